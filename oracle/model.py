@@ -1,0 +1,256 @@
+"""ORACLE (test infrastructure): the forward-only two-point zeroth-order QAT step,
+written out plainly in numpy (float64 arithmetic) on top of the C core.
+
+What it follows
+  * Eq. (1): g = [L(Q(W + eps u); B) - L(Q(W - eps u); B)] / (2 eps), one direction
+    (q = 1), u ~ N(0, I) regenerated from (seed, tensor id, element index).
+  * Eq. (2): W <- W - lr * g * u on every trainable tensor.
+  * Section 4.1: full-precision masters are kept; the forward pass sees their
+    quantised counterparts.  Section 2 quantiser, per group for weights and per
+    token (symmetric, 8 bit) for activations (Appendix "Quantization settings").
+  * Section 4.3 (lightweight variant): frozen tensors are quantised from the
+    unperturbed masters and are neither perturbed nor updated.
+
+Precision: float64 for every sum (linear layers, norms, softmax, loss).  The
+numbers that decide integer codes or operand roundings are taken in binary32,
+the precision the CUDA kernels use for the same decision: the perturbed weight
+and its quantiser (C core), the activation that enters the per-token quantiser,
+and the bfloat16 rounding of matrix-multiply operands.
+
+Only tests, the smoke check and the benchmark's CPU leg may import this module.
+"""
+from dataclasses import dataclass, field
+from typing import Callable, Optional
+
+import numpy as np
+
+from . import core
+
+F32 = np.float32
+
+# Block-linear roles.  tensor id of a block tensor = 16*(layer+1) + role;
+# the vocabulary projection has tensor id 0.
+ROLE_Q, ROLE_K, ROLE_V, ROLE_O, ROLE_GATE, ROLE_UP, ROLE_DOWN = range(7)
+ROLE_FC1, ROLE_FC2 = ROLE_GATE, ROLE_DOWN
+LM_HEAD_ID = 0
+
+
+def tensor_id(layer: int, role: int) -> int:
+    return 16 * (layer + 1) + role
+
+
+@dataclass
+class OracleConfig:
+    arch: str                 # "llama" (RMSNorm, RoPE, SiLU-gated FFN) or "opt" (LayerNorm, learned positions, ReLU FFN, biases)
+    n_layers: int
+    d_model: int
+    n_heads: int
+    d_ffn: int
+    vocab: int
+    w_bits: int = 4
+    w_group: int = 128
+    a_bits: int = 8           # 8 = per-token symmetric int8 on block-linear inputs, 0 = none
+    norm_eps: float = 1e-5
+    rope_base: float = 10000.0
+    first_trainable_layer: int = 0   # layers below are frozen (quantised from the unperturbed masters)
+    head_trainable: bool = True
+    operand_bf16: bool = True        # False (with w_bits = 0, a_bits = 0) gives the unquantised float64 model, used only to pin the forward
+
+
+def act_quant(x64):
+    """Per-token symmetric int8 quantiser (Section 2 symmetric form with N = 8:
+    Delta = max|x| / Q_P, z = 0, clamp to [-2^7, 2^7 - 1]); one Delta per row.
+    The decision is taken in binary32.  Returns integer codes (float64 array)
+    and the per-row Delta (float32)."""
+    x = x64.astype(F32)
+    amax = np.max(np.abs(x), axis=-1, keepdims=True).astype(F32)
+    s = (amax / F32(127.0)).astype(F32)
+    s = np.maximum(s, F32(1e-8))
+    inv = (F32(1.0) / s).astype(F32)
+    v = (x * inv).astype(F32)
+    q = np.clip(np.rint(v), -128.0, 127.0)
+    return q.astype(np.float64), s[..., 0]
+
+
+def rope_tables(seq, d_head, base):
+    """cos/sin of pos * base^(-2i/d_head), i < d_head/2, rounded to binary32."""
+    i = np.arange(d_head // 2, dtype=np.float64)
+    inv_freq = base ** (-2.0 * i / d_head)
+    ang = np.arange(seq, dtype=np.float64)[:, None] * inv_freq[None, :]
+    return np.cos(ang).astype(F32).astype(np.float64), np.sin(ang).astype(F32).astype(np.float64)
+
+
+def apply_rope(x, cos, sin):
+    """x [B, S, H, dh]; pairs (i, i + dh/2) rotated by the angle of position s."""
+    h = x.shape[-1] // 2
+    x1, x2 = x[..., :h], x[..., h:]
+    c = cos[None, :, None, :]
+    s = sin[None, :, None, :]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+class OracleModel:
+    """params: dict with 'embed' [V,d], 'lm_head' [V,d], 'final_norm_g' [d]
+    (+ 'final_norm_b', 'pos' [S_max,d] for arch 'opt'), and 'layers': list of
+    dicts with 'attn_norm_g', 'ffn_norm_g', 'wq','wk','wv','wo' [out,in] and
+    'w_gate','w_up','w_down' (llama) or 'fc1','fc2' plus biases 'bq','bk','bv',
+    'bo','b_fc1','b_fc2' and 'attn_norm_b','ffn_norm_b' (opt).  All float32."""
+
+    def __init__(self, cfg: OracleConfig, params: dict):
+        self.cfg = cfg
+        self.p = params
+        self.tap: Optional[Callable[[str, np.ndarray], None]] = None
+
+    # -- which tensors are perturbed / updated ---------------------------------
+    def linear_names(self):
+        return (["wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"] if self.cfg.arch == "llama"
+                else ["wq", "wk", "wv", "wo", "fc1", "fc2"])
+
+    _ROLE = {"wq": ROLE_Q, "wk": ROLE_K, "wv": ROLE_V, "wo": ROLE_O, "w_gate": ROLE_GATE,
+             "w_up": ROLE_UP, "w_down": ROLE_DOWN, "fc1": ROLE_FC1, "fc2": ROLE_FC2}
+
+    def trainable_tensors(self):
+        """(array, tensor id) of every tensor Eq. (2) updates."""
+        out = []
+        for l in range(self.cfg.first_trainable_layer, self.cfg.n_layers):
+            for n in self.linear_names():
+                out.append((self.p["layers"][l][n], tensor_id(l, self._ROLE[n])))
+        if self.cfg.head_trainable:
+            out.append((self.p["lm_head"], LM_HEAD_ID))
+        return out
+
+    # -- operands ----------------------------------------------------------------
+    def block_operand(self, l, name, seed, signed_eps):
+        """Fake-quantised weight of a block linear as the matmul sees it
+        (bfloat16-rounded dequantised value), float64 [out, in]."""
+        cfg = self.cfg
+        w = self.p["layers"][l][name]
+        if l >= cfg.first_trainable_layer and signed_eps != 0.0:
+            w = core.perturb(w, seed, tensor_id(l, self._ROLE[name]), signed_eps)
+        if cfg.w_bits == 0:
+            deq = w
+        else:
+            _, _, _, deq = core.weight_quant(w, cfg.w_group, cfg.w_bits)
+        return (core.round_bf16(deq) if cfg.operand_bf16 else deq).astype(np.float64)
+
+    def head_operand(self, seed, signed_eps):
+        w = self.p["lm_head"]
+        if self.cfg.head_trainable and signed_eps != 0.0:
+            w = core.perturb(w, seed, LM_HEAD_ID, signed_eps)
+        return (core.round_bf16(w) if self.cfg.operand_bf16 else w).astype(np.float64)
+
+    def _operand_round(self, x):
+        return core.round_bf16(x.astype(F32)).astype(np.float64) if self.cfg.operand_bf16 else x
+
+    def lin(self, x, l, name, seed, signed_eps, bias=None):
+        """x [T, in] float64 -> [T, out] float64 through the quantised linear."""
+        if self.cfg.a_bits == 8:
+            a, s = act_quant(x)
+            y = (a @ self.block_operand(l, name, seed, signed_eps).T) * s.astype(np.float64)[:, None]
+        else:
+            a = self._operand_round(x)
+            y = a @ self.block_operand(l, name, seed, signed_eps).T
+        if bias is not None:
+            y = y + bias.astype(np.float64)[None, :]
+        return y
+
+    def norm(self, h, g, b=None):
+        cfg = self.cfg
+        if cfg.arch == "llama":
+            ms = np.mean(h * h, axis=-1, keepdims=True)
+            y = h / np.sqrt(ms + np.float64(F32(cfg.norm_eps))) * g.astype(np.float64)
+        else:
+            mu = np.mean(h, axis=-1, keepdims=True)
+            var = np.mean((h - mu) ** 2, axis=-1, keepdims=True)
+            y = (h - mu) / np.sqrt(var + np.float64(F32(cfg.norm_eps))) * g.astype(np.float64)
+            y = y + b.astype(np.float64)
+        return y
+
+    def _tap(self, name, arr):
+        if self.tap is not None:
+            self.tap(name, arr)
+
+    # -- forward -------------------------------------------------------------------
+    def token_losses(self, tokens, labels, seed=0, signed_eps=0.0):
+        """tokens, labels int [B, S]; labels < 0 are ignored.  Returns the per-position
+        cross-entropy (float64 [B*S], 0 where ignored) and the valid mask."""
+        cfg = self.cfg
+        B, S = tokens.shape
+        T = B * S
+        d, H = cfg.d_model, cfg.n_heads
+        dh = d // H
+        h = self.p["embed"][tokens.reshape(-1)].astype(np.float64)
+        if cfg.arch == "opt":
+            pos = np.tile(np.arange(S), B)
+            h = h + self.p["pos"][pos].astype(np.float64)
+        else:
+            cos, sin = rope_tables(S, dh, cfg.rope_base)
+        causal = np.tril(np.ones((S, S), dtype=bool))
+        for l in range(cfg.n_layers):
+            P = self.p["layers"][l]
+            x = self.norm(h, P["attn_norm_g"], P.get("attn_norm_b"))
+            self._tap(f"l{l}.attn_norm", x)
+            q = self.lin(x, l, "wq", seed, signed_eps, P.get("bq"))
+            k = self.lin(x, l, "wk", seed, signed_eps, P.get("bk"))
+            v = self.lin(x, l, "wv", seed, signed_eps, P.get("bv"))
+            self._tap(f"l{l}.q", q); self._tap(f"l{l}.k", k); self._tap(f"l{l}.v", v)
+            q = q.reshape(B, S, H, dh); k = k.reshape(B, S, H, dh); v = v.reshape(B, S, H, dh)
+            if cfg.arch == "llama":
+                q = apply_rope(q, cos, sin)
+                k = apply_rope(k, cos, sin)
+            sc = np.einsum("bshd,bthd->bhst", q, k) / np.sqrt(np.float64(dh))
+            sc = np.where(causal[None, None], sc, -np.inf)
+            sc = sc - sc.max(axis=-1, keepdims=True)
+            pr = np.exp(sc)
+            pr = pr / pr.sum(axis=-1, keepdims=True)
+            att = np.einsum("bhst,bthd->bshd", pr, v).reshape(T, d)
+            self._tap(f"l{l}.attn", att)
+            h = h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo"))
+            self._tap(f"l{l}.h_mid", h)
+            x = self.norm(h, P["ffn_norm_g"], P.get("ffn_norm_b"))
+            if cfg.arch == "llama":
+                gate = self.lin(x, l, "w_gate", seed, signed_eps)
+                up = self.lin(x, l, "w_up", seed, signed_eps)
+                act = gate / (1.0 + np.exp(-gate)) * up
+                self._tap(f"l{l}.ffn_act", act)
+                h = h + self.lin(act, l, "w_down", seed, signed_eps)
+            else:
+                a1 = np.maximum(self.lin(x, l, "fc1", seed, signed_eps, P["b_fc1"]), 0.0)
+                self._tap(f"l{l}.ffn_act", a1)
+                h = h + self.lin(a1, l, "fc2", seed, signed_eps, P["b_fc2"])
+            self._tap(f"l{l}.h_out", h)
+        x = self.norm(h, self.p["final_norm_g"], self.p.get("final_norm_b"))
+        self._tap("final_norm", x)
+        a = self._operand_round(x)
+        logits = a @ self.head_operand(seed, signed_eps).T
+        self._tap("logits", logits)
+        lab = labels.reshape(-1)
+        valid = lab >= 0
+        mx = logits.max(axis=-1)
+        lse = mx + np.log(np.exp(logits - mx[:, None]).sum(axis=-1))
+        picked = logits[np.arange(T), np.where(valid, lab, 0)]
+        return np.where(valid, lse - picked, 0.0), valid
+
+    def loss(self, tokens, labels, seed=0, signed_eps=0.0):
+        """L(Q(W + signed_eps u); B): mean next-token cross-entropy over labelled positions."""
+        tl, valid = self.token_losses(tokens, labels, seed, signed_eps)
+        return float(tl.sum() / max(int(valid.sum()), 1))
+
+    # -- Eq. (1) and Eq. (2) ---------------------------------------------------------
+    def projected_gradient(self, tokens, labels, seed, eps):
+        eps32 = F32(eps)
+        lp = self.loss(tokens, labels, seed, float(eps32))
+        lm = self.loss(tokens, labels, seed, -float(eps32))
+        g = F32((lp - lm) / (2.0 * float(eps32)))
+        return lp, lm, g
+
+    def apply_update(self, seed, scale):
+        """W <- W - scale * u(seed) on every trainable tensor, in place (binary32 fma)."""
+        for w, tid in self.trainable_tensors():
+            core.update_(w, seed, tid, F32(scale))
+
+    def step(self, tokens, labels, seed, eps, lr):
+        lp, lm, g = self.projected_gradient(tokens, labels, seed, eps)
+        scale = F32(F32(lr) * g)
+        self.apply_update(seed, scale)
+        return lp, lm, float(g)
