@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the ZO-QAT step (two quantised forwards + seeded update) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one full pass of the hot path over one synthetic batch.  Default
+workload: LLaMA-7B shape, W4A8 (group-128 asymmetric weights, per-token int8
+activations), batch 4 x seq 1024.  Prints ONE JSON line (rank 0).
+--impl reference times the CPU oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ZO-QAT steps/s & fwd tokens/s, 7B-shape W4A8, 1 B200; % of roofline"
+UNIT = "steps/s"
+EPS, LR = 1e-3, 1e-6
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel from the committed ncu
+# capture (profiles/), keyed by workload; None until a capture exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sustained=p["bf16_tflops_sustained"], source="measured")
+    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+def workload_numbers(w):
+    """Algorithmic FLOPs and bytes of one step (both passes + update) of a workload."""
+    d, F, V, L = w["d_model"], w["d_ffn"], w["vocab"], w["n_layers"]
+    T = w["batch"] * w["seq"]
+    per_layer = 4 * d * d + (3 if w["arch"] == "llama" else 2) * d * F
+    ftl = w.get("first_trainable_layer", 0)
+    block = per_layer * L
+    trainable = per_layer * (L - ftl) + V * d
+    head = V * d
+    # frozen prefix layers are identical in both passes and are evaluated once
+    lin_flops = 2 * T * (per_layer * ftl + 2 * per_layer * (L - ftl) + 2 * head)
+    attn_flops = 2 * w["batch"] * w["seq"] ** 2 * d * (ftl + 2 * (L - ftl))
+    frozen = per_layer * ftl
+    bytes_step = 4 * trainable + (w["w_bits"] / 8 + 8 / w["w_group"]) * frozen + 8 * trainable
+    return dict(T=T, block_params=block, trainable_params=trainable, head_params=head,
+                linear_flops=lin_flops, attn_flops=attn_flops, flops=lin_flops + attn_flops, bytes=bytes_step)
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------
+def oracle_sample(w, budget_note=True):
+    """Times the oracle (as it stands) on a bounded sample of workload `w` and extrapolates one step.
+
+    Sample: ONE decoder layer of the workload's shape plus the vocabulary projection, at T1 and T2 = 2*T1
+    tokens (T1 = 32 for 7B-class shapes).  Step time is fitted as a + b*T per layer (a: weight-side work
+    - direction, perturbation, quantiser - independent of tokens; b: matmul/attention work per token) and
+    extrapolated to n_layers layers and the workload's tokens.
+    """
+    import numpy as np
+    from oracle.model import OracleConfig, OracleModel
+    from paper_2509_00031_b200 import synth
+    one = dict(w, n_layers=1)
+    small = w["d_model"] <= 512
+    seq1 = 32 if not small else w["seq"]
+    times = {}
+    cores = os.cpu_count() or 1
+    cfg = OracleConfig(arch=w["arch"], n_layers=1, d_model=w["d_model"], n_heads=w["n_heads"], d_ffn=w["d_ffn"],
+                       vocab=w["vocab"], w_bits=w["w_bits"], w_group=w["w_group"], a_bits=w["a_bits"])
+    params = synth.make_params(one, seed=0, max_seq=2 * seq1)
+    model = OracleModel(cfg, params)
+    for seq in (seq1, 2 * seq1):
+        tokens, labels = synth.make_batch(1, seq, w["vocab"], seed=1234)
+        t0 = time.perf_counter()
+        model.step(tokens, labels, 1000, EPS, LR)
+        times[seq] = time.perf_counter() - t0
+    b = (times[2 * seq1] - times[seq1]) / seq1
+    a = times[seq1] - b * seq1
+    nums = workload_numbers(w)
+    L = w["n_layers"]
+    # the single layer + head were timed together; scale the whole by layers (head counted L times: a small overestimate)
+    step_s = L * (max(a, 0.0) + max(b, 0.0) * nums["T"])
+    return dict(step_s=step_s, cores=cores, cpu_s=times[seq1] + times[2 * seq1],
+                sample=f"1 of {L} layers + vocabulary projection, full ZO step at {seq1} and {2 * seq1} tokens of {nums['T']}; "
+                       f"step time fitted as layers*(a + b*tokens), a={a:.3f}s b={b * 1e3:.3f}ms/token")
+
+
+def run_reference(args, w, rank, world):
+    if rank != 0:
+        return
+    reps = []
+    for _ in range(max(1, min(args.steps, 2))):
+        reps.append(oracle_sample(w))
+    step_s = sum(r["step_s"] for r in reps) / len(reps)
+    nums = workload_numbers(w)
+    value = 1.0 / step_s
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=step_s * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic", impl="reference", fwd_tokens_per_s=2 * nums["T"] * value,
+                config=dict(workload=args.workload, **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab",
+                                                                         "w_bits", "w_group", "a_bits", "batch", "seq")}),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=reps[0]["cores"], kind="oracle", sample=reps[0]["sample"]),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def make_device_params(w, torch, seed=0):
+    """Random-init parameters directly on the device (N(0, 0.02^2), bf16-rounded where the workload says so)."""
+    from paper_2509_00031_b200 import synth
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    d, f, v = w["d_model"], w["d_ffn"], w["vocab"]
+    opt = w["arch"] == "opt"
+
+    def rnd(*s):
+        t = torch.empty(s, dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=gen)
+        return t.bfloat16().float() if w.get("bf16_init") else t
+
+    ones = lambda n: torch.ones(n, dtype=torch.float32, device="cuda")
+    zeros = lambda n: torch.zeros(n, dtype=torch.float32, device="cuda")
+    p = {"embed": rnd(v, d), "lm_head": rnd(v, d), "final_norm_g": ones(d), "layers": []}
+    if opt:
+        p["final_norm_b"] = zeros(d)
+        p["pos"] = rnd(w["seq"], d)
+    for _ in range(w["n_layers"]):
+        L = {"attn_norm_g": ones(d), "ffn_norm_g": ones(d)}
+        for name, (o, i) in synth.linear_shapes(w).items():
+            L[name] = rnd(o, i)
+        if opt:
+            L["attn_norm_b"] = zeros(d); L["ffn_norm_b"] = zeros(d)
+            for name, n in (("bq", d), ("bk", d), ("bv", d), ("bo", d), ("b_fc1", f), ("b_fc2", d)):
+                L[name] = zeros(n)
+        p["layers"].append(L)
+    return p
+
+
+def run_ours(args, w, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_00031_b200 import binding, synth
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    binding.lib()
+    peaks = load_peaks()
+    nums = workload_numbers(w)
+    ftl = w.get("first_trainable_layer", 0)
+
+    params = make_device_params(w, torch, seed=0)          # every replica holds the same masters
+    model = binding.ZoqatModel(w, params, max_batch=w["batch"], max_seq=w["seq"], first_trainable_layer=ftl,
+                               packed_frozen=ftl > 0, gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05)
+    if ftl > 0:
+        model.zoqat_prequantize_frozen()
+        for l in range(ftl):                               # the fp32 copies of packed tensors are no longer needed
+            for name in synth.linear_shapes(w):
+                params["layers"][l][name] = None
+        torch.cuda.empty_cache()
+    # weak scaling: each rank gets its own batch shard of the workload's size
+    tok_np, lab_np = synth.make_batch(w["batch"], w["seq"], w["vocab"], seed=1234 + rank)
+    tokens, labels = torch.from_numpy(tok_np).cuda(), torch.from_numpy(lab_np).cuda()
+    tok_host, lab_host = torch.from_numpy(tok_np).pin_memory(), torch.from_numpy(lab_np).pin_memory()
+    result = torch.zeros(6, dtype=torch.float32, device="cuda")
+    sums = torch.zeros(3, dtype=torch.float64, device="cuda")
+
+    def step(t):
+        if world == 1:
+            model.zoqat_step(tokens, labels, 1000 + t, EPS, LR, result)
+        else:                                              # data-parallel replicas: 24-byte all-reduce between the halves
+            model.zoqat_step_begin(tokens, labels, 1000 + t, EPS, sums)
+            dist.all_reduce(sums)
+            model.zoqat_step_finish(sums, 1000 + t, EPS, LR, result)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        step(t)
+    model.zoqat_check()
+    barrier()
+    # ---- timed region: K steps, device-timed, per-category event pairs for the roofline of the dominant kernel
+    model.zoqat_profile_enable(True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = model.zoqat_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for t in range(args.steps):
+        step(args.warmup + t)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = model.zoqat_launch_count() - launches0
+    prof = {binding.PROF_NAMES[c]: model.zoqat_profile_read(c) for c in range(len(binding.PROF_NAMES))}
+    model.zoqat_profile_enable(False)
+    model.zoqat_check()
+    res = binding.decode_step_result(result)
+    # ---- end-to-end: the host-buffer entry point, copies inside the timed region
+    e2e_ms = None
+    if world == 1:
+        barrier()
+        t0 = time.perf_counter()
+        for t in range(args.steps):
+            model.zoqat_step_host(tok_host, lab_host, 5000 + t, EPS, LR)
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3
+    if world > 1:
+        tmax = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = ms / args.steps
+    steps_per_s = world * 1e3 / ms_per_step                 # whole job: every replica processes its own batch
+    gemm_ms, gemm_n = prof["gemm"]
+    gemm_flops_step = nums["linear_flops"]
+    achieved_tf = gemm_flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    peak_tf = peaks["tf_sustained"]
+    t_flop = nums["flops"] / (peaks["tf_burst"] * 1e12)
+    t_hbm = nums["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    roof_s = max(t_flop, t_hbm)
+    line = dict(
+        metric=METRIC, value=steps_per_s, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+        data="synthetic", fwd_tokens_per_s=2 * nums["T"] * steps_per_s,
+        config=dict(workload=args.workload, l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
+                    gemm="simt" if args.simt else "tcgen05",
+                    **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab", "w_bits", "w_group",
+                                         "a_bits", "batch", "seq")}),
+        step_roofline=dict(bound="tensor" if t_flop >= t_hbm else "hbm", flops_per_step=nums["flops"],
+                           bytes_per_step=nums["bytes"], roofline_ms=roof_s * 1e3,
+                           frac=(roof_s * 1e3) / ms_per_step, peak_source=peaks["source"] + " (burst bf16, copy HBM)"),
+        roofline=dict(bound="tensor", kernel="gemm_tc_kernel (all linear layers + fused vocabulary projection/cross-entropy)",
+                      achieved=achieved_tf, peak=peak_tf, unit="TFLOP/s",
+                      frac=(achieved_tf / peak_tf) if achieved_tf else None,
+                      peak_source=peaks["source"] + " sustained bf16 (kernel timed inside a long step)",
+                      launches_per_step=gemm_n / args.steps, avg_launch_ms=gemm_ms / max(gemm_n, 1),
+                      traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)),
+        kernel_ms_per_step={k: v[0] / args.steps for k, v in prof.items()},
+        gpu_launches=launches, clocks=clocks,
+        last_step=dict(loss_plus=res["loss_plus"], loss_minus=res["loss_minus"], proj_grad=res["proj_grad"], status=res["status"]),
+    )
+    if e2e_ms is not None:
+        line["e2e"] = dict(value=1e3 * args.steps / e2e_ms, unit=UNIT, h2d_bytes_per_step=2 * nums["T"] * 4, d2h_bytes_per_step=24)
+    # release the device before the CPU baseline runs
+    del model, params
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_cpu_baseline:
+        o = oracle_sample(w)
+        line["cpu_baseline"] = dict(value=1.0 / o["step_s"], unit=UNIT, cores=o["cores"], kind="oracle", sample=o["sample"])
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_w4a8")
+    ap.add_argument("--simt", action="store_true", help="use the CUDA-core cross-check GEMM instead of tcgen05")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2509_00031_b200 import synth
+    w = dict(synth.WORKLOADS[args.workload])
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, w, rank, world)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+    run_ours(args, w, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,313 @@
+/*
+ * zoqat.h - C ABI of libzoqat: the forward-only, two-point zeroth-order
+ * quantisation-aware training step of ZeroQAT on one NVIDIA B200 (sm_100a).
+ *
+ * One step (Section 4.1 of the paper):
+ *   Eq. (1)  g = [ L(Q(W + eps u); B) - L(Q(W - eps u); B) ] / (2 eps),  u ~ N(0, I), q = 1
+ *   Eq. (2)  W <- W - lr * g * u
+ * Q is the uniform quantiser of Section 2 (asymmetric, one step size and zero
+ * point per group of consecutive input channels for weights; symmetric 8-bit,
+ * one step size per token for the inputs of the block linears).  Full-precision
+ * masters are kept and only their quantised counterparts enter the forward
+ * pass.  The direction u is never stored: element i of tensor t under a 64-bit
+ * seed is regenerated from a Philox4x32-10 counter (block i/4, tensor id t)
+ * wherever it is needed (both passes and the update).  The lightweight variant
+ * of Section 4.3 keeps frozen tensors as packed low-bit codes.
+ *
+ * Conventions
+ *   - Every function returns an int status: ZOQAT_OK (0) or a negative error.
+ *     Nothing throws; zoqat_status_string() names a status and
+ *     zoqat_last_error() returns the text of the last failure on the calling
+ *     thread (arguments are validated on the host before any launch).
+ *   - "dev" pointers are device (global) memory of the current CUDA device,
+ *     "host" pointers are host memory.  The caller owns all device memory:
+ *     masters, packed buffers, workspace, inputs and outputs.  The library owns
+ *     only the host-side handle.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls are asynchronous with respect to the host unless stated otherwise.
+ *     One handle may be used from one stream at a time.
+ *   - Matrices are row-major; a linear weight is [out_features, in_features]
+ *     with quantisation groups contiguous along in_features.
+ *   - Device-side waits are bounded; a wait that runs out writes a non-zero
+ *     word to the handle's error flag, which zoqat_check() reads.  No kernel
+ *     traps the GPU.
+ */
+#ifndef ZOQAT_H
+#define ZOQAT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------- */
+#define ZOQAT_OK                     0
+#define ZOQAT_ERR_INVALID_ARG       -1
+#define ZOQAT_ERR_UNSUPPORTED       -2
+#define ZOQAT_ERR_WORKSPACE_SMALL   -3
+#define ZOQAT_ERR_CUDA              -4
+#define ZOQAT_ERR_BAD_STATE         -5
+#define ZOQAT_ERR_TIMEOUT           -6
+
+/* ---- model description --------------------------------------------------- */
+#define ZOQAT_ARCH_LLAMA 0   /* RMSNorm, rotary positions, SiLU-gated FFN, no biases   */
+#define ZOQAT_ARCH_OPT   1   /* LayerNorm, learned positions, ReLU FFN, linear biases  */
+
+/* Tensor roles.  The first seven are the block linears; their Philox tensor id
+ * is 16*(layer+1) + role.  The vocabulary projection has tensor id 0. */
+#define ZOQAT_ROLE_WQ            0
+#define ZOQAT_ROLE_WK            1
+#define ZOQAT_ROLE_WV            2
+#define ZOQAT_ROLE_WO            3
+#define ZOQAT_ROLE_W_GATE        4   /* OPT: fc1 */
+#define ZOQAT_ROLE_W_UP          5   /* LLaMA only */
+#define ZOQAT_ROLE_W_DOWN        6   /* OPT: fc2 */
+#define ZOQAT_ROLE_ATTN_NORM_G   7
+#define ZOQAT_ROLE_ATTN_NORM_B   8   /* OPT only */
+#define ZOQAT_ROLE_FFN_NORM_G    9
+#define ZOQAT_ROLE_FFN_NORM_B   10   /* OPT only */
+#define ZOQAT_ROLE_BQ           11   /* OPT only: biases */
+#define ZOQAT_ROLE_BK           12
+#define ZOQAT_ROLE_BV           13
+#define ZOQAT_ROLE_BO           14
+#define ZOQAT_ROLE_B_FC1        15
+#define ZOQAT_ROLE_B_FC2        16
+#define ZOQAT_ROLE_EMBED        17   /* layer = -1 from here on */
+#define ZOQAT_ROLE_POS_EMBED    18   /* OPT only */
+#define ZOQAT_ROLE_FINAL_NORM_G 19
+#define ZOQAT_ROLE_FINAL_NORM_B 20   /* OPT only */
+#define ZOQAT_ROLE_LM_HEAD      21
+#define ZOQAT_ROLE_COUNT        22
+
+/* Tensor flags (linear weights only; every other tensor is frozen fp32). */
+#define ZOQAT_TENSOR_TRAINABLE      1u  /* perturbed by +/- eps u in the forward, updated by Eq. (2) */
+#define ZOQAT_TENSOR_QUANTIZED      2u  /* forward sees the per-group fake-quantised weight         */
+#define ZOQAT_TENSOR_FROZEN_PACKED  4u  /* Section 4.3: forward reads packed codes + (step, zero point) written by
+                                           zoqat_prequantize_frozen(); never perturbed, never updated */
+
+#define ZOQAT_GEMM_TCGEN05 0   /* tcgen05/TMEM tensor-core kernel (default)                    */
+#define ZOQAT_GEMM_SIMT    1   /* plain CUDA-core kernel, kept as an on-device cross-check      */
+
+typedef struct zoqat_config {
+    int32_t arch;          /* ZOQAT_ARCH_*                                                        */
+    int32_t n_layers;
+    int32_t d_model;       /* multiple of 64                                                      */
+    int32_t n_heads;       /* d_model / n_heads in {32, 64, 128}                                  */
+    int32_t d_ffn;         /* multiple of 64                                                      */
+    int32_t vocab;
+    int32_t max_batch;     /* largest batch ...                                                   */
+    int32_t max_seq;       /* ... and sequence length a call will pass                            */
+    int32_t w_bits;        /* 2, 3 or 4                                                           */
+    int32_t w_group;       /* 32, 64 or 128; divides d_model and d_ffn                            */
+    int32_t a_bits;        /* 8 = per-token symmetric int8 on block-linear inputs, 0 = none        */
+    int32_t gemm_impl;     /* ZOQAT_GEMM_*                                                        */
+    float   norm_eps;
+    float   rope_base;     /* LLaMA only                                                          */
+} zoqat_config_t;
+
+typedef struct zoqat_tensor_desc {
+    int32_t role;          /* ZOQAT_ROLE_*                                                        */
+    int32_t layer;         /* 0..n_layers-1, or -1 for model-level tensors                        */
+    uint32_t flags;        /* ZOQAT_TENSOR_* (linear weights)                                     */
+    uint32_t reserved;
+    void*   data;          /* dev: fp32 values.  For FROZEN_PACKED tensors it is read only by
+                              zoqat_prequantize_frozen() and may be freed afterwards.            */
+    void*   packed;        /* dev: FROZEN_PACKED only, zoqat_packed_bytes() code bytes             */
+    void*   qparams;       /* dev: FROZEN_PACKED only, one (float step, float zero point) pair per group */
+} zoqat_tensor_desc_t;
+
+typedef struct zoqat_step_result {
+    float   loss_plus;     /* L(Q(W + eps u); B)                                                  */
+    float   loss_minus;    /* L(Q(W - eps u); B)                                                  */
+    float   proj_grad;     /* g of Eq. (1), formed in double precision and rounded                 */
+    float   update_scale;  /* lr * g, the factor the update multiplies u by                        */
+    int32_t status;        /* 0, or the device error word                                         */
+    int32_t n_labels;      /* labelled positions per pass                                         */
+} zoqat_step_result_t;
+
+typedef struct zoqat_model zoqat_model_t;
+
+/* ---- the step (Section 4.1, Section 4.3) ---------------------------------- */
+
+/* Bytes of device workspace zoqat_model_create() needs for `cfg` (host only). */
+int zoqat_query_workspace(const zoqat_config_t* cfg, size_t* bytes);
+
+/* Sizes of the packed representation of one [rows, cols] tensor: `code_bytes` of
+ * codes (rows * cols * bits / 8, rows padded to nothing: cols*bits must be a
+ * multiple of 8) and `qparam_bytes` = rows * cols/group * 8. */
+int zoqat_packed_bytes(int64_t rows, int64_t cols, int bits, int group,
+                       size_t* code_bytes, size_t* qparam_bytes);
+
+/* Builds a handle.  `tensors[0..n)` must name every tensor the architecture has
+ * (each role once per layer).  `workspace_dev` (256-byte aligned, `bytes` >=
+ * the queried size) is used by every later call on the handle.  Masters flagged
+ * TRAINABLE are updated in place by zoqat_step()/zoqat_apply_update(). */
+int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* tensors, int n_tensors,
+                       void* workspace_dev, size_t bytes, zoqat_model_t** out);
+int zoqat_model_destroy(zoqat_model_t* m);
+
+/* Section 4.3: quantises every FROZEN_PACKED tensor from its unperturbed fp32
+ * values into `packed` / `qparams`.  Idempotent.  Must run before the first
+ * forward when such tensors exist. */
+int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream);
+
+/* One forward pass: *loss_out_dev = L(Q(W + signed_eps u(seed)); B), the mean
+ * next-token cross-entropy over positions whose label is >= 0 (Eq. (1) argument).
+ * signed_eps = 0 gives the unperturbed quantised model.  tokens_dev / labels_dev:
+ * int32 [batch, seq] on the device.  Masters are not modified. */
+int zoqat_forward_loss(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                       int batch, int seq, uint64_t seed, float signed_eps,
+                       float* loss_out_dev, void* stream);
+
+/* One ZO-QAT step: both passes of Eq. (1) (evaluated side by side so that each
+ * master and each direction is produced once for the pair), g, and the update
+ * of Eq. (2) with the regenerated direction.  No host synchronisation.
+ * `result_dev` (device memory) receives the scalars. */
+int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+               int batch, int seq, uint64_t seed, float eps, float lr,
+               zoqat_step_result_t* result_dev, void* stream);
+
+/* The step in two halves, for data-parallel replicas that each hold all masters and a
+ * shard of the mini-batch (the loss of Eq. (1) is a mean over the mini-batch):
+ * zoqat_step_begin runs both passes on the local shard and writes
+ * sums_dev = (sum of per-position losses at +eps, the same at -eps, labelled positions)
+ * as three doubles; the caller sums sums_dev over replicas (one all-reduce of 24 bytes);
+ * zoqat_step_finish forms g from the global sums and applies Eq. (2), so every replica
+ * makes the same update and masters stay identical without any weight traffic.
+ * zoqat_step is begin + finish on one device. */
+int zoqat_step_begin(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                     int batch, int seq, uint64_t seed, float eps, double* sums_dev, void* stream);
+int zoqat_step_finish(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                      zoqat_step_result_t* result_dev, void* stream);
+
+/* Same step with HOST inputs and outputs: copies tokens/labels to the device,
+ * runs zoqat_step, copies the result back and synchronises the stream. */
+int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host,
+                    int batch, int seq, uint64_t seed, float eps, float lr,
+                    zoqat_step_result_t* result_host, void* stream);
+
+/* Eq. (2) alone: W <- W - scale * u(seed) on every TRAINABLE tensor. */
+int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream);
+
+/* Synchronises `stream` and returns ZOQAT_OK, ZOQAT_ERR_TIMEOUT if a bounded
+ * device wait ran out since the last check, or ZOQAT_ERR_CUDA. */
+int zoqat_check(zoqat_model_t* m, void* stream);
+
+/* Number of kernel launches the handle has issued so far. */
+int zoqat_launch_count(const zoqat_model_t* m, int64_t* launches);
+
+/* Optional device-side timing by category.  While enabled, every launch group of a
+ * forward/step is bracketed by a CUDA event pair on the caller's stream;
+ * zoqat_profile_read() synchronises `stream`, returns the milliseconds and the number
+ * of bracketed intervals accumulated for `category` since its last read, and clears them. */
+#define ZOQAT_PROF_GEMM       0   /* linear layers and the fused vocabulary projection / cross-entropy */
+#define ZOQAT_PROF_WEIGHT     1   /* perturb + quantise weight operands (and unpacking of frozen codes) */
+#define ZOQAT_PROF_ACT        2   /* embedding, norms, activation quantisers, FFN non-linearity         */
+#define ZOQAT_PROF_ATTENTION  3
+#define ZOQAT_PROF_LOSS       4   /* cross-entropy finalisation                                         */
+#define ZOQAT_PROF_UPDATE     5   /* Eq. (2)                                                            */
+#define ZOQAT_PROF_COUNT      6
+int zoqat_profile_enable(zoqat_model_t* m, int on);
+int zoqat_profile_read(zoqat_model_t* m, int category, double* ms, int64_t* intervals, void* stream);
+
+/* Device pointer and size of a workspace buffer holding intermediates of the
+ * most recent forward (last layer executed).  Parity hook. */
+#define ZOQAT_BUF_RESIDUAL   0   /* fp32 [passes*T, d_model]   residual stream after the last layer */
+#define ZOQAT_BUF_QKV        1   /* fp32 [passes*T, 3*d_model] q | k | v of the last layer (before RoPE) */
+#define ZOQAT_BUF_ATTN       2   /* fp32 [passes*T, d_model]   attention output of the last layer   */
+#define ZOQAT_BUF_FFN        3   /* fp32 [passes*T, 2*d_ffn or d_ffn] gate|up (LLaMA) or fc1 (OPT)   */
+#define ZOQAT_BUF_TOKEN_LOSS 4   /* fp32 [passes*T]            per-position cross-entropy            */
+int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* bytes);
+
+const char* zoqat_status_string(int status);
+const char* zoqat_last_error(void);
+
+/* ---- the steps of the path as single operations ---------------------------
+ * The same kernels the step launches, callable on raw device buffers so that
+ * each can be compared with the oracle at any size.  All asynchronous. */
+
+/* Raw Philox4x32-10 words of counter blocks [blk0, blk0+nblk) of a tensor:
+ * counter = (blk_lo, blk_hi, tensor_id, 0), key = (seed_lo, seed_hi).
+ * out_dev: uint32 [nblk, 4]. */
+int zoqat_op_philox_words(uint64_t seed, uint32_t tensor_id, uint64_t blk0, uint64_t nblk,
+                          uint32_t* out_dev, void* stream);
+
+/* u of Eq. (1) for elements [0, n) of a tensor: fp32 [n].  (Test hook: the step
+ * itself never writes u to memory.) */
+int zoqat_op_normal(uint64_t seed, uint32_t tensor_id, uint64_t n, float* out_dev, void* stream);
+
+/* Weight path of one [rows, cols] tensor (Eq. (1) argument + Section 2
+ * quantiser): w' = W + signed_eps u; per group of `group` columns the step,
+ * zero point and codes; the bf16 matmul operand (code - zp) * step.
+ * bits = 0 skips the quantiser (operand = bf16(w')).  Outputs may be NULL:
+ * codes_dev uint8 [rows, cols]; step_dev fp32 and zp_dev int32 [rows, cols/group];
+ * operand_dev bf16 [rows, cols]. */
+int zoqat_op_weight_quant(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
+                          uint64_t seed, uint32_t tensor_id, float signed_eps,
+                          uint8_t* codes_dev, float* step_dev, int32_t* zp_dev, void* operand_dev,
+                          void* stream);
+
+/* Both operands of a step from one read of W and one evaluation of u:
+ * operand_plus_dev from W + eps u, operand_minus_dev from W - eps u. */
+int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
+                                 uint64_t seed, uint32_t tensor_id, float eps,
+                                 void* operand_plus_dev, void* operand_minus_dev, void* stream);
+
+/* Packing of Section 4.3: quantise W (unperturbed) into packed codes + qparams,
+ * and expansion of a packed tensor into the bf16 operand. */
+int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
+                         void* packed_dev, void* qparams_dev, void* stream);
+int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols,
+                            int group, int bits, void* operand_dev, void* stream);
+
+/* Eq. (2) on one tensor: w[i] <- w[i] - scale * u_i, i in [0, n). */
+int zoqat_op_update(float* w_dev, uint64_t n, uint64_t seed, uint32_t tensor_id, float scale, void* stream);
+
+/* Optional normalisation followed by the activation operand of a linear:
+ * norm_kind 0 none, 1 RMSNorm (gain), 2 LayerNorm (gain, bias);
+ * a_bits 8: per-row symmetric int8 codes (as bf16 integers) + row step in
+ * row_step_dev; a_bits 0: bf16(x), row step 1.  x_dev fp32 [rows, cols];
+ * operand_dev bf16 [rows, cols]; row_step_dev fp32 [rows];
+ * normed_dev (may be NULL) fp32 [rows, cols] receives the normalised values. */
+int zoqat_op_norm_act_operand(const float* x_dev, int64_t rows, int64_t cols, int norm_kind,
+                              const float* gain_dev, const float* bias_dev, float norm_eps, int a_bits,
+                              void* operand_dev, float* row_step_dev, float* normed_dev, void* stream);
+
+/* FFN activation followed by the activation operand: LLaMA (gated = 1):
+ * silu(x[:, :cols]) * x[:, cols:2*cols] from x_dev fp32 [rows, 2*cols];
+ * OPT (gated = 0): relu(x) from fp32 [rows, cols]. */
+int zoqat_op_ffn_act_operand(const float* x_dev, int64_t rows, int64_t cols, int gated, int a_bits,
+                             void* operand_dev, float* row_step_dev, void* stream);
+
+/* out[m, n] (+)= row_step[m] * sum_k A[m, k] * B[n, k] (+ bias[n]), optional ReLU.
+ * a_dev bf16 [M, K], b_dev bf16 [N, K], out_dev fp32 [M, N] (ldo = N).
+ * row_step_dev / bias_dev may be NULL.  accumulate != 0 adds into out_dev.
+ * impl: ZOQAT_GEMM_*.  tcgen05 path: K % 8 == 0. err_flag_dev: int32 device word
+ * set non-zero if a bounded wait ran out (may be NULL for the SIMT kernel). */
+int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, int64_t K,
+                  const float* row_step_dev, const float* bias_dev, int relu, int accumulate,
+                  float* out_dev, int impl, int32_t* err_flag_dev, void* stream);
+
+/* Causal softmax attention of one layer.  qkv_dev fp32 [batch*seq, 3*d_model]
+ * (q | k | v, heads contiguous inside each); rotary tables cos_dev/sin_dev fp32
+ * [seq, d_head/2] or NULL (no rotation); out_dev fp32 [batch*seq, d_model]. */
+int zoqat_op_attention(const float* qkv_dev, int batch, int seq, int n_heads, int d_head,
+                       const float* cos_dev, const float* sin_dev, float* out_dev, void* stream);
+
+/* Vocabulary projection fused with the cross-entropy: logits = A B^T are never
+ * stored.  a_dev bf16 [T, d], b_dev bf16 [V, d], labels_dev int32 [T] (< 0 =
+ * ignored); token_loss_dev fp32 [T] (0 where ignored); loss_sum_dev double[1]
+ * (sum of the per-position losses) and count_dev int32[1] (labelled positions).
+ * scratch_dev: zoqat_op_head_loss_scratch_bytes(T, V) bytes. */
+int zoqat_op_head_loss_scratch_bytes(int64_t T, int64_t V, size_t* bytes);
+int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labels_dev,
+                       int64_t T, int64_t V, int64_t d, float* token_loss_dev,
+                       double* loss_sum_dev, int32_t* count_dev, void* scratch_dev,
+                       int impl, int32_t* err_flag_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZOQAT_H */

@@ -89,6 +89,23 @@ def apply_rope(x, cos, sin):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
+def causal_attention(q, k, v, n_heads, cos=None, sin=None):
+    """softmax(q k^T / sqrt(d_head) + causal mask) v per head, float64.
+    q, k, v: [B, S, d_model]; cos/sin: rotary tables [S, d_head/2] or None."""
+    B, S, d = q.shape
+    dh = d // n_heads
+    q = q.reshape(B, S, n_heads, dh); k = k.reshape(B, S, n_heads, dh); v = v.reshape(B, S, n_heads, dh)
+    if cos is not None:
+        q = apply_rope(q, cos, sin)
+        k = apply_rope(k, cos, sin)
+    sc = np.einsum("bshd,bthd->bhst", q, k) / np.sqrt(np.float64(dh))
+    sc = np.where(np.tril(np.ones((S, S), dtype=bool))[None, None], sc, -np.inf)
+    sc = sc - sc.max(axis=-1, keepdims=True)
+    pr = np.exp(sc)
+    pr = pr / pr.sum(axis=-1, keepdims=True)
+    return np.einsum("bhst,bthd->bshd", pr, v).reshape(B, S, d)
+
+
 class OracleModel:
     """params: dict with 'embed' [V,d], 'lm_head' [V,d], 'final_norm_g' [d]
     (+ 'final_norm_b', 'pos' [S_max,d] for arch 'opt'), and 'layers': list of
@@ -185,7 +202,6 @@ class OracleModel:
             h = h + self.p["pos"][pos].astype(np.float64)
         else:
             cos, sin = rope_tables(S, dh, cfg.rope_base)
-        causal = np.tril(np.ones((S, S), dtype=bool))
         for l in range(cfg.n_layers):
             P = self.p["layers"][l]
             x = self.norm(h, P["attn_norm_g"], P.get("attn_norm_b"))
@@ -194,16 +210,9 @@ class OracleModel:
             k = self.lin(x, l, "wk", seed, signed_eps, P.get("bk"))
             v = self.lin(x, l, "wv", seed, signed_eps, P.get("bv"))
             self._tap(f"l{l}.q", q); self._tap(f"l{l}.k", k); self._tap(f"l{l}.v", v)
-            q = q.reshape(B, S, H, dh); k = k.reshape(B, S, H, dh); v = v.reshape(B, S, H, dh)
-            if cfg.arch == "llama":
-                q = apply_rope(q, cos, sin)
-                k = apply_rope(k, cos, sin)
-            sc = np.einsum("bshd,bthd->bhst", q, k) / np.sqrt(np.float64(dh))
-            sc = np.where(causal[None, None], sc, -np.inf)
-            sc = sc - sc.max(axis=-1, keepdims=True)
-            pr = np.exp(sc)
-            pr = pr / pr.sum(axis=-1, keepdims=True)
-            att = np.einsum("bhst,bthd->bshd", pr, v).reshape(T, d)
+            att = causal_attention(q.reshape(B, S, d), k.reshape(B, S, d), v.reshape(B, S, d), H,
+                                   cos if cfg.arch == "llama" else None,
+                                   sin if cfg.arch == "llama" else None).reshape(T, d)
             self._tap(f"l{l}.attn", att)
             h = h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo"))
             self._tap(f"l{l}.h_mid", h)

@@ -1,0 +1,283 @@
+// Activation side of the forward pass outside the matrix multiplies: embedding
+// gather, RMSNorm / LayerNorm fused with the per-token activation quantiser
+// (Section 2 symmetric form, N = 8: step = max|x|/127, code = clamp(round(x/step),
+// -128, 127), one step per token), and the FFN non-linearity fused with the same
+// quantiser.  One CTA owns one token row, staged in shared memory; row statistics
+// are accumulated in double precision.  The operand written for the following
+// GEMM is bf16: the integer codes themselves (exact in bf16) with the step kept
+// per row for the GEMM epilogue, or bf16(x) when activations are not quantised.
+#include "common.cuh"
+
+namespace zq {
+namespace {
+
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ double block_sum(double v, double* red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int i = 0; i < kRowThreads / 32; ++i) t += red[i];
+    return t;
+}
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float t = red[0];
+#pragma unroll
+    for (int i = 1; i < kRowThreads / 32; ++i) t = fmaxf(t, red[i]);
+    return t;
+}
+
+// Writes the operand row from the fp32 row held in shared memory.
+__device__ __forceinline__ void write_operand_row(const float* row, int cols, int a_bits, __nv_bfloat16* op_row,
+                                                  float* row_step, float* redf) {
+    if (a_bits == 8) {
+        float amax = 0.0f;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) amax = fmaxf(amax, fabsf(row[c]));
+        amax = block_max(amax, redf);
+        const float step = fmaxf(__fdiv_rn(amax, 127.0f), 1e-8f);
+        const float inv = __fdiv_rn(1.0f, step);
+        if (threadIdx.x == 0) *row_step = step;
+        for (int c = 2 * threadIdx.x; c < cols; c += 2 * kRowThreads) {
+            const float q0 = fminf(fmaxf(rintf(__fmul_rn(row[c], inv)), -128.0f), 127.0f);
+            const float q1 = fminf(fmaxf(rintf(__fmul_rn(row[c + 1], inv)), -128.0f), 127.0f);
+            *reinterpret_cast<__nv_bfloat162*>(op_row + c) = __floats2bfloat162_rn(q0, q1);
+        }
+    } else {
+        if (threadIdx.x == 0) *row_step = 1.0f;
+        for (int c = 2 * threadIdx.x; c < cols; c += 2 * kRowThreads)
+            *reinterpret_cast<__nv_bfloat162*>(op_row + c) = __floats2bfloat162_rn(row[c], row[c + 1]);
+    }
+}
+
+__global__ void __launch_bounds__(kRowThreads)
+norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
+                        const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
+                        float* __restrict__ row_step, float* __restrict__ normed) {
+    extern __shared__ float row[];
+    __shared__ double redd[kRowThreads / 32];
+    __shared__ float redf[kRowThreads / 32];
+    const int64_t r = blockIdx.x;
+    const float* xr = x + r * cols;
+    for (int c = 4 * threadIdx.x; c < cols; c += 4 * kRowThreads)
+        *reinterpret_cast<float4*>(row + c) = *reinterpret_cast<const float4*>(xr + c);
+    __syncthreads();
+    if (norm_kind == 1) {            // RMSNorm: x / sqrt(mean(x^2) + eps) * gain
+        double ss = 0.0;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) { const double v = row[c]; ss += v * v; }
+        ss = block_sum(ss, redd);
+        const float rstd = (float)(1.0 / sqrt(ss / cols + (double)norm_eps));
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = row[c] * rstd * gain[c];
+    } else if (norm_kind == 2) {     // LayerNorm: (x - mean) / sqrt(var + eps) * gain + bias
+        double sm = 0.0;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) sm += (double)row[c];
+        const double mu = block_sum(sm, redd) / cols;
+        double sv = 0.0;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) { const double v = (double)row[c] - mu; sv += v * v; }
+        sv = block_sum(sv, redd);
+        const float rstd = (float)(1.0 / sqrt(sv / cols + (double)norm_eps));
+        const float muf = (float)mu;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = (row[c] - muf) * rstd * gain[c] + bias[c];
+    }
+    __syncthreads();
+    if (normed)
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) normed[r * cols + c] = row[c];
+    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
+}
+
+__global__ void __launch_bounds__(kRowThreads)
+ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
+                       float* __restrict__ row_step) {
+    extern __shared__ float row[];
+    __shared__ float redf[kRowThreads / 32];
+    const int64_t r = blockIdx.x;
+    if (gated) {                     // silu(gate) * up, gate | up concatenated along the row
+        const float* g = x + r * 2 * cols;
+        const float* u = g + cols;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) {
+            const float gv = g[c];
+            row[c] = __fdiv_rn(gv, 1.0f + expf(-gv)) * u[c];
+        }
+    } else {                         // relu
+        const float* g = x + r * cols;
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = fmaxf(g[c], 0.0f);
+    }
+    __syncthreads();
+    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
+}
+
+// h[p*T + t, :] = embed[token[t], :] (+ pos[t % seq, :]) for each of `passes` copies.
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const float4* __restrict__ embed,
+                             const float4* __restrict__ pos, int64_t T, int seq, int d4, int vocab, int passes,
+                             float4* __restrict__ h) {
+    const int64_t t = blockIdx.x;
+    int tok = tokens[t];
+    tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+    const float4* e = embed + (int64_t)tok * d4;
+    const float4* p = pos ? pos + (int64_t)(t % seq) * d4 : nullptr;
+    for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+        float4 v = e[c];
+        if (p) { const float4 q = p[c]; v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w; }
+        for (int k = 0; k < passes; ++k) h[((int64_t)k * T + t) * d4 + c] = v;
+    }
+}
+
+__global__ void copy_kernel(const float4* __restrict__ src, float4* __restrict__ dst, int64_t n4) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+
+// Per-position loss = logsumexp - logit[label] from the per-tile (max, sum exp) partials.
+__global__ void ce_token_kernel(const float2* __restrict__ partials, const float* __restrict__ label_logit,
+                                const int32_t* __restrict__ labels, int64_t M, int64_t rows, int n_tiles,
+                                float* __restrict__ token_loss) {
+    const int64_t r = blockIdx.x * (int64_t)(blockDim.x / 32) + (threadIdx.x >> 5);
+    if (r >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const int32_t lab = labels[r % M];
+    float mx = -INFINITY, sm = 0.0f;
+    for (int t = lane; t < n_tiles; t += 32) {
+        const float2 p = partials[r * n_tiles + t];
+        const float nm = fmaxf(mx, p.x);
+        sm = sm * expf(mx - nm) + p.y * expf(p.x - nm);
+        mx = nm;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, mx, o);
+        const float os = __shfl_xor_sync(0xffffffffu, sm, o);
+        const float nm = fmaxf(mx, om);
+        const float a = (mx == -INFINITY) ? 0.0f : sm * expf(mx - nm);
+        const float b = (om == -INFINITY) ? 0.0f : os * expf(om - nm);
+        sm = a + b;
+        mx = nm;
+    }
+    if (lane == 0) token_loss[r] = lab >= 0 ? (mx + logf(sm)) - label_logit[r] : 0.0f;
+}
+
+// Deterministic sum of the per-position losses of each pass (fixed tree, double).
+__global__ void __launch_bounds__(1024)
+ce_sum_kernel(const float* __restrict__ token_loss, const int32_t* __restrict__ labels, int64_t M,
+              double* __restrict__ loss_sum, int32_t* __restrict__ count) {
+    __shared__ double sd[32];
+    __shared__ int sc[32];
+    const int z = blockIdx.x;
+    double acc = 0.0;
+    int cnt = 0;
+    for (int64_t i = threadIdx.x; i < M; i += 1024) {
+        acc += (double)token_loss[z * M + i];
+        cnt += labels[i] >= 0;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    }
+    if ((threadIdx.x & 31) == 0) { sd[threadIdx.x >> 5] = acc; sc[threadIdx.x >> 5] = cnt; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0; int c = 0;
+        for (int i = 0; i < 32; ++i) { t += sd[i]; c += sc[i]; }
+        loss_sum[z] = t;
+        count[z] = c;
+    }
+}
+
+// Eq. (1): g = (L+ - L-) / (2 eps) in double, rounded to fp32; update factor lr*g.
+__global__ void pack_sums_kernel(const double* loss_sum, const int32_t* count, double* sums) {
+    sums[0] = loss_sum[0];
+    sums[1] = loss_sum[1];
+    sums[2] = (double)count[0];
+}
+
+// sums = (sum of per-position losses of the +eps pass, of the -eps pass, labelled positions).
+__global__ void finish_step_kernel(const double* sums, float eps, float lr,
+                                   const int32_t* err_flag, zoqat_step_result_dev* result) {
+    const double n = sums[2] > 0.0 ? sums[2] : 1.0;
+    const double lp = sums[0] / n, lm = sums[1] / n;
+    const float g = (float)((lp - lm) / (2.0 * (double)eps));
+    result->loss_plus = (float)lp;
+    result->loss_minus = (float)lm;
+    result->proj_grad = g;
+    result->update_scale = __fmul_rn(lr, g);
+    result->status = err_flag ? *err_flag : 0;
+    result->n_labels = (int32_t)sums[2];
+}
+
+__global__ void store_loss_kernel(const double* loss_sum, const int32_t* count, float* loss_out) {
+    const int n = count[0] > 0 ? count[0] : 1;
+    *loss_out = (float)(loss_sum[0] / n);
+}
+
+}  // namespace
+
+void launch_embed(const int32_t* tokens, const float* embed, const float* pos, int64_t T, int seq, int d, int vocab,
+                  int passes, float* h, cudaStream_t s) {
+    embed_kernel<<<(unsigned)T, 128, 0, s>>>(tokens, reinterpret_cast<const float4*>(embed),
+                                             reinterpret_cast<const float4*>(pos), T, seq, d / 4, vocab, passes,
+                                             reinterpret_cast<float4*>(h));
+    count_launch();
+}
+
+void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
+                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s) {
+    const size_t smem = (size_t)cols * sizeof(float);
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+    norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    count_launch();
+}
+
+void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
+                            float* row_step, cudaStream_t s) {
+    const size_t smem = (size_t)cols * sizeof(float);
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+    ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step);
+    count_launch();
+}
+
+void launch_ce_finalize(const float2* partials, const float* label_logit, const int32_t* labels, int64_t M, int Z,
+                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, cudaStream_t s) {
+    const int64_t rows = M * Z;
+    ce_token_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(partials, label_logit, labels, M, rows, n_tiles, token_loss);
+    ce_sum_kernel<<<Z, 1024, 0, s>>>(token_loss, labels, M, loss_sum, count);
+    count_launch(2);
+}
+
+void launch_pack_sums(const double* loss_sum, const int32_t* count, double* sums, cudaStream_t s) {
+    pack_sums_kernel<<<1, 1, 0, s>>>(loss_sum, count, sums);
+    count_launch();
+}
+
+void launch_finish_step(const double* sums, float eps, float lr, const int32_t* err_flag,
+                        zoqat_step_result_dev* result, cudaStream_t s) {
+    finish_step_kernel<<<1, 1, 0, s>>>(sums, eps, lr, err_flag, result);
+    count_launch();
+}
+
+void launch_store_loss(const double* loss_sum, const int32_t* count, float* loss_out, cudaStream_t s) {
+    store_loss_kernel<<<1, 1, 0, s>>>(loss_sum, count, loss_out);
+    count_launch();
+}
+
+void launch_copy_rows(const float* src, float* dst, int64_t n_floats, cudaStream_t s) {
+    const int64_t n4 = n_floats / 4;
+    int64_t blocks = (n4 + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    copy_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), n4);
+    count_launch();
+}
+
+}  // namespace zq

@@ -1,0 +1,765 @@
+// C ABI of libzoqat (see include/zoqat.h) and the host-side step engine: model
+// description, workspace layout, the layer loop of the quantised forward, the
+// two-pass schedule of Eq. (1) and the update of Eq. (2).  Host code only; every
+// arithmetic step of the path runs in the kernels of this directory.
+#include "common.cuh"
+#include "../../include/zoqat.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace zq;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int code, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    g_last_error = buf;
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char* what) {
+    return fail(ZOQAT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define CUDA_TRY(expr)                                              \
+    do {                                                            \
+        cudaError_t e__ = (expr);                                   \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr);       \
+    } while (0)
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Linear {
+    const float* w = nullptr;
+    float* w_mut = nullptr;
+    const float* bias = nullptr;
+    uint32_t flags = 0;
+    uint32_t tid = 0;
+    int64_t rows = 0, cols = 0;
+    const uint32_t* packed = nullptr;
+    const float2* qparams = nullptr;
+    bool present = false;
+    bool trainable() const { return (flags & ZOQAT_TENSOR_TRAINABLE) && !(flags & ZOQAT_TENSOR_FROZEN_PACKED); }
+    bool packed_frozen() const { return flags & ZOQAT_TENSOR_FROZEN_PACKED; }
+    int bits(int w_bits) const { return (flags & (ZOQAT_TENSOR_QUANTIZED | ZOQAT_TENSOR_FROZEN_PACKED)) ? w_bits : 0; }
+};
+
+struct Layer {
+    Linear lin[7];                      // indexed by ZOQAT_ROLE_WQ .. ZOQAT_ROLE_W_DOWN
+    const float* vec[ZOQAT_ROLE_COUNT] = {nullptr};   // norm gains / biases / linear biases by role
+    bool any_trainable = false;
+};
+
+struct Workspace {
+    int32_t *tokens, *labels;
+    float *h, *row_step, *qkv, *att, *ffn, *rope_cos, *rope_sin, *bias_qkv, *label_logit, *token_loss;
+    __nv_bfloat16 *xa, *bop;
+    float2* ce_partials;
+    double* loss_sum;
+    double* sums;                       // (sum L+, sum L-, labelled positions) of the last pair of passes
+    int32_t *count, *err_flag;
+    zoqat_step_result_dev* result;
+    size_t bop_elems;                   // elements of ONE pass' operand buffer
+    size_t total;
+};
+
+// Lays the workspace out; base may be NULL to only compute the size.
+void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
+    const size_t T = (size_t)c.max_batch * c.max_seq, R = 2 * T;
+    const size_t d = c.d_model, F = c.d_ffn, V = c.vocab;
+    const size_t ffn_cols = (c.arch == ZOQAT_ARCH_LLAMA) ? 2 * F : F;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { uint8_t* p = base ? base + off : nullptr; off += align_up(bytes); return p; };
+    w.tokens = (int32_t*)take(T * 4);
+    w.labels = (int32_t*)take(T * 4);
+    w.h = (float*)take(R * d * 4);
+    w.xa = (__nv_bfloat16*)take(R * (d > F ? d : F) * 2);
+    w.row_step = (float*)take(R * 4);
+    w.qkv = (float*)take(R * 3 * d * 4);
+    w.att = (float*)take(R * d * 4);
+    w.ffn = (float*)take(R * ffn_cols * 4);
+    size_t bmax = 3 * d * d;
+    if (ffn_cols * d > bmax) bmax = ffn_cols * d;
+    if (V * d > bmax) bmax = V * d;
+    w.bop_elems = bmax;
+    w.bop = (__nv_bfloat16*)take(2 * bmax * 2);
+    w.rope_cos = (float*)take((size_t)c.max_seq * (d / c.n_heads / 2) * 4);
+    w.rope_sin = (float*)take((size_t)c.max_seq * (d / c.n_heads / 2) * 4);
+    w.bias_qkv = (float*)take((size_t)c.n_layers * 3 * d * 4);
+    const size_t ce_tiles = (V + 127) / 128;          // enough for either GEMM implementation
+    w.ce_partials = (float2*)take(R * ce_tiles * 8);
+    w.label_logit = (float*)take(R * 4);
+    w.token_loss = (float*)take(R * 4);
+    w.loss_sum = (double*)take(2 * 8);
+    w.sums = (double*)take(3 * 8);
+    w.count = (int32_t*)take(2 * 4);
+    w.err_flag = (int32_t*)take(4);
+    w.result = (zoqat_step_result_dev*)take(sizeof(zoqat_step_result_dev));
+    w.total = off;
+}
+
+int validate_config(const zoqat_config_t* c) {
+    if (!c) return fail(ZOQAT_ERR_INVALID_ARG, "config is NULL");
+    if (c->arch != ZOQAT_ARCH_LLAMA && c->arch != ZOQAT_ARCH_OPT) return fail(ZOQAT_ERR_INVALID_ARG, "unknown arch %d", c->arch);
+    if (c->n_layers < 0 || c->d_model <= 0 || c->n_heads <= 0 || c->d_ffn <= 0 || c->vocab <= 0 || c->max_batch <= 0 || c->max_seq <= 0)
+        return fail(ZOQAT_ERR_INVALID_ARG, "sizes must be positive");
+    if (c->d_model % 64 || c->d_ffn % 64) return fail(ZOQAT_ERR_UNSUPPORTED, "d_model and d_ffn must be multiples of 64");
+    if (c->d_model % c->n_heads) return fail(ZOQAT_ERR_INVALID_ARG, "n_heads must divide d_model");
+    const int dh = c->d_model / c->n_heads;
+    if (dh != 64 && dh != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", dh);
+    if (c->w_bits != 2 && c->w_bits != 3 && c->w_bits != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "w_bits %d (supported: 2, 3, 4)", c->w_bits);
+    if (c->w_group != 32 && c->w_group != 64 && c->w_group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "w_group %d (supported: 32, 64, 128)", c->w_group);
+    if (c->d_model % c->w_group || c->d_ffn % c->w_group) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
+    if (c->a_bits != 0 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 8)", c->a_bits);
+    if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
+    if ((int64_t)c->max_batch * c->max_seq > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "max_batch*max_seq too large");
+    return ZOQAT_OK;
+}
+
+}  // namespace
+
+// Optional per-category device timing: a CUDA event pair around every launch group.
+struct Profiler {
+    static constexpr int kCats = ZOQAT_PROF_COUNT;
+    bool on = false;
+    std::vector<cudaEvent_t> pool;
+    std::vector<int> cat_of;            // category of event pair i
+    size_t used = 0;                    // pairs in flight since the last read
+    double ms[kCats] = {0};
+    long long n[kCats] = {0};
+    cudaEvent_t get(size_t i) {
+        while (pool.size() <= i) {
+            cudaEvent_t e;
+            cudaEventCreate(&e);
+            pool.push_back(e);
+        }
+        return pool[i];
+    }
+    void collect() {
+        for (size_t i = 0; i < used; ++i) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, pool[2 * i], pool[2 * i + 1]) == cudaSuccess) {
+                ms[cat_of[i]] += t;
+                n[cat_of[i]] += 1;
+            }
+        }
+        used = 0;
+    }
+    ~Profiler() { for (auto e : pool) cudaEventDestroy(e); }
+};
+
+struct zoqat_model {
+    Profiler prof;
+    zoqat_config_t cfg;
+    std::vector<Layer> layers;
+    const float *embed = nullptr, *pos = nullptr, *final_g = nullptr, *final_b = nullptr;
+    Linear head;
+    Workspace ws;
+    int first_trainable_layer = 0;      // n_layers if no block tensor is trainable
+    bool any_packed = false, prequantized = false;
+    long long launches_at_create = 0;
+};
+
+namespace {
+
+struct ProfScope {
+    Profiler& p; cudaStream_t s; size_t idx = 0; bool live;
+    ProfScope(zoqat_model* m, int cat, cudaStream_t st) : p(m->prof), s(st), live(m->prof.on) {
+        if (!live) return;
+        idx = p.used++;
+        if (p.cat_of.size() <= idx) p.cat_of.resize(idx + 1);
+        p.cat_of[idx] = cat;
+        p.get(2 * idx + 1);
+        cudaEventRecord(p.pool[2 * idx], s);
+    }
+    ~ProfScope() { if (live) cudaEventRecord(p.pool[2 * idx + 1], s); }
+};
+
+int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
+    ProfScope ps(m, ZOQAT_PROF_GEMM, s);
+    g.err_flag = m->ws.err_flag;
+    const int rc = (m->cfg.gemm_impl == ZOQAT_GEMM_SIMT) ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "GEMM launch rejected (M=%lld N=%lld K=%lld)", (long long)g.M, (long long)g.N, (long long)g.K);
+    return ZOQAT_OK;
+}
+
+// Writes the bf16 matmul operand(s) of one linear at `dst` (+ pass stride for the second pass).
+// passes == 1: operand of W + eps*u (eps signed).  passes == 2: +eps at dst, -eps at dst + pass_stride.
+void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t pass_stride, int passes,
+                     uint64_t seed, float eps, cudaStream_t s) {
+    ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
+    const int64_t n = L.rows * L.cols;
+    const int bits = L.bits(m->cfg.w_bits);
+    if (L.packed_frozen()) {
+        launch_unpack_operand(L.packed, L.qparams, n, m->cfg.w_group, m->cfg.w_bits, dst, s);
+        if (passes == 2) cudaMemcpyAsync(dst + pass_stride, dst, (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
+        return;
+    }
+    const int perturb = L.trainable() && eps != 0.0f;
+    if (passes == 2 && perturb) {
+        launch_weight_operand(L.w, n, m->cfg.w_group, bits, 1, seed, L.tid, eps, dst, dst + pass_stride, nullptr, nullptr, nullptr, s);
+    } else {
+        launch_weight_operand(L.w, n, m->cfg.w_group, bits, perturb, seed, L.tid, eps, dst, nullptr, nullptr, nullptr, nullptr, s);
+        if (passes == 2) cudaMemcpyAsync(dst + pass_stride, dst, (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
+    }
+}
+
+// The quantised forward.  passes = 1: loss of W + eps*u (eps signed) in loss_sum[0].
+// passes = 2: +eps in loss_sum[0] and -eps in loss_sum[1], evaluated side by side on 2T rows.
+// Layers before the first trainable one see the same weights in both passes and run once.
+int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int batch, int seq, uint64_t seed,
+            float eps, int passes, cudaStream_t s) {
+    const zoqat_config_t& c = m->cfg;
+    Workspace& w = m->ws;
+    const int64_t T = (int64_t)batch * seq;
+    const int d = c.d_model, F = c.d_ffn, H = c.n_heads, dh = d / H;
+    const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
+    const int norm_kind = llama ? 1 : 2;
+    const size_t ps = w.bop_elems;
+
+    int Z = (passes == 2 && m->first_trainable_layer == 0) ? 2 : 1;     // passes currently materialised as rows
+    { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_embed(tokens, m->embed, m->pos, T, seq, d, c.vocab, Z, w.h, s); }
+
+    for (int l = 0; l < c.n_layers; ++l) {
+        const Layer& Ly = m->layers[l];
+        if (passes == 2 && Z == 1 && l >= m->first_trainable_layer) {
+            { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_copy_rows(w.h, w.h + T * d, T * d, s); }   // the shared prefix ends here
+            Z = 2;
+        }
+        const int64_t R = Z * T;
+        // --- attention block
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
+          launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s); }
+        for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
+            produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s);
+        GemmArgs g{};
+        g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
+        g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
+        g.out = w.qkv; g.b_stride = ps;
+        if (int rc = run_gemm(m, g, s)) return rc;
+        { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s); launch_attention(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, w.att, s); }
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s);
+        g = GemmArgs{};
+        g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
+        g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
+        if (int rc = run_gemm(m, g, s)) return rc;
+        // --- feed-forward block
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
+          launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s); }
+        const int n_up = llama ? 2 * F : F;
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s);
+        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s);
+        g = GemmArgs{};
+        g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
+        g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
+        if (int rc = run_gemm(m, g, s)) return rc;
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s);
+        g = GemmArgs{};
+        g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
+        g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
+        if (int rc = run_gemm(m, g, s)) return rc;
+    }
+    if (passes == 2 && Z == 1) {
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_copy_rows(w.h, w.h + T * d, T * d, s); }
+        Z = 2;
+    }
+    // --- final norm, vocabulary projection fused with the cross-entropy
+    { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.h, Z * T, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s); }
+    produce_operand(m, m->head, w.bop, ps, Z, seed, eps, s);
+    GemmArgs g{};
+    g.A = w.xa; g.B = w.bop; g.M = T; g.N = c.vocab; g.K = d; g.Z = Z; g.b_stride = ps;
+    g.mode = 1; g.labels = labels; g.partials = w.ce_partials; g.label_logit = w.label_logit;
+    if (int rc = run_gemm(m, g, s)) return rc;
+    { ProfScope ps_(m, ZOQAT_PROF_LOSS, s);
+      launch_ce_finalize(w.ce_partials, w.label_logit, labels, T, Z, gemm_ce_tiles(c.vocab, c.gemm_impl), w.token_loss,
+                         w.loss_sum, w.count, s); }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "forward launch");
+    return ZOQAT_OK;
+}
+
+int check_call(zoqat_model* m, const void* tokens, const void* labels, int batch, int seq) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (!tokens || !labels) return fail(ZOQAT_ERR_INVALID_ARG, "tokens/labels are NULL");
+    if (batch <= 0 || seq <= 0 || batch > m->cfg.max_batch || seq > m->cfg.max_seq ||
+        (int64_t)batch * seq > (int64_t)m->cfg.max_batch * m->cfg.max_seq)
+        return fail(ZOQAT_ERR_INVALID_ARG, "batch %d x seq %d exceeds the configured maximum %d x %d", batch, seq,
+                    m->cfg.max_batch, m->cfg.max_seq);
+    if (m->any_packed && !m->prequantized)
+        return fail(ZOQAT_ERR_BAD_STATE, "frozen packed tensors present: call zoqat_prequantize_frozen first");
+    return ZOQAT_OK;
+}
+
+void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float scale_val, cudaStream_t s) {
+    ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r) {
+            Linear& L = Ly.lin[r];
+            if (L.present && L.trainable()) launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
+        }
+    if (m->head.trainable())
+        launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
+}
+
+}  // namespace
+
+// =============================================================================
+extern "C" {
+
+const char* zoqat_status_string(int status) {
+    switch (status) {
+        case ZOQAT_OK: return "ok";
+        case ZOQAT_ERR_INVALID_ARG: return "invalid argument";
+        case ZOQAT_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ZOQAT_ERR_WORKSPACE_SMALL: return "workspace too small";
+        case ZOQAT_ERR_CUDA: return "CUDA error";
+        case ZOQAT_ERR_BAD_STATE: return "call out of order";
+        case ZOQAT_ERR_TIMEOUT: return "a bounded device wait ran out";
+        default: return "unknown status";
+    }
+}
+
+const char* zoqat_last_error(void) { return g_last_error.c_str(); }
+
+int zoqat_query_workspace(const zoqat_config_t* cfg, size_t* bytes) {
+    if (int rc = validate_config(cfg)) return rc;
+    if (!bytes) return fail(ZOQAT_ERR_INVALID_ARG, "bytes is NULL");
+    Workspace w;
+    layout_workspace(*cfg, nullptr, w);
+    *bytes = w.total;
+    return ZOQAT_OK;
+}
+
+int zoqat_packed_bytes(int64_t rows, int64_t cols, int bits, int group, size_t* code_bytes, size_t* qparam_bytes) {
+    if (rows <= 0 || cols <= 0 || (bits != 2 && bits != 3 && bits != 4) || (group != 32 && group != 64 && group != 128))
+        return fail(ZOQAT_ERR_INVALID_ARG, "bad packed-size query");
+    if (cols % group || (rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128 and cols of the group");
+    if (code_bytes) *code_bytes = (size_t)(rows * cols / 128) * 16 * bits;
+    if (qparam_bytes) *qparam_bytes = (size_t)(rows * cols / group) * 8;
+    return ZOQAT_OK;
+}
+
+int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* tensors, int n_tensors,
+                       void* workspace_dev, size_t bytes, zoqat_model_t** out) {
+    if (int rc = validate_config(cfg)) return rc;
+    if (!tensors || n_tensors <= 0 || !out) return fail(ZOQAT_ERR_INVALID_ARG, "tensors/out are NULL");
+    if (!workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) & 255)) return fail(ZOQAT_ERR_INVALID_ARG, "workspace must be 256-byte aligned device memory");
+    int dev = 0, major = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    if (major != 10) return fail(ZOQAT_ERR_UNSUPPORTED, "this library is built for sm_100a only (device is sm_%d*)", major);
+
+    zoqat_model* m = new (std::nothrow) zoqat_model();
+    if (!m) return fail(ZOQAT_ERR_CUDA, "out of host memory");
+    m->cfg = *cfg;
+    layout_workspace(*cfg, static_cast<uint8_t*>(workspace_dev), m->ws);
+    if (bytes < m->ws.total) { size_t need = m->ws.total; delete m; return fail(ZOQAT_ERR_WORKSPACE_SMALL, "workspace %zu < %zu bytes", bytes, need); }
+    m->layers.resize(cfg->n_layers);
+    const bool llama = cfg->arch == ZOQAT_ARCH_LLAMA;
+    const int d = cfg->d_model, F = cfg->d_ffn;
+
+    for (int i = 0; i < n_tensors; ++i) {
+        const zoqat_tensor_desc_t& t = tensors[i];
+        if (t.role < 0 || t.role >= ZOQAT_ROLE_COUNT) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: unknown role %d", i, t.role); }
+        const bool is_packed = t.flags & ZOQAT_TENSOR_FROZEN_PACKED;
+        if (!t.data && !is_packed) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: data is NULL", i); }
+        if (reinterpret_cast<uintptr_t>(t.data) & 15) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: data must be 16-byte aligned", i); }
+        if (t.role <= ZOQAT_ROLE_B_FC2) {
+            if (t.layer < 0 || t.layer >= cfg->n_layers) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: layer %d out of range", i, t.layer); }
+            Layer& Ly = m->layers[t.layer];
+            if (t.role <= ZOQAT_ROLE_W_DOWN) {
+                Linear& L = Ly.lin[t.role];
+                if (L.present) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: role %d of layer %d given twice", i, t.role, t.layer); }
+                L.present = true;
+                L.w = static_cast<const float*>(t.data);
+                L.w_mut = static_cast<float*>(t.data);
+                L.flags = t.flags;
+                L.tid = 16u * (uint32_t)(t.layer + 1) + (uint32_t)t.role;
+                const bool up = t.role == ZOQAT_ROLE_W_GATE || t.role == ZOQAT_ROLE_W_UP;
+                L.rows = up ? F : d;
+                L.cols = t.role == ZOQAT_ROLE_W_DOWN ? F : d;
+                if (is_packed) {
+                    if (!t.packed || !t.qparams) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: packed/qparams are NULL", i); }
+                    if ((L.rows * L.cols) % 128) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need rows*cols %% 128 == 0", i); }
+                    L.packed = static_cast<const uint32_t*>(t.packed);
+                    L.qparams = static_cast<const float2*>(t.qparams);
+                    m->any_packed = true;
+                }
+                if (L.trainable()) Ly.any_trainable = true;
+            } else {
+                Ly.vec[t.role] = static_cast<const float*>(t.data);
+            }
+        } else if (t.role == ZOQAT_ROLE_EMBED) m->embed = static_cast<const float*>(t.data);
+        else if (t.role == ZOQAT_ROLE_POS_EMBED) m->pos = static_cast<const float*>(t.data);
+        else if (t.role == ZOQAT_ROLE_FINAL_NORM_G) m->final_g = static_cast<const float*>(t.data);
+        else if (t.role == ZOQAT_ROLE_FINAL_NORM_B) m->final_b = static_cast<const float*>(t.data);
+        else if (t.role == ZOQAT_ROLE_LM_HEAD) {
+            if (is_packed || (t.flags & ZOQAT_TENSOR_QUANTIZED)) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "the vocabulary projection is kept unquantised"); }
+            m->head.present = true;
+            m->head.w = static_cast<const float*>(t.data);
+            m->head.w_mut = static_cast<float*>(t.data);
+            m->head.flags = t.flags;
+            m->head.tid = 0;
+            m->head.rows = cfg->vocab;
+            m->head.cols = d;
+        }
+    }
+    // completeness
+    auto missing = [&](const char* what, int layer) {
+        delete m;
+        return fail(ZOQAT_ERR_INVALID_ARG, "missing tensor: %s (layer %d)", what, layer);
+    };
+    if (!m->embed) return missing("embedding", -1);
+    if (!m->final_g) return missing("final norm gain", -1);
+    if (!m->head.present) return missing("vocabulary projection", -1);
+    if (!llama && (!m->pos || !m->final_b)) return missing("positions / final norm bias", -1);
+    m->first_trainable_layer = cfg->n_layers;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        Layer& Ly = m->layers[l];
+        for (int r = 0; r < 7; ++r)
+            if (!Ly.lin[r].present && !(r == ZOQAT_ROLE_W_UP && !llama)) return missing("block linear", l);
+        if (!Ly.vec[ZOQAT_ROLE_ATTN_NORM_G] || !Ly.vec[ZOQAT_ROLE_FFN_NORM_G]) return missing("norm gain", l);
+        if (!llama)
+            for (int r : {ZOQAT_ROLE_ATTN_NORM_B, ZOQAT_ROLE_FFN_NORM_B, ZOQAT_ROLE_BQ, ZOQAT_ROLE_BK, ZOQAT_ROLE_BV,
+                          ZOQAT_ROLE_BO, ZOQAT_ROLE_B_FC1, ZOQAT_ROLE_B_FC2})
+                if (!Ly.vec[r]) return missing("bias", l);
+        if (Ly.any_trainable && m->first_trainable_layer == cfg->n_layers) m->first_trainable_layer = l;
+    }
+    // one-time tables: rotary cos/sin (evaluated in double, stored fp32) and concatenated q|k|v biases
+    if (llama) {
+        const int dh = d / cfg->n_heads, half = dh / 2;
+        std::vector<float> cs((size_t)cfg->max_seq * half), sn((size_t)cfg->max_seq * half);
+        for (int i = 0; i < half; ++i) {
+            const double inv_freq = std::pow((double)cfg->rope_base, -2.0 * i / dh);
+            for (int p = 0; p < cfg->max_seq; ++p) {
+                cs[(size_t)p * half + i] = (float)std::cos(p * inv_freq);
+                sn[(size_t)p * half + i] = (float)std::sin(p * inv_freq);
+            }
+        }
+        cudaError_t e = cudaMemcpy(m->ws.rope_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(m->ws.rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { delete m; return cuda_fail(e, "rotary table upload"); }
+    } else {
+        for (int l = 0; l < cfg->n_layers; ++l) {
+            const int roles[3] = {ZOQAT_ROLE_BQ, ZOQAT_ROLE_BK, ZOQAT_ROLE_BV};
+            for (int j = 0; j < 3; ++j) {
+                cudaError_t e = cudaMemcpy(m->ws.bias_qkv + ((size_t)l * 3 + j) * d, m->layers[l].vec[roles[j]], (size_t)d * 4, cudaMemcpyDeviceToDevice);
+                if (e != cudaSuccess) { delete m; return cuda_fail(e, "bias concatenation"); }
+            }
+        }
+    }
+    cudaError_t e = cudaMemset(m->ws.err_flag, 0, 4);
+    if (e != cudaSuccess) { delete m; return cuda_fail(e, "workspace init"); }
+    m->launches_at_create = g_launch_count;
+    *out = m;
+    return ZOQAT_OK;
+}
+
+int zoqat_model_destroy(zoqat_model_t* m) {
+    delete m;
+    return ZOQAT_OK;
+}
+
+int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r) {
+            Linear& L = Ly.lin[r];
+            if (!L.present || !L.packed_frozen()) continue;
+            if (!L.w) return fail(ZOQAT_ERR_BAD_STATE, "frozen tensor has no fp32 source to quantise");
+            launch_pack_frozen(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, const_cast<uint32_t*>(L.packed),
+                               const_cast<float2*>(L.qparams), s);
+        }
+    CUDA_TRY(cudaGetLastError());
+    m->prequantized = true;
+    return ZOQAT_OK;
+}
+
+int zoqat_forward_loss(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                       uint64_t seed, float signed_eps, float* loss_out_dev, void* stream) {
+    if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
+    if (!loss_out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "loss_out_dev is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, signed_eps, 1, s)) return rc;
+    launch_store_loss(m->ws.loss_sum, m->ws.count, loss_out_dev, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step_begin(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                     uint64_t seed, float eps, double* sums_dev, void* stream) {
+    if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
+    if (!sums_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev is NULL");
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, eps, 2, s)) return rc;
+    launch_pack_sums(m->ws.loss_sum, m->ws.count, sums_dev, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step_finish(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                      zoqat_step_result_t* result_dev, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (!sums_dev || !result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev/result_dev are NULL");
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(result_dev);
+    launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, res, s);
+    update_all(m, seed, &res->update_scale, 0.0f, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+               uint64_t seed, float eps, float lr, zoqat_step_result_t* result_dev, void* stream) {
+    if (!result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "result_dev is NULL");
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (int rc = zoqat_step_begin(m, tokens_dev, labels_dev, batch, seq, seed, eps, m->ws.sums, stream)) return rc;
+    return zoqat_step_finish(m, m->ws.sums, seed, eps, lr, result_dev, stream);
+}
+
+int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
+                    uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream) {
+    if (int rc = check_call(m, tokens_host, labels_host, batch, seq)) return rc;
+    if (!result_host) return fail(ZOQAT_ERR_INVALID_ARG, "result_host is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t nb = (size_t)batch * seq * 4;
+    CUDA_TRY(cudaMemcpyAsync(m->ws.tokens, tokens_host, nb, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(cudaMemcpyAsync(m->ws.labels, labels_host, nb, cudaMemcpyHostToDevice, s));
+    if (int rc = zoqat_step(m, m->ws.tokens, m->ws.labels, batch, seq, seed, eps, lr,
+                            reinterpret_cast<zoqat_step_result_t*>(m->ws.result), s))
+        return rc;
+    CUDA_TRY(cudaMemcpyAsync(result_host, m->ws.result, sizeof(zoqat_step_result_t), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    if (result_host->status != 0) return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", result_host->status);
+    return ZOQAT_OK;
+}
+
+int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    update_all(m, seed, nullptr, scale, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_check(zoqat_model_t* m, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t flag = 0;
+    CUDA_TRY(cudaMemcpyAsync(&flag, m->ws.err_flag, 4, cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    if (flag != 0) {
+        cudaMemsetAsync(m->ws.err_flag, 0, 4, s);
+        return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", flag);
+    }
+    return ZOQAT_OK;
+}
+
+int zoqat_launch_count(const zoqat_model_t* m, int64_t* launches) {
+    if (!m || !launches) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    *launches = g_launch_count - m->launches_at_create;
+    return ZOQAT_OK;
+}
+
+int zoqat_profile_enable(zoqat_model_t* m, int on) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    m->prof.on = on != 0;
+    return ZOQAT_OK;
+}
+
+int zoqat_profile_read(zoqat_model_t* m, int category, double* ms, int64_t* intervals, void* stream) {
+    if (!m || !ms || !intervals) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (category < 0 || category >= ZOQAT_PROF_COUNT) return fail(ZOQAT_ERR_INVALID_ARG, "unknown category %d", category);
+    CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    m->prof.collect();
+    *ms = m->prof.ms[category];
+    *intervals = m->prof.n[category];
+    m->prof.ms[category] = 0.0;
+    m->prof.n[category] = 0;
+    return ZOQAT_OK;
+}
+
+int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* bytes) {
+    if (!m || !dev_ptr || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    const zoqat_config_t& c = m->cfg;
+    const size_t R = 2 * (size_t)c.max_batch * c.max_seq;
+    const size_t ffn_cols = (c.arch == ZOQAT_ARCH_LLAMA) ? 2 * (size_t)c.d_ffn : (size_t)c.d_ffn;
+    switch (which) {
+        case ZOQAT_BUF_RESIDUAL: *dev_ptr = m->ws.h; *bytes = R * c.d_model * 4; break;
+        case ZOQAT_BUF_QKV: *dev_ptr = m->ws.qkv; *bytes = R * 3 * c.d_model * 4; break;
+        case ZOQAT_BUF_ATTN: *dev_ptr = m->ws.att; *bytes = R * c.d_model * 4; break;
+        case ZOQAT_BUF_FFN: *dev_ptr = m->ws.ffn; *bytes = R * ffn_cols * 4; break;
+        case ZOQAT_BUF_TOKEN_LOSS: *dev_ptr = m->ws.token_loss; *bytes = R * 4; break;
+        default: return fail(ZOQAT_ERR_INVALID_ARG, "unknown buffer %d", which);
+    }
+    return ZOQAT_OK;
+}
+
+// ---- single operations ---------------------------------------------------------
+static int check_group_bits(int64_t rows, int64_t cols, int group, int bits, bool allow_zero_bits) {
+    if (rows <= 0 || cols <= 0) return fail(ZOQAT_ERR_INVALID_ARG, "rows/cols must be positive");
+    if (group != 32 && group != 64 && group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "group %d (supported: 32, 64, 128)", group);
+    if (cols % group) return fail(ZOQAT_ERR_INVALID_ARG, "group must divide cols");
+    if (!((bits >= 2 && bits <= 4) || (allow_zero_bits && bits == 0))) return fail(ZOQAT_ERR_UNSUPPORTED, "bits %d", bits);
+    return ZOQAT_OK;
+}
+
+int zoqat_op_philox_words(uint64_t seed, uint32_t tensor_id, uint64_t blk0, uint64_t nblk, uint32_t* out_dev, void* stream) {
+    if (!out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "out_dev is NULL");
+    launch_philox_words(seed, tensor_id, blk0, nblk, out_dev, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_normal(uint64_t seed, uint32_t tensor_id, uint64_t n, float* out_dev, void* stream) {
+    if (!out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "out_dev is NULL");
+    launch_normal(seed, tensor_id, n, out_dev, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_weight_quant(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
+                          uint32_t tensor_id, float signed_eps, uint8_t* codes_dev, float* step_dev, int32_t* zp_dev,
+                          void* operand_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
+    if (!w_dev || !operand_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_dev are NULL");
+    launch_weight_operand(w_dev, rows * cols, group, bits, signed_eps != 0.0f, seed, tensor_id, signed_eps,
+                          static_cast<__nv_bfloat16*>(operand_dev), nullptr, codes_dev, step_dev, zp_dev,
+                          static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
+                                 uint32_t tensor_id, float eps, void* operand_plus_dev, void* operand_minus_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
+    if (!w_dev || !operand_plus_dev || !operand_minus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    launch_weight_operand(w_dev, rows * cols, group, bits, 1, seed, tensor_id, eps, static_cast<__nv_bfloat16*>(operand_plus_dev),
+                          static_cast<__nv_bfloat16*>(operand_minus_dev), nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, void* packed_dev,
+                         void* qparams_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
+    if (!w_dev || !packed_dev || !qparams_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    launch_pack_frozen(w_dev, rows * cols, group, bits, static_cast<uint32_t*>(packed_dev), static_cast<float2*>(qparams_dev),
+                       static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group,
+                            int bits, void* operand_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
+    if (!packed_dev || !qparams_dev || !operand_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    launch_unpack_operand(static_cast<const uint32_t*>(packed_dev), static_cast<const float2*>(qparams_dev), rows * cols,
+                          group, bits, static_cast<__nv_bfloat16*>(operand_dev), static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_update(float* w_dev, uint64_t n, uint64_t seed, uint32_t tensor_id, float scale, void* stream) {
+    if (!w_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev is NULL");
+    if (reinterpret_cast<uintptr_t>(w_dev) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev must be 16-byte aligned");
+    launch_update(w_dev, n, seed, tensor_id, nullptr, scale, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_norm_act_operand(const float* x_dev, int64_t rows, int64_t cols, int norm_kind, const float* gain_dev,
+                              const float* bias_dev, float norm_eps, int a_bits, void* operand_dev, float* row_step_dev,
+                              float* normed_dev, void* stream) {
+    if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
+    if (norm_kind < 0 || norm_kind > 2 || (norm_kind >= 1 && !gain_dev) || (norm_kind == 2 && !bias_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "bad norm arguments");
+    if (a_bits != 0 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
+    launch_norm_act_operand(x_dev, rows, (int)cols, norm_kind, gain_dev, bias_dev, norm_eps, a_bits,
+                            static_cast<__nv_bfloat16*>(operand_dev), row_step_dev, normed_dev, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_ffn_act_operand(const float* x_dev, int64_t rows, int64_t cols, int gated, int a_bits, void* operand_dev,
+                             float* row_step_dev, void* stream) {
+    if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
+    if (a_bits != 0 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
+    launch_ffn_act_operand(x_dev, rows, (int)cols, gated, a_bits, static_cast<__nv_bfloat16*>(operand_dev), row_step_dev,
+                           static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, int64_t K, const float* row_step_dev,
+                  const float* bias_dev, int relu, int accumulate, float* out_dev, int impl, int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = M; g.N = N; g.K = K; g.Z = 1; g.row_step = row_step_dev; g.bias = bias_dev; g.relu = relu; g.accumulate = accumulate;
+    g.out = out_dev; g.err_flag = err_flag_dev; g.b_stride = (size_t)N * K;
+    const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, static_cast<cudaStream_t>(stream))
+                                           : launch_gemm_tc(g, static_cast<cudaStream_t>(stream));
+    if (rc != ZOQAT_OK) return fail(rc, "GEMM rejected: M=%lld N=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers, err flag for tcgen05)",
+                                    (long long)M, (long long)N, (long long)K);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_attention(const float* qkv_dev, int batch, int seq, int n_heads, int d_head, const float* cos_dev,
+                       const float* sin_dev, float* out_dev, void* stream) {
+    if (!qkv_dev || !out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (batch <= 0 || seq <= 0 || n_heads <= 0 || (d_head != 64 && d_head != 128)) return fail(ZOQAT_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", d_head);
+    if ((cos_dev == nullptr) != (sin_dev == nullptr)) return fail(ZOQAT_ERR_INVALID_ARG, "cos/sin tables must both be given or both NULL");
+    launch_attention(qkv_dev, batch, seq, n_heads, d_head, cos_dev, sin_dev, out_dev, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_head_loss_scratch_bytes(int64_t T, int64_t V, size_t* bytes) {
+    if (T <= 0 || V <= 0 || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "bad arguments");
+    *bytes = align_up((size_t)T * ((V + 127) / 128) * 8) + align_up((size_t)T * 4);
+    return ZOQAT_OK;
+}
+
+int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labels_dev, int64_t T, int64_t V, int64_t d,
+                       float* token_loss_dev, double* loss_sum_dev, int32_t* count_dev, void* scratch_dev, int impl,
+                       int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !labels_dev || !token_loss_dev || !loss_sum_dev || !count_dev || !scratch_dev)
+        return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float2* partials = static_cast<float2*>(scratch_dev);
+    float* label_logit = reinterpret_cast<float*>(static_cast<uint8_t*>(scratch_dev) + align_up((size_t)T * ((V + 127) / 128) * 8));
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = T; g.N = V; g.K = d; g.Z = 1; g.mode = 1; g.labels = labels_dev; g.partials = partials; g.label_logit = label_logit;
+    g.err_flag = err_flag_dev; g.b_stride = (size_t)V * d;
+    const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
+    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,83 @@
+// Shared declarations of the zoqat CUDA library (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace zq {
+
+// Device error words written by kernels whose bounded waits ran out.
+constexpr int kErrWaitFull = 1;      // MMA warp: operands never arrived
+constexpr int kErrWaitEmpty = 2;     // TMA warp: stage never released
+constexpr int kErrWaitAccFull = 3;   // epilogue: accumulator never committed
+constexpr int kErrWaitAccEmpty = 4;  // MMA warp: accumulator never drained
+
+// Host-side launch bookkeeping (one counter per process, read through the handle).
+extern long long g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count += n; }
+
+// ---------------------------------------------------------------------------
+// Launch functions (host).  Every pointer is device memory.
+// ---------------------------------------------------------------------------
+void launch_philox_words(uint64_t seed, uint32_t tid, uint64_t blk0, uint64_t nblk, uint32_t* out, cudaStream_t s);
+void launch_normal(uint64_t seed, uint32_t tid, uint64_t n, float* out, cudaStream_t s);
+
+// Weight producer.  n = rows*cols elements (multiple of group); bits in {0,2,3,4};
+// perturb = 0 skips the direction entirely (frozen tensors).
+// op_plus from W + eps*u; op_minus (may be NULL) from W - eps*u.
+// Debug outputs (may be NULL) describe the op_plus side.
+void launch_weight_operand(const float* w, int64_t n, int group, int bits, int perturb,
+                           uint64_t seed, uint32_t tid, float eps,
+                           __nv_bfloat16* op_plus, __nv_bfloat16* op_minus,
+                           uint8_t* codes, float* step, int32_t* zp, cudaStream_t s);
+void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);
+void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,
+                           __nv_bfloat16* op, cudaStream_t s);
+// w <- w - scale*u; scale = *scale_ptr if scale_ptr != NULL else scale_val.
+void launch_update(float* w, uint64_t n, uint64_t seed, uint32_t tid, const float* scale_ptr, float scale_val, cudaStream_t s);
+
+void launch_embed(const int32_t* tokens, const float* embed, const float* pos, int64_t T, int seq, int d,
+                  int vocab, int passes, float* h, cudaStream_t s);
+void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
+                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s);
+void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
+                            __nv_bfloat16* op, float* row_step, cudaStream_t s);
+void launch_attention(const float* qkv, int batch, int seq, int n_heads, int d_head,
+                      const float* cos_t, const float* sin_t, float* out, cudaStream_t s);
+
+// out[z*M + m, n] (+)= row_step[z*M+m] * sum_k A[z*M+m, k] * B[z][n, k] (+ bias[n]) (relu)
+// mode 1: cross-entropy partials instead of a store (labels[m], partials [Z*M, n_tiles], label_logit [Z*M]).
+struct GemmArgs {
+    const __nv_bfloat16* A;   // [Z*M, K]
+    const __nv_bfloat16* B;   // [Z][N, K], pass z starts at B + z*b_stride
+    size_t b_stride;          // elements between the B matrices of consecutive passes (multiple of 8)
+    int64_t M, N, K;
+    int Z;
+    const float* row_step;    // [Z*M] or NULL
+    const float* bias;        // [N] or NULL
+    int relu;
+    int accumulate;
+    float* out;               // [Z*M, N]
+    int mode;                 // 0 store, 1 cross-entropy partials
+    const int32_t* labels;    // [M]
+    float2* partials;         // [Z*M, ce_tiles] (max, sum exp)
+    float* label_logit;       // [Z*M]
+    int32_t* err_flag;
+};
+int gemm_ce_tiles(int64_t N, int impl);                 // column tiles the cross-entropy epilogue produces
+int launch_gemm_simt(const GemmArgs& a, cudaStream_t s);   // returns 0 or a ZOQAT_ERR_* code
+int launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
+
+// Per-position loss from the partials, then the deterministic sum.
+void launch_ce_finalize(const float2* partials, const float* label_logit, const int32_t* labels, int64_t M, int Z,
+                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, cudaStream_t s);
+// g, lr*g and the result record from the two loss sums.
+struct zoqat_step_result_dev { float loss_plus, loss_minus, proj_grad, update_scale; int32_t status, n_labels; };
+void launch_pack_sums(const double* loss_sum, const int32_t* count, double* sums, cudaStream_t s);
+void launch_finish_step(const double* sums, float eps, float lr, const int32_t* err_flag,
+                        zoqat_step_result_dev* result, cudaStream_t s);
+void launch_store_loss(const double* loss_sum, const int32_t* count, float* loss_out, cudaStream_t s);
+void launch_copy_rows(const float* src, float* dst, int64_t n_floats, cudaStream_t s);
+
+}  // namespace zq

@@ -1,0 +1,426 @@
+// Tensor-core GEMM for sm_100a: out = row_step * (A B^T) (+ bias), bf16 operands,
+// fp32 accumulation in tensor memory (TMEM), written with tcgen05 / TMA inline PTX.
+//
+// Structure (one persistent CTA per SM, 192 threads):
+//   warp 0     TMA producer: streams 128x64 A tiles and BNx64 B tiles (128-byte
+//              swizzle) into a ring of shared-memory stages, one elected lane.
+//   warp 1     MMA issuer: one lane issues tcgen05.mma (M=128, N=BN, K=16) over
+//              each stage and commits to the stage's "empty" barrier; owns TMEM.
+//   warps 2-5  epilogue: tcgen05.ld the 128xBN fp32 accumulator (each warp its
+//              32-lane quarter), apply the per-row step / bias / ReLU / residual
+//              add, or reduce the tile to cross-entropy partials (max, sum exp)
+//              so that logits never reach memory.
+// Two accumulators (2*BN of the 512 TMEM columns) let the epilogue of tile i
+// overlap the MMAs of tile i+1.
+//
+// Every wait is bounded: a wait that runs out records a code in *err_flag and
+// the role leaves its loop; the CTA then drains, frees its TMEM and returns.
+#include "common.cuh"
+#include "../../include/zoqat.h"
+#include <cuda.h>
+
+namespace zq {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kThreadsTC = 192;
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz
+
+template <int BN> struct TileCfg {
+    static constexpr int kStages = (BN == 256) ? 4 : 6;
+    static constexpr int kABytes = BM * BK * 2;
+    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
+};
+
+// ---- PTX wrappers ------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> fp32, one CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The barrier is signalled once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread = lane (row), v[j] = column j.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand tile whose rows are 128 bytes
+// (64 bf16) written by TMA with the 128-byte swizzle; 8-row groups are 1024 bytes
+// apart (stride byte offset); the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // bits  0-13 start address / 16
+    d |= (uint64_t)1 << 16;                          // bits 16-29 leading byte offset / 16 (ignored)
+    d |= (uint64_t)(1024 >> 4) << 32;                // bits 32-45 stride byte offset / 16
+    d |= (uint64_t)1 << 46;                          // bits 46-47 descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                          // bits 61-63 layout: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both K-major.
+template <int BN>
+__device__ __forceinline__ uint32_t idesc_bf16() {
+    return (1u << 4)                      // D format: f32
+         | (1u << 7)                      // A format: bf16
+         | (1u << 10)                     // B format: bf16
+         | ((uint32_t)(BN >> 3) << 17)    // N / 8
+         | ((uint32_t)(BM >> 4) << 24);   // M / 16
+}
+
+__device__ __forceinline__ void ce_merge(float& m, float& s, float v) {
+    if (v > m) { s = s * expf(m - v) + 1.0f; m = v; }
+    else s += expf(v - m);
+}
+
+struct TcParams {
+    int64_t M, N, K;
+    int Z;
+    const float* row_step;
+    const float* bias;
+    int relu, accumulate;
+    float* out;
+    int mode;
+    const int32_t* labels;
+    float2* partials;
+    float* label_logit;
+    int32_t* err_flag;
+    int tiles_m, tiles_n;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreadsTC, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
+    using Cfg = TileCfg<BN>;
+    constexpr int S = Cfg::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;              // 1024-byte aligned stage ring
+    const uint32_t bars = tiles + S * Cfg::kStageBytes;         // barriers follow the ring
+    // barrier layout (8 bytes each): full[S], empty[S], acc_full[2], acc_empty[2], then the TMEM base word
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
+    auto acc_full_bar = [&](int a) { return bars + 8u * (2 * S + a); };
+    auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * S + 2 + a); };
+    const uint32_t tmem_slot = bars + 8u * (2 * S + 4);
+    uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - raw));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = (int)((p.K + BK - 1) / BK);
+    const int tiles_per_z = p.tiles_m * p.tiles_n;
+    const int total_tiles = tiles_per_z * p.Z;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&map_a);
+        prefetch_tmap(&map_b);
+    }
+    if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns
+        tmem_alloc(tmem_slot, 2 * BN);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int z = t / tiles_per_z, r = t % tiles_per_z;
+                const int tm = r % p.tiles_m, tn = r / p.tiles_m;     // m fastest: neighbours share B
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { atomicExch(p.err_flag, kErrWaitEmpty); ok = false; break; }
+                    mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
+                    const uint32_t a_dst = tiles + stage * Cfg::kStageBytes;
+                    tma_load_3d(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z);
+                    tma_load_3d(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // drain: every load issued above must land before the CTA may exit
+            // (a stage is "landed" once the consumer released it or its full barrier completed)
+            for (int i = 0; i < S; ++i) {
+                // wait until the consumer has released the stage the producer would reuse next
+                if (!mbar_wait(empty_bar(stage), phase ^ 1u)) break;
+                if (++stage == S) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16<BN>();
+            int stage = 0; uint32_t phase = 0;
+            int acc = 0; uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u)) { atomicExch(p.err_flag, kErrWaitAccEmpty); break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase)) { atomicExch(p.err_flag, kErrWaitFull); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = tiles + stage * Cfg::kStageBytes;
+                    const uint64_t a_desc = smem_desc_sw128(a_addr);
+                    const uint64_t b_desc = smem_desc_sw128(a_addr + Cfg::kABytes);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // advance 16 elements = 32 bytes inside the swizzled row: +2 in the (addr/16) field
+                        umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(acc_full_bar(acc));             // accumulator complete
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------- epilogue (warps 2..5) ----------------
+        const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter+32)
+        int acc = 0; uint32_t acc_phase = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+            const int z = t / tiles_per_z, r = t % tiles_per_z;
+            const int tm = r % p.tiles_m, tn = r / p.tiles_m;
+            // the whole warp takes the same decision: the TMEM loads below are warp-collective
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase))) {
+                if (lane == 0) atomicExch(p.err_flag, kErrWaitAccFull);
+                break;
+            }
+            tc_fence_after();
+            const int64_t m = (int64_t)tm * BM + quarter * 32 + lane;
+            const bool row_ok = m < p.M;
+            const int64_t row = (int64_t)z * p.M + (row_ok ? m : 0);
+            const float rs = (p.row_step && row_ok) ? p.row_step[row] : 1.0f;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+            const int64_t n_base = (int64_t)tn * BN;
+            float ce_m = -INFINITY, ce_s = 0.0f;
+            const int32_t lab = (p.mode == 1 && row_ok) ? p.labels[m] : -1;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                __syncwarp();
+                tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+                tmem_ld_wait();
+                const int64_t n0 = n_base + c * 32;
+                if (n0 >= p.N) continue;                      // uniform: whole chunk out of range
+                if (p.mode == 0) {
+                    if (!row_ok) continue;
+                    float* o = p.out + row * p.N + n0;
+                    if (n0 + 32 <= p.N && (p.N & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 x;
+                            x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
+                            x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
+                            if (p.bias) {
+                                const float4 b = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+                                x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
+                            }
+                            if (p.relu) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
+                            if (p.accumulate) {
+                                const float4 h = *reinterpret_cast<const float4*>(o + j);
+                                x.x += h.x; x.y += h.y; x.z += h.z; x.w += h.w;
+                            }
+                            *reinterpret_cast<float4*>(o + j) = x;
+                        }
+                    } else {
+                        for (int j = 0; j < 32; ++j) {
+                            if (n0 + j >= p.N) break;
+                            float x = rs * __uint_as_float(v[j]);
+                            if (p.bias) x += p.bias[n0 + j];
+                            if (p.relu) x = fmaxf(x, 0.f);
+                            if (p.accumulate) x += o[j];
+                            o[j] = x;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (n0 + j < p.N) {
+                            const float x = rs * __uint_as_float(v[j]);
+                            ce_merge(ce_m, ce_s, x);
+                            if (n0 + j == lab) p.label_logit[row] = x;
+                        }
+                    }
+                }
+            }
+            if (p.mode == 1 && row_ok) p.partials[row * p.tiles_n + tn] = make_float2(ce_m, ce_s);
+            // accumulator drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2 * BN);
+    }
+}
+
+// ---- host side ------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 3-D map over a [Z][rows][K] bf16 array (K innermost), box = 64 x box_rows x 1, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int Z, size_t z_stride_elems, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)Z};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)z_stride_elems * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int num_sms() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int BN>
+int launch_tc(const GemmArgs& a, cudaStream_t s) {
+    using Cfg = TileCfg<BN>;
+    alignas(64) CUtensorMap map_a, map_b;
+    const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
+    if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN))
+        return ZOQAT_ERR_CUDA;
+    TcParams p;
+    p.M = a.M; p.N = a.N; p.K = a.K; p.Z = a.Z;
+    p.row_step = a.row_step; p.bias = a.bias; p.relu = a.relu; p.accumulate = a.accumulate;
+    p.out = a.out; p.mode = a.mode; p.labels = a.labels; p.partials = a.partials; p.label_logit = a.label_logit;
+    p.err_flag = a.err_flag;
+    p.tiles_m = (int)((a.M + BM - 1) / BM);
+    p.tiles_n = (int)((a.N + BN - 1) / BN);
+    static bool attr = false;
+    if (!attr) {
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+            return ZOQAT_ERR_CUDA;
+        attr = true;
+    }
+    const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
+    const int grid = (int)(total < num_sms() ? total : num_sms());
+    gemm_tc_kernel<BN><<<grid, kThreadsTC, Cfg::kSmemBytes, s>>>(map_a, map_b, p);
+    count_launch();
+    return ZOQAT_OK;
+}
+
+}  // namespace
+
+int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
+    if (a.M <= 0 || a.N <= 0 || a.K <= 0 || a.Z <= 0) return ZOQAT_ERR_INVALID_ARG;
+    if (a.K % 8 != 0 || a.err_flag == nullptr || (a.Z > 1 && (a.b_stride % 8 != 0 || a.b_stride < (size_t)a.N * a.K))) return ZOQAT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.out) |
+         reinterpret_cast<uintptr_t>(a.bias)) & 15)
+        return ZOQAT_ERR_INVALID_ARG;
+    // the cross-entropy epilogue always uses 256-column tiles (gemm_ce_tiles)
+    if (a.mode == 1 || a.N > 128) return launch_tc<256>(a, s);
+    return launch_tc<128>(a, s);
+}
+
+}  // namespace zq

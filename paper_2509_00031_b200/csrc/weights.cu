@@ -1,0 +1,298 @@
+// Weight side of the step: the perturbation W +/- eps*u (Eq. (1)), the per-group
+// asymmetric quantiser of Section 2, the packed representation of Section 4.3
+// and the update of Eq. (2).  All kernels stream the fp32 masters once with
+// 16-byte accesses; the direction is regenerated in registers (rng.cuh).
+//
+// Thread mapping: a thread owns 4 consecutive elements (one Philox block), a
+// warp owns 128 consecutive elements = 128/group whole groups, so the group
+// min/max is a shuffle reduction over group/4 adjacent lanes.
+#include "common.cuh"
+#include "rng.cuh"
+
+namespace zq {
+
+long long g_launch_count = 0;
+
+namespace {
+
+constexpr int kThreads = 256;
+
+inline int stream_grid(int64_t work_items, int per_block) {
+    int64_t blocks = (work_items + per_block - 1) / per_block;
+    const int64_t cap = 148 * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+__global__ void philox_words_kernel(uint32_t k0, uint32_t k1, uint32_t tid, uint64_t blk0, uint64_t nblk, uint4* out) {
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < nblk; i += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t blk = blk0 + i;
+        out[i] = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), tid, 0u, k0, k1);
+    }
+}
+
+__global__ void normal_kernel(uint32_t k0, uint32_t k1, uint32_t tid, uint64_t n, float* out) {
+    const uint64_t nblk = (n + 3) / 4;
+    for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b < nblk; b += (uint64_t)gridDim.x * blockDim.x) {
+        const float4 z = direction4(k0, k1, tid, b);
+        const float v[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (4 * b + j < n) out[4 * b + j] = v[j];
+    }
+}
+
+// min / max over the LANES adjacent lanes that share a group.
+template <int LANES>
+__device__ __forceinline__ void group_minmax(float& mn, float& mx) {
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+}
+
+struct GroupQ { float step, inv, zp; };
+
+// Section 2, asymmetric: step = (max-min)/Q_P, zero point = -round(min/step); x/step is
+// evaluated as x * (1/step) with the reciprocal rounded once (round = nearest even).
+__device__ __forceinline__ GroupQ group_params(float mn, float mx, float qp) {
+    GroupQ g;
+    g.step = fmaxf(__fdiv_rn(__fadd_rn(mx, -mn), qp), 1e-8f);
+    g.inv = __fdiv_rn(1.0f, g.step);
+    g.zp = -rintf(__fmul_rn(mn, g.inv));
+    return g;
+}
+
+__device__ __forceinline__ float quant_code(float x, const GroupQ& g, float qp) {
+    const float q = __fadd_rn(rintf(__fmul_rn(x, g.inv)), g.zp);
+    return fminf(fmaxf(q, 0.0f), qp);
+}
+
+__device__ __forceinline__ float dequant(float code, const GroupQ& g) {
+    return __fmul_rn(__fadd_rn(code, -g.zp), g.step);
+}
+
+__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b);
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(c, d);
+    uint2 r;
+    r.x = *reinterpret_cast<const uint32_t*>(&lo);
+    r.y = *reinterpret_cast<const uint32_t*>(&hi);
+    return r;
+}
+
+// One pass over a tensor: perturb, quantise per group, write the bf16 operand(s).
+// GROUP in {32, 64, 128}; bits in {0 (no quantiser), 2, 3, 4}; DUAL writes the -eps operand too.
+template <int GROUP, bool DUAL, bool DEBUG>
+__global__ void __launch_bounds__(kThreads)
+weight_operand_kernel(const float4* __restrict__ w, int64_t n4, int bits, int perturb,
+                      uint32_t k0, uint32_t k1, uint32_t tid, float eps,
+                      uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
+                      uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp) {
+    constexpr int LANES = GROUP / 4;
+    const float qp = (float)((1 << bits) - 1);
+    // whole warps iterate together so that the shuffles always see 32 lanes
+    const int64_t n4_ceil = (n4 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n4;
+        float4 x = live ? __ldg(w + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 xm = x;
+        if (perturb) {
+            const float4 z = direction4(k0, k1, tid, (uint64_t)i);
+            if (DUAL) {
+                xm.x = __fmaf_rn(-eps, z.x, x.x); xm.y = __fmaf_rn(-eps, z.y, x.y);
+                xm.z = __fmaf_rn(-eps, z.z, x.z); xm.w = __fmaf_rn(-eps, z.w, x.w);
+            }
+            x.x = __fmaf_rn(eps, z.x, x.x); x.y = __fmaf_rn(eps, z.y, x.y);
+            x.z = __fmaf_rn(eps, z.z, x.z); x.w = __fmaf_rn(eps, z.w, x.w);
+        }
+        if (bits == 0) {
+            if (live) {
+                op_plus[i] = pack_bf16x4(x.x, x.y, x.z, x.w);
+                if (DUAL) op_minus[i] = pack_bf16x4(xm.x, xm.y, xm.z, xm.w);
+            }
+            continue;
+        }
+        {
+            float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
+            float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+            group_minmax<LANES>(mn, mx);
+            const GroupQ g = group_params(mn, mx, qp);
+            const float c0 = quant_code(x.x, g, qp), c1 = quant_code(x.y, g, qp);
+            const float c2 = quant_code(x.z, g, qp), c3 = quant_code(x.w, g, qp);
+            if (live) {
+                op_plus[i] = pack_bf16x4(dequant(c0, g), dequant(c1, g), dequant(c2, g), dequant(c3, g));
+                if (DEBUG) {
+                    if (codes) codes[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
+                    if ((i % LANES) == 0) {
+                        if (step) step[i / LANES] = g.step;
+                        if (zp) zp[i / LANES] = (int32_t)g.zp;
+                    }
+                }
+            }
+        }
+        if (DUAL) {
+            float mn = fminf(fminf(xm.x, xm.y), fminf(xm.z, xm.w));
+            float mx = fmaxf(fmaxf(xm.x, xm.y), fmaxf(xm.z, xm.w));
+            group_minmax<LANES>(mn, mx);
+            const GroupQ g = group_params(mn, mx, qp);
+            const float c0 = quant_code(xm.x, g, qp), c1 = quant_code(xm.y, g, qp);
+            const float c2 = quant_code(xm.z, g, qp), c3 = quant_code(xm.w, g, qp);
+            if (live) op_minus[i] = pack_bf16x4(dequant(c0, g), dequant(c1, g), dequant(c2, g), dequant(c3, g));
+        }
+    }
+}
+
+// Packed layout of Section 4.3 (any bit width with one code path): for every run of
+// 128 consecutive elements, 4*bits 32-bit words; word (j*bits + b) holds bit b of the
+// code of element 4*lane + j in bit `lane` (a warp ballot).  qparams: (step, zero point).
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads)
+pack_frozen_kernel(const float4* __restrict__ w, int64_t n4, int bits, uint32_t* __restrict__ packed,
+                   float2* __restrict__ qparams) {
+    constexpr int LANES = GROUP / 4;
+    const float qp = (float)((1 << bits) - 1);
+    const int lane = threadIdx.x & 31;
+    const int64_t n4_ceil = (n4 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n4;
+        const float4 x = live ? __ldg(w + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
+        float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+        group_minmax<LANES>(mn, mx);
+        const GroupQ g = group_params(mn, mx, qp);
+        const uint32_t c[4] = {(uint32_t)quant_code(x.x, g, qp), (uint32_t)quant_code(x.y, g, qp),
+                               (uint32_t)quant_code(x.z, g, qp), (uint32_t)quant_code(x.w, g, qp)};
+        if (live && (i % LANES) == 0) qparams[i / LANES] = make_float2(g.step, g.zp);
+        const int64_t chunk = i >> 5;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            for (int b = 0; b < bits; ++b) {
+                const uint32_t word = __ballot_sync(0xffffffffu, (c[j] >> b) & 1u);
+                if (lane == j * bits + b) packed[chunk * (4 * bits) + lane] = word;
+            }
+    }
+}
+
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads)
+unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restrict__ qparams, int64_t n4, int bits,
+                      uint2* __restrict__ op) {
+    constexpr int LANES = GROUP / 4;
+    const int lane = threadIdx.x & 31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t* words = packed + (i >> 5) * (4 * bits);
+        const float2 qpv = __ldg(qparams + i / LANES);
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t c = 0;
+            for (int b = 0; b < bits; ++b) c |= ((__ldg(words + j * bits + b) >> lane) & 1u) << b;
+            v[j] = __fmul_rn(__fadd_rn((float)c, -qpv.y), qpv.x);
+        }
+        op[i] = pack_bf16x4(v[0], v[1], v[2], v[3]);
+    }
+}
+
+// Eq. (2): w <- w - scale*u, one fused multiply-add per element.
+__global__ void __launch_bounds__(kThreads)
+update_kernel(float* __restrict__ w, uint64_t n, uint32_t k0, uint32_t k1, uint32_t tid,
+              const float* __restrict__ scale_ptr, float scale_val) {
+    const float c = -(scale_ptr ? *scale_ptr : scale_val);
+    const uint64_t nblk = (n + 3) / 4;
+    float4* w4 = reinterpret_cast<float4*>(w);
+    for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b < nblk; b += (uint64_t)gridDim.x * blockDim.x) {
+        const float4 z = direction4(k0, k1, tid, b);
+        if (4 * b + 4 <= n) {
+            float4 x = w4[b];
+            x.x = __fmaf_rn(c, z.x, x.x); x.y = __fmaf_rn(c, z.y, x.y);
+            x.z = __fmaf_rn(c, z.z, x.z); x.w = __fmaf_rn(c, z.w, x.w);
+            w4[b] = x;
+        } else {
+            const float zz[4] = {z.x, z.y, z.z, z.w};
+            for (int j = 0; j < 4; ++j)
+                if (4 * b + j < n) w[4 * b + j] = __fmaf_rn(c, zz[j], w[4 * b + j]);
+        }
+    }
+}
+
+}  // namespace
+
+void launch_philox_words(uint64_t seed, uint32_t tid, uint64_t blk0, uint64_t nblk, uint32_t* out, cudaStream_t s) {
+    if (nblk == 0) return;
+    philox_words_kernel<<<stream_grid((int64_t)nblk, kThreads), kThreads, 0, s>>>(
+        (uint32_t)seed, (uint32_t)(seed >> 32), tid, blk0, nblk, reinterpret_cast<uint4*>(out));
+    count_launch();
+}
+
+void launch_normal(uint64_t seed, uint32_t tid, uint64_t n, float* out, cudaStream_t s) {
+    if (n == 0) return;
+    normal_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(
+        (uint32_t)seed, (uint32_t)(seed >> 32), tid, n, out);
+    count_launch();
+}
+
+template <int GROUP>
+static void weight_operand_dispatch(const float* w, int64_t n, int bits, int perturb, uint64_t seed, uint32_t tid,
+                                    float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes,
+                                    float* step, int32_t* zp, cudaStream_t s) {
+    const int64_t n4 = n / 4;
+    const int grid = stream_grid(n4, kThreads * 2);
+    const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    const float4* w4 = reinterpret_cast<const float4*>(w);
+    uint2* p = reinterpret_cast<uint2*>(op_plus);
+    uint2* m = reinterpret_cast<uint2*>(op_minus);
+    uchar4* c4 = reinterpret_cast<uchar4*>(codes);
+    const bool debug = codes || step || zp;
+    if (op_minus) {
+        weight_operand_kernel<GROUP, true, false><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr);
+    } else if (debug) {
+        weight_operand_kernel<GROUP, false, true><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp);
+    } else {
+        weight_operand_kernel<GROUP, false, false><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr);
+    }
+    count_launch();
+}
+
+void launch_weight_operand(const float* w, int64_t n, int group, int bits, int perturb, uint64_t seed, uint32_t tid,
+                           float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes, float* step,
+                           int32_t* zp, cudaStream_t s) {
+    if (n == 0) return;
+    if (group == 32) weight_operand_dispatch<32>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
+    else if (group == 64) weight_operand_dispatch<64>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
+    else weight_operand_dispatch<128>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
+}
+
+void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s) {
+    if (n == 0) return;
+    const int64_t n4 = n / 4;
+    const int grid = stream_grid(n4, kThreads);
+    const float4* w4 = reinterpret_cast<const float4*>(w);
+    if (group == 32) pack_frozen_kernel<32><<<grid, kThreads, 0, s>>>(w4, n4, bits, packed, qparams);
+    else if (group == 64) pack_frozen_kernel<64><<<grid, kThreads, 0, s>>>(w4, n4, bits, packed, qparams);
+    else pack_frozen_kernel<128><<<grid, kThreads, 0, s>>>(w4, n4, bits, packed, qparams);
+    count_launch();
+}
+
+void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,
+                           __nv_bfloat16* op, cudaStream_t s) {
+    if (n == 0) return;
+    const int64_t n4 = n / 4;
+    const int grid = stream_grid(n4, kThreads);
+    uint2* o = reinterpret_cast<uint2*>(op);
+    if (group == 32) unpack_operand_kernel<32><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
+    else if (group == 64) unpack_operand_kernel<64><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
+    else unpack_operand_kernel<128><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
+    count_launch();
+}
+
+void launch_update(float* w, uint64_t n, uint64_t seed, uint32_t tid, const float* scale_ptr, float scale_val, cudaStream_t s) {
+    if (n == 0) return;
+    update_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(
+        w, n, (uint32_t)seed, (uint32_t)(seed >> 32), tid, scale_ptr, scale_val);
+    count_launch();
+}
+
+}  // namespace zq

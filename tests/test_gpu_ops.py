@@ -1,0 +1,271 @@
+"""GPU parity, kernel by kernel: every operation of the path, called through the
+C ABI on seeded inputs, against the CPU oracle.  Integer work (Philox words,
+weight codes, zero points, activation codes) and everything the binary32
+contract fixes (the direction, steps, operands, updated weights) is compared
+bit for bit; float results against the float64 oracle within stated bounds.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import core
+from oracle.model import act_quant, causal_attention, rope_tables
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zq():
+    from paper_2509_00031_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def bf16_to_f32(t):
+    return t.float().cpu().numpy()
+
+
+# ---- direction generator ----------------------------------------------------------------
+@pytest.mark.parametrize("seed,tid,blk0,nblk", [(0, 0, 0, 1000), (0x0123456789ABCDEF, 37, 5, 4099),
+                                                (2**64 - 1, 2**32 - 1, 2**32 - 3, 777), (1000, 16, 2**40, 513)])
+def test_philox_words_bit_exact(zq, seed, tid, blk0, nblk):
+    got = zq.zoqat_op_philox_words(seed, tid, blk0, nblk).cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, core.philox_words(seed, tid, blk0, nblk))
+
+
+@pytest.mark.parametrize("seed,tid,n", [(1, 0, 4096), (1000, 33, 1_000_003), (2**63 + 5, 500, 7)])
+def test_direction_bit_exact(zq, seed, tid, n):
+    got = zq.zoqat_op_normal(seed, tid, n).cpu().numpy()
+    want = core.normal(seed, tid, n)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+# ---- weight path ---------------------------------------------------------------------------
+@pytest.mark.parametrize("bits,group", [(4, 64), (4, 128), (3, 64), (2, 64), (2, 32), (4, 32)])
+@pytest.mark.parametrize("signed_eps", [0.0, 1e-3, -1e-3])
+def test_weight_quant_bit_exact(zq, bits, group, signed_eps):
+    rng = np.random.default_rng(bits * 100 + group)
+    rows, cols = 203, 3 * 128 + group          # several warps' worth plus a ragged tail
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    seed, tid = 4242, 48
+    codes, step, zp, operand = zq.zoqat_op_weight_quant(dev(w), group, bits, seed, tid, signed_eps)
+    wp = core.perturb(w, seed, tid, signed_eps)
+    o_codes, o_step, o_zp, o_deq = core.weight_quant(wp, group, bits)
+    assert np.array_equal(codes.cpu().numpy(), o_codes)            # zero codes excused
+    assert np.array_equal(step.cpu().numpy().view(np.uint32), o_step.view(np.uint32))
+    assert np.array_equal(zp.cpu().numpy(), o_zp)
+    assert np.array_equal(bf16_to_f32(operand), core.round_bf16(o_deq))
+
+
+def test_weight_operand_unquantised_and_pair(zq):
+    rng = np.random.default_rng(9)
+    w = (rng.standard_normal((130, 256)) * 0.02).astype(np.float32)
+    seed, tid, eps = 77, 0, np.float32(1e-3)
+    _, _, _, op = zq.zoqat_op_weight_quant(dev(w), 64, 0, seed, tid, float(eps))
+    assert np.array_equal(bf16_to_f32(op), core.round_bf16(core.perturb(w, seed, tid, eps)))
+    for bits in (0, 4):
+        plus, minus = zq.zoqat_op_weight_operand_pair(dev(w), 64, bits, seed, tid, float(eps))
+        _, _, _, sp = zq.zoqat_op_weight_quant(dev(w), 64, bits, seed, tid, float(eps), want_codes=False)
+        _, _, _, sm = zq.zoqat_op_weight_quant(dev(w), 64, bits, seed, tid, -float(eps), want_codes=False)
+        assert torch.equal(plus, sp) and torch.equal(minus, sm)
+        assert not torch.equal(plus, minus)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64), (2, 32)])
+def test_pack_unpack_frozen(zq, bits, group):
+    rng = np.random.default_rng(bits)
+    w = (rng.standard_normal((96, 512)) * 0.02).astype(np.float32)
+    packed, qparams = zq.zoqat_op_pack_frozen(dev(w), group, bits)
+    assert packed.numel() == 96 * 512 * bits // 8
+    op = zq.zoqat_op_unpack_operand(packed, qparams, 96, 512, group, bits)
+    o_codes, o_step, o_zp, o_deq = core.weight_quant(w, group, bits)
+    assert np.array_equal(bf16_to_f32(op), core.round_bf16(o_deq))
+    qp = qparams.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(qp[:, 0], o_step.ravel()) and np.array_equal(qp[:, 1], o_zp.ravel().astype(np.float32))
+    # the stored bit planes decode to the oracle's codes
+    words = packed.cpu().numpy().view(np.uint32).reshape(-1, 4, bits)
+    lanes = np.arange(32, dtype=np.uint32)
+    dec = np.zeros((words.shape[0], 32, 4), np.uint8)
+    for j in range(4):
+        for b in range(bits):
+            dec[:, :, j] |= (((words[:, j, b][:, None] >> lanes[None, :]) & 1) << b).astype(np.uint8)
+    assert np.array_equal(dec.reshape(96, 512), o_codes)
+
+
+@pytest.mark.parametrize("n", [4096, 1_000_003])
+def test_update_bit_exact(zq, n):
+    rng = np.random.default_rng(n)
+    w = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    wd = dev(w)
+    zq.zoqat_op_update(wd, 99, 21, 3.5e-6)
+    want = core.update_(w.copy(), 99, 21, np.float32(3.5e-6))
+    assert np.array_equal(wd.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+# ---- activation operands ---------------------------------------------------------------------
+def _oracle_norm(x, kind, g, b, eps):
+    x = x.astype(np.float64)
+    if kind == 0:
+        return x
+    if kind == 1:
+        return x / np.sqrt(np.mean(x * x, -1, keepdims=True) + np.float64(np.float32(eps))) * g.astype(np.float64)
+    mu = x.mean(-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + np.float64(np.float32(eps))) * g.astype(np.float64) + b.astype(np.float64)
+
+
+def _check_codes(codes_gpu, step_gpu, x_gpu_f32, x_oracle_f64):
+    """Codes of the GPU's own fp32 input reproduce the oracle quantiser exactly; against the
+    oracle's float64 input they may differ only where the pre-rounding value is within 1e-6
+    (relative) of a rounding boundary."""
+    q_self, s_self = act_quant(x_gpu_f32.astype(np.float64))
+    assert np.array_equal(codes_gpu, q_self)
+    assert np.array_equal(step_gpu, s_self)
+    q_or, s_or = act_quant(x_oracle_f64)
+    diff = codes_gpu != q_or
+    if diff.any():
+        inv = (np.float32(1.0) / s_or)[:, None]
+        v = x_oracle_f64.astype(np.float32) * inv
+        dist = np.abs(np.abs(v - np.floor(v)) - 0.5)
+        assert np.all(dist[diff] <= 1e-6 * np.maximum(1.0, np.abs(v[diff])) + 2e-5), "code differs away from a rounding boundary"
+    return int(diff.sum())
+
+
+@pytest.mark.parametrize("kind,cols", [(1, 256), (2, 2048), (0, 320), (1, 11008)])
+def test_norm_act_operand(zq, kind, cols):
+    rng = np.random.default_rng(cols + kind)
+    rows = 37
+    x = (rng.standard_normal((rows, cols)) * rng.uniform(0.2, 4.0, (rows, 1))).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(cols)).astype(np.float32)
+    b = (0.05 * rng.standard_normal(cols)).astype(np.float32)
+    op, step, normed = zq.zoqat_op_norm_act_operand(dev(x), kind, dev(g), dev(b), 1e-5, 8, want_normed=True)
+    want = _oracle_norm(x, kind, g, b, 1e-5)
+    normed = normed.cpu().numpy()
+    assert np.allclose(normed, want, rtol=2e-6, atol=2e-6)
+    excused = _check_codes(bf16_to_f32(op).astype(np.float64), step.cpu().numpy(), normed, want)
+    assert excused <= 3
+    # unquantised activations: operand = bf16(x), row step 1
+    op16, step16, _ = zq.zoqat_op_norm_act_operand(dev(x), kind, dev(g), dev(b), 1e-5, 0, want_normed=False)
+    assert np.array_equal(bf16_to_f32(op16), core.round_bf16(normed)) and np.all(step16.cpu().numpy() == 1.0)
+
+
+@pytest.mark.parametrize("gated,cols", [(1, 1024), (0, 8192), (1, 11008)])
+def test_ffn_act_operand(zq, gated, cols):
+    rng = np.random.default_rng(cols)
+    rows = 19
+    x = rng.standard_normal((rows, 2 * cols if gated else cols)).astype(np.float32) * 2
+    op, step = zq.zoqat_op_ffn_act_operand(dev(x), gated, 8)
+    x64 = x.astype(np.float64)
+    want = x64[:, :cols] / (1 + np.exp(-x64[:, :cols])) * x64[:, cols:] if gated else np.maximum(x64, 0)
+    codes = bf16_to_f32(op).astype(np.float64)
+    assert np.allclose(step.cpu().numpy(), np.abs(want).max(1) / 127, rtol=1e-6)
+    q_or, s_or = act_quant(want)
+    diff = codes != q_or
+    assert diff.mean() < 2e-4                      # only values that sit on a rounding boundary move
+    assert np.all(np.abs(codes - q_or) <= 1)
+    deq = codes * step.cpu().numpy()[:, None]
+    assert np.all(np.abs(deq - want) <= 0.5001 * s_or[:, None] + 1e-6)
+    op16, _ = zq.zoqat_op_ffn_act_operand(dev(x), gated, 0)
+    assert np.allclose(bf16_to_f32(op16), want, rtol=2 ** -8, atol=1e-30)
+
+
+# ---- matrix multiply --------------------------------------------------------------------------
+IMPLS = [pytest.param(1, id="simt"), pytest.param(0, id="tcgen05")]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 520, 192), (512, 768, 256), (1000, 136, 1024), (64, 64, 8)])
+def test_gemm_integer_operands_exact(zq, impl, M, N, K):
+    """int8 activation codes times small-integer weights: every product and partial sum is an
+    integer below 2^24, so fp32 accumulation is exact and the result must match bit for bit."""
+    rng = np.random.default_rng(M + N + K)
+    a = rng.integers(-127, 128, (M, K)).astype(np.float32)
+    b = rng.integers(-15, 16, (N, K)).astype(np.float32)
+    out, err = zq.zoqat_op_gemm(dev(a).bfloat16(), dev(b).bfloat16(), impl=impl)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    want = a.astype(np.float64) @ b.astype(np.float64).T
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_gemm_epilogues(zq, impl):
+    rng = np.random.default_rng(3)
+    M, N, K = 260, 392, 320
+    a = core.round_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    b = core.round_bf16((rng.standard_normal((N, K)) * 0.02).astype(np.float32))
+    rs = rng.uniform(0.01, 0.1, M).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    resid = rng.standard_normal((M, N)).astype(np.float32)
+    base = a.astype(np.float64) @ b.astype(np.float64).T
+    scale = np.abs(a).astype(np.float64) @ np.abs(b).astype(np.float64).T     # bound on the accumulation error
+    ad, bd = dev(a).bfloat16(), dev(b).bfloat16()
+    out, err = zq.zoqat_op_gemm(ad, bd, impl=impl)
+    assert np.all(np.abs(out.cpu().numpy() - base) <= 2e-6 * scale + 1e-7)
+    out, err = zq.zoqat_op_gemm(ad, bd, row_step=dev(rs), bias=dev(bias), impl=impl)
+    want = base * rs[:, None] + bias[None, :]
+    assert np.all(np.abs(out.cpu().numpy() - want) <= 2e-6 * (scale * rs[:, None] + np.abs(bias)[None, :]) + 1e-7)
+    out, err = zq.zoqat_op_gemm(ad, bd, row_step=dev(rs), bias=dev(bias), relu=True, impl=impl)
+    assert np.all(np.abs(out.cpu().numpy() - np.maximum(want, 0)) <= 2e-6 * (scale * rs[:, None] + np.abs(bias)[None, :]) + 1e-7)
+    acc = dev(resid.copy())
+    zq.zoqat_op_gemm(ad, bd, row_step=dev(rs), bias=dev(bias), out=acc, accumulate=True, impl=impl)
+    assert np.all(np.abs(acc.cpu().numpy() - (want + resid)) <= 2e-6 * (scale * rs[:, None] + np.abs(bias)[None, :] + np.abs(resid)) + 1e-7)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+
+
+def test_gemm_rejects_bad_arguments(zq):
+    a = torch.zeros((8, 12), dtype=torch.bfloat16, device="cuda")     # K not a multiple of 8
+    b = torch.zeros((8, 12), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(zq.ZoqatError) as e:
+        zq.zoqat_op_gemm(a, b)
+    assert e.value.status == zq.ERR_INVALID_ARG
+
+
+# ---- attention ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("B,S,H,dh,rope", [(2, 128, 4, 64, True), (1, 200, 2, 128, True), (3, 77, 2, 64, False),
+                                           (1, 512, 1, 128, False)])
+def test_attention(zq, B, S, H, dh, rope):
+    rng = np.random.default_rng(S + dh)
+    d = H * dh
+    qkv = rng.standard_normal((B * S, 3 * d)).astype(np.float32)
+    cos = sin = None
+    if rope:
+        cos, sin = rope_tables(S, dh, 10000.0)
+    out = zq.zoqat_op_attention(dev(qkv), B, S, H, dh,
+                                None if cos is None else dev(cos.astype(np.float32)),
+                                None if sin is None else dev(sin.astype(np.float32)))
+    x = qkv.astype(np.float64).reshape(B, S, 3 * d)
+    want = causal_attention(x[..., :d], x[..., d:2 * d], x[..., 2 * d:], H, cos, sin).reshape(B * S, d)
+    got = out.cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 5e-6 * max(1.0, np.abs(want).max())
+    # first position attends to itself only
+    assert np.allclose(got.reshape(B, S, d)[:, 0], x[:, 0, 2 * d:], atol=1e-6)
+
+
+# ---- vocabulary projection + cross-entropy ---------------------------------------------------------
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("T,V,d", [(130, 1024, 256), (257, 5000, 128), (64, 50272, 64)])
+def test_head_loss(zq, impl, T, V, d):
+    rng = np.random.default_rng(V)
+    a = core.round_bf16(rng.standard_normal((T, d)).astype(np.float32))
+    b = core.round_bf16((rng.standard_normal((V, d)) * 0.05).astype(np.float32))
+    labels = rng.integers(0, V, T).astype(np.int32)
+    labels[::7] = -1
+    labels[1] = V - 1
+    labels[2] = 0
+    tl, ls, cnt, err = zq.zoqat_op_head_loss(dev(a).bfloat16(), dev(b).bfloat16(), dev(labels), impl=impl)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    logits = a.astype(np.float64) @ b.astype(np.float64).T
+    mx = logits.max(-1)
+    lse = mx + np.log(np.exp(logits - mx[:, None]).sum(-1))
+    valid = labels >= 0
+    want = np.where(valid, lse - logits[np.arange(T), np.where(valid, labels, 0)], 0.0)
+    assert np.allclose(tl.cpu().numpy(), want, rtol=0, atol=3e-6 * np.abs(lse).max())
+    assert int(cnt.item()) == int(valid.sum())
+    assert abs(float(ls.item()) - want.sum()) <= 1e-6 * abs(want.sum())
