@@ -106,8 +106,8 @@ class ClockSampler:
 def oracle_sample(w, budget_note=True):
     """Times the oracle (as it stands) on a bounded sample of workload `w` and extrapolates one step.
 
-    Sample: ONE decoder layer of the workload's shape plus the vocabulary projection, at T1 and T2 = 2*T1
-    tokens (T1 = 32 for 7B-class shapes).  Step time is fitted as a + b*T per layer (a: weight-side work
+    Sample: ONE decoder layer of the workload's shape plus the vocabulary projection, at T1 and T2 tokens
+    (64 and 512 for 7B-class shapes).  Step time is fitted as a + b*T per layer (a: weight-side work
     - direction, perturbation, quantiser - independent of tokens; b: matmul/attention work per token) and
     extrapolated to n_layers layers and the workload's tokens.
     """
@@ -116,26 +116,27 @@ def oracle_sample(w, budget_note=True):
     from paper_2509_00031_b200 import synth
     one = dict(w, n_layers=1)
     small = w["d_model"] <= 512
-    seq1 = 32 if not small else w["seq"]
+    seq1 = 64 if not small else w["seq"] // 2
+    seq2 = 512 if not small else w["seq"]
     times = {}
     cores = os.cpu_count() or 1
     cfg = OracleConfig(arch=w["arch"], n_layers=1, d_model=w["d_model"], n_heads=w["n_heads"], d_ffn=w["d_ffn"],
                        vocab=w["vocab"], w_bits=w["w_bits"], w_group=w["w_group"], a_bits=w["a_bits"])
-    params = synth.make_params(one, seed=0, max_seq=2 * seq1)
+    params = synth.make_params(one, seed=0, max_seq=seq2)
     model = OracleModel(cfg, params)
-    for seq in (seq1, 2 * seq1):
+    for seq in (seq1, seq2):
         tokens, labels = synth.make_batch(1, seq, w["vocab"], seed=1234)
         t0 = time.perf_counter()
         model.step(tokens, labels, 1000, EPS, LR)
         times[seq] = time.perf_counter() - t0
-    b = (times[2 * seq1] - times[seq1]) / seq1
+    b = (times[seq2] - times[seq1]) / (seq2 - seq1)
     a = times[seq1] - b * seq1
     nums = workload_numbers(w)
     L = w["n_layers"]
     # the single layer + head were timed together; scale the whole by layers (head counted L times: a small overestimate)
     step_s = L * (max(a, 0.0) + max(b, 0.0) * nums["T"])
-    return dict(step_s=step_s, cores=cores, cpu_s=times[seq1] + times[2 * seq1],
-                sample=f"1 of {L} layers + vocabulary projection, full ZO step at {seq1} and {2 * seq1} tokens of {nums['T']}; "
+    return dict(step_s=step_s, cores=cores, cpu_s=times[seq1] + times[seq2],
+                sample=f"1 of {L} layers + vocabulary projection, full ZO step at {seq1} and {seq2} tokens of {nums['T']}; "
                        f"step time fitted as layers*(a + b*tokens), a={a:.3f}s b={b * 1e3:.3f}ms/token")
 
 

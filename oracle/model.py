@@ -54,6 +54,9 @@ class OracleConfig:
     rope_base: float = 10000.0
     first_trainable_layer: int = 0   # layers below are frozen (quantised from the unperturbed masters)
     head_trainable: bool = True
+    store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
+                                     # residual stream) to binary32, as an implementation that keeps activations in
+                                     # fp32 does; used only to measure how far two correct implementations can differ
     operand_bf16: bool = True        # False (with w_bits = 0, a_bits = 0) gives the unquantised float64 model, used only to pin the forward
 
 
@@ -169,7 +172,10 @@ class OracleModel:
             y = a @ self.block_operand(l, name, seed, signed_eps).T
         if bias is not None:
             y = y + bias.astype(np.float64)[None, :]
-        return y
+        return self._store(y)
+
+    def _store(self, x):
+        return x.astype(F32).astype(np.float64) if self.cfg.store_f32 else x
 
     def norm(self, h, g, b=None):
         cfg = self.cfg
@@ -181,7 +187,7 @@ class OracleModel:
             var = np.mean((h - mu) ** 2, axis=-1, keepdims=True)
             y = (h - mu) / np.sqrt(var + np.float64(F32(cfg.norm_eps))) * g.astype(np.float64)
             y = y + b.astype(np.float64)
-        return y
+        return self._store(y)
 
     def _tap(self, name, arr):
         if self.tap is not None:
@@ -213,20 +219,21 @@ class OracleModel:
             att = causal_attention(q.reshape(B, S, d), k.reshape(B, S, d), v.reshape(B, S, d), H,
                                    cos if cfg.arch == "llama" else None,
                                    sin if cfg.arch == "llama" else None).reshape(T, d)
+            att = self._store(att)
             self._tap(f"l{l}.attn", att)
-            h = h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo"))
+            h = self._store(h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo")))
             self._tap(f"l{l}.h_mid", h)
             x = self.norm(h, P["ffn_norm_g"], P.get("ffn_norm_b"))
             if cfg.arch == "llama":
                 gate = self.lin(x, l, "w_gate", seed, signed_eps)
                 up = self.lin(x, l, "w_up", seed, signed_eps)
-                act = gate / (1.0 + np.exp(-gate)) * up
+                act = self._store(gate / (1.0 + np.exp(-gate)) * up)
                 self._tap(f"l{l}.ffn_act", act)
-                h = h + self.lin(act, l, "w_down", seed, signed_eps)
+                h = self._store(h + self.lin(act, l, "w_down", seed, signed_eps))
             else:
                 a1 = np.maximum(self.lin(x, l, "fc1", seed, signed_eps, P["b_fc1"]), 0.0)
                 self._tap(f"l{l}.ffn_act", a1)
-                h = h + self.lin(a1, l, "fc2", seed, signed_eps, P["b_fc2"])
+                h = self._store(h + self.lin(a1, l, "fc2", seed, signed_eps, P["b_fc2"]))
             self._tap(f"l{l}.h_out", h)
         x = self.norm(h, self.p["final_norm_g"], self.p.get("final_norm_b"))
         self._tap("final_norm", x)
