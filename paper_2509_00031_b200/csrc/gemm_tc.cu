@@ -7,9 +7,11 @@
 //   warp 1     MMA issuer: one lane issues tcgen05.mma (M=128, N=BN, K=16) over
 //              each stage and commits to the stage's "empty" barrier; owns TMEM.
 //   warps 2-5  epilogue: tcgen05.ld the 128xBN fp32 accumulator (each warp its
-//              32-lane quarter), apply the per-row step / bias / ReLU / residual
-//              add, or reduce the tile to cross-entropy partials (max, sum exp)
-//              so that logits never reach memory.
+//              32-lane quarter), apply the per-row step / bias / ReLU, stage 32x32
+//              boxes in shared memory and let TMA store them (or add them into the
+//              residual stream with a TMA fp32 reduction, one add per element, so
+//              the result does not depend on timing); or reduce the tile to
+//              cross-entropy partials (max, sum exp) so that logits never reach memory.
 // Two accumulators (2*BN of the 512 TMEM columns) let the epilogue of tile i
 // overlap the MMAs of tile i+1.
 //
@@ -33,7 +35,10 @@ template <int BN> struct TileCfg {
     static constexpr int kABytes = BM * BK * 2;
     static constexpr int kBBytes = BN * BK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
+    // output staging for the TMA stores of the epilogue: two 32x32 fp32 boxes per epilogue warp
+    static constexpr int kOutBoxBytes = 32 * 32 * 4;
+    static constexpr int kOutStageBytes = 4 * 2 * kOutBoxBytes;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------
@@ -72,6 +77,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// shared -> global tile store (or fp32 add into global) of one box, tracked by the thread's bulk async-group
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// at most one group of this thread may still be reading its shared-memory source
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -155,17 +174,20 @@ struct TcParams {
     float* label_logit;
     int32_t* err_flag;
     int tiles_m, tiles_n;
+    int tma_out;              // 1: mode-0 results leave through map_out (needs N % 4 == 0)
 };
 
 template <int BN>
 __global__ void __launch_bounds__(kThreadsTC, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams p) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_out, TcParams p) {
     using Cfg = TileCfg<BN>;
     constexpr int S = Cfg::kStages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;              // 1024-byte aligned stage ring
-    const uint32_t bars = tiles + S * Cfg::kStageBytes;         // barriers follow the ring
+    const uint32_t out_stage = tiles + S * Cfg::kStageBytes;    // 1024-byte aligned: epilogue store staging
+    const uint32_t bars = out_stage + Cfg::kOutStageBytes;      // barriers follow
     // barrier layout (8 bytes each): full[S], empty[S], acc_full[2], acc_empty[2], then the TMEM base word
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (S + s); };
@@ -185,6 +207,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
+        if (p.tma_out) prefetch_tmap(&map_out);
     }
     if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns
         tmem_alloc(tmem_slot, 2 * BN);
@@ -255,6 +278,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ---------------- epilogue (warps 2..5) ----------------
         const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter+32)
         int acc = 0; uint32_t acc_phase = 0;
+        int out_buf = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const int z = t / tiles_per_z, r = t % tiles_per_z;
             const int tm = r % p.tiles_m, tn = r / p.tiles_m;
@@ -280,7 +304,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tmem_ld_wait();
                 const int64_t n0 = n_base + c * 32;
                 if (n0 >= p.N) continue;                      // uniform: whole chunk out of range
-                if (p.mode == 0) {
+                if (p.mode == 0 && p.tma_out) {
+                    // Stage the warp's 32x32 box in shared memory (128-byte rows, 16-byte chunks XOR-swizzled by
+                    // row so that the writes spread over all banks) and hand it to the TMA unit, which writes
+                    // whole rows (or adds them into the residual stream) and clips the box at the matrix edge.
+                    const uint32_t box = out_stage + (uint32_t)((quarter * 2 + out_buf) * Cfg::kOutBoxBytes);
+                    if (lane == 0) bulk_wait_read_1();          // the box written two chunks ago has been read
+                    __syncwarp();
+                    const bool full = n0 + 32 <= p.N;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        float4 x;
+                        x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
+                        x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
+                        if (p.bias) {
+                            if (full) {
+                                const float4 b = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+                                x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
+                            } else {
+                                if (n0 + j < p.N) x.x += p.bias[n0 + j];
+                                if (n0 + j + 1 < p.N) x.y += p.bias[n0 + j + 1];
+                                if (n0 + j + 2 < p.N) x.z += p.bias[n0 + j + 2];
+                                if (n0 + j + 3 < p.N) x.w += p.bias[n0 + j + 3];
+                            }
+                        }
+                        if (p.relu) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
+                        const uint32_t dst = box + (uint32_t)(lane * 128) + (uint32_t)((((j >> 2) ^ (lane & 7)) << 4));
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w) : "memory");
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int y0 = tm * BM + quarter * 32;
+                        if (p.accumulate) tma_reduce_add_3d(&map_out, box, (int)n0, y0, z);
+                        else tma_store_3d(&map_out, box, (int)n0, y0, z);
+                        bulk_commit();
+                    }
+                    out_buf ^= 1;
+                } else if (p.mode == 0) {
                     if (!row_ok) continue;
                     float* o = p.out + row * p.N + n0;
                     if (n0 + 32 <= p.N && (p.N & 3) == 0) {
@@ -328,6 +389,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (lane == 0) mbar_arrive(acc_empty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (lane == 0) bulk_wait_all();      // every store / add issued by this warp has completed
     }
 
     tc_fence_before();
@@ -372,6 +434,18 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int Z
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D map over the fp32 result [Z][M][N] (N innermost), box = 32 x 32 x 1 with the 128-byte swizzle.
+bool make_out_map(CUtensorMap* map, float* base, int64_t M, int64_t N, int Z) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)Z};
+    const cuuint64_t strides[2] = {(cuuint64_t)N * 4, (cuuint64_t)M * N * 4};
+    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int num_sms() {
     static int n = 0;
     if (n == 0) {
@@ -386,7 +460,7 @@ int num_sms() {
 template <int BN>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
     using Cfg = TileCfg<BN>;
-    alignas(64) CUtensorMap map_a, map_b;
+    alignas(64) CUtensorMap map_a, map_b, map_out;
     const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
     if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN))
         return ZOQAT_ERR_CUDA;
@@ -397,6 +471,12 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     p.err_flag = a.err_flag;
     p.tiles_m = (int)((a.M + BM - 1) / BM);
     p.tiles_n = (int)((a.N + BN - 1) / BN);
+    p.tma_out = (a.mode == 0 && a.N % 4 == 0) ? 1 : 0;
+    if (p.tma_out) {
+        if (!make_out_map(&map_out, a.out, a.M, a.N, a.Z)) return ZOQAT_ERR_CUDA;
+    } else {
+        map_out = map_a;      // never dereferenced
+    }
     static bool attr = false;
     if (!attr) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
@@ -405,7 +485,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
     const int grid = (int)(total < num_sms() ? total : num_sms());
-    gemm_tc_kernel<BN><<<grid, kThreadsTC, Cfg::kSmemBytes, s>>>(map_a, map_b, p);
+    gemm_tc_kernel<BN><<<grid, kThreadsTC, Cfg::kSmemBytes, s>>>(map_a, map_b, map_out, p);
     count_launch();
     return ZOQAT_OK;
 }
