@@ -307,6 +307,35 @@ int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labe
                        double* loss_sum_dev, int32_t* count_dev, void* scratch_dev,
                        int impl, int32_t* err_flag_dev, void* stream);
 
+/* The same operation as zoqat_op_head_loss for callers that must not allocate device
+ * memory and so cannot hand over a scratch buffer.  (The paper has no counterpart: this
+ * is a convenience of the library, not a step of the method.)  Typical cases: code that
+ * runs after another component has claimed the whole device for its own memory pool, a
+ * latency-critical loop in which a cudaMalloc/cudaFree would stall every stream of the
+ * device, or a plug-in whose host forbids allocation calls altogether.
+ *
+ * The scratch is a fixed array of ZOQAT_STATIC_SCRATCH_BYTES inside the library image;
+ * every device that loads the library keeps it resident until the process ends.  Inputs
+ * and outputs are still the caller's: a_dev bf16 [T, d], b_dev bf16 [V, d], labels_dev
+ * int32 [T]; token_loss_dev fp32 [T], loss_sum_dev double[1], count_dev int32[1],
+ * err_flag_dev int32[1] (required for ZOQAT_GEMM_TCGEN05) - all device memory.
+ *
+ *   - Limit: 256-byte-rounded T * ceil(V/128) * 8 plus 256-byte-rounded T * 4 bytes must
+ *     fit in the array (T = 4096 with V = 32000 does; T = 8192 with V = 50272 does not).
+ *     Larger problems return ZOQAT_ERR_WORKSPACE_SMALL and launch nothing.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called, on any call.
+ *   - All calls on a device share the one array, which still holds the previous call's
+ *     data; the part that has to start from zero is cleared on `stream` before use.  Two
+ *     calls whose kernels can overlap on the GPU (different streams without an ordering
+ *     between them, or different host threads doing so) race on it: serialise them. */
+#define ZOQAT_STATIC_SCRATCH_BYTES (16u << 20)
+int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_t* labels_dev,
+                              int64_t T, int64_t V, int64_t d, float* token_loss_dev,
+                              double* loss_sum_dev, int32_t* count_dev, int impl,
+                              int32_t* err_flag_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

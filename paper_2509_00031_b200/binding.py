@@ -30,7 +30,7 @@ EXPORTS = [
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
     "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_attention", "zoqat_op_head_loss_scratch_bytes",
-    "zoqat_op_head_loss",
+    "zoqat_op_head_loss", "zoqat_op_head_loss_static",
 ]
 
 
@@ -103,6 +103,7 @@ def lib():
             "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, vp],
             "zoqat_op_head_loss_scratch_bytes": [i64, i64, P(sz)],
             "zoqat_op_head_loss": [vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, vp, vp],
+            "zoqat_op_head_loss_static": [vp, vp, vp, i64, i64, i64, vp, vp, vp, i32, vp, vp],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -235,6 +236,19 @@ def zoqat_op_head_loss(a, b, labels, impl=GEMM_TCGEN05):
     err = torch.zeros(1, dtype=torch.int32, device=a.device)
     _check(lib().zoqat_op_head_loss(_p(a), _p(b), _p(labels), T, V, d, _p(token_loss), _p(loss_sum), _p(count),
                                     _p(scratch), impl, _p(err), _stream()))
+    return token_loss, loss_sum, count, err
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def zoqat_op_head_loss_static(a, b, labels, token_loss, loss_sum, count, err, impl=GEMM_TCGEN05):
+    """zoqat_op_head_loss for callers that cannot allocate: the library's built-in scratch array is
+    used, and every output tensor is supplied by the caller, so nothing is allocated here either."""
+    T, d = a.shape
+    V = b.shape[0]
+    _check(lib().zoqat_op_head_loss_static(_p(a), _p(b), _p(labels), T, V, d, _p(token_loss), _p(loss_sum), _p(count),
+                                           impl, _p(err), _stream()))
     return token_loss, loss_sum, count, err
 
 

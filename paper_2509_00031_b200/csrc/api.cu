@@ -9,6 +9,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -751,6 +752,68 @@ int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labe
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     float2* partials = static_cast<float2*>(scratch_dev);
     float* label_logit = reinterpret_cast<float*>(static_cast<uint8_t*>(scratch_dev) + align_up((size_t)T * ((V + 127) / 128) * 8));
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = T; g.N = V; g.K = d; g.Z = 1; g.mode = 1; g.labels = labels_dev; g.partials = partials; g.label_logit = label_logit;
+    g.err_flag = err_flag_dev; g.b_stride = (size_t)V * d;
+    const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
+    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+// ---- vocabulary projection + cross-entropy without any allocation ---------------------
+// Scratch for zoqat_op_head_loss_static lives in the library image itself, so the entry
+// point never asks the CUDA allocator (or anyone else) for memory.  Each device that loads
+// the library carries its own copy of the array until the process exits.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[ZOQAT_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxStaticDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxStaticDevices] = {nullptr};
+
+// Device address of g_static_scratch on the current device.  In host code the symbol is only a
+// handle, never an address a kernel may dereference, so the address is looked up once per device.
+int static_scratch_address(void** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxStaticDevices) return fail(ZOQAT_ERR_UNSUPPORTED, "device ordinal %d is beyond the %d this entry point tracks", dev, kMaxStaticDevices);
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return fail(ZOQAT_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return ZOQAT_OK;
+}
+
+}  // namespace
+
+int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_t* labels_dev, int64_t T, int64_t V,
+                              int64_t d, float* token_loss_dev, double* loss_sum_dev, int32_t* count_dev, int impl,
+                              int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !labels_dev || !token_loss_dev || !loss_sum_dev || !count_dev)
+        return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (T <= 0 || V <= 0 || d <= 0) return fail(ZOQAT_ERR_INVALID_ARG, "T, V and d must be positive");
+    const size_t partial_bytes = align_up((size_t)T * ((V + 127) / 128) * 8);
+    const size_t logit_bytes = align_up((size_t)T * 4);
+    if (partial_bytes + logit_bytes > (size_t)ZOQAT_STATIC_SCRATCH_BYTES)
+        return fail(ZOQAT_ERR_WORKSPACE_SMALL,
+                    "T=%lld x V=%lld needs %zu bytes of scratch; the built-in buffer holds %zu (use zoqat_op_head_loss with caller scratch)",
+                    (long long)T, (long long)V, partial_bytes + logit_bytes, (size_t)ZOQAT_STATIC_SCRATCH_BYTES);
+    void* base = nullptr;
+    if (int rc = static_scratch_address(&base)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float2* partials = static_cast<float2*>(base);
+    float* label_logit = reinterpret_cast<float*>(static_cast<uint8_t*>(base) + partial_bytes);
+    // The buffer still holds the previous call's values.  Every partial this call reads is rewritten by the
+    // projection kernel first; the label logits are only written for labels inside [0, V), so they start at zero.
+    CUDA_TRY(cudaMemsetAsync(label_logit, 0, (size_t)T * 4, s));
     GemmArgs g{};
     g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
     g.M = T; g.N = V; g.K = d; g.Z = 1; g.mode = 1; g.labels = labels_dev; g.partials = partials; g.label_logit = label_logit;
