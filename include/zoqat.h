@@ -290,11 +290,21 @@ int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, in
                   const float* row_step_dev, const float* bias_dev, int relu, int accumulate,
                   float* out_dev, int impl, int32_t* err_flag_dev, void* stream);
 
-/* Causal softmax attention of one layer.  qkv_dev fp32 [batch*seq, 3*d_model]
- * (q | k | v, heads contiguous inside each); rotary tables cos_dev/sin_dev fp32
- * [seq, d_head/2] or NULL (no rotation); out_dev fp32 [batch*seq, d_model]. */
+/* Causal softmax attention of one layer (the architecture of the workloads; the paper's
+ * forward pass of Section 4.1 runs the unmodified decoder between the quantised linears).
+ * qkv_dev fp32 [batch*seq, 3*d_model] (q | k | v, heads contiguous inside each); rotary
+ * tables cos_dev/sin_dev fp32 [seq, d_head/2] or NULL (no rotation); out_dev fp32
+ * [batch*seq, d_model].  All pointers 16-byte aligned.
+ * impl ZOQAT_GEMM_TCGEN05: tensor-core kernel; every operand is split into two binary16
+ * halves (hi + lo * 2^-11) and every product is formed from three tensor-core products, so
+ * the result is binary32-grade; |q|, |k|, |v| must stay below 65504.  Needs scratch_dev
+ * (256-byte aligned, zoqat_op_attention_scratch_bytes() bytes) and err_flag_dev (int32, set
+ * non-zero if a bounded wait ran out).  impl ZOQAT_GEMM_SIMT: fp32 CUDA-core kernel
+ * (cross-check); scratch_dev / err_flag_dev may be NULL. */
+int zoqat_op_attention_scratch_bytes(int batch, int seq, int n_heads, int d_head, size_t* bytes);
 int zoqat_op_attention(const float* qkv_dev, int batch, int seq, int n_heads, int d_head,
-                       const float* cos_dev, const float* sin_dev, float* out_dev, void* stream);
+                       const float* cos_dev, const float* sin_dev, float* out_dev,
+                       int impl, void* scratch_dev, int32_t* err_flag_dev, void* stream);
 
 /* Vocabulary projection fused with the cross-entropy: logits = A B^T are never
  * stored.  a_dev bf16 [T, d], b_dev bf16 [V, d], labels_dev int32 [T] (< 0 =

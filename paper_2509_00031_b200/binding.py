@@ -29,7 +29,8 @@ EXPORTS = [
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
-    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_attention", "zoqat_op_head_loss_scratch_bytes",
+    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
+    "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
 ]
 
@@ -100,7 +101,8 @@ def lib():
             "zoqat_op_norm_act_operand": [vp, i64, i64, i32, vp, vp, f32, i32, vp, vp, vp, vp],
             "zoqat_op_ffn_act_operand": [vp, i64, i64, i32, i32, vp, vp, vp],
             "zoqat_op_gemm": [vp, vp, i64, i64, i64, vp, vp, i32, i32, vp, i32, vp, vp],
-            "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, vp],
+            "zoqat_op_attention_scratch_bytes": [i32, i32, i32, i32, P(sz)],
+            "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp],
             "zoqat_op_head_loss_scratch_bytes": [i64, i64, P(sz)],
             "zoqat_op_head_loss": [vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, vp, vp],
             "zoqat_op_head_loss_static": [vp, vp, vp, i64, i64, i64, vp, vp, vp, i32, vp, vp],
@@ -218,10 +220,18 @@ def zoqat_op_gemm(a, b, row_step=None, bias=None, relu=False, out=None, accumula
     return out, err
 
 
-def zoqat_op_attention(qkv, batch, seq, n_heads, d_head, cos=None, sin=None):
+def zoqat_op_attention(qkv, batch, seq, n_heads, d_head, cos=None, sin=None, impl=GEMM_TCGEN05, scratch=None, err=None):
     out = torch.empty((batch * seq, n_heads * d_head), dtype=torch.float32, device=qkv.device)
-    _check(lib().zoqat_op_attention(_p(qkv), batch, seq, n_heads, d_head, _p(cos), _p(sin), _p(out), _stream()))
-    return out
+    if impl == GEMM_TCGEN05:
+        if scratch is None:
+            nb = ctypes.c_size_t()
+            _check(lib().zoqat_op_attention_scratch_bytes(batch, seq, n_heads, d_head, ctypes.byref(nb)))
+            scratch = torch.empty(nb.value, dtype=torch.uint8, device=qkv.device)
+        if err is None:
+            err = torch.zeros(1, dtype=torch.int32, device=qkv.device)
+    _check(lib().zoqat_op_attention(_p(qkv), batch, seq, n_heads, d_head, _p(cos), _p(sin), _p(out), impl, _p(scratch),
+                                    _p(err), _stream()))
+    return out, err
 
 
 def zoqat_op_head_loss(a, b, labels, impl=GEMM_TCGEN05):

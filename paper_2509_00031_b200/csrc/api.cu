@@ -72,6 +72,7 @@ struct Workspace {
     double* sums;                       // (sum L+, sum L-, labelled positions) of the last pair of passes
     int32_t *count, *err_flag;
     zoqat_step_result_dev* result;
+    void* attn_scratch;                 // fp16 hi/lo operands of the tensor-core attention
     size_t bop_elems;                   // elements of ONE pass' operand buffer
     size_t total;
 };
@@ -108,6 +109,7 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.count = (int32_t*)take(2 * 4);
     w.err_flag = (int32_t*)take(4);
     w.result = (zoqat_step_result_dev*)take(sizeof(zoqat_step_result_dev));
+    w.attn_scratch = take(attention_tc_scratch_bytes(2 * c.max_batch, c.max_seq, c.n_heads, c.d_model / c.n_heads));
     w.total = off;
 }
 
@@ -251,7 +253,13 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
         g.out = w.qkv; g.b_stride = ps;
         if (int rc = run_gemm(m, g, s)) return rc;
-        { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s); launch_attention(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, w.att, s); }
+        { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s);
+          if (c.gemm_impl == ZOQAT_GEMM_SIMT) {
+              launch_attention(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, w.att, s);
+          } else if (int rc = launch_attention_tc(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr,
+                                                  llama ? w.rope_sin : nullptr, w.att, w.attn_scratch, w.err_flag, s)) {
+              return fail(rc, "attention launch rejected");
+          } }
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s); }
         produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s);
         g = GemmArgs{};
@@ -728,12 +736,31 @@ int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, in
     return ZOQAT_OK;
 }
 
+int zoqat_op_attention_scratch_bytes(int batch, int seq, int n_heads, int d_head, size_t* bytes) {
+    if (batch <= 0 || seq <= 0 || n_heads <= 0 || (d_head != 64 && d_head != 128) || !bytes)
+        return fail(ZOQAT_ERR_INVALID_ARG, "bad attention scratch query");
+    *bytes = attention_tc_scratch_bytes(batch, seq, n_heads, d_head);
+    return ZOQAT_OK;
+}
+
 int zoqat_op_attention(const float* qkv_dev, int batch, int seq, int n_heads, int d_head, const float* cos_dev,
-                       const float* sin_dev, float* out_dev, void* stream) {
+                       const float* sin_dev, float* out_dev, int impl, void* scratch_dev, int32_t* err_flag_dev,
+                       void* stream) {
     if (!qkv_dev || !out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if (batch <= 0 || seq <= 0 || n_heads <= 0 || (d_head != 64 && d_head != 128)) return fail(ZOQAT_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", d_head);
     if ((cos_dev == nullptr) != (sin_dev == nullptr)) return fail(ZOQAT_ERR_INVALID_ARG, "cos/sin tables must both be given or both NULL");
-    launch_attention(qkv_dev, batch, seq, n_heads, d_head, cos_dev, sin_dev, out_dev, static_cast<cudaStream_t>(stream));
+    if ((reinterpret_cast<uintptr_t>(qkv_dev) | reinterpret_cast<uintptr_t>(out_dev) | reinterpret_cast<uintptr_t>(cos_dev) |
+         reinterpret_cast<uintptr_t>(sin_dev)) & 15)
+        return fail(ZOQAT_ERR_INVALID_ARG, "attention pointers must be 16-byte aligned");
+    if (impl == ZOQAT_GEMM_SIMT) {
+        launch_attention(qkv_dev, batch, seq, n_heads, d_head, cos_dev, sin_dev, out_dev, static_cast<cudaStream_t>(stream));
+    } else {
+        if (!scratch_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "the tensor-core attention needs scratch_dev and err_flag_dev");
+        if (reinterpret_cast<uintptr_t>(scratch_dev) & 255) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 256-byte aligned");
+        if (int rc = launch_attention_tc(qkv_dev, batch, seq, n_heads, d_head, cos_dev, sin_dev, out_dev, scratch_dev,
+                                         err_flag_dev, static_cast<cudaStream_t>(stream)))
+            return fail(rc, "attention launch rejected");
+    }
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -1,0 +1,557 @@
+// Causal softmax attention of one layer on the tensor cores (sm_100a: tcgen05 / TMEM / TMA).
+//
+// Precision.  The attention output feeds a per-token int8 quantiser, so it has to be
+// binary32-grade, not bf16-grade.  Every operand x (rotated and pre-scaled q, rotated k, v,
+// and the softmax numerators p) is therefore split into two binary16 numbers,
+//     hi = fp16(x),   lo = fp16((x - hi) * 2^11),        x = hi + lo * 2^-11 (to ~2^-22 relative),
+// and every product A B^T is evaluated as three tensor-core products with fp32 accumulation,
+//     A B^T ~= Ah Bh^T + 2^-11 (Ah Bl^T + Al Bh^T),
+// the main and the correction term in separate TMEM accumulators, combined in fp32 when read.
+// Operands must be finite in binary16 (|x| < 65504); larger values give inf/NaN, not a silently
+// wrong result.
+//
+// Two kernels:
+//   attn_prep_kernel   fp32 q|k|v -> rotary embedding, q * log2(e)/sqrt(d_head), hi/lo split;
+//                      q and k as [batch][head][seq][d_head], v transposed [batch][head][d_head][seq]
+//                      so that every tensor-core operand is K-major.
+//   attention_tc_kernel  persistent, one CTA per SM, 320 threads:
+//     warp 0     TMA producer: Q tile (128 queries) once per work item, then K / V^T tiles of 64 keys
+//                (hi and lo) into a two-stage ring.
+//     warp 1     MMA issuer: S_j = Q K_j^T (N = 64) into one of two TMEM score buffers - issued one
+//                tile ahead of the softmax - and O_j = P_j V_j (N = d_head).
+//     warps 2-9  softmax: two threads per query row (each half of the columns).  Read S_j from TMEM,
+//                running max / sum (base-2 exponentials), write P_j hi/lo to shared memory in the
+//                operand layout, and accumulate O_j from TMEM into registers with the usual
+//                rescaling; finally out = acc / sum.
+// Scores and probabilities never reach global memory.  Work items (query tile, head, batch) are
+// taken heaviest first.  Every wait is bounded and reports through *err_flag.
+#include "common.cuh"
+#include "../../include/zoqat.h"
+#include "tc_ptx.cuh"
+#include <cuda_fp16.h>
+
+namespace zq {
+namespace {
+
+constexpr int BQ = 128, BKV = 64;
+constexpr int kAttThreadsTC = 320;
+constexpr float kLoScale = 2048.0f, kLoInv = 1.0f / 2048.0f;
+constexpr int kErrAttnSmem = 16;       // dynamic shared memory window too small after alignment
+constexpr int kErrAttnWait = 17;       // a bounded wait of the attention kernel ran out
+
+template <int D> struct AttCfg {
+    static constexpr int kQBytes = BQ * D * 2;            // one of Qh / Ql
+    static constexpr int kKBytes = BKV * D * 2;           // one of Kh / Kl / Vth / Vtl of a stage
+    static constexpr int kStages = 2;
+    static constexpr int kStageBytes = 4 * kKBytes;
+    static constexpr int kPBytes = BQ * BKV * 2;          // one of Ph / Pl
+    static constexpr int kOffStage = 2 * kQBytes;
+    static constexpr int kOffP = kOffStage + kStages * kStageBytes;
+    static constexpr int kOffX = kOffP + 2 * kPBytes;     // row-max exchange: [2 slots][128 rows][2 halves] floats
+    static constexpr int kOffBar = kOffX + 2048;
+    static constexpr int kUsedBytes = kOffBar + 160;      // 18 mbarriers + the TMEM base word
+    // Request the whole opt-in window for d_head 128 (the tiles need all but ~860 bytes of it) and enough to
+    // keep a second CTA off the SM for d_head 64 (a CTA owns all 512 TMEM columns).
+    static constexpr int kSmemBytes = (D == 128) ? 232448 : (kUsedBytes + 1024 > 120 * 1024 ? kUsedBytes + 1024 : 120 * 1024);
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, fp16 x fp16 -> fp32, one CTA.
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// kind::f16 instruction descriptor: fp32 accumulate, fp16 A and B (format 0), both K-major, M = 128.
+__device__ __forceinline__ uint32_t idesc_f16(int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
+}
+
+struct AttParams {
+    int seq, n_heads, batch;
+    int n_qt;                 // query tiles per (batch, head)
+    int total_items;
+    float* out;               // [batch*seq, n_heads*D]
+    int32_t* err_flag;
+    uint32_t smem_bytes;
+};
+
+// hi / lo split of x into binary16
+__device__ __forceinline__ void split16(float x, __half& hi, __half& lo) {
+    hi = __float2half_rn(x);
+    lo = __float2half_rn((x - __half2float(hi)) * kLoScale);
+}
+
+// ---- preparation: rotary embedding, scaling, split, transpose of v ------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256)
+attn_prep_kernel(const float* __restrict__ qkv, int seq, int seq_pad, int n_heads, const float* __restrict__ cos_t,
+                 const float* __restrict__ sin_t, float q_mul, __half* __restrict__ qh, __half* __restrict__ ql,
+                 __half* __restrict__ kh, __half* __restrict__ kl, __half* __restrict__ vth, __half* __restrict__ vtl) {
+    constexpr int H4 = D / 8;                  // float4 per half row
+    constexpr int LDV = 64 + 8;                // padded token stride of the transposed v tile (halfs)
+    __shared__ __align__(16) __half vs_h[D * LDV];
+    __shared__ __align__(16) __half vs_l[D * LDV];
+    const int head = blockIdx.y, b = blockIdx.z;
+    const int d_model = n_heads * D, ld = 3 * d_model;
+    const int pos0 = blockIdx.x * 64;
+    const int tid = threadIdx.x;
+    const float* base = qkv + (int64_t)b * seq * ld + head * D;
+    const int64_t bh = (int64_t)b * n_heads + head;
+
+    // q and k: pairs (i, i + D/2) rotate together
+    for (int idx = tid; idx < 2 * 64 * H4; idx += 256) {
+        const int sel = idx / (64 * H4);       // 0 q, 1 k
+        const int r = (idx / H4) % 64, c4 = idx % H4;
+        const int pos = pos0 + r;
+        if (pos >= seq) continue;
+        const float* src = base + (int64_t)pos * ld + sel * d_model;
+        float4 lo = *reinterpret_cast<const float4*>(src + 4 * c4);
+        float4 hi = *reinterpret_cast<const float4*>(src + D / 2 + 4 * c4);
+        if (cos_t != nullptr) {
+            const float4 c = *reinterpret_cast<const float4*>(cos_t + (int64_t)pos * (D / 2) + 4 * c4);
+            const float4 s = *reinterpret_cast<const float4*>(sin_t + (int64_t)pos * (D / 2) + 4 * c4);
+            const float4 a = lo, bb = hi;
+            lo.x = a.x * c.x - bb.x * s.x; hi.x = bb.x * c.x + a.x * s.x;
+            lo.y = a.y * c.y - bb.y * s.y; hi.y = bb.y * c.y + a.y * s.y;
+            lo.z = a.z * c.z - bb.z * s.z; hi.z = bb.z * c.z + a.z * s.z;
+            lo.w = a.w * c.w - bb.w * s.w; hi.w = bb.w * c.w + a.w * s.w;
+        }
+        const float mul = sel == 0 ? q_mul : 1.0f;
+        const float v[8] = {lo.x * mul, lo.y * mul, lo.z * mul, lo.w * mul, hi.x * mul, hi.y * mul, hi.z * mul, hi.w * mul};
+        __align__(8) __half oh[8], ol[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) split16(v[i], oh[i], ol[i]);
+        __half* dh_ = (sel == 0 ? qh : kh) + (bh * seq + pos) * D;
+        __half* dl_ = (sel == 0 ? ql : kl) + (bh * seq + pos) * D;
+        *reinterpret_cast<uint2*>(dh_ + 4 * c4) = *reinterpret_cast<const uint2*>(oh);
+        *reinterpret_cast<uint2*>(dh_ + D / 2 + 4 * c4) = *reinterpret_cast<const uint2*>(oh + 4);
+        *reinterpret_cast<uint2*>(dl_ + 4 * c4) = *reinterpret_cast<const uint2*>(ol);
+        *reinterpret_cast<uint2*>(dl_ + D / 2 + 4 * c4) = *reinterpret_cast<const uint2*>(ol + 4);
+    }
+    // v: split, transpose through shared memory
+    for (int idx = tid; idx < 64 * (D / 4); idx += 256) {
+        const int r = idx / (D / 4), c4 = idx % (D / 4);
+        const int pos = pos0 + r;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (pos < seq) x = *reinterpret_cast<const float4*>(base + (int64_t)pos * ld + 2 * d_model + 4 * c4);
+        const float v[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __half h, l;
+            split16(v[i], h, l);
+            vs_h[(4 * c4 + i) * LDV + r] = h;
+            vs_l[(4 * c4 + i) * LDV + r] = l;
+        }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < D * 8; idx += 256) {          // 8 tokens (16 bytes) per store
+        const int dd = idx / 8, t8 = idx % 8;
+        const int pos = pos0 + 8 * t8;
+        if (pos >= seq_pad) continue;
+        const int64_t o = (bh * D + dd) * (int64_t)seq_pad + pos;
+        *reinterpret_cast<uint4*>(vth + o) = *reinterpret_cast<const uint4*>(vs_h + dd * LDV + 8 * t8);
+        *reinterpret_cast<uint4*>(vtl + o) = *reinterpret_cast<const uint4*>(vs_l + dd * LDV + 8 * t8);
+    }
+}
+
+// ---- the attention kernel ---------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kAttThreadsTC, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_constant__ CUtensorMap map_ql,
+                    const __grid_constant__ CUtensorMap map_kh, const __grid_constant__ CUtensorMap map_kl,
+                    const __grid_constant__ CUtensorMap map_vth, const __grid_constant__ CUtensorMap map_vtl,
+                    AttParams p) {
+    using Cfg = AttCfg<D>;
+    constexpr int KSUB = D / 64;               // 64-column (128-byte) sub-tiles along d_head
+    constexpr int DH = D / 2;                  // output columns per softmax thread
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const bool smem_ok = (base - raw) + (uint32_t)Cfg::kUsedBytes <= p.smem_bytes;
+    const uint32_t bars = base + Cfg::kOffBar;
+    // barriers (8 bytes each)
+    const uint32_t q_full = bars, q_empty = bars + 8;
+    auto kv_full = [&](int s) { return bars + 16u + 8u * s; };
+    auto kv_empty = [&](int s) { return bars + 32u + 8u * s; };
+    auto s_full = [&](int b) { return bars + 48u + 8u * b; };
+    auto s_empty = [&](int b) { return bars + 64u + 8u * b; };
+    const uint32_t p_full = bars + 80, p_empty = bars + 88, o_full = bars + 96, o_empty = bars + 104;
+    auto x_bar = [&](int q) { return bars + 112u + 8u * q; };
+    const uint32_t tmem_slot = bars + 144;
+    uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - raw));
+    float* xchg = reinterpret_cast<float*>(smem_raw + (base + Cfg::kOffX - raw));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (!smem_ok) {                              // uniform over the CTA: nothing has been set up yet
+        if (threadIdx.x == 0) atomicExch(p.err_flag, kErrAttnSmem);
+        return;
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1); mbar_init(q_empty, 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); mbar_init(s_full(s), 1); mbar_init(s_empty(s), 8); }
+        mbar_init(p_full, 8); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 8);
+        for (int q = 0; q < 4; ++q) mbar_init(x_bar(q), 2);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&map_qh); prefetch_tmap(&map_ql); prefetch_tmap(&map_kh);
+        prefetch_tmap(&map_kl); prefetch_tmap(&map_vth); prefetch_tmap(&map_vtl);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    const int HB = p.n_heads * p.batch;
+    // work item -> (query tile, batch*head); heaviest (latest) query tiles first
+    auto item_qt = [&](int it) { return p.n_qt - 1 - it / HB; };
+    auto item_bh = [&](int it) { return it % HB; };
+    auto n_kv_tiles = [&](int qt) { const int hi_ = min(p.seq, (qt + 1) * BQ); return (hi_ + BKV - 1) / BKV; };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t kv_it = 0, q_it = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
+                const int qt = item_qt(it), bh = item_bh(it), n = n_kv_tiles(qt);
+                if (!mbar_wait(q_empty, (q_it & 1u) ^ 1u)) { atomicExch(p.err_flag, kErrAttnWait); ok = false; break; }
+                mbar_arrive_expect_tx(q_full, 2 * Cfg::kQBytes);
+#pragma unroll
+                for (int sub = 0; sub < KSUB; ++sub) {
+                    tma_load_3d(base + sub * (BQ * 128), &map_qh, q_full, sub * 64, qt * BQ, bh);
+                    tma_load_3d(base + Cfg::kQBytes + sub * (BQ * 128), &map_ql, q_full, sub * 64, qt * BQ, bh);
+                }
+                for (int j = 0; j < n; ++j, ++kv_it) {
+                    const int st = kv_it & 1u;
+                    if (!mbar_wait(kv_empty(st), ((kv_it >> 1) & 1u) ^ 1u)) { atomicExch(p.err_flag, kErrAttnWait); ok = false; break; }
+                    mbar_arrive_expect_tx(kv_full(st), Cfg::kStageBytes);
+                    const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
+#pragma unroll
+                    for (int sub = 0; sub < KSUB; ++sub) {
+                        tma_load_3d(sb + sub * (BKV * 128), &map_kh, kv_full(st), sub * 64, j * BKV, bh);
+                        tma_load_3d(sb + Cfg::kKBytes + sub * (BKV * 128), &map_kl, kv_full(st), sub * 64, j * BKV, bh);
+                    }
+                    tma_load_3d(sb + 2 * Cfg::kKBytes, &map_vth, kv_full(st), j * BKV, 0, bh);
+                    tma_load_3d(sb + 3 * Cfg::kKBytes, &map_vtl, kv_full(st), j * BKV, 0, bh);
+                }
+            }
+            // every load issued above has to land before the CTA may leave
+            for (int i = 0; i < 2 && ok; ++i, ++kv_it)
+                if (!mbar_wait(kv_empty(kv_it & 1u), ((kv_it >> 1) & 1u) ^ 1u)) break;
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc_s = idesc_f16(BKV), idesc_o = idesc_f16(D);
+            uint32_t kv_it = 0, t_it = 0, q_it = 0;
+            bool ok = true;
+            // S of global tile g (stage / score buffer g & 1)
+            auto issue_s = [&](uint32_t g) -> bool {
+                const int st = g & 1u;
+                if (!mbar_wait(kv_full(st), (g >> 1) & 1u)) return false;
+                if (!mbar_wait(s_empty(st), ((g >> 1) & 1u) ^ 1u)) return false;
+                tc_fence_after();
+                const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
+                const uint32_t d_main = tmem_base + (uint32_t)(st * 128), d_corr = d_main + 64u;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (uint32_t)((k >> 2) * (BQ * 128)), offk = (uint32_t)((k >> 2) * (BKV * 128));
+                    const uint64_t aqh = smem_desc_sw128(base + off) + (uint64_t)(2 * (k & 3));
+                    const uint64_t bkh = smem_desc_sw128(sb + offk) + (uint64_t)(2 * (k & 3));
+                    umma_f16(d_main, aqh, bkh, idesc_s, k > 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (uint32_t)((k >> 2) * (BQ * 128)), offk = (uint32_t)((k >> 2) * (BKV * 128));
+                    const uint64_t aqh = smem_desc_sw128(base + off) + (uint64_t)(2 * (k & 3));
+                    const uint64_t aql = smem_desc_sw128(base + Cfg::kQBytes + off) + (uint64_t)(2 * (k & 3));
+                    const uint64_t bkh = smem_desc_sw128(sb + offk) + (uint64_t)(2 * (k & 3));
+                    const uint64_t bkl = smem_desc_sw128(sb + Cfg::kKBytes + offk) + (uint64_t)(2 * (k & 3));
+                    umma_f16(d_corr, aqh, bkl, idesc_s, k > 0 ? 1u : 0u);
+                    umma_f16(d_corr, aql, bkh, idesc_s, 1u);
+                }
+                umma_commit(s_full(st));
+                return true;
+            };
+            for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
+                const int n = n_kv_tiles(item_qt(it));
+                if (!mbar_wait(q_full, q_it & 1u)) { ok = false; break; }
+                if (!issue_s(kv_it)) { ok = false; break; }
+                if (n == 1) umma_commit(q_empty);
+                for (int j = 0; j < n; ++j, ++t_it) {
+                    if (j + 1 < n) {
+                        if (!issue_s(kv_it + j + 1)) { ok = false; break; }
+                        if (j + 2 == n) umma_commit(q_empty);     // Q is free once the last S of the item has completed
+                    }
+                    if (!mbar_wait(p_full, t_it & 1u) || !mbar_wait(o_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
+                    tc_fence_after();
+                    const int st = (kv_it + j) & 1u;
+                    const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
+                    const uint32_t ph = base + Cfg::kOffP, pl = ph + Cfg::kPBytes;
+                    const uint32_t o_main = tmem_base + 256u, o_corr = tmem_base + 384u;
+#pragma unroll
+                    for (int k = 0; k < BKV / 16; ++k) {
+                        const uint64_t aph = smem_desc_sw128(ph) + (uint64_t)(2 * k);
+                        const uint64_t bvh = smem_desc_sw128(sb + 2 * Cfg::kKBytes) + (uint64_t)(2 * k);
+                        umma_f16(o_main, aph, bvh, idesc_o, k > 0 ? 1u : 0u);
+                    }
+#pragma unroll
+                    for (int k = 0; k < BKV / 16; ++k) {
+                        const uint64_t aph = smem_desc_sw128(ph) + (uint64_t)(2 * k);
+                        const uint64_t apl = smem_desc_sw128(pl) + (uint64_t)(2 * k);
+                        const uint64_t bvh = smem_desc_sw128(sb + 2 * Cfg::kKBytes) + (uint64_t)(2 * k);
+                        const uint64_t bvl = smem_desc_sw128(sb + 3 * Cfg::kKBytes) + (uint64_t)(2 * k);
+                        umma_f16(o_corr, aph, bvl, idesc_o, k > 0 ? 1u : 0u);
+                        umma_f16(o_corr, apl, bvh, idesc_o, 1u);
+                    }
+                    umma_commit(o_full);
+                    umma_commit(kv_empty(st));
+                    umma_commit(p_empty);
+                }
+                kv_it += n;
+            }
+            if (!ok) atomicExch(p.err_flag, kErrAttnWait);
+        }
+    } else {
+        // ---------------- softmax / output warps (2..9) ----------------
+        const int quarter = warp & 3;                       // TMEM lanes [32*quarter, 32*quarter + 32)
+        const int half = (warp - 2) >> 2;                   // which half of the columns
+        const int row = quarter * 32 + lane;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int d_model = p.n_heads * D;
+        uint32_t s_it = 0, t_it = 0, x_it = 0;
+        bool ok = true;
+        // wait helper: the whole warp takes the same decision
+        auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)) != 0; };
+        for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x) {
+            const int qt = item_qt(it), bh = item_bh(it), n = n_kv_tiles(qt);
+            const int qpos = qt * BQ + row;
+            float m_run = -INFINITY, l_run = 0.0f, corr_prev = 1.0f;
+            float acc[DH];
+#pragma unroll
+            for (int c = 0; c < DH; ++c) acc[c] = 0.0f;
+
+            // acc <- acc * corr_prev + (O_main + 2^-11 O_corr) of the previous tile, then release the O buffer
+            auto take_o = [&]() -> bool {
+                if (!wait_all(o_full, (t_it & 1u) ^ 1u)) return false;     // tile t_it - 1
+                tc_fence_after();
+#pragma unroll
+                for (int c0 = 0; c0 < DH; c0 += 32) {
+                    uint32_t om[32], oc[32];
+                    tmem_ld32(t_lane + 256u + (uint32_t)(half * DH + c0), om);
+                    tmem_ld32(t_lane + 384u + (uint32_t)(half * DH + c0), oc);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        acc[c0 + c] = fmaf(acc[c0 + c], corr_prev, fmaf(__uint_as_float(oc[c]), kLoInv, __uint_as_float(om[c])));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(o_empty);
+                return true;
+            };
+
+            for (int j = 0; j < n; ++j, ++s_it, ++t_it, ++x_it) {
+                const int sbuf = s_it & 1u;
+                if (!wait_all(s_full(sbuf), (s_it >> 1) & 1u)) { ok = false; break; }
+                tc_fence_after();
+                float s[32];
+                {
+                    uint32_t sm[32], sc[32];
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + half * 32), sm);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64 + half * 32), sc);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s[c] = fmaf(__uint_as_float(sc[c]), kLoInv, __uint_as_float(sm[c]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty(sbuf));
+                // causal mask (keys beyond the sequence end are beyond every valid query as well)
+                const int k0 = j * BKV + half * 32;
+                if (j * BKV + BKV - 1 > qt * BQ) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (k0 + c > qpos) s[c] = -INFINITY;
+                }
+                float mx = s[0];
+#pragma unroll
+                for (int c = 1; c < 32; ++c) mx = fmaxf(mx, s[c]);
+                // exchange the half-row maxima with the partner warp of this quarter
+                xchg[((x_it & 1u) * BQ + row) * 2 + half] = mx;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(x_bar(quarter));
+                if (!wait_all(x_bar(quarter), x_it & 1u)) { ok = false; break; }
+                mx = fmaxf(mx, xchg[((x_it & 1u) * BQ + row) * 2 + (half ^ 1)]);
+                const float m_new = fmaxf(m_run, mx);         // finite: key 0 is visible to every query
+                const float corr = ex2(m_run - m_new);
+                float rs = 0.0f;
+#pragma unroll
+                for (int c = 0; c < 32; ++c) { s[c] = ex2(s[c] - m_new); rs += s[c]; }
+                l_run = fmaf(l_run, corr, rs);
+                m_run = m_new;
+                // O of the previous tile (frees the O accumulators for this tile's P V)
+                if (j > 0 && !take_o()) { ok = false; break; }
+                corr_prev = corr;
+                // P -> shared memory (operand layout: 128-byte rows, 16-byte chunks XOR-swizzled by row)
+                if (!wait_all(p_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
+                const uint32_t ph = base + Cfg::kOffP + (uint32_t)(row * 128), pl = ph + Cfg::kPBytes;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t wh[4], wl[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float a = s[8 * i + 2 * e], b2 = s[8 * i + 2 * e + 1];
+                        const __half2 h2 = __floats2half2_rn(a, b2);
+                        const float2 hf = __half22float2(h2);
+                        const __half2 l2 = __floats2half2_rn((a - hf.x) * kLoScale, (b2 - hf.y) * kLoScale);
+                        wh[e] = *reinterpret_cast<const uint32_t*>(&h2);
+                        wl[e] = *reinterpret_cast<const uint32_t*>(&l2);
+                    }
+                    const uint32_t chunk = (uint32_t)(((half * 4 + i) ^ (row & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ph + chunk), "r"(wh[0]), "r"(wh[1]), "r"(wh[2]), "r"(wh[3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pl + chunk), "r"(wl[0]), "r"(wl[1]), "r"(wl[2]), "r"(wl[3]) : "memory");
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full);
+            }
+            if (!ok) break;
+            if (!take_o()) { ok = false; break; }             // the last tile of the item
+            // total row sum = both halves
+            xchg[((x_it & 1u) * BQ + row) * 2 + half] = l_run;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_bar(quarter));
+            if (!wait_all(x_bar(quarter), x_it & 1u)) { ok = false; break; }
+            const float l_tot = l_run + xchg[((x_it & 1u) * BQ + row) * 2 + (half ^ 1)];
+            ++x_it;
+            if (qpos < p.seq) {
+                const float inv = 1.0f / l_tot;
+                const int b = bh / p.n_heads, head = bh % p.n_heads;
+                float* dst = p.out + ((int64_t)b * p.seq + qpos) * d_model + head * D + half * DH;
+#pragma unroll
+                for (int c = 0; c < DH; c += 4)
+                    *reinterpret_cast<float4*>(dst + c) = make_float4(acc[c] * inv, acc[c + 1] * inv, acc[c + 2] * inv, acc[c + 3] * inv);
+            }
+        }
+        if (!ok && lane == 0) atomicExch(p.err_flag, kErrAttnWait);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ---- host side --------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn att_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 3-D fp16 map {inner, rows, slabs}; box = 64 x box_rows x 1, 128-byte swizzle, zero fill outside.
+bool make_half_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t slabs, int64_t row_pitch,
+                   int box_rows) {
+    EncodeTiledFn fn = att_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)slabs};
+    const cuuint64_t strides[2] = {(cuuint64_t)row_pitch * 2, (cuuint64_t)row_pitch * rows * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+inline int pad8(int s) { return (s + 7) / 8 * 8; }
+
+template <int D>
+int attention_tc_launch(const float* qkv, int batch, int seq, int n_heads, const float* cos_t, const float* sin_t,
+                        float* out, void* scratch, int32_t* err_flag, cudaStream_t s) {
+    using Cfg = AttCfg<D>;
+    const int seq_pad = pad8(seq);
+    const int64_t bhs = (int64_t)batch * n_heads;
+    const size_t qk_bytes = up256((size_t)bhs * seq * D * 2), vt_bytes = up256((size_t)bhs * D * seq_pad * 2);
+    uint8_t* sp = static_cast<uint8_t*>(scratch);
+    __half* qh = reinterpret_cast<__half*>(sp);
+    __half* ql = reinterpret_cast<__half*>(sp + qk_bytes);
+    __half* kh = reinterpret_cast<__half*>(sp + 2 * qk_bytes);
+    __half* kl = reinterpret_cast<__half*>(sp + 3 * qk_bytes);
+    __half* vth = reinterpret_cast<__half*>(sp + 4 * qk_bytes);
+    __half* vtl = reinterpret_cast<__half*>(sp + 4 * qk_bytes + vt_bytes);
+
+    const float q_mul = (float)(1.4426950408889634 / sqrt((double)D));
+    dim3 pgrid((seq + 63) / 64, n_heads, batch);
+    attn_prep_kernel<D><<<pgrid, 256, 0, s>>>(qkv, seq, seq_pad, n_heads, cos_t, sin_t, q_mul, qh, ql, kh, kl, vth, vtl);
+
+    alignas(64) CUtensorMap m_qh, m_ql, m_kh, m_kl, m_vth, m_vtl;
+    if (!make_half_map(&m_qh, qh, D, seq, bhs, D, BQ) || !make_half_map(&m_ql, ql, D, seq, bhs, D, BQ) ||
+        !make_half_map(&m_kh, kh, D, seq, bhs, D, BKV) || !make_half_map(&m_kl, kl, D, seq, bhs, D, BKV) ||
+        !make_half_map(&m_vth, vth, seq, D, bhs, seq_pad, D) || !make_half_map(&m_vtl, vtl, seq, D, bhs, seq_pad, D))
+        return ZOQAT_ERR_CUDA;
+    static bool attr = false;
+    if (!attr) {
+        if (cudaFuncSetAttribute(attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+            return ZOQAT_ERR_CUDA;
+        attr = true;
+    }
+    AttParams p;
+    p.seq = seq; p.n_heads = n_heads; p.batch = batch;
+    p.n_qt = (seq + BQ - 1) / BQ;
+    p.total_items = p.n_qt * n_heads * batch;
+    p.out = out; p.err_flag = err_flag; p.smem_bytes = Cfg::kSmemBytes;
+    int sms = 0, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms <= 0) sms = 148;
+    const int grid = p.total_items < sms ? p.total_items : sms;
+    attention_tc_kernel<D><<<grid, kAttThreadsTC, Cfg::kSmemBytes, s>>>(m_qh, m_ql, m_kh, m_kl, m_vth, m_vtl, p);
+    count_launch(2);
+    return ZOQAT_OK;
+}
+
+}  // namespace
+
+size_t attention_tc_scratch_bytes(int batch, int seq, int n_heads, int d_head) {
+    const size_t bhs = (size_t)batch * n_heads;
+    return 4 * up256(bhs * seq * d_head * 2) + 2 * up256(bhs * d_head * pad8(seq) * 2);
+}
+
+int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d_head, const float* cos_t,
+                        const float* sin_t, float* out, void* scratch, int32_t* err_flag, cudaStream_t s) {
+    if (!scratch || !err_flag || (reinterpret_cast<uintptr_t>(scratch) & 255)) return ZOQAT_ERR_INVALID_ARG;
+    if (d_head == 64) return attention_tc_launch<64>(qkv, batch, seq, n_heads, cos_t, sin_t, out, scratch, err_flag, s);
+    if (d_head == 128) return attention_tc_launch<128>(qkv, batch, seq, n_heads, cos_t, sin_t, out, scratch, err_flag, s);
+    return ZOQAT_ERR_UNSUPPORTED;
+}
+
+}  // namespace zq

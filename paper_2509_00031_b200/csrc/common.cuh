@@ -43,8 +43,12 @@ void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_ki
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s);
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
                             __nv_bfloat16* op, float* row_step, cudaStream_t s);
+// fp32 CUDA-core attention (cross-check) and the tensor-core attention (needs scratch and an error word).
 void launch_attention(const float* qkv, int batch, int seq, int n_heads, int d_head,
                       const float* cos_t, const float* sin_t, float* out, cudaStream_t s);
+size_t attention_tc_scratch_bytes(int batch, int seq, int n_heads, int d_head);
+int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d_head, const float* cos_t,
+                        const float* sin_t, float* out, void* scratch, int32_t* err_flag, cudaStream_t s);
 
 // out[z*M + m, n] (+)= row_step[z*M+m] * sum_k A[z*M+m, k] * B[z][n, k] (+ bias[n]) (relu)
 // mode 1: cross-entropy partials instead of a store (labels[m], partials [Z*M, n_tiles], label_logit [Z*M]).

@@ -93,10 +93,16 @@ def main():
     elif a.op == "attention":
         d = a.heads * a.dh
         qkv = torch.randn(a.batch * a.seq, 3 * d, device=dev)
-        fn = lambda: zq.zoqat_op_attention(qkv, a.batch, a.seq, a.heads, a.dh)
+        import ctypes
+        nb = ctypes.c_size_t()
+        zq.lib().zoqat_op_attention_scratch_bytes(a.batch, a.seq, a.heads, a.dh, ctypes.byref(nb))
+        scratch = torch.empty(nb.value, dtype=torch.uint8, device=dev)
+        err = torch.zeros(1, dtype=torch.int32, device=dev)
+        fn = lambda: zq.zoqat_op_attention(qkv, a.batch, a.seq, a.heads, a.dh, impl=a.impl, scratch=scratch, err=err)
         med, best = timed(fn, a.iters, flush)
         flops = 2.0 * a.batch * a.seq * a.seq * d          # causal: half of 4*B*S^2*d
-        out.update(batch=a.batch, seq=a.seq, heads=a.heads, dh=a.dh, ms=med, ms_best=best, tflops=flops / med / 1e9)
+        out.update(batch=a.batch, seq=a.seq, heads=a.heads, dh=a.dh, impl=a.impl, ms=med, ms_best=best, tflops=flops / med / 1e9,
+                   err_flag=int(err.item()))
     elif a.op in ("norm_act", "ffn_act"):
         if a.op == "norm_act":
             x = torch.randn(a.rows, a.cols, device=dev)
