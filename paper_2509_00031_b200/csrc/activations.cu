@@ -117,6 +117,152 @@ ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_b
     write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
 }
 
+// ---- register-resident variants (rows up to 12288 columns) ------------------------------------------------
+// The row never leaves registers: VPT float4 per thread, 16-byte loads and 8-byte operand stores, one pass over
+// global memory in each direction.  Same arithmetic as the shared-memory kernels above.
+__device__ __forceinline__ float amax4(const float4& v) { return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))); }
+
+__device__ __forceinline__ uint2 bf16x4(float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
+template <int VPT>
+__device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n4, int a_bits, uint2* op_row, float* row_step,
+                                                   float* redf) {
+    if (a_bits == 8) {
+        float amax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) amax = fmaxf(amax, amax4(v[i]));      // slots beyond the row hold zeros
+        amax = block_max(amax, redf);
+        const float step = fmaxf(__fdiv_rn(amax, 127.0f), 1e-8f);
+        const float inv = __fdiv_rn(1.0f, step);
+        if (threadIdx.x == 0) *row_step = step;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4)
+                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), -128.0f), 127.0f));
+        }
+    } else {
+        if (threadIdx.x == 0) *row_step = 1.0f;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) op_row[idx] = bf16x4(v[i].x, v[i].y, v[i].z, v[i].w);
+        }
+    }
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kRowThreads)
+norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
+                            const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
+                            float* __restrict__ row_step, float* __restrict__ normed) {
+    __shared__ double redd[kRowThreads / 32];
+    __shared__ float redf[kRowThreads / 32];
+    const int64_t r = blockIdx.x;
+    const int n4 = cols >> 2;
+    const float4* xr = reinterpret_cast<const float4*>(x + r * cols);
+    float4 v[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int idx = threadIdx.x + i * kRowThreads;
+        v[i] = idx < n4 ? xr[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (norm_kind == 1) {
+        double ss = 0.0;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i)
+            ss += (double)v[i].x * v[i].x + (double)v[i].y * v[i].y + (double)v[i].z * v[i].z + (double)v[i].w * v[i].w;
+        ss = block_sum(ss, redd);
+        const float rstd = (float)(1.0 / sqrt(ss / cols + (double)norm_eps));
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) {
+                const float4 g = reinterpret_cast<const float4*>(gain)[idx];
+                v[i].x = v[i].x * rstd * g.x; v[i].y = v[i].y * rstd * g.y; v[i].z = v[i].z * rstd * g.z; v[i].w = v[i].w * rstd * g.w;
+            }
+        }
+    } else if (norm_kind == 2) {
+        double sm = 0.0;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) sm += (double)v[i].x + (double)v[i].y + (double)v[i].z + (double)v[i].w;
+        const double mu = block_sum(sm, redd) / cols;
+        double sv = 0.0;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) {
+                const double a = (double)v[i].x - mu, b = (double)v[i].y - mu, c = (double)v[i].z - mu, d = (double)v[i].w - mu;
+                sv += a * a + b * b + c * c + d * d;
+            }
+        }
+        sv = block_sum(sv, redd);
+        const float rstd = (float)(1.0 / sqrt(sv / cols + (double)norm_eps));
+        const float muf = (float)mu;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) {
+                const float4 g = reinterpret_cast<const float4*>(gain)[idx];
+                const float4 b = reinterpret_cast<const float4*>(bias)[idx];
+                v[i].x = (v[i].x - muf) * rstd * g.x + b.x; v[i].y = (v[i].y - muf) * rstd * g.y + b.y;
+                v[i].z = (v[i].z - muf) * rstd * g.z + b.z; v[i].w = (v[i].w - muf) * rstd * g.w + b.w;
+            }
+        }
+    }
+    if (normed) {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) reinterpret_cast<float4*>(normed + r * cols)[idx] = v[i];
+        }
+    }
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kRowThreads)
+ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
+                           float* __restrict__ row_step) {
+    __shared__ float redf[kRowThreads / 32];
+    const int64_t r = blockIdx.x;
+    const int n4 = cols >> 2;
+    float4 v[VPT];
+    if (gated) {
+        const float4* g4 = reinterpret_cast<const float4*>(x + r * 2 * cols);
+        const float4* u4 = g4 + n4;
+        float4 u[VPT];
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            v[i] = idx < n4 ? __ldcs(g4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+            u[i] = idx < n4 ? __ldcs(u4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            v[i].x = __fdiv_rn(v[i].x, 1.0f + expf(-v[i].x)) * u[i].x;
+            v[i].y = __fdiv_rn(v[i].y, 1.0f + expf(-v[i].y)) * u[i].y;
+            v[i].z = __fdiv_rn(v[i].z, 1.0f + expf(-v[i].z)) * u[i].z;
+            v[i].w = __fdiv_rn(v[i].w, 1.0f + expf(-v[i].w)) * u[i].w;
+        }
+    } else {
+        const float4* g4 = reinterpret_cast<const float4*>(x + r * cols);
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            const float4 g = idx < n4 ? __ldcs(g4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[i] = make_float4(fmaxf(g.x, 0.f), fmaxf(g.y, 0.f), fmaxf(g.z, 0.f), fmaxf(g.w, 0.f));
+        }
+    }
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
+}
+
 // h[p*T + t, :] = embed[token[t], :] (+ pos[t % seq, :]) for each of `passes` copies.
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const float4* __restrict__ embed,
                              const float4* __restrict__ pos, int64_t T, int seq, int d4, int vocab, int passes,
@@ -232,19 +378,40 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s) {
-    const size_t smem = (size_t)cols * sizeof(float);
-    static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-    norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    const int n4 = cols / 4;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(bias) |
+                           reinterpret_cast<uintptr_t>(normed)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
+    if (aligned && n4 <= 4 * kRowThreads) {
+        norm_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    } else if (aligned && n4 <= 8 * kRowThreads) {
+        norm_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    } else if (aligned && n4 <= 12 * kRowThreads) {
+        norm_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    } else {
+        const size_t smem = (size_t)cols * sizeof(float);
+        static bool attr = false;
+        if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+        norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+    }
     count_launch();
 }
 
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
                             float* row_step, cudaStream_t s) {
-    const size_t smem = (size_t)cols * sizeof(float);
-    static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-    ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step);
+    const int n4 = cols / 4;
+    const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
+    if (aligned && n4 <= 4 * kRowThreads) {
+        ffn_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+    } else if (aligned && n4 <= 8 * kRowThreads) {
+        ffn_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+    } else if (aligned && n4 <= 12 * kRowThreads) {
+        ffn_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+    } else {
+        const size_t smem = (size_t)cols * sizeof(float);
+        static bool attr = false;
+        if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+        ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step);
+    }
     count_launch();
 }
 
