@@ -3,9 +3,9 @@
 // and the update of Eq. (2).  All kernels stream the fp32 masters once with
 // 16-byte accesses; the direction is regenerated in registers (rng.cuh).
 //
-// Thread mapping: a thread owns 4 consecutive elements (one Philox block), a
-// warp owns 128 consecutive elements = 128/group whole groups, so the group
-// min/max is a shuffle reduction over group/4 adjacent lanes.
+// Thread mapping of the operand producer: a thread owns 16 consecutive elements
+// (four Philox blocks), so a group is shared by group/16 adjacent lanes.  The
+// packing and update kernels map one Philox block (4 elements) to a thread.
 #include "common.cuh"
 #include "rng.cuh"
 
@@ -83,49 +83,105 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
     return r;
 }
 
+// Quantises the 16 values a thread holds (one (step, zero point) per group of LANES adjacent lanes) and returns
+// the dequantised values in place; codes (optional) receive the integer codes.
+//   code = clamp(round(x * inv) + zp, 0, qp),  value = (code - zp) * step
+// evaluated as value = clamp(round(x * inv), -zp, qp - zp) * step, which is the same number: all terms are
+// integers far below 2^24.  round() is to nearest even; when every |x * inv| of the warp is below 2^22 it is
+// taken by adding and subtracting 1.5 * 2^23 (exact for such values), otherwise by rintf.
+template <int LANES>
+__device__ __forceinline__ GroupQ quantise16(float (&x)[16], float qp, float* codes) {
+    float mn = x[0], mx = x[0];
+#pragma unroll
+    for (int j = 1; j < 16; ++j) { mn = fminf(mn, x[j]); mx = fmaxf(mx, x[j]); }
+    group_minmax<LANES>(mn, mx);
+    const GroupQ g = group_params(mn, mx, qp);
+    const float lo = -g.zp, hi = __fadd_rn(qp, -g.zp);
+    const bool small = __fmul_rn(fmaxf(fabsf(mn), fabsf(mx)), g.inv) < 4.0e6f;
+    if (__all_sync(0xffffffffu, small)) {
+        constexpr float kMagic = 12582912.0f;           // 1.5 * 2^23
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float r = __fadd_rn(__fadd_rn(__fmul_rn(x[j], g.inv), kMagic), -kMagic);
+            const float c = fminf(fmaxf(r, lo), hi);
+            if (codes) codes[j] = __fadd_rn(c, g.zp);
+            x[j] = __fmul_rn(c, g.step);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float c = fminf(fmaxf(rintf(__fmul_rn(x[j], g.inv)), lo), hi);
+            if (codes) codes[j] = __fadd_rn(c, g.zp);
+            x[j] = __fmul_rn(c, g.step);
+        }
+    }
+    return g;
+}
+
+__device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&x)[16]) {
+    const uint2 a = pack_bf16x4(x[0], x[1], x[2], x[3]), b = pack_bf16x4(x[4], x[5], x[6], x[7]);
+    const uint2 c = pack_bf16x4(x[8], x[9], x[10], x[11]), d = pack_bf16x4(x[12], x[13], x[14], x[15]);
+    dst[0] = make_uint4(a.x, a.y, b.x, b.y);
+    dst[1] = make_uint4(c.x, c.y, d.x, d.y);
+}
+
 // One pass over a tensor: perturb, quantise per group, write the bf16 operand(s).
-// GROUP in {32, 64, 128}; bits in {0 (no quantiser), 2, 3, 4}; DUAL writes the -eps operand too.
+// A thread owns 16 consecutive elements (four Philox blocks), so a group of GROUP elements spans GROUP/16
+// adjacent lanes: the group parameters are computed once per 16 elements and the min/max reduction takes
+// log2(GROUP/16) shuffle steps.  GROUP in {32, 64, 128}; bits in {0 (no quantiser), 2, 3, 4}; DUAL writes the
+// -eps operand too.
 template <int GROUP, bool DUAL, bool DEBUG>
 __global__ void __launch_bounds__(kThreads)
-weight_operand_kernel(const float4* __restrict__ w, int64_t n4, int bits, int perturb,
+weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int perturb,
                       uint32_t k0, uint32_t k1, uint32_t tid, float eps,
-                      uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
+                      uint4* __restrict__ op_plus, uint4* __restrict__ op_minus,
                       uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp) {
-    constexpr int LANES = GROUP / 4;
+    constexpr int LANES = GROUP / 16;
     const float qp = (float)((1 << bits) - 1);
     // whole warps iterate together so that the shuffles always see 32 lanes
-    const int64_t n4_ceil = (n4 + 31) & ~(int64_t)31;
-    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4_ceil; i += (int64_t)gridDim.x * blockDim.x) {
-        const bool live = i < n4;
-        float4 x = live ? __ldg(w + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        float4 xm = x;
+    const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n16_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n16;
+        float x[16], xm[16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float4 v = live ? __ldg(w + 4 * i + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+        }
         if (perturb) {
-            const float4 z = direction4(k0, k1, tid, (uint64_t)i);
-            if (DUAL) {
-                xm.x = __fmaf_rn(-eps, z.x, x.x); xm.y = __fmaf_rn(-eps, z.y, x.y);
-                xm.z = __fmaf_rn(-eps, z.z, x.z); xm.w = __fmaf_rn(-eps, z.w, x.w);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 z = direction4(k0, k1, tid, (uint64_t)(4 * i + k));
+                const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (DUAL) xm[4 * k + j] = __fmaf_rn(-eps, zz[j], x[4 * k + j]);
+                    x[4 * k + j] = __fmaf_rn(eps, zz[j], x[4 * k + j]);
+                }
             }
-            x.x = __fmaf_rn(eps, z.x, x.x); x.y = __fmaf_rn(eps, z.y, x.y);
-            x.z = __fmaf_rn(eps, z.z, x.z); x.w = __fmaf_rn(eps, z.w, x.w);
+        } else if (DUAL) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) xm[j] = x[j];
         }
         if (bits == 0) {
             if (live) {
-                op_plus[i] = pack_bf16x4(x.x, x.y, x.z, x.w);
-                if (DUAL) op_minus[i] = pack_bf16x4(xm.x, xm.y, xm.z, xm.w);
+                store_bf16x16(op_plus + 2 * i, x);
+                if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
             }
             continue;
         }
         {
-            float mn = fminf(fminf(x.x, x.y), fminf(x.z, x.w));
-            float mx = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
-            group_minmax<LANES>(mn, mx);
-            const GroupQ g = group_params(mn, mx, qp);
-            const float c0 = quant_code(x.x, g, qp), c1 = quant_code(x.y, g, qp);
-            const float c2 = quant_code(x.z, g, qp), c3 = quant_code(x.w, g, qp);
+            float cd[16];
+            const GroupQ g = quantise16<LANES>(x, qp, DEBUG ? cd : nullptr);
             if (live) {
-                op_plus[i] = pack_bf16x4(dequant(c0, g), dequant(c1, g), dequant(c2, g), dequant(c3, g));
+                store_bf16x16(op_plus + 2 * i, x);
                 if (DEBUG) {
-                    if (codes) codes[i] = make_uchar4((unsigned char)c0, (unsigned char)c1, (unsigned char)c2, (unsigned char)c3);
+                    if (codes) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            codes[4 * i + k] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
+                                                           (unsigned char)cd[4 * k + 2], (unsigned char)cd[4 * k + 3]);
+                    }
                     if ((i % LANES) == 0) {
                         if (step) step[i / LANES] = g.step;
                         if (zp) zp[i / LANES] = (int32_t)g.zp;
@@ -134,13 +190,8 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n4, int bits, int pe
             }
         }
         if (DUAL) {
-            float mn = fminf(fminf(xm.x, xm.y), fminf(xm.z, xm.w));
-            float mx = fmaxf(fmaxf(xm.x, xm.y), fmaxf(xm.z, xm.w));
-            group_minmax<LANES>(mn, mx);
-            const GroupQ g = group_params(mn, mx, qp);
-            const float c0 = quant_code(xm.x, g, qp), c1 = quant_code(xm.y, g, qp);
-            const float c2 = quant_code(xm.z, g, qp), c3 = quant_code(xm.w, g, qp);
-            if (live) op_minus[i] = pack_bf16x4(dequant(c0, g), dequant(c1, g), dequant(c2, g), dequant(c3, g));
+            quantise16<LANES>(xm, qp, nullptr);
+            if (live) store_bf16x16(op_minus + 2 * i, xm);
         }
     }
 }
@@ -238,20 +289,20 @@ template <int GROUP>
 static void weight_operand_dispatch(const float* w, int64_t n, int bits, int perturb, uint64_t seed, uint32_t tid,
                                     float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes,
                                     float* step, int32_t* zp, cudaStream_t s) {
-    const int64_t n4 = n / 4;
-    const int grid = stream_grid(n4, kThreads * 2);
+    const int64_t n16 = n / 16;
+    const int grid = stream_grid(n16, kThreads);
     const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
     const float4* w4 = reinterpret_cast<const float4*>(w);
-    uint2* p = reinterpret_cast<uint2*>(op_plus);
-    uint2* m = reinterpret_cast<uint2*>(op_minus);
+    uint4* p = reinterpret_cast<uint4*>(op_plus);
+    uint4* m = reinterpret_cast<uint4*>(op_minus);
     uchar4* c4 = reinterpret_cast<uchar4*>(codes);
     const bool debug = codes || step || zp;
     if (op_minus) {
-        weight_operand_kernel<GROUP, true, false><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr);
+        weight_operand_kernel<GROUP, true, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr);
     } else if (debug) {
-        weight_operand_kernel<GROUP, false, true><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp);
+        weight_operand_kernel<GROUP, false, true><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp);
     } else {
-        weight_operand_kernel<GROUP, false, false><<<grid, kThreads, 0, s>>>(w4, n4, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr);
+        weight_operand_kernel<GROUP, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr);
     }
     count_launch();
 }
