@@ -87,8 +87,10 @@ extern "C" {
 #define ZOQAT_TENSOR_FROZEN_PACKED  4u  /* Section 4.3: forward reads packed codes + (step, zero point) written by
                                            zoqat_prequantize_frozen(); never perturbed, never updated */
 
-#define ZOQAT_GEMM_TCGEN05 0   /* tcgen05/TMEM tensor-core kernel (default)                    */
-#define ZOQAT_GEMM_SIMT    1   /* plain CUDA-core kernel, kept as an on-device cross-check      */
+#define ZOQAT_GEMM_TCGEN05 0   /* tcgen05/TMEM tensor-core kernels (default); GEMM tiles of 256 rows are computed by a
+                                  pair of CTAs on two SMs with one cta_group::2 MMA                                  */
+#define ZOQAT_GEMM_SIMT    1   /* plain CUDA-core kernels, kept as an on-device cross-check                          */
+#define ZOQAT_GEMM_TCGEN05_1CTA 2 /* as 0, but every GEMM tile (128 rows) belongs to a single CTA                    */
 
 typedef struct zoqat_config {
     int32_t arch;          /* ZOQAT_ARCH_*                                                        */

@@ -18,7 +18,7 @@ ARCH_LLAMA, ARCH_OPT = 0, 1
  ROLE_FFN_NORM_G, ROLE_FFN_NORM_B, ROLE_BQ, ROLE_BK, ROLE_BV, ROLE_BO, ROLE_B_FC1, ROLE_B_FC2, ROLE_EMBED,
  ROLE_POS_EMBED, ROLE_FINAL_NORM_G, ROLE_FINAL_NORM_B, ROLE_LM_HEAD) = range(22)
 TENSOR_TRAINABLE, TENSOR_QUANTIZED, TENSOR_FROZEN_PACKED = 1, 2, 4
-GEMM_TCGEN05, GEMM_SIMT = 0, 1
+GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_1CTA = 0, 1, 2
 BUF_RESIDUAL, BUF_QKV, BUF_ATTN, BUF_FFN, BUF_TOKEN_LOSS = range(5)
 PROF_GEMM, PROF_WEIGHT, PROF_ACT, PROF_ATTENTION, PROF_LOSS, PROF_UPDATE = range(6)
 PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "update"]

@@ -126,7 +126,7 @@ int validate_config(const zoqat_config_t* c) {
     if (c->w_group != 32 && c->w_group != 64 && c->w_group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "w_group %d (supported: 32, 64, 128)", c->w_group);
     if (c->d_model % c->w_group || c->d_ffn % c->w_group) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
     if (c->a_bits != 0 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 8)", c->a_bits);
-    if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
+    if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT && c->gemm_impl != ZOQAT_GEMM_TCGEN05_1CTA) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
     if ((int64_t)c->max_batch * c->max_seq > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "max_batch*max_seq too large");
     return ZOQAT_OK;
 }
@@ -193,6 +193,7 @@ struct ProfScope {
 int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
     ProfScope ps(m, ZOQAT_PROF_GEMM, s);
     g.err_flag = m->ws.err_flag;
+    g.single_cta = m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = (m->cfg.gemm_impl == ZOQAT_GEMM_SIMT) ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "GEMM launch rejected (M=%lld N=%lld K=%lld)", (long long)g.M, (long long)g.N, (long long)g.K);
     return ZOQAT_OK;
@@ -728,6 +729,7 @@ int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, in
     g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
     g.M = M; g.N = N; g.K = K; g.Z = 1; g.row_step = row_step_dev; g.bias = bias_dev; g.relu = relu; g.accumulate = accumulate;
     g.out = out_dev; g.err_flag = err_flag_dev; g.b_stride = (size_t)N * K;
+    g.single_cta = impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, static_cast<cudaStream_t>(stream))
                                            : launch_gemm_tc(g, static_cast<cudaStream_t>(stream));
     if (rc != ZOQAT_OK) return fail(rc, "GEMM rejected: M=%lld N=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers, err flag for tcgen05)",
@@ -783,6 +785,7 @@ int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labe
     g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
     g.M = T; g.N = V; g.K = d; g.Z = 1; g.mode = 1; g.labels = labels_dev; g.partials = partials; g.label_logit = label_logit;
     g.err_flag = err_flag_dev; g.b_stride = (size_t)V * d;
+    g.single_cta = impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
     launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
@@ -845,6 +848,7 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
     g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
     g.M = T; g.N = V; g.K = d; g.Z = 1; g.mode = 1; g.labels = labels_dev; g.partials = partials; g.label_logit = label_logit;
     g.err_flag = err_flag_dev; g.b_stride = (size_t)V * d;
+    g.single_cta = impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
     launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);

@@ -68,6 +68,7 @@ struct GemmArgs {
     float2* partials;         // [Z*M, ce_tiles] (max, sum exp)
     float* label_logit;       // [Z*M]
     int32_t* err_flag;
+    int single_cta;           // tcgen05 kernel: 1 = one CTA per 128-row tile instead of a CTA pair per 256-row tile
 };
 int gemm_ce_tiles(int64_t N, int impl);                 // column tiles the cross-entropy epilogue produces
 int launch_gemm_simt(const GemmArgs& a, cudaStream_t s);   // returns 0 or a ZOQAT_ERR_* code

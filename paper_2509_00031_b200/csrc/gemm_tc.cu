@@ -29,10 +29,12 @@ constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kThreadsTC = 192;
 
-template <int BN> struct TileCfg {
-    static constexpr int kStages = (BN == 256) ? 4 : 6;
+// CG = CTAs per tile: 1, or 2 (a cluster of two CTAs on an SM pair computes a 256 x BN tile with one
+// cta_group::2 MMA; each CTA stages its 128 rows of A and its half of the B rows, so a stage is a third smaller).
+template <int BN, int CG> struct TileCfg {
+    static constexpr int kStages = (BN == 256 && CG == 1) ? 4 : 6;
     static constexpr int kABytes = BM * BK * 2;
-    static constexpr int kBBytes = BN * BK * 2;
+    static constexpr int kBBytes = (BN / CG) * BK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     // output staging for the TMA stores of the epilogue: two 32x32 fp32 boxes per epilogue warp
     static constexpr int kOutBoxBytes = 32 * 32 * 4;
@@ -41,13 +43,13 @@ template <int BN> struct TileCfg {
 };
 
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, both K-major.
-template <int BN>
+template <int BN, int CG>
 __device__ __forceinline__ uint32_t idesc_bf16() {
-    return (1u << 4)                      // D format: f32
-         | (1u << 7)                      // A format: bf16
-         | (1u << 10)                     // B format: bf16
-         | ((uint32_t)(BN >> 3) << 17)    // N / 8
-         | ((uint32_t)(BM >> 4) << 24);   // M / 16
+    return (1u << 4)                           // D format: f32
+         | (1u << 7)                           // A format: bf16
+         | (1u << 10)                          // B format: bf16
+         | ((uint32_t)(BN >> 3) << 17)         // N / 8
+         | ((uint32_t)((BM * CG) >> 4) << 24); // M / 16
 }
 
 __device__ __forceinline__ void ce_merge(float& m, float& s, float v) {
@@ -71,12 +73,16 @@ struct TcParams {
     int tma_out;              // 1: mode-0 results leave through map_out (needs N % 4 == 0)
 };
 
-template <int BN>
+template <int BN, int CG>
 __global__ void __launch_bounds__(kThreadsTC, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, TcParams p) {
-    using Cfg = TileCfg<BN>;
+    using Cfg = TileCfg<BN, CG>;
     constexpr int S = Cfg::kStages;
+    constexpr int TM = BM * CG;                                  // rows of a tile
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // CTA 0 of a pair leads: it issues the MMAs
+    const int unit = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_units = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;              // 1024-byte aligned stage ring
@@ -97,18 +103,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4 * CG); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
         if (p.tma_out) prefetch_tmap(&map_out);
     }
-    if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns
-        tmem_alloc(tmem_slot, 2 * BN);
-        tmem_relinquish();
+    if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns (in each CTA of a pair)
+        if (CG == 2) { tmem_alloc_pair(tmem_slot, 2 * BN); tmem_relinquish_pair(); }
+        else { tmem_alloc(tmem_slot, 2 * BN); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();      // the partner's barriers and TMEM are ready before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
@@ -117,15 +124,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = unit; t < total_tiles && ok; t += n_units) {
                 const int z = t / tiles_per_z, r = t % tiles_per_z;
                 const int tm = r % p.tiles_m, tn = r / p.tiles_m;     // m fastest: neighbours share B
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { atomicExch(p.err_flag, kErrWaitEmpty); ok = false; break; }
-                    mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
                     const uint32_t a_dst = tiles + stage * Cfg::kStageBytes;
-                    tma_load_3d(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z);
-                    tma_load_3d(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z);
+                    if (CG == 2) {
+                        // both CTAs' bytes are counted on the leader's barrier, which expects them all
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::kStageBytes);
+                        const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
+                        tma_load_3d_pair(a_dst, &map_a, lead_full, kb * BK, tm * TM + (int)rank * BM, z);
+                        tma_load_3d_pair(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, tn * BN + (int)rank * (BN / 2), z);
+                    } else {
+                        mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
+                        tma_load_3d(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z);
+                        tma_load_3d(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z);
+                    }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -139,12 +154,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t idesc = idesc_bf16<BN>();
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = idesc_bf16<BN, CG>();
             int stage = 0; uint32_t phase = 0;
             int acc = 0; uint32_t acc_phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = unit; t < total_tiles && ok; t += n_units) {
                 if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u)) { atomicExch(p.err_flag, kErrWaitAccEmpty); break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -157,14 +172,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         // advance 16 elements = 32 bytes inside the swizzled row: +2 in the (addr/16) field
-                        umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                        if (CG == 2) umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                                    (kb > 0 || k > 0) ? 1u : 0u);
+                        else umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                       (kb > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty_bar(stage));          // stage reusable once these MMAs have read it
+                    // stage reusable (in both CTAs of a pair) once these MMAs have read it
+                    if (CG == 2) umma_commit_pair(empty_bar(stage)); else umma_commit(empty_bar(stage));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(acc_full_bar(acc));             // accumulator complete
+                if (CG == 2) umma_commit_pair(acc_full_bar(acc)); else umma_commit(acc_full_bar(acc));   // accumulator complete
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -173,7 +191,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter+32)
         int acc = 0; uint32_t acc_phase = 0;
         int out_buf = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        for (int t = unit; t < total_tiles; t += n_units) {
             const int z = t / tiles_per_z, r = t % tiles_per_z;
             const int tm = r % p.tiles_m, tn = r / p.tiles_m;
             // the whole warp takes the same decision: the TMEM loads below are warp-collective
@@ -182,7 +200,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 break;
             }
             tc_fence_after();
-            const int64_t m = (int64_t)tm * BM + quarter * 32 + lane;
+            const int64_t m = (int64_t)tm * TM + rank * BM + quarter * 32 + lane;
             const bool row_ok = m < p.M;
             const int64_t row = (int64_t)z * p.M + (row_ok ? m : 0);
             const float rs = (p.row_step && row_ok) ? p.row_step[row] : 1.0f;
@@ -229,7 +247,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        const int y0 = tm * BM + quarter * 32;
+                        const int y0 = tm * TM + (int)rank * BM + quarter * 32;
                         if (p.accumulate) tma_reduce_add_3d(&map_out, box, (int)n0, y0, z);
                         else tma_store_3d(&map_out, box, (int)n0, y0, z);
                         bulk_commit();
@@ -280,7 +298,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // accumulator drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+            if (lane == 0) {
+                if (CG == 2) mbar_arrive_cluster(mapa_shared(acc_empty_bar(acc), 0));     // the leader issues the MMAs
+                else mbar_arrive(acc_empty_bar(acc));
+            }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait_all();      // every store / add issued by this warp has completed
@@ -288,10 +309,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    if (CG == 2) cluster_sync_all();      // neither CTA leaves (or frees TMEM) while its partner may still signal it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, 2 * BN);
+        if (CG == 2) tmem_dealloc_pair(tmem_base, 2 * BN); else tmem_dealloc(tmem_base, 2 * BN);
     }
 }
 
@@ -351,19 +373,19 @@ int num_sms() {
     return n;
 }
 
-template <int BN>
+template <int BN, int CG>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
-    using Cfg = TileCfg<BN>;
+    using Cfg = TileCfg<BN, CG>;
     alignas(64) CUtensorMap map_a, map_b, map_out;
     const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
-    if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN))
+    if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN / CG))
         return ZOQAT_ERR_CUDA;
     TcParams p;
     p.M = a.M; p.N = a.N; p.K = a.K; p.Z = a.Z;
     p.row_step = a.row_step; p.bias = a.bias; p.relu = a.relu; p.accumulate = a.accumulate;
     p.out = a.out; p.mode = a.mode; p.labels = a.labels; p.partials = a.partials; p.label_logit = a.label_logit;
     p.err_flag = a.err_flag;
-    p.tiles_m = (int)((a.M + BM - 1) / BM);
+    p.tiles_m = (int)((a.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((a.N + BN - 1) / BN);
     p.tma_out = (a.mode == 0 && a.N % 4 == 0) ? 1 : 0;
     if (p.tma_out) {
@@ -373,13 +395,24 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     }
     static bool attr = false;
     if (!attr) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
             return ZOQAT_ERR_CUDA;
         attr = true;
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
-    const int grid = (int)(total < num_sms() ? total : num_sms());
-    gemm_tc_kernel<BN><<<grid, kThreadsTC, Cfg::kSmemBytes, s>>>(map_a, map_b, map_out, p);
+    const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)
+    const int grid = (int)(total < units ? total : units) * CG;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kThreadsTC, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, CG>, map_a, map_b, map_out, p) != cudaSuccess) return ZOQAT_ERR_CUDA;
     count_launch();
     return ZOQAT_OK;
 }
@@ -393,8 +426,8 @@ int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
          reinterpret_cast<uintptr_t>(a.bias)) & 15)
         return ZOQAT_ERR_INVALID_ARG;
     // the cross-entropy epilogue always uses 256-column tiles (gemm_ce_tiles)
-    if (a.mode == 1 || a.N > 128) return launch_tc<256>(a, s);
-    return launch_tc<128>(a, s);
+    if (a.mode == 1 || a.N > 128) return a.single_cta ? launch_tc<256, 1>(a, s) : launch_tc<256, 2>(a, s);
+    return launch_tc<128, 1>(a, s);
 }
 
 }  // namespace zq
