@@ -14,17 +14,21 @@
 //   attn_prep_kernel   fp32 q|k|v -> rotary embedding, q * log2(e)/sqrt(d_head), hi/lo split;
 //                      q and k as [batch][head][seq][d_head], v transposed [batch][head][d_head][seq]
 //                      so that every tensor-core operand is K-major.
-//   attention_tc_kernel  persistent, one CTA per SM, 320 threads:
+//   attention_tc_kernel  persistent, one CTA per SM, 192 threads:
 //     warp 0     TMA producer: Q tile (128 queries) once per work item, then K / V^T tiles of 64 keys
 //                (hi and lo) into a two-stage ring.
 //     warp 1     MMA issuer: S_j = Q K_j^T (N = 64) into one of two TMEM score buffers - issued one
-//                tile ahead of the softmax - and O_j = P_j V_j (N = d_head).
-//     warps 2-9  softmax: two threads per query row (each half of the columns).  Read S_j from TMEM,
-//                running max / sum (base-2 exponentials), write P_j hi/lo to shared memory in the
-//                operand layout, and accumulate O_j from TMEM into registers with the usual
-//                rescaling; finally out = acc / sum.
-// Scores and probabilities never reach global memory.  Work items (query tile, head, batch) are
-// taken heaviest first.  Every wait is bounded and reports through *err_flag.
+//                tile ahead of the softmax - and O += P_j V_j (N = d_head), accumulated in TMEM over
+//                the whole work item.
+//     warps 2-5  softmax, one thread per query row: read S_j from TMEM, base-2 exponentials relative
+//                to a reference maximum, write P_j hi/lo to shared memory in the operand layout.  The
+//                reference only moves when the row maximum has grown by more than 2^8 since it was
+//                set (the normalisation by the running sum makes any reference exact); only then is
+//                the O accumulator rescaled in TMEM, so on almost every tile the softmax warps do not
+//                touch O at all.  At the end of the item: out = O / sum.
+// Scores and probabilities never reach global memory.  Work items are ordered in groups of 32
+// (batch, head) pairs - so that a group's K/V stays in L2 while its query tiles are processed - and,
+// inside a group, heaviest query tile first.  Every wait is bounded and reports through *err_flag.
 #include "common.cuh"
 #include "../../include/zoqat.h"
 #include "tc_ptx.cuh"
@@ -34,7 +38,8 @@ namespace zq {
 namespace {
 
 constexpr int BQ = 128, BKV = 64;
-constexpr int kAttThreadsTC = 320;
+constexpr int kAttThreadsTC = 192;
+constexpr float kRefSlack = 8.0f;      // the softmax reference may lag the row maximum by up to 2^8
 constexpr float kLoScale = 2048.0f, kLoInv = 1.0f / 2048.0f;
 constexpr int kErrAttnSmem = 16;       // dynamic shared memory window too small after alignment
 constexpr int kErrAttnWait = 17;       // a bounded wait of the attention kernel ran out
@@ -47,12 +52,11 @@ template <int D> struct AttCfg {
     static constexpr int kPBytes = BQ * BKV * 2;          // one of Ph / Pl
     static constexpr int kOffStage = 2 * kQBytes;
     static constexpr int kOffP = kOffStage + kStages * kStageBytes;
-    static constexpr int kOffX = kOffP + 2 * kPBytes;     // row-max exchange: [2 slots][128 rows][2 halves] floats
-    static constexpr int kOffBar = kOffX + 2048;
+    static constexpr int kOffBar = kOffP + 2 * kPBytes;
     static constexpr int kUsedBytes = kOffBar + 160;      // 18 mbarriers + the TMEM base word
-    // Request the whole opt-in window for d_head 128 (the tiles need all but ~860 bytes of it) and enough to
-    // keep a second CTA off the SM for d_head 64 (a CTA owns all 512 TMEM columns).
-    static constexpr int kSmemBytes = (D == 128) ? 232448 : (kUsedBytes + 1024 > 120 * 1024 ? kUsedBytes + 1024 : 120 * 1024);
+    // 1 KB of slack for the 1024-byte alignment of the tiles; at least 120 KB so that a second CTA stays off
+    // the SM for d_head 64 (a CTA owns all 512 TMEM columns).
+    static constexpr int kSmemBytes = kUsedBytes + 1024 > 120 * 1024 ? kUsedBytes + 1024 : 120 * 1024;
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -60,6 +64,20 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+// 32 lanes x 32 consecutive fp32 columns back into TMEM: thread = lane (row), v[j] = column j.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] * B[smem]^T, fp16 x fp16 -> fp32, one CTA.
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -180,15 +198,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
     const uint32_t bars = base + Cfg::kOffBar;
     // barriers (8 bytes each)
     const uint32_t q_full = bars, q_empty = bars + 8;
-    auto kv_full = [&](int s) { return bars + 16u + 8u * s; };
-    auto kv_empty = [&](int s) { return bars + 32u + 8u * s; };
+    // K and V of a stage have their own barriers: a K tile is free as soon as its S product has completed, long
+    // before the stage's V tile, so the next K load starts a whole tile earlier
+    auto k_full = [&](int s) { return bars + 16u + 8u * s; };
+    auto k_empty = [&](int s) { return bars + 32u + 8u * s; };
+    auto v_full = [&](int s) { return bars + 120u + 8u * s; };
+    auto v_empty = [&](int s) { return bars + 136u + 8u * s; };
     auto s_full = [&](int b) { return bars + 48u + 8u * b; };
     auto s_empty = [&](int b) { return bars + 64u + 8u * b; };
     const uint32_t p_full = bars + 80, p_empty = bars + 88, o_full = bars + 96, o_empty = bars + 104;
-    auto x_bar = [&](int q) { return bars + 112u + 8u * q; };
-    const uint32_t tmem_slot = bars + 144;
+    const uint32_t tmem_slot = bars + 112;
     uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - raw));
-    float* xchg = reinterpret_cast<float*>(smem_raw + (base + Cfg::kOffX - raw));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (!smem_ok) {                              // uniform over the CTA: nothing has been set up yet
@@ -197,9 +217,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
     }
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(kv_full(s), 1); mbar_init(kv_empty(s), 1); mbar_init(s_full(s), 1); mbar_init(s_empty(s), 8); }
-        mbar_init(p_full, 8); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 8);
-        for (int q = 0; q < 4; ++q) mbar_init(x_bar(q), 2);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1);
+            mbar_init(s_full(s), 1); mbar_init(s_empty(s), 4);
+        }
+        mbar_init(p_full, 4); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_qh); prefetch_tmap(&map_ql); prefetch_tmap(&map_kh);
         prefetch_tmap(&map_kl); prefetch_tmap(&map_vth); prefetch_tmap(&map_vtl);
@@ -214,42 +236,78 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
     const uint32_t tmem_base = *tmem_slot_ptr;
 
     const int HB = p.n_heads * p.batch;
-    // work item -> (query tile, batch*head); heaviest (latest) query tiles first
-    auto item_qt = [&](int it) { return p.n_qt - 1 - it / HB; };
-    auto item_bh = [&](int it) { return it % HB; };
+    // work item -> (query tile, batch*head): groups of up to 32 (batch, head) pairs; inside a group the heaviest
+    // (latest) query tiles first
+    constexpr int kGroup = 32;
+    const int per_group = kGroup * p.n_qt;
+    auto item_qt = [&](int it) {
+        const int g = it / per_group, r = it - g * per_group;
+        const int gsz = min(kGroup, HB - g * kGroup);
+        return p.n_qt - 1 - r / gsz;
+    };
+    auto item_bh = [&](int it) {
+        const int g = it / per_group, r = it - g * per_group;
+        const int gsz = min(kGroup, HB - g * kGroup);
+        return g * kGroup + r % gsz;
+    };
     auto n_kv_tiles = [&](int qt) { const int hi_ = min(p.seq, (qt + 1) * BQ); return (hi_ + BKV - 1) / BKV; };
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            uint32_t kv_it = 0, q_it = 0;
+            // Two cursors walk the same sequence of (item, key tile): the K cursor runs one tile ahead of the V
+            // cursor, in the order the tensor pipe releases the slots (S_g completes before P V of tile g - 1).
+            struct Cursor { int it, j, n, bh; uint32_t g; };
+            auto start = [&](Cursor& c, int it) {
+                c.it = it; c.j = 0;
+                if (it < p.total_items) { c.n = n_kv_tiles(item_qt(it)); c.bh = item_bh(it); }
+            };
+            auto advance = [&](Cursor& c) { ++c.g; if (++c.j == c.n) start(c, c.it + (int)gridDim.x); };
+            Cursor kc, vc;
+            kc.g = vc.g = 0;
+            start(kc, blockIdx.x);
+            start(vc, blockIdx.x);
+            uint32_t q_it = 0;
             bool ok = true;
-            for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
-                const int qt = item_qt(it), bh = item_bh(it), n = n_kv_tiles(qt);
-                if (!mbar_wait(q_empty, (q_it & 1u) ^ 1u)) { atomicExch(p.err_flag, kErrAttnWait); ok = false; break; }
-                mbar_arrive_expect_tx(q_full, 2 * Cfg::kQBytes);
+            while (ok && vc.it < p.total_items) {
+                while (ok && kc.it < p.total_items && kc.g <= vc.g + 1) {
+                    if (kc.j == 0) {                   // first tile of an item: its Q tile
+                        if (!mbar_wait(q_empty, (q_it & 1u) ^ 1u)) { ok = false; break; }
+                        ++q_it;
+                        const int qt = item_qt(kc.it);
+                        mbar_arrive_expect_tx(q_full, 2 * Cfg::kQBytes);
 #pragma unroll
-                for (int sub = 0; sub < KSUB; ++sub) {
-                    tma_load_3d(base + sub * (BQ * 128), &map_qh, q_full, sub * 64, qt * BQ, bh);
-                    tma_load_3d(base + Cfg::kQBytes + sub * (BQ * 128), &map_ql, q_full, sub * 64, qt * BQ, bh);
-                }
-                for (int j = 0; j < n; ++j, ++kv_it) {
-                    const int st = kv_it & 1u;
-                    if (!mbar_wait(kv_empty(st), ((kv_it >> 1) & 1u) ^ 1u)) { atomicExch(p.err_flag, kErrAttnWait); ok = false; break; }
-                    mbar_arrive_expect_tx(kv_full(st), Cfg::kStageBytes);
+                        for (int sub = 0; sub < KSUB; ++sub) {
+                            tma_load_3d(base + sub * (BQ * 128), &map_qh, q_full, sub * 64, qt * BQ, kc.bh);
+                            tma_load_3d(base + Cfg::kQBytes + sub * (BQ * 128), &map_ql, q_full, sub * 64, qt * BQ, kc.bh);
+                        }
+                    }
+                    const int st = kc.g & 1u;
+                    if (!mbar_wait(k_empty(st), ((kc.g >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                    mbar_arrive_expect_tx(k_full(st), 2 * Cfg::kKBytes);
                     const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
 #pragma unroll
                     for (int sub = 0; sub < KSUB; ++sub) {
-                        tma_load_3d(sb + sub * (BKV * 128), &map_kh, kv_full(st), sub * 64, j * BKV, bh);
-                        tma_load_3d(sb + Cfg::kKBytes + sub * (BKV * 128), &map_kl, kv_full(st), sub * 64, j * BKV, bh);
+                        tma_load_3d(sb + sub * (BKV * 128), &map_kh, k_full(st), sub * 64, kc.j * BKV, kc.bh);
+                        tma_load_3d(sb + Cfg::kKBytes + sub * (BKV * 128), &map_kl, k_full(st), sub * 64, kc.j * BKV, kc.bh);
                     }
-                    tma_load_3d(sb + 2 * Cfg::kKBytes, &map_vth, kv_full(st), j * BKV, 0, bh);
-                    tma_load_3d(sb + 3 * Cfg::kKBytes, &map_vtl, kv_full(st), j * BKV, 0, bh);
+                    advance(kc);
                 }
+                if (!ok) break;
+                const int st = vc.g & 1u;
+                if (!mbar_wait(v_empty(st), ((vc.g >> 1) & 1u) ^ 1u)) { ok = false; break; }
+                mbar_arrive_expect_tx(v_full(st), 2 * Cfg::kKBytes);
+                const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
+                tma_load_3d(sb + 2 * Cfg::kKBytes, &map_vth, v_full(st), vc.j * BKV, 0, vc.bh);
+                tma_load_3d(sb + 3 * Cfg::kKBytes, &map_vtl, v_full(st), vc.j * BKV, 0, vc.bh);
+                advance(vc);
             }
+            if (!ok) atomicExch(p.err_flag, kErrAttnWait);
             // every load issued above has to land before the CTA may leave
-            for (int i = 0; i < 2 && ok; ++i, ++kv_it)
-                if (!mbar_wait(kv_empty(kv_it & 1u), ((kv_it >> 1) & 1u) ^ 1u)) break;
+            for (int i = 0; i < 2 && ok; ++i) {
+                if (!mbar_wait(k_empty((kc.g + i) & 1u), (((kc.g + i) >> 1) & 1u) ^ 1u)) break;
+                if (!mbar_wait(v_empty((vc.g + i) & 1u), (((vc.g + i) >> 1) & 1u) ^ 1u)) break;
+            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
@@ -260,7 +318,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
             // S of global tile g (stage / score buffer g & 1)
             auto issue_s = [&](uint32_t g) -> bool {
                 const int st = g & 1u;
-                if (!mbar_wait(kv_full(st), (g >> 1) & 1u)) return false;
+                if (!mbar_wait(k_full(st), (g >> 1) & 1u)) return false;
                 if (!mbar_wait(s_empty(st), ((g >> 1) & 1u) ^ 1u)) return false;
                 tc_fence_after();
                 const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
@@ -283,6 +341,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                     umma_f16(d_corr, aql, bkh, idesc_s, 1u);
                 }
                 umma_commit(s_full(st));
+                umma_commit(k_empty(st));          // the K tile is free once these products have completed
                 return true;
             };
             for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
@@ -290,14 +349,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 if (!mbar_wait(q_full, q_it & 1u)) { ok = false; break; }
                 if (!issue_s(kv_it)) { ok = false; break; }
                 if (n == 1) umma_commit(q_empty);
+                // the O accumulators are free once the softmax warps have read out the previous item
+                if (!mbar_wait(o_empty, (q_it & 1u) ^ 1u)) { ok = false; break; }
                 for (int j = 0; j < n; ++j, ++t_it) {
                     if (j + 1 < n) {
                         if (!issue_s(kv_it + j + 1)) { ok = false; break; }
                         if (j + 2 == n) umma_commit(q_empty);     // Q is free once the last S of the item has completed
                     }
-                    if (!mbar_wait(p_full, t_it & 1u) || !mbar_wait(o_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
-                    tc_fence_after();
                     const int st = (kv_it + j) & 1u;
+                    if (!mbar_wait(p_full, t_it & 1u) ||                         // P_j stored (and O rescaled if needed)
+                        !mbar_wait(v_full(st), ((kv_it + j) >> 1) & 1u)) { ok = false; break; }
+                    tc_fence_after();
                     const uint32_t sb = base + Cfg::kOffStage + st * Cfg::kStageBytes;
                     const uint32_t ph = base + Cfg::kOffP, pl = ph + Cfg::kPBytes;
                     const uint32_t o_main = tmem_base + 256u, o_corr = tmem_base + 384u;
@@ -305,7 +367,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                     for (int k = 0; k < BKV / 16; ++k) {
                         const uint64_t aph = smem_desc_sw128(ph) + (uint64_t)(2 * k);
                         const uint64_t bvh = smem_desc_sw128(sb + 2 * Cfg::kKBytes) + (uint64_t)(2 * k);
-                        umma_f16(o_main, aph, bvh, idesc_o, k > 0 ? 1u : 0u);
+                        umma_f16(o_main, aph, bvh, idesc_o, (j > 0 || k > 0) ? 1u : 0u);
                     }
 #pragma unroll
                     for (int k = 0; k < BKV / 16; ++k) {
@@ -313,11 +375,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                         const uint64_t apl = smem_desc_sw128(pl) + (uint64_t)(2 * k);
                         const uint64_t bvh = smem_desc_sw128(sb + 2 * Cfg::kKBytes) + (uint64_t)(2 * k);
                         const uint64_t bvl = smem_desc_sw128(sb + 3 * Cfg::kKBytes) + (uint64_t)(2 * k);
-                        umma_f16(o_corr, aph, bvl, idesc_o, k > 0 ? 1u : 0u);
+                        umma_f16(o_corr, aph, bvl, idesc_o, (j > 0 || k > 0) ? 1u : 0u);
                         umma_f16(o_corr, apl, bvh, idesc_o, 1u);
                     }
                     umma_commit(o_full);
-                    umma_commit(kv_empty(st));
+                    umma_commit(v_empty(st));
                     umma_commit(p_empty);
                 }
                 kv_it += n;
@@ -325,91 +387,84 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
             if (!ok) atomicExch(p.err_flag, kErrAttnWait);
         }
     } else {
-        // ---------------- softmax / output warps (2..9) ----------------
+        // ---------------- softmax / output warps (2..5), one thread per query row ----------------
         const int quarter = warp & 3;                       // TMEM lanes [32*quarter, 32*quarter + 32)
-        const int half = (warp - 2) >> 2;                   // which half of the columns
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int d_model = p.n_heads * D;
-        uint32_t s_it = 0, t_it = 0, x_it = 0;
+        uint32_t s_it = 0, t_it = 0, q_it = 0;
         bool ok = true;
         // wait helper: the whole warp takes the same decision
         auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)) != 0; };
-        for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x) {
+        for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
             const int qt = item_qt(it), bh = item_bh(it), n = n_kv_tiles(qt);
             const int qpos = qt * BQ + row;
-            float m_run = -INFINITY, l_run = 0.0f, corr_prev = 1.0f;
-            float acc[DH];
-#pragma unroll
-            for (int c = 0; c < DH; ++c) acc[c] = 0.0f;
+            float m_ref = -INFINITY, l_run = 0.0f;
 
-            // acc <- acc * corr_prev + (O_main + 2^-11 O_corr) of the previous tile, then release the O buffer
-            auto take_o = [&]() -> bool {
-                if (!wait_all(o_full, (t_it & 1u) ^ 1u)) return false;     // tile t_it - 1
-                tc_fence_after();
-#pragma unroll
-                for (int c0 = 0; c0 < DH; c0 += 32) {
-                    uint32_t om[32], oc[32];
-                    tmem_ld32(t_lane + 256u + (uint32_t)(half * DH + c0), om);
-                    tmem_ld32(t_lane + 384u + (uint32_t)(half * DH + c0), oc);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        acc[c0 + c] = fmaf(acc[c0 + c], corr_prev, fmaf(__uint_as_float(oc[c]), kLoInv, __uint_as_float(om[c])));
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_empty);
-                return true;
-            };
-
-            for (int j = 0; j < n; ++j, ++s_it, ++t_it, ++x_it) {
+            for (int j = 0; j < n; ++j, ++s_it, ++t_it) {
                 const int sbuf = s_it & 1u;
                 if (!wait_all(s_full(sbuf), (s_it >> 1) & 1u)) { ok = false; break; }
                 tc_fence_after();
-                float s[32];
-                {
+                float s[BKV];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
                     uint32_t sm[32], sc[32];
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + half * 32), sm);
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64 + half * 32), sc);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + h * 32), sm);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64 + h * 32), sc);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) s[c] = fmaf(__uint_as_float(sc[c]), kLoInv, __uint_as_float(sm[c]));
+                    for (int c = 0; c < 32; ++c) s[h * 32 + c] = fmaf(__uint_as_float(sc[c]), kLoInv, __uint_as_float(sm[c]));
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty(sbuf));
                 // causal mask (keys beyond the sequence end are beyond every valid query as well)
-                const int k0 = j * BKV + half * 32;
                 if (j * BKV + BKV - 1 > qt * BQ) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (k0 + c > qpos) s[c] = -INFINITY;
+                    for (int c = 0; c < BKV; ++c)
+                        if (j * BKV + c > qpos) s[c] = -INFINITY;
                 }
                 float mx = s[0];
 #pragma unroll
-                for (int c = 1; c < 32; ++c) mx = fmaxf(mx, s[c]);
-                // exchange the half-row maxima with the partner warp of this quarter
-                xchg[((x_it & 1u) * BQ + row) * 2 + half] = mx;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(x_bar(quarter));
-                if (!wait_all(x_bar(quarter), x_it & 1u)) { ok = false; break; }
-                mx = fmaxf(mx, xchg[((x_it & 1u) * BQ + row) * 2 + (half ^ 1)]);
-                const float m_new = fmaxf(m_run, mx);         // finite: key 0 is visible to every query
-                const float corr = ex2(m_run - m_new);
+                for (int c = 1; c < BKV; ++c) mx = fmaxf(mx, s[c]);
+                if (j == 0) {
+                    m_ref = mx;                                   // finite: key 0 is visible to every query; O is still empty
+                } else {
+                    const bool grow = mx > m_ref + kRefSlack;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        // rare: move the reference of the rows that need it and rescale their O rows in TMEM,
+                        // after the previous tile's P V has completed and before this tile's is issued
+                        if (!wait_all(o_full, (t_it & 1u) ^ 1u)) { ok = false; break; }
+                        tc_fence_after();
+                        const float f = grow ? ex2(m_ref - mx) : 1.0f;
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+#pragma unroll 1
+                            for (int part = 0; part < 2; ++part) {
+                                uint32_t o[32];
+                                const uint32_t addr = t_lane + (part == 0 ? 256u : 384u) + (uint32_t)c0;
+                                tmem_ld32(addr, o);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                                tmem_st32(addr, o);
+                            }
+                        }
+                        tmem_st_wait();
+                        tc_fence_before();
+                        l_run *= f;
+                        if (grow) m_ref = mx;
+                    }
+                }
                 float rs = 0.0f;
 #pragma unroll
-                for (int c = 0; c < 32; ++c) { s[c] = ex2(s[c] - m_new); rs += s[c]; }
-                l_run = fmaf(l_run, corr, rs);
-                m_run = m_new;
-                // O of the previous tile (frees the O accumulators for this tile's P V)
-                if (j > 0 && !take_o()) { ok = false; break; }
-                corr_prev = corr;
+                for (int c = 0; c < BKV; ++c) { s[c] = ex2(s[c] - m_ref); rs += s[c]; }
+                l_run += rs;
                 // P -> shared memory (operand layout: 128-byte rows, 16-byte chunks XOR-swizzled by row)
                 if (!wait_all(p_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
                 const uint32_t ph = base + Cfg::kOffP + (uint32_t)(row * 128), pl = ph + Cfg::kPBytes;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < 8; ++i) {
                     uint32_t wh[4], wl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -420,7 +475,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                         wh[e] = *reinterpret_cast<const uint32_t*>(&h2);
                         wl[e] = *reinterpret_cast<const uint32_t*>(&l2);
                     }
-                    const uint32_t chunk = (uint32_t)(((half * 4 + i) ^ (row & 7)) << 4);
+                    const uint32_t chunk = (uint32_t)((i ^ (row & 7)) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ph + chunk), "r"(wh[0]), "r"(wh[1]), "r"(wh[2]), "r"(wh[3]) : "memory");
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pl + chunk), "r"(wl[0]), "r"(wl[1]), "r"(wl[2]), "r"(wl[3]) : "memory");
                 }
@@ -429,22 +484,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 if (lane == 0) mbar_arrive(p_full);
             }
             if (!ok) break;
-            if (!take_o()) { ok = false; break; }             // the last tile of the item
-            // total row sum = both halves
-            xchg[((x_it & 1u) * BQ + row) * 2 + half] = l_run;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(x_bar(quarter));
-            if (!wait_all(x_bar(quarter), x_it & 1u)) { ok = false; break; }
-            const float l_tot = l_run + xchg[((x_it & 1u) * BQ + row) * 2 + (half ^ 1)];
-            ++x_it;
-            if (qpos < p.seq) {
-                const float inv = 1.0f / l_tot;
-                const int b = bh / p.n_heads, head = bh % p.n_heads;
-                float* dst = p.out + ((int64_t)b * p.seq + qpos) * d_model + head * D + half * DH;
+            // the item's last P V has completed: out = (O_main + 2^-11 O_corr) / sum
+            if (!wait_all(o_full, (t_it & 1u) ^ 1u)) { ok = false; break; }
+            tc_fence_after();
+            const float inv = 1.0f / l_run;
+            const int b = bh / p.n_heads, head = bh % p.n_heads;
+            float* dst = p.out + ((int64_t)b * p.seq + qpos) * d_model + head * D;
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                uint32_t om[32], oc[32];
+                tmem_ld32(t_lane + 256u + (uint32_t)c0, om);
+                tmem_ld32(t_lane + 384u + (uint32_t)c0, oc);
+                tmem_ld_wait();
+                if (qpos < p.seq) {
 #pragma unroll
-                for (int c = 0; c < DH; c += 4)
-                    *reinterpret_cast<float4*>(dst + c) = make_float4(acc[c] * inv, acc[c + 1] * inv, acc[c + 2] * inv, acc[c + 3] * inv);
+                    for (int c = 0; c < 32; c += 4) {
+                        float4 v;
+                        v.x = fmaf(__uint_as_float(oc[c]), kLoInv, __uint_as_float(om[c])) * inv;
+                        v.y = fmaf(__uint_as_float(oc[c + 1]), kLoInv, __uint_as_float(om[c + 1])) * inv;
+                        v.z = fmaf(__uint_as_float(oc[c + 2]), kLoInv, __uint_as_float(om[c + 2])) * inv;
+                        v.w = fmaf(__uint_as_float(oc[c + 3]), kLoInv, __uint_as_float(om[c + 3])) * inv;
+                        *reinterpret_cast<float4*>(dst + c0 + c) = v;
+                    }
+                }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(o_empty);
         }
         if (!ok && lane == 0) atomicExch(p.err_flag, kErrAttnWait);
     }
