@@ -23,9 +23,10 @@ if ROOT not in sys.path:
 METRIC = "ZO-QAT steps/s & fwd tokens/s, 7B-shape W4A8, 1 B200; % of roofline"
 UNIT = "steps/s"
 EPS, LR = 1e-3, 1e-6
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel from the committed ncu
-# capture (profiles/), keyed by workload; None until a capture exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, averaged over the 129 GEMM
+# launches of one step, from the committed ncu capture (profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by
+# workload; absent for workloads that have not been captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 946.5e6}
 
 
 def load_peaks():
@@ -84,7 +85,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
@@ -94,12 +95,16 @@ class ClockSampler:
                 sm.append(float(f[0])); mx.append(float(f[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(f[2]))
+            except ValueError:
+                pass
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        sm.sort()
+        sm.sort(); pw.sort()
         return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=sorted(reasons), samples=len(sm))
+                    power_w=pw[len(pw) // 2] if pw else None, reasons=sorted(reasons), samples=len(sm))
 
 
 # ---------------------------------------------------------------------------------------------
