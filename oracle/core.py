@@ -25,9 +25,10 @@ def lib():
         L.zq_update.argtypes = [vp, u64, u64, u32, f32]
         L.zq_weight_quant.argtypes = [vp, i64, i64, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp]
         L.zq_round_bf16.argtypes = [vp, u64, vp]
-        L.zq_box_muller.argtypes = [u32, u32, vp, vp]
+        L.zq_gauss_words.argtypes = [vp, u64, vp]
+        L.zq_icdf_table.argtypes = [vp, vp]
         for name in ("zq_philox_words", "zq_normal_fill", "zq_perturb", "zq_update",
-                     "zq_weight_quant", "zq_round_bf16", "zq_box_muller"):
+                     "zq_weight_quant", "zq_round_bf16", "zq_gauss_words", "zq_icdf_table"):
             getattr(L, name).restype = None
         _lib = L
     return _lib
@@ -51,11 +52,20 @@ def normal(seed, tensor_id, n):
     return z
 
 
-def box_muller(w0, w1):
-    a = np.zeros(1, np.float32)
-    b = np.zeros(1, np.float32)
-    lib().zq_box_muller(int(w0), int(w1), _ptr(a), _ptr(b))
-    return float(a[0]), float(b[0])
+def gauss_from_words(words):
+    """One standard normal per 32-bit word (the table-driven inverse distribution function): float32, same shape."""
+    w = np.ascontiguousarray(words, dtype=np.uint32)
+    z = np.empty(w.shape, np.float32)
+    lib().zq_gauss_words(_ptr(w), w.size, _ptr(z))
+    return z
+
+
+def icdf_table():
+    """The generator's knot table: (base, slope), 2048 float32 each."""
+    base = np.empty(2048, np.float32)
+    slope = np.empty(2048, np.float32)
+    lib().zq_icdf_table(_ptr(base), _ptr(slope))
+    return base, slope
 
 
 def perturb(w, seed, tensor_id, signed_eps):

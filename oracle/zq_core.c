@@ -18,19 +18,23 @@
  * (build with -ffp-contract=off).
  *
  * The direction generator (the paper only says u_i ~ N(0, I), Eq. (1)):
- *   words   = Philox4x32-10(counter = (blk_lo, blk_hi, tensor_id, 0),
- *                           key = (seed_lo, seed_hi)),  blk = index / 4
- *   (z[4blk], z[4blk+1]) = BoxMuller(words[0], words[1])
- *   (z[4blk+2], z[4blk+3]) = BoxMuller(words[2], words[3])
- * Box-Muller in binary32:
- *   radius: a = 2*(w0 >> 9) + 1 (odd, < 2^24, exact in binary32), u = a*2^-24,
- *           ln u = (e-24)*ln2 + ln m with a = m*2^e, m folded into
- *           (sqrt(1/2), sqrt 2], ln m = 2 s (1 + s^2/3 + s^4/5 + s^6/7 + s^8/9),
- *           s = (m-1)/(m+1);  r = sqrt(-2 ln u)
- *   angle:  phi = (2*((w1 >> 6) & 0x7fffff) + 1) * 2^-24 * pi/4 in (0, pi/4),
- *           sin/cos by their Taylor polynomials (through phi^9 and phi^8); the
- *           top three bits of w1 pick the octant (swap sin/cos, negate first,
- *           negate second), which maps the first octant onto the whole circle.
+ *   words = Philox4x32-10(counter = (blk_lo, blk_hi, tensor_id, 0),
+ *                         key = (seed_lo, seed_hi)),  blk = index / 4
+ *   z[4blk + j] = G(words[j]),  j = 0..3
+ * G is the inverse of the Gaussian distribution function applied to the word,
+ * evaluated by a piecewise-linear table so that every machine reproduces it bit
+ * for bit with a handful of integer operations and one fused multiply-add:
+ *   sign = w >> 31;  v = 2^31 - (w & 0x7fffffff)  in [1, 2^31]
+ *   |z| is the upper quantile of the half-normal at tail probability v / 2^31,
+ *         Q(v) = Phi^-1(1 - v / 2^32),
+ *   interpolated linearly in v between the knots v = 2^E (1 + j/64), E = 0..31,
+ *   j = 0..63 (64 knots per octave of the tail probability, so the tail is
+ *   resolved as finely, in relative terms, as the centre; largest |z| = 6.23).
+ *   f = (float)v (round to nearest); the knot index is the exponent and the top
+ *   six mantissa bits of f, the offset inside the segment its low 17 bits:
+ *   |z| = fmaf(offset, slope[idx], base[idx]).
+ * The knots are float roundings of Q computed in double by bisection on erfc().
+ * Interpolation error is below 3e-5 everywhere (tests pin it).
  */
 #include <math.h>
 #include <stdint.h>
@@ -62,45 +66,71 @@ void zq_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out
 static float bits_to_float(uint32_t b) { float f; memcpy(&f, &b, 4); return f; }
 static uint32_t float_to_bits(float f) { uint32_t b; memcpy(&b, &f, 4); return b; }
 
-/* One Box-Muller pair from two 32-bit words, binary32 throughout. */
-void zq_box_muller(uint32_t w0, uint32_t w1, float *za, float *zb)
+/* ---- table of the inverse Gaussian distribution function --------------------- */
+#define ZQ_ICDF_KNOTS (32 * 64)
+static float zq_icdf_base[ZQ_ICDF_KNOTS];
+static float zq_icdf_slope[ZQ_ICDF_KNOTS];
+static int zq_icdf_ready = 0;
+
+/* z >= 0 with 1 - Phi(z) = q for 0 < q < 1/2 (0 for q >= 1/2): bisection on
+ * 1 - Phi(z) = erfc(z / sqrt 2) / 2, which is decreasing in z. */
+static double zq_upper_quantile(double q)
 {
-    /* radius */
-    float a = (float)(2u * (w0 >> 9) + 1u);           /* odd integer < 2^24: exact */
-    uint32_t ab = float_to_bits(a);
-    int e = (int)(ab >> 23) - 127;                      /* a = m * 2^e, m in [1,2) */
-    float m = bits_to_float((ab & 0x007FFFFFu) | 0x3F800000u);
-    if (m > 1.41421354f) { m = m * 0.5f; e += 1; }     /* m in (sqrt(1/2), sqrt 2] */
-    float s = (m - 1.0f) / (m + 1.0f);
-    float s2 = s * s;
-    float p = fmaf(s2, 1.0f / 9.0f, 1.0f / 7.0f);
-    p = fmaf(p, s2, 1.0f / 5.0f);
-    p = fmaf(p, s2, 1.0f / 3.0f);
-    p = fmaf(p, s2, 1.0f);
-    float lnm = (2.0f * s) * p;
-    float lnu = fmaf((float)(e - 24), 0.693147182f, lnm);   /* ln(a * 2^-24) <= 0 */
-    float r = sqrtf(-2.0f * lnu);
-    /* angle in the first octant */
-    float f = (float)(2u * ((w1 >> 6) & 0x7FFFFFu) + 1u);   /* odd integer < 2^24 */
-    float phi = f * (0.785398185f * 5.9604644775390625e-08f); /* * pi/4 * 2^-24 */
-    float y = phi * phi;
-    float sp = fmaf(y, 1.0f / 362880.0f, -1.0f / 5040.0f);
-    sp = fmaf(sp, y, 1.0f / 120.0f);
-    sp = fmaf(sp, y, -1.0f / 6.0f);
-    sp = fmaf(sp, y, 1.0f);
-    float sn = phi * sp;
-    float cs = fmaf(y, 1.0f / 40320.0f, -1.0f / 720.0f);
-    cs = fmaf(cs, y, 1.0f / 24.0f);
-    cs = fmaf(cs, y, -0.5f);
-    cs = fmaf(cs, y, 1.0f);
-    /* octant: bit 29 swaps, bit 30 negates the first, bit 31 the second */
-    uint32_t oct = w1 >> 29;
-    float first = (oct & 1u) ? sn : cs;
-    float second = (oct & 1u) ? cs : sn;
-    if (oct & 2u) first = -first;
-    if (oct & 4u) second = -second;
-    *za = r * first;
-    *zb = r * second;
+    if (q >= 0.5) return 0.0;
+    double lo = 0.0, hi = 8.0;
+    for (int it = 0; it < 200; ++it) {
+        double mid = 0.5 * (lo + hi);
+        double tail = 0.5 * erfc(mid * 0.70710678118654752440);
+        if (tail > q) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+static double zq_knot(int k)      /* Q at v = 2^E (1 + j/64), k = 64 E + j (k may be 2048) */
+{
+    int e = k >> 6, j = k & 63;
+    double v = ldexp(1.0 + (double)j / 64.0, e);
+    return zq_upper_quantile(v / 4294967296.0);
+}
+
+void zq_icdf_init(void)
+{
+#pragma omp critical(zq_icdf_table)
+    {
+        if (!zq_icdf_ready) {
+            for (int k = 0; k < ZQ_ICDF_KNOTS; ++k) {
+                double z0 = zq_knot(k), z1 = zq_knot(k + 1);
+                zq_icdf_base[k] = (float)z0;
+                zq_icdf_slope[k] = (float)((z1 - z0) / 131072.0);
+            }
+            zq_icdf_ready = 1;
+        }
+    }
+}
+
+/* Copies of the table for tests: base and slope, ZQ_ICDF_KNOTS floats each. */
+void zq_icdf_table(float *base, float *slope)
+{
+    zq_icdf_init();
+    memcpy(base, zq_icdf_base, sizeof(zq_icdf_base));
+    memcpy(slope, zq_icdf_slope, sizeof(zq_icdf_slope));
+}
+
+/* One standard normal from one 32-bit word (see the header). */
+float zq_gauss_from_word(uint32_t w)
+{
+    uint32_t v = 0x80000000u - (w & 0x7FFFFFFFu);       /* 1 .. 2^31 */
+    uint32_t fb = float_to_bits((float)v);              /* round to nearest */
+    uint32_t idx = (fb >> 17) - (127u << 6);
+    float off = (float)(fb & 0x1FFFFu);
+    float z = fmaf(off, zq_icdf_slope[idx], zq_icdf_base[idx]);
+    return (w >> 31) ? -z : z;
+}
+
+void zq_gauss_words(const uint32_t *w, uint64_t n, float *z)
+{
+    zq_icdf_init();
+    for (uint64_t i = 0; i < n; ++i) z[i] = zq_gauss_from_word(w[i]);
 }
 
 /* z for elements [4*blk, 4*blk+4) of tensor `tensor_id` under `seed`. */
@@ -110,8 +140,7 @@ void zq_normal4(uint64_t seed, uint32_t tensor_id, uint64_t blk, float z[4])
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t w[4];
     zq_philox4x32_10(ctr, key, w);
-    zq_box_muller(w[0], w[1], &z[0], &z[1]);
-    zq_box_muller(w[2], w[3], &z[2], &z[3]);
+    for (int j = 0; j < 4; ++j) z[j] = zq_gauss_from_word(w[j]);
 }
 
 /* Raw words for blocks [blk0, blk0+nblk): out has 4*nblk entries. */
@@ -128,6 +157,7 @@ void zq_philox_words(uint64_t seed, uint32_t tensor_id, uint64_t blk0, uint64_t 
 /* z[i] for i in [0, n); n need not be a multiple of 4. */
 void zq_normal_fill(uint64_t seed, uint32_t tensor_id, uint64_t n, float *z)
 {
+    zq_icdf_init();
     uint64_t nblk = (n + 3) / 4;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < (int64_t)nblk; ++b) {
@@ -144,6 +174,7 @@ void zq_normal_fill(uint64_t seed, uint32_t tensor_id, uint64_t n, float *z)
 void zq_perturb(const float *w, uint64_t n, uint64_t seed, uint32_t tensor_id,
                 float signed_eps, float *w_out)
 {
+    zq_icdf_init();
     uint64_t nblk = (n + 3) / 4;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < (int64_t)nblk; ++b) {
@@ -159,6 +190,7 @@ void zq_perturb(const float *w, uint64_t n, uint64_t seed, uint32_t tensor_id,
 /* Eq. (2) with the one-direction estimate: W <- W - scale * z, scale = lr * g. */
 void zq_update(float *w, uint64_t n, uint64_t seed, uint32_t tensor_id, float scale)
 {
+    zq_icdf_init();
     uint64_t nblk = (n + 3) / 4;
 #pragma omp parallel for schedule(static)
     for (int64_t b = 0; b < (int64_t)nblk; ++b) {

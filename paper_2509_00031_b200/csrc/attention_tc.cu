@@ -190,7 +190,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                     AttParams p) {
     using Cfg = AttCfg<D>;
     constexpr int KSUB = D / 64;               // 64-column (128-byte) sub-tiles along d_head
-    constexpr int DH = D / 2;                  // output columns per softmax thread
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -406,14 +405,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 if (!wait_all(s_full(sbuf), (s_it >> 1) & 1u)) { ok = false; break; }
                 tc_fence_after();
                 float s[BKV];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t sm[32], sc[32];
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + h * 32), sm);
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64 + h * 32), sc);
+                {
+                    // all four loads in flight before the single wait
+                    uint32_t sm0[32], sc0[32], sm1[32], sc1[32];
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128), sm0);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64), sc0);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 32), sm1);
+                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 96), sc1);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) s[h * 32 + c] = fmaf(__uint_as_float(sc[c]), kLoInv, __uint_as_float(sm[c]));
+                    for (int c = 0; c < 32; ++c) {
+                        s[c] = fmaf(__uint_as_float(sc0[c]), kLoInv, __uint_as_float(sm0[c]));
+                        s[32 + c] = fmaf(__uint_as_float(sc1[c]), kLoInv, __uint_as_float(sm1[c]));
+                    }
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -424,9 +428,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                     for (int c = 0; c < BKV; ++c)
                         if (j * BKV + c > qpos) s[c] = -INFINITY;
                 }
-                float mx = s[0];
+                // row maximum by a balanced tree (max is exact in any order)
+                float mx;
+                {
+                    float t8[8];
 #pragma unroll
-                for (int c = 1; c < BKV; ++c) mx = fmaxf(mx, s[c]);
+                    for (int c = 0; c < 8; ++c) t8[c] = s[c];
+#pragma unroll
+                    for (int c = 8; c < BKV; ++c) t8[c & 7] = fmaxf(t8[c & 7], s[c]);
+                    mx = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
+                }
                 if (j == 0) {
                     m_ref = mx;                                   // finite: key 0 is visible to every query; O is still empty
                 } else {
@@ -456,10 +467,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                         if (grow) m_ref = mx;
                     }
                 }
-                float rs = 0.0f;
+                // exponentials; the row sum in four independent partial sums (fixed order)
+                float rs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int c = 0; c < BKV; ++c) { s[c] = ex2(s[c] - m_ref); rs += s[c]; }
-                l_run += rs;
+                for (int c = 0; c < BKV; ++c) { s[c] = ex2(s[c] - m_ref); rs4[c & 3] += s[c]; }
+                l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
                 // P -> shared memory (operand layout: 128-byte rows, 16-byte chunks XOR-swizzled by row)
                 if (!wait_all(p_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
                 const uint32_t ph = base + Cfg::kOffP + (uint32_t)(row * 128), pl = ph + Cfg::kPBytes;

@@ -52,11 +52,6 @@ __device__ __forceinline__ uint32_t idesc_bf16() {
          | ((uint32_t)((BM * CG) >> 4) << 24); // M / 16
 }
 
-__device__ __forceinline__ void ce_merge(float& m, float& s, float v) {
-    if (v > m) { s = s * expf(m - v) + 1.0f; m = v; }
-    else s += expf(v - m);
-}
-
 struct TcParams {
     int64_t M, N, K;
     int Z;
@@ -284,14 +279,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                 } else {
+                    // chunk maximum first, then one exponential per logit and one rescale of the running sum
+                    float x[32], cm = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (n0 + j < p.N) {
-                            const float x = rs * __uint_as_float(v[j]);
-                            ce_merge(ce_m, ce_s, x);
-                            if (n0 + j == lab) p.label_logit[row] = x;
-                        }
+                        x[j] = (n0 + j < p.N) ? rs * __uint_as_float(v[j]) : -INFINITY;
+                        cm = fmaxf(cm, x[j]);
+                        if (n0 + j == lab) p.label_logit[row] = x[j];
                     }
+                    const float nm = fmaxf(ce_m, cm);                 // finite: column n0 is inside the matrix
+                    float acc_s = ce_s * __expf(ce_m - nm);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) acc_s += __expf(x[j] - nm);
+                    ce_s = acc_s;
+                    ce_m = nm;
                 }
             }
             if (p.mode == 1 && row_ok) p.partials[row * p.tiles_n + tn] = make_float2(ce_m, ce_s);

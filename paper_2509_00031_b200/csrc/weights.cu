@@ -9,6 +9,10 @@
 #include "common.cuh"
 #include "rng.cuh"
 
+#include <cmath>
+#include <mutex>
+#include <vector>
+
 namespace zq {
 
 long long g_launch_count = 0;
@@ -17,9 +21,51 @@ namespace {
 
 constexpr int kThreads = 256;
 
+// ---- table of the inverse Gaussian distribution function (rng.cuh) -----------------------------------------
+__device__ float2 g_icdf_table[kIcdfKnots];
+
+// z >= 0 with upper tail probability q (0 for q >= 1/2), by bisection on erfc in double precision.
+double upper_quantile(double q) {
+    if (q >= 0.5) return 0.0;
+    double lo = 0.0, hi = 8.0;
+    for (int it = 0; it < 200; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (0.5 * erfc(mid * 0.70710678118654752440) > q) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+// Uploads the table to the current device the first time a generator kernel is launched on it.
+bool ensure_icdf_table() {
+    static std::mutex mu;
+    static bool ready[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    if (ready[dev]) return true;
+    static std::vector<float2> host;
+    if (host.empty()) {
+        std::vector<double> knot(kIcdfKnots + 1);
+        for (int k = 0; k <= kIcdfKnots; ++k)
+            knot[k] = upper_quantile(std::ldexp(1.0 + (k & 63) / 64.0, k >> 6) / 4294967296.0);
+        host.resize(kIcdfKnots);
+        for (int k = 0; k < kIcdfKnots; ++k)
+            host[k] = make_float2((float)knot[k], (float)((knot[k + 1] - knot[k]) / 131072.0));
+    }
+    if (cudaMemcpyToSymbol(g_icdf_table, host.data(), sizeof(float2) * kIcdfKnots) != cudaSuccess) return false;
+    ready[dev] = true;
+    return true;
+}
+
+// Every generator kernel starts by staging the table in shared memory.
+__device__ __forceinline__ void stage_icdf_table(float2* tab) {
+    for (int i = threadIdx.x; i < kIcdfKnots; i += blockDim.x) tab[i] = g_icdf_table[i];
+    __syncthreads();
+}
+
 inline int stream_grid(int64_t work_items, int per_block) {
     int64_t blocks = (work_items + per_block - 1) / per_block;
-    const int64_t cap = 148 * 16;
+    const int64_t cap = 148 * 8;       // one resident wave of 256-thread CTAs (each stages the 16 KB table once)
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return (int)blocks;
@@ -33,9 +79,11 @@ __global__ void philox_words_kernel(uint32_t k0, uint32_t k1, uint32_t tid, uint
 }
 
 __global__ void normal_kernel(uint32_t k0, uint32_t k1, uint32_t tid, uint64_t n, float* out) {
+    __shared__ float2 tab[kIcdfKnots];
+    stage_icdf_table(tab);
     const uint64_t nblk = (n + 3) / 4;
     for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b < nblk; b += (uint64_t)gridDim.x * blockDim.x) {
-        const float4 z = direction4(k0, k1, tid, b);
+        const float4 z = direction4(tab, k0, k1, tid, b);
         const float v[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j)
@@ -68,10 +116,6 @@ __device__ __forceinline__ GroupQ group_params(float mn, float mx, float qp) {
 __device__ __forceinline__ float quant_code(float x, const GroupQ& g, float qp) {
     const float q = __fadd_rn(rintf(__fmul_rn(x, g.inv)), g.zp);
     return fminf(fmaxf(q, 0.0f), qp);
-}
-
-__device__ __forceinline__ float dequant(float code, const GroupQ& g) {
-    return __fmul_rn(__fadd_rn(code, -g.zp), g.step);
 }
 
 __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
@@ -137,6 +181,8 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
                       uint4* __restrict__ op_plus, uint4* __restrict__ op_minus,
                       uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp) {
     constexpr int LANES = GROUP / 16;
+    __shared__ float2 tab[kIcdfKnots];
+    if (perturb) stage_icdf_table(tab);
     const float qp = (float)((1 << bits) - 1);
     // whole warps iterate together so that the shuffles always see 32 lanes
     const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
@@ -151,7 +197,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         if (perturb) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(k0, k1, tid, (uint64_t)(4 * i + k));
+                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)(4 * i + k));
                 const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -251,11 +297,28 @@ unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restr
 __global__ void __launch_bounds__(kThreads)
 update_kernel(float* __restrict__ w, uint64_t n, uint32_t k0, uint32_t k1, uint32_t tid,
               const float* __restrict__ scale_ptr, float scale_val) {
+    __shared__ float2 tab[kIcdfKnots];
+    stage_icdf_table(tab);
     const float c = -(scale_ptr ? *scale_ptr : scale_val);
     const uint64_t nblk = (n + 3) / 4;
     float4* w4 = reinterpret_cast<float4*>(w);
-    for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b < nblk; b += (uint64_t)gridDim.x * blockDim.x) {
-        const float4 z = direction4(k0, k1, tid, b);
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x;
+    // four Philox blocks per iteration: all loads are issued before any of them is used
+    for (; b + 3 * stride < nblk && 4 * (b + 3 * stride) + 4 <= n; b += 4 * stride) {
+        float4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = w4[b + u * stride];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float4 z = direction4(tab, k0, k1, tid, b + u * stride);
+            x[u].x = __fmaf_rn(c, z.x, x[u].x); x[u].y = __fmaf_rn(c, z.y, x[u].y);
+            x[u].z = __fmaf_rn(c, z.z, x[u].z); x[u].w = __fmaf_rn(c, z.w, x[u].w);
+            w4[b + u * stride] = x[u];
+        }
+    }
+    for (; b < nblk; b += stride) {
+        const float4 z = direction4(tab, k0, k1, tid, b);
         if (4 * b + 4 <= n) {
             float4 x = w4[b];
             x.x = __fmaf_rn(c, z.x, x.x); x.y = __fmaf_rn(c, z.y, x.y);
@@ -279,7 +342,7 @@ void launch_philox_words(uint64_t seed, uint32_t tid, uint64_t blk0, uint64_t nb
 }
 
 void launch_normal(uint64_t seed, uint32_t tid, uint64_t n, float* out, cudaStream_t s) {
-    if (n == 0) return;
+    if (n == 0 || !ensure_icdf_table()) return;
     normal_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(
         (uint32_t)seed, (uint32_t)(seed >> 32), tid, n, out);
     count_launch();
@@ -310,7 +373,7 @@ static void weight_operand_dispatch(const float* w, int64_t n, int bits, int per
 void launch_weight_operand(const float* w, int64_t n, int group, int bits, int perturb, uint64_t seed, uint32_t tid,
                            float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes, float* step,
                            int32_t* zp, cudaStream_t s) {
-    if (n == 0) return;
+    if (n == 0 || (perturb && !ensure_icdf_table())) return;
     if (group == 32) weight_operand_dispatch<32>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
     else if (group == 64) weight_operand_dispatch<64>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
     else weight_operand_dispatch<128>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
@@ -340,7 +403,7 @@ void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_
 }
 
 void launch_update(float* w, uint64_t n, uint64_t seed, uint32_t tid, const float* scale_ptr, float scale_val, cudaStream_t s) {
-    if (n == 0) return;
+    if (n == 0 || !ensure_icdf_table()) return;
     update_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(
         w, n, (uint32_t)seed, (uint32_t)(seed >> 32), tid, scale_ptr, scale_val);
     count_launch();

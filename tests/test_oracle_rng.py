@@ -3,7 +3,9 @@
 * raw Philox4x32-10 words against cuRAND's host generator (a library
   implementation of the same published cipher) and against a big-integer
   restatement of the round function for general counters;
-* the binary32 Box-Muller against float64 evaluation of its definition;
+* the word -> normal map (table-driven inverse distribution function) against a
+  float64 library evaluation of its definition, and its knot table against an
+  independent computation of every knot;
 * the generated distribution against the closed forms of the Gaussian tail
   lemma of the paper's theory appendix (Lemma "1-D Gaussian tail identities");
 * regeneration: the same (seed, tensor, index) always gives the same bits.
@@ -73,37 +75,54 @@ def test_streams_differ_by_tensor_block_and_seed():
     assert len({tuple(r) for r in a}) == 64
 
 
-def test_box_muller_matches_float64_definition():
-    rng = np.random.default_rng(11)
-    w = rng.integers(0, 2**32, size=(20000, 2), dtype=np.uint64)
-    # include the extremes of both words
-    w[:4] = [[0, 0], [2**32 - 1, 2**32 - 1], [0, 2**32 - 1], [2**32 - 1, 0]]
-    worst = 0.0
-    for w0, w1 in w:
-        w0, w1 = int(w0), int(w1)
-        za, zb = core.box_muller(w0, w1)
-        u = (2 * (w0 >> 9) + 1) / 2.0**24
-        r = math.sqrt(-2.0 * math.log(u))
-        phi = (2 * ((w1 >> 6) & 0x7FFFFF) + 1) / 2.0**24 * (math.pi / 4)
-        c, s = math.cos(phi), math.sin(phi)
-        octant = w1 >> 29
-        first, second = (s, c) if octant & 1 else (c, s)
-        if octant & 2:
-            first = -first
-        if octant & 4:
-            second = -second
-        worst = max(worst, abs(za - r * first), abs(zb - r * second))
-        assert abs(za - r * first) <= 2e-6 * max(1.0, r)
-        assert abs(zb - r * second) <= 2e-6 * max(1.0, r)
-    assert worst > 0.0   # binary32 evaluation, not a float64 copy
+def _words_with_extremes(n, seed):
+    w = np.random.default_rng(seed).integers(0, 2**32, size=n, dtype=np.uint64).astype(np.uint32)
+    w[:8] = [0, 1, 0x7FFFFFFE, 0x7FFFFFFF, 0x80000000, 0x80000001, 0xFFFFFFFE, 0xFFFFFFFF]
+    return w
 
 
-def test_octants_cover_the_circle_uniformly():
-    z = core.normal(2024, 9, 4_000_000).reshape(-1, 2)
-    ang = np.arctan2(z[:, 1].astype(np.float64), z[:, 0].astype(np.float64))
-    hist, _ = np.histogram(ang, bins=64, range=(-math.pi, math.pi))
-    expect = len(z) / 64
-    assert np.all(np.abs(hist - expect) < 6 * math.sqrt(expect))
+def test_word_to_normal_matches_float64_inverse_distribution_function():
+    """|z| = Phi^-1(1 - v / 2^32) with v = 2^31 - (w mod 2^31), sign from the top bit (scipy evaluates the
+    definition in float64); the piecewise-linear table stays within 3e-5 of it, tails included."""
+    from scipy.stats import norm
+    w = _words_with_extremes(400_000, 11)
+    z = core.gauss_from_words(w).astype(np.float64)
+    v = (2**31 - (w.astype(np.int64) & 0x7FFFFFFF)).astype(np.float64)
+    want = norm.isf(v / 2.0**32) * np.where(w >> 31, -1.0, 1.0)
+    err = np.abs(z - want)
+    assert err.max() <= 3e-5
+    assert err.max() > 0.0                       # an interpolated table, not a float64 copy
+    assert z[0] == 0.0 and abs(z[3] - 6.2302601) < 1e-6 and z[7] == -z[3]      # centre and the largest magnitude
+    # odd symmetry in the sign bit, monotone in the magnitude bits
+    assert np.array_equal(core.gauss_from_words(w ^ np.uint32(0x80000000)), -core.gauss_from_words(w))
+    m = np.sort(w & np.uint32(0x7FFFFFFF))
+    zm = core.gauss_from_words(m)
+    assert np.all(np.diff(zm) >= 0)
+
+
+def test_knot_table_against_independent_quantiles():
+    """Every knot v = 2^E (1 + j/64): base = float32(Phi^-1(1 - v/2^32)) (scipy's ndtri-based isf, a different
+    algorithm from the oracle's bisection on erfc), slopes join consecutive knots."""
+    from scipy.stats import norm
+    base, slope = core.icdf_table()
+    k = np.arange(2048)
+    v = np.ldexp(1.0 + (k & 63) / 64.0, k >> 6)
+    q = v / 2.0**32
+    want = np.where(q < 0.5, norm.isf(np.minimum(q, 0.5)), 0.0)
+    used = k <= 31 * 64                          # v <= 2^31
+    ulp = np.spacing(np.abs(want).astype(np.float32)).astype(np.float64)
+    assert np.all(np.abs(base.astype(np.float64) - want)[used] <= 0.5000001 * ulp[used] + 1e-12)
+    assert np.all(np.diff(base[: 31 * 64 + 1]) < 0)          # |z| falls as the tail probability grows
+    joined = base[:-1].astype(np.float64) + 131072.0 * slope[:-1].astype(np.float64)
+    assert np.all(np.abs(joined - base[1:])[: 31 * 64] <= 2e-6)
+
+
+def test_signs_are_fair_and_words_of_a_block_independent():
+    z = core.normal(2024, 9, 4_000_000)
+    assert abs((z > 0).mean() - 0.5) < 5 * 0.5 / math.sqrt(len(z))
+    q = z.reshape(-1, 4).astype(np.float64)                     # the four normals of one Philox block
+    c = np.corrcoef(q.T)
+    assert np.all(np.abs(c - np.eye(4)) < 5 / math.sqrt(len(q)))
 
 
 def _phi(t):
