@@ -219,7 +219,8 @@ int zoqat_profile_read(zoqat_model_t* m, int category, double* ms, int64_t* inte
 #define ZOQAT_BUF_RESIDUAL   0   /* fp32 [passes*T, d_model]   residual stream after the last layer */
 #define ZOQAT_BUF_QKV        1   /* fp32 [passes*T, 3*d_model] q | k | v of the last layer (before RoPE) */
 #define ZOQAT_BUF_ATTN       2   /* fp32 [passes*T, d_model]   attention output of the last layer   */
-#define ZOQAT_BUF_FFN        3   /* fp32 [passes*T, 2*d_ffn or d_ffn] gate|up (LLaMA) or fc1 (OPT)   */
+#define ZOQAT_BUF_FFN        3   /* fp32: fc1 output [passes*T, d_ffn] (OPT); LLaMA: silu(gate)*up [passes*T, d_ffn] when
+                                    d_ffn is a multiple of 128 with the default GEMM, else gate|up [passes*T, 2*d_ffn] */
 #define ZOQAT_BUF_TOKEN_LOSS 4   /* fp32 [passes*T]            per-position cross-entropy            */
 int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* bytes);
 
@@ -291,6 +292,16 @@ int zoqat_op_ffn_act_operand(const float* x_dev, int64_t rows, int64_t cols, int
 int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, int64_t K,
                   const float* row_step_dev, const float* bias_dev, int relu, int accumulate,
                   float* out_dev, int impl, int32_t* err_flag_dev, void* stream);
+
+/* The gate and up projections of a SiLU-gated FFN in one launch, with the non-linearity in the epilogue:
+ * act[m, f] = silu(g) * u,  g = row_step[m] * sum_k A[m, k] * B[f, k],  u = row_step[m] * sum_k A[m, k] * B[F + f, k]
+ * (the linear layers of the forward pass of Section 4.1; the architecture is the workloads').
+ * a_dev bf16 [M, K]; b_dev bf16 [2F, K] = gate rows then up rows; act_dev fp32 [M, F]; row_amax_dev uint32 [M]
+ * receives max_f |act[m, f]| as the bit pattern of a float (the per-token quantiser of the next linear starts
+ * from it); F % 128 == 0, K % 8 == 0; tcgen05 pair kernel only. */
+int zoqat_op_gemm_silu_gate(const void* a_dev, const void* b_dev, int64_t M, int64_t F, int64_t K,
+                            const float* row_step_dev, float* act_dev, uint32_t* row_amax_dev,
+                            int32_t* err_flag_dev, void* stream);
 
 /* Causal softmax attention of one layer (the architecture of the workloads; the paper's
  * forward pass of Section 4.1 runs the unmodified decoder between the quantised linears).

@@ -29,7 +29,7 @@ EXPORTS = [
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
-    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
+    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
 ]
@@ -101,6 +101,7 @@ def lib():
             "zoqat_op_norm_act_operand": [vp, i64, i64, i32, vp, vp, f32, i32, vp, vp, vp, vp],
             "zoqat_op_ffn_act_operand": [vp, i64, i64, i32, i32, vp, vp, vp],
             "zoqat_op_gemm": [vp, vp, i64, i64, i64, vp, vp, i32, i32, vp, i32, vp, vp],
+            "zoqat_op_gemm_silu_gate": [vp, vp, i64, i64, i64, vp, vp, vp, vp, vp],
             "zoqat_op_attention_scratch_bytes": [i32, i32, i32, i32, P(sz)],
             "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp],
             "zoqat_op_head_loss_scratch_bytes": [i64, i64, P(sz)],
@@ -218,6 +219,16 @@ def zoqat_op_gemm(a, b, row_step=None, bias=None, relu=False, out=None, accumula
     _check(lib().zoqat_op_gemm(_p(a), _p(b), M, N, K, _p(row_step), _p(bias), int(relu), int(accumulate), _p(out),
                                impl, _p(err), _stream()))
     return out, err
+
+
+def zoqat_op_gemm_silu_gate(a, b_gate_up, row_step=None):
+    M, K = a.shape
+    F = b_gate_up.shape[0] // 2
+    act = torch.empty((M, F), dtype=torch.float32, device=a.device)
+    amax = torch.empty(M, dtype=torch.int32, device=a.device)
+    err = torch.zeros(1, dtype=torch.int32, device=a.device)
+    _check(lib().zoqat_op_gemm_silu_gate(_p(a), _p(b_gate_up), M, F, K, _p(row_step), _p(act), _p(amax), _p(err), _stream()))
+    return act, amax.view(torch.float32), err
 
 
 def zoqat_op_attention(qkv, batch, seq, n_heads, d_head, cos=None, sin=None, impl=GEMM_TCGEN05, scratch=None, err=None):

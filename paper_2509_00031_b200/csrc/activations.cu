@@ -263,6 +263,44 @@ ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int
     write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
 }
 
+// Activation operand of a row whose max |x| has already been collected (by the GEMM that produced x).
+template <int VPT>
+__global__ void __launch_bounds__(kRowThreads)
+rows_operand_reg_kernel(const float* __restrict__ x, int cols, const uint32_t* __restrict__ amax_bits, int a_bits,
+                        __nv_bfloat16* __restrict__ op, float* __restrict__ row_step) {
+    const int64_t r = blockIdx.x;
+    const int n4 = cols >> 2;
+    const float4* xr = reinterpret_cast<const float4*>(x + r * cols);
+    uint2* op_row = reinterpret_cast<uint2*>(op + r * cols);
+    float4 v[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int idx = threadIdx.x + i * kRowThreads;
+        v[i] = idx < n4 ? __ldcs(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (a_bits == 8) {
+        const float step = fmaxf(__fdiv_rn(__uint_as_float(amax_bits[r]), 127.0f), 1e-8f);
+        const float inv = __fdiv_rn(1.0f, step);
+        if (threadIdx.x == 0) row_step[r] = step;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4)
+                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), -128.0f), 127.0f),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), -128.0f), 127.0f));
+        }
+    } else {
+        if (threadIdx.x == 0) row_step[r] = 1.0f;
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) op_row[idx] = bf16x4(v[i].x, v[i].y, v[i].z, v[i].w);
+        }
+    }
+}
+
 // h[p*T + t, :] = embed[token[t], :] (+ pos[t % seq, :]) for each of `passes` copies.
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const float4* __restrict__ embed,
                              const float4* __restrict__ pos, int64_t T, int seq, int d4, int vocab, int passes,
@@ -412,6 +450,16 @@ void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, i
         if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
         ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step);
     }
+    count_launch();
+}
+
+void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits, __nv_bfloat16* op,
+                         float* row_step, cudaStream_t s) {
+    const int n4 = cols / 4;       // callers guarantee cols % 4 == 0, cols <= 16384 and 16-byte aligned rows
+    if (n4 <= 4 * kRowThreads) rows_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
+    else if (n4 <= 8 * kRowThreads) rows_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
+    else if (n4 <= 12 * kRowThreads) rows_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
+    else rows_operand_reg_kernel<16><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
     count_launch();
 }
 

@@ -73,6 +73,7 @@ struct Workspace {
     int32_t *count, *err_flag;
     zoqat_step_result_dev* result;
     void* attn_scratch;                 // fp16 hi/lo operands of the tensor-core attention
+    uint32_t* row_amax;                 // max |act| per row collected by the gate/up GEMM epilogue
     size_t bop_elems;                   // elements of ONE pass' operand buffer
     size_t total;
 };
@@ -110,6 +111,7 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.err_flag = (int32_t*)take(4);
     w.result = (zoqat_step_result_dev*)take(sizeof(zoqat_step_result_dev));
     w.attn_scratch = take(attention_tc_scratch_bytes(2 * c.max_batch, c.max_seq, c.n_heads, c.d_model / c.n_heads));
+    w.row_amax = (uint32_t*)take(R * 4);
     w.total = off;
 }
 
@@ -277,8 +279,17 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
+        // SiLU-gated FFN on the pair kernel: the epilogue multiplies silu(gate) by up and collects the row maxima,
+        // so the intermediate is half as wide and the quantiser that follows needs a single pass
+        const bool fuse_gate = llama && c.gemm_impl == ZOQAT_GEMM_TCGEN05 && F % 128 == 0 && F <= 16384;
+        if (fuse_gate) {
+            cudaMemsetAsync(w.row_amax, 0, (size_t)R * 4, s);
+            g.mode = 3; g.row_amax = w.row_amax;
+        }
         if (int rc = run_gemm(m, g, s)) return rc;
-        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s); }
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
+          if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
+          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s); }
         produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
@@ -734,6 +745,22 @@ int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, in
                                            : launch_gemm_tc(g, static_cast<cudaStream_t>(stream));
     if (rc != ZOQAT_OK) return fail(rc, "GEMM rejected: M=%lld N=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers, err flag for tcgen05)",
                                     (long long)M, (long long)N, (long long)K);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_gemm_silu_gate(const void* a_dev, const void* b_dev, int64_t M, int64_t F, int64_t K, const float* row_step_dev,
+                            float* act_dev, uint32_t* row_amax_dev, int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !act_dev || !row_amax_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (M <= 0 || F <= 0 || K <= 0 || F % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "F must be a positive multiple of 128");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CUDA_TRY(cudaMemsetAsync(row_amax_dev, 0, (size_t)M * 4, s));
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = M; g.N = 2 * F; g.K = K; g.Z = 1; g.row_step = row_step_dev; g.out = act_dev; g.err_flag = err_flag_dev;
+    g.b_stride = (size_t)2 * F * K; g.mode = 3; g.row_amax = row_amax_dev;
+    const int rc = launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "gated GEMM rejected: M=%lld F=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers)", (long long)M, (long long)F, (long long)K);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

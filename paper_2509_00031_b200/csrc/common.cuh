@@ -43,6 +43,9 @@ void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_ki
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s);
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
                             __nv_bfloat16* op, float* row_step, cudaStream_t s);
+// Activation operand of rows whose max |x| is already known (amax: bits of a non-negative float per row).
+void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits,
+                         __nv_bfloat16* op, float* row_step, cudaStream_t s);
 // fp32 CUDA-core attention (cross-check) and the tensor-core attention (needs scratch and an error word).
 void launch_attention(const float* qkv, int batch, int seq, int n_heads, int d_head,
                       const float* cos_t, const float* sin_t, float* out, cudaStream_t s);
@@ -63,7 +66,9 @@ struct GemmArgs {
     int relu;
     int accumulate;
     float* out;               // [Z*M, N]
-    int mode;                 // 0 store, 1 cross-entropy partials
+    uint32_t* row_amax;       // mode 3: [Z*M] max |act| per row as the bits of a non-negative float (zeroed by the caller)
+    int mode;                 // 0 store, 1 cross-entropy partials, 3 SiLU-gated pair (tcgen05 pair kernel only):
+                              //   B = [gate rows; up rows], out[z*M+m, f] = silu(row_step*A.gate_f) * (row_step*A.up_f), ldo = N/2
     const int32_t* labels;    // [M]
     float2* partials;         // [Z*M, ce_tiles] (max, sum exp)
     float* label_logit;       // [Z*M]

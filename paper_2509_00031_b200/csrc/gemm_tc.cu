@@ -66,6 +66,7 @@ struct TcParams {
     int32_t* err_flag;
     int tiles_m, tiles_n;
     int tma_out;              // 1: mode-0 results leave through map_out (needs N % 4 == 0)
+    uint32_t* row_amax;       // mode 3: [Z*M] running max |act| per row (bit pattern of a non-negative float)
 };
 
 template <int BN, int CG>
@@ -102,7 +103,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
-        if (p.tma_out) prefetch_tmap(&map_out);
+        if (p.tma_out || p.mode == 3) prefetch_tmap(&map_out);
     }
     if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns (in each CTA of a pair)
         if (CG == 2) { tmem_alloc_pair(tmem_slot, 2 * BN); tmem_relinquish_pair(); }
@@ -130,7 +131,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::kStageBytes);
                         const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
                         tma_load_3d_pair(a_dst, &map_a, lead_full, kb * BK, tm * TM + (int)rank * BM, z);
-                        tma_load_3d_pair(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, tn * BN + (int)rank * (BN / 2), z);
+                        // mode 3: the tile's first 128 columns are gate features, the last 128 the matching up features
+                        const int b_row = p.mode == 3 ? (int)rank * (int)(p.N / 2) + tn * (BN / 2) : tn * BN + (int)rank * (BN / 2);
+                        tma_load_3d_pair(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, b_row, z);
                     } else {
                         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
                         tma_load_3d(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z);
@@ -203,8 +206,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int64_t n_base = (int64_t)tn * BN;
             float ce_m = -INFINITY, ce_s = 0.0f;
             const int32_t lab = (p.mode == 1 && row_ok) ? p.labels[m] : -1;
+            if (p.mode == 3) {
+                // SiLU-gated FFN: act = silu(gate) * up leaves as fp32 [rows, N/2]; the row maximum of |act| is
+                // collected for the activation quantiser that follows.
+                float amax = 0.0f;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+                for (int c = 0; c < BN / 64; ++c) {
+                    uint32_t vg[32], vu[32];
+                    __syncwarp();
+                    tmem_ld32(t_addr + (uint32_t)(c * 32), vg);
+                    tmem_ld32(t_addr + (uint32_t)(BN / 2 + c * 32), vu);
+                    tmem_ld_wait();
+                    const uint32_t box = out_stage + (uint32_t)((quarter * 2 + out_buf) * Cfg::kOutBoxBytes);
+                    if (lane == 0) bulk_wait_read_1();
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        float a4[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float g = rs * __uint_as_float(vg[j + e]);
+                            const float u = rs * __uint_as_float(vu[j + e]);
+                            a4[e] = __fdiv_rn(g, 1.0f + expf(-g)) * u;
+                            amax = fmaxf(amax, fabsf(a4[e]));
+                        }
+                        const uint32_t dst = box + (uint32_t)(lane * 128) + (uint32_t)((((j >> 2) ^ (lane & 7)) << 4));
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(a4[0]), "f"(a4[1]), "f"(a4[2]), "f"(a4[3]) : "memory");
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&map_out, box, tn * (BN / 2) + c * 32, tm * TM + (int)rank * BM + quarter * 32, z);
+                        bulk_commit();
+                    }
+                    out_buf ^= 1;
+                }
+                if (row_ok) atomicMax(p.row_amax + row, __float_as_uint(amax));
+            }
+#pragma unroll 1
+            for (int c = 0; c < (p.mode == 3 ? 0 : BN / 32); ++c) {
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)(c * 32), v);
@@ -389,7 +429,12 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     p.tiles_m = (int)((a.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((a.N + BN - 1) / BN);
     p.tma_out = (a.mode == 0 && a.N % 4 == 0) ? 1 : 0;
-    if (p.tma_out) {
+    p.row_amax = a.row_amax;
+    if (a.mode == 3) {
+        if (CG != 2 || BN != 256 || a.N % 256 != 0 || !a.row_amax || !a.out) return ZOQAT_ERR_INVALID_ARG;
+        p.tiles_n = (int)(a.N / 256);
+        if (!make_out_map(&map_out, a.out, a.M, a.N / 2, a.Z)) return ZOQAT_ERR_CUDA;
+    } else if (p.tma_out) {
         if (!make_out_map(&map_out, a.out, a.M, a.N, a.Z)) return ZOQAT_ERR_CUDA;
     } else {
         map_out = map_a;      // never dereferenced
@@ -427,7 +472,8 @@ int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
          reinterpret_cast<uintptr_t>(a.bias)) & 15)
         return ZOQAT_ERR_INVALID_ARG;
     // the cross-entropy epilogue always uses 256-column tiles (gemm_ce_tiles)
-    if (a.mode == 1 || a.N > 128) return a.single_cta ? launch_tc<256, 1>(a, s) : launch_tc<256, 2>(a, s);
+    if (a.mode == 3 && a.single_cta) return ZOQAT_ERR_UNSUPPORTED;
+    if (a.mode != 0 || a.N > 128) return a.single_cta ? launch_tc<256, 1>(a, s) : launch_tc<256, 2>(a, s);
     return launch_tc<128, 1>(a, s);
 }
 

@@ -220,6 +220,27 @@ def test_gemm_epilogues(zq, impl):
     assert int(err.item()) == 0
 
 
+@pytest.mark.parametrize("M,F,K", [(128, 128, 64), (300, 384, 192), (1000, 1024, 256)])
+def test_gemm_silu_gate(zq, M, F, K):
+    """Gate and up projections with silu(gate) * up in the epilogue, against float64; the collected row maximum is
+    exactly the maximum of the stored values."""
+    rng = np.random.default_rng(M + F)
+    a = core.round_bf16(rng.standard_normal((M, K)).astype(np.float32))
+    b = core.round_bf16((rng.standard_normal((2 * F, K)) * 0.1).astype(np.float32))
+    rs = rng.uniform(0.5, 1.5, M).astype(np.float32)
+    act, amax, err = zq.zoqat_op_gemm_silu_gate(dev(a).bfloat16(), dev(b).bfloat16(), dev(rs))
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    y = (a.astype(np.float64) @ b.astype(np.float64).T) * rs[:, None]
+    g, u = y[:, :F], y[:, F:]
+    want = g / (1 + np.exp(-g)) * u
+    got = act.cpu().numpy()
+    scale = (np.abs(a).astype(np.float64) @ np.abs(b).astype(np.float64).T) * rs[:, None]
+    bound = 4e-6 * (scale[:, :F] * (np.abs(u) + 1) + scale[:, F:] * (np.abs(g) + 1)) + 1e-7
+    assert np.all(np.abs(got - want) <= bound)
+    assert np.array_equal(amax.cpu().numpy(), np.abs(got).max(axis=1))
+
+
 def test_gemm_rejects_bad_arguments(zq):
     a = torch.zeros((8, 12), dtype=torch.bfloat16, device="cuda")     # K not a multiple of 8
     b = torch.zeros((8, 12), dtype=torch.bfloat16, device="cuda")
