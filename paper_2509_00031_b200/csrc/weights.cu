@@ -273,20 +273,28 @@ pack_frozen_kernel(const float4* __restrict__ w, int64_t n4, int bits, uint32_t*
     }
 }
 
-template <int GROUP>
+template <int GROUP, int BITS>
 __global__ void __launch_bounds__(kThreads)
-unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restrict__ qparams, int64_t n4, int bits,
+unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restrict__ qparams, int64_t n4,
                       uint2* __restrict__ op) {
     constexpr int LANES = GROUP / 4;
     const int lane = threadIdx.x & 31;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
-        const uint32_t* words = packed + (i >> 5) * (4 * bits);
+        // the 4*BITS words of this 128-element run, as BITS 16-byte loads (the same address in every lane)
+        const uint4* run = reinterpret_cast<const uint4*>(packed + (i >> 5) * (4 * BITS));
+        uint32_t wd[4 * BITS];
+#pragma unroll
+        for (int q = 0; q < BITS; ++q) {
+            const uint4 t = __ldg(run + q);
+            wd[4 * q] = t.x; wd[4 * q + 1] = t.y; wd[4 * q + 2] = t.z; wd[4 * q + 3] = t.w;
+        }
         const float2 qpv = __ldg(qparams + i / LANES);
         float v[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t c = 0;
-            for (int b = 0; b < bits; ++b) c |= ((__ldg(words + j * bits + b) >> lane) & 1u) << b;
+#pragma unroll
+            for (int b = 0; b < BITS; ++b) c |= ((wd[j * BITS + b] >> lane) & 1u) << b;
             v[j] = __fmul_rn(__fadd_rn((float)c, -qpv.y), qpv.x);
         }
         op[i] = pack_bf16x4(v[0], v[1], v[2], v[3]);
@@ -390,15 +398,22 @@ void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t
     count_launch();
 }
 
+template <int GROUP>
+static void unpack_dispatch(const uint32_t* packed, const float2* qparams, int64_t n4, int bits, uint2* o, int grid, cudaStream_t s) {
+    if (bits == 2) unpack_operand_kernel<GROUP, 2><<<grid, kThreads, 0, s>>>(packed, qparams, n4, o);
+    else if (bits == 3) unpack_operand_kernel<GROUP, 3><<<grid, kThreads, 0, s>>>(packed, qparams, n4, o);
+    else unpack_operand_kernel<GROUP, 4><<<grid, kThreads, 0, s>>>(packed, qparams, n4, o);
+}
+
 void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,
                            __nv_bfloat16* op, cudaStream_t s) {
     if (n == 0) return;
     const int64_t n4 = n / 4;
     const int grid = stream_grid(n4, kThreads);
     uint2* o = reinterpret_cast<uint2*>(op);
-    if (group == 32) unpack_operand_kernel<32><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
-    else if (group == 64) unpack_operand_kernel<64><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
-    else unpack_operand_kernel<128><<<grid, kThreads, 0, s>>>(packed, qparams, n4, bits, o);
+    if (group == 32) unpack_dispatch<32>(packed, qparams, n4, bits, o, grid, s);
+    else if (group == 64) unpack_dispatch<64>(packed, qparams, n4, bits, o, grid, s);
+    else unpack_dispatch<128>(packed, qparams, n4, bits, o, grid, s);
     count_launch();
 }
 
