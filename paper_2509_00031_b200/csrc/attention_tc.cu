@@ -20,7 +20,8 @@
 //     warp 1     MMA issuer: S_j = Q K_j^T (N = 64) into one of two TMEM score buffers - issued one
 //                tile ahead of the softmax - and O += P_j V_j (N = d_head), accumulated in TMEM over
 //                the whole work item.
-//     warps 2-5  softmax, one thread per query row: read S_j from TMEM, base-2 exponentials relative
+//     warps 2-5  softmax, one thread per query row (kRowThreads = 2 gives each row two threads that share the
+//                columns and exchange their maxima; it measured no faster): read S_j from TMEM, base-2 exponentials relative
 //                to a reference maximum, write P_j hi/lo to shared memory in the operand layout.  The
 //                reference only moves when the row maximum has grown by more than 2^8 since it was
 //                set (the normalisation by the running sum makes any reference exact); only then is
@@ -38,7 +39,8 @@ namespace zq {
 namespace {
 
 constexpr int BQ = 128, BKV = 64;
-constexpr int kAttThreadsTC = 192;
+constexpr int kRowThreads = 1;          // softmax threads per query row (each takes 1/kRowThreads of the columns)
+constexpr int kAttThreadsTC = 64 + 128 * kRowThreads;
 constexpr float kRefSlack = 8.0f;      // the softmax reference may lag the row maximum by up to 2^8
 constexpr float kLoScale = 2048.0f, kLoInv = 1.0f / 2048.0f;
 constexpr int kErrAttnSmem = 16;       // dynamic shared memory window too small after alignment
@@ -52,11 +54,13 @@ template <int D> struct AttCfg {
     static constexpr int kPBytes = BQ * BKV * 2;          // one of Ph / Pl
     static constexpr int kOffStage = 2 * kQBytes;
     static constexpr int kOffP = kOffStage + kStages * kStageBytes;
-    static constexpr int kOffBar = kOffP + 2 * kPBytes;
-    static constexpr int kUsedBytes = kOffBar + 160;      // 18 mbarriers + the TMEM base word
+    static constexpr int kOffX = kOffP + 2 * kPBytes;     // row-max exchange between the threads of a row: [2 slots][128 rows][2] floats
+    static constexpr int kOffBar = kOffX + (kRowThreads == 2 ? 2048 : 0);
+    static constexpr int kUsedBytes = kOffBar + 192;      // 22 mbarriers + the TMEM base word
     // 1 KB of slack for the 1024-byte alignment of the tiles; at least 120 KB so that a second CTA stays off
     // the SM for d_head 64 (a CTA owns all 512 TMEM columns).
-    static constexpr int kSmemBytes = kUsedBytes + 1024 > 120 * 1024 ? kUsedBytes + 1024 : 120 * 1024;
+    static constexpr int kWant = kUsedBytes + 1024 > 120 * 1024 ? kUsedBytes + 1024 : 120 * 1024;
+    static constexpr int kSmemBytes = kWant > 232448 ? 232448 : kWant;     // the kernel checks that the tiles fit after alignment
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -208,6 +212,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
     const uint32_t p_full = bars + 80, p_empty = bars + 88, o_full = bars + 96, o_empty = bars + 104;
     const uint32_t tmem_slot = bars + 112;
     uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - raw));
+    auto x_bar = [&](int q) { return bars + 152u + 8u * q; };
+    float* xchg = reinterpret_cast<float*>(smem_raw + (base + Cfg::kOffX - raw));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (!smem_ok) {                              // uniform over the CTA: nothing has been set up yet
@@ -218,9 +224,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
         mbar_init(q_full, 1); mbar_init(q_empty, 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1);
-            mbar_init(s_full(s), 1); mbar_init(s_empty(s), 4);
+            mbar_init(s_full(s), 1); mbar_init(s_empty(s), 4 * kRowThreads);
         }
-        mbar_init(p_full, 4); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 4);
+        mbar_init(p_full, 4 * kRowThreads); mbar_init(p_empty, 1); mbar_init(o_full, 1); mbar_init(o_empty, 4 * kRowThreads);
+        for (int q = 0; q < 4; ++q) mbar_init(x_bar(q), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_qh); prefetch_tmap(&map_ql); prefetch_tmap(&map_kh);
         prefetch_tmap(&map_kl); prefetch_tmap(&map_vth); prefetch_tmap(&map_vtl);
@@ -386,16 +393,29 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
             if (!ok) atomicExch(p.err_flag, kErrAttnWait);
         }
     } else {
-        // ---------------- softmax / output warps (2..5), one thread per query row ----------------
+        // ---------------- softmax / output warps: kRowThreads threads per query row, each on its share of the columns
+        constexpr int CW = BKV / kRowThreads;               // score columns per thread
+        constexpr int DW = D / kRowThreads;                 // output columns per thread
         const int quarter = warp & 3;                       // TMEM lanes [32*quarter, 32*quarter + 32)
+        const int half = (warp - 2) >> 2;                   // which share of the columns
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int d_model = p.n_heads * D;
-        uint32_t s_it = 0, t_it = 0, q_it = 0;
+        uint32_t s_it = 0, t_it = 0, x_it = 0;
         bool ok = true;
         // wait helper: the whole warp takes the same decision
         auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait(bar, parity)) != 0; };
-        for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
+        // the two threads of a row swap one float through shared memory (two slots, so one barrier per swap suffices)
+        auto swap_with_partner = [&](float mine, float& theirs) -> bool {
+            xchg[((x_it & 1u) * BQ + row) * 2 + half] = mine;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_bar(quarter));
+            if (!wait_all(x_bar(quarter), x_it & 1u)) return false;
+            theirs = xchg[((x_it & 1u) * BQ + row) * 2 + (half ^ 1)];
+            ++x_it;
+            return true;
+        };
+        for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x) {
             const int qt = item_qt(it), bh = item_bh(it), n = n_kv_tiles(qt);
             const int qpos = qt * BQ + row;
             float m_ref = -INFINITY, l_run = 0.0f;
@@ -404,29 +424,30 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 const int sbuf = s_it & 1u;
                 if (!wait_all(s_full(sbuf), (s_it >> 1) & 1u)) { ok = false; break; }
                 tc_fence_after();
-                float s[BKV];
+                float s[CW];
                 {
-                    // all four loads in flight before the single wait
-                    uint32_t sm0[32], sc0[32], sm1[32], sc1[32];
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128), sm0);
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64), sc0);
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 32), sm1);
-                    tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 96), sc1);
+                    // all loads in flight before the single wait
+                    uint32_t sm[CW / 32][32], sc[CW / 32][32];
+#pragma unroll
+                    for (int h = 0; h < CW / 32; ++h) {
+                        tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + half * CW + h * 32), sm[h]);
+                        tmem_ld32(t_lane + (uint32_t)(sbuf * 128 + 64 + half * CW + h * 32), sc[h]);
+                    }
                     tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        s[c] = fmaf(__uint_as_float(sc0[c]), kLoInv, __uint_as_float(sm0[c]));
-                        s[32 + c] = fmaf(__uint_as_float(sc1[c]), kLoInv, __uint_as_float(sm1[c]));
-                    }
+                    for (int h = 0; h < CW / 32; ++h)
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) s[h * 32 + c] = fmaf(__uint_as_float(sc[h][c]), kLoInv, __uint_as_float(sm[h][c]));
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty(sbuf));
                 // causal mask (keys beyond the sequence end are beyond every valid query as well)
+                const int k0 = j * BKV + half * CW;
                 if (j * BKV + BKV - 1 > qt * BQ) {
 #pragma unroll
-                    for (int c = 0; c < BKV; ++c)
-                        if (j * BKV + c > qpos) s[c] = -INFINITY;
+                    for (int c = 0; c < CW; ++c)
+                        if (k0 + c > qpos) s[c] = -INFINITY;
                 }
                 // row maximum by a balanced tree (max is exact in any order)
                 float mx;
@@ -435,8 +456,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
 #pragma unroll
                     for (int c = 0; c < 8; ++c) t8[c] = s[c];
 #pragma unroll
-                    for (int c = 8; c < BKV; ++c) t8[c & 7] = fmaxf(t8[c & 7], s[c]);
+                    for (int c = 8; c < CW; ++c) t8[c & 7] = fmaxf(t8[c & 7], s[c]);
                     mx = fmaxf(fmaxf(fmaxf(t8[0], t8[1]), fmaxf(t8[2], t8[3])), fmaxf(fmaxf(t8[4], t8[5]), fmaxf(t8[6], t8[7])));
+                }
+                if (kRowThreads == 2) {
+                    float other;
+                    if (!swap_with_partner(mx, other)) { ok = false; break; }
+                    mx = fmaxf(mx, other);
                 }
                 if (j == 0) {
                     m_ref = mx;                                   // finite: key 0 is visible to every query; O is still empty
@@ -449,11 +475,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                         tc_fence_after();
                         const float f = grow ? ex2(m_ref - mx) : 1.0f;
 #pragma unroll 1
-                        for (int c0 = 0; c0 < D; c0 += 32) {
+                        for (int c0 = 0; c0 < DW; c0 += 32) {
 #pragma unroll 1
                             for (int part = 0; part < 2; ++part) {
                                 uint32_t o[32];
-                                const uint32_t addr = t_lane + (part == 0 ? 256u : 384u) + (uint32_t)c0;
+                                const uint32_t addr = t_lane + (part == 0 ? 256u : 384u) + (uint32_t)(half * DW + c0);
                                 tmem_ld32(addr, o);
                                 tmem_ld_wait();
 #pragma unroll
@@ -470,24 +496,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 // exponentials; the row sum in four independent partial sums (fixed order)
                 float rs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int c = 0; c < BKV; ++c) { s[c] = ex2(s[c] - m_ref); rs4[c & 3] += s[c]; }
+                for (int c = 0; c < CW; ++c) { s[c] = ex2(s[c] - m_ref); rs4[c & 3] += s[c]; }
                 l_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
                 // P -> shared memory (operand layout: 128-byte rows, 16-byte chunks XOR-swizzled by row)
                 if (!wait_all(p_empty, (t_it & 1u) ^ 1u)) { ok = false; break; }
                 const uint32_t ph = base + Cfg::kOffP + (uint32_t)(row * 128), pl = ph + Cfg::kPBytes;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < CW / 8; ++i) {
                     uint32_t wh[4], wl[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
+                        // hi = the leading 11 significant bits (by masking: exact in binary16 without a conversion
+                        // round trip; below the binary16 normal range hi = 0 and lo carries the value)
                         const float a = s[8 * i + 2 * e], b2 = s[8 * i + 2 * e + 1];
-                        const __half2 h2 = __floats2half2_rn(a, b2);
-                        const float2 hf = __half22float2(h2);
-                        const __half2 l2 = __floats2half2_rn((a - hf.x) * kLoScale, (b2 - hf.y) * kLoScale);
+                        const float ha = a >= 6.103515625e-05f ? __uint_as_float(__float_as_uint(a) & 0xFFFFE000u) : 0.0f;
+                        const float hb = b2 >= 6.103515625e-05f ? __uint_as_float(__float_as_uint(b2) & 0xFFFFE000u) : 0.0f;
+                        const __half2 h2 = __floats2half2_rn(ha, hb);
+                        const __half2 l2 = __floats2half2_rn((a - ha) * kLoScale, (b2 - hb) * kLoScale);
                         wh[e] = *reinterpret_cast<const uint32_t*>(&h2);
                         wl[e] = *reinterpret_cast<const uint32_t*>(&l2);
                     }
-                    const uint32_t chunk = (uint32_t)((i ^ (row & 7)) << 4);
+                    const uint32_t chunk = (uint32_t)(((half * (CW / 8) + i) ^ (row & 7)) << 4);
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ph + chunk), "r"(wh[0]), "r"(wh[1]), "r"(wh[2]), "r"(wh[3]) : "memory");
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pl + chunk), "r"(wl[0]), "r"(wl[1]), "r"(wl[2]), "r"(wl[3]) : "memory");
                 }
@@ -496,17 +525,24 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 if (lane == 0) mbar_arrive(p_full);
             }
             if (!ok) break;
+            // the row sum over all columns
+            float l_tot = l_run;
+            if (kRowThreads == 2) {
+                float other;
+                if (!swap_with_partner(l_run, other)) { ok = false; break; }
+                l_tot = l_run + other;
+            }
             // the item's last P V has completed: out = (O_main + 2^-11 O_corr) / sum
             if (!wait_all(o_full, (t_it & 1u) ^ 1u)) { ok = false; break; }
             tc_fence_after();
-            const float inv = 1.0f / l_run;
+            const float inv = 1.0f / l_tot;
             const int b = bh / p.n_heads, head = bh % p.n_heads;
-            float* dst = p.out + ((int64_t)b * p.seq + qpos) * d_model + head * D;
+            float* dst = p.out + ((int64_t)b * p.seq + qpos) * d_model + head * D + half * DW;
 #pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 32) {
+            for (int c0 = 0; c0 < DW; c0 += 32) {
                 uint32_t om[32], oc[32];
-                tmem_ld32(t_lane + 256u + (uint32_t)c0, om);
-                tmem_ld32(t_lane + 384u + (uint32_t)c0, oc);
+                tmem_ld32(t_lane + 256u + (uint32_t)(half * DW + c0), om);
+                tmem_ld32(t_lane + 384u + (uint32_t)(half * DW + c0), oc);
                 tmem_ld_wait();
                 if (qpos < p.seq) {
 #pragma unroll
