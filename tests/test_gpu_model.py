@@ -256,3 +256,55 @@ def test_step_host_buffers(zq):
     assert res.status == 0
     assert abs(res.loss_plus - lp) <= 1e-3 * abs(lp) and abs(res.loss_minus - lm) <= 1e-3 * abs(lm)
     assert abs(res.proj_grad - g) <= 0.1 * max(abs(g), 1.0)          # see the module docstring on g
+
+
+# ---- the five workloads at their real layer dimensions ------------------------------------------------------------
+def _cut(name, n_layers, **over):
+    w = dict(synth.WORKLOADS[name])
+    w.update(n_layers=n_layers, **over)
+    return w
+
+
+WORKLOAD_CUTS = [
+    pytest.param(_cut("opt1p3b_w4", 1), 1, 192, 0, False, id="opt1p3b_w4"),
+    pytest.param(_cut("llama7b_w4a8", 1), 1, 160, 0, False, id="llama7b_w4a8"),
+    pytest.param(_cut("llama7b_w2", 1), 1, 128, 0, False, id="llama7b_w2"),
+    pytest.param(_cut("llama7b_w3", 1), 1, 128, 0, False, id="llama7b_w3"),
+    pytest.param(_cut("llama13b_light", 2), 1, 96, 1, True, id="llama13b_light"),
+]
+
+
+@pytest.mark.parametrize("shape,batch,seq,first_trainable,packed", WORKLOAD_CUTS)
+def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packed):
+    """Every workload with its real d_model / heads / d_ffn / vocabulary / quantiser, cut to one layer (two for the
+    lightweight one: a frozen packed layer under a trainable one) and a short sequence so that the oracle finishes:
+    one full step against the oracle - both losses, the update of a block tensor and of the vocabulary projection."""
+    params = synth.make_params(shape, seed=3, max_seq=seq)
+    oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable), synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq,
+                          first_trainable_layer=first_trainable, packed_frozen=packed)
+    if packed:
+        model.zoqat_prequantize_frozen()
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
+    eps, lr, seed = 1e-3, 1e-6, 1000
+    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), seed, eps, lr))
+    model.zoqat_check()
+    lp, lm, g = oracle.step(tokens, labels, seed, eps, lr)
+    assert res["status"] == 0
+    assert abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
+    print(f"[{shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} W{shape['w_bits']}A{shape['a_bits']}] "
+          f"L+ {res['loss_plus']:.6f} / {lp:.6f}  L- {res['loss_minus']:.6f} / {lm:.6f}  g {res['proj_grad']:.4f} / {g:.4f}")
+    last = shape["n_layers"] - 1
+    name = "w_down" if shape["arch"] == "llama" else "fc2"
+    # the update uses the step's own g: compare against the oracle's update with that factor (bit for bit), and
+    # against the oracle's own step within the weight tolerance scaled by the difference in g
+    from oracle import core
+    from oracle.model import tensor_id, LM_HEAD_ID
+    w0 = params["layers"][last][name]
+    want = core.update_(w0.copy(), seed, tensor_id(last, oracle._ROLE[name]), np.float32(res["update_scale"]))
+    assert np.array_equal(model.params["layers"][last][name].cpu().numpy().view(np.uint32), want.view(np.uint32))
+    want_h = core.update_(params["lm_head"].copy(), seed, LM_HEAD_ID, np.float32(res["update_scale"]))
+    assert np.array_equal(model.params["lm_head"].cpu().numpy().view(np.uint32), want_h.view(np.uint32))
+    assert np.abs(model.params["layers"][last][name].cpu().numpy() - oracle.p["layers"][last][name]).max() <= 1e-5
+    if first_trainable:
+        assert np.array_equal(model.params["layers"][0]["wq"].cpu().numpy(), params["layers"][0]["wq"])
