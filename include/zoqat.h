@@ -171,6 +171,15 @@ int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* label
                int batch, int seq, uint64_t seed, float eps, float lr,
                zoqat_step_result_t* result_dev, void* stream);
 
+/* Eq. (1) with q = n_dirs directions per step (the paper's estimator averages over q directions u_1..u_q; it never
+ * states q): direction i uses seed + i, every g_i is the two-point estimate at the SAME weights, and Eq. (2) then
+ * applies W <- W - (lr / q) sum_i g_i u_i, direction by direction in one pass over each trainable tensor.
+ * results_dev: n_dirs records (device memory); record i holds L+, L-, g_i and its update factor fl((lr/q) g_i).
+ * n_dirs = 1 is zoqat_step.  2 * n_dirs forward passes. */
+int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                     int batch, int seq, uint64_t seed, int n_dirs, float eps, float lr,
+                     zoqat_step_result_t* results_dev, void* stream);
+
 /* The step in two halves, for data-parallel replicas that each hold all masters and a
  * shard of the mini-batch (the loss of Eq. (1) is a mean over the mini-batch):
  * zoqat_step_begin runs both passes on the local shard and writes

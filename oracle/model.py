@@ -270,3 +270,13 @@ class OracleModel:
         scale = F32(F32(lr) * g)
         self.apply_update(seed, scale)
         return lp, lm, float(g)
+
+    def step_multi(self, tokens, labels, seed, n_dirs, eps, lr):
+        """Eq. (1) with q = n_dirs directions u_1..u_q (seeds seed, seed+1, ...), all evaluated at the same W, then
+        Eq. (2): W <- W - (lr/q) sum_i g_i u_i, applied direction by direction (one binary32 fma per element each).
+        Returns the list of (L+, L-, g_i)."""
+        out = [self.projected_gradient(tokens, labels, seed + i, eps) for i in range(n_dirs)]
+        lr_q = F32(F32(lr) / F32(n_dirs))
+        for i, (_, _, g) in enumerate(out):
+            self.apply_update(seed + i, F32(lr_q * g))
+        return [(lp, lm, float(g)) for lp, lm, g in out]

@@ -25,7 +25,7 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
-    "zoqat_prequantize_frozen", "zoqat_forward_loss", "zoqat_step", "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_host", "zoqat_apply_update",
+    "zoqat_prequantize_frozen", "zoqat_forward_loss", "zoqat_step", "zoqat_step_multi", "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_host", "zoqat_apply_update",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
@@ -82,6 +82,7 @@ def lib():
             "zoqat_prequantize_frozen": [vp, vp],
             "zoqat_forward_loss": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step": [vp, vp, vp, i32, i32, u64, f32, f32, vp, vp],
+            "zoqat_step_multi": [vp, vp, vp, i32, i32, u64, i32, f32, f32, vp, vp],
             "zoqat_step_host": [vp, vp, vp, i32, i32, u64, f32, f32, P(StepResult), vp],
             "zoqat_step_begin": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step_finish": [vp, vp, u64, f32, f32, vp, vp],
@@ -359,6 +360,13 @@ class ZoqatModel:
         b, s = tokens.shape
         _check(lib().zoqat_step(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, _p(result), _stream()))
         return result
+
+    def zoqat_step_multi(self, tokens, labels, seed, n_dirs, eps, lr, results=None):
+        """results: float32 device tensor [n_dirs, 6] (one zoqat_step_result_t per direction)."""
+        results = torch.empty((n_dirs, 6), dtype=torch.float32, device="cuda") if results is None else results
+        b, s = tokens.shape
+        _check(lib().zoqat_step_multi(self.handle, _p(tokens), _p(labels), b, s, seed, n_dirs, eps, lr, _p(results), _stream()))
+        return results
 
     def zoqat_step_begin(self, tokens, labels, seed, eps, sums=None):
         """sums: float64 device tensor [3] = (sum L+, sum L-, labelled positions) of this shard."""

@@ -557,6 +557,38 @@ int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* label
     return zoqat_step_finish(m, m->ws.sums, seed, eps, lr, result_dev, stream);
 }
 
+int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                     uint64_t seed, int n_dirs, float eps, float lr, zoqat_step_result_t* results_dev, void* stream) {
+    if (!results_dev) return fail(ZOQAT_ERR_INVALID_ARG, "results_dev is NULL");
+    if (n_dirs < 1 || n_dirs > 64) return fail(ZOQAT_ERR_INVALID_ARG, "n_dirs %d (supported: 1..64)", n_dirs);
+    if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const float lr_q = lr / (float)n_dirs;                        // binary32 division, as in Eq. (1)'s 1/q
+    zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(results_dev);
+    // every direction is evaluated at the same W ...
+    for (int i = 0; i < n_dirs; ++i) {
+        if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed + (uint64_t)i, eps, 2, s)) return rc;
+        launch_pack_sums(m->ws.loss_sum, m->ws.count, m->ws.sums, s);
+        launch_finish_step(m->ws.sums, eps, lr_q, m->ws.err_flag, res + i, s);
+    }
+    // ... then Eq. (2) for all of them in one pass over each trainable tensor
+    {
+        ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
+        const int stride = (int)(sizeof(zoqat_step_result_dev) / sizeof(float));
+        for (auto& Ly : m->layers)
+            for (int r = 0; r < 7; ++r) {
+                Linear& L = Ly.lin[r];
+                if (L.present && L.trainable())
+                    launch_update_multi(L.w_mut, (uint64_t)(L.rows * L.cols), seed, n_dirs, L.tid, &res->update_scale, stride, s);
+            }
+        if (m->head.trainable())
+            launch_update_multi(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, n_dirs, m->head.tid, &res->update_scale, stride, s);
+    }
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
 int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
                     uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream) {
     if (int rc = check_call(m, tokens_host, labels_host, batch, seq)) return rc;

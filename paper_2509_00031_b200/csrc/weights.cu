@@ -340,7 +340,40 @@ update_kernel(float* __restrict__ w, uint64_t n, uint32_t k0, uint32_t k1, uint3
     }
 }
 
+// Eq. (2) with q directions in one pass over the tensor: w <- fma(-c_i, u_i, w) for i = 0..q-1 in that order,
+// direction i under seed + i, c_i read from scales[i * scale_stride] (device memory).
+__global__ void __launch_bounds__(kThreads)
+update_multi_kernel(float* __restrict__ w, uint64_t n, uint64_t seed, int n_dirs, uint32_t tid,
+                    const float* __restrict__ scales, int scale_stride) {
+    __shared__ float2 tab[kIcdfKnots];
+    stage_icdf_table(tab);
+    const uint64_t nblk = (n + 3) / 4;
+    float4* w4 = reinterpret_cast<float4*>(w);
+    for (uint64_t b = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; b < nblk; b += (uint64_t)gridDim.x * blockDim.x) {
+        const bool whole = 4 * b + 4 <= n;
+        float x[4];
+        if (whole) { const float4 t = w4[b]; x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+        else for (int j = 0; j < 4; ++j) x[j] = 4 * b + j < n ? w[4 * b + j] : 0.0f;
+        for (int i = 0; i < n_dirs; ++i) {
+            const uint64_t sd = seed + (uint64_t)i;
+            const float c = -scales[(size_t)i * scale_stride];
+            const float4 z = direction4(tab, (uint32_t)sd, (uint32_t)(sd >> 32), tid, b);
+            x[0] = __fmaf_rn(c, z.x, x[0]); x[1] = __fmaf_rn(c, z.y, x[1]);
+            x[2] = __fmaf_rn(c, z.z, x[2]); x[3] = __fmaf_rn(c, z.w, x[3]);
+        }
+        if (whole) w4[b] = make_float4(x[0], x[1], x[2], x[3]);
+        else for (int j = 0; j < 4; ++j) if (4 * b + j < n) w[4 * b + j] = x[j];
+    }
+}
+
 }  // namespace
+
+void launch_update_multi(float* w, uint64_t n, uint64_t seed, int n_dirs, uint32_t tid, const float* scales,
+                         int scale_stride, cudaStream_t s) {
+    if (n == 0 || n_dirs <= 0 || !ensure_icdf_table()) return;
+    update_multi_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(w, n, seed, n_dirs, tid, scales, scale_stride);
+    count_launch();
+}
 
 void launch_philox_words(uint64_t seed, uint32_t tid, uint64_t blk0, uint64_t nblk, uint32_t* out, cudaStream_t s) {
     if (nblk == 0) return;

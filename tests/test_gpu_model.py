@@ -308,3 +308,38 @@ def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packe
     assert np.abs(model.params["layers"][last][name].cpu().numpy() - oracle.p["layers"][last][name]).max() <= 1e-5
     if first_trainable:
         assert np.array_equal(model.params["layers"][0]["wq"].cpu().numpy(), params["layers"][0]["wq"])
+
+
+def test_step_multi_directions(zq):
+    """q = 3 directions per step: every g_i at the same weights, one fused update; against the oracle, and
+    q = 1 against zoqat_step bit for bit."""
+    from oracle import core
+    from oracle.model import tensor_id
+    shape, batch, seq = SMALL_LLAMA, 2, 96
+    model, oracle = build_pair(zq, shape, batch, seq, 0)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=16)
+    td, ld = dev(tokens), dev(labels)
+    eps, lr, seed, q = 1e-3, 1e-4, 400, 3
+    w0 = oracle.p["layers"][1]["w_down"].copy()
+    res = model.zoqat_step_multi(td, ld, seed, q, eps, lr).cpu()
+    model.zoqat_check()
+    recs = [zq.decode_step_result(res[i]) for i in range(q)]
+    want = oracle.step_multi(tokens, labels, seed, q, eps, lr)
+    lr_q = np.float32(np.float32(lr) / np.float32(q))
+    upd = w0.copy()
+    for i, (r, (lp, lm, g)) in enumerate(zip(recs, want)):
+        assert r["status"] == 0
+        assert abs(r["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(r["loss_minus"] - lm) <= 1e-3 * abs(lm)
+        assert abs(r["proj_grad"] - g) <= 0.1 * max(abs(g), 1.0)          # see the module docstring on g
+        assert r["update_scale"] == float(lr_q * np.float32(r["proj_grad"]))
+        core.update_(upd, seed + i, tensor_id(1, oracle._ROLE["w_down"]), np.float32(r["update_scale"]))
+    got = model.params["layers"][1]["w_down"].cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), upd.view(np.uint32))     # the fused update, given the step's own factors
+    assert np.abs(got - oracle.p["layers"][1]["w_down"]).max() <= 1e-5
+    # q = 1 is zoqat_step
+    a, _ = build_pair(zq, shape, batch, seq, 0)
+    b, _ = build_pair(zq, shape, batch, seq, 0)
+    ra = zq.decode_step_result(a.zoqat_step(td, ld, seed, eps, lr))
+    rb = zq.decode_step_result(b.zoqat_step_multi(td, ld, seed, 1, eps, lr)[0])
+    assert ra == rb
+    assert torch.equal(a.params["layers"][0]["wq"], b.params["layers"][0]["wq"]) and torch.equal(a.params["lm_head"], b.params["lm_head"])

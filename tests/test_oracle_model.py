@@ -255,3 +255,49 @@ def test_estimate_is_unbiased_in_expectation():
     assert cos > 0.85 * expect, (cos, expect, P)
     # scale: <avg, grad>/|grad|^2 -> 1
     assert abs(float(acc @ grad / (grad @ grad)) - 1.0) < 0.25
+
+
+def test_more_directions_reduce_the_estimator_error():
+    """Eq. (1) with q directions and Proposition 1 (ii): the mean squared error of the estimate falls like 1/q.
+    Quantiser off; the squared distance between (1/q) sum g_i u_i and the autograd gradient, averaged over
+    independent draws, is compared for q = 1 and q = 8."""
+    shape = dict(arch="llama", n_layers=1, d_model=8, n_heads=2, d_ffn=16, vocab=12)
+    p = synth.make_params(shape, seed=3, jitter=True)
+    cfg = OracleConfig(arch="llama", n_layers=1, d_model=8, n_heads=2, d_ffn=16, vocab=12, w_bits=0, a_bits=0, operand_bf16=False)
+    m = OracleModel(cfg, p)
+    tokens, labels = synth.make_batch(2, 6, 12, seed=12)
+    tp = torch_params(p, True)
+    torch_loss(tp, shape, tokens, labels).backward()
+    names = [(0, n) for n in m.linear_names()] + ["lm_head"]
+    grad = np.concatenate([(tp["lm_head"].grad if k == "lm_head" else tp["layers"][0][k[1]].grad).numpy().ravel() for k in names])
+    gu = []
+    for seed in range(240):
+        _, _, g = m.projected_gradient(tokens, labels, 5000 + seed, 1e-3)
+        u = _materialised_direction(m, 5000 + seed)
+        gu.append(float(g) * np.concatenate([u[k].ravel() for k in names]))
+    gu = np.array(gu)
+    mse1 = np.mean(np.sum((gu - grad) ** 2, axis=1))
+    mse8 = np.mean(np.sum((gu.reshape(30, 8, -1).mean(axis=1) - grad) ** 2, axis=1))
+    assert 5.0 < mse1 / mse8 < 12.0, (mse1, mse8)
+
+
+def test_step_multi_reduces_to_step_and_uses_one_w_for_all_directions():
+    m1, shape = make("llama", quant=True)
+    m2, _ = make("llama", quant=True)
+    tokens, labels = synth.make_batch(2, 12, shape["vocab"], seed=6)
+    a = m1.step(tokens, labels, 77, 1e-3, 1e-3)
+    b = m2.step_multi(tokens, labels, 77, 1, 1e-3, 1e-3)
+    assert b == [a]
+    for l in range(shape["n_layers"]):
+        for n in m1.linear_names():
+            assert np.array_equal(m1.p["layers"][l][n], m2.p["layers"][l][n])
+    # q = 3: every g_i is the two-point estimate at the ORIGINAL weights
+    m3, _ = make("llama", quant=True)
+    m4, _ = make("llama", quant=True)
+    want = [m4.projected_gradient(tokens, labels, 77 + i, 1e-3) for i in range(3)]
+    got = m3.step_multi(tokens, labels, 77, 3, 1e-3, 1e-3)
+    assert [g for _, _, g in got] == [float(g) for _, _, g in want]
+    lr_q = np.float32(np.float32(1e-3) / np.float32(3))
+    for i, (_, _, g) in enumerate(want):
+        m4.apply_update(77 + i, np.float32(lr_q * g))
+    assert np.array_equal(m3.p["layers"][0]["wq"], m4.p["layers"][0]["wq"])
