@@ -44,12 +44,14 @@ def workload_numbers(w):
     per_layer = 4 * d * d + (3 if w["arch"] == "llama" else 2) * d * F
     ftl = w.get("first_trainable_layer", 0)
     block = per_layer * L
-    trainable = per_layer * (L - ftl) + V * d
     head = V * d
+    names = w.get("trainable_names")
+    per_layer_trainable = per_layer if names is None else len(names) * d * d      # the selectable subsets are d x d projections
+    trainable = per_layer_trainable * (L - ftl) + (head if w.get("head_trainable", True) else 0)
     # frozen prefix layers are identical in both passes and are evaluated once
     lin_flops = 2 * T * (per_layer * ftl + 2 * per_layer * (L - ftl) + 2 * head)
     attn_flops = 2 * w["batch"] * w["seq"] ** 2 * d * (ftl + 2 * (L - ftl))
-    frozen = per_layer * ftl
+    frozen = per_layer * L - per_layer_trainable * (L - ftl)
     bytes_step = 4 * trainable + (w["w_bits"] / 8 + 8 / w["w_group"]) * frozen + 8 * trainable
     return dict(T=T, block_params=block, trainable_params=trainable, head_params=head,
                 linear_flops=lin_flops, attn_flops=attn_flops, flops=lin_flops + attn_flops, bytes=bytes_step)
@@ -209,13 +211,17 @@ def run_ours(args, w, rank, world, local_rank):
     ftl = w.get("first_trainable_layer", 0)
 
     params = make_device_params(w, torch, seed=0)          # every replica holds the same masters
+    names = w.get("trainable_names")
+    any_packed = ftl > 0 or names is not None
     model = binding.ZoqatModel(w, params, max_batch=w["batch"], max_seq=w["seq"], first_trainable_layer=ftl,
-                               packed_frozen=ftl > 0, gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05)
-    if ftl > 0:
+                               packed_frozen=any_packed, trainable_names=names, head_trainable=w.get("head_trainable", True),
+                               gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05)
+    if any_packed:
         model.zoqat_prequantize_frozen()
-        for l in range(ftl):                               # the fp32 copies of packed tensors are no longer needed
+        for l in range(w["n_layers"]):                     # the fp32 copies of packed tensors are no longer needed
             for name in synth.linear_shapes(w):
-                params["layers"][l][name] = None
+                if l < ftl or (names is not None and name not in names):
+                    params["layers"][l][name] = None
         torch.cuda.empty_cache()
     # weak scaling: each rank gets its own batch shard of the workload's size
     tok_np, lab_np = synth.make_batch(w["batch"], w["seq"], w["vocab"], seed=1234 + rank)
@@ -325,7 +331,7 @@ def run_ours(args, w, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b_w4a8")

@@ -54,6 +54,8 @@ class OracleConfig:
     rope_base: float = 10000.0
     first_trainable_layer: int = 0   # layers below are frozen (quantised from the unperturbed masters)
     head_trainable: bool = True
+    trainable_names: Optional[tuple] = None   # block linears that are trainable in the trainable layers (None = all);
+                                              # Section 4.3 keeps only the query and value projections trainable
     store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
                                      # residual stream) to binary32, as an implementation that keeps activations in
                                      # fp32 does; used only to measure how far two correct implementations can differ
@@ -129,12 +131,16 @@ class OracleModel:
     _ROLE = {"wq": ROLE_Q, "wk": ROLE_K, "wv": ROLE_V, "wo": ROLE_O, "w_gate": ROLE_GATE,
              "w_up": ROLE_UP, "w_down": ROLE_DOWN, "fc1": ROLE_FC1, "fc2": ROLE_FC2}
 
+    def is_trainable(self, l, name):
+        return l >= self.cfg.first_trainable_layer and (self.cfg.trainable_names is None or name in self.cfg.trainable_names)
+
     def trainable_tensors(self):
         """(array, tensor id) of every tensor Eq. (2) updates."""
         out = []
         for l in range(self.cfg.first_trainable_layer, self.cfg.n_layers):
             for n in self.linear_names():
-                out.append((self.p["layers"][l][n], tensor_id(l, self._ROLE[n])))
+                if self.is_trainable(l, n):
+                    out.append((self.p["layers"][l][n], tensor_id(l, self._ROLE[n])))
         if self.cfg.head_trainable:
             out.append((self.p["lm_head"], LM_HEAD_ID))
         return out
@@ -145,7 +151,7 @@ class OracleModel:
         (bfloat16-rounded dequantised value), float64 [out, in]."""
         cfg = self.cfg
         w = self.p["layers"][l][name]
-        if l >= cfg.first_trainable_layer and signed_eps != 0.0:
+        if self.is_trainable(l, name) and signed_eps != 0.0:
             w = core.perturb(w, seed, tensor_id(l, self._ROLE[name]), signed_eps)
         if cfg.w_bits == 0:
             deq = w

@@ -291,11 +291,13 @@ class ZoqatModel:
     (model-level entries plus ``layers``: a list of per-layer dicts).
     first_trainable_layer: block linears of earlier layers are frozen; with
     packed_frozen=True they are FROZEN_PACKED (Section 4.3), else quantised on
-    the fly from their fp32 values every pass.
+    the fly from their fp32 values every pass.  trainable_names: the block linears
+    that are trainable inside the trainable layers (None = all; Section 4.3 keeps
+    only ("wq", "wv")); the others are frozen like the earlier layers.
     """
 
     def __init__(self, shape, params, max_batch, max_seq, gemm_impl=GEMM_TCGEN05, first_trainable_layer=0,
-                 head_trainable=True, packed_frozen=False, norm_eps=1e-5, rope_base=10000.0):
+                 head_trainable=True, packed_frozen=False, norm_eps=1e-5, rope_base=10000.0, trainable_names=None):
         L = lib()
         self.shape = dict(shape)
         self.params = params
@@ -316,7 +318,7 @@ class ZoqatModel:
         for l, P in enumerate(params["layers"]):
             for name, t in P.items():
                 if name in _LINEAR_ROLES:
-                    if l >= first_trainable_layer:
+                    if l >= first_trainable_layer and (trainable_names is None or name in trainable_names):
                         descs.append(TensorDesc(_LINEAR_ROLES[name], l, TENSOR_TRAINABLE | TENSOR_QUANTIZED, 0, t.data_ptr(), None, None))
                     elif packed_frozen:
                         cb, qb = zoqat_packed_bytes(t.shape[0], t.shape[1], shape["w_bits"], shape["w_group"])

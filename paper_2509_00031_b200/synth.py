@@ -23,6 +23,10 @@ WORKLOADS = {
     "llama13b_light": dict(arch="llama", n_layers=40, d_model=5120, n_heads=40, d_ffn=13824, vocab=32000,
                            w_bits=4, w_group=128, a_bits=8, batch=8, seq=512, bf16_init=True,
                            first_trainable_layer=36),
+    # Section 4.3 as the paper runs it: only the query and value projections trainable, the rest packed
+    "llama7b_qv_light": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                             w_bits=4, w_group=128, a_bits=8, batch=4, seq=1024, bf16_init=True,
+                             trainable_names=("wq", "wv"), head_trainable=False),
 }
 
 

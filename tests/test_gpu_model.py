@@ -343,3 +343,33 @@ def test_step_multi_directions(zq):
     rb = zq.decode_step_result(b.zoqat_step_multi(td, ld, seed, 1, eps, lr)[0])
     assert ra == rb
     assert torch.equal(a.params["layers"][0]["wq"], b.params["layers"][0]["wq"]) and torch.equal(a.params["lm_head"], b.params["lm_head"])
+
+
+def test_query_value_only_selection(zq):
+    """Section 4.3 as the paper runs it: only the query and value projections keep full-precision masters and are
+    perturbed / updated; every other block linear is frozen and pre-quantised to packed codes."""
+    shape = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=512, w_bits=4, w_group=128, a_bits=8)
+    batch, seq = 2, 64
+    params = synth.make_params(shape, seed=5, max_seq=seq, jitter=True)
+    names = ("wq", "wv")
+    oracle = OracleModel(oracle_cfg(shape, trainable_names=names, head_trainable=False), synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, packed_frozen=True,
+                          trainable_names=names, head_trainable=False)
+    model.zoqat_prequantize_frozen()
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=17)
+    eps, lr, seed = 1e-3, 1e-4, 9
+    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), seed, eps, lr))
+    model.zoqat_check()
+    lp, lm, g = oracle.step(tokens, labels, seed, eps, lr)
+    assert res["status"] == 0
+    assert abs(res["loss_plus"] - lp) <= 1e-4 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-4 * abs(lm)
+    assert abs(res["proj_grad"] - g) <= 0.1 * max(abs(g), 1.0)
+    for l in range(2):
+        for n in oracle.linear_names():
+            got = model.params["layers"][l][n].cpu().numpy()
+            if n in names:
+                assert not np.array_equal(got, params["layers"][l][n])
+                assert np.abs(got - oracle.p["layers"][l][n]).max() <= 1e-5
+            else:
+                assert np.array_equal(got, params["layers"][l][n])
+    assert np.array_equal(model.params["lm_head"].cpu().numpy(), params["lm_head"])
