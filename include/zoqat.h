@@ -103,7 +103,7 @@ typedef struct zoqat_config {
     int32_t max_seq;       /* ... and sequence length a call will pass                            */
     int32_t w_bits;        /* 2, 3 or 4                                                           */
     int32_t w_group;       /* 32, 64 or 128; divides d_model and d_ffn                            */
-    int32_t a_bits;        /* 8 = per-token symmetric int8 on block-linear inputs, 0 = none        */
+    int32_t a_bits;        /* 4, 6 or 8 = per-token symmetric N-bit codes on block-linear inputs, 0 = none */
     int32_t gemm_impl;     /* ZOQAT_GEMM_*                                                        */
     float   norm_eps;
     float   rope_base;     /* LLaMA only                                                          */
@@ -279,7 +279,7 @@ int zoqat_op_update(float* w_dev, uint64_t n, uint64_t seed, uint32_t tensor_id,
 
 /* Optional normalisation followed by the activation operand of a linear:
  * norm_kind 0 none, 1 RMSNorm (gain), 2 LayerNorm (gain, bias);
- * a_bits 8: per-row symmetric int8 codes (as bf16 integers) + row step in
+ * a_bits 4 / 6 / 8: per-row symmetric N-bit codes (as bf16 integers) + row step in
  * row_step_dev; a_bits 0: bf16(x), row step 1.  x_dev fp32 [rows, cols];
  * operand_dev bf16 [rows, cols]; row_step_dev fp32 [rows];
  * normed_dev (may be NULL) fp32 [rows, cols] receives the normalised values. */

@@ -49,7 +49,7 @@ class OracleConfig:
     vocab: int
     w_bits: int = 4
     w_group: int = 128
-    a_bits: int = 8           # 8 = per-token symmetric int8 on block-linear inputs, 0 = none
+    a_bits: int = 8           # 4 / 6 / 8 = per-token symmetric N-bit codes on block-linear inputs, 0 = none
     norm_eps: float = 1e-5
     rope_base: float = 10000.0
     first_trainable_layer: int = 0   # layers below are frozen (quantised from the unperturbed masters)
@@ -62,18 +62,19 @@ class OracleConfig:
     operand_bf16: bool = True        # False (with w_bits = 0, a_bits = 0) gives the unquantised float64 model, used only to pin the forward
 
 
-def act_quant(x64):
-    """Per-token symmetric int8 quantiser (Section 2 symmetric form with N = 8:
-    Delta = max|x| / Q_P, z = 0, clamp to [-2^7, 2^7 - 1]); one Delta per row.
+def act_quant(x64, bits=8):
+    """Per-token symmetric N-bit quantiser (Section 2 symmetric form: Q_P = 2^(N-1) - 1,
+    Delta = max|x| / Q_P, z = 0, clamp to [-2^(N-1), 2^(N-1) - 1]); one Delta per row.
     The decision is taken in binary32.  Returns integer codes (float64 array)
     and the per-row Delta (float32)."""
     x = x64.astype(F32)
     amax = np.max(np.abs(x), axis=-1, keepdims=True).astype(F32)
-    s = (amax / F32(127.0)).astype(F32)
+    qp = float(2 ** (bits - 1) - 1)
+    s = (amax / F32(qp)).astype(F32)
     s = np.maximum(s, F32(1e-8))
     inv = (F32(1.0) / s).astype(F32)
     v = (x * inv).astype(F32)
-    q = np.clip(np.rint(v), -128.0, 127.0)
+    q = np.clip(np.rint(v), -qp - 1.0, qp)
     return q.astype(np.float64), s[..., 0]
 
 
@@ -170,8 +171,8 @@ class OracleModel:
 
     def lin(self, x, l, name, seed, signed_eps, bias=None):
         """x [T, in] float64 -> [T, out] float64 through the quantised linear."""
-        if self.cfg.a_bits == 8:
-            a, s = act_quant(x)
+        if self.cfg.a_bits:
+            a, s = act_quant(x, self.cfg.a_bits)
             y = (a @ self.block_operand(l, name, seed, signed_eps).T) * s.astype(np.float64)[:, None]
         else:
             a = self._operand_round(x)

@@ -1,7 +1,7 @@
 // Activation side of the forward pass outside the matrix multiplies: embedding
 // gather, RMSNorm / LayerNorm fused with the per-token activation quantiser
-// (Section 2 symmetric form, N = 8: step = max|x|/127, code = clamp(round(x/step),
-// -128, 127), one step per token), and the FFN non-linearity fused with the same
+// (Section 2 symmetric form, N = a_bits in {4, 6, 8}: Q_P = 2^(N-1) - 1, step = max|x|/Q_P,
+// code = clamp(round(x/step), -Q_P - 1, Q_P), one step per token), and the FFN non-linearity fused with the same
 // quantiser.  One CTA owns one token row, staged in shared memory; row statistics
 // are accumulated in double precision.  The operand written for the following
 // GEMM is bf16: the integer codes themselves (exact in bf16) with the step kept
@@ -42,16 +42,17 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 // Writes the operand row from the fp32 row held in shared memory.
 __device__ __forceinline__ void write_operand_row(const float* row, int cols, int a_bits, __nv_bfloat16* op_row,
                                                   float* row_step, float* redf) {
-    if (a_bits == 8) {
+    if (a_bits != 0) {
+        const float qmax = (float)((1 << (a_bits - 1)) - 1), qmin = -qmax - 1.0f;     // symmetric N-bit range
         float amax = 0.0f;
         for (int c = threadIdx.x; c < cols; c += kRowThreads) amax = fmaxf(amax, fabsf(row[c]));
         amax = block_max(amax, redf);
-        const float step = fmaxf(__fdiv_rn(amax, 127.0f), 1e-8f);
+        const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
         for (int c = 2 * threadIdx.x; c < cols; c += 2 * kRowThreads) {
-            const float q0 = fminf(fmaxf(rintf(__fmul_rn(row[c], inv)), -128.0f), 127.0f);
-            const float q1 = fminf(fmaxf(rintf(__fmul_rn(row[c + 1], inv)), -128.0f), 127.0f);
+            const float q0 = fminf(fmaxf(rintf(__fmul_rn(row[c], inv)), qmin), qmax);
+            const float q1 = fminf(fmaxf(rintf(__fmul_rn(row[c + 1], inv)), qmin), qmax);
             *reinterpret_cast<__nv_bfloat162*>(op_row + c) = __floats2bfloat162_rn(q0, q1);
         }
     } else {
@@ -130,22 +131,23 @@ __device__ __forceinline__ uint2 bf16x4(float a, float b, float c, float d) {
 template <int VPT>
 __device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n4, int a_bits, uint2* op_row, float* row_step,
                                                    float* redf) {
-    if (a_bits == 8) {
+    if (a_bits != 0) {
+        const float qmax = (float)((1 << (a_bits - 1)) - 1), qmin = -qmax - 1.0f;     // symmetric N-bit range
         float amax = 0.0f;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) amax = fmaxf(amax, amax4(v[i]));      // slots beyond the row hold zeros
         amax = block_max(amax, redf);
-        const float step = fmaxf(__fdiv_rn(amax, 127.0f), 1e-8f);
+        const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = threadIdx.x + i * kRowThreads;
             if (idx < n4)
-                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), -128.0f), 127.0f));
+                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), qmin), qmax));
         }
     } else {
         if (threadIdx.x == 0) *row_step = 1.0f;
@@ -278,18 +280,19 @@ rows_operand_reg_kernel(const float* __restrict__ x, int cols, const uint32_t* _
         const int idx = threadIdx.x + i * kRowThreads;
         v[i] = idx < n4 ? __ldcs(xr + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    if (a_bits == 8) {
-        const float step = fmaxf(__fdiv_rn(__uint_as_float(amax_bits[r]), 127.0f), 1e-8f);
+    if (a_bits != 0) {
+        const float qmax = (float)((1 << (a_bits - 1)) - 1), qmin = -qmax - 1.0f;     // symmetric N-bit range
+        const float step = fmaxf(__fdiv_rn(__uint_as_float(amax_bits[r]), qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) row_step[r] = step;
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = threadIdx.x + i * kRowThreads;
             if (idx < n4)
-                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), -128.0f), 127.0f),
-                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), -128.0f), 127.0f));
+                op_row[idx] = bf16x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), qmin), qmax),
+                                     fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), qmin), qmax));
         }
     } else {
         if (threadIdx.x == 0) row_step[r] = 1.0f;

@@ -127,7 +127,7 @@ int validate_config(const zoqat_config_t* c) {
     if (c->w_bits != 2 && c->w_bits != 3 && c->w_bits != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "w_bits %d (supported: 2, 3, 4)", c->w_bits);
     if (c->w_group != 32 && c->w_group != 64 && c->w_group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "w_group %d (supported: 32, 64, 128)", c->w_group);
     if (c->d_model % c->w_group || c->d_ffn % c->w_group) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
-    if (c->a_bits != 0 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 8)", c->a_bits);
+    if (c->a_bits != 0 && c->a_bits != 4 && c->a_bits != 6 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 4, 6, 8)", c->a_bits);
     if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT && c->gemm_impl != ZOQAT_GEMM_TCGEN05_1CTA) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
     if ((int64_t)c->max_batch * c->max_seq > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "max_batch*max_seq too large");
     return ZOQAT_OK;
@@ -747,7 +747,7 @@ int zoqat_op_norm_act_operand(const float* x_dev, int64_t rows, int64_t cols, in
     if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
     if (norm_kind < 0 || norm_kind > 2 || (norm_kind >= 1 && !gain_dev) || (norm_kind == 2 && !bias_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "bad norm arguments");
-    if (a_bits != 0 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
+    if (a_bits != 0 && a_bits != 4 && a_bits != 6 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
     launch_norm_act_operand(x_dev, rows, (int)cols, norm_kind, gain_dev, bias_dev, norm_eps, a_bits,
                             static_cast<__nv_bfloat16*>(operand_dev), row_step_dev, normed_dev, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
@@ -758,7 +758,7 @@ int zoqat_op_ffn_act_operand(const float* x_dev, int64_t rows, int64_t cols, int
                              float* row_step_dev, void* stream) {
     if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
-    if (a_bits != 0 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
+    if (a_bits != 0 && a_bits != 4 && a_bits != 6 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
     launch_ffn_act_operand(x_dev, rows, (int)cols, gated, a_bits, static_cast<__nv_bfloat16*>(operand_dev), row_step_dev,
                            static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());

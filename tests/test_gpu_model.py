@@ -60,11 +60,14 @@ SMALL_LLAMA = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=320, 
 SMALL_OPT = dict(arch="opt", n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=777, w_bits=4, w_group=128, a_bits=0)
 SMALL_W2 = dict(arch="llama", n_layers=1, d_model=256, n_heads=2, d_ffn=512, vocab=512, w_bits=2, w_group=64, a_bits=0)
 SMALL_W3A8 = dict(arch="opt", n_layers=1, d_model=128, n_heads=2, d_ffn=384, vocab=300, w_bits=3, w_group=32, a_bits=8)
+SMALL_W4A4 = dict(arch="llama", n_layers=2, d_model=256, n_heads=2, d_ffn=512, vocab=400, w_bits=4, w_group=128, a_bits=4)
+SMALL_W4A6 = dict(arch="opt", n_layers=1, d_model=128, n_heads=2, d_ffn=256, vocab=300, w_bits=4, w_group=64, a_bits=6)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("shape,batch,seq", [(SMALL_LLAMA, 2, 96), (SMALL_OPT, 3, 50), (SMALL_W2, 1, 130), (SMALL_W3A8, 2, 64)],
-                         ids=["llama_w4a8", "opt_w4", "llama_w2", "opt_w3a8"])
+@pytest.mark.parametrize("shape,batch,seq", [(SMALL_LLAMA, 2, 96), (SMALL_OPT, 3, 50), (SMALL_W2, 1, 130), (SMALL_W3A8, 2, 64),
+                                             (SMALL_W4A4, 2, 64), (SMALL_W4A6, 2, 64)],
+                         ids=["llama_w4a8", "opt_w4", "llama_w2", "opt_w3a8", "llama_w4a4", "opt_w4a6"])
 def test_forward_loss_matches_oracle(zq, impl, shape, batch, seq):
     model, oracle = build_pair(zq, shape, batch, seq, impl)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=11)

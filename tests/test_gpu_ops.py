@@ -156,6 +156,19 @@ def test_norm_act_operand(zq, kind, cols):
     assert np.array_equal(bf16_to_f32(op16), core.round_bf16(normed)) and np.all(step16.cpu().numpy() == 1.0)
 
 
+@pytest.mark.parametrize("bits", [4, 6])
+def test_low_bit_activation_codes(zq, bits):
+    """W-A settings below 8 activation bits: the codes of the GPU's own normalised row reproduce the oracle's
+    N-bit quantiser exactly."""
+    rng = np.random.default_rng(bits)
+    x = (rng.standard_normal((41, 2048)) * rng.uniform(0.2, 4.0, (41, 1))).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(2048)).astype(np.float32)
+    op, step, normed = zq.zoqat_op_norm_act_operand(dev(x), 1, dev(g), None, 1e-5, bits, want_normed=True)
+    q, s = act_quant(normed.cpu().numpy().astype(np.float64), bits)
+    assert np.array_equal(bf16_to_f32(op).astype(np.float64), q) and np.array_equal(step.cpu().numpy(), s)
+    assert q.max() == 2 ** (bits - 1) - 1 or q.min() == -(2 ** (bits - 1) - 1)
+
+
 @pytest.mark.parametrize("gated,cols", [(1, 1024), (0, 8192), (1, 11008)])
 def test_ffn_act_operand(zq, gated, cols):
     rng = np.random.default_rng(cols)

@@ -42,7 +42,7 @@ def test_query_workspace_and_validation(zq):
     assert L.zoqat_query_workspace(ctypes.byref(big), ctypes.byref(n)) == zq.OK
     assert n.value < 4 << 30          # scratch for the 7B shape stays far below the 26 GB of masters
     for field, bad, code in [("w_bits", 5, zq.ERR_UNSUPPORTED), ("w_group", 48, zq.ERR_UNSUPPORTED),
-                             ("a_bits", 4, zq.ERR_UNSUPPORTED), ("arch", 7, zq.ERR_INVALID_ARG),
+                             ("a_bits", 5, zq.ERR_UNSUPPORTED), ("arch", 7, zq.ERR_INVALID_ARG),
                              ("n_heads", 3, zq.ERR_INVALID_ARG), ("d_model", 200, zq.ERR_UNSUPPORTED)]:
         c2 = zq.Config.from_buffer_copy(cfg)
         setattr(c2, field, bad)

@@ -30,6 +30,13 @@ def test_symmetric_int8_hand_cases(case):
     assert float(s[0]) == case["delta"]
 
 
+@pytest.mark.parametrize("case", GOLD["symmetric_low_bits"], ids=lambda c: c["note"][:30])
+def test_symmetric_low_bit_hand_cases(case):
+    q, s = act_quant(np.array(case["x"], np.float64)[None, :], case["bits"])
+    assert q[0].tolist() == case["codes"]
+    assert float(s[0]) == case["delta"]
+
+
 def test_degenerate_group_and_zero_row():
     x = np.full((1, 8), 0.3, np.float32)
     codes, delta, zp, deq = core.weight_quant(x, 8, 4)
