@@ -130,8 +130,9 @@ __device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d)
 // Quantises the 16 values a thread holds (one (step, zero point) per group of LANES adjacent lanes) and returns
 // the dequantised values in place; codes (optional) receive the integer codes.
 //   code = clamp(round(x * inv) + zp, 0, qp),  value = (code - zp) * step
-// evaluated as value = clamp(round(x * inv), -zp, qp - zp) * step, which is the same number: all terms are
-// integers far below 2^24.  round() is to nearest even; when every |x * inv| of the warp is below 2^22 it is
+// evaluated as value = min(round(x * inv), qp - zp) * step, which is the same number: all terms are integers far
+// below 2^24, and the lower clamp can never act (x >= min of the group, multiplication by inv > 0 and rounding
+// are monotone, so round(x * inv) >= round(min * inv) = -zp).  round() is to nearest even; when every |x * inv| of the warp is below 2^22 it is
 // taken by adding and subtracting 1.5 * 2^23 (exact for such values), otherwise by rintf.
 template <int LANES>
 __device__ __forceinline__ GroupQ quantise16(float (&x)[16], float qp, float* codes) {
@@ -140,21 +141,21 @@ __device__ __forceinline__ GroupQ quantise16(float (&x)[16], float qp, float* co
     for (int j = 1; j < 16; ++j) { mn = fminf(mn, x[j]); mx = fmaxf(mx, x[j]); }
     group_minmax<LANES>(mn, mx);
     const GroupQ g = group_params(mn, mx, qp);
-    const float lo = -g.zp, hi = __fadd_rn(qp, -g.zp);
+    const float hi = __fadd_rn(qp, -g.zp);
     const bool small = __fmul_rn(fmaxf(fabsf(mn), fabsf(mx)), g.inv) < 4.0e6f;
     if (__all_sync(0xffffffffu, small)) {
         constexpr float kMagic = 12582912.0f;           // 1.5 * 2^23
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
             const float r = __fadd_rn(__fadd_rn(__fmul_rn(x[j], g.inv), kMagic), -kMagic);
-            const float c = fminf(fmaxf(r, lo), hi);
+            const float c = fminf(r, hi);
             if (codes) codes[j] = __fadd_rn(c, g.zp);
             x[j] = __fmul_rn(c, g.step);
         }
     } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            const float c = fminf(fmaxf(rintf(__fmul_rn(x[j], g.inv)), lo), hi);
+            const float c = fminf(rintf(__fmul_rn(x[j], g.inv)), hi);
             if (codes) codes[j] = __fadd_rn(c, g.zp);
             x[j] = __fmul_rn(c, g.step);
         }
