@@ -26,7 +26,7 @@ EPS, LR = 1e-3, 1e-6
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, averaged over the 129 GEMM
 # launches of one step, from the committed ncu capture (profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by
 # workload; absent for workloads that have not been captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 946.5e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 832.9e6}
 
 
 def load_peaks():
