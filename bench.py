@@ -248,7 +248,7 @@ def run_ours(args, w, rank, world, local_rank):
     model.zoqat_check()
     barrier()
     # ---- timed region: K steps, device-timed, per-category event pairs for the roofline of the dominant kernel
-    model.zoqat_profile_enable(True)
+    model.zoqat_profile_enable(1 if args.breakdown else 2)     # event pairs around the GEMM launches (all kernels with --breakdown)
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -311,7 +311,7 @@ def run_ours(args, w, rank, world, local_rank):
                       peak_source=peaks["source"] + " sustained bf16 (kernel timed inside a long step)",
                       launches_per_step=gemm_n / args.steps, avg_launch_ms=gemm_ms / max(gemm_n, 1),
                       traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)),
-        kernel_ms_per_step={k: v[0] / args.steps for k, v in prof.items()},
+        kernel_ms_per_step={k: v[0] / args.steps for k, v in prof.items() if v[1] > 0},
         gpu_launches=launches, clocks=clocks,
         last_step=dict(loss_plus=res["loss_plus"], loss_minus=res["loss_minus"], proj_grad=res["proj_grad"], status=res["status"]),
     )
@@ -337,6 +337,7 @@ def main():
     ap.add_argument("--workload", default="llama7b_w4a8")
     ap.add_argument("--simt", action="store_true", help="use the CUDA-core cross-check GEMM instead of tcgen05")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--breakdown", action="store_true", help="time every kernel category, not only the GEMM launches (adds ~1 %% to the step)")
     args = ap.parse_args()
     from paper_2509_00031_b200 import synth
     w = dict(synth.WORKLOADS[args.workload])

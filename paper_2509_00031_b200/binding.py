@@ -402,6 +402,7 @@ class ZoqatModel:
         return n.value
 
     def zoqat_profile_enable(self, on):
+        """on: 0 off, 1 (or True) every category, 2 the GEMM launches only."""
         _check(lib().zoqat_profile_enable(self.handle, int(on)))
 
     def zoqat_profile_read(self, category):

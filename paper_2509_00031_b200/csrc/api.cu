@@ -138,7 +138,7 @@ int validate_config(const zoqat_config_t* c) {
 // Optional per-category device timing: a CUDA event pair around every launch group.
 struct Profiler {
     static constexpr int kCats = ZOQAT_PROF_COUNT;
-    bool on = false;
+    int on = 0;                         // 0 off, 1 every category, 2 the GEMM launches only
     std::vector<cudaEvent_t> pool;
     std::vector<int> cat_of;            // category of event pair i
     size_t used = 0;                    // pairs in flight since the last read
@@ -181,7 +181,8 @@ namespace {
 
 struct ProfScope {
     Profiler& p; cudaStream_t s; size_t idx = 0; bool live;
-    ProfScope(zoqat_model* m, int cat, cudaStream_t st) : p(m->prof), s(st), live(m->prof.on) {
+    ProfScope(zoqat_model* m, int cat, cudaStream_t st)
+        : p(m->prof), s(st), live(m->prof.on == 1 || (m->prof.on == 2 && cat == ZOQAT_PROF_GEMM)) {
         if (!live) return;
         idx = p.used++;
         if (p.cat_of.size() <= idx) p.cat_of.resize(idx + 1);
@@ -634,7 +635,7 @@ int zoqat_launch_count(const zoqat_model_t* m, int64_t* launches) {
 
 int zoqat_profile_enable(zoqat_model_t* m, int on) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
-    m->prof.on = on != 0;
+    m->prof.on = (on == 2) ? 2 : (on != 0);
     return ZOQAT_OK;
 }
 
