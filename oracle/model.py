@@ -10,6 +10,11 @@ What it follows
     token (symmetric, 8 bit) for activations (Appendix "Quantization settings").
   * Section 4.3 (lightweight variant): frozen tensors are quantised from the
     unperturbed masters and are neither perturbed nor updated.
+  * Section 4.2 (optional): the adaptive weight quantiser (learnable step, zero point and
+    clipping coefficients per group) and the adaptive outlier smoothing (learnable
+    per-channel scale s and shift delta at the input of every block linear); both sets of
+    parameters are perturbed and updated by the same two-point estimate as the weights,
+    each class with its own learning rate (hyperparameter table of the appendix).
 
 Precision: float64 for every sum (linear layers, norms, softmax, loss).  The
 numbers that decide integer codes or operand roundings are taken in binary32,
@@ -39,6 +44,54 @@ def tensor_id(layer: int, role: int) -> int:
     return 16 * (layer + 1) + role
 
 
+# Section 4.2 parameters live in the same counter space under their own tensor ids:
+# quantiser parameters of a linear = its weight's id + QPARAM_ID; smoothing scale / shift of
+# quantisation point p of a layer = SMOOTH_SCALE_ID / SMOOTH_SHIFT_ID + 16*(layer+1) + p.
+QPARAM_ID = 0x10000
+SMOOTH_SCALE_ID = 0x20000
+SMOOTH_SHIFT_ID = 0x30000
+# the four inputs of block linears that are quantised (and smoothed): which linears read them
+POINTS = ("attn_in", "attn_out", "ffn_in", "ffn_out")
+POINT_OF = {"wq": 0, "wk": 0, "wv": 0, "wo": 1, "w_gate": 2, "w_up": 2, "fc1": 2, "w_down": 3, "fc2": 3}
+
+
+def adaptive_weight_quant(w, theta, group, bits):
+    """Adaptive weight quantiser of Section 4.2:
+        code = clamp(round(w / Delta) + z, alpha * Q_P, beta * Q_P),   value = (code - z) * Delta
+    with one learnable (Delta, z, alpha, beta) per group of `group` consecutive input
+    channels: theta float32 [rows, cols/group, 4].  Codes stay integers in [0, Q_P]: the zero
+    point and the two clipping levels enter rounded to the nearest integer (ties to even),
+    the levels limited to [0, Q_P] and the upper one to at least the lower one; Delta is
+    floored at 1e-8 and w / Delta is w * (1 / Delta) with the reciprocal rounded once, as in
+    the min/max quantiser.  All decisions in binary32.
+    Returns (codes, dequantised values), float32 [rows, cols]."""
+    w = np.ascontiguousarray(w, dtype=F32)
+    rows, cols = w.shape
+    x = w.reshape(rows, cols // group, group)
+    th = np.asarray(theta, dtype=F32).reshape(rows, cols // group, 4)
+    qp = F32(2 ** bits - 1)
+    d = np.maximum(th[..., 0], F32(1e-8))[..., None]
+    inv = (F32(1.0) / d).astype(F32)
+    zr = np.rint(th[..., 1])[..., None]
+    lo = np.clip(np.rint((th[..., 2] * qp).astype(F32)), F32(0), qp)
+    hi = np.clip(np.rint((th[..., 3] * qp).astype(F32)), lo, qp)
+    q = np.clip((np.rint((x * inv).astype(F32)) + zr).astype(F32), lo[..., None], hi[..., None])
+    deq = ((q - zr).astype(F32) * d).astype(F32)
+    return q.reshape(rows, cols), deq.reshape(rows, cols)
+
+
+def init_quant_params(w, group, bits):
+    """Initial (Delta, z, alpha, beta) per group: Delta and z from the default asymmetric
+    min/max scheme on the unperturbed weights, alpha = 0, beta = 1 (Section 4.2)."""
+    _, delta, zp, _ = core.weight_quant(w, group, bits)
+    th = np.empty(delta.shape + (4,), F32)
+    th[..., 0] = delta
+    th[..., 1] = zp.astype(F32)
+    th[..., 2] = 0.0
+    th[..., 3] = 1.0
+    return th
+
+
 @dataclass
 class OracleConfig:
     arch: str                 # "llama" (RMSNorm, RoPE, SiLU-gated FFN) or "opt" (LayerNorm, learned positions, ReLU FFN, biases)
@@ -56,6 +109,10 @@ class OracleConfig:
     head_trainable: bool = True
     trainable_names: Optional[tuple] = None   # block linears that are trainable in the trainable layers (None = all);
                                               # Section 4.3 keeps only the query and value projections trainable
+    adaptive_quant: bool = False     # Section 4.2: trainable block linears use the learnable quantiser ('theta_<name>')
+    smoothing: bool = False          # Section 4.2: learnable per-channel scale / shift at the inputs of the block linears
+                                     # of the trainable layers ('smooth_s_<point>', 'smooth_d_<point>'); needs
+                                     # trainable_names = None
     store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
                                      # residual stream) to binary32, as an implementation that keeps activations in
                                      # fp32 does; used only to measure how far two correct implementations can differ
@@ -135,27 +192,81 @@ class OracleModel:
     def is_trainable(self, l, name):
         return l >= self.cfg.first_trainable_layer and (self.cfg.trainable_names is None or name in self.cfg.trainable_names)
 
+    def has_smoothing(self, l):
+        return self.cfg.smoothing and l >= self.cfg.first_trainable_layer
+
+    def has_adaptive(self, l, name):
+        return self.cfg.adaptive_quant and self.cfg.w_bits != 0 and self.is_trainable(l, name)
+
+    def init_learnable(self):
+        """Adds the Section 4.2 parameters at their initial values: quantiser parameters from the
+        min/max scheme of the current weights, smoothing scale 1 and shift 0 (the model is then
+        the same function as without them)."""
+        cfg = self.cfg
+        for l in range(cfg.first_trainable_layer, cfg.n_layers):
+            P = self.p["layers"][l]
+            for n in self.linear_names():
+                if self.has_adaptive(l, n):
+                    P["theta_" + n] = init_quant_params(P[n], cfg.w_group, cfg.w_bits)
+            if self.has_smoothing(l):
+                for n in self.linear_names():
+                    pt = POINTS[POINT_OF[n]]
+                    P["smooth_s_" + pt] = np.ones(P[n].shape[1], F32)
+                    P["smooth_d_" + pt] = np.zeros(P[n].shape[1], F32)
+
     def trainable_tensors(self):
-        """(array, tensor id) of every tensor Eq. (2) updates."""
+        """(array, tensor id, class) of every tensor Eq. (2) updates; class 'w' (weights),
+        'q' (quantiser parameters) or 's' (smoothing parameters) selects the learning rate."""
         out = []
         for l in range(self.cfg.first_trainable_layer, self.cfg.n_layers):
+            P = self.p["layers"][l]
             for n in self.linear_names():
                 if self.is_trainable(l, n):
-                    out.append((self.p["layers"][l][n], tensor_id(l, self._ROLE[n])))
+                    out.append((P[n], tensor_id(l, self._ROLE[n]), "w"))
+                    if self.has_adaptive(l, n):
+                        out.append((P["theta_" + n], tensor_id(l, self._ROLE[n]) + QPARAM_ID, "q"))
+            if self.has_smoothing(l):
+                for i, pt in enumerate(POINTS):
+                    out.append((P["smooth_s_" + pt], SMOOTH_SCALE_ID + tensor_id(l, i), "s"))
+                    out.append((P["smooth_d_" + pt], SMOOTH_SHIFT_ID + tensor_id(l, i), "s"))
         if self.cfg.head_trainable:
-            out.append((self.p["lm_head"], LM_HEAD_ID))
+            out.append((self.p["lm_head"], LM_HEAD_ID, "w"))
         return out
 
     # -- operands ----------------------------------------------------------------
-    def block_operand(self, l, name, seed, signed_eps):
-        """Fake-quantised weight of a block linear as the matmul sees it
-        (bfloat16-rounded dequantised value), float64 [out, in]."""
-        cfg = self.cfg
+    def smoothing_params(self, l, name, seed, signed_eps):
+        """(s, delta) of the quantisation point `name` reads, perturbed like every learnable tensor."""
+        i = POINT_OF[name]
+        P = self.p["layers"][l]
+        s_ = P["smooth_s_" + POINTS[i]]
+        d_ = P["smooth_d_" + POINTS[i]]
+        if signed_eps != 0.0:
+            s_ = core.perturb(s_, seed, SMOOTH_SCALE_ID + tensor_id(l, i), signed_eps)
+            d_ = core.perturb(d_, seed, SMOOTH_SHIFT_ID + tensor_id(l, i), signed_eps)
+        return s_, d_
+
+    def perturbed_weight(self, l, name, seed, signed_eps):
         w = self.p["layers"][l][name]
         if self.is_trainable(l, name) and signed_eps != 0.0:
             w = core.perturb(w, seed, tensor_id(l, self._ROLE[name]), signed_eps)
+        return w
+
+    def block_operand(self, l, name, seed, signed_eps):
+        """Fake-quantised weight of a block linear as the matmul sees it
+        (bfloat16-rounded dequantised value), float64 [out, in].  With smoothing the quantiser
+        sees s (.) W (Section 4.2, first equation)."""
+        cfg = self.cfg
+        w = self.perturbed_weight(l, name, seed, signed_eps)
+        if self.has_smoothing(l):
+            s_, _ = self.smoothing_params(l, name, seed, signed_eps)
+            w = (w * s_[None, :]).astype(F32)
         if cfg.w_bits == 0:
             deq = w
+        elif self.has_adaptive(l, name):
+            th = self.p["layers"][l]["theta_" + name]
+            if signed_eps != 0.0:
+                th = core.perturb(th, seed, tensor_id(l, self._ROLE[name]) + QPARAM_ID, signed_eps)
+            _, deq = adaptive_weight_quant(w, th, cfg.w_group, cfg.w_bits)
         else:
             _, _, _, deq = core.weight_quant(w, cfg.w_group, cfg.w_bits)
         return (core.round_bf16(deq) if cfg.operand_bf16 else deq).astype(np.float64)
@@ -170,7 +281,15 @@ class OracleModel:
         return core.round_bf16(x.astype(F32)).astype(np.float64) if self.cfg.operand_bf16 else x
 
     def lin(self, x, l, name, seed, signed_eps, bias=None):
-        """x [T, in] float64 -> [T, out] float64 through the quantised linear."""
+        """x [T, in] float64 -> [T, out] float64 through the quantised linear.  With smoothing
+        (Section 4.2): Y = Q_a((X - delta) / s) Q_w(s (.) W)^T + (B + delta W^T), the division taken in
+        binary32 as a multiplication by 1/s rounded once, the shift term with the unquantised W."""
+        extra = None
+        if self.has_smoothing(l):
+            s_, d_ = self.smoothing_params(l, name, seed, signed_eps)
+            inv = (F32(1.0) / s_).astype(F32)
+            x = (((x.astype(F32) - d_[None, :]).astype(F32)) * inv[None, :]).astype(F32).astype(np.float64)
+            extra = self.perturbed_weight(l, name, seed, signed_eps).astype(np.float64) @ d_.astype(np.float64)
         if self.cfg.a_bits:
             a, s = act_quant(x, self.cfg.a_bits)
             y = (a @ self.block_operand(l, name, seed, signed_eps).T) * s.astype(np.float64)[:, None]
@@ -179,6 +298,8 @@ class OracleModel:
             y = a @ self.block_operand(l, name, seed, signed_eps).T
         if bias is not None:
             y = y + bias.astype(np.float64)[None, :]
+        if extra is not None:
+            y = y + extra[None, :]
         return self._store(y)
 
     def _store(self, x):
@@ -267,15 +388,21 @@ class OracleModel:
         g = F32((lp - lm) / (2.0 * float(eps32)))
         return lp, lm, g
 
-    def apply_update(self, seed, scale):
-        """W <- W - scale * u(seed) on every trainable tensor, in place (binary32 fma)."""
-        for w, tid in self.trainable_tensors():
-            core.update_(w, seed, tid, F32(scale))
+    def apply_update(self, seed, scale, scale_quant=None, scale_smooth=None):
+        """W <- W - scale * u(seed) on every trainable tensor, in place (binary32 fma); quantiser and
+        smoothing parameters use their own factors (default: the same one)."""
+        by_class = {"w": F32(scale), "q": F32(scale if scale_quant is None else scale_quant),
+                    "s": F32(scale if scale_smooth is None else scale_smooth)}
+        for w, tid, cls in self.trainable_tensors():
+            core.update_(w.reshape(-1), seed, tid, by_class[cls])
 
-    def step(self, tokens, labels, seed, eps, lr):
+    def step(self, tokens, labels, seed, eps, lr, lr_quant=None, lr_smooth=None):
+        """One step.  lr_quant / lr_smooth: learning rates of the quantiser ("clipping") and smoothing
+        parameters of Section 4.2 (default lr)."""
         lp, lm, g = self.projected_gradient(tokens, labels, seed, eps)
-        scale = F32(F32(lr) * g)
-        self.apply_update(seed, scale)
+        lrq = lr if lr_quant is None else lr_quant
+        lrs = lr if lr_smooth is None else lr_smooth
+        self.apply_update(seed, F32(F32(lr) * g), F32(F32(lrq) * g), F32(F32(lrs) * g))
         return lp, lm, float(g)
 
     def step_multi(self, tokens, labels, seed, n_dirs, eps, lr):
