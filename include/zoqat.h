@@ -79,13 +79,27 @@ extern "C" {
 #define ZOQAT_ROLE_FINAL_NORM_G 19
 #define ZOQAT_ROLE_FINAL_NORM_B 20   /* OPT only */
 #define ZOQAT_ROLE_LM_HEAD      21
-#define ZOQAT_ROLE_COUNT        22
+/* Section 4.2, adaptive outlier smoothing: per-input-channel scale s and shift delta at the four quantised
+ * inputs of a layer's linears (point 0: input of q/k/v, 1: input of the output projection, 2: input of
+ * gate/up (fc1), 3: input of down (fc2)); fp32 vectors of d_model (d_ffn for point 3) elements, layer >= 0.
+ * Role = base + point.  A layer has either all eight or none; with them every block linear of the layer must
+ * be TRAINABLE.  They are perturbed and updated like the weights: Philox tensor ids
+ * 0x20000 + 16*(layer+1) + point (scale) and 0x30000 + 16*(layer+1) + point (shift). */
+#define ZOQAT_ROLE_SMOOTH_SCALE 22   /* .. 25 */
+#define ZOQAT_ROLE_SMOOTH_SHIFT 26   /* .. 29 */
+#define ZOQAT_ROLE_COUNT        30
 
 /* Tensor flags (linear weights only; every other tensor is frozen fp32). */
 #define ZOQAT_TENSOR_TRAINABLE      1u  /* perturbed by +/- eps u in the forward, updated by Eq. (2) */
 #define ZOQAT_TENSOR_QUANTIZED      2u  /* forward sees the per-group fake-quantised weight         */
 #define ZOQAT_TENSOR_FROZEN_PACKED  4u  /* Section 4.3: forward reads packed codes + (step, zero point) written by
                                            zoqat_prequantize_frozen(); never perturbed, never updated */
+#define ZOQAT_TENSOR_ADAPTIVE       8u  /* Section 4.2 adaptive weight quantiser (with TRAINABLE | QUANTIZED): `qparams` holds
+                                           one learnable (step, zero point, alpha, beta) per group, code =
+                                           clamp(round(w/step) + z, alpha*Q_P, beta*Q_P); perturbed and updated like
+                                           the weights under Philox tensor id 0x10000 + the weight's id, element
+                                           4*group + {0,1,2,3}.  Codes stay integers in [0, Q_P]: z and the two levels
+                                           enter rounded to nearest even, the levels limited to [0, Q_P], upper >= lower */
 
 #define ZOQAT_GEMM_TCGEN05 0   /* tcgen05/TMEM tensor-core kernels (default); GEMM tiles of 256 rows are computed by a
                                   pair of CTAs on two SMs with one cta_group::2 MMA                                  */
@@ -117,7 +131,9 @@ typedef struct zoqat_tensor_desc {
     void*   data;          /* dev: fp32 values.  For FROZEN_PACKED tensors it is read only by
                               zoqat_prequantize_frozen() and may be freed afterwards.            */
     void*   packed;        /* dev: FROZEN_PACKED only, zoqat_packed_bytes() code bytes             */
-    void*   qparams;       /* dev: FROZEN_PACKED only, one (float step, float zero point) pair per group */
+    void*   qparams;       /* dev: FROZEN_PACKED: one (float step, float zero point) pair per group;
+                              ADAPTIVE: four floats (step, zero point, alpha, beta) per group, 16-byte aligned,
+                              updated in place (zoqat_init_qparams() writes the initial values)         */
 } zoqat_tensor_desc_t;
 
 typedef struct zoqat_step_result {
@@ -155,6 +171,12 @@ int zoqat_model_destroy(zoqat_model_t* m);
  * forward when such tensors exist. */
 int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream);
 
+/* Section 4.2: writes the initial quantiser parameters of every ADAPTIVE tensor - step and zero point of the
+ * default min/max scheme on the current (unperturbed) weights, alpha = 0, beta = 1 - at which the adaptive
+ * quantiser reproduces the min/max quantiser exactly.  (Smoothing vectors are the caller's to initialise:
+ * scale 1 and shift 0 leave the model unchanged.) */
+int zoqat_init_qparams(zoqat_model_t* m, void* stream);
+
 /* One forward pass: *loss_out_dev = L(Q(W + signed_eps u(seed)); B), the mean
  * next-token cross-entropy over positions whose label is >= 0 (Eq. (1) argument).
  * signed_eps = 0 gives the unperturbed quantised model.  tokens_dev / labels_dev:
@@ -170,6 +192,13 @@ int zoqat_forward_loss(zoqat_model_t* m, const int32_t* tokens_dev, const int32_
 int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
                int batch, int seq, uint64_t seed, float eps, float lr,
                zoqat_step_result_t* result_dev, void* stream);
+
+/* zoqat_step with one learning rate per parameter class (hyperparameter table of the appendix: the weights, the
+ * quantiser parameters of ADAPTIVE tensors - its "clipping" rate -, the smoothing vectors).  All classes share the
+ * one g of Eq. (1); class c moves by -fl(lr_c * g) u.  zoqat_step(lr) is zoqat_step_rates(lr, lr, lr). */
+int zoqat_step_rates(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                     int batch, int seq, uint64_t seed, float eps, float lr, float lr_quant, float lr_smooth,
+                     zoqat_step_result_t* result_dev, void* stream);
 
 /* Eq. (1) with q = n_dirs directions per step (the paper's estimator averages over q directions u_1..u_q; it never
  * states q): direction i uses seed + i, every g_i is the two-point estimate at the SAME weights, and Eq. (2) then
@@ -192,6 +221,8 @@ int zoqat_step_begin(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
                      int batch, int seq, uint64_t seed, float eps, double* sums_dev, void* stream);
 int zoqat_step_finish(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
                       zoqat_step_result_t* result_dev, void* stream);
+int zoqat_step_finish_rates(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                            float lr_quant, float lr_smooth, zoqat_step_result_t* result_dev, void* stream);
 
 /* Same step with HOST inputs and outputs: copies tokens/labels to the device,
  * runs zoqat_step, copies the result back and synchronises the stream. */
@@ -199,8 +230,11 @@ int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t*
                     int batch, int seq, uint64_t seed, float eps, float lr,
                     zoqat_step_result_t* result_host, void* stream);
 
-/* Eq. (2) alone: W <- W - scale * u(seed) on every TRAINABLE tensor. */
+/* Eq. (2) alone: W <- W - scale * u(seed) on every TRAINABLE tensor (and on the Section 4.2 parameters);
+ * the _rates form takes one factor per parameter class. */
 int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream);
+int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float scale_quant, float scale_smooth,
+                             void* stream);
 
 /* Synchronises `stream` and returns ZOQAT_OK, ZOQAT_ERR_TIMEOUT if a bounded
  * device wait ran out since the last check, or ZOQAT_ERR_CUDA. */
@@ -267,6 +301,38 @@ int zoqat_op_weight_quant(const float* w_dev, int64_t rows, int64_t cols, int gr
 int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
                                  uint64_t seed, uint32_t tensor_id, float eps,
                                  void* operand_plus_dev, void* operand_minus_dev, void* stream);
+
+/* The weight producer with the learnable parts of Section 4.2, on one [rows, cols] tensor.
+ *   theta_dev (may be NULL = min/max quantiser): fp32 [rows, cols/group, 4] = (step, zero point, alpha, beta) per
+ *     group, perturbed by +/- eps u under tensor id 0x10000 + tensor_id.
+ *   smooth_dev (may be NULL = no smoothing): fp32 [2][3][cols], the vectors zoqat_op_smooth_perturb wrote: the
+ *     quantiser sees scale' (.) w', and bias_dev[sign * rows + r] = bias0_dev[r] (or 0) + sum_k shift'[k] * w'[r, k]
+ *     (first equation of Section 4.2: the smoothed bias uses the unscaled, unquantised perturbed weight).
+ *     scratch_dev: 2 * rows * cols / group floats.
+ * operand_minus_dev may be NULL: one operand (and one bias vector) with eps signed.
+ * codes_dev (may be NULL): uint8 [rows, cols] codes of the +eps side. */
+int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
+                                    uint64_t seed, uint32_t tensor_id, float eps,
+                                    const float* theta_dev, const float* smooth_dev,
+                                    const float* bias0_dev, float* bias_dev, float* scratch_dev,
+                                    void* operand_plus_dev, void* operand_minus_dev, uint8_t* codes_dev, void* stream);
+
+/* Perturbed smoothing vectors of one quantisation point (Section 4.2): out_dev fp32 [2][3][cols] =
+ * [sign][scale' | shift' | 1/scale'], scale' = scale +/- eps u(seed, scale_id), shift' likewise with shift_id;
+ * sign 0 is +eps, sign 1 is -eps.  cols % 4 == 0. */
+int zoqat_op_smooth_perturb(const float* scale_dev, const float* shift_dev, int64_t cols, uint64_t seed,
+                            uint32_t scale_id, uint32_t shift_id, float eps, float* out_dev, void* stream);
+
+/* zoqat_op_norm_act_operand with the activation side of the smoothing: the quantiser sees
+ * (x - shift') * (1/scale') (both operations rounded once) with the vectors of sign 0 of smooth_dev
+ * (zoqat_op_smooth_perturb layout) for rows [0, rows_per_pass) and of sign 1 for the rest. */
+int zoqat_op_smooth_act_operand(const float* x_dev, int64_t rows, int64_t cols, int norm_kind, const float* gain_dev,
+                                const float* bias_dev, float norm_eps, int a_bits, const float* smooth_dev,
+                                int64_t rows_per_pass, void* operand_dev, float* row_step_dev, void* stream);
+
+/* Initial quantiser parameters of one tensor (what zoqat_init_qparams writes): theta_dev fp32 [rows, cols/group, 4]. */
+int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, float* theta_dev,
+                          void* stream);
 
 /* Packing of Section 4.3: quantise W (unperturbed) into packed codes + qparams,
  * and expansion of a packed tensor into the bf16 operand. */

@@ -17,7 +17,9 @@ ARCH_LLAMA, ARCH_OPT = 0, 1
 (ROLE_WQ, ROLE_WK, ROLE_WV, ROLE_WO, ROLE_W_GATE, ROLE_W_UP, ROLE_W_DOWN, ROLE_ATTN_NORM_G, ROLE_ATTN_NORM_B,
  ROLE_FFN_NORM_G, ROLE_FFN_NORM_B, ROLE_BQ, ROLE_BK, ROLE_BV, ROLE_BO, ROLE_B_FC1, ROLE_B_FC2, ROLE_EMBED,
  ROLE_POS_EMBED, ROLE_FINAL_NORM_G, ROLE_FINAL_NORM_B, ROLE_LM_HEAD) = range(22)
-TENSOR_TRAINABLE, TENSOR_QUANTIZED, TENSOR_FROZEN_PACKED = 1, 2, 4
+ROLE_SMOOTH_SCALE, ROLE_SMOOTH_SHIFT = 22, 26      # + quantisation point 0..3 (Section 4.2)
+SMOOTH_POINTS = ("attn_in", "attn_out", "ffn_in", "ffn_out")
+TENSOR_TRAINABLE, TENSOR_QUANTIZED, TENSOR_FROZEN_PACKED, TENSOR_ADAPTIVE = 1, 2, 4, 8
 GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_1CTA = 0, 1, 2
 BUF_RESIDUAL, BUF_QKV, BUF_ATTN, BUF_FFN, BUF_TOKEN_LOSS = range(5)
 PROF_GEMM, PROF_WEIGHT, PROF_ACT, PROF_ATTENTION, PROF_LOSS, PROF_UPDATE = range(6)
@@ -25,9 +27,11 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
-    "zoqat_prequantize_frozen", "zoqat_forward_loss", "zoqat_step", "zoqat_step_multi", "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_host", "zoqat_apply_update",
+    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_multi",
+    "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_apply_update", "zoqat_apply_update_rates",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
+    "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
     "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
@@ -80,6 +84,14 @@ def lib():
             "zoqat_model_create": [P(Config), P(TensorDesc), i32, vp, sz, P(vp)],
             "zoqat_model_destroy": [vp],
             "zoqat_prequantize_frozen": [vp, vp],
+            "zoqat_init_qparams": [vp, vp],
+            "zoqat_step_rates": [vp, vp, vp, i32, i32, u64, f32, f32, f32, f32, vp, vp],
+            "zoqat_step_finish_rates": [vp, vp, u64, f32, f32, f32, f32, vp, vp],
+            "zoqat_apply_update_rates": [vp, u64, f32, f32, f32, vp],
+            "zoqat_op_weight_operand_learned": [vp, i64, i64, i32, i32, u64, u32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "zoqat_op_smooth_perturb": [vp, vp, i64, u64, u32, u32, f32, vp, vp],
+            "zoqat_op_smooth_act_operand": [vp, i64, i64, i32, vp, vp, f32, i32, vp, i64, vp, vp, vp],
+            "zoqat_op_init_qparams": [vp, i64, i64, i32, i32, vp, vp],
             "zoqat_forward_loss": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step": [vp, vp, vp, i32, i32, u64, f32, f32, vp, vp],
             "zoqat_step_multi": [vp, vp, vp, i32, i32, u64, i32, f32, f32, vp, vp],
@@ -164,6 +176,46 @@ def zoqat_op_weight_operand_pair(w, group, bits, seed, tensor_id, eps):
     minus = torch.empty_like(plus)
     _check(lib().zoqat_op_weight_operand_pair(_p(w), rows, cols, group, bits, seed, tensor_id, eps, _p(plus), _p(minus), _stream()))
     return plus, minus
+
+
+def zoqat_op_init_qparams(w, group, bits):
+    rows, cols = w.shape
+    theta = torch.empty((rows, cols // group, 4), dtype=torch.float32, device=w.device)
+    _check(lib().zoqat_op_init_qparams(_p(w), rows, cols, group, bits, _p(theta), _stream()))
+    return theta
+
+
+def zoqat_op_smooth_perturb(scale, shift, seed, scale_id, shift_id, eps):
+    """-> float32 [2, 3, cols]: [sign][scale', shift', 1/scale']."""
+    cols = scale.numel()
+    out = torch.empty((2, 3, cols), dtype=torch.float32, device=scale.device)
+    _check(lib().zoqat_op_smooth_perturb(_p(scale), _p(shift), cols, seed, scale_id, shift_id, eps, _p(out), _stream()))
+    return out
+
+
+def zoqat_op_weight_operand_learned(w, group, bits, seed, tensor_id, eps, theta=None, smooth=None, bias0=None,
+                                    dual=True, want_codes=False):
+    """-> (operand_plus, operand_minus or None, bias [signs, rows] or None, codes or None)."""
+    rows, cols = w.shape
+    plus = torch.empty((rows, cols), dtype=torch.bfloat16, device=w.device)
+    minus = torch.empty_like(plus) if dual else None
+    bias = scratch = None
+    if smooth is not None:
+        bias = torch.empty((2 if dual else 1, rows), dtype=torch.float32, device=w.device)
+        scratch = torch.empty(2 * rows * (cols // group), dtype=torch.float32, device=w.device)
+    codes = torch.empty((rows, cols), dtype=torch.uint8, device=w.device) if want_codes else None
+    _check(lib().zoqat_op_weight_operand_learned(_p(w), rows, cols, group, bits, seed, tensor_id, eps, _p(theta), _p(smooth),
+                                                 _p(bias0), _p(bias), _p(scratch), _p(plus), _p(minus), _p(codes), _stream()))
+    return plus, minus, bias, codes
+
+
+def zoqat_op_smooth_act_operand(x, norm_kind, gain, bias, norm_eps, a_bits, smooth, rows_per_pass):
+    rows, cols = x.shape
+    operand = torch.empty((rows, cols), dtype=torch.bfloat16, device=x.device)
+    row_step = torch.empty(rows, dtype=torch.float32, device=x.device)
+    _check(lib().zoqat_op_smooth_act_operand(_p(x), rows, cols, norm_kind, _p(gain), _p(bias), norm_eps, a_bits, _p(smooth),
+                                             rows_per_pass, _p(operand), _p(row_step), _stream()))
+    return operand, row_step
 
 
 def zoqat_packed_bytes(rows, cols, bits, group):
@@ -294,10 +346,15 @@ class ZoqatModel:
     the fly from their fp32 values every pass.  trainable_names: the block linears
     that are trainable inside the trainable layers (None = all; Section 4.3 keeps
     only ("wq", "wv")); the others are frozen like the earlier layers.
+    adaptive_quant / smoothing (Section 4.2): trainable block linears get learnable quantiser
+    parameters (layer entry ``theta_<name>``, float32 [out, in/group, 4]; created here when absent -
+    call zoqat_init_qparams() to fill them) and the trainable layers get smoothing vectors
+    (``smooth_s_<point>``, ``smooth_d_<point>``; created as ones / zeros when absent).
     """
 
     def __init__(self, shape, params, max_batch, max_seq, gemm_impl=GEMM_TCGEN05, first_trainable_layer=0,
-                 head_trainable=True, packed_frozen=False, norm_eps=1e-5, rope_base=10000.0, trainable_names=None):
+                 head_trainable=True, packed_frozen=False, norm_eps=1e-5, rope_base=10000.0, trainable_names=None,
+                 adaptive_quant=False, smoothing=False):
         L = lib()
         self.shape = dict(shape)
         self.params = params
@@ -316,10 +373,26 @@ class ZoqatModel:
                 flags = TENSOR_TRAINABLE if (name == "lm_head" and head_trainable) else 0
                 descs.append(TensorDesc(role, -1, flags, 0, params[name].data_ptr(), None, None))
         for l, P in enumerate(params["layers"]):
-            for name, t in P.items():
-                if name in _LINEAR_ROLES:
+            if smoothing and l >= first_trainable_layer:
+                for i, pt in enumerate(SMOOTH_POINTS):
+                    n = shape["d_ffn"] if i == 3 else shape["d_model"]
+                    P.setdefault("smooth_s_" + pt, torch.ones(n, dtype=torch.float32, device="cuda"))
+                    P.setdefault("smooth_d_" + pt, torch.zeros(n, dtype=torch.float32, device="cuda"))
+            for name, t in list(P.items()):
+                if name.startswith("theta_"):
+                    continue
+                if name.startswith("smooth_s_") or name.startswith("smooth_d_"):
+                    base = ROLE_SMOOTH_SCALE if name.startswith("smooth_s_") else ROLE_SMOOTH_SHIFT
+                    descs.append(TensorDesc(base + SMOOTH_POINTS.index(name[9:]), l, 0, 0, t.data_ptr(), None, None))
+                elif name in _LINEAR_ROLES:
                     if l >= first_trainable_layer and (trainable_names is None or name in trainable_names):
-                        descs.append(TensorDesc(_LINEAR_ROLES[name], l, TENSOR_TRAINABLE | TENSOR_QUANTIZED, 0, t.data_ptr(), None, None))
+                        flags, th = TENSOR_TRAINABLE | TENSOR_QUANTIZED, None
+                        if adaptive_quant:
+                            th = P.setdefault("theta_" + name, torch.empty((t.shape[0], t.shape[1] // shape["w_group"], 4),
+                                                                           dtype=torch.float32, device="cuda"))
+                            flags |= TENSOR_ADAPTIVE
+                        descs.append(TensorDesc(_LINEAR_ROLES[name], l, flags, 0, t.data_ptr(), None,
+                                                th.data_ptr() if th is not None else None))
                     elif packed_frozen:
                         cb, qb = zoqat_packed_bytes(t.shape[0], t.shape[1], shape["w_bits"], shape["w_group"])
                         pk = torch.empty(cb, dtype=torch.uint8, device="cuda")
@@ -349,6 +422,24 @@ class ZoqatModel:
 
     def zoqat_prequantize_frozen(self):
         _check(lib().zoqat_prequantize_frozen(self.handle, _stream()))
+
+    def zoqat_init_qparams(self):
+        _check(lib().zoqat_init_qparams(self.handle, _stream()))
+
+    def zoqat_step_rates(self, tokens, labels, seed, eps, lr, lr_quant, lr_smooth, result=None):
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        b, s = tokens.shape
+        _check(lib().zoqat_step_rates(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, lr_quant, lr_smooth,
+                                      _p(result), _stream()))
+        return result
+
+    def zoqat_step_finish_rates(self, sums, seed, eps, lr, lr_quant, lr_smooth, result=None):
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        _check(lib().zoqat_step_finish_rates(self.handle, _p(sums), seed, eps, lr, lr_quant, lr_smooth, _p(result), _stream()))
+        return result
+
+    def zoqat_apply_update_rates(self, seed, scale, scale_quant, scale_smooth):
+        _check(lib().zoqat_apply_update_rates(self.handle, seed, scale, scale_quant, scale_smooth, _stream()))
 
     def zoqat_forward_loss(self, tokens, labels, seed, signed_eps, out=None):
         out = torch.empty(1, dtype=torch.float32, device="cuda") if out is None else out

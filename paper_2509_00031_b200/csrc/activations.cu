@@ -39,6 +39,16 @@ __device__ __forceinline__ float block_max(float v, float* red) {
     return t;
 }
 
+// Section 4.2 smoothing on the activation side: x <- (x - shift') * (1 / scale'), each operation rounded once.
+__device__ __forceinline__ float smooth1(float x, float shift, float inv) { return __fmul_rn(__fsub_rn(x, shift), inv); }
+__device__ __forceinline__ void smooth4(float4& v, const float4& d, const float4& i) {
+    v.x = smooth1(v.x, d.x, i.x); v.y = smooth1(v.y, d.y, i.y); v.z = smooth1(v.z, d.z, i.z); v.w = smooth1(v.w, d.w, i.w);
+}
+// Vectors of the pass that row r belongs to: shift at +ld, reciprocal scale at +2*ld of the sign's block.
+__device__ __forceinline__ const float* smooth_base(const SmoothAct& sm, int64_t r) {
+    return sm.smooth + (r >= sm.rows_per_pass ? 3 * (size_t)sm.ld : 0);
+}
+
 // Writes the operand row from the fp32 row held in shared memory.
 __device__ __forceinline__ void write_operand_row(const float* row, int cols, int a_bits, __nv_bfloat16* op_row,
                                                   float* row_step, float* redf) {
@@ -65,7 +75,7 @@ __device__ __forceinline__ void write_operand_row(const float* row, int cols, in
 __global__ void __launch_bounds__(kRowThreads)
 norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
                         const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
-                        float* __restrict__ row_step, float* __restrict__ normed) {
+                        float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm) {
     extern __shared__ float row[];
     __shared__ double redd[kRowThreads / 32];
     __shared__ float redf[kRowThreads / 32];
@@ -94,12 +104,17 @@ norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, co
     __syncthreads();
     if (normed)
         for (int c = threadIdx.x; c < cols; c += kRowThreads) normed[r * cols + c] = row[c];
+    if (sm.smooth) {
+        const float* b = smooth_base(sm, r);
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
+        __syncthreads();
+    }
     write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
 }
 
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                       float* __restrict__ row_step) {
+                       float* __restrict__ row_step, SmoothAct sm) {
     extern __shared__ float row[];
     __shared__ float redf[kRowThreads / 32];
     const int64_t r = blockIdx.x;
@@ -113,6 +128,10 @@ ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_b
     } else {                         // relu
         const float* g = x + r * cols;
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = fmaxf(g[c], 0.0f);
+    }
+    if (sm.smooth) {
+        const float* b = smooth_base(sm, r);
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
     }
     __syncthreads();
     write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
@@ -160,10 +179,23 @@ __device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n
 }
 
 template <int VPT>
+__device__ __forceinline__ void smooth_regs(float4 (&v)[VPT], int n4, const SmoothAct& sm, int64_t r) {
+    if (!sm.smooth) return;
+    const float* b = smooth_base(sm, r);
+    const float4* d4 = reinterpret_cast<const float4*>(b + sm.ld);
+    const float4* i4 = reinterpret_cast<const float4*>(b + 2 * (size_t)sm.ld);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int idx = threadIdx.x + i * kRowThreads;
+        if (idx < n4) smooth4(v[i], __ldg(d4 + idx), __ldg(i4 + idx));
+    }
+}
+
+template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
                             const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
-                            float* __restrict__ row_step, float* __restrict__ normed) {
+                            float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm) {
     __shared__ double redd[kRowThreads / 32];
     __shared__ float redf[kRowThreads / 32];
     const int64_t r = blockIdx.x;
@@ -225,13 +257,14 @@ norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind
             if (idx < n4) reinterpret_cast<float4*>(normed + r * cols)[idx] = v[i];
         }
     }
+    smooth_regs<VPT>(v, n4, sm, r);
     write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
 }
 
 template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                           float* __restrict__ row_step) {
+                           float* __restrict__ row_step, SmoothAct sm) {
     __shared__ float redf[kRowThreads / 32];
     const int64_t r = blockIdx.x;
     const int n4 = cols >> 2;
@@ -262,6 +295,7 @@ ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int
             v[i] = make_float4(fmaxf(g.x, 0.f), fmaxf(g.y, 0.f), fmaxf(g.z, 0.f), fmaxf(g.w, 0.f));
         }
     }
+    smooth_regs<VPT>(v, n4, sm, r);
     write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
 }
 
@@ -418,40 +452,41 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 }
 
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
-                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s) {
+                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
+                             SmoothAct sm) {
     const int n4 = cols / 4;
     const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(bias) |
                            reinterpret_cast<uintptr_t>(normed)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        norm_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+        norm_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        norm_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+        norm_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        norm_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+        norm_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static bool attr = false;
         if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed);
+        norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
     }
     count_launch();
 }
 
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
-                            float* row_step, cudaStream_t s) {
+                            float* row_step, cudaStream_t s, SmoothAct sm) {
     const int n4 = cols / 4;
     const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        ffn_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+        ffn_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        ffn_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+        ffn_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        ffn_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step);
+        ffn_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static bool attr = false;
         if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step);
+        ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step, sm);
     }
     count_launch();
 }

@@ -51,7 +51,10 @@ struct Linear {
     int64_t rows = 0, cols = 0;
     const uint32_t* packed = nullptr;
     const float2* qparams = nullptr;
+    float* theta = nullptr;             // Section 4.2: learnable (step, zero point, alpha, beta) per group
     bool present = false;
+    bool adaptive() const { return theta != nullptr; }
+    uint32_t tid_q() const { return tid + 0x10000u; }
     bool trainable() const { return (flags & ZOQAT_TENSOR_TRAINABLE) && !(flags & ZOQAT_TENSOR_FROZEN_PACKED); }
     bool packed_frozen() const { return flags & ZOQAT_TENSOR_FROZEN_PACKED; }
     int bits(int w_bits) const { return (flags & (ZOQAT_TENSOR_QUANTIZED | ZOQAT_TENSOR_FROZEN_PACKED)) ? w_bits : 0; }
@@ -60,6 +63,9 @@ struct Linear {
 struct Layer {
     Linear lin[7];                      // indexed by ZOQAT_ROLE_WQ .. ZOQAT_ROLE_W_DOWN
     const float* vec[ZOQAT_ROLE_COUNT] = {nullptr};   // norm gains / biases / linear biases by role
+    float* smooth_s[4] = {nullptr, nullptr, nullptr, nullptr};   // Section 4.2 smoothing scale / shift per quantisation point
+    float* smooth_d[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool smoothing = false;
     bool any_trainable = false;
 };
 
@@ -74,6 +80,11 @@ struct Workspace {
     zoqat_step_result_dev* result;
     void* attn_scratch;                 // fp16 hi/lo operands of the tensor-core attention
     uint32_t* row_amax;                 // max |act| per row collected by the gate/up GEMM epilogue
+    float* smooth_buf;                  // Section 4.2: [sign 2][scale', shift', 1/scale'][smooth_ld] of the current point
+    float* bias_part;                   // per-group partial sums of shift' . w' ([sign][group])
+    float* bias_pm;                     // smoothed bias per pass: [sign][bias_ld]
+    float* class_scales;                // {lr_quant * g, lr_smooth * g}
+    int smooth_ld, bias_ld;
     size_t bop_elems;                   // elements of ONE pass' operand buffer
     size_t total;
 };
@@ -112,6 +123,13 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.result = (zoqat_step_result_dev*)take(sizeof(zoqat_step_result_dev));
     w.attn_scratch = take(attention_tc_scratch_bytes(2 * c.max_batch, c.max_seq, c.n_heads, c.d_model / c.n_heads));
     w.row_amax = (uint32_t*)take(R * 4);
+    w.smooth_ld = (int)(d > F ? d : F);
+    w.smooth_buf = (float*)take((size_t)6 * w.smooth_ld * 4);
+    const size_t lin_max = (3 * d * d > ffn_cols * d) ? 3 * d * d : ffn_cols * d;
+    w.bias_part = (float*)take(2 * (lin_max / c.w_group) * 4);
+    w.bias_ld = (int)(3 * d > ffn_cols ? 3 * d : ffn_cols);
+    w.bias_pm = (float*)take((size_t)2 * w.bias_ld * 4);
+    w.class_scales = (float*)take(2 * 4);
     w.total = off;
 }
 
@@ -174,6 +192,7 @@ struct zoqat_model {
     Workspace ws;
     int first_trainable_layer = 0;      // n_layers if no block tensor is trainable
     bool any_packed = false, prequantized = false;
+    bool any_learnable = false;         // a tensor is ADAPTIVE or a layer has smoothing vectors (Section 4.2)
     long long launches_at_create = 0;
 };
 
@@ -204,11 +223,29 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
 
 // Writes the bf16 matmul operand(s) of one linear at `dst` (+ pass stride for the second pass).
 // passes == 1: operand of W + eps*u (eps signed).  passes == 2: +eps at dst, -eps at dst + pass_stride.
+// smoothing (Section 4.2): the layer's current point has its perturbed vectors in ws.smooth_buf; the smoothed bias
+// of this linear goes to ws.bias_pm + bias_off (per pass: + ws.bias_ld), starting from bias0 (may be NULL).
 void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t pass_stride, int passes,
-                     uint64_t seed, float eps, cudaStream_t s) {
+                     uint64_t seed, float eps, cudaStream_t s, bool smoothing = false, size_t bias_off = 0,
+                     const float* bias0 = nullptr) {
     ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
     const int64_t n = L.rows * L.cols;
     const int bits = L.bits(m->cfg.w_bits);
+    if (smoothing || (L.adaptive() && bits != 0)) {
+        LearnedOperandArgs a{};
+        a.w = L.w; a.rows = L.rows; a.cols = L.cols; a.group = m->cfg.w_group; a.bits = bits;
+        a.perturb = L.trainable() && eps != 0.0f;
+        a.seed = seed; a.tid = L.tid; a.tid_q = L.tid_q(); a.eps = eps;
+        a.op_plus = dst; a.op_minus = passes == 2 ? dst + pass_stride : nullptr;
+        a.theta = L.adaptive() ? L.theta : nullptr;
+        if (smoothing) {
+            a.smooth = m->ws.smooth_buf; a.smooth_ld = m->ws.smooth_ld;
+            a.bias_part = m->ws.bias_part; a.bias0 = bias0;
+            a.bias_out = m->ws.bias_pm + bias_off; a.bias_out_stride = m->ws.bias_ld;
+        }
+        launch_weight_operand_learned(a, s);
+        return;
+    }
     if (L.packed_frozen()) {
         launch_unpack_operand(L.packed, L.qparams, n, m->cfg.w_group, m->cfg.w_bits, dst, s);
         if (passes == 2) cudaMemcpyAsync(dst + pass_stride, dst, (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
@@ -246,15 +283,29 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             Z = 2;
         }
         const int64_t R = Z * T;
+        // Section 4.2 smoothing: the perturbed vectors of a quantisation point are written to ws.smooth_buf just
+        // before the kernels that read them (the activation operand, the producers of the point's linears)
+        const bool smo = Ly.smoothing;
+        SmoothAct sa;
+        if (smo) { sa.smooth = w.smooth_buf; sa.ld = w.smooth_ld; sa.rows_per_pass = T; }
+        auto smooth_point = [&](int point, int cols) {
+            ProfScope ps_(m, ZOQAT_PROF_WEIGHT, s);
+            const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)point;
+            launch_smooth_perturb(Ly.smooth_s[point], Ly.smooth_d[point], cols, seed, 0x20000u + base, 0x30000u + base, eps,
+                                  eps != 0.0f, Z, w.smooth_buf, w.smooth_ld, s);
+        };
         // --- attention block
+        if (smo) smooth_point(0, d);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
-            produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s);
+            produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
+                            Ly.vec[ZOQAT_ROLE_BQ + r]);
         GemmArgs g{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
+        if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         g.out = w.qkv; g.b_stride = ps;
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s);
@@ -264,22 +315,26 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                                   llama ? w.rope_sin : nullptr, w.att, w.attn_scratch, w.err_flag, s)) {
               return fail(rc, "attention launch rejected");
           } }
-        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s);
+        if (smo) smooth_point(1, d);
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO]);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
+        if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         if (int rc = run_gemm(m, g, s)) return rc;
         // --- feed-forward block
+        if (smo) smooth_point(2, d);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
         const int n_up = llama ? 2 * F : F;
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s);
-        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1]);
+        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
+        if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         // SiLU-gated FFN on the pair kernel: the epilogue multiplies silu(gate) by up and collects the row maxima,
         // so the intermediate is half as wide and the quantiser that follows needs a single pass
         const bool fuse_gate = llama && c.gemm_impl == ZOQAT_GEMM_TCGEN05 && F % 128 == 0 && F <= 16384;
@@ -288,13 +343,17 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             g.mode = 3; g.row_amax = w.row_amax;
         }
         if (int rc = run_gemm(m, g, s)) return rc;
+        if (smo) smooth_point(3, F);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
-          if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
-          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s);
+          // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
+          if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, sa);
+          else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
+          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, sa); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2]);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
+        if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         if (int rc = run_gemm(m, g, s)) return rc;
     }
     if (passes == 2 && Z == 1) {
@@ -328,13 +387,29 @@ int check_call(zoqat_model* m, const void* tokens, const void* labels, int batch
     return ZOQAT_OK;
 }
 
-void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float scale_val, cudaStream_t s) {
+// Eq. (2) on every trainable tensor.  Factors: weights scale_ptr / scale_val; quantiser parameters and smoothing
+// vectors (Section 4.2) class_ptr[0] / class_ptr[1] when class_ptr != NULL, else scale_q / scale_s.
+void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float scale_val, cudaStream_t s,
+                const float* class_ptr = nullptr, float scale_q = 0.0f, float scale_s = 0.0f) {
     ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
-    for (auto& Ly : m->layers)
+    const int d = m->cfg.d_model, F = m->cfg.d_ffn;
+    for (size_t l = 0; l < m->layers.size(); ++l) {
+        Layer& Ly = m->layers[l];
         for (int r = 0; r < 7; ++r) {
             Linear& L = Ly.lin[r];
-            if (L.present && L.trainable()) launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
+            if (!(L.present && L.trainable())) continue;
+            launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
+            if (L.adaptive())
+                launch_update(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, seed, L.tid_q(), class_ptr, scale_q, s);
         }
+        if (Ly.smoothing)
+            for (int pt = 0; pt < 4; ++pt) {
+                const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
+                const uint64_t n = pt == 3 ? (uint64_t)F : (uint64_t)d;
+                launch_update(Ly.smooth_s[pt], n, seed, 0x20000u + base, class_ptr ? class_ptr + 1 : nullptr, scale_s, s);
+                launch_update(Ly.smooth_d[pt], n, seed, 0x30000u + base, class_ptr ? class_ptr + 1 : nullptr, scale_s, s);
+            }
+    }
     if (m->head.trainable())
         launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
 }
@@ -402,7 +477,14 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
         const bool is_packed = t.flags & ZOQAT_TENSOR_FROZEN_PACKED;
         if (!t.data && !is_packed) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: data is NULL", i); }
         if (reinterpret_cast<uintptr_t>(t.data) & 15) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: data must be 16-byte aligned", i); }
-        if (t.role <= ZOQAT_ROLE_B_FC2) {
+        if (t.role >= ZOQAT_ROLE_SMOOTH_SCALE && t.role < ZOQAT_ROLE_SMOOTH_SHIFT + 4) {
+            if (t.layer < 0 || t.layer >= cfg->n_layers) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: layer %d out of range", i, t.layer); }
+            Layer& Ly = m->layers[t.layer];
+            float** slot = t.role < ZOQAT_ROLE_SMOOTH_SHIFT ? &Ly.smooth_s[t.role - ZOQAT_ROLE_SMOOTH_SCALE]
+                                                             : &Ly.smooth_d[t.role - ZOQAT_ROLE_SMOOTH_SHIFT];
+            if (*slot) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: smoothing role %d of layer %d given twice", i, t.role, t.layer); }
+            *slot = static_cast<float*>(t.data);
+        } else if (t.role <= ZOQAT_ROLE_B_FC2) {
             if (t.layer < 0 || t.layer >= cfg->n_layers) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: layer %d out of range", i, t.layer); }
             Layer& Ly = m->layers[t.layer];
             if (t.role <= ZOQAT_ROLE_W_DOWN) {
@@ -422,6 +504,12 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
                     L.packed = static_cast<const uint32_t*>(t.packed);
                     L.qparams = static_cast<const float2*>(t.qparams);
                     m->any_packed = true;
+                }
+                if (t.flags & ZOQAT_TENSOR_ADAPTIVE) {
+                    const uint32_t need = ZOQAT_TENSOR_TRAINABLE | ZOQAT_TENSOR_QUANTIZED;
+                    if (is_packed || (t.flags & need) != need) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: ADAPTIVE needs TRAINABLE | QUANTIZED and excludes FROZEN_PACKED", i); }
+                    if (!t.qparams || (reinterpret_cast<uintptr_t>(t.qparams) & 15)) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: ADAPTIVE needs 16-byte aligned qparams", i); }
+                    L.theta = static_cast<float*>(t.qparams);
                 }
                 if (L.trainable()) Ly.any_trainable = true;
             } else {
@@ -462,6 +550,16 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
                           ZOQAT_ROLE_BO, ZOQAT_ROLE_B_FC1, ZOQAT_ROLE_B_FC2})
                 if (!Ly.vec[r]) return missing("bias", l);
         if (Ly.any_trainable && m->first_trainable_layer == cfg->n_layers) m->first_trainable_layer = l;
+        int n_smooth = 0;
+        for (int pt = 0; pt < 4; ++pt) n_smooth += (Ly.smooth_s[pt] != nullptr) + (Ly.smooth_d[pt] != nullptr);
+        if (n_smooth != 0 && n_smooth != 8) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "layer %d: smoothing needs the scale and the shift of all four points", l); }
+        if (n_smooth == 8) {
+            for (int r = 0; r < 7; ++r)
+                if (Ly.lin[r].present && !Ly.lin[r].trainable()) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "layer %d: smoothing needs every block linear of the layer trainable", l); }
+            Ly.smoothing = true;
+        }
+        if (Ly.smoothing) m->any_learnable = true;
+        for (int r = 0; r < 7; ++r) if (Ly.lin[r].adaptive()) m->any_learnable = true;
     }
     // one-time tables: rotary cos/sin (evaluated in double, stored fp32) and concatenated q|k|v biases
     if (llama) {
@@ -514,6 +612,18 @@ int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream) {
     return ZOQAT_OK;
 }
 
+int zoqat_init_qparams(zoqat_model_t* m, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r) {
+            Linear& L = Ly.lin[r];
+            if (L.present && L.adaptive()) launch_init_qparams(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, L.theta, s);
+        }
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
 int zoqat_forward_loss(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
                        uint64_t seed, float signed_eps, float* loss_out_dev, void* stream) {
     if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
@@ -545,9 +655,37 @@ int zoqat_step_finish(zoqat_model_t* m, const double* sums_dev, uint64_t seed, f
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(result_dev);
     launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, res, s);
-    update_all(m, seed, &res->update_scale, 0.0f, s);
+    if (m->any_learnable) {        // Section 4.2 parameters move with the same rate
+        launch_class_scales(&res->proj_grad, lr, lr, m->ws.class_scales, s);
+        update_all(m, seed, &res->update_scale, 0.0f, s, m->ws.class_scales);
+    } else {
+        update_all(m, seed, &res->update_scale, 0.0f, s);
+    }
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
+}
+
+int zoqat_step_finish_rates(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr, float lr_quant,
+                            float lr_smooth, zoqat_step_result_t* result_dev, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (!sums_dev || !result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev/result_dev are NULL");
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(result_dev);
+    launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, res, s);
+    launch_class_scales(&res->proj_grad, lr_quant, lr_smooth, m->ws.class_scales, s);
+    update_all(m, seed, &res->update_scale, 0.0f, s, m->ws.class_scales);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step_rates(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                     uint64_t seed, float eps, float lr, float lr_quant, float lr_smooth, zoqat_step_result_t* result_dev,
+                     void* stream) {
+    if (!result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "result_dev is NULL");
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (int rc = zoqat_step_begin(m, tokens_dev, labels_dev, batch, seq, seed, eps, m->ws.sums, stream)) return rc;
+    return zoqat_step_finish_rates(m, m->ws.sums, seed, eps, lr, lr_quant, lr_smooth, result_dev, stream);
 }
 
 int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
@@ -580,9 +718,22 @@ int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
         for (auto& Ly : m->layers)
             for (int r = 0; r < 7; ++r) {
                 Linear& L = Ly.lin[r];
-                if (L.present && L.trainable())
+                if (L.present && L.trainable()) {
                     launch_update_multi(L.w_mut, (uint64_t)(L.rows * L.cols), seed, n_dirs, L.tid, &res->update_scale, stride, s);
+                    if (L.adaptive())
+                        launch_update_multi(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, seed, n_dirs, L.tid_q(), &res->update_scale, stride, s);
+                }
             }
+        for (size_t l = 0; l < m->layers.size(); ++l) {
+            Layer& Ly = m->layers[l];
+            if (!Ly.smoothing) continue;
+            for (int pt = 0; pt < 4; ++pt) {
+                const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
+                const uint64_t n = pt == 3 ? (uint64_t)m->cfg.d_ffn : (uint64_t)m->cfg.d_model;
+                launch_update_multi(Ly.smooth_s[pt], n, seed, n_dirs, 0x20000u + base, &res->update_scale, stride, s);
+                launch_update_multi(Ly.smooth_d[pt], n, seed, n_dirs, 0x30000u + base, &res->update_scale, stride, s);
+            }
+        }
         if (m->head.trainable())
             launch_update_multi(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, n_dirs, m->head.tid, &res->update_scale, stride, s);
     }
@@ -607,11 +758,15 @@ int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t*
     return ZOQAT_OK;
 }
 
-int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream) {
+int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float scale_quant, float scale_smooth, void* stream) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
-    update_all(m, seed, nullptr, scale, static_cast<cudaStream_t>(stream));
+    update_all(m, seed, nullptr, scale, static_cast<cudaStream_t>(stream), nullptr, scale_quant, scale_smooth);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
+}
+
+int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream) {
+    return zoqat_apply_update_rates(m, seed, scale, scale, scale, stream);
 }
 
 int zoqat_check(zoqat_model_t* m, void* stream) {
@@ -708,6 +863,65 @@ int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols,
     if (!w_dev || !operand_plus_dev || !operand_minus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     launch_weight_operand(w_dev, rows * cols, group, bits, 1, seed, tensor_id, eps, static_cast<__nv_bfloat16*>(operand_plus_dev),
                           static_cast<__nv_bfloat16*>(operand_minus_dev), nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
+                                    uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
+                                    const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
+                                    void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
+    if (!w_dev || !operand_plus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_plus_dev are NULL");
+    if (!theta_dev && !smooth_dev) return fail(ZOQAT_ERR_INVALID_ARG, "neither theta_dev nor smooth_dev given: use zoqat_op_weight_quant");
+    if (smooth_dev && (!bias_dev || !scratch_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "smoothing needs bias_dev and scratch_dev");
+    if ((reinterpret_cast<uintptr_t>(theta_dev) | reinterpret_cast<uintptr_t>(smooth_dev) | reinterpret_cast<uintptr_t>(w_dev)) & 15)
+        return fail(ZOQAT_ERR_INVALID_ARG, "w_dev, theta_dev and smooth_dev must be 16-byte aligned");
+    LearnedOperandArgs a{};
+    a.w = w_dev; a.rows = rows; a.cols = cols; a.group = group; a.bits = bits; a.perturb = eps != 0.0f;
+    a.seed = seed; a.tid = tensor_id; a.tid_q = tensor_id + 0x10000u; a.eps = eps;
+    a.op_plus = static_cast<__nv_bfloat16*>(operand_plus_dev); a.op_minus = static_cast<__nv_bfloat16*>(operand_minus_dev);
+    a.theta = theta_dev; a.smooth = smooth_dev; a.smooth_ld = (int)cols;
+    a.bias_part = scratch_dev; a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
+    a.codes = codes_dev;
+    launch_weight_operand_learned(a, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_smooth_perturb(const float* scale_dev, const float* shift_dev, int64_t cols, uint64_t seed, uint32_t scale_id,
+                            uint32_t shift_id, float eps, float* out_dev, void* stream) {
+    if (!scale_dev || !shift_dev || !out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (cols <= 0 || cols % 4 || cols > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a positive multiple of 4");
+    if ((reinterpret_cast<uintptr_t>(scale_dev) | reinterpret_cast<uintptr_t>(shift_dev) | reinterpret_cast<uintptr_t>(out_dev)) & 15)
+        return fail(ZOQAT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    launch_smooth_perturb(scale_dev, shift_dev, (int)cols, seed, scale_id, shift_id, eps, eps != 0.0f, 2, out_dev, (int)cols,
+                          static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_smooth_act_operand(const float* x_dev, int64_t rows, int64_t cols, int norm_kind, const float* gain_dev,
+                                const float* bias_dev, float norm_eps, int a_bits, const float* smooth_dev,
+                                int64_t rows_per_pass, void* operand_dev, float* row_step_dev, void* stream) {
+    if (!x_dev || !operand_dev || !row_step_dev || !smooth_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
+    if (norm_kind < 0 || norm_kind > 2 || (norm_kind >= 1 && !gain_dev) || (norm_kind == 2 && !bias_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "bad norm arguments");
+    if (a_bits != 0 && a_bits != 4 && a_bits != 6 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d", a_bits);
+    if (reinterpret_cast<uintptr_t>(smooth_dev) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "smooth_dev must be 16-byte aligned");
+    SmoothAct sa;
+    sa.smooth = smooth_dev; sa.ld = (int)cols; sa.rows_per_pass = rows_per_pass;
+    launch_norm_act_operand(x_dev, rows, (int)cols, norm_kind, gain_dev, bias_dev, norm_eps, a_bits,
+                            static_cast<__nv_bfloat16*>(operand_dev), row_step_dev, nullptr, static_cast<cudaStream_t>(stream), sa);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, float* theta_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if (!w_dev || !theta_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if ((reinterpret_cast<uintptr_t>(w_dev) | reinterpret_cast<uintptr_t>(theta_dev)) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    launch_init_qparams(w_dev, rows * cols, group, bits, theta_dev, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -31,6 +31,25 @@ void launch_weight_operand(const float* w, int64_t n, int group, int bits, int p
                            uint64_t seed, uint32_t tid, float eps,
                            __nv_bfloat16* op_plus, __nv_bfloat16* op_minus,
                            uint8_t* codes, float* step, int32_t* zp, cudaStream_t s);
+// Producer with the learnable parts of Section 4.2.  theta != NULL: per-group (step, z, alpha, beta) replace min/max
+// (perturbed with tensor id tid_q).  smooth != NULL: [sign][kind][smooth_ld] perturbed smoothing vectors (kind 0
+// scale, 1 shift, 2 reciprocal scale); the quantiser sees scale (.) w' and bias_out[sign * bias_out_stride + row] =
+// bias0[row] (or 0) + shift . w'[row, :] (bias_part: scratch of 2 * rows * cols / group floats).
+// op_minus == NULL: one operand with eps signed.  codes (may be NULL): uint8 codes of the op_plus side.
+struct LearnedOperandArgs {
+    const float* w; int64_t rows, cols; int group, bits, perturb;
+    uint64_t seed; uint32_t tid, tid_q; float eps;
+    __nv_bfloat16 *op_plus, *op_minus;
+    const float* theta;
+    const float* smooth; int smooth_ld;
+    float* bias_part; const float* bias0; float* bias_out; int64_t bias_out_stride;
+    uint8_t* codes;
+};
+void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s);
+void launch_smooth_perturb(const float* scale, const float* shift, int cols, uint64_t seed, uint32_t tid_s, uint32_t tid_d,
+                           float eps, int perturb, int signs, float* out, int ld, cudaStream_t s);
+void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s);
+void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s);
 void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);
 void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,
                            __nv_bfloat16* op, cudaStream_t s);
@@ -43,10 +62,14 @@ void launch_update_multi(float* w, uint64_t n, uint64_t seed, int n_dirs, uint32
 
 void launch_embed(const int32_t* tokens, const float* embed, const float* pos, int64_t T, int seq, int d,
                   int vocab, int passes, float* h, cudaStream_t s);
+// Smoothing of Section 4.2 on the activation side (smooth may be NULL): the quantiser sees (x - shift') * (1 / scale')
+// with the vectors of launch_smooth_perturb; rows [0, rows_per_pass) use sign 0, the rest sign 1.
+struct SmoothAct { const float* smooth = nullptr; int ld = 0; int64_t rows_per_pass = 0; };
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
-                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s);
+                             float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
+                             SmoothAct sm = SmoothAct());
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
-                            __nv_bfloat16* op, float* row_step, cudaStream_t s);
+                            __nv_bfloat16* op, float* row_step, cudaStream_t s, SmoothAct sm = SmoothAct());
 // Activation operand of rows whose max |x| is already known (amax: bits of a non-negative float per row).
 void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits,
                          __nv_bfloat16* op, float* row_step, cudaStream_t s);
@@ -66,7 +89,8 @@ struct GemmArgs {
     int64_t M, N, K;
     int Z;
     const float* row_step;    // [Z*M] or NULL
-    const float* bias;        // [N] or NULL
+    const float* bias;        // [N] or NULL; pass z reads bias + z*bias_stride
+    size_t bias_stride;       // 0: one bias for every pass
     int relu;
     int accumulate;
     float* out;               // [Z*M, N]

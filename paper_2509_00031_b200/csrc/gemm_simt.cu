@@ -75,7 +75,7 @@ gemm_simt_kernel(GemmArgs g, int n_tiles_n) {
                 const int64_t n = n0 + tx * 8 + j;
                 if (n >= g.N) continue;
                 float v = rs * acc[i][j];
-                if (g.bias) v += g.bias[n];
+                if (g.bias) v += g.bias[(size_t)z * g.bias_stride + n];
                 if (g.relu) v = fmaxf(v, 0.0f);
                 float* o = g.out + r * g.N + n;
                 *o = g.accumulate ? *o + v : v;

@@ -57,6 +57,7 @@ struct TcParams {
     int Z;
     const float* row_step;
     const float* bias;
+    int64_t bias_stride;      // elements between the bias vectors of consecutive passes (0: shared)
     int relu, accumulate;
     float* out;
     int mode;
@@ -206,6 +207,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int64_t n_base = (int64_t)tn * BN;
             float ce_m = -INFINITY, ce_s = 0.0f;
             const int32_t lab = (p.mode == 1 && row_ok) ? p.labels[m] : -1;
+            const float* bias = p.bias ? p.bias + (int64_t)z * p.bias_stride : nullptr;
             if (p.mode == 3) {
                 // SiLU-gated FFN: act = silu(gate) * up leaves as fp32 [rows, N/2]; the row maximum of |act| is
                 // collected for the activation quantiser that follows.
@@ -220,13 +222,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint32_t box = out_stage + (uint32_t)((quarter * 2 + out_buf) * Cfg::kOutBoxBytes);
                     if (lane == 0) bulk_wait_read_1();
                     __syncwarp();
+                    const int64_t f0 = (int64_t)tn * (BN / 2) + c * 32;     // feature of column 0 of this chunk
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         float a4[4];
+                        float4 bg = make_float4(0.f, 0.f, 0.f, 0.f), bu = bg;
+                        if (bias) {
+                            bg = *reinterpret_cast<const float4*>(bias + f0 + j);
+                            bu = *reinterpret_cast<const float4*>(bias + p.N / 2 + f0 + j);
+                        }
+                        const float bgs[4] = {bg.x, bg.y, bg.z, bg.w}, bus[4] = {bu.x, bu.y, bu.z, bu.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float g = rs * __uint_as_float(vg[j + e]);
-                            const float u = rs * __uint_as_float(vu[j + e]);
+                            const float g = rs * __uint_as_float(vg[j + e]) + bgs[e];
+                            const float u = rs * __uint_as_float(vu[j + e]) + bus[e];
                             a4[e] = __fdiv_rn(g, 1.0f + expf(-g)) * u;
                             amax = fmaxf(amax, fabsf(a4[e]));
                         }
@@ -264,15 +273,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         float4 x;
                         x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
                         x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
-                        if (p.bias) {
+                        if (bias) {
                             if (full) {
-                                const float4 b = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+                                const float4 b = *reinterpret_cast<const float4*>(bias + n0 + j);
                                 x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
                             } else {
-                                if (n0 + j < p.N) x.x += p.bias[n0 + j];
-                                if (n0 + j + 1 < p.N) x.y += p.bias[n0 + j + 1];
-                                if (n0 + j + 2 < p.N) x.z += p.bias[n0 + j + 2];
-                                if (n0 + j + 3 < p.N) x.w += p.bias[n0 + j + 3];
+                                if (n0 + j < p.N) x.x += bias[n0 + j];
+                                if (n0 + j + 1 < p.N) x.y += bias[n0 + j + 1];
+                                if (n0 + j + 2 < p.N) x.z += bias[n0 + j + 2];
+                                if (n0 + j + 3 < p.N) x.w += bias[n0 + j + 3];
                             }
                         }
                         if (p.relu) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
@@ -297,8 +306,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             float4 x;
                             x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
                             x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
-                            if (p.bias) {
-                                const float4 b = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+                            if (bias) {
+                                const float4 b = *reinterpret_cast<const float4*>(bias + n0 + j);
                                 x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
                             }
                             if (p.relu) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
@@ -312,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int j = 0; j < 32; ++j) {
                             if (n0 + j >= p.N) break;
                             float x = rs * __uint_as_float(v[j]);
-                            if (p.bias) x += p.bias[n0 + j];
+                            if (bias) x += bias[n0 + j];
                             if (p.relu) x = fmaxf(x, 0.f);
                             if (p.accumulate) x += o[j];
                             o[j] = x;
@@ -423,7 +432,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
         return ZOQAT_ERR_CUDA;
     TcParams p;
     p.M = a.M; p.N = a.N; p.K = a.K; p.Z = a.Z;
-    p.row_step = a.row_step; p.bias = a.bias; p.relu = a.relu; p.accumulate = a.accumulate;
+    p.row_step = a.row_step; p.bias = a.bias; p.bias_stride = (int64_t)a.bias_stride; p.relu = a.relu; p.accumulate = a.accumulate;
     p.out = a.out; p.mode = a.mode; p.labels = a.labels; p.partials = a.partials; p.label_logit = a.label_logit;
     p.err_flag = a.err_flag;
     p.tiles_m = (int)((a.M + BM * CG - 1) / (BM * CG));
@@ -468,6 +477,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
 int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     if (a.M <= 0 || a.N <= 0 || a.K <= 0 || a.Z <= 0) return ZOQAT_ERR_INVALID_ARG;
     if (a.K % 8 != 0 || a.err_flag == nullptr || (a.Z > 1 && (a.b_stride % 8 != 0 || a.b_stride < (size_t)a.N * a.K))) return ZOQAT_ERR_INVALID_ARG;
+    if (a.bias_stride % 4 != 0) return ZOQAT_ERR_INVALID_ARG;      // the epilogue reads the bias with 16-byte loads
     if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.out) |
          reinterpret_cast<uintptr_t>(a.bias)) & 15)
         return ZOQAT_ERR_INVALID_ARG;

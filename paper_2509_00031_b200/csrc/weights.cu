@@ -243,6 +243,214 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
     }
 }
 
+// ---- Section 4.2: learnable quantiser and smoothing ---------------------------------------------------------
+// Adaptive weight quantiser: code = clamp(round(x / step) + z, alpha * Q_P, beta * Q_P), value = (code - z) * step,
+// one learnable (step, z, alpha, beta) per group.  Codes stay integers in [0, Q_P]: z and the two levels enter
+// rounded to nearest even, the levels limited to [0, Q_P] and the upper one to at least the lower one.
+struct AdaptQ { float step, inv, zr, lo, hi; };
+
+__device__ __forceinline__ AdaptQ adapt_params(const float4& th, float qp) {
+    AdaptQ a;
+    a.step = fmaxf(th.x, 1e-8f);
+    a.inv = __fdiv_rn(1.0f, a.step);
+    a.zr = rintf(th.y);
+    a.lo = fminf(fmaxf(rintf(__fmul_rn(th.z, qp)), 0.0f), qp);
+    a.hi = fminf(fmaxf(rintf(__fmul_rn(th.w, qp)), a.lo), qp);
+    return a;
+}
+
+__device__ __forceinline__ void quantise16_adaptive(float (&x)[16], const AdaptQ& a, float* codes) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float q = fminf(fmaxf(__fadd_rn(rintf(__fmul_rn(x[j], a.inv)), a.zr), a.lo), a.hi);
+        if (codes) codes[j] = q;
+        x[j] = __fmul_rn(__fadd_rn(q, -a.zr), a.step);
+    }
+}
+
+// The operand producer with the learnable parts of Section 4.2 (same thread mapping as weight_operand_kernel):
+//   SMOOTH  the quantiser sees s' (.) w' (s' = perturbed per-input-channel scale); the per-group partial sums of
+//           delta' . w' (the shift term of the smoothed bias, with the unscaled perturbed weight) go to bias_part,
+//           [sign][group], and are reduced per output row by bias_reduce_kernel;
+//   ADAPT   the group's (step, z, alpha, beta) are read from theta and perturbed with their own direction
+//           (tensor id tid_q, one Philox block per group) instead of being derived from min/max.
+// smooth: [sign][kind][smooth_ld] floats, kind 0 = scale, 1 = shift (2 = 1/scale, used by the activation side).
+template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH>
+__global__ void __launch_bounds__(kThreads)
+weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols16, int bits, int perturb,
+                              uint32_t k0, uint32_t k1, uint32_t tid, uint32_t tid_q, float eps,
+                              uint4* __restrict__ op_plus, uint4* __restrict__ op_minus,
+                              const float4* __restrict__ theta, const float* __restrict__ smooth, int smooth_ld,
+                              float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes) {
+    constexpr int LANES = GROUP / 16;
+    __shared__ float2 tab[kIcdfKnots];
+    if (perturb) stage_icdf_table(tab);
+    const float qp = (float)((1 << bits) - 1);
+    const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n16_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n16;
+        float x[16], xm[16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float4 v = live ? __ldg(w + 4 * i + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+        }
+        if (perturb) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)(4 * i + k));
+                const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (DUAL) xm[4 * k + j] = __fmaf_rn(-eps, zz[j], x[4 * k + j]);
+                    x[4 * k + j] = __fmaf_rn(eps, zz[j], x[4 * k + j]);
+                }
+            }
+        } else if (DUAL) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) xm[j] = x[j];
+        }
+        if (SMOOTH) {
+            const int col0 = (int)(i % cols16) * 16;
+            const float4* sp = reinterpret_cast<const float4*>(smooth + col0);
+            const float4* dp = reinterpret_cast<const float4*>(smooth + smooth_ld + col0);
+            const float4* sm = reinterpret_cast<const float4*>(smooth + 3 * (size_t)smooth_ld + col0);
+            const float4* dm = reinterpret_cast<const float4*>(smooth + 4 * (size_t)smooth_ld + col0);
+            float bp = 0.0f, bm = 0.0f;
+            if (live) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float4 s4 = __ldg(sp + k), d4 = __ldg(dp + k);
+                    const float ss[4] = {s4.x, s4.y, s4.z, s4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        bp = __fmaf_rn(dd[j], x[4 * k + j], bp);
+                        x[4 * k + j] = __fmul_rn(x[4 * k + j], ss[j]);
+                    }
+                    if (DUAL) {
+                        const float4 t4 = __ldg(sm + k), e4 = __ldg(dm + k);
+                        const float ts[4] = {t4.x, t4.y, t4.z, t4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            bm = __fmaf_rn(ee[j], xm[4 * k + j], bm);
+                            xm[4 * k + j] = __fmul_rn(xm[4 * k + j], ts[j]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = LANES / 2; o > 0; o >>= 1) {
+                bp += __shfl_xor_sync(0xffffffffu, bp, o);
+                if (DUAL) bm += __shfl_xor_sync(0xffffffffu, bm, o);
+            }
+            if (live && (i % LANES) == 0) {
+                bias_part[i / LANES] = bp;
+                if (DUAL) bias_part[n_groups + i / LANES] = bm;
+            }
+        }
+        if (bits == 0) {
+            if (live) {
+                store_bf16x16(op_plus + 2 * i, x);
+                if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
+            }
+            continue;
+        }
+        float cd[16];
+        if (ADAPT) {
+            const float4 th = live ? __ldg(theta + i / LANES) : make_float4(1.f, 0.f, 0.f, 1.f);
+            float4 tp = th, tm = th;
+            if (perturb) {
+                const float4 u = direction4(tab, k0, k1, tid_q, (uint64_t)(i / LANES));
+                tp = make_float4(__fmaf_rn(eps, u.x, th.x), __fmaf_rn(eps, u.y, th.y), __fmaf_rn(eps, u.z, th.z), __fmaf_rn(eps, u.w, th.w));
+                if (DUAL) tm = make_float4(__fmaf_rn(-eps, u.x, th.x), __fmaf_rn(-eps, u.y, th.y), __fmaf_rn(-eps, u.z, th.z), __fmaf_rn(-eps, u.w, th.w));
+            }
+            quantise16_adaptive(x, adapt_params(tp, qp), codes ? cd : nullptr);
+            if (DUAL) quantise16_adaptive(xm, adapt_params(tm, qp), nullptr);
+        } else {
+            quantise16<LANES>(x, qp, codes ? cd : nullptr);
+            if (DUAL) quantise16<LANES>(xm, qp, nullptr);
+        }
+        if (live) {
+            store_bf16x16(op_plus + 2 * i, x);
+            if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
+            if (codes) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    codes[4 * i + k] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
+                                                   (unsigned char)cd[4 * k + 2], (unsigned char)cd[4 * k + 3]);
+            }
+        }
+    }
+}
+
+// out[sign][row] = bias0[row] + sum over the row's groups of bias_part[sign][row * gpr + g], in a fixed order.
+__global__ void bias_reduce_kernel(const float* __restrict__ part, int64_t n_groups, int gpr, int rows, int signs,
+                                   const float* __restrict__ bias0, float* __restrict__ out, int64_t out_sign_stride) {
+    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)rows * signs) return;
+    const int sgn = (int)(idx / rows), r = (int)(idx % rows);
+    const float* p = part + (int64_t)sgn * n_groups + (int64_t)r * gpr;
+    double acc = 0.0;
+    for (int g = 0; g < gpr; ++g) acc += (double)p[g];
+    out[(int64_t)sgn * out_sign_stride + r] = (float)(acc + (bias0 ? (double)bias0[r] : 0.0));
+}
+
+// Perturbed smoothing vectors of one quantisation point: out[sign][kind][ld], kind 0 = s' = s +/- eps u_s,
+// 1 = delta' = delta +/- eps u_delta, 2 = 1 / s' (rounded once).  sign 0 uses +eps (eps may be signed), sign 1 -eps.
+__global__ void __launch_bounds__(kThreads)
+smooth_perturb_kernel(const float4* __restrict__ s, const float4* __restrict__ d, int n4, uint32_t k0, uint32_t k1,
+                      uint32_t tid_s, uint32_t tid_d, float eps, int perturb, int signs, float* __restrict__ out, int ld) {
+    __shared__ float2 tab[kIcdfKnots];
+    if (perturb) stage_icdf_table(tab);
+    for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < n4; b += gridDim.x * blockDim.x) {
+        const float4 s4 = s[b], d4 = d[b];
+        float4 us = make_float4(0.f, 0.f, 0.f, 0.f), ud = us;
+        if (perturb) { us = direction4(tab, k0, k1, tid_s, (uint64_t)b); ud = direction4(tab, k0, k1, tid_d, (uint64_t)b); }
+        for (int sg = 0; sg < signs; ++sg) {
+            const float e = sg == 0 ? eps : -eps;
+            float4 a = s4, c = d4;
+            if (perturb) {
+                a = make_float4(__fmaf_rn(e, us.x, s4.x), __fmaf_rn(e, us.y, s4.y), __fmaf_rn(e, us.z, s4.z), __fmaf_rn(e, us.w, s4.w));
+                c = make_float4(__fmaf_rn(e, ud.x, d4.x), __fmaf_rn(e, ud.y, d4.y), __fmaf_rn(e, ud.z, d4.z), __fmaf_rn(e, ud.w, d4.w));
+            }
+            float* o = out + (size_t)sg * 3 * ld;
+            reinterpret_cast<float4*>(o)[b] = a;
+            reinterpret_cast<float4*>(o + ld)[b] = c;
+            reinterpret_cast<float4*>(o + 2 * (size_t)ld)[b] =
+                make_float4(__fdiv_rn(1.0f, a.x), __fdiv_rn(1.0f, a.y), __fdiv_rn(1.0f, a.z), __fdiv_rn(1.0f, a.w));
+        }
+    }
+}
+
+// Initial quantiser parameters (Section 4.2): step and zero point of the min/max scheme on the unperturbed
+// weights, alpha = 0, beta = 1.
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads)
+init_qparams_kernel(const float4* __restrict__ w, int64_t n16, int bits, float4* __restrict__ theta) {
+    constexpr int LANES = GROUP / 16;
+    const float qp = (float)((1 << bits) - 1);
+    const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n16_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n16;
+        float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float4 v = live ? __ldg(w + 4 * i + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            mn = fminf(mn, fminf(fminf(v.x, v.y), fminf(v.z, v.w)));
+            mx = fmaxf(mx, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+        }
+        group_minmax<LANES>(mn, mx);
+        const GroupQ g = group_params(mn, mx, qp);
+        if (live && (i % LANES) == 0) theta[i / LANES] = make_float4(g.step, __fadd_rn(g.zp, 0.0f), 0.0f, 1.0f);   // -0 -> +0
+    }
+}
+
+// {lr_quant * g, lr_smooth * g} next to the step record (Eq. (2) factors of the Section 4.2 parameter classes).
+__global__ void class_scales_kernel(const float* __restrict__ proj_grad, float lr_quant, float lr_smooth, float* __restrict__ out) {
+    out[0] = __fmul_rn(lr_quant, *proj_grad);
+    out[1] = __fmul_rn(lr_smooth, *proj_grad);
+}
+
 // Packed layout of Section 4.3 (any bit width with one code path): for every run of
 // 128 consecutive elements, 4*bits 32-bit words; word (j*bits + b) holds bit b of the
 // code of element 4*lane + j in bit `lane` (a warp ballot).  qparams: (step, zero point).
@@ -419,6 +627,78 @@ void launch_weight_operand(const float* w, int64_t n, int group, int bits, int p
     if (group == 32) weight_operand_dispatch<32>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
     else if (group == 64) weight_operand_dispatch<64>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
     else weight_operand_dispatch<128>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
+}
+
+template <int GROUP, bool ADAPT, bool SMOOTH>
+static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
+    const int64_t n16 = a.rows * a.cols / 16;
+    const int grid = stream_grid(n16, kThreads);
+    const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
+    const float4* w4 = reinterpret_cast<const float4*>(a.w);
+    uint4* p = reinterpret_cast<uint4*>(a.op_plus);
+    uint4* m = reinterpret_cast<uint4*>(a.op_minus);
+    const float4* th = reinterpret_cast<const float4*>(a.theta);
+    const int64_t n_groups = a.rows * a.cols / GROUP;
+    uchar4* c4 = reinterpret_cast<uchar4*>(a.codes);
+    if (a.op_minus)
+        weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
+            w4, n16, (int)(a.cols / 16), a.bits, a.perturb, k0, k1, a.tid, a.tid_q, a.eps, p, m, th, a.smooth, a.smooth_ld,
+            a.bias_part, n_groups, c4);
+    else
+        weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
+            w4, n16, (int)(a.cols / 16), a.bits, a.perturb, k0, k1, a.tid, a.tid_q, a.eps, p, nullptr, th, a.smooth, a.smooth_ld,
+            a.bias_part, n_groups, c4);
+    count_launch();
+    if (SMOOTH) {
+        const int signs = a.op_minus ? 2 : 1;
+        const int64_t work = a.rows * signs;
+        bias_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(a.bias_part, n_groups, (int)(a.cols / GROUP), (int)a.rows,
+                                                                          signs, a.bias0, a.bias_out, a.bias_out_stride);
+        count_launch();
+    }
+}
+
+template <int GROUP>
+static void learned_dispatch_group(const LearnedOperandArgs& a, cudaStream_t s) {
+    const bool adapt = a.theta != nullptr && a.bits != 0, smooth = a.smooth != nullptr;
+    if (adapt && smooth) learned_dispatch<GROUP, true, true>(a, s);
+    else if (adapt) learned_dispatch<GROUP, true, false>(a, s);
+    else learned_dispatch<GROUP, false, true>(a, s);
+}
+
+void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s) {
+    if (a.rows * a.cols == 0 || (a.perturb && !ensure_icdf_table())) return;
+    if (a.group == 32) learned_dispatch_group<32>(a, s);
+    else if (a.group == 64) learned_dispatch_group<64>(a, s);
+    else learned_dispatch_group<128>(a, s);
+}
+
+void launch_smooth_perturb(const float* scale, const float* shift, int cols, uint64_t seed, uint32_t tid_s, uint32_t tid_d,
+                           float eps, int perturb, int signs, float* out, int ld, cudaStream_t s) {
+    if (cols == 0 || (perturb && !ensure_icdf_table())) return;
+    const int n4 = cols / 4;
+    int blocks = (n4 + kThreads - 1) / kThreads;
+    if (blocks > 8) blocks = 8;
+    smooth_perturb_kernel<<<blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(scale), reinterpret_cast<const float4*>(shift), n4,
+                                                      (uint32_t)seed, (uint32_t)(seed >> 32), tid_s, tid_d, eps, perturb, signs, out, ld);
+    count_launch();
+}
+
+void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s) {
+    if (n == 0) return;
+    const int64_t n16 = n / 16;
+    const int grid = stream_grid(n16, kThreads);
+    const float4* w4 = reinterpret_cast<const float4*>(w);
+    float4* th = reinterpret_cast<float4*>(theta);
+    if (group == 32) init_qparams_kernel<32><<<grid, kThreads, 0, s>>>(w4, n16, bits, th);
+    else if (group == 64) init_qparams_kernel<64><<<grid, kThreads, 0, s>>>(w4, n16, bits, th);
+    else init_qparams_kernel<128><<<grid, kThreads, 0, s>>>(w4, n16, bits, th);
+    count_launch();
+}
+
+void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s) {
+    class_scales_kernel<<<1, 1, 0, s>>>(proj_grad, lr_quant, lr_smooth, out);
+    count_launch();
 }
 
 void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s) {
