@@ -23,6 +23,7 @@ if ROOT not in sys.path:
 METRIC = "ZO-QAT steps/s & fwd tokens/s, 7B-shape W4A8, 1 B200; % of roofline"
 UNIT = "steps/s"
 EPS, LR = 1e-3, 1e-6
+LR_QUANT, LR_SMOOTH = 1e-5, 5e-6      # rates of the Section 4.2 parameter classes (the paper's hyperparameter table)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, averaged over the 129 GEMM
 # launches of one step, from the committed ncu capture (profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by
 # workload; absent for workloads that have not been captured.
@@ -53,6 +54,8 @@ def workload_numbers(w):
     attn_flops = 2 * w["batch"] * w["seq"] ** 2 * d * (ftl + 2 * (L - ftl))
     frozen = per_layer * L - per_layer_trainable * (L - ftl)
     bytes_step = 4 * trainable + (w["w_bits"] / 8 + 8 / w["w_group"]) * frozen + 8 * trainable
+    if w.get("adaptive_quant"):         # four fp32 quantiser parameters per group: read once per step pair, read + written by Eq. (2)
+        bytes_step += 12 * 4 * per_layer_trainable * (L - ftl) / w["w_group"]
     return dict(T=T, block_params=block, trainable_params=trainable, head_params=head,
                 linear_flops=lin_flops, attn_flops=attn_flops, flops=lin_flops + attn_flops, bytes=bytes_step)
 
@@ -128,13 +131,15 @@ def oracle_sample(w, budget_note=True):
     times = {}
     cores = os.cpu_count() or 1
     cfg = OracleConfig(arch=w["arch"], n_layers=1, d_model=w["d_model"], n_heads=w["n_heads"], d_ffn=w["d_ffn"],
-                       vocab=w["vocab"], w_bits=w["w_bits"], w_group=w["w_group"], a_bits=w["a_bits"])
+                       vocab=w["vocab"], w_bits=w["w_bits"], w_group=w["w_group"], a_bits=w["a_bits"],
+                       adaptive_quant=bool(w.get("adaptive_quant")), smoothing=bool(w.get("smoothing")))
     params = synth.make_params(one, seed=0, max_seq=seq2)
     model = OracleModel(cfg, params)
+    model.init_learnable()
     for seq in (seq1, seq2):
         tokens, labels = synth.make_batch(1, seq, w["vocab"], seed=1234)
         t0 = time.perf_counter()
-        model.step(tokens, labels, 1000, EPS, LR)
+        model.step(tokens, labels, 1000, EPS, LR, LR_QUANT, LR_SMOOTH)
         times[seq] = time.perf_counter() - t0
     b = (times[seq2] - times[seq1]) / (seq2 - seq1)
     a = times[seq1] - b * seq1
@@ -215,7 +220,10 @@ def run_ours(args, w, rank, world, local_rank):
     any_packed = ftl > 0 or names is not None
     model = binding.ZoqatModel(w, params, max_batch=w["batch"], max_seq=w["seq"], first_trainable_layer=ftl,
                                packed_frozen=any_packed, trainable_names=names, head_trainable=w.get("head_trainable", True),
-                               gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05)
+                               gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05,
+                               adaptive_quant=bool(w.get("adaptive_quant")), smoothing=bool(w.get("smoothing")))
+    if w.get("adaptive_quant"):
+        model.zoqat_init_qparams()
     if any_packed:
         model.zoqat_prequantize_frozen()
         for l in range(w["n_layers"]):                     # the fp32 copies of packed tensors are no longer needed
@@ -230,13 +238,20 @@ def run_ours(args, w, rank, world, local_rank):
     result = torch.zeros(6, dtype=torch.float32, device="cuda")
     sums = torch.zeros(3, dtype=torch.float64, device="cuda")
 
+    learned = bool(w.get("adaptive_quant") or w.get("smoothing"))
+
     def step(t):
-        if world == 1:
+        if world == 1 and learned:
+            model.zoqat_step_rates(tokens, labels, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
+        elif world == 1:
             model.zoqat_step(tokens, labels, 1000 + t, EPS, LR, result)
         else:                                              # data-parallel replicas: 24-byte all-reduce between the halves
             model.zoqat_step_begin(tokens, labels, 1000 + t, EPS, sums)
             dist.all_reduce(sums)
-            model.zoqat_step_finish(sums, 1000 + t, EPS, LR, result)
+            if learned:
+                model.zoqat_step_finish_rates(sums, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
+            else:
+                model.zoqat_step_finish(sums, 1000 + t, EPS, LR, result)
 
     def barrier():
         if world > 1:

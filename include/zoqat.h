@@ -308,7 +308,7 @@ int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols,
  *   smooth_dev (may be NULL = no smoothing): fp32 [2][3][cols], the vectors zoqat_op_smooth_perturb wrote: the
  *     quantiser sees scale' (.) w', and bias_dev[sign * rows + r] = bias0_dev[r] (or 0) + sum_k shift'[k] * w'[r, k]
  *     (first equation of Section 4.2: the smoothed bias uses the unscaled, unquantised perturbed weight).
- *     scratch_dev: 2 * rows * cols / group floats.
+ *   scratch_dev: 18 * rows * cols / group floats, 16-byte aligned (prepared group parameters, bias partial sums).
  * operand_minus_dev may be NULL: one operand (and one bias vector) with eps signed.
  * codes_dev (may be NULL): uint8 [rows, cols] codes of the +eps side. */
 int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,

@@ -199,10 +199,10 @@ def zoqat_op_weight_operand_learned(w, group, bits, seed, tensor_id, eps, theta=
     rows, cols = w.shape
     plus = torch.empty((rows, cols), dtype=torch.bfloat16, device=w.device)
     minus = torch.empty_like(plus) if dual else None
-    bias = scratch = None
+    bias = None
+    scratch = torch.empty(18 * rows * (cols // group), dtype=torch.float32, device=w.device)
     if smooth is not None:
         bias = torch.empty((2 if dual else 1, rows), dtype=torch.float32, device=w.device)
-        scratch = torch.empty(2 * rows * (cols // group), dtype=torch.float32, device=w.device)
     codes = torch.empty((rows, cols), dtype=torch.uint8, device=w.device) if want_codes else None
     _check(lib().zoqat_op_weight_operand_learned(_p(w), rows, cols, group, bits, seed, tensor_id, eps, _p(theta), _p(smooth),
                                                  _p(bias0), _p(bias), _p(scratch), _p(plus), _p(minus), _p(codes), _stream()))

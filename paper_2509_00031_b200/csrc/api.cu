@@ -80,8 +80,10 @@ struct Workspace {
     zoqat_step_result_dev* result;
     void* attn_scratch;                 // fp16 hi/lo operands of the tensor-core attention
     uint32_t* row_amax;                 // max |act| per row collected by the gate/up GEMM epilogue
-    float* smooth_buf;                  // Section 4.2: [sign 2][scale', shift', 1/scale'][smooth_ld] of the current point
+    float* smooth_buf;                  // Section 4.2: [point 4][sign 2][scale', shift', 1/scale'][smooth_ld] of the current layer
     float* bias_part;                   // per-group partial sums of shift' . w' ([sign][group])
+    uint8_t* qprep;                     // prepared (perturbed) quantiser parameters of the current layer's linears
+    size_t qprep_off[8];                // byte offset of each block linear's block inside qprep
     float* bias_pm;                     // smoothed bias per pass: [sign][bias_ld]
     float* class_scales;                // {lr_quant * g, lr_smooth * g}
     int smooth_ld, bias_ld;
@@ -124,9 +126,16 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.attn_scratch = take(attention_tc_scratch_bytes(2 * c.max_batch, c.max_seq, c.n_heads, c.d_model / c.n_heads));
     w.row_amax = (uint32_t*)take(R * 4);
     w.smooth_ld = (int)(d > F ? d : F);
-    w.smooth_buf = (float*)take((size_t)6 * w.smooth_ld * 4);
+    w.smooth_buf = (float*)take((size_t)4 * 6 * w.smooth_ld * 4);
     const size_t lin_max = (3 * d * d > ffn_cols * d) ? 3 * d * d : ffn_cols * d;
     w.bias_part = (float*)take(2 * (lin_max / c.w_group) * 4);
+    {   // per linear: 2 passes x (A, B) x groups float4; q, k, v, o, gate, up, down back to back
+        const size_t lin_elems[7] = {d * d, d * d, d * d, d * d, F * d, (c.arch == ZOQAT_ARCH_LLAMA) ? F * d : 0, d * F};
+        size_t o = 0;
+        for (int r = 0; r < 7; ++r) { w.qprep_off[r] = o; o += align_up(4 * (lin_elems[r] / c.w_group) * 16); }
+        w.qprep_off[7] = o;
+        w.qprep = take(o);
+    }
     w.bias_ld = (int)(3 * d > ffn_cols ? 3 * d : ffn_cols);
     w.bias_pm = (float*)take((size_t)2 * w.bias_ld * 4);
     w.class_scales = (float*)take(2 * 4);
@@ -223,11 +232,12 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
 
 // Writes the bf16 matmul operand(s) of one linear at `dst` (+ pass stride for the second pass).
 // passes == 1: operand of W + eps*u (eps signed).  passes == 2: +eps at dst, -eps at dst + pass_stride.
-// smoothing (Section 4.2): the layer's current point has its perturbed vectors in ws.smooth_buf; the smoothed bias
-// of this linear goes to ws.bias_pm + bias_off (per pass: + ws.bias_ld), starting from bias0 (may be NULL).
+// smoothing (Section 4.2): quantisation point `point` of the layer has its perturbed vectors in ws.smooth_buf; the
+// smoothed bias of this linear goes to ws.bias_pm + bias_off (per pass: + ws.bias_ld), starting from bias0 (may be
+// NULL).  Adaptive tensors read the parameters forward() prepared for block linear `role`.
 void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t pass_stride, int passes,
                      uint64_t seed, float eps, cudaStream_t s, bool smoothing = false, size_t bias_off = 0,
-                     const float* bias0 = nullptr) {
+                     const float* bias0 = nullptr, int role = 0, int point = 0) {
     ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
     const int64_t n = L.rows * L.cols;
     const int bits = L.bits(m->cfg.w_bits);
@@ -238,8 +248,9 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
         a.seed = seed; a.tid = L.tid; a.tid_q = L.tid_q(); a.eps = eps;
         a.op_plus = dst; a.op_minus = passes == 2 ? dst + pass_stride : nullptr;
         a.theta = L.adaptive() ? L.theta : nullptr;
+        a.prep = m->ws.qprep + m->ws.qprep_off[role]; a.prepared = 1;      // forward() prepared the whole layer
         if (smoothing) {
-            a.smooth = m->ws.smooth_buf; a.smooth_ld = m->ws.smooth_ld;
+            a.smooth = m->ws.smooth_buf + (size_t)point * 6 * m->ws.smooth_ld; a.smooth_ld = m->ws.smooth_ld;
             a.bias_part = m->ws.bias_part; a.bias0 = bias0;
             a.bias_out = m->ws.bias_pm + bias_off; a.bias_out_stride = m->ws.bias_ld;
         }
@@ -283,25 +294,49 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             Z = 2;
         }
         const int64_t R = Z * T;
-        // Section 4.2 smoothing: the perturbed vectors of a quantisation point are written to ws.smooth_buf just
-        // before the kernels that read them (the activation operand, the producers of the point's linears)
+        // Section 4.2: one launch perturbs the smoothing vectors of the layer's four quantisation points, one more
+        // prepares the perturbed quantiser parameters of its adaptive linears
         const bool smo = Ly.smoothing;
-        SmoothAct sa;
-        if (smo) { sa.smooth = w.smooth_buf; sa.ld = w.smooth_ld; sa.rows_per_pass = T; }
-        auto smooth_point = [&](int point, int cols) {
-            ProfScope ps_(m, ZOQAT_PROF_WEIGHT, s);
-            const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)point;
-            launch_smooth_perturb(Ly.smooth_s[point], Ly.smooth_d[point], cols, seed, 0x20000u + base, 0x30000u + base, eps,
-                                  eps != 0.0f, Z, w.smooth_buf, w.smooth_ld, s);
+        auto smooth_at = [&](int point) {
+            SmoothAct sa;
+            if (smo) { sa.smooth = w.smooth_buf + (size_t)point * 6 * w.smooth_ld; sa.ld = w.smooth_ld; sa.rows_per_pass = T; }
+            return sa;
         };
+        if (smo) {
+            ProfScope ps_(m, ZOQAT_PROF_WEIGHT, s);
+            SmoothBatch sb{};
+            sb.count = 4; sb.prefix[0] = 0;
+            for (int pt = 0; pt < 4; ++pt) {
+                const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
+                sb.scale[pt] = Ly.smooth_s[pt]; sb.shift[pt] = Ly.smooth_d[pt];
+                sb.out[pt] = w.smooth_buf + (size_t)pt * 6 * w.smooth_ld;
+                sb.tid_s[pt] = 0x20000u + base; sb.tid_d[pt] = 0x30000u + base;
+                sb.prefix[pt + 1] = sb.prefix[pt] + (pt == 3 ? F : d) / 4;
+            }
+            launch_smooth_perturb(sb, seed, eps, eps != 0.0f, Z, w.smooth_ld, s);
+        }
+        {
+            PrepareBatch pb{};
+            pb.prefix[0] = 0;
+            for (int r = 0; r < 7; ++r) {
+                const Linear& L = Ly.lin[r];
+                if (!(L.present && L.adaptive() && L.bits(c.w_bits) != 0)) continue;
+                const int k = pb.count++;
+                pb.theta[k] = L.theta; pb.prep[k] = w.qprep + w.qprep_off[r]; pb.tid_q[k] = L.tid_q();
+                pb.prefix[k + 1] = pb.prefix[k] + L.rows * L.cols / c.w_group;
+            }
+            if (pb.count) {
+                ProfScope ps_(m, ZOQAT_PROF_WEIGHT, s);
+                launch_adapt_prepare(pb, c.w_bits, eps != 0.0f, seed, eps, Z, s);
+            }
+        }
         // --- attention block
-        if (smo) smooth_point(0, d);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(0)); }
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
             produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
-                            Ly.vec[ZOQAT_ROLE_BQ + r]);
+                            Ly.vec[ZOQAT_ROLE_BQ + r], r, 0);
         GemmArgs g{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
@@ -315,22 +350,20 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                                   llama ? w.rope_sin : nullptr, w.att, w.attn_scratch, w.err_flag, s)) {
               return fail(rc, "attention launch rejected");
           } }
-        if (smo) smooth_point(1, d);
-        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO]);
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1)); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         if (int rc = run_gemm(m, g, s)) return rc;
         // --- feed-forward block
-        if (smo) smooth_point(2, d);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, sa); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(2)); }
         const int n_up = llama ? 2 * F : F;
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1]);
-        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2);
+        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
@@ -343,13 +376,12 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             g.mode = 3; g.row_amax = w.row_amax;
         }
         if (int rc = run_gemm(m, g, s)) return rc;
-        if (smo) smooth_point(3, F);
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
-          if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, sa);
+          if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(3));
           else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
-          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, sa); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2]);
+          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3)); }
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
@@ -395,20 +427,27 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
     const int d = m->cfg.d_model, F = m->cfg.d_ffn;
     for (size_t l = 0; l < m->layers.size(); ++l) {
         Layer& Ly = m->layers[l];
+        UpdateBatch ub{};            // the layer's quantiser parameters and smoothing vectors: one launch
+        ub.prefix[0] = 0;
+        auto add = [&](float* ptr, uint64_t n, uint32_t tid, int smooth_class) {
+            const int k = ub.count++;
+            ub.ptr[k] = ptr; ub.tid[k] = tid; ub.smooth_class[k] = smooth_class;
+            ub.prefix[k + 1] = ub.prefix[k] + (int64_t)(n / 4);
+        };
         for (int r = 0; r < 7; ++r) {
             Linear& L = Ly.lin[r];
             if (!(L.present && L.trainable())) continue;
             launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
-            if (L.adaptive())
-                launch_update(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, seed, L.tid_q(), class_ptr, scale_q, s);
+            if (L.adaptive()) add(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, L.tid_q(), 0);
         }
         if (Ly.smoothing)
             for (int pt = 0; pt < 4; ++pt) {
                 const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
                 const uint64_t n = pt == 3 ? (uint64_t)F : (uint64_t)d;
-                launch_update(Ly.smooth_s[pt], n, seed, 0x20000u + base, class_ptr ? class_ptr + 1 : nullptr, scale_s, s);
-                launch_update(Ly.smooth_d[pt], n, seed, 0x30000u + base, class_ptr ? class_ptr + 1 : nullptr, scale_s, s);
+                add(Ly.smooth_s[pt], n, 0x20000u + base, 1);
+                add(Ly.smooth_d[pt], n, 0x30000u + base, 1);
             }
+        launch_update_batch(ub, seed, class_ptr, scale_q, scale_s, s);
     }
     if (m->head.trainable())
         launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
@@ -871,10 +910,11 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
                                     uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
                                     const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
                                     void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
+    if (!scratch_dev || (reinterpret_cast<uintptr_t>(scratch_dev) & 15)) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 16-byte aligned device memory");
     if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
     if (!w_dev || !operand_plus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_plus_dev are NULL");
     if (!theta_dev && !smooth_dev) return fail(ZOQAT_ERR_INVALID_ARG, "neither theta_dev nor smooth_dev given: use zoqat_op_weight_quant");
-    if (smooth_dev && (!bias_dev || !scratch_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "smoothing needs bias_dev and scratch_dev");
+    if (smooth_dev && !bias_dev) return fail(ZOQAT_ERR_INVALID_ARG, "smoothing needs bias_dev");
     if ((reinterpret_cast<uintptr_t>(theta_dev) | reinterpret_cast<uintptr_t>(smooth_dev) | reinterpret_cast<uintptr_t>(w_dev)) & 15)
         return fail(ZOQAT_ERR_INVALID_ARG, "w_dev, theta_dev and smooth_dev must be 16-byte aligned");
     LearnedOperandArgs a{};
@@ -882,7 +922,9 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
     a.seed = seed; a.tid = tensor_id; a.tid_q = tensor_id + 0x10000u; a.eps = eps;
     a.op_plus = static_cast<__nv_bfloat16*>(operand_plus_dev); a.op_minus = static_cast<__nv_bfloat16*>(operand_minus_dev);
     a.theta = theta_dev; a.smooth = smooth_dev; a.smooth_ld = (int)cols;
-    a.bias_part = scratch_dev; a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
+    // scratch: 16 floats per group for the prepared parameters, then 2 per group for the bias partial sums
+    a.prep = scratch_dev;
+    a.bias_part = scratch_dev + 16 * (rows * cols / group); a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
     a.codes = codes_dev;
     launch_weight_operand_learned(a, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
@@ -895,8 +937,10 @@ int zoqat_op_smooth_perturb(const float* scale_dev, const float* shift_dev, int6
     if (cols <= 0 || cols % 4 || cols > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a positive multiple of 4");
     if ((reinterpret_cast<uintptr_t>(scale_dev) | reinterpret_cast<uintptr_t>(shift_dev) | reinterpret_cast<uintptr_t>(out_dev)) & 15)
         return fail(ZOQAT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-    launch_smooth_perturb(scale_dev, shift_dev, (int)cols, seed, scale_id, shift_id, eps, eps != 0.0f, 2, out_dev, (int)cols,
-                          static_cast<cudaStream_t>(stream));
+    SmoothBatch sb{};
+    sb.count = 1; sb.scale[0] = scale_dev; sb.shift[0] = shift_dev; sb.out[0] = out_dev; sb.tid_s[0] = scale_id; sb.tid_d[0] = shift_id;
+    sb.prefix[0] = 0; sb.prefix[1] = (int)(cols / 4);
+    launch_smooth_perturb(sb, seed, eps, eps != 0.0f, 2, (int)cols, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -35,19 +35,32 @@ void launch_weight_operand(const float* w, int64_t n, int group, int bits, int p
 // (perturbed with tensor id tid_q).  smooth != NULL: [sign][kind][smooth_ld] perturbed smoothing vectors (kind 0
 // scale, 1 shift, 2 reciprocal scale); the quantiser sees scale (.) w' and bias_out[sign * bias_out_stride + row] =
 // bias0[row] (or 0) + shift . w'[row, :] (bias_part: scratch of 2 * rows * cols / group floats).
+// prep (theta != NULL): scratch of 2 passes * 2 * rows * cols / group float4 for the prepared group parameters.
 // op_minus == NULL: one operand with eps signed.  codes (may be NULL): uint8 codes of the op_plus side.
+constexpr int kMaxBatch = 16;
+// Batches of small per-layer work items served by one launch each.
+struct PrepareBatch {       // quantiser parameters of up to kMaxBatch tensors -> prepared per (group, sign) blocks
+    const float* theta[kMaxBatch]; void* prep[kMaxBatch]; uint32_t tid_q[kMaxBatch]; int64_t prefix[kMaxBatch + 1]; int count;
+};
+struct SmoothBatch {        // smoothing vectors of up to 4 quantisation points; prefix in 16-byte chunks
+    const float* scale[4]; const float* shift[4]; float* out[4]; uint32_t tid_s[4], tid_d[4]; int prefix[5]; int count;
+};
+struct UpdateBatch {        // Eq. (2) on up to kMaxBatch small tensors; prefix in Philox blocks (4 elements)
+    float* ptr[kMaxBatch]; uint32_t tid[kMaxBatch]; int smooth_class[kMaxBatch]; int64_t prefix[kMaxBatch + 1]; int count;
+};
+void launch_adapt_prepare(const PrepareBatch& b, int bits, int perturb, uint64_t seed, float eps, int signs, cudaStream_t s);
+void launch_smooth_perturb(const SmoothBatch& b, uint64_t seed, float eps, int perturb, int signs, int ld, cudaStream_t s);
+void launch_update_batch(const UpdateBatch& b, uint64_t seed, const float* class_ptr, float scale_q, float scale_s, cudaStream_t s);
 struct LearnedOperandArgs {
     const float* w; int64_t rows, cols; int group, bits, perturb;
     uint64_t seed; uint32_t tid, tid_q; float eps;
     __nv_bfloat16 *op_plus, *op_minus;
-    const float* theta;
+    const float* theta; void* prep; int prepared;   // prepared = 1: prep already holds this tensor's parameters
     const float* smooth; int smooth_ld;
     float* bias_part; const float* bias0; float* bias_out; int64_t bias_out_stride;
     uint8_t* codes;
 };
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s);
-void launch_smooth_perturb(const float* scale, const float* shift, int cols, uint64_t seed, uint32_t tid_s, uint32_t tid_d,
-                           float eps, int perturb, int signs, float* out, int ld, cudaStream_t s);
 void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s);
 void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s);
 void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);

@@ -3,9 +3,12 @@
 // and the update of Eq. (2).  All kernels stream the fp32 masters once with
 // 16-byte accesses; the direction is regenerated in registers (rng.cuh).
 //
-// Thread mapping of the operand producer: a thread owns 16 consecutive elements
-// (four Philox blocks), so a group is shared by group/16 adjacent lanes.  The
-// packing and update kernels map one Philox block (4 elements) to a thread.
+// Thread mapping of the operand producer: the group/16 adjacent lanes that share a
+// group own its elements interleaved - lane j takes the 16-byte chunks (Philox
+// blocks) j, j + group/16, j + 2*group/16, j + 3*group/16 of the group's span - so a
+// load instruction of the warp touches whole 128-byte lines (group 128) and every
+// thread still holds 16 elements of one group.  The packing and update kernels
+// map one Philox block (4 elements) to a thread.
 #include "common.cuh"
 #include "rng.cuh"
 
@@ -63,9 +66,9 @@ __device__ __forceinline__ void stage_icdf_table(float2* tab) {
     __syncthreads();
 }
 
-inline int stream_grid(int64_t work_items, int per_block) {
+inline int stream_grid(int64_t work_items, int per_block, int ctas_per_sm = 8) {
     int64_t blocks = (work_items + per_block - 1) / per_block;
-    const int64_t cap = 148 * 8;       // one resident wave of 256-thread CTAs (each stages the 16 KB table once)
+    const int64_t cap = 148 * ctas_per_sm;       // one resident wave of 256-thread CTAs (each stages the 16 KB table once)
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return (int)blocks;
@@ -163,11 +166,17 @@ __device__ __forceinline__ GroupQ quantise16(float (&x)[16], float qp, float* co
     return g;
 }
 
-__device__ __forceinline__ void store_bf16x16(uint4* dst, const float (&x)[16]) {
-    const uint2 a = pack_bf16x4(x[0], x[1], x[2], x[3]), b = pack_bf16x4(x[4], x[5], x[6], x[7]);
-    const uint2 c = pack_bf16x4(x[8], x[9], x[10], x[11]), d = pack_bf16x4(x[12], x[13], x[14], x[15]);
-    dst[0] = make_uint4(a.x, a.y, b.x, b.y);
-    dst[1] = make_uint4(c.x, c.y, d.x, d.y);
+// 16-byte chunk (= Philox block) k of the 16 elements that thread-item i owns: the LANES items of a group span
+// interleave their chunks.
+template <int LANES>
+__device__ __forceinline__ int64_t chunk_of(int64_t i, int k) {
+    return (i / LANES) * (4 * LANES) + (i % LANES) + LANES * k;
+}
+
+template <int LANES>
+__device__ __forceinline__ void store_bf16x16(uint2* dst, int64_t i, const float (&x)[16]) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) dst[chunk_of<LANES>(i, k)] = pack_bf16x4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
 }
 
 // One pass over a tensor: perturb, quantise per group, write the bf16 operand(s).
@@ -179,7 +188,7 @@ template <int GROUP, bool DUAL, bool DEBUG>
 __global__ void __launch_bounds__(kThreads)
 weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int perturb,
                       uint32_t k0, uint32_t k1, uint32_t tid, float eps,
-                      uint4* __restrict__ op_plus, uint4* __restrict__ op_minus,
+                      uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
                       uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp) {
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
@@ -192,13 +201,13 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         float x[16], xm[16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float4 v = live ? __ldg(w + 4 * i + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 v = live ? __ldg(w + chunk_of<LANES>(i, k)) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
         }
         if (perturb) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)(4 * i + k));
+                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk_of<LANES>(i, k));
                 const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -212,8 +221,8 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         }
         if (bits == 0) {
             if (live) {
-                store_bf16x16(op_plus + 2 * i, x);
-                if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
+                store_bf16x16<LANES>(op_plus, i, x);
+                if (DUAL) store_bf16x16<LANES>(op_minus, i, xm);
             }
             continue;
         }
@@ -221,12 +230,12 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
             float cd[16];
             const GroupQ g = quantise16<LANES>(x, qp, DEBUG ? cd : nullptr);
             if (live) {
-                store_bf16x16(op_plus + 2 * i, x);
+                store_bf16x16<LANES>(op_plus, i, x);
                 if (DEBUG) {
                     if (codes) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            codes[4 * i + k] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
+                            codes[chunk_of<LANES>(i, k)] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
                                                            (unsigned char)cd[4 * k + 2], (unsigned char)cd[4 * k + 3]);
                     }
                     if ((i % LANES) == 0) {
@@ -238,7 +247,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         }
         if (DUAL) {
             quantise16<LANES>(xm, qp, nullptr);
-            if (live) store_bf16x16(op_minus + 2 * i, xm);
+            if (live) store_bf16x16<LANES>(op_minus, i, xm);
         }
     }
 }
@@ -268,19 +277,61 @@ __device__ __forceinline__ void quantise16_adaptive(float (&x)[16], const AdaptQ
     }
 }
 
+// The same quantiser with the zero point folded into the clamp: value = clamp(round(x * inv), lo - z, hi - z) * step.
+// Every term is an integer, so this is the same number whenever lo - z and hi - z are exact in binary32
+// (|z| < 2^24 - 16; when round(x * inv) + z would round, it lies far outside [lo, hi] and both forms clamp).
+__device__ __forceinline__ void quantise16_folded(float (&x)[16], const float4& a) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = __fmul_rn(fminf(fmaxf(rintf(__fmul_rn(x[j], a.y)), a.z), a.w), a.x);
+}
+
+// Perturbs the quantiser parameters of every group once (one Philox block per group, tensor id tid_q) and derives
+// what the producer needs, per (group, sign): A = (step, 1/step, lo - z, hi - z), B = (z, lo, hi, 0), all after
+// rounding / limiting.  A.z is NaN when the folded form is not exact for the group (|z| >= 2^24 - 16).
+// One launch serves up to kMaxBatch tensors (the linears of a layer): tensor t owns groups [prefix[t], prefix[t+1])
+// and writes its A block, then its B block, at prep[t].
+__global__ void __launch_bounds__(kThreads)
+adapt_prepare_kernel(PrepareBatch b, int bits, int perturb, uint32_t k0, uint32_t k1, float eps, int signs) {
+    __shared__ float2 tab[kIcdfKnots];
+    if (perturb) stage_icdf_table(tab);
+    const float qp = (float)((1 << bits) - 1);
+    const int64_t total = b.prefix[b.count];
+    for (int64_t gi = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; gi < total; gi += (int64_t)gridDim.x * blockDim.x) {
+        int t = 0;
+        while (t + 1 < b.count && gi >= b.prefix[t + 1]) ++t;
+        const int64_t g = gi - b.prefix[t];
+        const float4 th = __ldg(reinterpret_cast<const float4*>(b.theta[t]) + g);
+        float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (perturb) u = direction4(tab, k0, k1, b.tid_q[t], (uint64_t)g);
+        float4* out_a = reinterpret_cast<float4*>(b.prep[t]);
+        float4* out_b = out_a + (b.prefix[t + 1] - b.prefix[t]) * signs;
+        for (int sg = 0; sg < signs; ++sg) {
+            const float e = sg == 0 ? eps : -eps;
+            float4 v = th;
+            if (perturb) v = make_float4(__fmaf_rn(e, u.x, th.x), __fmaf_rn(e, u.y, th.y), __fmaf_rn(e, u.z, th.z), __fmaf_rn(e, u.w, th.w));
+            const AdaptQ a = adapt_params(v, qp);
+            const bool exact = fabsf(a.zr) < 16777200.0f;
+            out_a[g * signs + sg] = make_float4(a.step, a.inv, exact ? __fadd_rn(a.lo, -a.zr) : __int_as_float(0x7fc00000),
+                                                __fadd_rn(a.hi, -a.zr));
+            out_b[g * signs + sg] = make_float4(a.zr, a.lo, a.hi, 0.0f);
+        }
+    }
+}
+
 // The operand producer with the learnable parts of Section 4.2 (same thread mapping as weight_operand_kernel):
 //   SMOOTH  the quantiser sees s' (.) w' (s' = perturbed per-input-channel scale); the per-group partial sums of
 //           delta' . w' (the shift term of the smoothed bias, with the unscaled perturbed weight) go to bias_part,
 //           [sign][group], and are reduced per output row by bias_reduce_kernel;
-//   ADAPT   the group's (step, z, alpha, beta) are read from theta and perturbed with their own direction
-//           (tensor id tid_q, one Philox block per group) instead of being derived from min/max.
+//   ADAPT   the group's quantiser comes from the learnable parameters, perturbed and prepared per (group, sign) by
+//           adapt_prepare_kernel (prep_a / prep_b), instead of being derived from min/max.
 // smooth: [sign][kind][smooth_ld] floats, kind 0 = scale, 1 = shift (2 = 1/scale, used by the activation side).
 template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH>
-__global__ void __launch_bounds__(kThreads)
-weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols16, int bits, int perturb,
-                              uint32_t k0, uint32_t k1, uint32_t tid, uint32_t tid_q, float eps,
-                              uint4* __restrict__ op_plus, uint4* __restrict__ op_minus,
-                              const float4* __restrict__ theta, const float* __restrict__ smooth, int smooth_ld,
+__global__ void __launch_bounds__(kThreads, 3)
+weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols4, int bits, int perturb,
+                              uint32_t k0, uint32_t k1, uint32_t tid, float eps,
+                              uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
+                              const float4* __restrict__ prep_a, const float4* __restrict__ prep_b,
+                              const float* __restrict__ smooth, int smooth_ld,
                               float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes) {
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
@@ -292,13 +343,13 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
         float x[16], xm[16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float4 v = live ? __ldg(w + 4 * i + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 v = live ? __ldg(w + chunk_of<LANES>(i, k)) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
         }
         if (perturb) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)(4 * i + k));
+                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk_of<LANES>(i, k));
                 const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -311,16 +362,17 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
             for (int j = 0; j < 16; ++j) xm[j] = x[j];
         }
         if (SMOOTH) {
-            const int col0 = (int)(i % cols16) * 16;
-            const float4* sp = reinterpret_cast<const float4*>(smooth + col0);
-            const float4* dp = reinterpret_cast<const float4*>(smooth + smooth_ld + col0);
-            const float4* sm = reinterpret_cast<const float4*>(smooth + 3 * (size_t)smooth_ld + col0);
-            const float4* dm = reinterpret_cast<const float4*>(smooth + 4 * (size_t)smooth_ld + col0);
+            // column (in 16-byte chunks) of chunk 0; the following chunks are LANES further, wrapping at the row end
+            int c4 = (int)(chunk_of<LANES>(i, 0) % cols4);
+            const float4* sp = reinterpret_cast<const float4*>(smooth);
+            const float4* dp = reinterpret_cast<const float4*>(smooth + smooth_ld);
+            const float4* sm = reinterpret_cast<const float4*>(smooth + 3 * (size_t)smooth_ld);
+            const float4* dm = reinterpret_cast<const float4*>(smooth + 4 * (size_t)smooth_ld);
             float bp = 0.0f, bm = 0.0f;
             if (live) {
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const float4 s4 = __ldg(sp + k), d4 = __ldg(dp + k);
+                    const float4 s4 = __ldg(sp + c4), d4 = __ldg(dp + c4);
                     const float ss[4] = {s4.x, s4.y, s4.z, s4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -328,7 +380,7 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                         x[4 * k + j] = __fmul_rn(x[4 * k + j], ss[j]);
                     }
                     if (DUAL) {
-                        const float4 t4 = __ldg(sm + k), e4 = __ldg(dm + k);
+                        const float4 t4 = __ldg(sm + c4), e4 = __ldg(dm + c4);
                         const float ts[4] = {t4.x, t4.y, t4.z, t4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -336,6 +388,8 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                             xm[4 * k + j] = __fmul_rn(xm[4 * k + j], ts[j]);
                         }
                     }
+                    c4 += LANES;
+                    if (c4 >= cols4) c4 -= cols4;
                 }
             }
 #pragma unroll
@@ -350,62 +404,74 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
         }
         if (bits == 0) {
             if (live) {
-                store_bf16x16(op_plus + 2 * i, x);
-                if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
+                store_bf16x16<LANES>(op_plus, i, x);
+                if (DUAL) store_bf16x16<LANES>(op_minus, i, xm);
             }
             continue;
         }
+        // one sign at a time, so that only one set of group parameters and one operand is live
         float cd[16];
-        if (ADAPT) {
-            const float4 th = live ? __ldg(theta + i / LANES) : make_float4(1.f, 0.f, 0.f, 1.f);
-            float4 tp = th, tm = th;
-            if (perturb) {
-                const float4 u = direction4(tab, k0, k1, tid_q, (uint64_t)(i / LANES));
-                tp = make_float4(__fmaf_rn(eps, u.x, th.x), __fmaf_rn(eps, u.y, th.y), __fmaf_rn(eps, u.z, th.z), __fmaf_rn(eps, u.w, th.w));
-                if (DUAL) tm = make_float4(__fmaf_rn(-eps, u.x, th.x), __fmaf_rn(-eps, u.y, th.y), __fmaf_rn(-eps, u.z, th.z), __fmaf_rn(-eps, u.w, th.w));
-            }
-            quantise16_adaptive(x, adapt_params(tp, qp), codes ? cd : nullptr);
-            if (DUAL) quantise16_adaptive(xm, adapt_params(tm, qp), nullptr);
-        } else {
-            quantise16<LANES>(x, qp, codes ? cd : nullptr);
-            if (DUAL) quantise16<LANES>(xm, qp, nullptr);
-        }
-        if (live) {
-            store_bf16x16(op_plus + 2 * i, x);
-            if (DUAL) store_bf16x16(op_minus + 2 * i, xm);
-            if (codes) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    codes[4 * i + k] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
-                                                   (unsigned char)cd[4 * k + 2], (unsigned char)cd[4 * k + 3]);
+        for (int sg = 0; sg < (DUAL ? 2 : 1); ++sg) {
+            float (&v)[16] = sg == 0 ? x : xm;
+            float* cdp = (sg == 0 && codes) ? cd : nullptr;
+            if (ADAPT) {
+                constexpr int SG = DUAL ? 2 : 1;
+                const int64_t slot = (i / LANES) * SG + sg;
+                const float4 a = live ? __ldg(prep_a + slot) : make_float4(1.f, 1.f, 0.f, 0.f);
+                const bool literal = (a.z != a.z) || cdp != nullptr;
+                if (__any_sync(0xffffffffu, literal)) {       // zero point beyond exact integer arithmetic, or codes wanted
+                    const float4 b = live ? __ldg(prep_b + slot) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const AdaptQ q = {a.x, a.y, b.x, b.y, b.z};
+                    quantise16_adaptive(v, q, cdp);
+                } else {
+                    quantise16_folded(v, a);
+                }
+            } else {
+                quantise16<LANES>(v, qp, cdp);
             }
+            if (live) store_bf16x16<LANES>(sg == 0 ? op_plus : op_minus, i, v);
+        }
+        if (live && codes) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                codes[chunk_of<LANES>(i, k)] = make_uchar4((unsigned char)cd[4 * k], (unsigned char)cd[4 * k + 1],
+                                               (unsigned char)cd[4 * k + 2], (unsigned char)cd[4 * k + 3]);
         }
     }
 }
 
-// out[sign][row] = bias0[row] + sum over the row's groups of bias_part[sign][row * gpr + g], in a fixed order.
+// out[sign][row] = bias0[row] + sum over the row's groups of bias_part[sign][row * gpr + g]; one warp per (sign, row),
+// lane-strided partial sums in double and a fixed shuffle tree, so the result does not depend on timing.
 __global__ void bias_reduce_kernel(const float* __restrict__ part, int64_t n_groups, int gpr, int rows, int signs,
                                    const float* __restrict__ bias0, float* __restrict__ out, int64_t out_sign_stride) {
-    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t idx = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     if (idx >= (int64_t)rows * signs) return;
+    const int lane = threadIdx.x & 31;
     const int sgn = (int)(idx / rows), r = (int)(idx % rows);
     const float* p = part + (int64_t)sgn * n_groups + (int64_t)r * gpr;
     double acc = 0.0;
-    for (int g = 0; g < gpr; ++g) acc += (double)p[g];
-    out[(int64_t)sgn * out_sign_stride + r] = (float)(acc + (bias0 ? (double)bias0[r] : 0.0));
+    for (int g = lane; g < gpr; g += 32) acc += (double)p[g];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) out[(int64_t)sgn * out_sign_stride + r] = (float)(acc + (bias0 ? (double)bias0[r] : 0.0));
 }
 
-// Perturbed smoothing vectors of one quantisation point: out[sign][kind][ld], kind 0 = s' = s +/- eps u_s,
-// 1 = delta' = delta +/- eps u_delta, 2 = 1 / s' (rounded once).  sign 0 uses +eps (eps may be signed), sign 1 -eps.
+// Perturbed smoothing vectors of up to four quantisation points in one launch: out[t][sign][kind][ld], kind 0 = s' =
+// s +/- eps u_s, 1 = delta' = delta +/- eps u_delta, 2 = 1 / s' (rounded once).  sign 0 uses +eps (eps may be signed),
+// sign 1 -eps.  Point t owns 16-byte chunks [prefix[t], prefix[t+1]).
 __global__ void __launch_bounds__(kThreads)
-smooth_perturb_kernel(const float4* __restrict__ s, const float4* __restrict__ d, int n4, uint32_t k0, uint32_t k1,
-                      uint32_t tid_s, uint32_t tid_d, float eps, int perturb, int signs, float* __restrict__ out, int ld) {
+smooth_perturb_kernel(SmoothBatch sb, uint32_t k0, uint32_t k1, float eps, int perturb, int signs, int ld) {
     __shared__ float2 tab[kIcdfKnots];
     if (perturb) stage_icdf_table(tab);
-    for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < n4; b += gridDim.x * blockDim.x) {
-        const float4 s4 = s[b], d4 = d[b];
+    const int total = sb.prefix[sb.count];
+    for (int gi = blockIdx.x * blockDim.x + threadIdx.x; gi < total; gi += gridDim.x * blockDim.x) {
+        int t = 0;
+        while (t + 1 < sb.count && gi >= sb.prefix[t + 1]) ++t;
+        const int b = gi - sb.prefix[t];
+        const float4 s4 = reinterpret_cast<const float4*>(sb.scale[t])[b], d4 = reinterpret_cast<const float4*>(sb.shift[t])[b];
         float4 us = make_float4(0.f, 0.f, 0.f, 0.f), ud = us;
-        if (perturb) { us = direction4(tab, k0, k1, tid_s, (uint64_t)b); ud = direction4(tab, k0, k1, tid_d, (uint64_t)b); }
+        if (perturb) { us = direction4(tab, k0, k1, sb.tid_s[t], (uint64_t)b); ud = direction4(tab, k0, k1, sb.tid_d[t], (uint64_t)b); }
         for (int sg = 0; sg < signs; ++sg) {
             const float e = sg == 0 ? eps : -eps;
             float4 a = s4, c = d4;
@@ -413,12 +479,33 @@ smooth_perturb_kernel(const float4* __restrict__ s, const float4* __restrict__ d
                 a = make_float4(__fmaf_rn(e, us.x, s4.x), __fmaf_rn(e, us.y, s4.y), __fmaf_rn(e, us.z, s4.z), __fmaf_rn(e, us.w, s4.w));
                 c = make_float4(__fmaf_rn(e, ud.x, d4.x), __fmaf_rn(e, ud.y, d4.y), __fmaf_rn(e, ud.z, d4.z), __fmaf_rn(e, ud.w, d4.w));
             }
-            float* o = out + (size_t)sg * 3 * ld;
+            float* o = sb.out[t] + (size_t)sg * 3 * ld;
             reinterpret_cast<float4*>(o)[b] = a;
             reinterpret_cast<float4*>(o + ld)[b] = c;
             reinterpret_cast<float4*>(o + 2 * (size_t)ld)[b] =
                 make_float4(__fdiv_rn(1.0f, a.x), __fdiv_rn(1.0f, a.y), __fdiv_rn(1.0f, a.z), __fdiv_rn(1.0f, a.w));
         }
+    }
+}
+
+// Eq. (2) on a batch of small tensors (the quantiser parameters and smoothing vectors of a layer) in one launch:
+// tensor t owns Philox blocks [prefix[t], prefix[t+1]); every tensor has a multiple of 4 elements.
+__global__ void __launch_bounds__(kThreads)
+update_batch_kernel(UpdateBatch ub, uint32_t k0, uint32_t k1, const float* __restrict__ class_ptr, float scale_q, float scale_s) {
+    __shared__ float2 tab[kIcdfKnots];
+    stage_icdf_table(tab);
+    const float cq = -(class_ptr ? class_ptr[0] : scale_q), cs = -(class_ptr ? class_ptr[1] : scale_s);
+    const int64_t total = ub.prefix[ub.count];
+    for (int64_t gi = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; gi < total; gi += (int64_t)gridDim.x * blockDim.x) {
+        int t = 0;
+        while (t + 1 < ub.count && gi >= ub.prefix[t + 1]) ++t;
+        const int64_t b = gi - ub.prefix[t];
+        const float c = ub.smooth_class[t] ? cs : cq;
+        const float4 z = direction4(tab, k0, k1, ub.tid[t], (uint64_t)b);
+        float4* w4 = reinterpret_cast<float4*>(ub.ptr[t]) + b;
+        float4 x = *w4;
+        x.x = __fmaf_rn(c, z.x, x.x); x.y = __fmaf_rn(c, z.y, x.y); x.z = __fmaf_rn(c, z.z, x.z); x.w = __fmaf_rn(c, z.w, x.w);
+        *w4 = x;
     }
 }
 
@@ -606,8 +693,8 @@ static void weight_operand_dispatch(const float* w, int64_t n, int bits, int per
     const int grid = stream_grid(n16, kThreads);
     const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
     const float4* w4 = reinterpret_cast<const float4*>(w);
-    uint4* p = reinterpret_cast<uint4*>(op_plus);
-    uint4* m = reinterpret_cast<uint4*>(op_minus);
+    uint2* p = reinterpret_cast<uint2*>(op_plus);
+    uint2* m = reinterpret_cast<uint2*>(op_minus);
     uchar4* c4 = reinterpret_cast<uchar4*>(codes);
     const bool debug = codes || step || zp;
     if (op_minus) {
@@ -632,26 +719,32 @@ void launch_weight_operand(const float* w, int64_t n, int group, int bits, int p
 template <int GROUP, bool ADAPT, bool SMOOTH>
 static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
     const int64_t n16 = a.rows * a.cols / 16;
-    const int grid = stream_grid(n16, kThreads);
+    const int grid = stream_grid(n16, kThreads, 3);        // 80 registers: three CTAs per SM
     const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
     const float4* w4 = reinterpret_cast<const float4*>(a.w);
-    uint4* p = reinterpret_cast<uint4*>(a.op_plus);
-    uint4* m = reinterpret_cast<uint4*>(a.op_minus);
-    const float4* th = reinterpret_cast<const float4*>(a.theta);
+    uint2* p = reinterpret_cast<uint2*>(a.op_plus);
+    uint2* m = reinterpret_cast<uint2*>(a.op_minus);
     const int64_t n_groups = a.rows * a.cols / GROUP;
+    const int signs = a.op_minus ? 2 : 1;
+    float4* pa = reinterpret_cast<float4*>(a.prep);
+    float4* pb = pa + n_groups * signs;
     uchar4* c4 = reinterpret_cast<uchar4*>(a.codes);
+    if (ADAPT && !a.prepared) {
+        PrepareBatch pb1{};
+        pb1.count = 1; pb1.theta[0] = a.theta; pb1.prep[0] = a.prep; pb1.tid_q[0] = a.tid_q; pb1.prefix[0] = 0; pb1.prefix[1] = n_groups;
+        launch_adapt_prepare(pb1, a.bits, a.perturb, a.seed, a.eps, signs, s);
+    }
     if (a.op_minus)
         weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 16), a.bits, a.perturb, k0, k1, a.tid, a.tid_q, a.eps, p, m, th, a.smooth, a.smooth_ld,
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
             a.bias_part, n_groups, c4);
     else
         weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 16), a.bits, a.perturb, k0, k1, a.tid, a.tid_q, a.eps, p, nullptr, th, a.smooth, a.smooth_ld,
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
             a.bias_part, n_groups, c4);
     count_launch();
     if (SMOOTH) {
-        const int signs = a.op_minus ? 2 : 1;
-        const int64_t work = a.rows * signs;
+        const int64_t work = a.rows * signs * 32;
         bias_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(a.bias_part, n_groups, (int)(a.cols / GROUP), (int)a.rows,
                                                                           signs, a.bias0, a.bias_out, a.bias_out_stride);
         count_launch();
@@ -673,14 +766,25 @@ void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s) 
     else learned_dispatch_group<128>(a, s);
 }
 
-void launch_smooth_perturb(const float* scale, const float* shift, int cols, uint64_t seed, uint32_t tid_s, uint32_t tid_d,
-                           float eps, int perturb, int signs, float* out, int ld, cudaStream_t s) {
-    if (cols == 0 || (perturb && !ensure_icdf_table())) return;
-    const int n4 = cols / 4;
-    int blocks = (n4 + kThreads - 1) / kThreads;
-    if (blocks > 8) blocks = 8;
-    smooth_perturb_kernel<<<blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(scale), reinterpret_cast<const float4*>(shift), n4,
-                                                      (uint32_t)seed, (uint32_t)(seed >> 32), tid_s, tid_d, eps, perturb, signs, out, ld);
+void launch_adapt_prepare(const PrepareBatch& b, int bits, int perturb, uint64_t seed, float eps, int signs, cudaStream_t s) {
+    if (b.count == 0 || b.prefix[b.count] == 0 || (perturb && !ensure_icdf_table())) return;
+    adapt_prepare_kernel<<<stream_grid(b.prefix[b.count], kThreads), kThreads, 0, s>>>(b, bits, perturb, (uint32_t)seed,
+                                                                                       (uint32_t)(seed >> 32), eps, signs);
+    count_launch();
+}
+
+void launch_smooth_perturb(const SmoothBatch& b, uint64_t seed, float eps, int perturb, int signs, int ld, cudaStream_t s) {
+    if (b.count == 0 || b.prefix[b.count] == 0 || (perturb && !ensure_icdf_table())) return;
+    int blocks = (b.prefix[b.count] + kThreads - 1) / kThreads;
+    if (blocks > 32) blocks = 32;
+    smooth_perturb_kernel<<<blocks, kThreads, 0, s>>>(b, (uint32_t)seed, (uint32_t)(seed >> 32), eps, perturb, signs, ld);
+    count_launch();
+}
+
+void launch_update_batch(const UpdateBatch& b, uint64_t seed, const float* class_ptr, float scale_q, float scale_s, cudaStream_t s) {
+    if (b.count == 0 || b.prefix[b.count] == 0 || !ensure_icdf_table()) return;
+    update_batch_kernel<<<stream_grid(b.prefix[b.count], kThreads), kThreads, 0, s>>>(b, (uint32_t)seed, (uint32_t)(seed >> 32),
+                                                                                      class_ptr, scale_q, scale_s);
     count_launch();
 }
 

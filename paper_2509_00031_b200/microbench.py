@@ -3,6 +3,7 @@ between iterations) and prints one JSON line per kernel with its achieved rate.
 
   python -m paper_2509_00031_b200.microbench --op gemm --M 8192 --N 4096 --K 4096 [--iters 10]
   python -m paper_2509_00031_b200.microbench --op weight_pair --rows 11008 --cols 4096 --bits 4 --group 128
+  python -m paper_2509_00031_b200.microbench --op weight_learned --rows 11008 --cols 4096     (Section 4.2 producer)
   python -m paper_2509_00031_b200.microbench --op update --rows 11008 --cols 4096
   python -m paper_2509_00031_b200.microbench --op attention --batch 8 --seq 1024 --heads 32 --dh 128
   python -m paper_2509_00031_b200.microbench --op norm_act --rows 8192 --cols 4096
@@ -71,10 +72,15 @@ def main():
         med, best = timed(fn, a.iters, flush)
         flops = 2.0 * a.M * a.N * a.K
         out.update(M=a.M, N=a.N, K=a.K, ms=med, ms_best=best, tflops=flops / med / 1e9, tflops_best=flops / best / 1e9)
-    elif a.op in ("weight_pair", "weight_single", "update", "unpack"):
+    elif a.op in ("weight_pair", "weight_single", "weight_learned", "update", "unpack"):
         W = torch.randn(a.rows, a.cols, device=dev) * 0.02
         n = a.rows * a.cols
-        if a.op == "weight_pair":
+        if a.op == "weight_learned":
+            theta = zq.zoqat_op_init_qparams(W, a.group, a.bits)
+            smooth = zq.zoqat_op_smooth_perturb(torch.ones(a.cols, device=dev), torch.zeros(a.cols, device=dev), 1000, 0x20010, 0x30010, 1e-3)
+            fn = lambda: zq.zoqat_op_weight_operand_learned(W, a.group, a.bits, 1000, 16, 1e-3, theta=theta, smooth=smooth)
+            nbytes = n * (4 + 2 + 2 + 16 / a.group)
+        elif a.op == "weight_pair":
             fn = lambda: zq.zoqat_op_weight_operand_pair(W, a.group, a.bits, 1000, 16, 1e-3)
             nbytes = n * (4 + 2 + 2)
         elif a.op == "weight_single":

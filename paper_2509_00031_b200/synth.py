@@ -27,6 +27,13 @@ WORKLOADS = {
     "llama7b_qv_light": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
                              w_bits=4, w_group=128, a_bits=8, batch=4, seq=1024, bf16_init=True,
                              trainable_names=("wq", "wv"), head_trainable=False),
+    # Section 4.2 on the 7B shape: learnable per-group quantiser parameters and per-channel smoothing in every layer
+    "llama7b_w4a8_learned": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                 w_bits=4, w_group=128, a_bits=8, batch=4, seq=1024, bf16_init=True,
+                                 adaptive_quant=True, smoothing=True),
+    "llama7b_w4a4_learned": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                 w_bits=4, w_group=128, a_bits=4, batch=4, seq=1024, bf16_init=True,
+                                 adaptive_quant=True, smoothing=True),
 }
 
 
