@@ -143,3 +143,35 @@ def test_ffn_and_norm_operands_bench_shape_sampled(zq):
     assert np.allclose(normed[rows].cpu().numpy(), wantn, rtol=2e-6, atol=2e-6)
     q_self, s_self = act_quant(normed[rows].double().cpu().numpy())
     assert np.array_equal(op[rows].float().cpu().numpy(), q_self) and np.array_equal(step[rows].cpu().numpy(), s_self)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (2, 64)])
+def test_learned_producer_full_tensor(zq, bits, group):
+    """Section 4.2 producer (learnable group parameters + smoothing) on one down-projection-sized tensor
+    (4096 x 11008: rows that are not a multiple of the 128-byte line pattern, many grid-stride iterations):
+    sampled rows bit for bit, the shift term of the bias to binary32 accuracy on every row."""
+    from oracle.model import adaptive_weight_quant, init_quant_params, QPARAM_ID
+    rng = np.random.default_rng(bits)
+    w = _weights(D, F, 8)
+    w_np = w.cpu().numpy()
+    theta = init_quant_params(w_np, group, bits)
+    theta[..., 0] *= rng.uniform(0.8, 1.15, theta.shape[:-1]).astype(np.float32)
+    theta[..., 2] = rng.uniform(0.0, 0.2, theta.shape[:-1]).astype(np.float32)
+    theta[..., 3] = rng.uniform(0.7, 1.0, theta.shape[:-1]).astype(np.float32)
+    s = rng.uniform(0.5, 2.0, F).astype(np.float32)
+    d = (0.3 * rng.standard_normal(F)).astype(np.float32)
+    seed, tid, eps = 1009, 16 * 7 + 6, np.float32(1e-3)
+    smooth = zq.zoqat_op_smooth_perturb(torch.from_numpy(s).cuda(), torch.from_numpy(d).cuda(), seed, 0x20073, 0x30073, float(eps))
+    plus, minus, bias, _ = zq.zoqat_op_weight_operand_learned(w, group, bits, seed, tid, float(eps), theta=torch.from_numpy(theta).cuda(),
+                                                              smooth=smooth)
+    rows = np.array([0, 1, 2047, 2048, 4094, 4095])
+    for sg, (e, op) in enumerate(((eps, plus), (-eps, minus))):
+        wp = core.perturb(w_np, seed, tid, e)
+        sp = core.perturb(s, seed, 0x20073, e)
+        dp = core.perturb(d, seed, 0x30073, e)
+        thp = core.perturb(theta, seed, tid + QPARAM_ID, e)
+        _, deq = adaptive_weight_quant((wp[rows] * sp[None, :]).astype(np.float32), thp[rows], group, bits)
+        assert np.array_equal(op[rows].float().cpu().numpy(), core.round_bf16(deq))
+        want_bias = wp.astype(np.float64) @ dp.astype(np.float64)
+        scale = np.abs(wp.astype(np.float64)) @ np.abs(dp.astype(np.float64))
+        assert np.all(np.abs(bias[sg].cpu().numpy() - want_bias) <= 2e-6 * scale + 1e-9)
