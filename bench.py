@@ -53,9 +53,10 @@ def workload_numbers(w):
     lin_flops = 2 * T * (per_layer * ftl + 2 * per_layer * (L - ftl) + 2 * head)
     attn_flops = 2 * w["batch"] * w["seq"] ** 2 * d * (ftl + 2 * (L - ftl))
     frozen = per_layer * L - per_layer_trainable * (L - ftl)
-    bytes_step = 4 * trainable + (w["w_bits"] / 8 + 8 / w["w_group"]) * frozen + 8 * trainable
+    group = w["w_group"] or d           # 0 = one group per output row (rows of d or F columns: d is the smaller)
+    bytes_step = 4 * trainable + ((w["w_bits"] / 8 + 8 / group) * frozen if frozen else 0) + 8 * trainable
     if w.get("adaptive_quant"):         # four fp32 quantiser parameters per group: read once per step pair, read + written by Eq. (2)
-        bytes_step += 12 * 4 * per_layer_trainable * (L - ftl) / w["w_group"]
+        bytes_step += 12 * 4 * per_layer_trainable * (L - ftl) / group
     return dict(T=T, block_params=block, trainable_params=trainable, head_params=head,
                 linear_flops=lin_flops, attn_flops=attn_flops, flops=lin_flops + attn_flops, bytes=bytes_step)
 

@@ -115,8 +115,10 @@ typedef struct zoqat_config {
     int32_t vocab;
     int32_t max_batch;     /* largest batch ...                                                   */
     int32_t max_seq;       /* ... and sequence length a call will pass                            */
-    int32_t w_bits;        /* 2, 3 or 4                                                           */
-    int32_t w_group;       /* 32, 64 or 128; divides d_model and d_ffn                            */
+    int32_t w_bits;        /* 2..8 (FROZEN_PACKED tensors: 2, 3 or 4)                             */
+    int32_t w_group;       /* 32, 64 or 128 (divides d_model and d_ffn), or 0 = one group per output
+                              row ("per-channel" weights; d_model, d_ffn multiples of 128; not for
+                              FROZEN_PACKED tensors)                                              */
     int32_t a_bits;        /* 4, 6 or 8 = per-token symmetric N-bit codes on block-linear inputs, 0 = none */
     int32_t gemm_impl;     /* ZOQAT_GEMM_*                                                        */
     float   norm_eps;
@@ -310,7 +312,9 @@ int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols,
  *     (first equation of Section 4.2: the smoothed bias uses the unscaled, unquantised perturbed weight).
  *   scratch_dev: 18 * rows * cols / group floats, 16-byte aligned (prepared group parameters, bias partial sums).
  * operand_minus_dev may be NULL: one operand (and one bias vector) with eps signed.
- * codes_dev (may be NULL): uint8 [rows, cols] codes of the +eps side. */
+ * codes_dev (may be NULL): uint8 [rows, cols] codes of the +eps side.
+ * group = 0: one quantisation group per row (cols % 128 == 0; theta_dev then [rows, 1, 4]; theta_dev and
+ * smooth_dev may both be NULL: plain min/max over the row); the scratch size is that of group 128. */
 int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
                                     uint64_t seed, uint32_t tensor_id, float eps,
                                     const float* theta_dev, const float* smooth_dev,
@@ -330,7 +334,8 @@ int zoqat_op_smooth_act_operand(const float* x_dev, int64_t rows, int64_t cols, 
                                 const float* bias_dev, float norm_eps, int a_bits, const float* smooth_dev,
                                 int64_t rows_per_pass, void* operand_dev, float* row_step_dev, void* stream);
 
-/* Initial quantiser parameters of one tensor (what zoqat_init_qparams writes): theta_dev fp32 [rows, cols/group, 4]. */
+/* Initial quantiser parameters of one tensor (what zoqat_init_qparams writes): theta_dev fp32 [rows, cols/group, 4]
+ * (group = 0: [rows, 1, 4], one group per row). */
 int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, float* theta_dev,
                           void* stream);
 

@@ -101,7 +101,7 @@ class OracleConfig:
     d_ffn: int
     vocab: int
     w_bits: int = 4
-    w_group: int = 128
+    w_group: int = 128        # 0 = one group per output row ("per-channel" weights of the appendix on quantisation settings)
     a_bits: int = 8           # 4 / 6 / 8 = per-token symmetric N-bit codes on block-linear inputs, 0 = none
     norm_eps: float = 1e-5
     rope_base: float = 10000.0
@@ -192,6 +192,9 @@ class OracleModel:
     def is_trainable(self, l, name):
         return l >= self.cfg.first_trainable_layer and (self.cfg.trainable_names is None or name in self.cfg.trainable_names)
 
+    def group_of(self, w):
+        return self.cfg.w_group if self.cfg.w_group else w.shape[1]
+
     def has_smoothing(self, l):
         return self.cfg.smoothing and l >= self.cfg.first_trainable_layer
 
@@ -207,7 +210,7 @@ class OracleModel:
             P = self.p["layers"][l]
             for n in self.linear_names():
                 if self.has_adaptive(l, n):
-                    P["theta_" + n] = init_quant_params(P[n], cfg.w_group, cfg.w_bits)
+                    P["theta_" + n] = init_quant_params(P[n], self.group_of(P[n]), cfg.w_bits)
             if self.has_smoothing(l):
                 for n in self.linear_names():
                     pt = POINTS[POINT_OF[n]]
@@ -266,9 +269,9 @@ class OracleModel:
             th = self.p["layers"][l]["theta_" + name]
             if signed_eps != 0.0:
                 th = core.perturb(th, seed, tensor_id(l, self._ROLE[name]) + QPARAM_ID, signed_eps)
-            _, deq = adaptive_weight_quant(w, th, cfg.w_group, cfg.w_bits)
+            _, deq = adaptive_weight_quant(w, th, self.group_of(w), cfg.w_bits)
         else:
-            _, _, _, deq = core.weight_quant(w, cfg.w_group, cfg.w_bits)
+            _, _, _, deq = core.weight_quant(w, self.group_of(w), cfg.w_bits)
         return (core.round_bf16(deq) if cfg.operand_bf16 else deq).astype(np.float64)
 
     def head_operand(self, seed, signed_eps):

@@ -179,8 +179,9 @@ def zoqat_op_weight_operand_pair(w, group, bits, seed, tensor_id, eps):
 
 
 def zoqat_op_init_qparams(w, group, bits):
+    """group = 0: one group per row."""
     rows, cols = w.shape
-    theta = torch.empty((rows, cols // group, 4), dtype=torch.float32, device=w.device)
+    theta = torch.empty((rows, cols // group if group else 1, 4), dtype=torch.float32, device=w.device)
     _check(lib().zoqat_op_init_qparams(_p(w), rows, cols, group, bits, _p(theta), _stream()))
     return theta
 
@@ -200,7 +201,7 @@ def zoqat_op_weight_operand_learned(w, group, bits, seed, tensor_id, eps, theta=
     plus = torch.empty((rows, cols), dtype=torch.bfloat16, device=w.device)
     minus = torch.empty_like(plus) if dual else None
     bias = None
-    scratch = torch.empty(18 * rows * (cols // group), dtype=torch.float32, device=w.device)
+    scratch = torch.empty(18 * rows * (cols // (group or 128)), dtype=torch.float32, device=w.device)
     if smooth is not None:
         bias = torch.empty((2 if dual else 1, rows), dtype=torch.float32, device=w.device)
     codes = torch.empty((rows, cols), dtype=torch.uint8, device=w.device) if want_codes else None
@@ -388,8 +389,8 @@ class ZoqatModel:
                     if l >= first_trainable_layer and (trainable_names is None or name in trainable_names):
                         flags, th = TENSOR_TRAINABLE | TENSOR_QUANTIZED, None
                         if adaptive_quant:
-                            th = P.setdefault("theta_" + name, torch.empty((t.shape[0], t.shape[1] // shape["w_group"], 4),
-                                                                           dtype=torch.float32, device="cuda"))
+                            ng = t.shape[1] // shape["w_group"] if shape["w_group"] else 1
+                            th = P.setdefault("theta_" + name, torch.empty((t.shape[0], ng, 4), dtype=torch.float32, device="cuda"))
                             flags |= TENSOR_ADAPTIVE
                         descs.append(TensorDesc(_LINEAR_ROLES[name], l, flags, 0, t.data_ptr(), None,
                                                 th.data_ptr() if th is not None else None))

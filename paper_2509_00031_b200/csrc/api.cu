@@ -55,6 +55,7 @@ struct Linear {
     bool present = false;
     bool adaptive() const { return theta != nullptr; }
     uint32_t tid_q() const { return tid + 0x10000u; }
+    int64_t n_qgroups(int w_group) const { return w_group ? rows * cols / w_group : rows; }
     bool trainable() const { return (flags & ZOQAT_TENSOR_TRAINABLE) && !(flags & ZOQAT_TENSOR_FROZEN_PACKED); }
     bool packed_frozen() const { return flags & ZOQAT_TENSOR_FROZEN_PACKED; }
     int bits(int w_bits) const { return (flags & (ZOQAT_TENSOR_QUANTIZED | ZOQAT_TENSOR_FROZEN_PACKED)) ? w_bits : 0; }
@@ -128,11 +129,12 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.smooth_ld = (int)(d > F ? d : F);
     w.smooth_buf = (float*)take((size_t)4 * 6 * w.smooth_ld * 4);
     const size_t lin_max = (3 * d * d > ffn_cols * d) ? 3 * d * d : ffn_cols * d;
-    w.bias_part = (float*)take(2 * (lin_max / c.w_group) * 4);
+    const size_t span = c.w_group ? (size_t)c.w_group : 128;       // per-channel weights: partial sums per 128 columns
+    w.bias_part = (float*)take(2 * (lin_max / span) * 4);
     {   // per linear: 2 passes x (A, B) x groups float4; q, k, v, o, gate, up, down back to back
         const size_t lin_elems[7] = {d * d, d * d, d * d, d * d, F * d, (c.arch == ZOQAT_ARCH_LLAMA) ? F * d : 0, d * F};
         size_t o = 0;
-        for (int r = 0; r < 7; ++r) { w.qprep_off[r] = o; o += align_up(4 * (lin_elems[r] / c.w_group) * 16); }
+        for (int r = 0; r < 7; ++r) { w.qprep_off[r] = o; o += align_up(4 * (lin_elems[r] / span) * 16); }
         w.qprep_off[7] = o;
         w.qprep = take(o);
     }
@@ -151,9 +153,10 @@ int validate_config(const zoqat_config_t* c) {
     if (c->d_model % c->n_heads) return fail(ZOQAT_ERR_INVALID_ARG, "n_heads must divide d_model");
     const int dh = c->d_model / c->n_heads;
     if (dh != 64 && dh != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "head size %d (supported: 64, 128)", dh);
-    if (c->w_bits != 2 && c->w_bits != 3 && c->w_bits != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "w_bits %d (supported: 2, 3, 4)", c->w_bits);
-    if (c->w_group != 32 && c->w_group != 64 && c->w_group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "w_group %d (supported: 32, 64, 128)", c->w_group);
-    if (c->d_model % c->w_group || c->d_ffn % c->w_group) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
+    if (c->w_bits < 2 || c->w_bits > 8) return fail(ZOQAT_ERR_UNSUPPORTED, "w_bits %d (supported: 2..8; packed tensors 2..4)", c->w_bits);
+    if (c->w_group != 0 && c->w_group != 32 && c->w_group != 64 && c->w_group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "w_group %d (supported: 32, 64, 128, 0 = per output row)", c->w_group);
+    if (c->w_group == 0 && (c->d_model % 128 || c->d_ffn % 128)) return fail(ZOQAT_ERR_UNSUPPORTED, "per-row weight groups need d_model and d_ffn to be multiples of 128");
+    if (c->w_group != 0 && (c->d_model % c->w_group || c->d_ffn % c->w_group)) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
     if (c->a_bits != 0 && c->a_bits != 4 && c->a_bits != 6 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 4, 6, 8)", c->a_bits);
     if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT && c->gemm_impl != ZOQAT_GEMM_TCGEN05_1CTA) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
     if ((int64_t)c->max_batch * c->max_seq > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "max_batch*max_seq too large");
@@ -241,14 +244,17 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
     ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
     const int64_t n = L.rows * L.cols;
     const int bits = L.bits(m->cfg.w_bits);
-    if (smoothing || (L.adaptive() && bits != 0)) {
+    const bool per_channel = m->cfg.w_group == 0 && bits != 0;
+    if (smoothing || per_channel || (L.adaptive() && bits != 0)) {
         LearnedOperandArgs a{};
-        a.w = L.w; a.rows = L.rows; a.cols = L.cols; a.group = m->cfg.w_group; a.bits = bits;
+        a.w = L.w; a.rows = L.rows; a.cols = L.cols; a.group = m->cfg.w_group ? m->cfg.w_group : 128; a.bits = bits;
+        a.per_channel = per_channel;
         a.perturb = L.trainable() && eps != 0.0f;
         a.seed = seed; a.tid = L.tid; a.tid_q = L.tid_q(); a.eps = eps;
         a.op_plus = dst; a.op_minus = passes == 2 ? dst + pass_stride : nullptr;
         a.theta = L.adaptive() ? L.theta : nullptr;
-        a.prep = m->ws.qprep + m->ws.qprep_off[role]; a.prepared = 1;      // forward() prepared the whole layer
+        a.prep = m->ws.qprep + m->ws.qprep_off[role];
+        a.prepared = L.adaptive() ? 1 : 0;     // forward() prepared the layer's learnable parameters; row min/max is found here
         if (smoothing) {
             a.smooth = m->ws.smooth_buf + (size_t)point * 6 * m->ws.smooth_ld; a.smooth_ld = m->ws.smooth_ld;
             a.bias_part = m->ws.bias_part; a.bias0 = bias0;
@@ -323,7 +329,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                 if (!(L.present && L.adaptive() && L.bits(c.w_bits) != 0)) continue;
                 const int k = pb.count++;
                 pb.theta[k] = L.theta; pb.prep[k] = w.qprep + w.qprep_off[r]; pb.tid_q[k] = L.tid_q();
-                pb.prefix[k + 1] = pb.prefix[k] + L.rows * L.cols / c.w_group;
+                pb.prefix[k + 1] = pb.prefix[k] + L.n_qgroups(c.w_group);
             }
             if (pb.count) {
                 ProfScope ps_(m, ZOQAT_PROF_WEIGHT, s);
@@ -438,7 +444,7 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
             Linear& L = Ly.lin[r];
             if (!(L.present && L.trainable())) continue;
             launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
-            if (L.adaptive()) add(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, L.tid_q(), 0);
+            if (L.adaptive()) add(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, L.tid_q(), 0);
         }
         if (Ly.smoothing)
             for (int pt = 0; pt < 4; ++pt) {
@@ -540,6 +546,7 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
                 if (is_packed) {
                     if (!t.packed || !t.qparams) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: packed/qparams are NULL", i); }
                     if ((L.rows * L.cols) % 128) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need rows*cols %% 128 == 0", i); }
+                    if (cfg->w_bits > 4 || cfg->w_group == 0) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need w_bits <= 4 and a column group of 32, 64 or 128", i); }
                     L.packed = static_cast<const uint32_t*>(t.packed);
                     L.qparams = static_cast<const float2*>(t.qparams);
                     m->any_packed = true;
@@ -657,7 +664,9 @@ int zoqat_init_qparams(zoqat_model_t* m, void* stream) {
     for (auto& Ly : m->layers)
         for (int r = 0; r < 7; ++r) {
             Linear& L = Ly.lin[r];
-            if (L.present && L.adaptive()) launch_init_qparams(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, L.theta, s);
+            if (!(L.present && L.adaptive())) continue;
+            if (m->cfg.w_group) launch_init_qparams(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, L.theta, s);
+            else launch_init_qparams_rows(L.w, L.rows, L.cols, m->cfg.w_bits, L.theta, s);
         }
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
@@ -760,7 +769,7 @@ int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
                 if (L.present && L.trainable()) {
                     launch_update_multi(L.w_mut, (uint64_t)(L.rows * L.cols), seed, n_dirs, L.tid, &res->update_scale, stride, s);
                     if (L.adaptive())
-                        launch_update_multi(L.theta, (uint64_t)(L.rows * L.cols / m->cfg.w_group) * 4, seed, n_dirs, L.tid_q(), &res->update_scale, stride, s);
+                        launch_update_multi(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, seed, n_dirs, L.tid_q(), &res->update_scale, stride, s);
                 }
             }
         for (size_t l = 0; l < m->layers.size(); ++l) {
@@ -862,11 +871,16 @@ int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* byte
 }
 
 // ---- single operations ---------------------------------------------------------
-static int check_group_bits(int64_t rows, int64_t cols, int group, int bits, bool allow_zero_bits) {
+static int check_group_bits(int64_t rows, int64_t cols, int group, int bits, bool allow_zero_bits, int max_bits = 8,
+                            bool allow_rows = false) {
     if (rows <= 0 || cols <= 0) return fail(ZOQAT_ERR_INVALID_ARG, "rows/cols must be positive");
-    if (group != 32 && group != 64 && group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "group %d (supported: 32, 64, 128)", group);
-    if (cols % group) return fail(ZOQAT_ERR_INVALID_ARG, "group must divide cols");
-    if (!((bits >= 2 && bits <= 4) || (allow_zero_bits && bits == 0))) return fail(ZOQAT_ERR_UNSUPPORTED, "bits %d", bits);
+    if (group == 0 && allow_rows) {
+        if (cols % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "one group per row needs cols %% 128 == 0");
+    } else {
+        if (group != 32 && group != 64 && group != 128) return fail(ZOQAT_ERR_UNSUPPORTED, "group %d (supported: 32, 64, 128)", group);
+        if (cols % group) return fail(ZOQAT_ERR_INVALID_ARG, "group must divide cols");
+    }
+    if (!((bits >= 2 && bits <= max_bits) || (allow_zero_bits && bits == 0))) return fail(ZOQAT_ERR_UNSUPPORTED, "bits %d", bits);
     return ZOQAT_OK;
 }
 
@@ -911,20 +925,21 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
                                     const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
                                     void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
     if (!scratch_dev || (reinterpret_cast<uintptr_t>(scratch_dev) & 15)) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 16-byte aligned device memory");
-    if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, true, 8, true)) return rc;
     if (!w_dev || !operand_plus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_plus_dev are NULL");
-    if (!theta_dev && !smooth_dev) return fail(ZOQAT_ERR_INVALID_ARG, "neither theta_dev nor smooth_dev given: use zoqat_op_weight_quant");
+    if (!theta_dev && !smooth_dev && group != 0) return fail(ZOQAT_ERR_INVALID_ARG, "neither theta_dev nor smooth_dev given: use zoqat_op_weight_quant");
     if (smooth_dev && !bias_dev) return fail(ZOQAT_ERR_INVALID_ARG, "smoothing needs bias_dev");
     if ((reinterpret_cast<uintptr_t>(theta_dev) | reinterpret_cast<uintptr_t>(smooth_dev) | reinterpret_cast<uintptr_t>(w_dev)) & 15)
         return fail(ZOQAT_ERR_INVALID_ARG, "w_dev, theta_dev and smooth_dev must be 16-byte aligned");
     LearnedOperandArgs a{};
-    a.w = w_dev; a.rows = rows; a.cols = cols; a.group = group; a.bits = bits; a.perturb = eps != 0.0f;
+    a.w = w_dev; a.rows = rows; a.cols = cols; a.group = group ? group : 128; a.bits = bits; a.perturb = eps != 0.0f;
+    a.per_channel = group == 0 && bits != 0;
     a.seed = seed; a.tid = tensor_id; a.tid_q = tensor_id + 0x10000u; a.eps = eps;
     a.op_plus = static_cast<__nv_bfloat16*>(operand_plus_dev); a.op_minus = static_cast<__nv_bfloat16*>(operand_minus_dev);
     a.theta = theta_dev; a.smooth = smooth_dev; a.smooth_ld = (int)cols;
     // scratch: 16 floats per group for the prepared parameters, then 2 per group for the bias partial sums
     a.prep = scratch_dev;
-    a.bias_part = scratch_dev + 16 * (rows * cols / group); a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
+    a.bias_part = scratch_dev + 16 * (rows * cols / a.group); a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
     a.codes = codes_dev;
     launch_weight_operand_learned(a, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
@@ -962,17 +977,18 @@ int zoqat_op_smooth_act_operand(const float* x_dev, int64_t rows, int64_t cols, 
 }
 
 int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, float* theta_dev, void* stream) {
-    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 8, true)) return rc;
     if (!w_dev || !theta_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if ((reinterpret_cast<uintptr_t>(w_dev) | reinterpret_cast<uintptr_t>(theta_dev)) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-    launch_init_qparams(w_dev, rows * cols, group, bits, theta_dev, static_cast<cudaStream_t>(stream));
+    if (group) launch_init_qparams(w_dev, rows * cols, group, bits, theta_dev, static_cast<cudaStream_t>(stream));
+    else launch_init_qparams_rows(w_dev, rows, cols, bits, theta_dev, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
 
 int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, void* packed_dev,
                          void* qparams_dev, void* stream) {
-    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 4)) return rc;
     if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
     if (!w_dev || !packed_dev || !qparams_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     launch_pack_frozen(w_dev, rows * cols, group, bits, static_cast<uint32_t*>(packed_dev), static_cast<float2*>(qparams_dev),
@@ -983,7 +999,7 @@ int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int gro
 
 int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group,
                             int bits, void* operand_dev, void* stream) {
-    if (int rc = check_group_bits(rows, cols, group, bits, false)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 4)) return rc;
     if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
     if (!packed_dev || !qparams_dev || !operand_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     launch_unpack_operand(static_cast<const uint32_t*>(packed_dev), static_cast<const float2*>(qparams_dev), rows * cols,

@@ -53,6 +53,7 @@ void launch_smooth_perturb(const SmoothBatch& b, uint64_t seed, float eps, int p
 void launch_update_batch(const UpdateBatch& b, uint64_t seed, const float* class_ptr, float scale_q, float scale_s, cudaStream_t s);
 struct LearnedOperandArgs {
     const float* w; int64_t rows, cols; int group, bits, perturb;
+    int per_channel;          // 1: one quantisation group per row (cols % 128 == 0); `group` is then ignored
     uint64_t seed; uint32_t tid, tid_q; float eps;
     __nv_bfloat16 *op_plus, *op_minus;
     const float* theta; void* prep; int prepared;   // prepared = 1: prep already holds this tensor's parameters
@@ -62,6 +63,7 @@ struct LearnedOperandArgs {
 };
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s);
 void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s);
+void launch_init_qparams_rows(const float* w, int64_t rows, int64_t cols, int bits, float* theta, cudaStream_t s);   // one group per row
 void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s);
 void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);
 void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,

@@ -318,6 +318,72 @@ adapt_prepare_kernel(PrepareBatch b, int bits, int perturb, uint32_t k0, uint32_
     }
 }
 
+// One quantisation group per output row ("per-channel" weights): a first pass over the row finds min and max of the
+// perturbed (and, with smoothing, scaled) weights of both signs and writes the same prepared parameters as
+// adapt_prepare_kernel, A = (step, 1/step, -z, Q_P - z), B = (z, 0, Q_P, 0), so the producer runs its folded form.
+// theta_out != NULL instead writes the initial learnable parameters (step, z, 0, 1) of the unperturbed row.
+// One CTA per row; cols4 = cols / 4.
+__global__ void __launch_bounds__(kThreads)
+row_prepare_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, int perturb, uint32_t k0, uint32_t k1,
+                   uint32_t tid, float eps, int signs, const float* __restrict__ smooth, int smooth_ld,
+                   float4* __restrict__ out_a, float4* __restrict__ out_b, float4* __restrict__ theta_out) {
+    __shared__ float2 tab[kIcdfKnots];
+    __shared__ float red[4][kThreads / 32];
+    if (perturb) stage_icdf_table(tab);
+    const float qp = (float)((1 << bits) - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        float mnp = INFINITY, mxp = -INFINITY, mnm = INFINITY, mxm = -INFINITY;
+        for (int c = threadIdx.x; c < cols4; c += kThreads) {
+            const int64_t chunk = (int64_t)r * cols4 + c;
+            const float4 v = __ldg(w + chunk);
+            float xp[4] = {v.x, v.y, v.z, v.w}, xm[4] = {v.x, v.y, v.z, v.w};
+            if (perturb) {
+                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk);
+                const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { xm[j] = __fmaf_rn(-eps, zz[j], xp[j]); xp[j] = __fmaf_rn(eps, zz[j], xp[j]); }
+            }
+            if (smooth) {
+                const float4 sp = __ldg(reinterpret_cast<const float4*>(smooth) + c);
+                const float4 sm = signs == 2 ? __ldg(reinterpret_cast<const float4*>(smooth + 3 * (size_t)smooth_ld) + c) : sp;
+                const float a[4] = {sp.x, sp.y, sp.z, sp.w}, b[4] = {sm.x, sm.y, sm.z, sm.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { xp[j] = __fmul_rn(xp[j], a[j]); xm[j] = __fmul_rn(xm[j], b[j]); }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                mnp = fminf(mnp, xp[j]); mxp = fmaxf(mxp, xp[j]);
+                mnm = fminf(mnm, xm[j]); mxm = fmaxf(mxm, xm[j]);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mnp = fminf(mnp, __shfl_xor_sync(0xffffffffu, mnp, o)); mxp = fmaxf(mxp, __shfl_xor_sync(0xffffffffu, mxp, o));
+            mnm = fminf(mnm, __shfl_xor_sync(0xffffffffu, mnm, o)); mxm = fmaxf(mxm, __shfl_xor_sync(0xffffffffu, mxm, o));
+        }
+        __syncthreads();
+        if (lane == 0) { red[0][warp] = mnp; red[1][warp] = mxp; red[2][warp] = mnm; red[3][warp] = mxm; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int i = 1; i < kThreads / 32; ++i) {
+                red[0][0] = fminf(red[0][0], red[0][i]); red[1][0] = fmaxf(red[1][0], red[1][i]);
+                red[2][0] = fminf(red[2][0], red[2][i]); red[3][0] = fmaxf(red[3][0], red[3][i]);
+            }
+            for (int sg = 0; sg < signs; ++sg) {
+                const GroupQ g = group_params(red[2 * sg][0], red[2 * sg + 1][0], qp);
+                const float z = __fadd_rn(g.zp, 0.0f);          // -0 -> +0
+                if (theta_out) {
+                    theta_out[r] = make_float4(g.step, z, 0.0f, 1.0f);
+                } else {
+                    out_a[(int64_t)r * signs + sg] = make_float4(g.step, g.inv, -z, __fadd_rn(qp, -z));
+                    out_b[(int64_t)r * signs + sg] = make_float4(z, 0.0f, qp, 0.0f);
+                }
+            }
+        }
+    }
+}
+
 // The operand producer with the learnable parts of Section 4.2 (same thread mapping as weight_operand_kernel):
 //   SMOOTH  the quantiser sees s' (.) w' (s' = perturbed per-input-channel scale); the per-group partial sums of
 //           delta' . w' (the shift term of the smoothed bias, with the unscaled perturbed weight) go to bias_part,
@@ -332,7 +398,10 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                               uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
                               const float4* __restrict__ prep_a, const float4* __restrict__ prep_b,
                               const float* __restrict__ smooth, int smooth_ld,
-                              float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes) {
+                              float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes,
+                              int qgroup_items) {
+    // qgroup_items: 16-element items per quantisation group when that is not the GROUP-element span (one group per
+    // row: cols / 16); 0 = the span itself.  The bias partial sums stay per span either way.
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
     if (perturb) stage_icdf_table(tab);
@@ -417,7 +486,8 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
             float* cdp = (sg == 0 && codes) ? cd : nullptr;
             if (ADAPT) {
                 constexpr int SG = DUAL ? 2 : 1;
-                const int64_t slot = (i / LANES) * SG + sg;
+                const int64_t qg = qgroup_items ? (int64_t)((uint32_t)i / (uint32_t)qgroup_items) : i / LANES;
+                const int64_t slot = qg * SG + sg;
                 const float4 a = live ? __ldg(prep_a + slot) : make_float4(1.f, 1.f, 0.f, 0.f);
                 const bool literal = (a.z != a.z) || cdp != nullptr;
                 if (__any_sync(0xffffffffu, literal)) {       // zero point beyond exact integer arithmetic, or codes wanted
@@ -724,24 +794,33 @@ static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
     const float4* w4 = reinterpret_cast<const float4*>(a.w);
     uint2* p = reinterpret_cast<uint2*>(a.op_plus);
     uint2* m = reinterpret_cast<uint2*>(a.op_minus);
-    const int64_t n_groups = a.rows * a.cols / GROUP;
+    const int64_t n_groups = a.rows * a.cols / GROUP;                      // spans of the bias partial sums
+    const int64_t n_q = a.per_channel ? a.rows : n_groups;                 // quantisation groups
     const int signs = a.op_minus ? 2 : 1;
     float4* pa = reinterpret_cast<float4*>(a.prep);
-    float4* pb = pa + n_groups * signs;
+    float4* pb = pa + n_q * signs;
     uchar4* c4 = reinterpret_cast<uchar4*>(a.codes);
     if (ADAPT && !a.prepared) {
-        PrepareBatch pb1{};
-        pb1.count = 1; pb1.theta[0] = a.theta; pb1.prep[0] = a.prep; pb1.tid_q[0] = a.tid_q; pb1.prefix[0] = 0; pb1.prefix[1] = n_groups;
-        launch_adapt_prepare(pb1, a.bits, a.perturb, a.seed, a.eps, signs, s);
+        if (a.theta) {
+            PrepareBatch pb1{};
+            pb1.count = 1; pb1.theta[0] = a.theta; pb1.prep[0] = a.prep; pb1.tid_q[0] = a.tid_q; pb1.prefix[0] = 0; pb1.prefix[1] = n_q;
+            launch_adapt_prepare(pb1, a.bits, a.perturb, a.seed, a.eps, signs, s);
+        } else {       // one min/max group per row
+            const int rgrid = (int)(a.rows < 148 * 8 ? a.rows : 148 * 8);
+            row_prepare_kernel<<<rgrid, kThreads, 0, s>>>(w4, (int)a.rows, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps,
+                                                          signs, a.smooth, a.smooth_ld, pa, pb, nullptr);
+            count_launch();
+        }
     }
+    const int qgi = a.per_channel ? (int)(a.cols / 16) : 0;
     if (a.op_minus)
         weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
             w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
-            a.bias_part, n_groups, c4);
+            a.bias_part, n_groups, c4, qgi);
     else
         weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
             w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
-            a.bias_part, n_groups, c4);
+            a.bias_part, n_groups, c4, qgi);
     count_launch();
     if (SMOOTH) {
         const int64_t work = a.rows * signs * 32;
@@ -753,7 +832,8 @@ static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
 
 template <int GROUP>
 static void learned_dispatch_group(const LearnedOperandArgs& a, cudaStream_t s) {
-    const bool adapt = a.theta != nullptr && a.bits != 0, smooth = a.smooth != nullptr;
+    // prepared group parameters: learnable ones, or the row-wide min/max of per-channel weights
+    const bool adapt = (a.theta != nullptr || a.per_channel) && a.bits != 0, smooth = a.smooth != nullptr;
     if (adapt && smooth) learned_dispatch<GROUP, true, true>(a, s);
     else if (adapt) learned_dispatch<GROUP, true, false>(a, s);
     else learned_dispatch<GROUP, false, true>(a, s);
@@ -761,6 +841,7 @@ static void learned_dispatch_group(const LearnedOperandArgs& a, cudaStream_t s) 
 
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s) {
     if (a.rows * a.cols == 0 || (a.perturb && !ensure_icdf_table())) return;
+    if (a.per_channel) { learned_dispatch_group<128>(a, s); return; }      // cols % 128 == 0 (checked by the callers)
     if (a.group == 32) learned_dispatch_group<32>(a, s);
     else if (a.group == 64) learned_dispatch_group<64>(a, s);
     else learned_dispatch_group<128>(a, s);
@@ -785,6 +866,14 @@ void launch_update_batch(const UpdateBatch& b, uint64_t seed, const float* class
     if (b.count == 0 || b.prefix[b.count] == 0 || !ensure_icdf_table()) return;
     update_batch_kernel<<<stream_grid(b.prefix[b.count], kThreads), kThreads, 0, s>>>(b, (uint32_t)seed, (uint32_t)(seed >> 32),
                                                                                       class_ptr, scale_q, scale_s);
+    count_launch();
+}
+
+void launch_init_qparams_rows(const float* w, int64_t rows, int64_t cols, int bits, float* theta, cudaStream_t s) {
+    if (rows * cols == 0) return;
+    const int rgrid = (int)(rows < 148 * 8 ? rows : 148 * 8);
+    row_prepare_kernel<<<rgrid, kThreads, 0, s>>>(reinterpret_cast<const float4*>(w), (int)rows, (int)(cols / 4), bits, 0, 0u, 0u, 0u, 0.0f,
+                                                  1, nullptr, 0, nullptr, nullptr, reinterpret_cast<float4*>(theta));
     count_launch();
 }
 

@@ -34,6 +34,12 @@ WORKLOADS = {
     "llama7b_w4a4_learned": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
                                  w_bits=4, w_group=128, a_bits=4, batch=4, seq=1024, bf16_init=True,
                                  adaptive_quant=True, smoothing=True),
+    # the paper's weight-activation setting: one weight group per output row ("per-channel"), per-token activations
+    "llama7b_w4a4_perchannel": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                    w_bits=4, w_group=0, a_bits=4, batch=4, seq=1024, bf16_init=True,
+                                    adaptive_quant=True, smoothing=True),
+    "llama7b_w6a6_perchannel": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                    w_bits=6, w_group=0, a_bits=6, batch=4, seq=1024, bf16_init=True),
 }
 
 

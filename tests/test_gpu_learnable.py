@@ -161,10 +161,46 @@ def test_smooth_act_operand(zq, kind, cols, a_bits):
             assert np.all(step[rows_sg] == 1.0)
 
 
+@pytest.mark.parametrize("bits,adaptive,smoothing", [(4, False, False), (6, False, True), (4, True, True), (8, True, False)],
+                         ids=["w4_minmax", "w6_smooth", "w4_both", "w8_adaptive"])
+def test_per_row_groups_match_oracle(zq, bits, adaptive, smoothing):
+    """One quantisation group per output row ("per-channel" weights of the appendix on quantisation settings)."""
+    rng = np.random.default_rng(bits)
+    rows, cols = 301, 5 * 128
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    w[7] += 0.1
+    seed, tid, eps = 99, 36, np.float32(1e-3)
+    theta = random_theta(w, cols, bits, rng) if adaptive else None
+    assert zq.zoqat_op_init_qparams(dev(w), 0, bits).cpu().numpy().tobytes() == init_quant_params(w, cols, bits).tobytes()
+    smooth = None
+    if smoothing:
+        s = rng.uniform(0.5, 2.0, cols).astype(np.float32)
+        d = (0.3 * rng.standard_normal(cols)).astype(np.float32)
+        smooth = zq.zoqat_op_smooth_perturb(dev(s), dev(d), seed, 0x20021, 0x30021, float(eps))
+    plus, minus, bias, codes = zq.zoqat_op_weight_operand_learned(dev(w), 0, bits, seed, tid, float(eps), theta=dev(theta) if adaptive else None,
+                                                                  smooth=smooth, want_codes=True)
+    for sg, (e, op) in enumerate(((eps, plus), (-eps, minus))):
+        wp = core.perturb(w, seed, tid, e)
+        x = wp
+        if smoothing:
+            x = (wp * core.perturb(s, seed, 0x20021, e)[None, :]).astype(np.float32)
+            want_bias = wp.astype(np.float64) @ core.perturb(d, seed, 0x30021, e).astype(np.float64)
+            assert np.allclose(bias[sg].cpu().numpy(), want_bias, rtol=0, atol=2e-6 * np.abs(want_bias).max() + 1e-7)
+        if adaptive:
+            q, deq = adaptive_weight_quant(x, core.perturb(theta, seed, tid + QPARAM_ID, e), cols, bits)
+        else:
+            q, _, _, deq = core.weight_quant(x, cols, bits)
+        assert np.array_equal(bf16_to_f32(op), core.round_bf16(deq)), sg
+        if sg == 0:
+            assert np.array_equal(codes.cpu().numpy(), np.asarray(q).astype(np.uint8))
+
+
 # ---- the model ---------------------------------------------------------------------------------------------------
 SMALL_LLAMA = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=600, w_bits=4, w_group=64, a_bits=8)
 SMALL_LLAMA_UNFUSED = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=320, vocab=600, w_bits=4, w_group=64, a_bits=8)
 SMALL_OPT = dict(arch="opt", n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=777, w_bits=3, w_group=128, a_bits=0)
+PER_ROW_W6A6 = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=500, w_bits=6, w_group=0, a_bits=6)
+PER_ROW_W4A4 = dict(arch="opt", n_layers=1, d_model=128, n_heads=2, d_ffn=256, vocab=300, w_bits=4, w_group=0, a_bits=4)
 
 
 def oracle_cfg(shape, **kw):
@@ -179,7 +215,7 @@ def randomise_learnables(oracle, rng):
         P = oracle.p["layers"][l]
         for n in oracle.linear_names():
             if "theta_" + n in P:
-                P["theta_" + n][:] = random_theta(P[n], cfg.w_group, cfg.w_bits, rng)
+                P["theta_" + n][:] = random_theta(P[n], oracle.group_of(P[n]), cfg.w_bits, rng)
         for pt in POINTS:
             if "smooth_s_" + pt in P:
                 k = P["smooth_s_" + pt].size
@@ -210,8 +246,10 @@ def learnable_keys(oracle):
 
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("shape,adaptive,smoothing", [(SMALL_LLAMA, True, True), (SMALL_LLAMA_UNFUSED, False, True),
-                                                       (SMALL_OPT, True, True), (SMALL_LLAMA, True, False)],
-                         ids=["llama_both", "llama_unfused_smooth", "opt_both", "llama_adaptive"])
+                                                       (SMALL_OPT, True, True), (SMALL_LLAMA, True, False),
+                                                       (PER_ROW_W6A6, False, False), (PER_ROW_W6A6, True, True), (PER_ROW_W4A4, True, True)],
+                         ids=["llama_both", "llama_unfused_smooth", "opt_both", "llama_adaptive", "per_row_w6a6_minmax",
+                              "per_row_w6a6_both", "per_row_w4a4_opt_both"])
 def test_forward_loss_matches_oracle(zq, impl, shape, adaptive, smoothing):
     batch, seq = 2, 80
     model, oracle = build_pair(zq, shape, batch, seq, impl, adaptive, smoothing)
@@ -241,7 +279,7 @@ def test_initial_learnables_leave_the_model_unchanged(zq, shape):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("shape,first", [(SMALL_LLAMA, 0), (SMALL_OPT, 1)], ids=["llama", "opt_last_layer"])
+@pytest.mark.parametrize("shape,first", [(SMALL_LLAMA, 0), (SMALL_OPT, 1), (PER_ROW_W6A6, 0)], ids=["llama", "opt_last_layer", "per_row_w6a6"])
 def test_step_rates_match_oracle(zq, impl, shape, first):
     batch, seq, eps, lr, lrq, lrs = 2, 80, 1e-3, 1e-4, 3e-5, 5e-4
     model, oracle = build_pair(zq, shape, batch, seq, impl, True, True, first=first)

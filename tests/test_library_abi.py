@@ -41,7 +41,7 @@ def test_query_workspace_and_validation(zq):
                     max_seq=1024, w_bits=4, w_group=128, a_bits=8, gemm_impl=0, norm_eps=1e-5, rope_base=10000.0)
     assert L.zoqat_query_workspace(ctypes.byref(big), ctypes.byref(n)) == zq.OK
     assert n.value < 4 << 30          # scratch for the 7B shape stays far below the 26 GB of masters
-    for field, bad, code in [("w_bits", 5, zq.ERR_UNSUPPORTED), ("w_group", 48, zq.ERR_UNSUPPORTED),
+    for field, bad, code in [("w_bits", 9, zq.ERR_UNSUPPORTED), ("w_group", 48, zq.ERR_UNSUPPORTED),
                              ("a_bits", 5, zq.ERR_UNSUPPORTED), ("arch", 7, zq.ERR_INVALID_ARG),
                              ("n_heads", 3, zq.ERR_INVALID_ARG), ("d_model", 200, zq.ERR_UNSUPPORTED)]:
         c2 = zq.Config.from_buffer_copy(cfg)
