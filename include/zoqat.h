@@ -263,7 +263,9 @@ int zoqat_profile_read(zoqat_model_t* m, int category, double* ms, int64_t* inte
 /* Device pointer and size of a workspace buffer holding intermediates of the
  * most recent forward (last layer executed).  Parity hook. */
 #define ZOQAT_BUF_RESIDUAL   0   /* fp32 [passes*T, d_model]   residual stream after the last layer */
-#define ZOQAT_BUF_QKV        1   /* fp32 [passes*T, 3*d_model] q | k | v of the last layer (before RoPE) */
+#define ZOQAT_BUF_QKV        1   /* fp32 [passes*T, 3*d_model] q | k | v of the last layer (before RoPE); only written when
+                                    the projection's epilogue does not feed the attention kernel directly (CUDA-core or
+                                    single-CTA GEMM, d_model % 256 != 0 or seq % 32 != 0) */
 #define ZOQAT_BUF_ATTN       2   /* fp32 [passes*T, d_model]   attention output of the last layer   */
 #define ZOQAT_BUF_FFN        3   /* fp32: fc1 output [passes*T, d_ffn] (OPT); LLaMA: silu(gate)*up [passes*T, d_ffn] when
                                     d_ffn is a multiple of 128 with the default GEMM, else gate|up [passes*T, 2*d_ffn] */
@@ -399,6 +401,17 @@ int zoqat_op_attention_scratch_bytes(int batch, int seq, int n_heads, int d_head
 int zoqat_op_attention(const float* qkv_dev, int batch, int seq, int n_heads, int d_head,
                        const float* cos_dev, const float* sin_dev, float* out_dev,
                        int impl, void* scratch_dev, int32_t* err_flag_dev, void* stream);
+
+/* The q | k | v projection and the attention behind it as the step runs them on the default GEMM: the projection's
+ * epilogue applies the rotary embedding, scales q, splits every value into the two binary16 halves and writes the
+ * attention kernel's operand layouts itself, so q | k | v never exist as fp32 in memory and no preparation pass
+ * runs.  a_dev bf16 [batch*seq, K]; b_dev bf16 [3*d_model, K] (q rows, k rows, v rows; d_model = n_heads*d_head);
+ * row_step_dev / bias_dev ([3*d_model]) may be NULL; out_dev fp32 [batch*seq, d_model]; scratch_dev as for
+ * zoqat_op_attention.  Needs d_model % 256 == 0, seq % 32 == 0, K % 8 == 0.  Same result as zoqat_op_gemm followed
+ * by zoqat_op_attention up to the binary32 rounding of the rotation. */
+int zoqat_op_qkv_attention(const void* a_dev, const void* b_dev, int batch, int seq, int n_heads, int d_head, int64_t K,
+                           const float* row_step_dev, const float* bias_dev, const float* cos_dev, const float* sin_dev,
+                           float* out_dev, void* scratch_dev, int32_t* err_flag_dev, void* stream);
 
 /* Vocabulary projection fused with the cross-entropy: logits = A B^T are never
  * stored.  a_dev bf16 [T, d], b_dev bf16 [V, d], labels_dev int32 [T] (< 0 =

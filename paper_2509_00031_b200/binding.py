@@ -33,7 +33,7 @@ EXPORTS = [
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
-    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
+    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_qkv_attention", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
 ]
@@ -116,6 +116,7 @@ def lib():
             "zoqat_op_gemm": [vp, vp, i64, i64, i64, vp, vp, i32, i32, vp, i32, vp, vp],
             "zoqat_op_gemm_silu_gate": [vp, vp, i64, i64, i64, vp, vp, vp, vp, vp],
             "zoqat_op_attention_scratch_bytes": [i32, i32, i32, i32, P(sz)],
+            "zoqat_op_qkv_attention": [vp, vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp],
             "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp],
             "zoqat_op_head_loss_scratch_bytes": [i64, i64, P(sz)],
             "zoqat_op_head_loss": [vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, vp, vp],
@@ -296,6 +297,19 @@ def zoqat_op_attention(qkv, batch, seq, n_heads, d_head, cos=None, sin=None, imp
             err = torch.zeros(1, dtype=torch.int32, device=qkv.device)
     _check(lib().zoqat_op_attention(_p(qkv), batch, seq, n_heads, d_head, _p(cos), _p(sin), _p(out), impl, _p(scratch),
                                     _p(err), _stream()))
+    return out, err
+
+
+def zoqat_op_qkv_attention(a, b_qkv, batch, seq, n_heads, d_head, row_step=None, bias=None, cos=None, sin=None):
+    """Fused q|k|v projection + attention; returns (out [batch*seq, d_model], err)."""
+    K = a.shape[1]
+    out = torch.empty((batch * seq, n_heads * d_head), dtype=torch.float32, device=a.device)
+    nb = ctypes.c_size_t()
+    _check(lib().zoqat_op_attention_scratch_bytes(batch, seq, n_heads, d_head, ctypes.byref(nb)))
+    scratch = torch.empty(nb.value, dtype=torch.uint8, device=a.device)
+    err = torch.zeros(1, dtype=torch.int32, device=a.device)
+    _check(lib().zoqat_op_qkv_attention(_p(a), _p(b_qkv), batch, seq, n_heads, d_head, K, _p(row_step), _p(bias), _p(cos), _p(sin),
+                                        _p(out), _p(scratch), _p(err), _stream()))
     return out, err
 
 

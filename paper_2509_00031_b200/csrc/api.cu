@@ -348,11 +348,20 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         g.out = w.qkv; g.b_stride = ps;
+        // on the pair kernel the epilogue of this GEMM writes the attention operands itself (rotary embedding, q
+        // scaling, binary16 hi / lo split, v transposed): q | k | v never exist as fp32 and no preparation kernel runs
+        const bool fuse_qkv = c.gemm_impl == ZOQAT_GEMM_TCGEN05 && d % 256 == 0 && seq % 32 == 0;
+        if (fuse_qkv) {
+            g.mode = 2; g.out = nullptr;
+            g.att = attention_tc_operands(w.attn_scratch, Z * batch, seq, H, dh);
+            g.seq = seq; g.n_heads = H; g.d_head = dh;
+            g.cos_t = llama ? w.rope_cos : nullptr; g.sin_t = llama ? w.rope_sin : nullptr;
+        }
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s);
           if (c.gemm_impl == ZOQAT_GEMM_SIMT) {
               launch_attention(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, w.att, s);
-          } else if (int rc = launch_attention_tc(w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr,
+          } else if (int rc = launch_attention_tc(fuse_qkv ? nullptr : w.qkv, Z * batch, seq, H, dh, llama ? w.rope_cos : nullptr,
                                                   llama ? w.rope_sin : nullptr, w.att, w.attn_scratch, w.err_flag, s)) {
               return fail(rc, "attention launch rejected");
           } }
@@ -1068,6 +1077,30 @@ int zoqat_op_gemm_silu_gate(const void* a_dev, const void* b_dev, int64_t M, int
     g.b_stride = (size_t)2 * F * K; g.mode = 3; g.row_amax = row_amax_dev;
     const int rc = launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "gated GEMM rejected: M=%lld F=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers)", (long long)M, (long long)F, (long long)K);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_qkv_attention(const void* a_dev, const void* b_dev, int batch, int seq, int n_heads, int d_head, int64_t K,
+                           const float* row_step_dev, const float* bias_dev, const float* cos_dev, const float* sin_dev,
+                           float* out_dev, void* scratch_dev, int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !out_dev || !scratch_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (batch <= 0 || seq <= 0 || n_heads <= 0 || K <= 0 || (d_head != 64 && d_head != 128)) return fail(ZOQAT_ERR_UNSUPPORTED, "bad shape");
+    const int64_t dm = (int64_t)n_heads * d_head;
+    if (dm % 256 || seq % 32) return fail(ZOQAT_ERR_UNSUPPORTED, "the fused projection needs n_heads*d_head %% 256 == 0 and seq %% 32 == 0");
+    if ((cos_dev == nullptr) != (sin_dev == nullptr)) return fail(ZOQAT_ERR_INVALID_ARG, "cos/sin tables must both be given or both NULL");
+    if (reinterpret_cast<uintptr_t>(scratch_dev) & 255) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 256-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = (int64_t)batch * seq; g.N = 3 * dm; g.K = K; g.Z = 1; g.row_step = row_step_dev; g.bias = bias_dev;
+    g.err_flag = err_flag_dev; g.b_stride = (size_t)(3 * dm * K); g.mode = 2;
+    g.att = attention_tc_operands(scratch_dev, batch, seq, n_heads, d_head);
+    g.seq = seq; g.n_heads = n_heads; g.d_head = d_head; g.cos_t = cos_dev; g.sin_t = sin_dev;
+    int rc = launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "fused q|k|v GEMM rejected (K %% 8 == 0, 16-byte aligned pointers)");
+    rc = launch_attention_tc(nullptr, batch, seq, n_heads, d_head, cos_dev, sin_dev, out_dev, scratch_dev, err_flag_dev, s);
+    if (rc != ZOQAT_OK) return fail(rc, "attention launch rejected");
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -624,8 +624,11 @@ int attention_tc_launch(const float* qkv, int batch, int seq, int n_heads, const
     __half* vtl = reinterpret_cast<__half*>(sp + 4 * qk_bytes + vt_bytes);
 
     const float q_mul = (float)(1.4426950408889634 / sqrt((double)D));
-    dim3 pgrid((seq + 63) / 64, n_heads, batch);
-    attn_prep_kernel<D><<<pgrid, 256, 0, s>>>(qkv, seq, seq_pad, n_heads, cos_t, sin_t, q_mul, qh, ql, kh, kl, vth, vtl);
+    if (qkv != nullptr) {        // otherwise the operands are already in the scratch (written by the q|k|v GEMM epilogue)
+        dim3 pgrid((seq + 63) / 64, n_heads, batch);
+        attn_prep_kernel<D><<<pgrid, 256, 0, s>>>(qkv, seq, seq_pad, n_heads, cos_t, sin_t, q_mul, qh, ql, kh, kl, vth, vtl);
+        count_launch();
+    }
 
     alignas(64) CUtensorMap m_qh, m_ql, m_kh, m_kl, m_vth, m_vtl;
     if (!make_half_map(&m_qh, qh, D, seq, bhs, D, BQ) || !make_half_map(&m_ql, ql, D, seq, bhs, D, BQ) ||
@@ -649,7 +652,7 @@ int attention_tc_launch(const float* qkv, int batch, int seq, int n_heads, const
     if (sms <= 0) sms = 148;
     const int grid = p.total_items < sms ? p.total_items : sms;
     attention_tc_kernel<D><<<grid, kAttThreadsTC, Cfg::kSmemBytes, s>>>(m_qh, m_ql, m_kh, m_kl, m_vth, m_vtl, p);
-    count_launch(2);
+    count_launch();
     return ZOQAT_OK;
 }
 
@@ -658,6 +661,19 @@ int attention_tc_launch(const float* qkv, int batch, int seq, int n_heads, const
 size_t attention_tc_scratch_bytes(int batch, int seq, int n_heads, int d_head) {
     const size_t bhs = (size_t)batch * n_heads;
     return 4 * up256(bhs * seq * d_head * 2) + 2 * up256(bhs * d_head * pad8(seq) * 2);
+}
+
+AttnOperands attention_tc_operands(void* scratch, int batch, int seq, int n_heads, int d_head) {
+    const size_t bhs = (size_t)batch * n_heads;
+    const int seq_pad = pad8(seq);
+    const size_t qk_bytes = up256(bhs * seq * d_head * 2), vt_bytes = up256(bhs * d_head * seq_pad * 2);
+    uint8_t* sp = static_cast<uint8_t*>(scratch);
+    AttnOperands o;
+    o.qh = sp; o.ql = sp + qk_bytes; o.kh = sp + 2 * qk_bytes; o.kl = sp + 3 * qk_bytes;
+    o.vth = sp + 4 * qk_bytes; o.vtl = sp + 4 * qk_bytes + vt_bytes;
+    o.seq_pad = seq_pad;
+    o.q_mul = (float)(1.4426950408889634 / sqrt((double)d_head));
+    return o;
 }
 
 int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d_head, const float* cos_t,

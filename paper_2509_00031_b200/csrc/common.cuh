@@ -92,6 +92,11 @@ void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t*
 void launch_attention(const float* qkv, int batch, int seq, int n_heads, int d_head,
                       const float* cos_t, const float* sin_t, float* out, cudaStream_t s);
 size_t attention_tc_scratch_bytes(int batch, int seq, int n_heads, int d_head);
+// Operand arrays of the tensor-core attention inside its scratch: q and k as binary16 hi / lo halves
+// [batch*heads][seq][d_head] (q already times log2(e)/sqrt(d_head)), v transposed [batch*heads][d_head][seq_pad].
+// launch_attention_tc(qkv = NULL) runs on operands some other kernel (the q|k|v GEMM epilogue) has written there.
+struct AttnOperands { void *qh, *ql, *kh, *kl, *vth, *vtl; int seq_pad; float q_mul; };
+AttnOperands attention_tc_operands(void* scratch, int batch, int seq, int n_heads, int d_head);
 int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d_head, const float* cos_t,
                         const float* sin_t, float* out, void* scratch, int32_t* err_flag, cudaStream_t s);
 
@@ -112,6 +117,13 @@ struct GemmArgs {
     uint32_t* row_amax;       // mode 3: [Z*M] max |act| per row as the bits of a non-negative float (zeroed by the caller)
     int mode;                 // 0 store, 1 cross-entropy partials, 3 SiLU-gated pair (tcgen05 pair kernel only):
                               //   B = [gate rows; up rows], out[z*M+m, f] = silu(row_step*A.gate_f) * (row_step*A.up_f), ldo = N/2
+                              // 2 (tcgen05 pair kernel only): N = 3*d_model columns q | k | v; nothing is stored as fp32 -
+                              //   the epilogue applies the rotary embedding, scales q, splits into binary16 hi / lo and
+                              //   writes the attention operands `att` directly (M = batch*seq rows per pass, seq % 32 == 0,
+                              //   d_model % 256 == 0)
+    AttnOperands att;         // mode 2
+    int seq, n_heads, d_head; // mode 2
+    const float *cos_t, *sin_t;   // mode 2: rotary tables [seq, d_head/2] or NULL
     const int32_t* labels;    // [M]
     float2* partials;         // [Z*M, ce_tiles] (max, sum exp)
     float* label_logit;       // [Z*M]

@@ -20,6 +20,7 @@
 #include "common.cuh"
 #include "../../include/zoqat.h"
 #include "tc_ptx.cuh"
+#include <cuda_fp16.h>
 
 namespace zq {
 namespace {
@@ -68,12 +69,29 @@ struct TcParams {
     int tiles_m, tiles_n;
     int tma_out;              // 1: mode-0 results leave through map_out (needs N % 4 == 0)
     uint32_t* row_amax;       // mode 3: [Z*M] running max |act| per row (bit pattern of a non-negative float)
+    // mode 2: the q | k | v projection writes the attention operands
+    int seq, n_heads, d_head, d_model;
+    const float *cos_t, *sin_t;
+    float q_mul;
 };
+
+// Six tensor maps over the binary16 attention operands (mode 2): q / k hi and lo [batch*heads][seq][d_head], boxes of
+// 32 positions x 32 features; v^T hi and lo [batch*heads][d_head][seq_pad], boxes of 32 features x 32 positions.
+struct AttMaps { CUtensorMap qh, ql, kh, kl, vh, vl; };
+
+// x -> binary16 hi and lo with x ~ hi + lo * 2^-11 (the split the attention kernel's three-product scheme expects)
+__device__ __forceinline__ void split_half(float x, __half& hi, __half& lo) {
+    hi = __float2half_rn(x);
+    lo = __float2half_rn((x - __half2float(hi)) * 2048.0f);
+}
+__device__ __forceinline__ uint32_t pack_half2(__half a, __half b) {
+    return (uint32_t)__half_as_ushort(a) | ((uint32_t)__half_as_ushort(b) << 16);
+}
 
 template <int BN, int CG>
 __global__ void __launch_bounds__(kThreadsTC, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_out, TcParams p) {
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ AttMaps att, TcParams p) {
     using Cfg = TileCfg<BN, CG>;
     constexpr int S = Cfg::kStages;
     constexpr int TM = BM * CG;                                  // rows of a tile
@@ -105,6 +123,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
         if (p.tma_out || p.mode == 3) prefetch_tmap(&map_out);
+        if (p.mode == 2) { prefetch_tmap(&att.qh); prefetch_tmap(&att.ql); prefetch_tmap(&att.kh); prefetch_tmap(&att.kl); prefetch_tmap(&att.vh); prefetch_tmap(&att.vl); }
     }
     if (warp == 1) {            // TMEM: 2 accumulators of BN fp32 columns (in each CTA of a pair)
         if (CG == 2) { tmem_alloc_pair(tmem_slot, 2 * BN); tmem_relinquish_pair(); }
@@ -208,6 +227,122 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             float ce_m = -INFINITY, ce_s = 0.0f;
             const int32_t lab = (p.mode == 1 && row_ok) ? p.labels[m] : -1;
             const float* bias = p.bias ? p.bias + (int64_t)z * p.bias_stride : nullptr;
+            (void)lab;
+            if (p.mode == 2) {
+                // q | k | v projection: rotary embedding, q scaling, hi / lo split and the layouts of the attention kernel,
+                // written from here so that q | k | v never exist as fp32 in memory.  A warp's 32 rows are 32 consecutive
+                // positions of one sequence (seq % 32 == 0).
+                const int64_t m0 = (int64_t)tm * TM + rank * BM + quarter * 32;
+                if (m0 < p.M) {
+                    const int64_t r0 = (int64_t)z * p.M + m0;
+                    const int bseq = (int)(r0 / p.seq), pos0 = (int)(r0 % p.seq);
+                    const int dh = p.d_head, hd = dh >> 1;
+                    const int sel = (int)((int64_t)tn * BN / p.d_model);           // 0 q, 1 k, 2 v
+                    const int head0 = (int)(((int64_t)tn * BN - (int64_t)sel * p.d_model) / dh);
+                    const uint32_t stage = out_stage + (uint32_t)(quarter * 2 * Cfg::kOutBoxBytes);     // 8 KB of this warp
+                    if (sel < 2) {
+                        const CUtensorMap* mh = sel == 0 ? &att.qh : &att.kh;
+                        const CUtensorMap* ml = sel == 0 ? &att.ql : &att.kl;
+                        const float mul = sel == 0 ? p.q_mul : 1.0f;
+#pragma unroll 1
+                        for (int part = 0; part < hd / 32; ++part) {
+                            // cos / sin of this thread's position for the 32 rotation pairs of the part, kept for every head
+                            float cs[32], sn[32];
+                            if (p.cos_t) {
+                                const float4* c4 = reinterpret_cast<const float4*>(p.cos_t + (int64_t)(pos0 + lane) * hd + part * 32);
+                                const float4* s4 = reinterpret_cast<const float4*>(p.sin_t + (int64_t)(pos0 + lane) * hd + part * 32);
+#pragma unroll
+                                for (int q4 = 0; q4 < 8; ++q4) {
+                                    const float4 c = __ldg(c4 + q4), sv = __ldg(s4 + q4);
+                                    cs[4 * q4] = c.x; cs[4 * q4 + 1] = c.y; cs[4 * q4 + 2] = c.z; cs[4 * q4 + 3] = c.w;
+                                    sn[4 * q4] = sv.x; sn[4 * q4 + 1] = sv.y; sn[4 * q4 + 2] = sv.z; sn[4 * q4 + 3] = sv.w;
+                                }
+                            }
+#pragma unroll 1
+                            for (int hh = 0; hh < BN / dh; ++hh) {
+                                uint32_t va[32], vb[32];
+                                __syncwarp();
+                                tmem_ld32(t_addr + (uint32_t)(hh * dh + part * 32), va);
+                                tmem_ld32(t_addr + (uint32_t)(hh * dh + hd + part * 32), vb);
+                                tmem_ld_wait();
+                                if (lane == 0) bulk_wait_read_0();          // the four boxes of the previous round have been read
+                                __syncwarp();
+                                const int64_t n_lo = n_base + hh * dh + part * 32;       // global column of va[0]
+#pragma unroll
+                                for (int j = 0; j < 32; j += 8) {
+                                    uint32_t w[4][4];       // [lo-half hi, lo-half lo, hi-half hi, hi-half lo][4 x half2]
+#pragma unroll
+                                    for (int e = 0; e < 8; e += 2) {
+                                        __half h[4][2];
+#pragma unroll
+                                        for (int u = 0; u < 2; ++u) {
+                                            float a = rs * __uint_as_float(va[j + e + u]);
+                                            float b = rs * __uint_as_float(vb[j + e + u]);
+                                            if (bias) { a += bias[n_lo + j + e + u]; b += bias[n_lo + hd + j + e + u]; }
+                                            float lo = a, hi = b;
+                                            if (p.cos_t) {
+                                                lo = a * cs[j + e + u] - b * sn[j + e + u];
+                                                hi = b * cs[j + e + u] + a * sn[j + e + u];
+                                            }
+                                            split_half(lo * mul, h[0][u], h[1][u]);
+                                            split_half(hi * mul, h[2][u], h[3][u]);
+                                        }
+#pragma unroll
+                                        for (int k = 0; k < 4; ++k) w[k][e >> 1] = pack_half2(h[k][0], h[k][1]);
+                                    }
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        const uint32_t dst = stage + (uint32_t)(k * 2048 + lane * 64 + j * 2);
+                                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[k][0]), "r"(w[k][1]), "r"(w[k][2]), "r"(w[k][3]) : "memory");
+                                    }
+                                }
+                                fence_async_smem();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    const int bh = bseq * p.n_heads + head0 + hh;
+                                    tma_store_3d(mh, stage, part * 32, pos0, bh);
+                                    tma_store_3d(ml, stage + 2048, part * 32, pos0, bh);
+                                    tma_store_3d(mh, stage + 4096, hd + part * 32, pos0, bh);
+                                    tma_store_3d(ml, stage + 6144, hd + part * 32, pos0, bh);
+                                    bulk_commit();
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int c = 0; c < BN / 32; ++c) {
+                            uint32_t v[32];
+                            __syncwarp();
+                            tmem_ld32(t_addr + (uint32_t)(c * 32), v);
+                            tmem_ld_wait();
+                            const uint32_t box = stage + (uint32_t)((c & 1) * 4096);    // hi box, lo box 2 KB further
+                            if (lane == 0) bulk_wait_read_1();
+                            __syncwarp();
+                            const int64_t n0 = n_base + c * 32;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                float x = rs * __uint_as_float(v[j]);
+                                if (bias) x += bias[n0 + j];
+                                __half h, l;
+                                split_half(x, h, l);
+                                // transposed: row = feature j, column = position (this lane)
+                                const uint32_t dst = box + (uint32_t)(j * 64 + lane * 2);
+                                asm volatile("st.shared.b16 [%0], %1;" ::"r"(dst), "h"(__half_as_ushort(h)) : "memory");
+                                asm volatile("st.shared.b16 [%0], %1;" ::"r"(dst + 2048), "h"(__half_as_ushort(l)) : "memory");
+                            }
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                const int hh = (c * 32) / dh, d0 = (c * 32) % dh;
+                                const int bh = bseq * p.n_heads + head0 + hh;
+                                tma_store_3d(&att.vh, box, pos0, d0, bh);
+                                tma_store_3d(&att.vl, box + 2048, pos0, d0, bh);
+                                bulk_commit();
+                            }
+                        }
+                    }
+                }
+            }
             if (p.mode == 3) {
                 // SiLU-gated FFN: act = silu(gate) * up leaves as fp32 [rows, N/2]; the row maximum of |act| is
                 // collected for the activation quantiser that follows.
@@ -253,7 +388,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (row_ok) atomicMax(p.row_amax + row, __float_as_uint(amax));
             }
 #pragma unroll 1
-            for (int c = 0; c < (p.mode == 3 ? 0 : BN / 32); ++c) {
+            for (int c = 0; c < ((p.mode == 3 || p.mode == 2) ? 0 : BN / 32); ++c) {
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)(c * 32), v);
@@ -412,6 +547,18 @@ bool make_out_map(CUtensorMap* map, float* base, int64_t M, int64_t N, int Z) {
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D binary16 map {inner, rows, slabs} with 32 x 32 x 1 boxes (64-byte rows, no swizzle) for the mode-2 stores.
+bool make_half_box_map(CUtensorMap* map, void* base, int64_t inner, int64_t rows, int64_t slabs, int64_t row_pitch) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)slabs};
+    const cuuint64_t strides[2] = {(cuuint64_t)row_pitch * 2, (cuuint64_t)row_pitch * rows * 2};
+    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int num_sms() {
     static int n = 0;
     if (n == 0) {
@@ -427,6 +574,7 @@ template <int BN, int CG>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
     using Cfg = TileCfg<BN, CG>;
     alignas(64) CUtensorMap map_a, map_b, map_out;
+    alignas(64) AttMaps att;
     const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
     if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN / CG))
         return ZOQAT_ERR_CUDA;
@@ -437,15 +585,31 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     p.err_flag = a.err_flag;
     p.tiles_m = (int)((a.M + BM * CG - 1) / (BM * CG));
     p.tiles_n = (int)((a.N + BN - 1) / BN);
-    p.tma_out = (a.mode == 0 && a.N % 4 == 0) ? 1 : 0;
+    p.tma_out = (a.mode == 0 && a.N % 4 == 0) ? 1 : 0;      // mode 2 never stores fp32
     p.row_amax = a.row_amax;
+    p.seq = a.seq; p.n_heads = a.n_heads; p.d_head = a.d_head; p.d_model = a.n_heads * a.d_head;
+    p.cos_t = a.cos_t; p.sin_t = a.sin_t; p.q_mul = a.att.q_mul;
+    if (a.mode == 2) {
+        const int64_t dm = (int64_t)a.n_heads * a.d_head;
+        if (CG != 2 || BN != 256 || a.N != 3 * dm || dm % 256 != 0 || a.seq <= 0 || a.seq % 32 != 0 || a.M % a.seq != 0 ||
+            (a.d_head != 64 && a.d_head != 128) || (a.cos_t == nullptr) != (a.sin_t == nullptr) || !a.att.qh)
+            return ZOQAT_ERR_INVALID_ARG;
+        const int64_t bhs = (int64_t)a.Z * (a.M / a.seq) * a.n_heads;
+        if (!make_half_box_map(&att.qh, a.att.qh, a.d_head, a.seq, bhs, a.d_head) || !make_half_box_map(&att.ql, a.att.ql, a.d_head, a.seq, bhs, a.d_head) ||
+            !make_half_box_map(&att.kh, a.att.kh, a.d_head, a.seq, bhs, a.d_head) || !make_half_box_map(&att.kl, a.att.kl, a.d_head, a.seq, bhs, a.d_head) ||
+            !make_half_box_map(&att.vh, a.att.vth, a.seq, a.d_head, bhs, a.att.seq_pad) || !make_half_box_map(&att.vl, a.att.vtl, a.seq, a.d_head, bhs, a.att.seq_pad))
+            return ZOQAT_ERR_CUDA;
+        map_out = map_a;      // never dereferenced
+    } else {
+        att.qh = att.ql = att.kh = att.kl = att.vh = att.vl = map_a;     // never dereferenced
+    }
     if (a.mode == 3) {
         if (CG != 2 || BN != 256 || a.N % 256 != 0 || !a.row_amax || !a.out) return ZOQAT_ERR_INVALID_ARG;
         p.tiles_n = (int)(a.N / 256);
         if (!make_out_map(&map_out, a.out, a.M, a.N / 2, a.Z)) return ZOQAT_ERR_CUDA;
     } else if (p.tma_out) {
         if (!make_out_map(&map_out, a.out, a.M, a.N, a.Z)) return ZOQAT_ERR_CUDA;
-    } else {
+    } else if (a.mode != 2) {
         map_out = map_a;      // never dereferenced
     }
     static bool attr = false;
@@ -467,7 +631,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, CG>, map_a, map_b, map_out, p) != cudaSuccess) return ZOQAT_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, CG>, map_a, map_b, map_out, att, p) != cudaSuccess) return ZOQAT_ERR_CUDA;
     count_launch();
     return ZOQAT_OK;
 }
@@ -482,7 +646,7 @@ int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
          reinterpret_cast<uintptr_t>(a.bias)) & 15)
         return ZOQAT_ERR_INVALID_ARG;
     // the cross-entropy epilogue always uses 256-column tiles (gemm_ce_tiles)
-    if (a.mode == 3 && a.single_cta) return ZOQAT_ERR_UNSUPPORTED;
+    if ((a.mode == 3 || a.mode == 2) && a.single_cta) return ZOQAT_ERR_UNSUPPORTED;
     if (a.mode != 0 || a.N > 128) return a.single_cta ? launch_tc<256, 1>(a, s) : launch_tc<256, 2>(a, s);
     return launch_tc<128, 1>(a, s);
 }

@@ -309,6 +309,56 @@ def test_attention_kernels_agree_on_activation_like_inputs(zq):
     assert float(((a - b).abs() / scale).max()) <= 5e-6
 
 
+@pytest.mark.parametrize("B,S,H,dh,K,rope,bias", [(2, 96, 2, 128, 256, True, False), (1, 160, 4, 64, 128, True, True),
+                                                     (3, 64, 4, 128, 192, False, True), (2, 1024, 4, 128, 512, True, False)],
+                         ids=["dh128_rope", "dh64_rope_bias", "dh128_bias_only", "seq1024"])
+def test_qkv_projection_feeding_attention(zq, B, S, H, dh, K, rope, bias):
+    """The q|k|v projection whose epilogue writes the attention operands (rotary embedding, q scaling, binary16
+    hi / lo split, v transposed) against the float64 definition, and against the two-kernel route (fp32 q|k|v,
+    then the attention with its own preparation pass)."""
+    rng = np.random.default_rng(S + dh + K)
+    d = H * dh
+    a = rng.integers(-127, 128, (B * S, K)).astype(np.float32)
+    w = (rng.standard_normal((3 * d, K)) * 0.02).astype(np.float32)
+    rs = rng.uniform(0.005, 0.02, B * S).astype(np.float32)
+    bv = (0.1 * rng.standard_normal(3 * d)).astype(np.float32) if bias else None
+    cos = sin = None
+    if rope:
+        cos, sin = rope_tables(S, dh, 10000.0)
+    a_d, w_d = dev(a).bfloat16(), dev(w).bfloat16()
+    c_d = None if cos is None else dev(cos.astype(np.float32))
+    s_d = None if sin is None else dev(sin.astype(np.float32))
+    out, err = zq.zoqat_op_qkv_attention(a_d, w_d, B, S, H, dh, row_step=dev(rs), bias=None if bv is None else dev(bv), cos=c_d, sin=s_d)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    qkv = (a.astype(np.float64) @ w_d.float().cpu().numpy().astype(np.float64).T) * rs.astype(np.float64)[:, None]
+    if bv is not None:
+        qkv = qkv + bv.astype(np.float64)[None, :]
+    x = qkv.reshape(B, S, 3 * d)
+    want = causal_attention(x[..., :d], x[..., d:2 * d], x[..., 2 * d:], H, cos, sin).reshape(B * S, d)
+    got = out.cpu().numpy()
+    worst = np.max(np.abs(got - want))
+    print(f"[fused qkv+attention B={B} S={S} H={H} dh={dh}] max abs err {worst:.2e}")
+    assert worst <= 5e-6 * max(1.0, np.abs(want).max())
+    # the two-kernel route
+    qkv32, e2 = zq.zoqat_op_gemm(a_d, w_d, row_step=dev(rs), bias=None if bv is None else dev(bv))
+    ref, e3 = zq.zoqat_op_attention(qkv32, B, S, H, dh, c_d, s_d)
+    torch.cuda.synchronize()
+    assert int(e2.item()) == 0 and int(e3.item()) == 0
+    assert float((out - ref).abs().max()) <= 2e-6 * max(1.0, float(ref.abs().max()))
+
+
+def test_qkv_projection_rejects_unfusable_shapes(zq):
+    a = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((3 * 128, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(zq.ZoqatError):                      # d_model = 128 is not a multiple of 256
+        zq.zoqat_op_qkv_attention(a, w, 1, 64, 1, 128)
+    w2 = torch.zeros((3 * 256, 64), dtype=torch.bfloat16, device="cuda")
+    a2 = torch.zeros((40, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(zq.ZoqatError):                      # 40 positions: not a multiple of 32
+        zq.zoqat_op_qkv_attention(a2, w2, 1, 40, 2, 128)
+
+
 # ---- vocabulary projection + cross-entropy ---------------------------------------------------------
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("T,V,d", [(130, 1024, 256), (257, 5000, 128), (64, 50272, 64)])
