@@ -113,6 +113,9 @@ class OracleConfig:
     smoothing: bool = False          # Section 4.2: learnable per-channel scale / shift at the inputs of the block linears
                                      # of the trainable layers ('smooth_s_<point>', 'smooth_d_<point>'); needs
                                      # trainable_names = None
+    integer_linear: bool = False     # deployment arithmetic of the frozen (packed) linears, used by the decode path: integer
+                                     # dot products of activation codes and weight codes inside each group, the group step
+                                     # and the token step applied outside (no bfloat16 rounding of the dequantised weight)
     store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
                                      # residual stream) to binary32, as an implementation that keeps activations in
                                      # fp32 does; used only to measure how far two correct implementations can differ
@@ -283,10 +286,31 @@ class OracleModel:
     def _operand_round(self, x):
         return core.round_bf16(x.astype(F32)).astype(np.float64) if self.cfg.operand_bf16 else x
 
+    def lin_integer(self, x, l, name, bias=None):
+        """The linear as an integer runtime evaluates it (Section 4.3 representation: stored codes, one step and zero
+        point per group; per-token activation codes):
+            y[t, n] = s_t * sum_g Delta[n, g] * ( sum_{k in g} a[t, k] * (c[n, k] - z[n, g]) )
+        with the inner sums exact integers."""
+        cfg = self.cfg
+        w = self.p["layers"][l][name]
+        g = self.group_of(w)
+        codes, delta, zp, _ = core.weight_quant(w, g, cfg.w_bits)
+        a, s = act_quant(x, cfg.a_bits)
+        T, K = a.shape
+        N = w.shape[0]
+        cz = codes.reshape(N, K // g, g).astype(np.float64) - zp.astype(np.float64)[:, :, None]
+        inner = np.einsum("tgk,ngk->tng", a.reshape(T, K // g, g), cz)          # exact: integers far below 2^53
+        y = (inner * delta.astype(np.float64)[None, :, :]).sum(axis=-1) * s.astype(np.float64)[:, None]
+        if bias is not None:
+            y = y + bias.astype(np.float64)[None, :]
+        return self._store(y)
+
     def lin(self, x, l, name, seed, signed_eps, bias=None):
         """x [T, in] float64 -> [T, out] float64 through the quantised linear.  With smoothing
         (Section 4.2): Y = Q_a((X - delta) / s) Q_w(s (.) W)^T + (B + delta W^T), the division taken in
         binary32 as a multiplication by 1/s rounded once, the shift term with the unquantised W."""
+        if self.cfg.integer_linear and self.cfg.a_bits and self.cfg.w_bits and not self.is_trainable(l, name):
+            return self.lin_integer(x, l, name, bias)
         extra = None
         if self.has_smoothing(l):
             s_, d_ = self.smoothing_params(l, name, seed, signed_eps)
@@ -328,6 +352,19 @@ class OracleModel:
     def token_losses(self, tokens, labels, seed=0, signed_eps=0.0):
         """tokens, labels int [B, S]; labels < 0 are ignored.  Returns the per-position
         cross-entropy (float64 [B*S], 0 where ignored) and the valid mask."""
+        logits = self.logits(tokens, seed, signed_eps)
+        T = logits.shape[0]
+        lab = labels.reshape(-1)
+        valid = lab >= 0
+        mx = logits.max(axis=-1)
+        lse = mx + np.log(np.exp(logits - mx[:, None]).sum(axis=-1))
+        picked = logits[np.arange(T), np.where(valid, lab, 0)]
+        return np.where(valid, lse - picked, 0.0), valid
+
+    def logits(self, tokens, seed=0, signed_eps=0.0):
+        """Next-token logits of every position: float64 [B*S, vocab].  Row b*S + s depends on tokens[b, :s+1] only
+        (causal attention), so the logits a decoder produces at position s with a key/value cache are row s of the
+        forward over the prefix."""
         cfg = self.cfg
         B, S = tokens.shape
         T = B * S
@@ -371,12 +408,7 @@ class OracleModel:
         a = self._operand_round(x)
         logits = a @ self.head_operand(seed, signed_eps).T
         self._tap("logits", logits)
-        lab = labels.reshape(-1)
-        valid = lab >= 0
-        mx = logits.max(axis=-1)
-        lse = mx + np.log(np.exp(logits - mx[:, None]).sum(axis=-1))
-        picked = logits[np.arange(T), np.where(valid, lab, 0)]
-        return np.where(valid, lse - picked, 0.0), valid
+        return logits
 
     def loss(self, tokens, labels, seed=0, signed_eps=0.0):
         """L(Q(W + signed_eps u); B): mean next-token cross-entropy over labelled positions."""

@@ -301,3 +301,33 @@ def test_step_multi_reduces_to_step_and_uses_one_w_for_all_directions():
     for i, (_, _, g) in enumerate(want):
         m4.apply_update(77 + i, np.float32(lr_q * g))
     assert np.array_equal(m3.p["layers"][0]["wq"], m4.p["layers"][0]["wq"])
+
+
+# ---- deployment arithmetic of the packed linears (decode path) ---------------------------------------------
+def test_integer_linear_hand_case_and_agreement_with_folded_forward():
+    """lin_integer on a hand-computed case, and on a model: the integer evaluation differs from the training
+    forward (bfloat16-rounded dequantised weights) only by that rounding, 2^-9 relative per weight."""
+    from oracle.model import OracleModel, OracleConfig
+    cfg = OracleConfig(arch="llama", n_layers=1, d_model=4, n_heads=1, d_ffn=4, vocab=4, w_bits=2, w_group=4, a_bits=8,
+                       first_trainable_layer=1, head_trainable=False, integer_linear=True)
+    # one row of weights [-1, -0.25, 0.5, 2]: Delta = 1, z = 1, codes [0, 1, 1, 3] (golden case 1); a second row of zeros+3
+    w = np.array([[-1.0, -0.25, 0.5, 2.0], [0.0, 1.5, 2.5, 3.0]], np.float32)
+    m = OracleModel(cfg, {"layers": [{"wq": w}]})
+    x = np.array([[127.0, -64.0, 32.0, 1.0]])          # step = 1: codes are the values themselves
+    y = m.lin_integer(x, 0, "wq")
+    # row 0: codes - z = [-1, 0, 0, 2] -> 127*(-1) + 1*2 = -125; row 1 (Delta 1, z 0, codes [0, 2, 2, 3]): -128 + 64 + 3 = -61
+    assert y.tolist() == [[-125.0, -61.0]]
+
+    model, shape = make("llama", quant=True, first_trainable_layer=2, head_trainable=False)
+    tokens, _ = synth.make_batch(2, 12, shape["vocab"], seed=3)
+    folded = model.logits(tokens)
+    model.cfg.integer_linear = True
+    integer = model.logits(tokens)
+    model.cfg.integer_linear = False
+    rel = np.abs(integer - folded).max() / np.abs(folded).max()
+    assert 0 < rel < 2e-2          # different arithmetic, same model
+    # causality: the logits of position s do not depend on later tokens
+    t2 = tokens.copy()
+    t2[:, 8:] = (t2[:, 8:] + 7) % shape["vocab"]
+    model.cfg.integer_linear = True
+    assert np.array_equal(model.logits(t2).reshape(2, 12, -1)[:, :8], integer.reshape(2, 12, -1)[:, :8])
