@@ -453,6 +453,42 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
                               double* loss_sum_dev, int32_t* count_dev, int impl,
                               int32_t* err_flag_dev, void* stream);
 
+/* ---- decode-time inference over the packed representation -------------------------------
+ * The deployment side of the method (the paper's on-device tokens-per-second table): one new
+ * token per sequence and call, keys and values cached, every block linear read once per
+ * token as stored low-bit codes.  Needs a model whose block linears are all FROZEN_PACKED
+ * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups, a_bits in {4, 6, 8};
+ * batch in {1, 2, 4} sequences advance in lock step.
+ *
+ * Arithmetic: a packed linear is evaluated as an integer runtime does,
+ *     y[t, n] = s_t * sum_g Delta[n, g] * ( sum_{k in g} a[t, k] * (c[n, k] - z[n, g]) ) (+ bias),
+ * the inner sums exact integers (dp4a), the steps applied in fp32; it differs from the
+ * training forward only by that forward's bf16 rounding of (c - z) * Delta.  Norms,
+ * rotary embedding, attention (fp32, over an fp32 cache) and the bf16 vocabulary
+ * projection are those of the forward pass.
+ *
+ * zoqat_decode_begin converts the packed tensors once into `buffer_dev` (zoqat_decode_bytes()
+ * bytes, 256-byte aligned, caller-owned, in use until the handle is destroyed or begin is
+ * called again): 4-bit nibbles in input-channel order, contiguous group parameters, the
+ * vocabulary projection as bf16, and the key/value cache [layer][2][batch][head][max_len][d_head].
+ * zoqat_decode_step feeds tokens_dev[batch] at position `pos` (0-based; positions must be fed
+ * in order, each overwriting its cache slot) and writes logits_dev fp32 [batch, vocab]
+ * and/or next_token_dev int32 [batch] = argmax (lowest index on ties); either may be NULL.
+ * Asynchronous, no host synchronisation: a loop of steps can be captured in a CUDA graph. */
+int zoqat_decode_bytes(const zoqat_model_t* m, int batch, int max_len, size_t* bytes);
+int zoqat_decode_begin(zoqat_model_t* m, void* buffer_dev, size_t bytes, int batch, int max_len, void* stream);
+int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, float* logits_dev,
+                      int32_t* next_token_dev, void* stream);
+
+/* One packed linear of the decode path on raw buffers: packed_dev / qparams_dev as written by
+ * zoqat_op_pack_frozen for a [rows, cols] tensor; act_codes_dev bf16 [batch, cols] integer codes
+ * with their steps row_step_dev[batch] (zoqat_op_norm_act_operand output); out_dev fp32
+ * [batch, rows] (accumulate != 0 adds); nibble_scratch_dev: rows*cols/2 bytes, 16-byte aligned
+ * (the repacked codes).  batch in {1, 2, 4}; cols % 32 == 0. */
+int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group, int bits,
+                         const void* act_codes_dev, const float* row_step_dev, int batch, const float* bias_dev,
+                         int accumulate, float* out_dev, void* nibble_scratch_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

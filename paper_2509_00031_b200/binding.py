@@ -36,6 +36,7 @@ EXPORTS = [
     "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_qkv_attention", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
+    "zoqat_decode_bytes", "zoqat_decode_begin", "zoqat_decode_step", "zoqat_op_decode_gemv",
 ]
 
 
@@ -121,6 +122,10 @@ def lib():
             "zoqat_op_head_loss_scratch_bytes": [i64, i64, P(sz)],
             "zoqat_op_head_loss": [vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, i32, vp, vp],
             "zoqat_op_head_loss_static": [vp, vp, vp, i64, i64, i64, vp, vp, vp, i32, vp, vp],
+            "zoqat_decode_bytes": [vp, i32, i32, P(sz)],
+            "zoqat_decode_begin": [vp, vp, sz, i32, i32, vp],
+            "zoqat_decode_step": [vp, vp, i32, vp, vp, vp],
+            "zoqat_op_decode_gemv": [vp, vp, i64, i64, i32, i32, vp, vp, i32, vp, i32, vp, vp, vp],
         }
         for name, args in sigs.items():
             fn = getattr(L, name)
@@ -328,6 +333,16 @@ def zoqat_op_head_loss(a, b, labels, impl=GEMM_TCGEN05):
     return token_loss, loss_sum, count, err
 
 
+def zoqat_op_decode_gemv(packed, qparams, rows, cols, group, bits, act_codes, row_step, bias=None, out=None, accumulate=False):
+    batch = act_codes.shape[0]
+    if out is None:
+        out = torch.empty((batch, rows), dtype=torch.float32, device=packed.device)
+    scratch = torch.empty(rows * cols // 2, dtype=torch.uint8, device=packed.device)
+    _check(lib().zoqat_op_decode_gemv(_p(packed), _p(qparams), rows, cols, group, bits, _p(act_codes), _p(row_step), batch, _p(bias),
+                                      int(accumulate), _p(out), _p(scratch), _stream()))
+    return out
+
+
 STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -437,6 +452,24 @@ class ZoqatModel:
 
     def zoqat_prequantize_frozen(self):
         _check(lib().zoqat_prequantize_frozen(self.handle, _stream()))
+
+    def zoqat_decode_begin(self, batch, max_len):
+        """Allocates the decode buffer (kept alive by this object) and converts the packed model for decoding."""
+        nb = ctypes.c_size_t()
+        _check(lib().zoqat_decode_bytes(self.handle, batch, max_len, ctypes.byref(nb)))
+        self.decode_buffer = torch.empty(nb.value, dtype=torch.uint8, device="cuda")
+        self.decode_batch = batch
+        _check(lib().zoqat_decode_begin(self.handle, _p(self.decode_buffer), nb.value, batch, max_len, _stream()))
+        return nb.value
+
+    def zoqat_decode_step(self, tokens, pos, logits=None, next_token=None, want_logits=True):
+        """tokens: int32 device tensor [batch].  Returns (logits [batch, vocab] or None, next_token [batch])."""
+        if logits is None and want_logits:
+            logits = torch.empty((self.decode_batch, self.shape["vocab"]), dtype=torch.float32, device="cuda")
+        if next_token is None:
+            next_token = torch.empty(self.decode_batch, dtype=torch.int32, device="cuda")
+        _check(lib().zoqat_decode_step(self.handle, _p(tokens), pos, _p(logits), _p(next_token), _stream()))
+        return logits, next_token
 
     def zoqat_init_qparams(self):
         _check(lib().zoqat_init_qparams(self.handle, _stream()))

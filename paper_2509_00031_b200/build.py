@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libzoqat.so")
-SOURCES = ["api.cu", "weights.cu", "activations.cu", "attention.cu", "attention_tc.cu", "gemm_simt.cu", "gemm_tc.cu"]
+SOURCES = ["api.cu", "weights.cu", "activations.cu", "attention.cu", "attention_tc.cu", "gemm_simt.cu", "gemm_tc.cu", "decode.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -195,8 +195,24 @@ struct Profiler {
     ~Profiler() { for (auto e : pool) cudaEventDestroy(e); }
 };
 
+// Decode-time state (zoqat_decode_begin): nibble weights and contiguous group parameters per layer, the bf16 vocabulary
+// projection, the key/value cache and two small buffers, all inside the caller's decode buffer.
+struct DecodeLayer {
+    const void *w_qkv, *w_o, *w_up, *w_down;            // nibble codes; q|k|v and gate|up stored back to back
+    const float2 *q_qkv, *q_o, *q_up, *q_down;           // (step, zero point) per group, same order
+    float *cache_k, *cache_v;                            // [batch][heads][max_len][d_head]
+};
+struct DecodeState {
+    bool ready = false;
+    int batch = 0, max_len = 0;
+    std::vector<DecodeLayer> layers;
+    __nv_bfloat16* head = nullptr;
+    float *logits = nullptr, *q_rot = nullptr;
+};
+
 struct zoqat_model {
     Profiler prof;
+    DecodeState dec;
     zoqat_config_t cfg;
     std::vector<Layer> layers;
     const float *embed = nullptr, *pos = nullptr, *final_g = nullptr, *final_b = nullptr;
@@ -1219,6 +1235,153 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
     launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+}  // extern "C"
+
+// ---- decode-time inference over the packed representation ------------------------------------------------------
+namespace {
+
+struct DecodeSizes { size_t nib[4], qp_qkv, qp_up, head, cache, logits, q_rot, total; };
+
+int decode_sizes(const zoqat_model* m, int batch, int max_len, DecodeSizes& z) {
+    const zoqat_config_t& c = m->cfg;
+    if (batch != 1 && batch != 2 && batch != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode batch %d (supported: 1, 2, 4)", batch);
+    if (max_len <= 0 || max_len > c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "max_len %d must be in 1..max_seq (%d)", max_len, c.max_seq);
+    if (batch > c.max_batch * c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "batch exceeds the workspace");
+    if (c.a_bits == 0) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs quantised activations (a_bits 4, 6 or 8)");
+    if (c.w_group == 0 || c.w_bits > 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs column groups of 32, 64 or 128 and w_bits <= 4");
+    const size_t d = c.d_model, F = c.d_ffn, n_up = c.arch == ZOQAT_ARCH_LLAMA ? 2 * F : F;
+    z.nib[0] = align_up(3 * d * d / 2); z.nib[1] = align_up(d * d / 2); z.nib[2] = align_up(n_up * d / 2); z.nib[3] = align_up(d * F / 2);
+    z.qp_qkv = align_up(3 * d * (d / c.w_group) * 8);
+    z.qp_up = align_up(n_up * (d / c.w_group) * 8);
+    z.head = align_up((size_t)c.vocab * d * 2);
+    z.cache = align_up((size_t)batch * d * max_len * 4);           // one of K / V of one layer
+    z.logits = align_up((size_t)batch * c.vocab * 4);
+    z.q_rot = align_up((size_t)batch * d * 4);
+    z.total = (size_t)c.n_layers * (z.nib[0] + z.nib[1] + z.nib[2] + z.nib[3] + z.qp_qkv + z.qp_up + 2 * z.cache) + z.head + z.logits + z.q_rot;
+    return ZOQAT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int zoqat_decode_bytes(const zoqat_model_t* m, int batch, int max_len, size_t* bytes) {
+    if (!m || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    DecodeSizes z;
+    if (int rc = decode_sizes(m, batch, max_len, z)) return rc;
+    *bytes = z.total;
+    return ZOQAT_OK;
+}
+
+int zoqat_decode_begin(zoqat_model_t* m, void* buffer_dev, size_t bytes, int batch, int max_len, void* stream) {
+    if (!m || !buffer_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (reinterpret_cast<uintptr_t>(buffer_dev) & 255) return fail(ZOQAT_ERR_INVALID_ARG, "buffer_dev must be 256-byte aligned");
+    DecodeSizes z;
+    if (int rc = decode_sizes(m, batch, max_len, z)) return rc;
+    if (bytes < z.total) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "decode buffer %zu < %zu bytes", bytes, z.total);
+    if (!m->prequantized) return fail(ZOQAT_ERR_BAD_STATE, "call zoqat_prequantize_frozen first");
+    const zoqat_config_t& c = m->cfg;
+    const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r)
+            if (Ly.lin[r].present && !Ly.lin[r].packed_frozen())
+                return fail(ZOQAT_ERR_UNSUPPORTED, "decode runs on the packed representation: every block linear must be FROZEN_PACKED");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t d = c.d_model, F = c.d_ffn, G = c.w_group;
+    uint8_t* p = static_cast<uint8_t*>(buffer_dev);
+    auto take = [&](size_t n) { uint8_t* q = p; p += n; return q; };
+    DecodeState& D = m->dec;
+    D.layers.assign(c.n_layers, DecodeLayer());
+    for (int l = 0; l < c.n_layers; ++l) {
+        Layer& Ly = m->layers[l];
+        DecodeLayer& dl = D.layers[l];
+        uint8_t* nq = take(z.nib[0]); uint8_t* no = take(z.nib[1]); uint8_t* nu = take(z.nib[2]); uint8_t* nd = take(z.nib[3]);
+        float2* qq = reinterpret_cast<float2*>(take(z.qp_qkv));
+        float2* qu = reinterpret_cast<float2*>(take(z.qp_up));
+        for (int r = 0; r < 3; ++r) {
+            launch_repack_nibbles(Ly.lin[r].packed, (int64_t)(d * d), c.w_bits, nq + (size_t)r * d * d / 2, s);
+            CUDA_TRY(cudaMemcpyAsync(qq + (size_t)r * d * (d / G), Ly.lin[r].qparams, d * (d / G) * 8, cudaMemcpyDeviceToDevice, s));
+        }
+        launch_repack_nibbles(Ly.lin[ZOQAT_ROLE_WO].packed, (int64_t)(d * d), c.w_bits, no, s);
+        launch_repack_nibbles(Ly.lin[ZOQAT_ROLE_W_GATE].packed, (int64_t)(F * d), c.w_bits, nu, s);
+        CUDA_TRY(cudaMemcpyAsync(qu, Ly.lin[ZOQAT_ROLE_W_GATE].qparams, F * (d / G) * 8, cudaMemcpyDeviceToDevice, s));
+        if (llama) {
+            launch_repack_nibbles(Ly.lin[ZOQAT_ROLE_W_UP].packed, (int64_t)(F * d), c.w_bits, nu + F * d / 2, s);
+            CUDA_TRY(cudaMemcpyAsync(qu + F * (d / G), Ly.lin[ZOQAT_ROLE_W_UP].qparams, F * (d / G) * 8, cudaMemcpyDeviceToDevice, s));
+        }
+        launch_repack_nibbles(Ly.lin[ZOQAT_ROLE_W_DOWN].packed, (int64_t)(d * F), c.w_bits, nd, s);
+        dl.w_qkv = nq; dl.w_o = no; dl.w_up = nu; dl.w_down = nd;
+        dl.q_qkv = qq; dl.q_o = Ly.lin[ZOQAT_ROLE_WO].qparams; dl.q_up = qu; dl.q_down = Ly.lin[ZOQAT_ROLE_W_DOWN].qparams;
+        dl.cache_k = reinterpret_cast<float*>(take(z.cache));
+        dl.cache_v = reinterpret_cast<float*>(take(z.cache));
+    }
+    D.head = reinterpret_cast<__nv_bfloat16*>(take(z.head));
+    D.logits = reinterpret_cast<float*>(take(z.logits));
+    D.q_rot = reinterpret_cast<float*>(take(z.q_rot));
+    launch_to_bf16(m->head.w, D.head, (int64_t)c.vocab * d, s);
+    CUDA_TRY(cudaGetLastError());
+    D.batch = batch; D.max_len = max_len; D.ready = true;
+    return ZOQAT_OK;
+}
+
+int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group, int bits,
+                         const void* act_codes_dev, const float* row_step_dev, int batch, const float* bias_dev, int accumulate,
+                         float* out_dev, void* nibble_scratch_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 4)) return rc;
+    if ((rows * cols) % 128 || cols % 32) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128 and cols of 32");
+    if (!packed_dev || !qparams_dev || !act_codes_dev || !row_step_dev || !out_dev || !nibble_scratch_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (reinterpret_cast<uintptr_t>(nibble_scratch_dev) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "nibble_scratch_dev must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_repack_nibbles(static_cast<const uint32_t*>(packed_dev), rows * cols, bits, nibble_scratch_dev, s);
+    if (launch_decode_gemv(nibble_scratch_dev, static_cast<const float2*>(qparams_dev), (int)rows, (int)cols, group, batch,
+                           static_cast<const __nv_bfloat16*>(act_codes_dev), row_step_dev, bias_dev, accumulate, out_dev, s) != 0)
+        return fail(ZOQAT_ERR_UNSUPPORTED, "batch %d (supported: 1, 2, 4) or shape rejected", batch);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, float* logits_dev, int32_t* next_token_dev, void* stream) {
+    if (!m || !tokens_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    DecodeState& D = m->dec;
+    if (!D.ready) return fail(ZOQAT_ERR_BAD_STATE, "call zoqat_decode_begin first");
+    if (pos < 0 || pos >= D.max_len) return fail(ZOQAT_ERR_INVALID_ARG, "pos %d outside the cache (max_len %d)", pos, D.max_len);
+    const zoqat_config_t& c = m->cfg;
+    Workspace& w = m->ws;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
+    const int B = D.batch, d = c.d_model, F = c.d_ffn, H = c.n_heads, dh = d / H, G = c.w_group;
+    const int norm_kind = llama ? 1 : 2, n_up = llama ? 2 * F : F;
+    auto gemv = [&](const void* wq, const float2* qp, int N, int K, const float* bias, int accumulate, float* out) {
+        if (launch_decode_gemv(wq, qp, N, K, G, B, w.xa, w.row_step, bias, accumulate, out, s) != 0)
+            return fail(ZOQAT_ERR_UNSUPPORTED, "decode matrix-vector product rejected (N=%d K=%d)", N, K);
+        return (int)ZOQAT_OK;
+    };
+    launch_embed(tokens_dev, m->embed, m->pos ? m->pos + (size_t)pos * d : nullptr, B, 1, d, c.vocab, 1, w.h, s);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const Layer& Ly = m->layers[l];
+        const DecodeLayer& dl = D.layers[l];
+        launch_norm_act_operand(w.h, B, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B], c.norm_eps,
+                                c.a_bits, w.xa, w.row_step, nullptr, s);
+        if (int rc = gemv(dl.w_qkv, dl.q_qkv, 3 * d, d, llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d, 0, w.qkv)) return rc;
+        launch_decode_rope_cache(w.qkv, B, H, dh, pos, D.max_len, llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr,
+                                 D.q_rot, dl.cache_k, dl.cache_v, s);
+        launch_decode_attention(D.q_rot, dl.cache_k, dl.cache_v, B, H, dh, pos, D.max_len, w.att, s);
+        launch_norm_act_operand(w.att, B, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s);
+        if (int rc = gemv(dl.w_o, dl.q_o, d, d, Ly.vec[ZOQAT_ROLE_BO], 1, w.h)) return rc;
+        launch_norm_act_operand(w.h, B, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B], c.norm_eps,
+                                c.a_bits, w.xa, w.row_step, nullptr, s);
+        if (int rc = gemv(dl.w_up, dl.q_up, n_up, d, Ly.vec[ZOQAT_ROLE_B_FC1], 0, w.ffn)) return rc;
+        launch_ffn_act_operand(w.ffn, B, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s);
+        if (int rc = gemv(dl.w_down, dl.q_down, d, F, Ly.vec[ZOQAT_ROLE_B_FC2], 1, w.h)) return rc;
+    }
+    launch_norm_act_operand(w.h, B, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s);
+    float* logits = logits_dev ? logits_dev : D.logits;
+    if (launch_decode_head(D.head, c.vocab, d, B, w.xa, logits, s) != 0) return fail(ZOQAT_ERR_UNSUPPORTED, "vocabulary projection rejected");
+    if (next_token_dev) launch_decode_argmax(logits, B, c.vocab, next_token_dev, s);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -100,6 +100,19 @@ AttnOperands attention_tc_operands(void* scratch, int batch, int seq, int n_head
 int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d_head, const float* cos_t,
                         const float* sin_t, float* out, void* scratch, int32_t* err_flag, cudaStream_t s);
 
+// Decode-time inference over the packed representation (decode.cu).  launch_decode_gemv / launch_decode_head return 0 or -1
+// (unsupported shape: K % 32, group, batch not in {1, 2, 4}).
+void launch_repack_nibbles(const uint32_t* packed, int64_t n, int bits, void* out, cudaStream_t s);
+void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
+int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
+                       const float* row_step, const float* bias, int accumulate, float* out, cudaStream_t s);
+void launch_decode_rope_cache(const float* qkv, int batch, int n_heads, int dh, int pos, int max_len, const float* cos_t,
+                              const float* sin_t, float* q_out, float* cache_k, float* cache_v, cudaStream_t s);
+void launch_decode_attention(const float* q, const float* cache_k, const float* cache_v, int batch, int n_heads, int dh, int pos,
+                             int max_len, float* out, cudaStream_t s);
+int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_bfloat16* x, float* logits, cudaStream_t s);
+void launch_decode_argmax(const float* logits, int batch, int V, int32_t* next, cudaStream_t s);
+
 // out[z*M + m, n] (+)= row_step[z*M+m] * sum_k A[z*M+m, k] * B[z][n, k] (+ bias[n]) (relu)
 // mode 1: cross-entropy partials instead of a store (labels[m], partials [Z*M, n_tiles], label_logit [Z*M]).
 struct GemmArgs {

@@ -1,0 +1,332 @@
+// Decode-time inference with the packed representation of Section 4.3 (one new token per sequence and step, keys and
+// values cached): the deployment side of the method.  Every block linear is a matrix-vector product over stored
+// low-bit codes, so the step is bound by reading the weights once from HBM:
+//
+//   repack_nibbles_kernel   once per model: the bit-plane packing (built for warp ballots in the training path) is
+//                           turned into 4-bit nibbles in input-channel order, the layout integer dot products want.
+//   decode_gemv_kernel      y[m, n] (+)= s_m * sum_g Delta[n, g] * ( sum_{k in g} a[m, k] * (c[n, k] - z[n, g]) ) (+ bias)
+//                           for up to 4 sequences m: one warp per output row n, 32 codes (16 bytes) per lane and load,
+//                           dp4a on the nibble pairs against int8 activation codes staged in shared memory, the inner
+//                           sums exact integers, steps applied in fp32.
+//   decode_rope_cache_kernel / decode_attention_kernel   rotary embedding of the new q and k, append k and v to the
+//                           cache, softmax(q K^T / sqrt(d_head)) V over the cached positions (fp32).
+//   decode_head_kernel      logits = bf16(x) . bf16(W_head) (the vocabulary projection is unquantised), fp32 accumulate.
+//   decode_argmax_kernel    greedy next token (lowest index on ties).
+#include "common.cuh"
+
+namespace zq {
+namespace {
+
+constexpr int kGemvThreads = 256;
+
+// ---- layout conversion ---------------------------------------------------------------------------------------
+// packed: per 128 consecutive elements 4*BITS words, bit `lane` of word j*BITS + b = bit b of the code of element
+// 4*lane + j.  out: one byte per two elements, element 2i in the low nibble.
+template <int BITS>
+__global__ void repack_nibbles_kernel(const uint32_t* __restrict__ packed, int64_t n4, uint16_t* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t* run = packed + (i >> 5) * (4 * BITS);
+        uint32_t c[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            c[j] = 0;
+#pragma unroll
+            for (int b = 0; b < BITS; ++b) c[j] |= ((__ldg(run + j * BITS + b) >> lane) & 1u) << b;
+        }
+        out[i] = (uint16_t)(c[0] | (c[1] << 4) | (c[2] << 8) | (c[3] << 12));
+    }
+}
+
+__global__ void to_bf16_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, int64_t n4) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const float4 v = src[i];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        dst[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+    }
+}
+
+// ---- matrix-vector product over nibble codes --------------------------------------------------------------------
+// act: bf16 integer codes [MB, K] (as the activation-operand kernels write them) with their steps row_step[MB].
+// Shared memory: per sequence the even-k and odd-k codes as int8 (so that four consecutive bytes pair with the low / high
+// nibbles of one weight word) and the sum of the codes of every 32-element chunk (for the zero-point term).
+template <int MB>
+__global__ void __launch_bounds__(kGemvThreads)
+decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qparams, int N, int K, int group,
+                   const __nv_bfloat16* __restrict__ act, const float* __restrict__ row_step, const float* __restrict__ bias,
+                   int accumulate, float* __restrict__ out) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    int8_t* even = reinterpret_cast<int8_t*>(smem);                        // [MB][K/2]
+    int8_t* odd = even + (size_t)MB * (K / 2);                             // [MB][K/2]
+    int32_t* csum = reinterpret_cast<int32_t*>(odd + (size_t)MB * (K / 2));   // [MB][K/32]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < MB * (K / 2); i += kGemvThreads) {
+        const int m = i / (K / 2), k2 = i % (K / 2);
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(act + (size_t)m * K + 2 * k2);
+        even[i] = (int8_t)__bfloat162float(v.x);
+        odd[i] = (int8_t)__bfloat162float(v.y);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < MB * (K / 32); i += kGemvThreads) {
+        const int m = i / (K / 32), ch = i % (K / 32);
+        int sum = 0;
+        for (int j = 0; j < 16; ++j) sum += even[(size_t)m * (K / 2) + ch * 16 + j] + odd[(size_t)m * (K / 2) + ch * 16 + j];
+        csum[i] = sum;
+    }
+    __syncthreads();
+    const int chunks = K / 32;                 // 16-byte weight loads per row
+    const int gpr = K / group;
+    for (int n = blockIdx.x * (kGemvThreads / 32) + warp; n < N; n += gridDim.x * (kGemvThreads / 32)) {
+        const uint4* wrow = wq + (size_t)n * chunks;
+        const float2* qrow = qparams + (size_t)n * gpr;
+        float acc[MB];
+#pragma unroll
+        for (int m = 0; m < MB; ++m) acc[m] = 0.0f;
+        for (int ch = lane; ch < chunks; ch += 32) {
+            const uint4 w = __ldg(wrow + ch);
+            const float2 qp = __ldg(qrow + (ch * 32) / group);
+            const int zp = (int)qp.y;
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+                const uint4 e = *reinterpret_cast<const uint4*>(even + (size_t)m * (K / 2) + ch * 16);
+                const uint4 o = *reinterpret_cast<const uint4*>(odd + (size_t)m * (K / 2) + ch * 16);
+                const uint32_t ee[4] = {e.x, e.y, e.z, e.w}, oo[4] = {o.x, o.y, o.z, o.w};
+                int dp = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    dp = __dp4a((int)(ww[q] & 0x0F0F0F0Fu), (int)ee[q], dp);
+                    dp = __dp4a((int)((ww[q] >> 4) & 0x0F0F0F0Fu), (int)oo[q], dp);
+                }
+                acc[m] = __fmaf_rn((float)(dp - zp * csum[m * (K / 32) + ch]), qp.x, acc[m]);
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < MB; ++m) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+                float y = row_step[m] * acc[m];
+                if (bias) y += bias[n];
+                float* o = out + (size_t)m * N + n;
+                *o = accumulate ? *o + y : y;
+            }
+        }
+    }
+}
+
+// ---- attention over the cache -----------------------------------------------------------------------------------
+// qkv fp32 [B, 3*d]; cache_k / cache_v fp32 [B][H][max_len][dh] of one layer.  One CTA per (sequence, head): rotates q
+// and k by the angle of `pos`, appends k and v at `pos`, leaves the rotated q in q_out [B, d].
+__global__ void decode_rope_cache_kernel(const float* __restrict__ qkv, int n_heads, int dh, int pos, int max_len,
+                                         const float* __restrict__ cos_t, const float* __restrict__ sin_t,
+                                         float* __restrict__ q_out, float* __restrict__ cache_k, float* __restrict__ cache_v) {
+    const int b = blockIdx.y, h = blockIdx.x, d = n_heads * dh, hd = dh / 2;
+    const float* q = qkv + (size_t)b * 3 * d + h * dh;
+    const float* k = q + d;
+    const float* v = q + 2 * d;
+    float* ck = cache_k + (((size_t)b * n_heads + h) * max_len + pos) * dh;
+    float* cv = cache_v + (((size_t)b * n_heads + h) * max_len + pos) * dh;
+    float* qo = q_out + (size_t)b * d + h * dh;
+    for (int i = threadIdx.x; i < hd; i += blockDim.x) {
+        float c = 1.0f, s = 0.0f;
+        if (cos_t) { c = cos_t[(size_t)pos * hd + i]; s = sin_t[(size_t)pos * hd + i]; }
+        const float q1 = q[i], q2 = q[i + hd], k1 = k[i], k2 = k[i + hd];
+        qo[i] = q1 * c - q2 * s; qo[i + hd] = q2 * c + q1 * s;
+        ck[i] = k1 * c - k2 * s; ck[i + hd] = k2 * c + k1 * s;
+    }
+    for (int i = threadIdx.x; i < dh; i += blockDim.x) cv[i] = v[i];
+}
+
+// out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA (128 threads) per (sequence, head).
+__global__ void __launch_bounds__(128)
+decode_attention_kernel(const float* __restrict__ q_in, const float* __restrict__ cache_k, const float* __restrict__ cache_v,
+                        int n_heads, int dh, int pos, int max_len, float* __restrict__ out) {
+    extern __shared__ float sc[];              // scores of positions 0..pos, then dh floats of q
+    __shared__ float red[4];
+    const int b = blockIdx.y, h = blockIdx.x, d = n_heads * dh;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* qs = sc + (pos + 1);
+    const float* q = q_in + (size_t)b * d + h * dh;
+    const float* kc = cache_k + ((size_t)b * n_heads + h) * max_len * dh;
+    const float* vc = cache_v + ((size_t)b * n_heads + h) * max_len * dh;
+    for (int i = threadIdx.x; i < dh; i += 128) qs[i] = q[i];
+    __syncthreads();
+    const float scale = 1.0f / sqrtf((float)dh);
+    float mx = -INFINITY;
+    for (int t = warp; t <= pos; t += 4) {                      // a warp per cached position
+        float acc = 0.0f;
+        for (int i = lane; i < dh; i += 32) acc = __fmaf_rn(qs[i], kc[(size_t)t * dh + i], acc);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        acc *= scale;
+        if (lane == 0) sc[t] = acc;
+        mx = fmaxf(mx, acc);
+    }
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    __syncthreads();
+    float sum = 0.0f;
+    for (int t = threadIdx.x; t <= pos; t += 128) { const float p = expf(sc[t] - mx); sc[t] = p; sum += p; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) red[warp] = sum;
+    __syncthreads();
+    const float inv = 1.0f / (red[0] + red[1] + red[2] + red[3]);
+    for (int i = threadIdx.x; i < dh; i += 128) {
+        float acc = 0.0f;
+        for (int t = 0; t <= pos; ++t) acc = __fmaf_rn(sc[t], vc[(size_t)t * dh + i], acc);
+        out[(size_t)b * d + h * dh + i] = acc * inv;
+    }
+}
+
+// ---- vocabulary projection and greedy choice -----------------------------------------------------------------------
+// logits[m, v] = sum_k x[m, k] * W[v, k], both bf16, fp32 accumulation; one warp per vocabulary row.
+template <int MB>
+__global__ void __launch_bounds__(kGemvThreads)
+decode_head_kernel(const uint4* __restrict__ w, int V, int d, const __nv_bfloat16* __restrict__ x, float* __restrict__ logits) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem);            // [MB][d]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < MB * d; i += kGemvThreads) xs[i] = x[i];
+    __syncthreads();
+    const int chunks = d / 8;
+    for (int v = blockIdx.x * (kGemvThreads / 32) + warp; v < V; v += gridDim.x * (kGemvThreads / 32)) {
+        float acc[MB];
+#pragma unroll
+        for (int m = 0; m < MB; ++m) acc[m] = 0.0f;
+        for (int ch = lane; ch < chunks; ch += 32) {
+            const uint4 wv = __ldg(w + (size_t)v * chunks + ch);
+            const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)m * d + ch * 8);
+                const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&xv);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 a = __bfloat1622float2(w2[q]), bb = __bfloat1622float2(x2[q]);
+                    acc[m] = __fmaf_rn(a.x, bb.x, acc[m]);
+                    acc[m] = __fmaf_rn(a.y, bb.y, acc[m]);
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < MB; ++m) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], o);
+            if (lane == 0) logits[(size_t)m * V + v] = acc[m];
+        }
+    }
+}
+
+// next[m] = index of the largest logit of row m (the lowest index among equals); one CTA per row.
+__global__ void __launch_bounds__(1024)
+decode_argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ next) {
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    const float* row = logits + (size_t)blockIdx.x * V;
+    float best = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int v = threadIdx.x; v < V; v += 1024) {
+        const float x = row[v];
+        if (x > best || (x == best && v < idx)) { best = x; idx = v; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (ob > best || (ob == best && oi < idx)) { best = ob; idx = oi; }
+    }
+    if ((threadIdx.x & 31) == 0) { bv[threadIdx.x >> 5] = best; bi[threadIdx.x >> 5] = idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 32; ++i)
+            if (bv[i] > bv[0] || (bv[i] == bv[0] && bi[i] < bi[0])) { bv[0] = bv[i]; bi[0] = bi[i]; }
+        next[blockIdx.x] = bi[0];
+    }
+}
+
+inline int capped_blocks(int64_t work, int per_block, int cap) {
+    int64_t b = (work + per_block - 1) / per_block;
+    if (b > cap) b = cap;
+    return (int)(b < 1 ? 1 : b);
+}
+
+}  // namespace
+
+void launch_repack_nibbles(const uint32_t* packed, int64_t n, int bits, void* out, cudaStream_t s) {
+    if (n == 0) return;
+    const int64_t n4 = n / 4;
+    const int grid = capped_blocks(n4, 256, 148 * 8);
+    uint16_t* o = static_cast<uint16_t*>(out);
+    if (bits == 2) repack_nibbles_kernel<2><<<grid, 256, 0, s>>>(packed, n4, o);
+    else if (bits == 3) repack_nibbles_kernel<3><<<grid, 256, 0, s>>>(packed, n4, o);
+    else repack_nibbles_kernel<4><<<grid, 256, 0, s>>>(packed, n4, o);
+    count_launch();
+}
+
+void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s) {
+    if (n == 0) return;
+    to_bf16_kernel<<<capped_blocks(n / 4, 256, 148 * 8), 256, 0, s>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<uint2*>(dst), n / 4);
+    count_launch();
+}
+
+size_t decode_gemv_smem_bytes(int mb, int K) { return (size_t)mb * K + (size_t)mb * (K / 32) * 4; }
+
+int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
+                       const float* row_step, const float* bias, int accumulate, float* out, cudaStream_t s) {
+    if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
+    const size_t smem = decode_gemv_smem_bytes(mb, K);
+    if (smem > 160 * 1024) return -1;
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * 4);
+    const uint4* w4 = static_cast<const uint4*>(wq);
+#define ZQ_GEMV(MBV)                                                                                                      \
+    {                                                                                                                     \
+        static bool attr = false;                                                                                         \
+        if (!attr) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
+        decode_gemv_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, group, act, row_step, bias, accumulate, out); \
+    }
+    if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else return -1;
+#undef ZQ_GEMV
+    count_launch();
+    return 0;
+}
+
+void launch_decode_rope_cache(const float* qkv, int batch, int n_heads, int dh, int pos, int max_len, const float* cos_t,
+                              const float* sin_t, float* q_out, float* cache_k, float* cache_v, cudaStream_t s) {
+    decode_rope_cache_kernel<<<dim3(n_heads, batch), 64, 0, s>>>(qkv, n_heads, dh, pos, max_len, cos_t, sin_t, q_out, cache_k, cache_v);
+    count_launch();
+}
+
+void launch_decode_attention(const float* q, const float* cache_k, const float* cache_v, int batch, int n_heads, int dh, int pos,
+                             int max_len, float* out, cudaStream_t s) {
+    const size_t smem = (size_t)(pos + 1 + dh) * 4;
+    static bool attr = false;
+    if (!attr) { cudaFuncSetAttribute(decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024); attr = true; }
+    decode_attention_kernel<<<dim3(n_heads, batch), 128, smem, s>>>(q, cache_k, cache_v, n_heads, dh, pos, max_len, out);
+    count_launch();
+}
+
+int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_bfloat16* x, float* logits, cudaStream_t s) {
+    if (d % 8) return -1;
+    const size_t smem = (size_t)mb * d * 2;
+    const int grid = capped_blocks(V, kGemvThreads / 32, 148 * 4);
+    const uint4* w4 = reinterpret_cast<const uint4*>(w);
+    if (mb == 1) decode_head_kernel<1><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+    else if (mb == 2) decode_head_kernel<2><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+    else if (mb == 4) decode_head_kernel<4><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+    else return -1;
+    count_launch();
+    return 0;
+}
+
+void launch_decode_argmax(const float* logits, int batch, int V, int32_t* next, cudaStream_t s) {
+    decode_argmax_kernel<<<batch, 1024, 0, s>>>(logits, V, next);
+    count_launch();
+}
+
+}  // namespace zq

@@ -1,0 +1,106 @@
+"""GPU parity of decode-time inference over the packed representation (Section 4.3 codes, key/value cache) against
+the oracle: the packed matrix-vector product against exact integer arithmetic, then whole models token by token -
+the logits the cached decoder produces at position s against row s of the oracle's forward over the prefix (its
+integer-linear arithmetic), for both decoder families, several bit widths and batch sizes, and the greedy choice."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import core
+from oracle.model import OracleConfig, OracleModel, act_quant
+from paper_2509_00031_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def zq():
+    from paper_2509_00031_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+@pytest.mark.parametrize("bits,group,rows,cols,batch", [(4, 128, 300, 512, 1), (4, 64, 96, 1024 + 64, 2), (2, 32, 256, 4096, 4),
+                                                         (3, 128, 64, 11008, 4)])
+def test_packed_gemv_is_exact_integer_arithmetic(zq, bits, group, rows, cols, batch):
+    if (rows * cols) % 128:
+        pytest.skip("packed tensors need rows*cols % 128 == 0")
+    rng = np.random.default_rng(rows + cols)
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    x = (rng.standard_normal((batch, cols)) * rng.uniform(0.5, 3.0, (batch, 1))).astype(np.float32)
+    bias = (0.1 * rng.standard_normal(rows)).astype(np.float32)
+    packed, qparams = zq.zoqat_op_pack_frozen(dev(w), group, bits)
+    op, step, _ = zq.zoqat_op_norm_act_operand(dev(x), 0, None, None, 0.0, 8)
+    out = zq.zoqat_op_decode_gemv(packed, qparams, rows, cols, group, bits, op, step, bias=dev(bias))
+    codes, delta, zp, _ = core.weight_quant(w, group, bits)
+    a, s = act_quant(x.astype(np.float64), 8)
+    assert np.array_equal(op.float().cpu().numpy(), a)
+    cz = codes.reshape(rows, cols // group, group).astype(np.float64) - zp.astype(np.float64)[:, :, None]
+    inner = np.einsum("tgk,ngk->tng", a.reshape(batch, cols // group, group), cz)
+    want = (inner * delta.astype(np.float64)[None]).sum(-1) * s.astype(np.float64)[:, None] + bias[None, :]
+    bound = (np.abs(inner) * delta.astype(np.float64)[None]).sum(-1) * s.astype(np.float64)[:, None]
+    got = out.cpu().numpy()
+    assert np.all(np.abs(got - want) <= 2e-6 * bound + 1e-6 * np.abs(want) + 1e-9)
+    # accumulate adds onto what is there
+    base = torch.full((batch, rows), 0.5, dtype=torch.float32, device="cuda")
+    out2 = zq.zoqat_op_decode_gemv(packed, qparams, rows, cols, group, bits, op, step, out=base.clone(), accumulate=True)
+    assert torch.allclose(out2, out - dev(bias)[None, :] + 0.5, rtol=0, atol=1e-5 * float(out.abs().max()))
+
+
+SHAPES = {
+    "llama_w4a8": dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=600, w_bits=4, w_group=64, a_bits=8),
+    "opt_w3a8": dict(arch="opt", n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=333, w_bits=3, w_group=128, a_bits=8),
+    "llama_w2a4": dict(arch="llama", n_layers=1, d_model=256, n_heads=2, d_ffn=512, vocab=512, w_bits=2, w_group=32, a_bits=4),
+}
+
+
+@pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33)])
+def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
+    shape = SHAPES[name]
+    params = synth.make_params(shape, seed=5, max_seq=seq, jitter=True)
+    L = shape["n_layers"]
+    oracle = OracleModel(OracleConfig(arch=shape["arch"], n_layers=L, d_model=shape["d_model"], n_heads=shape["n_heads"],
+                                      d_ffn=shape["d_ffn"], vocab=shape["vocab"], w_bits=shape["w_bits"], w_group=shape["w_group"],
+                                      a_bits=shape["a_bits"], first_trainable_layer=L, head_trainable=False, integer_linear=True),
+                         synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, first_trainable_layer=L,
+                          head_trainable=False, packed_frozen=True)
+    model.zoqat_prequantize_frozen()
+    model.zoqat_decode_begin(batch, seq)
+    tokens, _ = synth.make_batch(batch, seq, shape["vocab"], seed=21)
+    want = oracle.logits(tokens).reshape(batch, seq, -1)
+    scale = np.abs(want).max()
+    agree = total = 0
+    for pos in range(seq):
+        logits, nxt = model.zoqat_decode_step(dev(tokens[:, pos].copy()), pos)
+        got = logits.cpu().numpy()
+        model.zoqat_check()
+        err = np.abs(got - want[:, pos]).max()
+        assert err <= 2e-4 * scale, (pos, err, scale)
+        # greedy choice: the device's argmax of its own logits, and the oracle's wherever its top two are well apart
+        assert np.array_equal(nxt.cpu().numpy(), got.argmax(-1))
+        top2 = np.sort(want[:, pos], axis=-1)[:, -2:]
+        clear = (top2[:, 1] - top2[:, 0]) > 1e-3 * scale
+        agree += int((nxt.cpu().numpy()[clear] == want[:, pos].argmax(-1)[clear]).sum())
+        total += int(clear.sum())
+    assert total > 0 and agree == total
+
+
+def test_decode_rejects_models_that_are_not_packed(zq):
+    shape = SHAPES["llama_w4a8"]
+    params = synth.make_params(shape, seed=5, max_seq=16)
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=1, max_seq=16)
+    with pytest.raises(zq.ZoqatError):
+        model.zoqat_decode_begin(1, 16)
+    packed = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=1, max_seq=16, first_trainable_layer=2, head_trainable=False,
+                           packed_frozen=True)
+    packed.zoqat_prequantize_frozen()
+    with pytest.raises(zq.ZoqatError):
+        packed.zoqat_decode_begin(3, 16)                 # batch 3
+    packed.zoqat_decode_begin(1, 16)
+    with pytest.raises(zq.ZoqatError):
+        packed.zoqat_decode_step(torch.zeros(1, dtype=torch.int32, device="cuda"), 16)       # position beyond the cache
