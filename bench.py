@@ -173,36 +173,6 @@ def run_reference(args, w, rank, world):
 
 
 # ---------------------------------------------------------------------------------------------
-def make_device_params(w, torch, seed=0):
-    """Random-init parameters directly on the device (N(0, 0.02^2), bf16-rounded where the workload says so)."""
-    from paper_2509_00031_b200 import synth
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(seed)
-    d, f, v = w["d_model"], w["d_ffn"], w["vocab"]
-    opt = w["arch"] == "opt"
-
-    def rnd(*s):
-        t = torch.empty(s, dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=gen)
-        return t.bfloat16().float() if w.get("bf16_init") else t
-
-    ones = lambda n: torch.ones(n, dtype=torch.float32, device="cuda")
-    zeros = lambda n: torch.zeros(n, dtype=torch.float32, device="cuda")
-    p = {"embed": rnd(v, d), "lm_head": rnd(v, d), "final_norm_g": ones(d), "layers": []}
-    if opt:
-        p["final_norm_b"] = zeros(d)
-        p["pos"] = rnd(w["seq"], d)
-    for _ in range(w["n_layers"]):
-        L = {"attn_norm_g": ones(d), "ffn_norm_g": ones(d)}
-        for name, (o, i) in synth.linear_shapes(w).items():
-            L[name] = rnd(o, i)
-        if opt:
-            L["attn_norm_b"] = zeros(d); L["ffn_norm_b"] = zeros(d)
-            for name, n in (("bq", d), ("bk", d), ("bv", d), ("bo", d), ("b_fc1", f), ("b_fc2", d)):
-                L[name] = zeros(n)
-        p["layers"].append(L)
-    return p
-
-
 def run_ours(args, w, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -216,7 +186,7 @@ def run_ours(args, w, rank, world, local_rank):
     nums = workload_numbers(w)
     ftl = w.get("first_trainable_layer", 0)
 
-    params = make_device_params(w, torch, seed=0)          # every replica holds the same masters
+    params = synth.make_device_params(w, seed=0)           # every replica holds the same masters
     names = w.get("trainable_names")
     any_packed = ftl > 0 or names is not None
     model = binding.ZoqatModel(w, params, max_batch=w["batch"], max_seq=w["seq"], first_trainable_layer=ftl,

@@ -8,8 +8,8 @@
 //                           for up to 4 sequences m: one warp per output row n, 32 codes (16 bytes) per lane and load,
 //                           dp4a on the nibble pairs against int8 activation codes staged in shared memory, the inner
 //                           sums exact integers, steps applied in fp32.
-//   decode_rope_cache_kernel / decode_attention_kernel   rotary embedding of the new q and k, append k and v to the
-//                           cache, softmax(q K^T / sqrt(d_head)) V over the cached positions (fp32).
+//   decode_attention_kernel rotary embedding of the new q and k, append k and v to the cache,
+//                           softmax(q K^T / sqrt(d_head)) V over the cached positions (fp32), one launch.
 //   decode_head_kernel      logits = bf16(x) . bf16(W_head) (the vocabulary projection is unquantised), fp32 accumulate.
 //   decode_argmax_kernel    greedy next token (lowest index on ties).
 #include "common.cuh"
@@ -52,53 +52,98 @@ __global__ void to_bf16_kernel(const float4* __restrict__ src, uint2* __restrict
 // nibbles of one weight word) and the sum of the codes of every 32-element chunk (for the zero-point term).
 template <int MB>
 __global__ void __launch_bounds__(kGemvThreads)
-decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qparams, int N, int K, int group,
+decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qparams, int N, int K, int group_shift,
                    const __nv_bfloat16* __restrict__ act, const float* __restrict__ row_step, const float* __restrict__ bias,
                    int accumulate, float* __restrict__ out) {
     extern __shared__ __align__(16) uint8_t smem[];
-    int8_t* even = reinterpret_cast<int8_t*>(smem);                        // [MB][K/2]
-    int8_t* odd = even + (size_t)MB * (K / 2);                             // [MB][K/2]
-    int32_t* csum = reinterpret_cast<int32_t*>(odd + (size_t)MB * (K / 2));   // [MB][K/32]
+    const int chunks = K >> 5;                 // 16-byte weight loads (32 codes) per row
+    uint4* even4 = reinterpret_cast<uint4*>(smem);                         // [MB][chunks]: the 16 even-k codes of a chunk
+    uint4* odd4 = even4 + MB * chunks;                                     // [MB][chunks]: the 16 odd-k codes
+    int32_t* csum = reinterpret_cast<int32_t*>(odd4 + MB * chunks);        // [MB][chunks]: sum of the chunk's 32 codes
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < MB * (K / 2); i += kGemvThreads) {
-        const int m = i / (K / 2), k2 = i % (K / 2);
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(act + (size_t)m * K + 2 * k2);
-        even[i] = (int8_t)__bfloat162float(v.x);
-        odd[i] = (int8_t)__bfloat162float(v.y);
+    const int gpr = K >> group_shift;
+    const int cshift = group_shift - 5;        // chunk -> group
+    // the first weights of this warp's first row are requested before anything else, so that the HBM latency runs
+    // under the staging of the activation codes
+    uint4 w[4];
+    float2 qp[4];
+    int n = blockIdx.x * (kGemvThreads / 32) + warp;
+    if (n < N) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int ch = lane + 32 * u;
+            if (ch < chunks) { w[u] = __ldg(wq + (size_t)n * chunks + ch); qp[u] = __ldg(qparams + (size_t)n * gpr + (ch >> cshift)); }
+        }
+    }
+    // staging: a thread converts 8 bf16 codes (one 16-byte load) into 4 even and 4 odd int8; the four threads of a
+    // chunk add up their code sums
+    {
+        uint32_t* even1 = reinterpret_cast<uint32_t*>(even4);
+        uint32_t* odd1 = reinterpret_cast<uint32_t*>(odd4);
+        const int per_row = K >> 3;
+        const int total = MB * per_row;
+        // every thread of the CTA runs every round (the shuffles below need whole warps); loads and stores are guarded
+        for (int base = 0; base < total; base += kGemvThreads) {
+            const int i = base + threadIdx.x;
+            const bool live = i < total;
+            uint32_t e = 0, o = 0;
+            int sum = 0;
+            if (live) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4*>(act) + i);
+                const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 f = __bfloat1622float2(p2[q]);
+                    const int a0 = (int)f.x, a1 = (int)f.y;
+                    sum += a0 + a1;
+                    e |= ((uint32_t)a0 & 0xFFu) << (8 * q);
+                    o |= ((uint32_t)a1 & 0xFFu) << (8 * q);
+                }
+                even1[i] = e;
+                odd1[i] = o;
+            }
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            if (live && (i & 3) == 0) csum[i >> 2] = sum;      // total is a multiple of 4: quads are whole
+        }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < MB * (K / 32); i += kGemvThreads) {
-        const int m = i / (K / 32), ch = i % (K / 32);
-        int sum = 0;
-        for (int j = 0; j < 16; ++j) sum += even[(size_t)m * (K / 2) + ch * 16 + j] + odd[(size_t)m * (K / 2) + ch * 16 + j];
-        csum[i] = sum;
-    }
-    __syncthreads();
-    const int chunks = K / 32;                 // 16-byte weight loads per row
-    const int gpr = K / group;
-    for (int n = blockIdx.x * (kGemvThreads / 32) + warp; n < N; n += gridDim.x * (kGemvThreads / 32)) {
+    bool first = true;                         // the first four loads of the first row are already in registers
+    for (; n < N; n += gridDim.x * (kGemvThreads / 32)) {
         const uint4* wrow = wq + (size_t)n * chunks;
         const float2* qrow = qparams + (size_t)n * gpr;
         float acc[MB];
 #pragma unroll
         for (int m = 0; m < MB; ++m) acc[m] = 0.0f;
-        for (int ch = lane; ch < chunks; ch += 32) {
-            const uint4 w = __ldg(wrow + ch);
-            const float2 qp = __ldg(qrow + (ch * 32) / group);
-            const int zp = (int)qp.y;
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        for (int ch0 = lane; ch0 < chunks; ch0 += 128) {      // four loads in flight per lane
+            if (!first) {
 #pragma unroll
-            for (int m = 0; m < MB; ++m) {
-                const uint4 e = *reinterpret_cast<const uint4*>(even + (size_t)m * (K / 2) + ch * 16);
-                const uint4 o = *reinterpret_cast<const uint4*>(odd + (size_t)m * (K / 2) + ch * 16);
-                const uint32_t ee[4] = {e.x, e.y, e.z, e.w}, oo[4] = {o.x, o.y, o.z, o.w};
-                int dp = 0;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    dp = __dp4a((int)(ww[q] & 0x0F0F0F0Fu), (int)ee[q], dp);
-                    dp = __dp4a((int)((ww[q] >> 4) & 0x0F0F0F0Fu), (int)oo[q], dp);
+                for (int u = 0; u < 4; ++u) {
+                    const int ch = ch0 + 32 * u;
+                    if (ch < chunks) { w[u] = __ldg(wrow + ch); qp[u] = __ldg(qrow + (ch >> cshift)); }
                 }
-                acc[m] = __fmaf_rn((float)(dp - zp * csum[m * (K / 32) + ch]), qp.x, acc[m]);
+            }
+            first = false;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int ch = ch0 + 32 * u;
+                if (ch < chunks) {
+                    const int zp = __float2int_rn(qp[u].y);
+                    const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                    for (int m = 0; m < MB; ++m) {
+                        const uint4 e = even4[m * chunks + ch];
+                        const uint4 o = odd4[m * chunks + ch];
+                        const uint32_t ee[4] = {e.x, e.y, e.z, e.w}, oo[4] = {o.x, o.y, o.z, o.w};
+                        int dp = 0;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            dp = __dp4a((int)(ww[q] & 0x0F0F0F0Fu), (int)ee[q], dp);
+                            dp = __dp4a((int)((ww[q] >> 4) & 0x0F0F0F0Fu), (int)oo[q], dp);
+                        }
+                        acc[m] = __fmaf_rn((float)(dp - zp * csum[m * chunks + ch]), qp[u].x, acc[m]);
+                    }
+                }
             }
         }
 #pragma unroll
@@ -119,68 +164,108 @@ decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qpar
 }
 
 // ---- attention over the cache -----------------------------------------------------------------------------------
-// qkv fp32 [B, 3*d]; cache_k / cache_v fp32 [B][H][max_len][dh] of one layer.  One CTA per (sequence, head): rotates q
-// and k by the angle of `pos`, appends k and v at `pos`, leaves the rotated q in q_out [B, d].
-__global__ void decode_rope_cache_kernel(const float* __restrict__ qkv, int n_heads, int dh, int pos, int max_len,
-                                         const float* __restrict__ cos_t, const float* __restrict__ sin_t,
-                                         float* __restrict__ q_out, float* __restrict__ cache_k, float* __restrict__ cache_v) {
-    const int b = blockIdx.y, h = blockIdx.x, d = n_heads * dh, hd = dh / 2;
-    const float* q = qkv + (size_t)b * 3 * d + h * dh;
-    const float* k = q + d;
-    const float* v = q + 2 * d;
-    float* ck = cache_k + (((size_t)b * n_heads + h) * max_len + pos) * dh;
-    float* cv = cache_v + (((size_t)b * n_heads + h) * max_len + pos) * dh;
-    float* qo = q_out + (size_t)b * d + h * dh;
-    for (int i = threadIdx.x; i < hd; i += blockDim.x) {
-        float c = 1.0f, s = 0.0f;
-        if (cos_t) { c = cos_t[(size_t)pos * hd + i]; s = sin_t[(size_t)pos * hd + i]; }
-        const float q1 = q[i], q2 = q[i + hd], k1 = k[i], k2 = k[i + hd];
-        qo[i] = q1 * c - q2 * s; qo[i + hd] = q2 * c + q1 * s;
-        ck[i] = k1 * c - k2 * s; ck[i + hd] = k2 * c + k1 * s;
-    }
-    for (int i = threadIdx.x; i < dh; i += blockDim.x) cv[i] = v[i];
-}
-
-// out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA (128 threads) per (sequence, head).
-__global__ void __launch_bounds__(128)
-decode_attention_kernel(const float* __restrict__ q_in, const float* __restrict__ cache_k, const float* __restrict__ cache_v,
-                        int n_heads, int dh, int pos, int max_len, float* __restrict__ out) {
-    extern __shared__ float sc[];              // scores of positions 0..pos, then dh floats of q
-    __shared__ float red[4];
-    const int b = blockIdx.y, h = blockIdx.x, d = n_heads * dh;
+// cache_k / cache_v: fp32 [B][H][max_len][dh] of one layer.
+// out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA of 8 warps per (sequence, head).  Warp s takes
+// the cached positions t = s, s + 8, ...: a lane holds 4 (d_head 128) or 2 (d_head 64) features, so one load instruction
+// of the warp reads a whole cached row; scores are reduced by shuffles, the output partial sums of the 8 warps through
+// shared memory.
+// qkv != NULL: the CTA first rotates the new q and k by the angle of `pos` (cos_t / sin_t, or none), appends k and v to
+// the cache at `pos` and uses the rotated q (q_in is then ignored) - the work of decode_rope_cache_kernel, in the same launch.
+template <int DH>
+__global__ void __launch_bounds__(256)
+decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cache_k, float* __restrict__ cache_v,
+                        int n_heads, int pos, int max_len, float* __restrict__ out, const float* __restrict__ qkv,
+                        const float* __restrict__ cos_t, const float* __restrict__ sin_t) {
+    constexpr int VPL = DH / 32;               // features per lane
+    extern __shared__ float sc[];              // scores / probabilities of positions 0..pos, then [8][DH] partial outputs
+    __shared__ float red[8];
+    const int b = blockIdx.y, h = blockIdx.x, d = n_heads * DH;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float* qs = sc + (pos + 1);
-    const float* q = q_in + (size_t)b * d + h * dh;
-    const float* kc = cache_k + ((size_t)b * n_heads + h) * max_len * dh;
-    const float* vc = cache_v + ((size_t)b * n_heads + h) * max_len * dh;
-    for (int i = threadIdx.x; i < dh; i += 128) qs[i] = q[i];
-    __syncthreads();
-    const float scale = 1.0f / sqrtf((float)dh);
-    float mx = -INFINITY;
-    for (int t = warp; t <= pos; t += 4) {                      // a warp per cached position
-        float acc = 0.0f;
-        for (int i = lane; i < dh; i += 32) acc = __fmaf_rn(qs[i], kc[(size_t)t * dh + i], acc);
+    float* part = sc + ((pos + 1 + 3) & ~3);
+    float* kc = cache_k + ((size_t)b * n_heads + h) * max_len * DH;
+    float* vc = cache_v + ((size_t)b * n_heads + h) * max_len * DH;
+    float q[VPL];
+    if (qkv) {
+        float* qs = part;                      // the rotated q passes through the (not yet used) partial-sum area
+        const float* qn = qkv + (size_t)b * 3 * d + h * DH;
+        const float* kn = qn + d;
+        const float* vn = qn + 2 * d;
+        constexpr int HD = DH / 2;
+        for (int i = threadIdx.x; i < HD; i += 256) {
+            float c = 1.0f, s = 0.0f;
+            if (cos_t) { c = cos_t[(size_t)pos * HD + i]; s = sin_t[(size_t)pos * HD + i]; }
+            const float q1 = qn[i], q2 = qn[i + HD], k1 = kn[i], k2 = kn[i + HD];
+            qs[i] = q1 * c - q2 * s; qs[i + HD] = q2 * c + q1 * s;
+            kc[(size_t)pos * DH + i] = k1 * c - k2 * s; kc[(size_t)pos * DH + i + HD] = k2 * c + k1 * s;
+        }
+        for (int i = threadIdx.x; i < DH; i += 256) vc[(size_t)pos * DH + i] = vn[i];
+        __syncthreads();                       // the new cache row and q are visible to the whole CTA
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        acc *= scale;
-        if (lane == 0) sc[t] = acc;
-        mx = fmaxf(mx, acc);
+        for (int j = 0; j < VPL; ++j) q[j] = qs[lane * VPL + j];
+        __syncthreads();
+    } else {
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) q[j] = q_in[(size_t)b * d + h * DH + lane * VPL + j];
+    }
+    const float scale = 1.0f / sqrtf((float)DH);
+    float mx = -INFINITY;
+    for (int t0 = warp; t0 <= pos; t0 += 32) {                 // four positions of this warp in flight
+        float a[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int t = t0 + 8 * u;
+            a[u] = 0.0f;
+            if (t <= pos) {
+#pragma unroll
+                for (int j = 0; j < VPL; ++j) a[u] = __fmaf_rn(q[j], kc[(size_t)t * DH + lane * VPL + j], a[u]);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int t = t0 + 8 * u;
+            if (t <= pos) {
+                a[u] *= scale;
+                if (lane == 0) sc[t] = a[u];
+                mx = fmaxf(mx, a[u]);
+            }
+        }
     }
     if (lane == 0) red[warp] = mx;
     __syncthreads();
-    mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    mx = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
     __syncthreads();
     float sum = 0.0f;
-    for (int t = threadIdx.x; t <= pos; t += 128) { const float p = expf(sc[t] - mx); sc[t] = p; sum += p; }
+    for (int t = threadIdx.x; t <= pos; t += 256) { const float p = expf(sc[t] - mx); sc[t] = p; sum += p; }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     if (lane == 0) red[warp] = sum;
     __syncthreads();
-    const float inv = 1.0f / (red[0] + red[1] + red[2] + red[3]);
-    for (int i = threadIdx.x; i < dh; i += 128) {
-        float acc = 0.0f;
-        for (int t = 0; t <= pos; ++t) acc = __fmaf_rn(sc[t], vc[(size_t)t * dh + i], acc);
-        out[(size_t)b * d + h * dh + i] = acc * inv;
+    float total = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) total += red[i];
+    float acc[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) acc[j] = 0.0f;
+    for (int t = warp; t <= pos; t += 8) {
+        const float p = sc[t];
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p, vc[(size_t)t * DH + lane * VPL + j], acc[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) part[warp * DH + lane * VPL + j] = acc[j];
+    __syncthreads();
+    for (int i = threadIdx.x; i < DH; i += 256) {
+        float o = 0.0f;
+#pragma unroll
+        for (int s8 = 0; s8 < 8; ++s8) o += part[s8 * DH + i];
+        out[(size_t)b * d + h * DH + i] = o / total;
     }
 }
 
@@ -282,13 +367,14 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
     const size_t smem = decode_gemv_smem_bytes(mb, K);
     if (smem > 160 * 1024) return -1;
-    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * 4);
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * 8);
+    const int gshift = group == 32 ? 5 : (group == 64 ? 6 : 7);
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV(MBV)                                                                                                      \
     {                                                                                                                     \
         static bool attr = false;                                                                                         \
         if (!attr) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
-        decode_gemv_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, group, act, row_step, bias, accumulate, out); \
+        decode_gemv_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, row_step, bias, accumulate, out); \
     }
     if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else return -1;
 #undef ZQ_GEMV
@@ -296,18 +382,17 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     return 0;
 }
 
-void launch_decode_rope_cache(const float* qkv, int batch, int n_heads, int dh, int pos, int max_len, const float* cos_t,
-                              const float* sin_t, float* q_out, float* cache_k, float* cache_v, cudaStream_t s) {
-    decode_rope_cache_kernel<<<dim3(n_heads, batch), 64, 0, s>>>(qkv, n_heads, dh, pos, max_len, cos_t, sin_t, q_out, cache_k, cache_v);
-    count_launch();
-}
-
-void launch_decode_attention(const float* q, const float* cache_k, const float* cache_v, int batch, int n_heads, int dh, int pos,
-                             int max_len, float* out, cudaStream_t s) {
-    const size_t smem = (size_t)(pos + 1 + dh) * 4;
+void launch_decode_attention(const float* q, float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos,
+                             int max_len, float* out, const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s) {
+    const size_t smem = (size_t)(((pos + 1 + 3) & ~3) + 8 * dh) * 4;
     static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024); attr = true; }
-    decode_attention_kernel<<<dim3(n_heads, batch), 128, smem, s>>>(q, cache_k, cache_v, n_heads, dh, pos, max_len, out);
+    if (!attr) {
+        cudaFuncSetAttribute(decode_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        cudaFuncSetAttribute(decode_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+        attr = true;
+    }
+    if (dh == 64) decode_attention_kernel<64><<<dim3(n_heads, batch), 256, smem, s>>>(q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
+    else decode_attention_kernel<128><<<dim3(n_heads, batch), 256, smem, s>>>(q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
     count_launch();
 }
 

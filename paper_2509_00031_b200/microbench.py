@@ -9,6 +9,8 @@ between iterations) and prints one JSON line per kernel with its achieved rate.
   python -m paper_2509_00031_b200.microbench --op norm_act --rows 8192 --cols 4096
   python -m paper_2509_00031_b200.microbench --op ffn_act --rows 8192 --cols 11008
   python -m paper_2509_00031_b200.microbench --op head_loss --M 8192 --N 32000 --K 4096
+  python -m paper_2509_00031_b200.microbench --op decode --workload llama7b_w4a8 --batch 1 --context 256 --tokens 64
+      (decode-time inference over the packed model: tokens/s, bytes per token against the HBM copy rate)
 
 It is also the small, self-contained command used for ncu captures of one kernel.
 """
@@ -36,6 +38,79 @@ def timed(fn, iters, flush):
     return ts[len(ts) // 2], ts[0]
 
 
+def decode_bench(a):
+    """Greedy decoding over the packed model of a workload's shape: `context` teacher-forced tokens fill the cache,
+    then `tokens` steps feed each step's choice back (no host synchronisation inside the timed loop)."""
+    import os
+    from . import synth
+    w = dict(synth.WORKLOADS[a.workload])
+    L = w["n_layers"]
+    max_len = a.context + a.tokens
+    w["seq"] = max(w["seq"], max_len)
+    params = synth.make_device_params(w, seed=0)
+    model = zq.ZoqatModel(w, params, max_batch=a.batch, max_seq=w["seq"], first_trainable_layer=L, head_trainable=False,
+                          packed_frozen=True)
+    model.zoqat_prequantize_frozen()
+    for l in range(L):
+        for name in synth.linear_shapes(w):
+            params["layers"][l][name] = None
+    torch.cuda.empty_cache()
+    nbytes = model.zoqat_decode_begin(a.batch, max_len)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1234)
+    ctx = torch.randint(0, w["vocab"], (a.context, a.batch), generator=g, device="cuda", dtype=torch.int32)
+    nxt = torch.zeros(a.batch, dtype=torch.int32, device="cuda")
+    for p in range(a.context):
+        model.zoqat_decode_step(ctx[p], p, next_token=nxt, want_logits=False)
+    model.zoqat_check()
+    launches0 = model.zoqat_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def steps():
+        for t in range(a.tokens):
+            model.zoqat_decode_step(nxt, a.context + t, next_token=nxt, want_logits=False)
+
+    if a.graph:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                steps()
+        torch.cuda.current_stream().wait_stream(side)
+        launches = model.zoqat_launch_count() - launches0
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+    else:
+        torch.cuda.synchronize()
+        e0.record()
+        steps()
+        e1.record()
+        launches = model.zoqat_launch_count() - launches0
+    torch.cuda.synchronize()
+    model.zoqat_check()
+    ms = e0.elapsed_time(e1) / a.tokens
+    d, F, V, H = w["d_model"], w["d_ffn"], w["vocab"], w["n_heads"]
+    per_layer = 4 * d * d + (3 if w["arch"] == "llama" else 2) * d * F
+    weight_bytes = L * per_layer * (0.5 + 8.0 / w["w_group"]) + V * d * 2
+    mean_len = a.context + (a.tokens + 1) / 2
+    cache_bytes = L * 2 * a.batch * d * mean_len * 4
+    peak = 6451.5
+    try:
+        import json as _json
+        peak = _json.load(open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")))["hbm_gbs"]
+    except Exception:
+        pass
+    out = dict(op="decode", workload=a.workload, batch=a.batch, context=a.context, tokens=a.tokens, graph=bool(a.graph),
+               ms_per_step=ms, tokens_per_s=a.batch * 1e3 / ms, launches_per_step=launches / a.tokens,
+               bytes_per_step=weight_bytes + cache_bytes, weight_bytes=weight_bytes, cache_bytes=cache_bytes,
+               achieved_gbs=(weight_bytes + cache_bytes) / ms / 1e6, hbm_peak_gbs=peak,
+               frac_of_hbm=(weight_bytes + cache_bytes) / ms / 1e6 / peak, decode_buffer_bytes=nbytes)
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--op", required=True)
@@ -54,7 +129,13 @@ def main():
     ap.add_argument("--impl", type=int, default=0)
     ap.add_argument("--accumulate", action="store_true")
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--workload", default="llama7b_w4a8")
+    ap.add_argument("--context", type=int, default=256)
+    ap.add_argument("--tokens", type=int, default=64)
+    ap.add_argument("--graph", action="store_true", help="decode: replay the timed steps from one captured CUDA graph")
     a = ap.parse_args()
+    if a.op == "decode":
+        return decode_bench(a)
     zq.lib()
     dev = "cuda"
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -96,6 +177,17 @@ def main():
         med, best = timed(fn, a.iters, flush)
         out.update(rows=a.rows, cols=a.cols, ms=med, ms_best=best, gbs=nbytes / med / 1e6, gbs_best=nbytes / best / 1e6,
                    gweights_per_s=n / med / 1e6)
+    elif a.op == "decode_gemv":
+        W = torch.randn(a.rows, a.cols, device=dev) * 0.02
+        pk, qp = zq.zoqat_op_pack_frozen(W, a.group, a.bits)
+        x = torch.randn(a.batch, a.cols, device=dev)
+        codes, step, _ = zq.zoqat_op_norm_act_operand(x, 0, None, None, 0.0, 8)
+        y = torch.empty((a.batch, a.rows), dtype=torch.float32, device=dev)
+        fn = lambda: zq.zoqat_op_decode_gemv(pk, qp, a.rows, a.cols, a.group, a.bits, codes, step, out=y)
+        med, best = timed(fn, a.iters, flush)
+        nbytes = a.rows * a.cols * (0.5 + 8.0 / a.group)
+        out.update(rows=a.rows, cols=a.cols, batch=a.batch, ms=med, ms_best=best, note="includes the nibble repack of every call",
+                   gbs_weights_only=nbytes / med / 1e6)
     elif a.op == "attention":
         d = a.heads * a.dh
         qkv = torch.randn(a.batch * a.seq, 3 * d, device=dev)

@@ -113,3 +113,33 @@ def make_batch(batch, seq, vocab, seed=1234):
     labels = np.full((batch, seq), -1, np.int32)
     labels[:, :-1] = tokens[:, 1:]
     return tokens, labels
+
+
+def make_device_params(w, seed=0):
+    """Random-init parameters directly on the device (N(0, 0.02^2), bf16-rounded where the workload says so)."""
+    import torch
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    d, f, v = w["d_model"], w["d_ffn"], w["vocab"]
+    opt = w["arch"] == "opt"
+
+    def rnd(*s):
+        t = torch.empty(s, dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=gen)
+        return t.bfloat16().float() if w.get("bf16_init") else t
+
+    ones = lambda n: torch.ones(n, dtype=torch.float32, device="cuda")
+    zeros = lambda n: torch.zeros(n, dtype=torch.float32, device="cuda")
+    p = {"embed": rnd(v, d), "lm_head": rnd(v, d), "final_norm_g": ones(d), "layers": []}
+    if opt:
+        p["final_norm_b"] = zeros(d)
+        p["pos"] = rnd(w["seq"], d)
+    for _ in range(w["n_layers"]):
+        L = {"attn_norm_g": ones(d), "ffn_norm_g": ones(d)}
+        for name, (o, i) in linear_shapes(w).items():
+            L[name] = rnd(o, i)
+        if opt:
+            L["attn_norm_b"] = zeros(d); L["ffn_norm_b"] = zeros(d)
+            for name, n in (("bq", d), ("bk", d), ("bv", d), ("bo", d), ("b_fc1", f), ("b_fc2", d)):
+                L[name] = zeros(n)
+        p["layers"].append(L)
+    return p
