@@ -215,14 +215,15 @@ def run_ours(args, w, rank, world, local_rank):
         if world == 1 and learned:
             model.zoqat_step_rates(tokens, labels, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
         elif world == 1:
-            model.zoqat_step(tokens, labels, 1000 + t, EPS, LR, result)
+            # Eq. (2) of step t rides on the operand producers of step t + 1; the last one is flushed inside the timed region
+            model.zoqat_step_deferred(tokens, labels, 1000 + t, EPS, LR, result)
         else:                                              # data-parallel replicas: 24-byte all-reduce between the halves
             model.zoqat_step_begin(tokens, labels, 1000 + t, EPS, sums)
             dist.all_reduce(sums)
             if learned:
                 model.zoqat_step_finish_rates(sums, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
             else:
-                model.zoqat_step_finish(sums, 1000 + t, EPS, LR, result)
+                model.zoqat_step_finish_deferred(sums, 1000 + t, EPS, LR, result)
 
     def barrier():
         if world > 1:
@@ -244,6 +245,7 @@ def run_ours(args, w, rank, world, local_rank):
     e0.record()
     for t in range(args.steps):
         step(args.warmup + t)
+    model.zoqat_flush_update()
     e1.record()
     barrier()
     ms = e0.elapsed_time(e1)

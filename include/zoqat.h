@@ -202,6 +202,22 @@ int zoqat_step_rates(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
                      int batch, int seq, uint64_t seed, float eps, float lr, float lr_quant, float lr_smooth,
                      zoqat_step_result_t* result_dev, void* stream);
 
+/* zoqat_step with Eq. (2) deferred: the call returns after both passes and g, and the update W <- W - lr g u is
+ * applied by the NEXT zoqat_step_deferred while its operand producers read the masters anyway (one pass over every
+ * trainable tensor per step instead of two), or by zoqat_flush_update().  The masters then lag one update behind the
+ * returned result until that happens; every other entry point that reads or changes them (zoqat_forward_loss,
+ * zoqat_step*, zoqat_apply_update*, zoqat_init_qparams) flushes first, and a caller that reads the master tensors
+ * itself calls zoqat_flush_update() before.  Same arithmetic, same bits as zoqat_step.  Models with Section 4.2
+ * parameters or per-row weight groups run zoqat_step instead (nothing is deferred). */
+int zoqat_step_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                        int batch, int seq, uint64_t seed, float eps, float lr,
+                        zoqat_step_result_t* result_dev, void* stream);
+int zoqat_flush_update(zoqat_model_t* m, void* stream);
+/* The deferred form of zoqat_step_finish for replicas: forms g from the global sums and leaves Eq. (2) to the next
+ * zoqat_step_begin (whose producers apply it) or to zoqat_flush_update(). */
+int zoqat_step_finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                               zoqat_step_result_t* result_dev, void* stream);
+
 /* Eq. (1) with q = n_dirs directions per step (the paper's estimator averages over q directions u_1..u_q; it never
  * states q): direction i uses seed + i, every g_i is the two-point estimate at the SAME weights, and Eq. (2) then
  * applies W <- W - (lr / q) sum_i g_i u_i, direction by direction in one pass over each trainable tensor.

@@ -27,7 +27,7 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
-    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_multi",
+    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_finish_deferred", "zoqat_flush_update", "zoqat_step_multi",
     "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_apply_update", "zoqat_apply_update_rates",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
@@ -96,6 +96,9 @@ def lib():
             "zoqat_forward_loss": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step": [vp, vp, vp, i32, i32, u64, f32, f32, vp, vp],
             "zoqat_step_multi": [vp, vp, vp, i32, i32, u64, i32, f32, f32, vp, vp],
+            "zoqat_step_deferred": [vp, vp, vp, i32, i32, u64, f32, f32, vp, vp],
+            "zoqat_flush_update": [vp, vp],
+            "zoqat_step_finish_deferred": [vp, vp, u64, f32, f32, vp, vp],
             "zoqat_step_host": [vp, vp, vp, i32, i32, u64, f32, f32, P(StepResult), vp],
             "zoqat_step_begin": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step_finish": [vp, vp, u64, f32, f32, vp, vp],
@@ -501,6 +504,21 @@ class ZoqatModel:
         b, s = tokens.shape
         _check(lib().zoqat_step(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, _p(result), _stream()))
         return result
+
+    def zoqat_step_deferred(self, tokens, labels, seed, eps, lr, result=None):
+        """zoqat_step whose update is applied by the next deferred step (or zoqat_flush_update)."""
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        b, s = tokens.shape
+        _check(lib().zoqat_step_deferred(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, _p(result), _stream()))
+        return result
+
+    def zoqat_step_finish_deferred(self, sums, seed, eps, lr, result=None):
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        _check(lib().zoqat_step_finish_deferred(self.handle, _p(sums), seed, eps, lr, _p(result), _stream()))
+        return result
+
+    def zoqat_flush_update(self):
+        _check(lib().zoqat_flush_update(self.handle, _stream()))
 
     def zoqat_step_multi(self, tokens, labels, seed, n_dirs, eps, lr, results=None):
         """results: float32 device tensor [n_dirs, 6] (one zoqat_step_result_t per direction)."""

@@ -87,6 +87,7 @@ struct Workspace {
     size_t qprep_off[8];                // byte offset of each block linear's block inside qprep
     float* bias_pm;                     // smoothed bias per pass: [sign][bias_ld]
     float* class_scales;                // {lr_quant * g, lr_smooth * g}
+    float* pending_scale;               // factor lr * g of a deferred update
     int smooth_ld, bias_ld;
     size_t bop_elems;                   // elements of ONE pass' operand buffer
     size_t total;
@@ -141,6 +142,7 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     w.bias_ld = (int)(3 * d > ffn_cols ? 3 * d : ffn_cols);
     w.bias_pm = (float*)take((size_t)2 * w.bias_ld * 4);
     w.class_scales = (float*)take(2 * 4);
+    w.pending_scale = (float*)take(4);
     w.total = off;
 }
 
@@ -221,6 +223,9 @@ struct zoqat_model {
     int first_trainable_layer = 0;      // n_layers if no block tensor is trainable
     bool any_packed = false, prequantized = false;
     bool any_learnable = false;         // a tensor is ADAPTIVE or a layer has smoothing vectors (Section 4.2)
+    // zoqat_step_deferred: Eq. (2) of the last step still to be applied (by the next step's producers, or by a flush)
+    bool pending = false;
+    uint64_t pending_seed = 0;
     long long launches_at_create = 0;
 };
 
@@ -256,7 +261,7 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
 // NULL).  Adaptive tensors read the parameters forward() prepared for block linear `role`.
 void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t pass_stride, int passes,
                      uint64_t seed, float eps, cudaStream_t s, bool smoothing = false, size_t bias_off = 0,
-                     const float* bias0 = nullptr, int role = 0, int point = 0) {
+                     const float* bias0 = nullptr, int role = 0, int point = 0, const PendingUpdate* pend = nullptr) {
     ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
     const int64_t n = L.rows * L.cols;
     const int bits = L.bits(m->cfg.w_bits);
@@ -286,7 +291,7 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
     }
     const int perturb = L.trainable() && eps != 0.0f;
     if (passes == 2 && perturb) {
-        launch_weight_operand(L.w, n, m->cfg.w_group, bits, 1, seed, L.tid, eps, dst, dst + pass_stride, nullptr, nullptr, nullptr, s);
+        launch_weight_operand(L.w, n, m->cfg.w_group, bits, 1, seed, L.tid, eps, dst, dst + pass_stride, nullptr, nullptr, nullptr, s, pend);
     } else {
         launch_weight_operand(L.w, n, m->cfg.w_group, bits, perturb, seed, L.tid, eps, dst, nullptr, nullptr, nullptr, nullptr, s);
         if (passes == 2) cudaMemcpyAsync(dst + pass_stride, dst, (size_t)n * 2, cudaMemcpyDeviceToDevice, s);
@@ -296,8 +301,9 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
 // The quantised forward.  passes = 1: loss of W + eps*u (eps signed) in loss_sum[0].
 // passes = 2: +eps in loss_sum[0] and -eps in loss_sum[1], evaluated side by side on 2T rows.
 // Layers before the first trainable one see the same weights in both passes and run once.
+// pend: a deferred update that the producers of the trainable tensors apply on the way (passes == 2 only).
 int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int batch, int seq, uint64_t seed,
-            float eps, int passes, cudaStream_t s) {
+            float eps, int passes, cudaStream_t s, const PendingUpdate* pend = nullptr) {
     const zoqat_config_t& c = m->cfg;
     Workspace& w = m->ws;
     const int64_t T = (int64_t)batch * seq;
@@ -358,7 +364,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                   c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(0)); }
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
             produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
-                            Ly.vec[ZOQAT_ROLE_BQ + r], r, 0);
+                            Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend);
         GemmArgs g{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
@@ -382,7 +388,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
               return fail(rc, "attention launch rejected");
           } }
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1)); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
@@ -393,8 +399,8 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
                                   c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(2)); }
         const int n_up = llama ? 2 * F : F;
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2);
-        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend);
+        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
@@ -412,7 +418,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(3));
           else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
           else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3)); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
@@ -425,7 +431,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     }
     // --- final norm, vocabulary projection fused with the cross-entropy
     { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.h, Z * T, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s); }
-    produce_operand(m, m->head, w.bop, ps, Z, seed, eps, s);
+    produce_operand(m, m->head, w.bop, ps, Z, seed, eps, s, false, 0, nullptr, 0, 0, pend);
     GemmArgs g{};
     g.A = w.xa; g.B = w.bop; g.M = T; g.N = c.vocab; g.K = d; g.Z = Z; g.b_stride = ps;
     g.mode = 1; g.labels = labels; g.partials = w.ce_partials; g.label_logit = w.label_logit;
@@ -482,6 +488,13 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
     }
     if (m->head.trainable())
         launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
+}
+
+// Applies a deferred update now (every entry point that reads or changes the masters starts with this).
+void flush_pending(zoqat_model* m, cudaStream_t s) {
+    if (!m->pending) return;
+    update_all(m, m->pending_seed, m->ws.pending_scale, 0.0f, s);
+    m->pending = false;
 }
 
 }  // namespace
@@ -686,6 +699,7 @@ int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream) {
 int zoqat_init_qparams(zoqat_model_t* m, void* stream) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);
     for (auto& Ly : m->layers)
         for (int r = 0; r < 7; ++r) {
             Linear& L = Ly.lin[r];
@@ -702,6 +716,7 @@ int zoqat_forward_loss(zoqat_model_t* m, const int32_t* tokens_dev, const int32_
     if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
     if (!loss_out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "loss_out_dev is NULL");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);
     if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, signed_eps, 1, s)) return rc;
     launch_store_loss(m->ws.loss_sum, m->ws.count, loss_out_dev, s);
     CUDA_TRY(cudaGetLastError());
@@ -714,7 +729,10 @@ int zoqat_step_begin(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
     if (!sums_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev is NULL");
     if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, eps, 2, s)) return rc;
+    // a deferred update rides on this forward's producers (same bits as applying it first)
+    PendingUpdate pend{m->pending_seed, m->ws.pending_scale};
+    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, eps, 2, s, m->pending ? &pend : nullptr)) return rc;
+    m->pending = false;
     launch_pack_sums(m->ws.loss_sum, m->ws.count, sums_dev, s);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
@@ -769,6 +787,41 @@ int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* label
     return zoqat_step_finish(m, m->ws.sums, seed, eps, lr, result_dev, stream);
 }
 
+int zoqat_step_finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                               zoqat_step_result_t* result_dev, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (!sums_dev || !result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev/result_dev are NULL");
+    if (m->any_learnable || m->cfg.w_group == 0) return zoqat_step_finish(m, sums_dev, seed, eps, lr, result_dev, stream);
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);            // nothing is pending after a step_begin; kept for callers that skip it
+    zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(result_dev);
+    launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, res, s);
+    CUDA_TRY(cudaMemcpyAsync(m->ws.pending_scale, &res->update_scale, 4, cudaMemcpyDeviceToDevice, s));
+    m->pending = true;
+    m->pending_seed = seed;
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_flush_update(zoqat_model_t* m, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    flush_pending(m, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                        uint64_t seed, float eps, float lr, zoqat_step_result_t* result_dev, void* stream) {
+    if (!result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "result_dev is NULL");
+    if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    // the producers that can carry an update are those of the plain per-group min/max path
+    if (m->any_learnable || m->cfg.w_group == 0) return zoqat_step(m, tokens_dev, labels_dev, batch, seq, seed, eps, lr, result_dev, stream);
+    if (int rc = zoqat_step_begin(m, tokens_dev, labels_dev, batch, seq, seed, eps, m->ws.sums, stream)) return rc;
+    return zoqat_step_finish_deferred(m, m->ws.sums, seed, eps, lr, result_dev, stream);
+}
+
 int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
                      uint64_t seed, int n_dirs, float eps, float lr, zoqat_step_result_t* results_dev, void* stream) {
     if (!results_dev) return fail(ZOQAT_ERR_INVALID_ARG, "results_dev is NULL");
@@ -776,6 +829,7 @@ int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
     if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
     if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);
     const float lr_q = lr / (float)n_dirs;                        // binary32 division, as in Eq. (1)'s 1/q
     zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(results_dev);
     // every direction is evaluated at the same W ...
@@ -833,6 +887,7 @@ int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t*
 
 int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float scale_quant, float scale_smooth, void* stream) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    flush_pending(m, static_cast<cudaStream_t>(stream));
     update_all(m, seed, nullptr, scale, static_cast<cudaStream_t>(stream), nullptr, scale_quant, scale_smooth);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;

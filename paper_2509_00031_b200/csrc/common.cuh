@@ -27,10 +27,13 @@ void launch_normal(uint64_t seed, uint32_t tid, uint64_t n, float* out, cudaStre
 // perturb = 0 skips the direction entirely (frozen tensors).
 // op_plus from W + eps*u; op_minus (may be NULL) from W - eps*u.
 // Debug outputs (may be NULL) describe the op_plus side.
+// pend (with op_minus only): the previous step's update, w <- fma(-*scale, u(pend->seed), w), is applied to the master
+// (which is then written, hence not really const) before this step's perturbation.
+struct PendingUpdate { uint64_t seed; const float* scale; };
 void launch_weight_operand(const float* w, int64_t n, int group, int bits, int perturb,
                            uint64_t seed, uint32_t tid, float eps,
                            __nv_bfloat16* op_plus, __nv_bfloat16* op_minus,
-                           uint8_t* codes, float* step, int32_t* zp, cudaStream_t s);
+                           uint8_t* codes, float* step, int32_t* zp, cudaStream_t s, const PendingUpdate* pend = nullptr);
 // Producer with the learnable parts of Section 4.2.  theta != NULL: per-group (step, z, alpha, beta) replace min/max
 // (perturbed with tensor id tid_q).  smooth != NULL: [sign][kind][smooth_ld] perturbed smoothing vectors (kind 0
 // scale, 1 shift, 2 reciprocal scale); the quantiser sees scale (.) w' and bias_out[sign * bias_out_stride + row] =

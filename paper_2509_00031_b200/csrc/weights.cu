@@ -184,15 +184,20 @@ __device__ __forceinline__ void store_bf16x16(uint2* dst, int64_t i, const float
 // adjacent lanes: the group parameters are computed once per 16 elements and the min/max reduction takes
 // log2(GROUP/16) shuffle steps.  GROUP in {32, 64, 128}; bits in {0 (no quantiser), 2, 3, 4}; DUAL writes the
 // -eps operand too.
-template <int GROUP, bool DUAL, bool DEBUG>
+// UPD: the update of the previous step (Eq. (2) with that step's seed (uk0, uk1) and factor *upd_scale) is applied to the
+// master on the way in - w <- fma(-c, u_prev, w), written back to w_out - before this step's perturbation, so a
+// deferred update costs no pass of its own over the tensor.
+template <int GROUP, bool DUAL, bool DEBUG, bool UPD>
 __global__ void __launch_bounds__(kThreads)
 weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int perturb,
                       uint32_t k0, uint32_t k1, uint32_t tid, float eps,
                       uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
-                      uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp) {
+                      uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp,
+                      float4* __restrict__ w_out, const float* __restrict__ upd_scale, uint32_t uk0, uint32_t uk1) {
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
-    if (perturb) stage_icdf_table(tab);
+    if (perturb || UPD) stage_icdf_table(tab);
+    const float upd_c = UPD ? -(*upd_scale) : 0.0f;
     const float qp = (float)((1 << bits) - 1);
     // whole warps iterate together so that the shuffles always see 32 lanes
     const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
@@ -201,8 +206,17 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         float x[16], xm[16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float4 v = live ? __ldg(w + chunk_of<LANES>(i, k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 v = live ? (UPD ? w[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+        }
+        if (UPD) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 z = direction4(tab, uk0, uk1, tid, (uint64_t)chunk_of<LANES>(i, k));
+                x[4 * k] = __fmaf_rn(upd_c, z.x, x[4 * k]); x[4 * k + 1] = __fmaf_rn(upd_c, z.y, x[4 * k + 1]);
+                x[4 * k + 2] = __fmaf_rn(upd_c, z.z, x[4 * k + 2]); x[4 * k + 3] = __fmaf_rn(upd_c, z.w, x[4 * k + 3]);
+                if (live) w_out[chunk_of<LANES>(i, k)] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+            }
         }
         if (perturb) {
 #pragma unroll
@@ -758,7 +772,7 @@ void launch_normal(uint64_t seed, uint32_t tid, uint64_t n, float* out, cudaStre
 template <int GROUP>
 static void weight_operand_dispatch(const float* w, int64_t n, int bits, int perturb, uint64_t seed, uint32_t tid,
                                     float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes,
-                                    float* step, int32_t* zp, cudaStream_t s) {
+                                    float* step, int32_t* zp, cudaStream_t s, const PendingUpdate* pend) {
     const int64_t n16 = n / 16;
     const int grid = stream_grid(n16, kThreads);
     const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
@@ -767,23 +781,27 @@ static void weight_operand_dispatch(const float* w, int64_t n, int bits, int per
     uint2* m = reinterpret_cast<uint2*>(op_minus);
     uchar4* c4 = reinterpret_cast<uchar4*>(codes);
     const bool debug = codes || step || zp;
-    if (op_minus) {
-        weight_operand_kernel<GROUP, true, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr);
+    if (op_minus && pend) {
+        weight_operand_kernel<GROUP, true, false, true><<<grid, kThreads, 0, s>>>(
+            w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr, reinterpret_cast<float4*>(const_cast<float*>(w)),
+            pend->scale, (uint32_t)pend->seed, (uint32_t)(pend->seed >> 32));
+    } else if (op_minus) {
+        weight_operand_kernel<GROUP, true, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr, nullptr, nullptr, 0u, 0u);
     } else if (debug) {
-        weight_operand_kernel<GROUP, false, true><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp);
+        weight_operand_kernel<GROUP, false, true, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp, nullptr, nullptr, 0u, 0u);
     } else {
-        weight_operand_kernel<GROUP, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr);
+        weight_operand_kernel<GROUP, false, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0u, 0u);
     }
     count_launch();
 }
 
 void launch_weight_operand(const float* w, int64_t n, int group, int bits, int perturb, uint64_t seed, uint32_t tid,
                            float eps, __nv_bfloat16* op_plus, __nv_bfloat16* op_minus, uint8_t* codes, float* step,
-                           int32_t* zp, cudaStream_t s) {
-    if (n == 0 || (perturb && !ensure_icdf_table())) return;
-    if (group == 32) weight_operand_dispatch<32>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
-    else if (group == 64) weight_operand_dispatch<64>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
-    else weight_operand_dispatch<128>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s);
+                           int32_t* zp, cudaStream_t s, const PendingUpdate* pend) {
+    if (n == 0 || ((perturb || pend) && !ensure_icdf_table())) return;
+    if (group == 32) weight_operand_dispatch<32>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s, pend);
+    else if (group == 64) weight_operand_dispatch<64>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s, pend);
+    else weight_operand_dispatch<128>(w, n, bits, perturb, seed, tid, eps, op_plus, op_minus, codes, step, zp, s, pend);
 }
 
 template <int GROUP, bool ADAPT, bool SMOOTH>

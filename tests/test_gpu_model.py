@@ -376,3 +376,47 @@ def test_query_value_only_selection(zq):
             else:
                 assert np.array_equal(got, params["layers"][l][n])
     assert np.array_equal(model.params["lm_head"].cpu().numpy(), params["lm_head"])
+
+
+@pytest.mark.parametrize("shape,batch,seq,first", [(SMALL_LLAMA, 2, 96, 0), (SMALL_OPT, 3, 50, 1)], ids=["llama_w4a8", "opt_w4_last_layer"])
+def test_deferred_update_gives_the_same_bits(zq, shape, batch, seq, first):
+    """zoqat_step_deferred applies Eq. (2) inside the next step's operand producers: results and masters are bit for
+    bit those of zoqat_step, and entry points that read the masters flush the pending update first."""
+    params = synth.make_params(shape, seed=2, max_seq=seq, jitter=True)
+    eager = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, first_trainable_layer=first)
+    lazy = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, first_trainable_layer=first)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=15)
+    t, l = dev(tokens), dev(labels)
+    for step in range(4):
+        a = eager.zoqat_step(t, l, 300 + step, 1e-3, 1e-3).cpu()
+        b = lazy.zoqat_step_deferred(t, l, 300 + step, 1e-3, 1e-3).cpu()
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32)), step
+    # the last update is still pending: the masters lag one step behind ...
+    name = "wq" if shape["arch"] == "llama" else "fc1"
+    last = shape["n_layers"] - 1
+    assert not torch.equal(eager.params["layers"][last][name], lazy.params["layers"][last][name])
+    # ... until something reads them through the library
+    la = eager.zoqat_forward_loss(t, l, 1, 0.0)
+    lb = lazy.zoqat_forward_loss(t, l, 1, 0.0)
+    lazy.zoqat_check()
+    assert torch.equal(la, lb)
+    for li in range(shape["n_layers"]):
+        for k, v in eager.params["layers"][li].items():
+            assert torch.equal(v, lazy.params["layers"][li][k]), (li, k)
+    assert torch.equal(eager.params["lm_head"], lazy.params["lm_head"])
+    # the two halves used by replicas, deferred; a plain zoqat_step afterwards carries the pending update along
+    sums = lazy.zoqat_step_begin(t, l, 350, 1e-3)
+    b = lazy.zoqat_step_finish_deferred(sums, 350, 1e-3, 1e-3).cpu()
+    a = eager.zoqat_step(t, l, 350, 1e-3, 1e-3).cpu()
+    assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    a = eager.zoqat_step(t, l, 351, 1e-3, 1e-3).cpu()
+    b = lazy.zoqat_step(t, l, 351, 1e-3, 1e-3).cpu()
+    assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    assert torch.equal(eager.params["layers"][last][name], lazy.params["layers"][last][name])
+    # explicit flush, and a flush with nothing pending changes nothing
+    lazy.zoqat_step_deferred(t, l, 400, 1e-3, 1e-3)
+    eager.zoqat_step(t, l, 400, 1e-3, 1e-3)
+    lazy.zoqat_flush_update()
+    lazy.zoqat_flush_update()
+    assert torch.equal(eager.params["layers"][last][name], lazy.params["layers"][last][name])
+    assert torch.equal(eager.params["lm_head"], lazy.params["lm_head"])
