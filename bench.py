@@ -27,7 +27,7 @@ LR_QUANT, LR_SMOOTH = 1e-5, 5e-6      # rates of the Section 4.2 parameter class
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, averaged over the 129 GEMM
 # launches of one step, from the committed ncu capture (profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by
 # workload; absent for workloads that have not been captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 854.7e6}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 842.7e6}
 
 
 def load_peaks():
