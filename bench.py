@@ -261,7 +261,8 @@ def run_ours(args, w, rank, world, local_rank):
         barrier()
         t0 = time.perf_counter()
         for t in range(args.steps):
-            model.zoqat_step_host(tok_host, lab_host, 5000 + t, EPS, LR)
+            model.zoqat_step_host(tok_host, lab_host, 5000 + t, EPS, LR, deferred=not learned)
+        model.zoqat_flush_update()
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3
     if world > 1:

@@ -248,6 +248,12 @@ int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t*
                     int batch, int seq, uint64_t seed, float eps, float lr,
                     zoqat_step_result_t* result_host, void* stream);
 
+/* zoqat_step_host around zoqat_step_deferred: the result is back on the host when the call returns, the update of
+ * the masters rides on the next step (or zoqat_flush_update()). */
+int zoqat_step_host_deferred(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host,
+                             int batch, int seq, uint64_t seed, float eps, float lr,
+                             zoqat_step_result_t* result_host, void* stream);
+
 /* Eq. (2) alone: W <- W - scale * u(seed) on every TRAINABLE tensor (and on the Section 4.2 parameters);
  * the _rates form takes one factor per parameter class. */
 int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream);

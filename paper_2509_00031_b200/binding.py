@@ -28,7 +28,7 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
     "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_finish_deferred", "zoqat_flush_update", "zoqat_step_multi",
-    "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_apply_update", "zoqat_apply_update_rates",
+    "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
@@ -100,6 +100,7 @@ def lib():
             "zoqat_flush_update": [vp, vp],
             "zoqat_step_finish_deferred": [vp, vp, u64, f32, f32, vp, vp],
             "zoqat_step_host": [vp, vp, vp, i32, i32, u64, f32, f32, P(StepResult), vp],
+            "zoqat_step_host_deferred": [vp, vp, vp, i32, i32, u64, f32, f32, P(StepResult), vp],
             "zoqat_step_begin": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step_finish": [vp, vp, u64, f32, f32, vp, vp],
             "zoqat_apply_update": [vp, u64, f32, vp],
@@ -539,12 +540,13 @@ class ZoqatModel:
         _check(lib().zoqat_step_finish(self.handle, _p(sums), seed, eps, lr, _p(result), _stream()))
         return result
 
-    def zoqat_step_host(self, tokens_host, labels_host, seed, eps, lr):
-        """tokens_host / labels_host: pinned (or pageable) CPU int32 tensors [batch, seq]."""
+    def zoqat_step_host(self, tokens_host, labels_host, seed, eps, lr, deferred=False):
+        """tokens_host / labels_host: pinned (or pageable) CPU int32 tensors [batch, seq].  deferred: the update of the
+        masters rides on the next step (zoqat_step_host_deferred)."""
         res = StepResult()
         b, s = tokens_host.shape
-        _check(lib().zoqat_step_host(self.handle, _p(tokens_host), _p(labels_host), b, s, seed, eps, lr,
-                                     ctypes.byref(res), _stream()))
+        fn = lib().zoqat_step_host_deferred if deferred else lib().zoqat_step_host
+        _check(fn(self.handle, _p(tokens_host), _p(labels_host), b, s, seed, eps, lr, ctypes.byref(res), _stream()))
         return res
 
     def zoqat_apply_update(self, seed, scale):

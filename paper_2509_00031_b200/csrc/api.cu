@@ -868,21 +868,32 @@ int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
     return ZOQAT_OK;
 }
 
-int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
-                    uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream) {
+static int step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
+                     uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream, bool deferred) {
     if (int rc = check_call(m, tokens_host, labels_host, batch, seq)) return rc;
     if (!result_host) return fail(ZOQAT_ERR_INVALID_ARG, "result_host is NULL");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t nb = (size_t)batch * seq * 4;
     CUDA_TRY(cudaMemcpyAsync(m->ws.tokens, tokens_host, nb, cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaMemcpyAsync(m->ws.labels, labels_host, nb, cudaMemcpyHostToDevice, s));
-    if (int rc = zoqat_step(m, m->ws.tokens, m->ws.labels, batch, seq, seed, eps, lr,
-                            reinterpret_cast<zoqat_step_result_t*>(m->ws.result), s))
+    zoqat_step_result_t* res = reinterpret_cast<zoqat_step_result_t*>(m->ws.result);
+    if (int rc = deferred ? zoqat_step_deferred(m, m->ws.tokens, m->ws.labels, batch, seq, seed, eps, lr, res, s)
+                          : zoqat_step(m, m->ws.tokens, m->ws.labels, batch, seq, seed, eps, lr, res, s))
         return rc;
     CUDA_TRY(cudaMemcpyAsync(result_host, m->ws.result, sizeof(zoqat_step_result_t), cudaMemcpyDeviceToHost, s));
     CUDA_TRY(cudaStreamSynchronize(s));
     if (result_host->status != 0) return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", result_host->status);
     return ZOQAT_OK;
+}
+
+int zoqat_step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
+                    uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream) {
+    return step_host(m, tokens_host, labels_host, batch, seq, seed, eps, lr, result_host, stream, false);
+}
+
+int zoqat_step_host_deferred(zoqat_model_t* m, const int32_t* tokens_host, const int32_t* labels_host, int batch, int seq,
+                             uint64_t seed, float eps, float lr, zoqat_step_result_t* result_host, void* stream) {
+    return step_host(m, tokens_host, labels_host, batch, seq, seed, eps, lr, result_host, stream, true);
 }
 
 int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float scale_quant, float scale_smooth, void* stream) {

@@ -413,6 +413,10 @@ def test_deferred_update_gives_the_same_bits(zq, shape, batch, seq, first):
     b = lazy.zoqat_step(t, l, 351, 1e-3, 1e-3).cpu()
     assert torch.equal(a.view(torch.int32), b.view(torch.int32))
     assert torch.equal(eager.params["layers"][last][name], lazy.params["layers"][last][name])
+    # host-buffer entry point, deferred
+    ra = eager.zoqat_step_host(torch.from_numpy(tokens), torch.from_numpy(labels), 352, 1e-3, 1e-3)
+    rb = lazy.zoqat_step_host(torch.from_numpy(tokens), torch.from_numpy(labels), 352, 1e-3, 1e-3, deferred=True)
+    assert (ra.loss_plus, ra.loss_minus, ra.proj_grad, ra.update_scale) == (rb.loss_plus, rb.loss_minus, rb.proj_grad, rb.update_scale)
     # explicit flush, and a flush with nothing pending changes nothing
     lazy.zoqat_step_deferred(t, l, 400, 1e-3, 1e-3)
     eager.zoqat_step(t, l, 400, 1e-3, 1e-3)
