@@ -64,3 +64,21 @@ def test_missing_library_is_loud(zq, monkeypatch):
     monkeypatch.setattr(zq, "LIB_PATH", "/nonexistent/libzoqat.so")
     with pytest.raises(ImportError):
         zq.lib()
+
+
+def test_null_handles_and_new_config_values_are_rejected_on_the_host(zq):
+    L = zq.lib()
+    n = ctypes.c_size_t()
+    assert L.zoqat_flush_update(None, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_decode_bytes(None, 1, 16, ctypes.byref(n)) == zq.ERR_INVALID_ARG
+    assert L.zoqat_decode_step(None, None, 0, None, None, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_init_qparams(None, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_step_deferred(None, None, None, 1, 1, 0, 1e-3, 1e-3, None, None) == zq.ERR_INVALID_ARG
+    # one weight group per output row needs row lengths that are multiples of 128; weight bit widths 2..8
+    cfg = zq.Config(arch=zq.ARCH_LLAMA, n_layers=1, d_model=192, n_heads=3, d_ffn=384, vocab=64, max_batch=1,
+                    max_seq=32, w_bits=6, w_group=0, a_bits=6, gemm_impl=0, norm_eps=1e-5, rope_base=10000.0)
+    assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.ERR_UNSUPPORTED
+    cfg.d_model, cfg.n_heads = 256, 4
+    assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.OK
+    cfg.w_bits = 1
+    assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.ERR_UNSUPPORTED
