@@ -366,3 +366,37 @@ def test_create_rejects_inconsistent_learnables(zq):
     params2["layers"][0]["smooth_s_attn_in"] = torch.ones(shape["d_model"], device="cuda")
     with pytest.raises(zq.ZoqatError):
         zq.ZoqatModel(shape, params2, max_batch=1, max_seq=32)
+
+
+def test_step_multi_and_replica_halves_with_learnables(zq):
+    """q directions per step, and the begin / finish halves used by replicas, on a model with Section 4.2 parameters."""
+    shape, batch, seq = SMALL_LLAMA, 2, 64
+    model, oracle = build_pair(zq, shape, batch, seq, 0, True, True)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=16)
+    keys = learnable_keys(oracle)
+    ids = {id(a): (tid, cls) for a, tid, cls in oracle.trainable_tensors()}
+    # q = 3: every g_i at the same parameters, then the updates in order with the factor fl(fl(lr / q) * g_i) for every class
+    before = {(l, k): oracle.p["layers"][l][k].copy() for l, k in keys}
+    res = model.zoqat_step_multi(dev(tokens), dev(labels), 500, 3, 1e-3, 3e-4).cpu().numpy()
+    model.zoqat_check()
+    want = oracle.step_multi(tokens, labels, 500, 3, 1e-3, 3e-4)
+    lr_q = np.float32(np.float32(3e-4) / np.float32(3))
+    for i, (lp, lm, g) in enumerate(want):
+        assert abs(res[i, 0] - lp) <= 1e-3 * abs(lp) and abs(res[i, 1] - lm) <= 1e-3 * abs(lm)
+    for (l, k), wb in before.items():
+        tid, _ = ids[id(oracle.p["layers"][l][k])]
+        cur = wb.copy().reshape(-1)
+        for i in range(3):
+            core.update_(cur, 500 + i, tid, np.float32(lr_q * np.float32(res[i, 2])))
+        assert np.array_equal(model.params["layers"][l][k].cpu().numpy().reshape(-1).view(np.uint32), cur.view(np.uint32)), (l, k)
+    # begin + finish_rates == step_rates (same seed, same data) on a second, identical model
+    twin, _ = build_pair(zq, shape, batch, seq, 0, True, True)
+    for l, k in keys:
+        twin.params["layers"][l][k].copy_(model.params["layers"][l][k])
+    twin.params["lm_head"].copy_(model.params["lm_head"])
+    a = model.zoqat_step_rates(dev(tokens), dev(labels), 600, 1e-3, 1e-4, 2e-4, 3e-4).cpu()
+    sums = twin.zoqat_step_begin(dev(tokens), dev(labels), 600, 1e-3)
+    b = twin.zoqat_step_finish_rates(sums, 600, 1e-3, 1e-4, 2e-4, 3e-4).cpu()
+    assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+    for l, k in keys:
+        assert torch.equal(model.params["layers"][l][k], twin.params["layers"][l][k]), (l, k)
