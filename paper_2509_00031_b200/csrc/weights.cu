@@ -190,10 +190,10 @@ __device__ __forceinline__ void store_bf16x16(uint2* dst, int64_t i, const float
 template <int GROUP, bool DUAL, bool DEBUG, bool UPD>
 __global__ void __launch_bounds__(kThreads)
 weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int perturb,
-                      uint32_t k0, uint32_t k1, uint32_t tid, float eps,
+                      const PhiloxKeys rk, uint32_t tid, float eps,
                       uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
                       uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp,
-                      float4* __restrict__ w_out, const float* __restrict__ upd_scale, uint32_t uk0, uint32_t uk1) {
+                      float4* __restrict__ w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk) {
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
     if (perturb || UPD) stage_icdf_table(tab);
@@ -212,7 +212,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         if (UPD) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(tab, uk0, uk1, tid, (uint64_t)chunk_of<LANES>(i, k));
+                const float4 z = direction4(tab, urk, tid, (uint64_t)chunk_of<LANES>(i, k));
                 x[4 * k] = __fmaf_rn(upd_c, z.x, x[4 * k]); x[4 * k + 1] = __fmaf_rn(upd_c, z.y, x[4 * k + 1]);
                 x[4 * k + 2] = __fmaf_rn(upd_c, z.z, x[4 * k + 2]); x[4 * k + 3] = __fmaf_rn(upd_c, z.w, x[4 * k + 3]);
                 if (live) w_out[chunk_of<LANES>(i, k)] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
@@ -221,7 +221,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         if (perturb) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk_of<LANES>(i, k));
+                const float4 z = direction4(tab, rk, tid, (uint64_t)chunk_of<LANES>(i, k));
                 const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -408,7 +408,7 @@ row_prepare_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, 
 template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH>
 __global__ void __launch_bounds__(kThreads, 3)
 weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols4, int bits, int perturb,
-                              uint32_t k0, uint32_t k1, uint32_t tid, float eps,
+                              const PhiloxKeys rk, uint32_t tid, float eps,
                               uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
                               const float4* __restrict__ prep_a, const float4* __restrict__ prep_b,
                               const float* __restrict__ smooth, int smooth_ld,
@@ -432,7 +432,7 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
         if (perturb) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk_of<LANES>(i, k));
+                const float4 z = direction4(tab, rk, tid, (uint64_t)chunk_of<LANES>(i, k));
                 const float zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -683,7 +683,7 @@ unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restr
 
 // Eq. (2): w <- w - scale*u, one fused multiply-add per element.
 __global__ void __launch_bounds__(kThreads)
-update_kernel(float* __restrict__ w, uint64_t n, uint32_t k0, uint32_t k1, uint32_t tid,
+update_kernel(float* __restrict__ w, uint64_t n, const PhiloxKeys rk, uint32_t tid,
               const float* __restrict__ scale_ptr, float scale_val) {
     __shared__ float2 tab[kIcdfKnots];
     stage_icdf_table(tab);
@@ -699,14 +699,14 @@ update_kernel(float* __restrict__ w, uint64_t n, uint32_t k0, uint32_t k1, uint3
         for (int u = 0; u < 4; ++u) x[u] = w4[b + u * stride];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float4 z = direction4(tab, k0, k1, tid, b + u * stride);
+            const float4 z = direction4(tab, rk, tid, b + u * stride);
             x[u].x = __fmaf_rn(c, z.x, x[u].x); x[u].y = __fmaf_rn(c, z.y, x[u].y);
             x[u].z = __fmaf_rn(c, z.z, x[u].z); x[u].w = __fmaf_rn(c, z.w, x[u].w);
             w4[b + u * stride] = x[u];
         }
     }
     for (; b < nblk; b += stride) {
-        const float4 z = direction4(tab, k0, k1, tid, b);
+        const float4 z = direction4(tab, rk, tid, b);
         if (4 * b + 4 <= n) {
             float4 x = w4[b];
             x.x = __fmaf_rn(c, z.x, x.x); x.y = __fmaf_rn(c, z.y, x.y);
@@ -775,7 +775,7 @@ static void weight_operand_dispatch(const float* w, int64_t n, int bits, int per
                                     float* step, int32_t* zp, cudaStream_t s, const PendingUpdate* pend) {
     const int64_t n16 = n / 16;
     const int grid = stream_grid(n16, kThreads);
-    const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    const PhiloxKeys rk = philox_keys(seed);
     const float4* w4 = reinterpret_cast<const float4*>(w);
     uint2* p = reinterpret_cast<uint2*>(op_plus);
     uint2* m = reinterpret_cast<uint2*>(op_minus);
@@ -783,14 +783,14 @@ static void weight_operand_dispatch(const float* w, int64_t n, int bits, int per
     const bool debug = codes || step || zp;
     if (op_minus && pend) {
         weight_operand_kernel<GROUP, true, false, true><<<grid, kThreads, 0, s>>>(
-            w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr, reinterpret_cast<float4*>(const_cast<float*>(w)),
-            pend->scale, (uint32_t)pend->seed, (uint32_t)(pend->seed >> 32));
+            w4, n16, bits, perturb, rk, tid, eps, p, m, nullptr, nullptr, nullptr, reinterpret_cast<float4*>(const_cast<float*>(w)),
+            pend->scale, philox_keys(pend->seed));
     } else if (op_minus) {
-        weight_operand_kernel<GROUP, true, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, m, nullptr, nullptr, nullptr, nullptr, nullptr, 0u, 0u);
+        weight_operand_kernel<GROUP, true, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, rk, tid, eps, p, m, nullptr, nullptr, nullptr, nullptr, nullptr, rk);
     } else if (debug) {
-        weight_operand_kernel<GROUP, false, true, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, c4, step, zp, nullptr, nullptr, 0u, 0u);
+        weight_operand_kernel<GROUP, false, true, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, rk, tid, eps, p, nullptr, c4, step, zp, nullptr, nullptr, rk);
     } else {
-        weight_operand_kernel<GROUP, false, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, k0, k1, tid, eps, p, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0u, 0u);
+        weight_operand_kernel<GROUP, false, false, false><<<grid, kThreads, 0, s>>>(w4, n16, bits, perturb, rk, tid, eps, p, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, rk);
     }
     count_launch();
 }
@@ -833,11 +833,11 @@ static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
     const int qgi = a.per_channel ? (int)(a.cols / 16) : 0;
     if (a.op_minus)
         weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, philox_keys(a.seed), a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
             a.bias_part, n_groups, c4, qgi);
     else
         weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, philox_keys(a.seed), a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
             a.bias_part, n_groups, c4, qgi);
     count_launch();
     if (SMOOTH) {
@@ -944,8 +944,7 @@ void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_
 
 void launch_update(float* w, uint64_t n, uint64_t seed, uint32_t tid, const float* scale_ptr, float scale_val, cudaStream_t s) {
     if (n == 0 || !ensure_icdf_table()) return;
-    update_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(
-        w, n, (uint32_t)seed, (uint32_t)(seed >> 32), tid, scale_ptr, scale_val);
+    update_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(w, n, philox_keys(seed), tid, scale_ptr, scale_val);
     count_launch();
 }
 
