@@ -209,10 +209,10 @@ decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cach
     }
     const float scale = 1.0f / sqrtf((float)DH);
     float mx = -INFINITY;
-    for (int t0 = warp; t0 <= pos; t0 += 32) {                 // four positions of this warp in flight
-        float a[4];
+    for (int t0 = warp; t0 <= pos; t0 += 64) {                 // eight positions of this warp in flight
+        float a[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const int t = t0 + 8 * u;
             a[u] = 0.0f;
             if (t <= pos) {
@@ -223,10 +223,10 @@ decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cach
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
+            for (int u = 0; u < 8; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
             const int t = t0 + 8 * u;
             if (t <= pos) {
                 a[u] *= scale;
@@ -253,10 +253,25 @@ decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cach
     float acc[VPL];
 #pragma unroll
     for (int j = 0; j < VPL; ++j) acc[j] = 0.0f;
-    for (int t = warp; t <= pos; t += 8) {
-        const float p = sc[t];
+    for (int t0 = warp; t0 <= pos; t0 += 64) {                 // eight cached rows of this warp in flight
+        float v[8][VPL], p[8];
 #pragma unroll
-        for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p, vc[(size_t)t * DH + lane * VPL + j], acc[j]);
+        for (int u = 0; u < 8; ++u) {
+            const int t = t0 + 8 * u;
+            p[u] = 0.0f;
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) v[u][j] = 0.0f;
+            if (t <= pos) {
+                p[u] = sc[t];
+#pragma unroll
+                for (int j = 0; j < VPL; ++j) v[u][j] = vc[(size_t)t * DH + lane * VPL + j];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p[u], v[u][j], acc[j]);
+        }
     }
 #pragma unroll
     for (int j = 0; j < VPL; ++j) part[warp * DH + lane * VPL + j] = acc[j];

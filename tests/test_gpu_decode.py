@@ -58,7 +58,7 @@ SHAPES = {
 }
 
 
-@pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33)])
+@pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33), ("llama_w4a8", 1, 150)])
 def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     shape = SHAPES[name]
     params = synth.make_params(shape, seed=5, max_seq=seq, jitter=True)
