@@ -207,7 +207,8 @@ int zoqat_step_rates(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
  * trainable tensor per step instead of two), or by zoqat_flush_update().  The masters then lag one update behind the
  * returned result until that happens; every other entry point that reads or changes them (zoqat_forward_loss,
  * zoqat_step*, zoqat_apply_update*, zoqat_init_qparams) flushes first, and a caller that reads the master tensors
- * itself calls zoqat_flush_update() before.  Same arithmetic, same bits as zoqat_step.  Models with Section 4.2
+ * itself calls zoqat_flush_update() before (zoqat_model_destroy() does not: a pending update is dropped with the handle).
+ * Same arithmetic, same bits as zoqat_step.  Models with Section 4.2
  * parameters or per-row weight groups run zoqat_step instead (nothing is deferred). */
 int zoqat_step_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
                         int batch, int seq, uint64_t seed, float eps, float lr,
