@@ -292,7 +292,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                     }
 #pragma unroll
                                     for (int k = 0; k < 4; ++k) {
-                                        const uint32_t dst = stage + (uint32_t)(k * 2048 + lane * 64 + j * 2);
+                                        // 64-byte rows with the 64-byte swizzle of the tensor map (16-byte chunk index XOR bits 1-2
+                                        // of the row): the 32 rows of a store instruction spread over all banks
+                                        const uint32_t dst = stage + (uint32_t)(k * 2048 + lane * 64 + (((j >> 3) ^ ((lane >> 1) & 3)) << 4));
                                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[k][0]), "r"(w[k][1]), "r"(w[k][2]), "r"(w[k][3]) : "memory");
                                     }
                                 }
@@ -547,8 +549,9 @@ bool make_out_map(CUtensorMap* map, float* base, int64_t M, int64_t N, int Z) {
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 3-D binary16 map {inner, rows, slabs} with 32 x 32 x 1 boxes (64-byte rows, no swizzle) for the mode-2 stores.
-bool make_half_box_map(CUtensorMap* map, void* base, int64_t inner, int64_t rows, int64_t slabs, int64_t row_pitch) {
+// 3-D binary16 map {inner, rows, slabs} with 32 x 32 x 1 boxes (64-byte rows) for the mode-2 stores; swizzle64 selects the
+// 64-byte swizzle (q / k boxes, written 16 bytes per row at a time) or none (v boxes, written 2 bytes per column at a time).
+bool make_half_box_map(CUtensorMap* map, void* base, int64_t inner, int64_t rows, int64_t slabs, int64_t row_pitch, bool swizzle64) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)slabs};
@@ -556,7 +559,8 @@ bool make_half_box_map(CUtensorMap* map, void* base, int64_t inner, int64_t rows
     const cuuint32_t box[3] = {32, 32, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int num_sms() {
@@ -595,9 +599,9 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
             (a.d_head != 64 && a.d_head != 128) || (a.cos_t == nullptr) != (a.sin_t == nullptr) || !a.att.qh)
             return ZOQAT_ERR_INVALID_ARG;
         const int64_t bhs = (int64_t)a.Z * (a.M / a.seq) * a.n_heads;
-        if (!make_half_box_map(&att.qh, a.att.qh, a.d_head, a.seq, bhs, a.d_head) || !make_half_box_map(&att.ql, a.att.ql, a.d_head, a.seq, bhs, a.d_head) ||
-            !make_half_box_map(&att.kh, a.att.kh, a.d_head, a.seq, bhs, a.d_head) || !make_half_box_map(&att.kl, a.att.kl, a.d_head, a.seq, bhs, a.d_head) ||
-            !make_half_box_map(&att.vh, a.att.vth, a.seq, a.d_head, bhs, a.att.seq_pad) || !make_half_box_map(&att.vl, a.att.vtl, a.seq, a.d_head, bhs, a.att.seq_pad))
+        if (!make_half_box_map(&att.qh, a.att.qh, a.d_head, a.seq, bhs, a.d_head, true) || !make_half_box_map(&att.ql, a.att.ql, a.d_head, a.seq, bhs, a.d_head, true) ||
+            !make_half_box_map(&att.kh, a.att.kh, a.d_head, a.seq, bhs, a.d_head, true) || !make_half_box_map(&att.kl, a.att.kl, a.d_head, a.seq, bhs, a.d_head, true) ||
+            !make_half_box_map(&att.vh, a.att.vth, a.seq, a.d_head, bhs, a.att.seq_pad, false) || !make_half_box_map(&att.vl, a.att.vtl, a.seq, a.d_head, bhs, a.att.seq_pad, false))
             return ZOQAT_ERR_CUDA;
         map_out = map_a;      // never dereferenced
     } else {
