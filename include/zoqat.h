@@ -480,13 +480,15 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
  * The deployment side of the method (the paper's on-device tokens-per-second table): one new
  * token per sequence and call, keys and values cached, every block linear read once per
  * token as stored low-bit codes.  Needs a model whose block linears are all FROZEN_PACKED
- * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups, a_bits in {4, 6, 8};
- * batch in {1, 2, 4} sequences advance in lock step.
+ * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups; batch in {1, 2, 4}
+ * sequences advance in lock step.
  *
  * Arithmetic: a packed linear is evaluated as an integer runtime does,
  *     y[t, n] = s_t * sum_g Delta[n, g] * ( sum_{k in g} a[t, k] * (c[n, k] - z[n, g]) ) (+ bias),
  * the inner sums exact integers (dp4a), the steps applied in fp32; it differs from the
- * training forward only by that forward's bf16 rounding of (c - z) * Delta.  Norms,
+ * training forward only by that forward's bf16 rounding of (c - z) * Delta.  Weight-only
+ * models (a_bits = 0) use the forward's own operands, bf16(x) and bf16((c - z) * Delta),
+ * with fp32 accumulation.  Norms,
  * rotary embedding, attention (fp32, over an fp32 cache) and the bf16 vocabulary
  * projection are those of the forward pass.
  *

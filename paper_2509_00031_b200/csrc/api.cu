@@ -1317,7 +1317,6 @@ int decode_sizes(const zoqat_model* m, int batch, int max_len, DecodeSizes& z) {
     if (batch != 1 && batch != 2 && batch != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode batch %d (supported: 1, 2, 4)", batch);
     if (max_len <= 0 || max_len > c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "max_len %d must be in 1..max_seq (%d)", max_len, c.max_seq);
     if (batch > c.max_batch * c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "batch exceeds the workspace");
-    if (c.a_bits == 0) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs quantised activations (a_bits 4, 6 or 8)");
     if (c.w_group == 0 || c.w_bits > 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs column groups of 32, 64 or 128 and w_bits <= 4");
     const size_t d = c.d_model, F = c.d_ffn, n_up = c.arch == ZOQAT_ARCH_LLAMA ? 2 * F : F;
     z.nib[0] = align_up(3 * d * d / 2); z.nib[1] = align_up(d * d / 2); z.nib[2] = align_up(n_up * d / 2); z.nib[3] = align_up(d * F / 2);
@@ -1422,8 +1421,9 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
     const int B = D.batch, d = c.d_model, F = c.d_ffn, H = c.n_heads, dh = d / H, G = c.w_group;
     const int norm_kind = llama ? 1 : 2, n_up = llama ? 2 * F : F;
     auto gemv = [&](const void* wq, const float2* qp, int N, int K, const float* bias, int accumulate, float* out) {
-        if (launch_decode_gemv(wq, qp, N, K, G, B, w.xa, w.row_step, bias, accumulate, out, s) != 0)
-            return fail(ZOQAT_ERR_UNSUPPORTED, "decode matrix-vector product rejected (N=%d K=%d)", N, K);
+        const int rc = c.a_bits ? launch_decode_gemv(wq, qp, N, K, G, B, w.xa, w.row_step, bias, accumulate, out, s)
+                                : launch_decode_gemv_fp(wq, qp, N, K, G, B, w.xa, bias, accumulate, out, s);     // weight-only
+        if (rc != 0) return fail(ZOQAT_ERR_UNSUPPORTED, "decode matrix-vector product rejected (N=%d K=%d)", N, K);
         return (int)ZOQAT_OK;
     };
     launch_embed(tokens_dev, m->embed, m->pos ? m->pos + (size_t)pos * d : nullptr, B, 1, d, c.vocab, 1, w.h, s);

@@ -109,6 +109,9 @@ void launch_repack_nibbles(const uint32_t* packed, int64_t n, int bits, void* ou
 void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
 int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
                        const float* row_step, const float* bias, int accumulate, float* out, cudaStream_t s);
+// weight-only models: act = bf16(x) [mb, K], operands bf16((c - z) * Delta) as in the training forward
+int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
+                          const float* bias, int accumulate, float* out, cudaStream_t s);
 // qkv != NULL: q | k | v of the new token, fp32 [batch, 3*d]: rotated (cos_t / sin_t or none), k and v appended at `pos`.
 void launch_decode_attention(const float* q, float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos,
                              int max_len, float* out, const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s);

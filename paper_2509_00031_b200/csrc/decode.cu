@@ -164,6 +164,81 @@ decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qpar
 }
 
 // ---- attention over the cache -----------------------------------------------------------------------------------
+// Weight-only models (activations not quantised): y[m, n] (+)= sum_k bf16(x[m, k]) * bf16((c[n, k] - z) * Delta) (+ bias), the
+// operands of the training forward (bf16-rounded dequantised weight, bf16 activation), fp32 accumulation.  Same mapping
+// as decode_gemv_kernel; the activations sit in shared memory as bf16.
+template <int MB>
+__global__ void __launch_bounds__(kGemvThreads)
+decode_gemv_fp_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qparams, int N, int K, int group_shift,
+                      const __nv_bfloat16* __restrict__ act, const float* __restrict__ bias, int accumulate,
+                      float* __restrict__ out) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    uint4* xs = reinterpret_cast<uint4*>(smem);                            // [MB][K] bf16, 8 per uint4
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int chunks = K >> 5, gpr = K >> group_shift, cshift = group_shift - 5;
+    for (int i = threadIdx.x; i < MB * (K >> 3); i += kGemvThreads) xs[i] = __ldg(reinterpret_cast<const uint4*>(act) + i);
+    __syncthreads();
+    for (int n = blockIdx.x * (kGemvThreads / 32) + warp; n < N; n += gridDim.x * (kGemvThreads / 32)) {
+        const uint4* wrow = wq + (size_t)n * chunks;
+        const float2* qrow = qparams + (size_t)n * gpr;
+        float acc[MB];
+#pragma unroll
+        for (int m = 0; m < MB; ++m) acc[m] = 0.0f;
+        for (int ch0 = lane; ch0 < chunks; ch0 += 64) {       // two loads in flight per lane
+            uint4 w[2];
+            float2 qp[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int ch = ch0 + 32 * u;
+                if (ch < chunks) { w[u] = __ldg(wrow + ch); qp[u] = __ldg(qrow + (ch >> cshift)); }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int ch = ch0 + 32 * u;
+                if (ch < chunks) {
+                    const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+                    // (c - z) exactly: the nibble goes into the mantissa of 2^23, then one subtraction of 2^23 + z
+                    const float zoff = 8388608.0f + qp[u].y;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float v[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float cf = __uint_as_float(((ww[q] >> (4 * e)) & 0xFu) | 0x4B000000u);
+                            v[e] = __bfloat162float(__float2bfloat16_rn(__fmul_rn(__fadd_rn(cf, -zoff), qp[u].x)));
+                        }
+#pragma unroll
+                        for (int m = 0; m < MB; ++m) {
+                            const uint4 xv = xs[m * (K >> 3) + ch * 4 + q];
+                            const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&xv);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 xf = __bfloat1622float2(x2[e]);
+                                acc[m] = __fmaf_rn(v[2 * e], xf.x, acc[m]);
+                                acc[m] = __fmaf_rn(v[2 * e + 1], xf.y, acc[m]);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < MB; ++m) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int m = 0; m < MB; ++m) {
+                float y = acc[m];
+                if (bias) y += bias[n];
+                float* o = out + (size_t)m * N + n;
+                *o = accumulate ? *o + y : y;
+            }
+        }
+    }
+}
+
 // cache_k / cache_v: fp32 [B][H][max_len][dh] of one layer.
 // out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA of 8 warps per (sequence, head).  Warp s takes
 // the cached positions t = s, s + 8, ...: a lane holds 4 (d_head 128) or 2 (d_head 64) features, so one load instruction
@@ -394,6 +469,26 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     }
     if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else return -1;
 #undef ZQ_GEMV
+    count_launch();
+    return 0;
+}
+
+int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
+                          const float* bias, int accumulate, float* out, cudaStream_t s) {
+    if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
+    const size_t smem = (size_t)mb * K * 2;
+    if (smem > 160 * 1024) return -1;
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : 3)));
+    const int gshift = group == 32 ? 5 : (group == 64 ? 6 : 7);
+    const uint4* w4 = static_cast<const uint4*>(wq);
+#define ZQ_GEMV_FP(MBV)                                                                                                   \
+    {                                                                                                                     \
+        static bool attr = false;                                                                                         \
+        if (!attr) { cudaFuncSetAttribute(decode_gemv_fp_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
+        decode_gemv_fp_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, bias, accumulate, out); \
+    }
+    if (mb == 1) ZQ_GEMV_FP(1) else if (mb == 2) ZQ_GEMV_FP(2) else if (mb == 4) ZQ_GEMV_FP(4) else return -1;
+#undef ZQ_GEMV_FP
     count_launch();
     return 0;
 }

@@ -55,10 +55,13 @@ SHAPES = {
     "llama_w4a8": dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=600, w_bits=4, w_group=64, a_bits=8),
     "opt_w3a8": dict(arch="opt", n_layers=2, d_model=128, n_heads=2, d_ffn=256, vocab=333, w_bits=3, w_group=128, a_bits=8),
     "llama_w2a4": dict(arch="llama", n_layers=1, d_model=256, n_heads=2, d_ffn=512, vocab=512, w_bits=2, w_group=32, a_bits=4),
+    "llama_w4": dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=600, w_bits=4, w_group=128, a_bits=0),
+    "opt_w3": dict(arch="opt", n_layers=1, d_model=128, n_heads=2, d_ffn=256, vocab=333, w_bits=3, w_group=64, a_bits=0),
 }
 
 
-@pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33), ("llama_w4a8", 1, 150)])
+@pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33), ("llama_w4a8", 1, 150),
+                                            ("llama_w4", 2, 40), ("opt_w3", 4, 20)])
 def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     shape = SHAPES[name]
     params = synth.make_params(shape, seed=5, max_seq=seq, jitter=True)
@@ -74,17 +77,24 @@ def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     tokens, _ = synth.make_batch(batch, seq, shape["vocab"], seed=21)
     want = oracle.logits(tokens).reshape(batch, seq, -1)
     scale = np.abs(want).max()
+    # How far two correct implementations differ: the oracle against itself with its stored activations re-rounded to
+    # binary32.  With quantised activations that is nothing on these models; weight-only models round every linear input
+    # to a bfloat16 operand, and one rounding that falls the other way in a cached key or value moves every later
+    # position (measured: the GPU then sits on the binary32-storage oracle, 2e-3 of the logit scale from the float64 one).
+    cfg32 = OracleConfig(**{**oracle.cfg.__dict__, "store_f32": True})
+    band = np.abs(OracleModel(cfg32, synth.copy_params(params)).logits(tokens).reshape(batch, seq, -1) - want).max()
+    tol = 2e-4 * scale + 1.5 * band
     agree = total = 0
     for pos in range(seq):
         logits, nxt = model.zoqat_decode_step(dev(tokens[:, pos].copy()), pos)
         got = logits.cpu().numpy()
         model.zoqat_check()
         err = np.abs(got - want[:, pos]).max()
-        assert err <= 2e-4 * scale, (pos, err, scale)
+        assert err <= tol, (pos, err, tol, scale)
         # greedy choice: the device's argmax of its own logits, and the oracle's wherever its top two are well apart
         assert np.array_equal(nxt.cpu().numpy(), got.argmax(-1))
         top2 = np.sort(want[:, pos], axis=-1)[:, -2:]
-        clear = (top2[:, 1] - top2[:, 0]) > 1e-3 * scale
+        clear = (top2[:, 1] - top2[:, 0]) > 5 * tol
         agree += int((nxt.cpu().numpy()[clear] == want[:, pos].argmax(-1)[clear]).sum())
         total += int(clear.sum())
     assert total > 0 and agree == total
