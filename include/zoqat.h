@@ -480,7 +480,7 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
  * The deployment side of the method (the paper's on-device tokens-per-second table): one new
  * token per sequence and call, keys and values cached, every block linear read once per
  * token as stored low-bit codes.  Needs a model whose block linears are all FROZEN_PACKED
- * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups; batch in {1, 2, 4}
+ * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups; batch in {1, 2, 4, 8}
  * sequences advance in lock step.
  *
  * Arithmetic: a packed linear is evaluated as an integer runtime does,
@@ -509,7 +509,7 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
  * zoqat_op_pack_frozen for a [rows, cols] tensor; act_codes_dev bf16 [batch, cols] integer codes
  * with their steps row_step_dev[batch] (zoqat_op_norm_act_operand output); out_dev fp32
  * [batch, rows] (accumulate != 0 adds); nibble_scratch_dev: rows*cols/2 bytes, 16-byte aligned
- * (the repacked codes).  batch in {1, 2, 4}; cols % 32 == 0. */
+ * (the repacked codes).  batch in {1, 2, 4, 8}; cols % 32 == 0. */
 int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group, int bits,
                          const void* act_codes_dev, const float* row_step_dev, int batch, const float* bias_dev,
                          int accumulate, float* out_dev, void* nibble_scratch_dev, void* stream);

@@ -1314,7 +1314,7 @@ struct DecodeSizes { size_t nib[4], qp_qkv, qp_up, head, cache, logits, q_rot, t
 
 int decode_sizes(const zoqat_model* m, int batch, int max_len, DecodeSizes& z) {
     const zoqat_config_t& c = m->cfg;
-    if (batch != 1 && batch != 2 && batch != 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode batch %d (supported: 1, 2, 4)", batch);
+    if (batch != 1 && batch != 2 && batch != 4 && batch != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "decode batch %d (supported: 1, 2, 4, 8)", batch);
     if (max_len <= 0 || max_len > c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "max_len %d must be in 1..max_seq (%d)", max_len, c.max_seq);
     if (batch > c.max_batch * c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "batch exceeds the workspace");
     if (c.w_group == 0 || c.w_bits > 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs column groups of 32, 64 or 128 and w_bits <= 4");
@@ -1404,7 +1404,7 @@ int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_
     launch_repack_nibbles(static_cast<const uint32_t*>(packed_dev), rows * cols, bits, nibble_scratch_dev, s);
     if (launch_decode_gemv(nibble_scratch_dev, static_cast<const float2*>(qparams_dev), (int)rows, (int)cols, group, batch,
                            static_cast<const __nv_bfloat16*>(act_codes_dev), row_step_dev, bias_dev, accumulate, out_dev, s) != 0)
-        return fail(ZOQAT_ERR_UNSUPPORTED, "batch %d (supported: 1, 2, 4) or shape rejected", batch);
+        return fail(ZOQAT_ERR_UNSUPPORTED, "batch %d (supported: 1, 2, 4, 8) or shape rejected", batch);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

@@ -104,7 +104,7 @@ int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d
                         const float* sin_t, float* out, void* scratch, int32_t* err_flag, cudaStream_t s);
 
 // Decode-time inference over the packed representation (decode.cu).  launch_decode_gemv / launch_decode_head return 0 or -1
-// (unsupported shape: K % 32, group, batch not in {1, 2, 4}).
+// (unsupported shape: K % 32, group, batch not in {1, 2, 4, 8}).
 void launch_repack_nibbles(const uint32_t* packed, int64_t n, int bits, void* out, cudaStream_t s);
 void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
 int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,

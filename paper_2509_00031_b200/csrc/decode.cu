@@ -5,7 +5,7 @@
 //   repack_nibbles_kernel   once per model: the bit-plane packing (built for warp ballots in the training path) is
 //                           turned into 4-bit nibbles in input-channel order, the layout integer dot products want.
 //   decode_gemv_kernel      y[m, n] (+)= s_m * sum_g Delta[n, g] * ( sum_{k in g} a[m, k] * (c[n, k] - z[n, g]) ) (+ bias)
-//                           for up to 4 sequences m: one warp per output row n, 32 codes (16 bytes) per lane and load,
+//                           for up to 8 sequences m: one warp per output row n, 32 codes (16 bytes) per lane and load,
 //                           dp4a on the nibble pairs against int8 activation codes staged in shared memory, the inner
 //                           sums exact integers, steps applied in fp32.
 //   decode_attention_kernel rotary embedding of the new q and k, append k and v to the cache,
@@ -458,7 +458,7 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     const size_t smem = decode_gemv_smem_bytes(mb, K);
     if (smem > 160 * 1024) return -1;
     // every CTA stages the activation codes of all sequences: more sequences, fewer and longer-lived CTAs (measured)
-    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : 3)));
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : (mb == 4 ? 3 : 2))));
     const int gshift = group == 32 ? 5 : (group == 64 ? 6 : 7);
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV(MBV)                                                                                                      \
@@ -467,7 +467,7 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
         if (!attr) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
         decode_gemv_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, row_step, bias, accumulate, out); \
     }
-    if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else return -1;
+    if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else if (mb == 8) ZQ_GEMV(8) else return -1;
 #undef ZQ_GEMV
     count_launch();
     return 0;
@@ -478,7 +478,7 @@ int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, i
     if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
     const size_t smem = (size_t)mb * K * 2;
     if (smem > 160 * 1024) return -1;
-    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : 3)));
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : (mb == 4 ? 3 : 2))));
     const int gshift = group == 32 ? 5 : (group == 64 ? 6 : 7);
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV_FP(MBV)                                                                                                   \
@@ -487,7 +487,7 @@ int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, i
         if (!attr) { cudaFuncSetAttribute(decode_gemv_fp_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
         decode_gemv_fp_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, bias, accumulate, out); \
     }
-    if (mb == 1) ZQ_GEMV_FP(1) else if (mb == 2) ZQ_GEMV_FP(2) else if (mb == 4) ZQ_GEMV_FP(4) else return -1;
+    if (mb == 1) ZQ_GEMV_FP(1) else if (mb == 2) ZQ_GEMV_FP(2) else if (mb == 4) ZQ_GEMV_FP(4) else if (mb == 8) ZQ_GEMV_FP(8) else return -1;
 #undef ZQ_GEMV_FP
     count_launch();
     return 0;
@@ -515,7 +515,11 @@ int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_
     if (mb == 1) decode_head_kernel<1><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
     else if (mb == 2) decode_head_kernel<2><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
     else if (mb == 4) decode_head_kernel<4><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
-    else return -1;
+    else if (mb == 8) {
+        static bool attr = false;
+        if (!attr) { cudaFuncSetAttribute(decode_head_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+        decode_head_kernel<8><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+    } else return -1;
     count_launch();
     return 0;
 }

@@ -25,7 +25,7 @@ def dev(a):
 
 
 @pytest.mark.parametrize("bits,group,rows,cols,batch", [(4, 128, 300, 512, 1), (4, 64, 96, 1024 + 64, 2), (2, 32, 256, 4096, 4),
-                                                         (3, 128, 64, 11008, 4)])
+                                                         (3, 128, 64, 11008, 4), (4, 128, 128, 11008, 8)])
 def test_packed_gemv_is_exact_integer_arithmetic(zq, bits, group, rows, cols, batch):
     if (rows * cols) % 128:
         pytest.skip("packed tensors need rows*cols % 128 == 0")
@@ -61,7 +61,7 @@ SHAPES = {
 
 
 @pytest.mark.parametrize("name,batch,seq", [("llama_w4a8", 2, 40), ("opt_w3a8", 4, 24), ("llama_w2a4", 1, 33), ("llama_w4a8", 1, 150),
-                                            ("llama_w4", 2, 40), ("opt_w3", 4, 20)])
+                                            ("llama_w4", 2, 40), ("opt_w3", 4, 20), ("llama_w4a8", 8, 20), ("opt_w3", 8, 12)])
 def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     shape = SHAPES[name]
     params = synth.make_params(shape, seed=5, max_seq=seq, jitter=True)
@@ -83,7 +83,9 @@ def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     # position (measured: the GPU then sits on the binary32-storage oracle, 2e-3 of the logit scale from the float64 one).
     cfg32 = OracleConfig(**{**oracle.cfg.__dict__, "store_f32": True})
     band = np.abs(OracleModel(cfg32, synth.copy_params(params)).logits(tokens).reshape(batch, seq, -1) - want).max()
-    tol = 2e-4 * scale + 1.5 * band
+    # (the binary32-storage oracle still normalises in float64, so it does not produce every flip a binary32
+    # implementation can: weight-only models get a floor of 2e-3 of the logit scale, the size of one such flip here)
+    tol = (2e-4 if shape["a_bits"] else 2e-3) * scale + 1.5 * band
     agree = total = 0
     for pos in range(seq):
         logits, nxt = model.zoqat_decode_step(dev(tokens[:, pos].copy()), pos)
