@@ -193,7 +193,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
                       const PhiloxKeys rk, uint32_t tid, float eps,
                       uint2* __restrict__ op_plus, uint2* __restrict__ op_minus,
                       uchar4* __restrict__ codes, float* __restrict__ step, int32_t* __restrict__ zp,
-                      float4* __restrict__ w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk) {
+                      float4* w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk) {
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
     if (perturb || UPD) stage_icdf_table(tab);
@@ -206,7 +206,8 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         float x[16], xm[16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float4 v = live ? (UPD ? w[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
+            // with UPD the master is read through the pointer it is written back through (w itself is then not dereferenced)
+            const float4 v = live ? (UPD ? w_out[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
         }
         if (UPD) {
