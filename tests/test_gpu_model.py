@@ -424,3 +424,16 @@ def test_deferred_update_gives_the_same_bits(zq, shape, batch, seq, first):
     lazy.zoqat_flush_update()
     assert torch.equal(eager.params["layers"][last][name], lazy.params["layers"][last][name])
     assert torch.equal(eager.params["lm_head"], lazy.params["lm_head"])
+
+
+def test_step_without_any_labelled_position(zq):
+    """Every label ignored: both losses are 0, g is 0 and the masters do not move (no division by zero)."""
+    shape, batch, seq = SMALL_LLAMA, 1, 32
+    model, _ = build_pair(zq, shape, batch, seq, 0)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=3)
+    before = model.params["layers"][0]["wq"].clone()
+    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(np.full_like(labels, -1)), 9, 1e-3, 1e-2))
+    model.zoqat_check()
+    assert res["n_labels"] == 0 and res["loss_plus"] == 0.0 and res["loss_minus"] == 0.0
+    assert res["proj_grad"] == 0.0 and res["update_scale"] == 0.0 and res["status"] == 0
+    assert torch.equal(before, model.params["layers"][0]["wq"])

@@ -381,3 +381,32 @@ def test_head_loss(zq, impl, T, V, d):
     assert np.allclose(tl.cpu().numpy(), want, rtol=0, atol=3e-6 * np.abs(lse).max())
     assert int(cnt.item()) == int(valid.sum())
     assert abs(float(ls.item()) - want.sum()) <= 1e-6 * abs(want.sum())
+
+
+# ---- degenerate inputs ------------------------------------------------------------------------------------------
+def test_degenerate_groups_and_rows(zq):
+    """Constant groups (step floored at 1e-8, huge x / step), an all-zero token row, and huge magnitudes: the kernels
+    take the same decisions as the oracle and produce no NaN."""
+    w = np.full((64, 256), 0.3, np.float32)
+    w[1, :128] = 0.0                       # a group of zeros
+    w[2, 128:] = -7.5                      # a constant negative group
+    w[3] = np.linspace(-1e4, 1e4, 256, dtype=np.float32)     # large magnitudes
+    for bits, group in [(4, 128), (2, 32)]:
+        codes, step, zp, operand = zq.zoqat_op_weight_quant(dev(w), group, bits, 0, 0, 0.0)
+        o_codes, o_step, o_zp, o_deq = core.weight_quant(w, group, bits)
+        assert np.array_equal(codes.cpu().numpy(), o_codes)
+        assert np.array_equal(step.cpu().numpy().view(np.uint32), o_step.view(np.uint32))
+        assert np.array_equal(zp.cpu().numpy(), o_zp)
+        got = bf16_to_f32(operand)
+        assert np.all(np.isfinite(got)) and np.array_equal(got, core.round_bf16(o_deq))
+        # and through the packed representation
+        packed, qparams = zq.zoqat_op_pack_frozen(dev(w), group, bits)
+        op2 = zq.zoqat_op_unpack_operand(packed, qparams, 64, 256, group, bits)
+        assert np.array_equal(bf16_to_f32(op2), core.round_bf16(o_deq))
+    x = np.zeros((3, 512), np.float32)
+    x[1] = 1e30
+    x[2, 5] = -3.0
+    op, st, _ = zq.zoqat_op_norm_act_operand(dev(x), 0, None, None, 0.0, 8)
+    q, s = act_quant(x.astype(np.float64))
+    assert np.array_equal(bf16_to_f32(op), q) and np.array_equal(st.cpu().numpy(), s)
+    assert float(st[0]) == np.float32(1e-8) and np.all(bf16_to_f32(op)[0] == 0)
