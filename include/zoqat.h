@@ -508,8 +508,9 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
 /* One packed linear of the decode path on raw buffers: packed_dev / qparams_dev as written by
  * zoqat_op_pack_frozen for a [rows, cols] tensor; act_codes_dev bf16 [batch, cols] integer codes
  * with their steps row_step_dev[batch] (zoqat_op_norm_act_operand output); out_dev fp32
- * [batch, rows] (accumulate != 0 adds); nibble_scratch_dev: rows*cols/2 bytes, 16-byte aligned
- * (the repacked codes).  batch in {1, 2, 4, 8}; cols % 32 == 0. */
+ * [batch, rows] (accumulate != 0 adds); nibble_scratch_dev: rows*cols/2 + 2*batch*cols bytes,
+ * 16-byte aligned (the repacked codes, then the activation rows as int8).  batch in
+ * {1, 2, 4, 8}; cols % 32 == 0. */
 int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group, int bits,
                          const void* act_codes_dev, const float* row_step_dev, int batch, const float* bias_dev,
                          int accumulate, float* out_dev, void* nibble_scratch_dev, void* stream);

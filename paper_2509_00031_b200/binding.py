@@ -341,7 +341,7 @@ def zoqat_op_decode_gemv(packed, qparams, rows, cols, group, bits, act_codes, ro
     batch = act_codes.shape[0]
     if out is None:
         out = torch.empty((batch, rows), dtype=torch.float32, device=packed.device)
-    scratch = torch.empty(rows * cols // 2, dtype=torch.uint8, device=packed.device)
+    scratch = torch.empty(rows * cols // 2 + 2 * batch * cols, dtype=torch.uint8, device=packed.device)
     _check(lib().zoqat_op_decode_gemv(_p(packed), _p(qparams), rows, cols, group, bits, _p(act_codes), _p(row_step), batch, _p(bias),
                                       int(accumulate), _p(out), _p(scratch), _stream()))
     return out

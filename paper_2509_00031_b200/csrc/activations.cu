@@ -49,9 +49,32 @@ __device__ __forceinline__ const float* smooth_base(const SmoothAct& sm, int64_t
     return sm.smooth + (r >= sm.rows_per_pass ? 3 * (size_t)sm.ld : 0);
 }
 
+// Integer form of a quantised operand row for the decode-time matrix-vector kernels, inside the row's 2 * cols bytes:
+// the codes of even columns as int8 [cols / 2], those of odd columns [cols / 2], then the sum of the codes of every 32
+// columns as int32 [cols / 32] (cols % 32 == 0).  store_code_planes: the thread holding columns 4 * idx .. 4 * idx + 3
+// writes its two bytes of each plane; the eight threads of a 32-column chunk add up their sums by shuffles, so whole
+// warps must call it (live = 0 for slots beyond the row, whose codes are 0).
+struct CodePlanes { uint16_t* even; uint16_t* odd; int32_t* csum; };
+__device__ __forceinline__ CodePlanes code_planes(__nv_bfloat16* op_row, int cols) {
+    uint8_t* b = reinterpret_cast<uint8_t*>(op_row);
+    return {reinterpret_cast<uint16_t*>(b), reinterpret_cast<uint16_t*>(b + (cols >> 1)), reinterpret_cast<int32_t*>(b + cols)};
+}
+__device__ __forceinline__ void store_code_planes(const CodePlanes& pl, int idx, bool live, float q0, float q1, float q2, float q3) {
+    const int c0 = (int)q0, c1 = (int)q1, c2 = (int)q2, c3 = (int)q3;
+    int sum = c0 + c1 + c2 + c3;
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+    if (live) {
+        pl.even[idx] = (uint16_t)(((uint32_t)c0 & 0xFFu) | (((uint32_t)c2 & 0xFFu) << 8));
+        pl.odd[idx] = (uint16_t)(((uint32_t)c1 & 0xFFu) | (((uint32_t)c3 & 0xFFu) << 8));
+        if ((idx & 7) == 0) pl.csum[idx >> 3] = sum;
+    }
+}
+
 // Writes the operand row from the fp32 row held in shared memory.
 __device__ __forceinline__ void write_operand_row(const float* row, int cols, int a_bits, __nv_bfloat16* op_row,
-                                                  float* row_step, float* redf) {
+                                                  float* row_step, float* redf, int planes = 0) {
     if (a_bits != 0) {
         const float qmax = (float)((1 << (a_bits - 1)) - 1), qmin = -qmax - 1.0f;     // symmetric N-bit range
         float amax = 0.0f;
@@ -60,6 +83,20 @@ __device__ __forceinline__ void write_operand_row(const float* row, int cols, in
         const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
+        if (planes) {                          // cols % 32 == 0: every warp runs every round, loads and stores are guarded
+            const CodePlanes pl = code_planes(op_row, cols);
+            const int n4 = cols >> 2;
+            for (int base = 0; base < n4; base += kRowThreads) {
+                const int idx = base + threadIdx.x;
+                float q[4] = {0.f, 0.f, 0.f, 0.f};
+                if (idx < n4) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) q[j] = fminf(fmaxf(rintf(__fmul_rn(row[4 * idx + j], inv)), qmin), qmax);
+                }
+                store_code_planes(pl, idx, idx < n4, q[0], q[1], q[2], q[3]);
+            }
+            return;
+        }
         for (int c = 2 * threadIdx.x; c < cols; c += 2 * kRowThreads) {
             const float q0 = fminf(fmaxf(rintf(__fmul_rn(row[c], inv)), qmin), qmax);
             const float q1 = fminf(fmaxf(rintf(__fmul_rn(row[c + 1], inv)), qmin), qmax);
@@ -75,10 +112,12 @@ __device__ __forceinline__ void write_operand_row(const float* row, int cols, in
 __global__ void __launch_bounds__(kRowThreads)
 norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
                         const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
-                        float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm) {
+                        float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm, int planes) {
     extern __shared__ float row[];
     __shared__ double redd[kRowThreads / 32];
     __shared__ float redf[kRowThreads / 32];
+    grid_dependency_release();
+    grid_dependency_wait();       // x comes from the preceding kernel
     const int64_t r = blockIdx.x;
     const float* xr = x + r * cols;
     for (int c = 4 * threadIdx.x; c < cols; c += 4 * kRowThreads)
@@ -109,14 +148,16 @@ norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, co
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
         __syncthreads();
     }
-    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
+    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf, planes);
 }
 
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                       float* __restrict__ row_step, SmoothAct sm) {
+                       float* __restrict__ row_step, SmoothAct sm, int planes) {
     extern __shared__ float row[];
     __shared__ float redf[kRowThreads / 32];
+    grid_dependency_release();
+    grid_dependency_wait();       // x comes from the preceding kernel
     const int64_t r = blockIdx.x;
     if (gated) {                     // silu(gate) * up, gate | up concatenated along the row
         const float* g = x + r * 2 * cols;
@@ -134,7 +175,7 @@ ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_b
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
     }
     __syncthreads();
-    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf);
+    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf, planes);
 }
 
 // ---- register-resident variants (rows up to 12288 columns) ------------------------------------------------
@@ -149,7 +190,7 @@ __device__ __forceinline__ uint2 bf16x4(float a, float b, float c, float d) {
 
 template <int VPT>
 __device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n4, int a_bits, uint2* op_row, float* row_step,
-                                                   float* redf) {
+                                                   float* redf, int planes = 0) {
     if (a_bits != 0) {
         const float qmax = (float)((1 << (a_bits - 1)) - 1), qmin = -qmax - 1.0f;     // symmetric N-bit range
         float amax = 0.0f;
@@ -159,6 +200,18 @@ __device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n
         const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
+        if (planes) {
+            const CodePlanes pl = code_planes(reinterpret_cast<__nv_bfloat16*>(op_row), 4 * n4);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int idx = threadIdx.x + i * kRowThreads;
+                store_code_planes(pl, idx, idx < n4, fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), qmin), qmax));
+            }
+            return;
+        }
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = threadIdx.x + i * kRowThreads;
@@ -195,9 +248,11 @@ template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
                             const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
-                            float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm) {
+                            float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm, int planes) {
     __shared__ double redd[kRowThreads / 32];
     __shared__ float redf[kRowThreads / 32];
+    grid_dependency_release();
+    grid_dependency_wait();       // x comes from the preceding kernel
     const int64_t r = blockIdx.x;
     const int n4 = cols >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + r * cols);
@@ -258,14 +313,16 @@ norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind
         }
     }
     smooth_regs<VPT>(v, n4, sm, r);
-    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf, planes);
 }
 
 template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                           float* __restrict__ row_step, SmoothAct sm) {
+                           float* __restrict__ row_step, SmoothAct sm, int planes) {
     __shared__ float redf[kRowThreads / 32];
+    grid_dependency_release();
+    grid_dependency_wait();       // x comes from the preceding kernel
     const int64_t r = blockIdx.x;
     const int n4 = cols >> 2;
     float4 v[VPT];
@@ -296,7 +353,7 @@ ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int
         }
     }
     smooth_regs<VPT>(v, n4, sm, r);
-    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf);
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf, planes);
 }
 
 // Activation operand of a row whose max |x| has already been collected (by the GEMM that produced x).
@@ -342,6 +399,7 @@ rows_operand_reg_kernel(const float* __restrict__ x, int cols, const uint32_t* _
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const float4* __restrict__ embed,
                              const float4* __restrict__ pos, int64_t T, int seq, int d4, int vocab, int passes,
                              float4* __restrict__ h) {
+    grid_dependency_release();
     const int64_t t = blockIdx.x;
     int tok = tokens[t];
     tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
@@ -453,40 +511,40 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
-                             SmoothAct sm) {
+                             SmoothAct sm, bool dependent, bool planes) {
     const int n4 = cols / 4;
     const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(bias) |
                            reinterpret_cast<uintptr_t>(normed)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        norm_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
+        launch_kernel(norm_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        norm_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
+        launch_kernel(norm_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        norm_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
+        launch_kernel(norm_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static bool attr = false;
         if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        norm_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm);
+        launch_kernel(norm_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     }
     count_launch();
 }
 
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
-                            float* row_step, cudaStream_t s, SmoothAct sm) {
+                            float* row_step, cudaStream_t s, SmoothAct sm, bool dependent, bool planes) {
     const int n4 = cols / 4;
     const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        ffn_act_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
+        launch_kernel(ffn_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        ffn_act_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
+        launch_kernel(ffn_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        ffn_act_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, gated, a_bits, op, row_step, sm);
+        launch_kernel(ffn_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static bool attr = false;
         if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        ffn_act_operand_kernel<<<(unsigned)rows, kRowThreads, smem, s>>>(x, cols, gated, a_bits, op, row_step, sm);
+        launch_kernel(ffn_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
     }
     count_launch();
 }

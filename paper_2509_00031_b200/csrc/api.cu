@@ -1401,9 +1401,13 @@ int zoqat_op_decode_gemv(const void* packed_dev, const void* qparams_dev, int64_
     if (!packed_dev || !qparams_dev || !act_codes_dev || !row_step_dev || !out_dev || !nibble_scratch_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if (reinterpret_cast<uintptr_t>(nibble_scratch_dev) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "nibble_scratch_dev must be 16-byte aligned");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (batch != 1 && batch != 2 && batch != 4 && batch != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "batch %d (supported: 1, 2, 4, 8)", batch);
     launch_repack_nibbles(static_cast<const uint32_t*>(packed_dev), rows * cols, bits, nibble_scratch_dev, s);
+    // the kernel reads the activation rows in their integer form, which follows the repacked codes in the scratch
+    uint8_t* planes = static_cast<uint8_t*>(nibble_scratch_dev) + rows * cols / 2;
+    launch_codes_to_planes(static_cast<const __nv_bfloat16*>(act_codes_dev), batch, (int)cols, planes, s);
     if (launch_decode_gemv(nibble_scratch_dev, static_cast<const float2*>(qparams_dev), (int)rows, (int)cols, group, batch,
-                           static_cast<const __nv_bfloat16*>(act_codes_dev), row_step_dev, bias_dev, accumulate, out_dev, s) != 0)
+                           reinterpret_cast<const __nv_bfloat16*>(planes), row_step_dev, bias_dev, accumulate, out_dev, s) != 0)
         return fail(ZOQAT_ERR_UNSUPPORTED, "batch %d (supported: 1, 2, 4, 8) or shape rejected", batch);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
@@ -1420,6 +1424,7 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
     const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
     const int B = D.batch, d = c.d_model, F = c.d_ffn, H = c.n_heads, dh = d / H, G = c.w_group;
     const int norm_kind = llama ? 1 : 2, n_up = llama ? 2 * F : F;
+    const bool planes = c.a_bits != 0;          // the integer kernels read int8 code planes, the weight-only ones bf16 rows
     auto gemv = [&](const void* wq, const float2* qp, int N, int K, const float* bias, int accumulate, float* out) {
         const int rc = c.a_bits ? launch_decode_gemv(wq, qp, N, K, G, B, w.xa, w.row_step, bias, accumulate, out, s)
                                 : launch_decode_gemv_fp(wq, qp, N, K, G, B, w.xa, bias, accumulate, out, s);     // weight-only
@@ -1431,19 +1436,19 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
         const Layer& Ly = m->layers[l];
         const DecodeLayer& dl = D.layers[l];
         launch_norm_act_operand(w.h, B, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B], c.norm_eps,
-                                c.a_bits, w.xa, w.row_step, nullptr, s);
+                                c.a_bits, w.xa, w.row_step, nullptr, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_qkv, dl.q_qkv, 3 * d, d, llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d, 0, w.qkv)) return rc;
         launch_decode_attention(nullptr, dl.cache_k, dl.cache_v, B, H, dh, pos, D.max_len, w.att, w.qkv,
                                 llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, s);
-        launch_norm_act_operand(w.att, B, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s);
+        launch_norm_act_operand(w.att, B, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_o, dl.q_o, d, d, Ly.vec[ZOQAT_ROLE_BO], 1, w.h)) return rc;
         launch_norm_act_operand(w.h, B, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B], c.norm_eps,
-                                c.a_bits, w.xa, w.row_step, nullptr, s);
+                                c.a_bits, w.xa, w.row_step, nullptr, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_up, dl.q_up, n_up, d, Ly.vec[ZOQAT_ROLE_B_FC1], 0, w.ffn)) return rc;
-        launch_ffn_act_operand(w.ffn, B, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s);
+        launch_ffn_act_operand(w.ffn, B, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_down, dl.q_down, d, F, Ly.vec[ZOQAT_ROLE_B_FC2], 1, w.h)) return rc;
     }
-    launch_norm_act_operand(w.h, B, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s);
+    launch_norm_act_operand(w.h, B, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s, SmoothAct(), true);
     float* logits = logits_dev ? logits_dev : D.logits;
     if (launch_decode_head(D.head, c.vocab, d, B, w.xa, logits, s) != 0) return fail(ZOQAT_ERR_UNSUPPORTED, "vocabulary projection rejected");
     if (next_token_dev) launch_decode_argmax(logits, B, c.vocab, next_token_dev, s);

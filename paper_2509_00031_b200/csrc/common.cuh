@@ -17,6 +17,32 @@ constexpr int kErrWaitAccEmpty = 4;  // MMA warp: accumulator never drained
 extern long long g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count += n; }
 
+// Programmatic dependent launch.  A kernel launched with dependent = true may start while its predecessor in the stream
+// is still running; it must call grid_dependency_wait() before it touches anything an earlier kernel writes (what it
+// reads before that must be constant for the whole chain: packed weights, tables).  grid_dependency_release() lets the
+// successor's CTAs be scheduled as soon as every CTA of this grid has issued it or exited.  Both are no-ops in a launch
+// without the attribute, so kernels shared with the training step carry them at no cost.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool dependent,
+                                 Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------------------
 // Launch functions (host).  Every pointer is device memory.
 // ---------------------------------------------------------------------------
@@ -83,11 +109,14 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 // Smoothing of Section 4.2 on the activation side (smooth may be NULL): the quantiser sees (x - shift') * (1 / scale')
 // with the vectors of launch_smooth_perturb; rows [0, rows_per_pass) use sign 0, the rest sign 1.
 struct SmoothAct { const float* smooth = nullptr; int ld = 0; int64_t rows_per_pass = 0; };
+// planes = true (a_bits != 0, cols % 32 == 0): the operand row holds, instead of bf16 codes, the integer form the
+// decode-time matrix-vector kernels read (int8 codes of even columns, of odd columns, int32 sums of every 32 codes).
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
-                             SmoothAct sm = SmoothAct());
+                             SmoothAct sm = SmoothAct(), bool dependent = false, bool planes = false);
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
-                            __nv_bfloat16* op, float* row_step, cudaStream_t s, SmoothAct sm = SmoothAct());
+                            __nv_bfloat16* op, float* row_step, cudaStream_t s, SmoothAct sm = SmoothAct(),
+                            bool dependent = false, bool planes = false);
 // Activation operand of rows whose max |x| is already known (amax: bits of a non-negative float per row).
 void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits,
                          __nv_bfloat16* op, float* row_step, cudaStream_t s);
@@ -107,6 +136,7 @@ int launch_attention_tc(const float* qkv, int batch, int seq, int n_heads, int d
 // (unsupported shape: K % 32, group, batch not in {1, 2, 4, 8}).
 void launch_repack_nibbles(const uint32_t* packed, int64_t n, int bits, void* out, cudaStream_t s);
 void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t s);
+void launch_codes_to_planes(const __nv_bfloat16* codes, int rows, int K, void* planes, cudaStream_t s);
 int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
                        const float* row_step, const float* bias, int accumulate, float* out, cudaStream_t s);
 // weight-only models: act = bf16(x) [mb, K], operands bf16((c - z) * Delta) as in the training forward

@@ -47,9 +47,41 @@ __global__ void to_bf16_kernel(const float4* __restrict__ src, uint2* __restrict
 }
 
 // ---- matrix-vector product over nibble codes --------------------------------------------------------------------
-// act: bf16 integer codes [MB, K] (as the activation-operand kernels write them) with their steps row_step[MB].
-// Shared memory: per sequence the even-k and odd-k codes as int8 (so that four consecutive bytes pair with the low / high
-// nibbles of one weight word) and the sum of the codes of every 32-element chunk (for the zero-point term).
+// act: [MB] operand rows of 2 * K bytes in their integer form (the activation-operand kernels write it with planes = 1):
+// int8 codes of even k [K / 2], of odd k [K / 2] (so that four consecutive bytes pair with the low / high nibbles of one
+// weight word), int32 sums of the codes of every 32-element chunk [K / 32] (for the zero-point term); steps row_step[MB].
+// Shared memory holds the same three arrays for all MB rows.
+// bf16 integer codes [rows, K] -> the integer form described below, rows of 2 * K bytes (one CTA per row).
+__global__ void __launch_bounds__(256)
+codes_to_planes_kernel(const __nv_bfloat16* __restrict__ codes, int K, uint8_t* __restrict__ planes) {
+    const __nv_bfloat16* src = codes + (size_t)blockIdx.x * K;
+    uint8_t* row = planes + (size_t)blockIdx.x * 2 * K;
+    uint16_t* even = reinterpret_cast<uint16_t*>(row);
+    uint16_t* odd = reinterpret_cast<uint16_t*>(row + (K >> 1));
+    int32_t* csum = reinterpret_cast<int32_t*>(row + K);
+    const int n4 = K >> 2;
+    for (int base = 0; base < n4; base += 256) {               // whole warps run every round (shuffles below)
+        const int idx = base + threadIdx.x;
+        const bool live = idx < n4;
+        int c[4] = {0, 0, 0, 0};
+        if (live) {
+            const uint2 v = __ldg(reinterpret_cast<const uint2*>(src) + idx);
+            const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+            const float2 a = __bfloat1622float2(p2[0]), b = __bfloat1622float2(p2[1]);
+            c[0] = (int)a.x; c[1] = (int)a.y; c[2] = (int)b.x; c[3] = (int)b.y;
+        }
+        int sum = c[0] + c[1] + c[2] + c[3];
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (live) {
+            even[idx] = (uint16_t)(((uint32_t)c[0] & 0xFFu) | (((uint32_t)c[2] & 0xFFu) << 8));
+            odd[idx] = (uint16_t)(((uint32_t)c[1] & 0xFFu) | (((uint32_t)c[3] & 0xFFu) << 8));
+            if ((idx & 7) == 0) csum[idx >> 3] = sum;
+        }
+    }
+}
+
 template <int MB>
 __global__ void __launch_bounds__(kGemvThreads)
 decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qparams, int N, int K, int group_shift,
@@ -75,36 +107,18 @@ decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qpar
             if (ch < chunks) { w[u] = __ldg(wq + (size_t)n * chunks + ch); qp[u] = __ldg(qparams + (size_t)n * gpr + (ch >> cshift)); }
         }
     }
-    // staging: a thread converts 8 bf16 codes (one 16-byte load) into 4 even and 4 odd int8; the four threads of a
-    // chunk add up their code sums
+    grid_dependency_wait();                    // the packed weights are constant; everything below reads the preceding kernels' output
+    // staging: the rows' integer form (written by the activation-operand kernels) is copied as it is
     {
-        uint32_t* even1 = reinterpret_cast<uint32_t*>(even4);
-        uint32_t* odd1 = reinterpret_cast<uint32_t*>(odd4);
-        const int per_row = K >> 3;
-        const int total = MB * per_row;
-        // every thread of the CTA runs every round (the shuffles below need whole warps); loads and stores are guarded
-        for (int base = 0; base < total; base += kGemvThreads) {
-            const int i = base + threadIdx.x;
-            const bool live = i < total;
-            uint32_t e = 0, o = 0;
-            int sum = 0;
-            if (live) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4*>(act) + i);
-                const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float2 f = __bfloat1622float2(p2[q]);
-                    const int a0 = (int)f.x, a1 = (int)f.y;
-                    sum += a0 + a1;
-                    e |= ((uint32_t)a0 & 0xFFu) << (8 * q);
-                    o |= ((uint32_t)a1 & 0xFFu) << (8 * q);
-                }
-                even1[i] = e;
-                odd1[i] = o;
-            }
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            if (live && (i & 3) == 0) csum[i >> 2] = sum;      // total is a multiple of 4: quads are whole
+        const int row16 = K >> 3;              // 16-byte words of one operand row (2 * K bytes)
+        for (int i = threadIdx.x; i < MB * 2 * chunks; i += kGemvThreads) {
+            const int m = i / (2 * chunks), c = i - m * 2 * chunks;
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(act) + (size_t)m * row16 + c);
+            if (c < chunks) even4[m * chunks + c] = v; else odd4[m * chunks + c - chunks] = v;
+        }
+        for (int i = threadIdx.x; i < MB * chunks; i += kGemvThreads) {
+            const int m = i / chunks, c = i - m * chunks;
+            csum[i] = __ldg(reinterpret_cast<const int32_t*>(act + (size_t)m * K + (K >> 1)) + c);
         }
     }
     __syncthreads();
@@ -161,6 +175,9 @@ decode_gemv_kernel(const uint4* __restrict__ wq, const float2* __restrict__ qpar
             }
         }
     }
+    // the successor is scheduled while the last CTAs drain; released earlier, waiting CTAs of later kernels would take
+    // residency slots and skew the distribution of this grid over the SMs
+    grid_dependency_release();
 }
 
 // ---- attention over the cache -----------------------------------------------------------------------------------
@@ -176,6 +193,7 @@ decode_gemv_fp_kernel(const uint4* __restrict__ wq, const float2* __restrict__ q
     uint4* xs = reinterpret_cast<uint4*>(smem);                            // [MB][K] bf16, 8 per uint4
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int chunks = K >> 5, gpr = K >> group_shift, cshift = group_shift - 5;
+    grid_dependency_wait();
     for (int i = threadIdx.x; i < MB * (K >> 3); i += kGemvThreads) xs[i] = __ldg(reinterpret_cast<const uint4*>(act) + i);
     __syncthreads();
     for (int n = blockIdx.x * (kGemvThreads / 32) + warp; n < N; n += gridDim.x * (kGemvThreads / 32)) {
@@ -237,6 +255,9 @@ decode_gemv_fp_kernel(const uint4* __restrict__ wq, const float2* __restrict__ q
             }
         }
     }
+    // the successor is scheduled while the last CTAs drain; released earlier, waiting CTAs of later kernels would take
+    // residency slots and skew the distribution of this grid over the SMs
+    grid_dependency_release();
 }
 
 // cache_k / cache_v: fp32 [B][H][max_len][dh] of one layer.
@@ -254,6 +275,8 @@ decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cach
     constexpr int VPL = DH / 32;               // features per lane
     extern __shared__ float sc[];              // scores / probabilities of positions 0..pos, then [8][DH] partial outputs
     __shared__ float red[8];
+    grid_dependency_release();
+    grid_dependency_wait();
     const int b = blockIdx.y, h = blockIdx.x, d = n_heads * DH;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float* part = sc + ((pos + 1 + 3) & ~3);
@@ -367,6 +390,7 @@ decode_head_kernel(const uint4* __restrict__ w, int V, int d, const __nv_bfloat1
     extern __shared__ __align__(16) uint8_t smem[];
     __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(smem);            // [MB][d]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    grid_dependency_wait();
     for (int i = threadIdx.x; i < MB * d; i += kGemvThreads) xs[i] = x[i];
     __syncthreads();
     const int chunks = d / 8;
@@ -396,6 +420,9 @@ decode_head_kernel(const uint4* __restrict__ w, int V, int d, const __nv_bfloat1
             if (lane == 0) logits[(size_t)m * V + v] = acc[m];
         }
     }
+    // the successor is scheduled while the last CTAs drain; released earlier, waiting CTAs of later kernels would take
+    // residency slots and skew the distribution of this grid over the SMs
+    grid_dependency_release();
 }
 
 // next[m] = index of the largest logit of row m (the lowest index among equals); one CTA per row.
@@ -403,6 +430,7 @@ __global__ void __launch_bounds__(1024)
 decode_argmax_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ next) {
     __shared__ float bv[32];
     __shared__ int bi[32];
+    grid_dependency_wait();
     const float* row = logits + (size_t)blockIdx.x * V;
     float best = -INFINITY;
     int idx = 0x7fffffff;
@@ -452,6 +480,11 @@ void launch_to_bf16(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_
 
 size_t decode_gemv_smem_bytes(int mb, int K) { return (size_t)mb * K + (size_t)mb * (K / 32) * 4; }
 
+void launch_codes_to_planes(const __nv_bfloat16* codes, int rows, int K, void* planes, cudaStream_t s) {
+    codes_to_planes_kernel<<<rows, 256, 0, s>>>(codes, K, static_cast<uint8_t*>(planes));
+    count_launch();
+}
+
 int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
                        const float* row_step, const float* bias, int accumulate, float* out, cudaStream_t s) {
     if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
@@ -465,7 +498,7 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     {                                                                                                                     \
         static bool attr = false;                                                                                         \
         if (!attr) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
-        decode_gemv_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, row_step, bias, accumulate, out); \
+        launch_kernel(decode_gemv_kernel<MBV>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, qparams, N, K, gshift, act, row_step, bias, accumulate, out); \
     }
     if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else if (mb == 8) ZQ_GEMV(8) else return -1;
 #undef ZQ_GEMV
@@ -485,7 +518,7 @@ int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, i
     {                                                                                                                     \
         static bool attr = false;                                                                                         \
         if (!attr) { cudaFuncSetAttribute(decode_gemv_fp_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
-        decode_gemv_fp_kernel<MBV><<<grid, kGemvThreads, smem, s>>>(w4, qparams, N, K, gshift, act, bias, accumulate, out); \
+        launch_kernel(decode_gemv_fp_kernel<MBV>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, qparams, N, K, gshift, act, bias, accumulate, out); \
     }
     if (mb == 1) ZQ_GEMV_FP(1) else if (mb == 2) ZQ_GEMV_FP(2) else if (mb == 4) ZQ_GEMV_FP(4) else if (mb == 8) ZQ_GEMV_FP(8) else return -1;
 #undef ZQ_GEMV_FP
@@ -502,8 +535,8 @@ void launch_decode_attention(const float* q, float* cache_k, float* cache_v, int
         cudaFuncSetAttribute(decode_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
         attr = true;
     }
-    if (dh == 64) decode_attention_kernel<64><<<dim3(n_heads, batch), 256, smem, s>>>(q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
-    else decode_attention_kernel<128><<<dim3(n_heads, batch), 256, smem, s>>>(q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
+    if (dh == 64) launch_kernel(decode_attention_kernel<64>, dim3(dim3(n_heads, batch)), dim3(256), smem, s, true, q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
+    else launch_kernel(decode_attention_kernel<128>, dim3(dim3(n_heads, batch)), dim3(256), smem, s, true, q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
     count_launch();
 }
 
@@ -512,20 +545,20 @@ int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_
     const size_t smem = (size_t)mb * d * 2;
     const int grid = capped_blocks(V, kGemvThreads / 32, 148 * 4);
     const uint4* w4 = reinterpret_cast<const uint4*>(w);
-    if (mb == 1) decode_head_kernel<1><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
-    else if (mb == 2) decode_head_kernel<2><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
-    else if (mb == 4) decode_head_kernel<4><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+    if (mb == 1) launch_kernel(decode_head_kernel<1>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
+    else if (mb == 2) launch_kernel(decode_head_kernel<2>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
+    else if (mb == 4) launch_kernel(decode_head_kernel<4>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
     else if (mb == 8) {
         static bool attr = false;
         if (!attr) { cudaFuncSetAttribute(decode_head_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        decode_head_kernel<8><<<grid, kGemvThreads, smem, s>>>(w4, V, d, x, logits);
+        launch_kernel(decode_head_kernel<8>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
     } else return -1;
     count_launch();
     return 0;
 }
 
 void launch_decode_argmax(const float* logits, int batch, int V, int32_t* next, cudaStream_t s) {
-    decode_argmax_kernel<<<batch, 1024, 0, s>>>(logits, V, next);
+    launch_kernel(decode_argmax_kernel, dim3(batch), dim3(1024), 0, s, true, logits, V, next);
     count_launch();
 }
 
