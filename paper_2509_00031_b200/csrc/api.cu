@@ -1438,7 +1438,7 @@ int zoqat_decode_step(zoqat_model_t* m, const int32_t* tokens_dev, int pos, floa
         launch_norm_act_operand(w.h, B, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B], c.norm_eps,
                                 c.a_bits, w.xa, w.row_step, nullptr, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_qkv, dl.q_qkv, 3 * d, d, llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d, 0, w.qkv)) return rc;
-        launch_decode_attention(nullptr, dl.cache_k, dl.cache_v, B, H, dh, pos, D.max_len, w.att, w.qkv,
+        launch_decode_attention(dl.cache_k, dl.cache_v, B, H, dh, pos, D.max_len, w.att, w.qkv,
                                 llama ? w.rope_cos : nullptr, llama ? w.rope_sin : nullptr, s);
         launch_norm_act_operand(w.att, B, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, SmoothAct(), true, planes);
         if (int rc = gemv(dl.w_o, dl.q_o, d, d, Ly.vec[ZOQAT_ROLE_BO], 1, w.h)) return rc;

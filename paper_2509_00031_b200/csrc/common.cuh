@@ -142,9 +142,10 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
 // weight-only models: act = bf16(x) [mb, K], operands bf16((c - z) * Delta) as in the training forward
 int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, int group, int mb, const __nv_bfloat16* act,
                           const float* bias, int accumulate, float* out, cudaStream_t s);
-// qkv != NULL: q | k | v of the new token, fp32 [batch, 3*d]: rotated (cos_t / sin_t or none), k and v appended at `pos`.
-void launch_decode_attention(const float* q, float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos,
-                             int max_len, float* out, const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s);
+// qkv: q | k | v of the new token, fp32 [batch, 3*d]: rotated (cos_t / sin_t or none), k and v appended at `pos`; rows
+// [0, pos) of the cache must be complete before the preceding kernel in the stream was launched.
+void launch_decode_attention(float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos, int max_len, float* out,
+                             const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s);
 int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_bfloat16* x, float* logits, cudaStream_t s);
 void launch_decode_argmax(const float* logits, int batch, int V, int32_t* next, cudaStream_t s);
 

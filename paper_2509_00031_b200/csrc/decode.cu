@@ -261,30 +261,40 @@ decode_gemv_fp_kernel(const uint4* __restrict__ wq, const float2* __restrict__ q
 }
 
 // cache_k / cache_v: fp32 [B][H][max_len][dh] of one layer.
-// out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA of 8 warps per (sequence, head).  Warp s takes
-// the cached positions t = s, s + 8, ...: a lane holds 4 (d_head 128) or 2 (d_head 64) features, so one load instruction
-// of the warp reads a whole cached row; scores are reduced by shuffles, the output partial sums of the 8 warps through
-// shared memory.
-// qkv != NULL: the CTA first rotates the new q and k by the angle of `pos` (cos_t / sin_t, or none), appends k and v to
-// the cache at `pos` and uses the rotated q (q_in is then ignored) - the work of decode_rope_cache_kernel, in the same launch.
+// out[b, h*dh + :] = softmax(q . K[0..pos] / sqrt(dh)) V[0..pos]; one CTA of 8 warps per (sequence, head).  The CTA first
+// rotates the new q and k (qkv: fp32 [B, 3*d] of this step) by the angle of `pos` (cos_t / sin_t, or none) and appends k
+// and v to the cache at `pos`.  Warp s then takes the cached positions t = s, s + 8, ... < pos, eight at a time with both
+// their key and value rows in flight: a lane holds 4 (d_head 128) or 2 (d_head 64) features, so one load instruction of
+// the warp reads a whole cached row.  Each warp keeps a running maximum, sum and weighted value sum (one pass over the
+// cache); warp 0 also takes the new position from shared memory; the 8 partial results are merged through shared memory.
+// The rows of earlier positions were written by earlier steps, so the first eight of every warp are requested before the
+// wait on the preceding kernel.
 template <int DH>
 __global__ void __launch_bounds__(256)
-decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cache_k, float* __restrict__ cache_v,
-                        int n_heads, int pos, int max_len, float* __restrict__ out, const float* __restrict__ qkv,
-                        const float* __restrict__ cos_t, const float* __restrict__ sin_t) {
+decode_attention_kernel(float* __restrict__ cache_k, float* __restrict__ cache_v, int n_heads, int pos, int max_len,
+                        float* __restrict__ out, const float* __restrict__ qkv, const float* __restrict__ cos_t,
+                        const float* __restrict__ sin_t) {
     constexpr int VPL = DH / 32;               // features per lane
-    extern __shared__ float sc[];              // scores / probabilities of positions 0..pos, then [8][DH] partial outputs
-    __shared__ float red[8];
+    __shared__ float qs[DH], ks[DH], vs[DH];   // rotated q and k, and v, of the new position
+    __shared__ float part[8][DH];
+    __shared__ float wmax[8], wsum[8];
     grid_dependency_release();
-    grid_dependency_wait();
     const int b = blockIdx.y, h = blockIdx.x, d = n_heads * DH;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float* part = sc + ((pos + 1 + 3) & ~3);
     float* kc = cache_k + ((size_t)b * n_heads + h) * max_len * DH;
     float* vc = cache_v + ((size_t)b * n_heads + h) * max_len * DH;
-    float q[VPL];
-    if (qkv) {
-        float* qs = part;                      // the rotated q passes through the (not yet used) partial-sum area
+    float kr[8][VPL], vr[8][VPL];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int t = warp + 8 * u;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            kr[u][j] = t < pos ? kc[(size_t)t * DH + lane * VPL + j] : 0.0f;
+            vr[u][j] = t < pos ? vc[(size_t)t * DH + lane * VPL + j] : 0.0f;
+        }
+    }
+    grid_dependency_wait();                    // qkv comes from the preceding kernel
+    {
         const float* qn = qkv + (size_t)b * 3 * d + h * DH;
         const float* kn = qn + d;
         const float* vn = qn + 2 * d;
@@ -294,90 +304,91 @@ decode_attention_kernel(const float* __restrict__ q_in, float* __restrict__ cach
             if (cos_t) { c = cos_t[(size_t)pos * HD + i]; s = sin_t[(size_t)pos * HD + i]; }
             const float q1 = qn[i], q2 = qn[i + HD], k1 = kn[i], k2 = kn[i + HD];
             qs[i] = q1 * c - q2 * s; qs[i + HD] = q2 * c + q1 * s;
-            kc[(size_t)pos * DH + i] = k1 * c - k2 * s; kc[(size_t)pos * DH + i + HD] = k2 * c + k1 * s;
+            const float ka = k1 * c - k2 * s, kb = k2 * c + k1 * s;
+            ks[i] = ka; ks[i + HD] = kb;
+            kc[(size_t)pos * DH + i] = ka; kc[(size_t)pos * DH + i + HD] = kb;
         }
-        for (int i = threadIdx.x; i < DH; i += 256) vc[(size_t)pos * DH + i] = vn[i];
-        __syncthreads();                       // the new cache row and q are visible to the whole CTA
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) q[j] = qs[lane * VPL + j];
-        __syncthreads();
-    } else {
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) q[j] = q_in[(size_t)b * d + h * DH + lane * VPL + j];
+        for (int i = threadIdx.x; i < DH; i += 256) { const float v = vn[i]; vs[i] = v; vc[(size_t)pos * DH + i] = v; }
     }
+    __syncthreads();
+    float q[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) q[j] = qs[lane * VPL + j];
     const float scale = 1.0f / sqrtf((float)DH);
-    float mx = -INFINITY;
-    for (int t0 = warp; t0 <= pos; t0 += 64) {                 // eight positions of this warp in flight
+    float mx = -INFINITY, sum = 0.0f, acc[VPL];
+#pragma unroll
+    for (int j = 0; j < VPL; ++j) acc[j] = 0.0f;
+    for (int t0 = warp; t0 < pos; t0 += 64) {
+        if (t0 != warp) {                      // the first eight rows are already in registers
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int t = t0 + 8 * u;
+#pragma unroll
+                for (int j = 0; j < VPL; ++j) {
+                    kr[u][j] = t < pos ? kc[(size_t)t * DH + lane * VPL + j] : 0.0f;
+                    vr[u][j] = t < pos ? vc[(size_t)t * DH + lane * VPL + j] : 0.0f;
+                }
+            }
+        }
         float a[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int t = t0 + 8 * u;
             a[u] = 0.0f;
-            if (t <= pos) {
 #pragma unroll
-                for (int j = 0; j < VPL; ++j) a[u] = __fmaf_rn(q[j], kc[(size_t)t * DH + lane * VPL + j], a[u]);
-            }
+            for (int j = 0; j < VPL; ++j) a[u] = __fmaf_rn(q[j], kr[u][j], a[u]);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
             for (int u = 0; u < 8; ++u) a[u] += __shfl_xor_sync(0xffffffffu, a[u], o);
         }
+        float m_new = mx;                      // t0 < pos: the first row of the round is valid, so m_new becomes finite
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int t = t0 + 8 * u;
-            if (t <= pos) {
-                a[u] *= scale;
-                if (lane == 0) sc[t] = a[u];
-                mx = fmaxf(mx, a[u]);
-            }
+            a[u] = t0 + 8 * u < pos ? a[u] * scale : -INFINITY;
+            m_new = fmaxf(m_new, a[u]);
         }
+        const float corr = expf(mx - m_new);   // 0 on the first round (mx = -inf)
+        sum *= corr;
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) acc[j] *= corr;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float p = expf(a[u] - m_new);                // 0 for rows beyond the cache
+            sum += p;
+#pragma unroll
+            for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p, vr[u][j], acc[j]);
+        }
+        mx = m_new;
     }
-    if (lane == 0) red[warp] = mx;
-    __syncthreads();
-    mx = red[0];
+    if (warp == 0) {                           // the new position
+        float a = 0.0f;
 #pragma unroll
-    for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
-    __syncthreads();
-    float sum = 0.0f;
-    for (int t = threadIdx.x; t <= pos; t += 256) { const float p = expf(sc[t] - mx); sc[t] = p; sum += p; }
+        for (int j = 0; j < VPL; ++j) a = __fmaf_rn(q[j], ks[lane * VPL + j], a);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) red[warp] = sum;
-    __syncthreads();
-    float total = 0.0f;
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        a *= scale;
+        const float m_new = fmaxf(mx, a);
+        const float corr = expf(mx - m_new), p = expf(a - m_new);
+        sum = sum * corr + p;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) total += red[i];
-    float acc[VPL];
-#pragma unroll
-    for (int j = 0; j < VPL; ++j) acc[j] = 0.0f;
-    for (int t0 = warp; t0 <= pos; t0 += 64) {                 // eight cached rows of this warp in flight
-        float v[8][VPL], p[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int t = t0 + 8 * u;
-            p[u] = 0.0f;
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) v[u][j] = 0.0f;
-            if (t <= pos) {
-                p[u] = sc[t];
-#pragma unroll
-                for (int j = 0; j < VPL; ++j) v[u][j] = vc[(size_t)t * DH + lane * VPL + j];
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-#pragma unroll
-            for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p[u], v[u][j], acc[j]);
-        }
+        for (int j = 0; j < VPL; ++j) acc[j] = __fmaf_rn(p, vs[lane * VPL + j], acc[j] * corr);
+        mx = m_new;
     }
 #pragma unroll
-    for (int j = 0; j < VPL; ++j) part[warp * DH + lane * VPL + j] = acc[j];
+    for (int j = 0; j < VPL; ++j) part[warp][lane * VPL + j] = acc[j];
+    if (lane == 0) { wmax[warp] = mx; wsum[warp] = sum; }
     __syncthreads();
+    float top = wmax[0];                       // finite: warp 0 holds the new position
+#pragma unroll
+    for (int w = 1; w < 8; ++w) top = fmaxf(top, wmax[w]);
+    float total = 0.0f, f[8];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { f[w] = expf(wmax[w] - top); total = __fmaf_rn(f[w], wsum[w], total); }   // 0 for a warp without rows
     for (int i = threadIdx.x; i < DH; i += 256) {
         float o = 0.0f;
 #pragma unroll
-        for (int s8 = 0; s8 < 8; ++s8) o += part[s8 * DH + i];
+        for (int w = 0; w < 8; ++w) o = __fmaf_rn(f[w], part[w][i], o);
         out[(size_t)b * d + h * DH + i] = o / total;
     }
 }
@@ -526,17 +537,10 @@ int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, i
     return 0;
 }
 
-void launch_decode_attention(const float* q, float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos,
-                             int max_len, float* out, const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s) {
-    const size_t smem = (size_t)(((pos + 1 + 3) & ~3) + 8 * dh) * 4;
-    static bool attr = false;
-    if (!attr) {
-        cudaFuncSetAttribute(decode_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        cudaFuncSetAttribute(decode_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
-        attr = true;
-    }
-    if (dh == 64) launch_kernel(decode_attention_kernel<64>, dim3(dim3(n_heads, batch)), dim3(256), smem, s, true, q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
-    else launch_kernel(decode_attention_kernel<128>, dim3(dim3(n_heads, batch)), dim3(256), smem, s, true, q, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
+void launch_decode_attention(float* cache_k, float* cache_v, int batch, int n_heads, int dh, int pos, int max_len, float* out,
+                             const float* qkv, const float* cos_t, const float* sin_t, cudaStream_t s) {
+    if (dh == 64) launch_kernel(decode_attention_kernel<64>, dim3(n_heads, batch), dim3(256), 0, s, true, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
+    else launch_kernel(decode_attention_kernel<128>, dim3(n_heads, batch), dim3(256), 0, s, true, cache_k, cache_v, n_heads, pos, max_len, out, qkv, cos_t, sin_t);
     count_launch();
 }
 
