@@ -102,6 +102,56 @@ def test_cached_decode_matches_oracle_forward(zq, name, batch, seq):
     assert total > 0 and agree == total
 
 
+@pytest.mark.parametrize("name,batch", [("llama_w4a8", 2), ("opt_w3", 1)])
+def test_greedy_decode_from_a_captured_graph_equals_eager_launches(zq, name, batch):
+    """A loop of steps (each kernel a programmatic dependent of the one before) is captured once and replayed: the
+    tokens and the last logits must be those of the same steps launched one by one."""
+    shape = SHAPES[name]
+    ctx, new = 9, 6
+    seq = ctx + new
+    params = synth.make_params(shape, seed=8, max_seq=seq, jitter=True)
+    L = shape["n_layers"]
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, first_trainable_layer=L,
+                          head_trainable=False, packed_frozen=True)
+    model.zoqat_prequantize_frozen()
+    tokens, _ = synth.make_batch(batch, ctx, shape["vocab"], seed=4)
+
+    def run(captured):
+        model.zoqat_decode_begin(batch, seq)
+        nxt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+        for pos in range(ctx):
+            model.zoqat_decode_step(dev(tokens[:, pos].copy()), pos, next_token=nxt, want_logits=False)
+        out = torch.zeros((new, batch), dtype=torch.int32, device="cuda")
+        logits = torch.zeros((batch, shape["vocab"]), dtype=torch.float32, device="cuda")
+
+        def steps():
+            for t in range(new):
+                model.zoqat_decode_step(nxt, ctx + t, logits=logits, next_token=nxt)
+                out[t].copy_(nxt)
+
+        if captured:
+            graph = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    steps()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graph.replay()
+        else:
+            steps()
+        torch.cuda.synchronize()
+        model.zoqat_check()
+        return out.cpu().numpy(), logits.cpu().numpy()
+
+    eager_tokens, eager_logits = run(False)
+    graph_tokens, graph_logits = run(True)
+    assert np.array_equal(eager_tokens, graph_tokens)
+    assert np.array_equal(eager_logits, graph_logits)
+    assert np.isfinite(eager_logits).all()
+
+
 def test_decode_rejects_models_that_are_not_packed(zq):
     shape = SHAPES["llama_w4a8"]
     params = synth.make_params(shape, seed=5, max_seq=16)
