@@ -480,8 +480,12 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
  * The deployment side of the method (the paper's on-device tokens-per-second table): one new
  * token per sequence and call, keys and values cached, every block linear read once per
  * token as stored low-bit codes.  Needs a model whose block linears are all FROZEN_PACKED
- * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups; batch in {1, 2, 4, 8}
- * sequences advance in lock step.
+ * (zoqat_prequantize_frozen() done), w_bits <= 4 with column groups, d_model and d_ffn
+ * multiples of 32 (ZOQAT_ERR_UNSUPPORTED otherwise); batch in {1, 2, 4, 8} sequences advance
+ * in lock step.  The kernels of a step are launched as programmatic dependents of one
+ * another (each may start while its predecessor drains and reads only constant data until
+ * the predecessor has completed); the first kernel of a step is an ordinary launch, so a step
+ * is ordered after all earlier work of the stream as usual.
  *
  * Arithmetic: a packed linear is evaluated as an integer runtime does,
  *     y[t, n] = s_t * sum_g Delta[n, g] * ( sum_{k in g} a[t, k] * (c[n, k] - z[n, g]) ) (+ bias),

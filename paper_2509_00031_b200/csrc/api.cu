@@ -1318,6 +1318,7 @@ int decode_sizes(const zoqat_model* m, int batch, int max_len, DecodeSizes& z) {
     if (max_len <= 0 || max_len > c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "max_len %d must be in 1..max_seq (%d)", max_len, c.max_seq);
     if (batch > c.max_batch * c.max_seq) return fail(ZOQAT_ERR_INVALID_ARG, "batch exceeds the workspace");
     if (c.w_group == 0 || c.w_bits > 4) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs column groups of 32, 64 or 128 and w_bits <= 4");
+    if (c.d_model % 32 || c.d_ffn % 32) return fail(ZOQAT_ERR_UNSUPPORTED, "decode needs d_model and d_ffn to be multiples of 32");
     const size_t d = c.d_model, F = c.d_ffn, n_up = c.arch == ZOQAT_ARCH_LLAMA ? 2 * F : F;
     z.nib[0] = align_up(3 * d * d / 2); z.nib[1] = align_up(d * d / 2); z.nib[2] = align_up(n_up * d / 2); z.nib[3] = align_up(d * F / 2);
     z.qp_qkv = align_up(3 * d * (d / c.w_group) * 8);
