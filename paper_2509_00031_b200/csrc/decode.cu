@@ -501,8 +501,9 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     if (N <= 0 || K <= 0 || K % 32 || K % group || (group != 32 && group != 64 && group != 128)) return -1;
     const size_t smem = decode_gemv_smem_bytes(mb, K);
     if (smem > 160 * 1024) return -1;
-    // every CTA stages the activation codes of all sequences: more sequences, fewer and longer-lived CTAs (measured)
-    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 8 : (mb == 2 ? 4 : (mb == 4 ? 3 : 2))));
+    // every CTA stages the activation codes of all sequences: more sequences, fewer and longer-lived CTAs (measured);
+    // 5 per SM is what 48 registers per thread keep resident
+    const int grid = capped_blocks(N, kGemvThreads / 32, 148 * (mb == 1 ? 5 : (mb == 2 ? 4 : (mb == 4 ? 3 : 2))));
     const int gshift = group == 32 ? 5 : (group == 64 ? 6 : 7);
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV(MBV)                                                                                                      \
