@@ -245,9 +245,10 @@ __device__ __forceinline__ void smooth_regs(float4 (&v)[VPT], int n4, const Smoo
 }
 
 // (rows of up to 4096 columns: held to 40 registers so that six CTAs share an SM; 8192 x 4096 rows in 43 us against 49 us
-// with four.  Up to 8192 columns: 64 registers, four CTAs instead of two at 128; 8192 x 5120 in 57 us against 143 us.)
+// with four.  Up to 8192 columns: 64 registers, four CTAs instead of two at 128; 8192 x 5120 in 57 us against 143 us.
+// Up to 12288 columns: 80 registers with a few spilled values, three CTAs instead of two; 8192 x 12288 in 102 us against 197 us.)
 template <int VPT>
-__global__ void __launch_bounds__(kRowThreads, VPT == 4 ? 6 : (VPT == 8 ? 4 : 1))
+__global__ void __launch_bounds__(kRowThreads, VPT == 4 ? 6 : (VPT == 8 ? 4 : 3))
 norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind, const float* __restrict__ gain,
                             const float* __restrict__ bias, float norm_eps, int a_bits, __nv_bfloat16* __restrict__ op,
                             float* __restrict__ row_step, float* __restrict__ normed, SmoothAct sm, int planes) {
