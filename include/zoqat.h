@@ -295,6 +295,23 @@ int zoqat_profile_read(zoqat_model_t* m, int category, double* ms, int64_t* inte
 #define ZOQAT_BUF_TOKEN_LOSS 4   /* fp32 [passes*T]            per-position cross-entropy            */
 int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* bytes);
 
+/* Parity hook for the activation quantisers as a whole forward runs them (Section 2 symmetric form, Appendix
+ * "Quantization settings": per-token activation quantisation at the input of every block linear).  While a capture
+ * buffer is set, every forward copies, at each of the four quantisation points of each layer (attn_in, attn_out,
+ * ffn_in, ffn_out) and in execution order, one record into `buf_dev`:
+ *   input   fp32 [rows, cols]   the value the quantiser saw (after the norm / non-linearity, before the Section 4.2
+ *                               shift and scale if the layer has them)
+ *   operand bf16 [rows, cols]   what the quantiser wrote for the GEMM (integer codes, or bf16(x) when a_bits = 0)
+ *   step    fp32 [rows]         the per-token step
+ * each part padded to a multiple of 256 bytes; rows = passes * batch * seq as materialised at that layer (a frozen
+ * prefix is evaluated once: rows = batch * seq there), cols = d_model (d_ffn at ffn_out).  One more record follows
+ * the last layer: the final norm's output, its bf16 rounding (the vocabulary projection's operand) and steps of 1,
+ * rows = passes * batch * seq, cols = d_model.  A forward that would
+ * overrun `bytes` fails with ZOQAT_ERR_WORKSPACE_SMALL before launching anything.  buf_dev = NULL switches the hook
+ * off.  The caller owns the buffer; zoqat_debug_capture_bytes gives the size one forward of `passes` passes needs. */
+int zoqat_debug_capture(zoqat_model_t* m, void* buf_dev, size_t bytes);
+int zoqat_debug_capture_bytes(const zoqat_model_t* m, int batch, int seq, int passes, size_t* bytes);
+
 const char* zoqat_status_string(int status);
 const char* zoqat_last_error(void);
 

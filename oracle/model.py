@@ -392,6 +392,7 @@ class OracleModel:
             h = self._store(h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo")))
             self._tap(f"l{l}.h_mid", h)
             x = self.norm(h, P["ffn_norm_g"], P.get("ffn_norm_b"))
+            self._tap(f"l{l}.ffn_norm", x)
             if cfg.arch == "llama":
                 gate = self.lin(x, l, "w_gate", seed, signed_eps)
                 up = self.lin(x, l, "w_up", seed, signed_eps)

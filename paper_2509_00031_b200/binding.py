@@ -29,7 +29,7 @@ EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
     "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_finish_deferred", "zoqat_flush_update", "zoqat_step_multi",
     "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates",
-    "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_status_string", "zoqat_last_error",
+    "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_debug_capture", "zoqat_debug_capture_bytes", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
@@ -107,6 +107,8 @@ def lib():
             "zoqat_check": [vp, vp],
             "zoqat_launch_count": [vp, P(i64)],
             "zoqat_debug_buffer": [vp, i32, P(vp), P(sz)],
+            "zoqat_debug_capture": [vp, vp, sz],
+            "zoqat_debug_capture_bytes": [vp, i32, i32, i32, P(sz)],
             "zoqat_profile_enable": [vp, i32],
             "zoqat_profile_read": [vp, i32, P(ctypes.c_double), P(i64), vp],
             "zoqat_op_philox_words": [u64, u32, u64, u64, vp, vp],
@@ -574,6 +576,37 @@ class ZoqatModel:
         _check(lib().zoqat_debug_buffer(self.handle, which, ctypes.byref(ptr), ctypes.byref(nb)))
         off = ptr.value - self.workspace.data_ptr()
         return self.workspace[off:off + nb.value].view(dtype)
+
+
+    def zoqat_debug_capture(self, batch, seq, passes=1):
+        """Switches the quantiser capture on for forwards of this size (the buffer is allocated here and kept alive
+        by this object); passes = 0 switches it off.  Returns the buffer (uint8) or None."""
+        if passes == 0:
+            _check(lib().zoqat_debug_capture(self.handle, None, 0))
+            self.capture_buffer = None
+            return None
+        nb = ctypes.c_size_t()
+        _check(lib().zoqat_debug_capture_bytes(self.handle, batch, seq, passes, ctypes.byref(nb)))
+        self.capture_buffer = torch.zeros(nb.value, dtype=torch.uint8, device="cuda")
+        _check(lib().zoqat_debug_capture(self.handle, _p(self.capture_buffer), nb.value))
+        return self.capture_buffer
+
+    def capture_records(self, rows_per_layer):
+        """Splits the capture buffer of the last forward into records, in execution order:
+        [(layer, point, input fp32 [rows, cols], operand bf16 [rows, cols], step fp32 [rows])], rows_per_layer[l] =
+        rows materialised at layer l (passes * batch * seq; batch * seq inside a frozen prefix).  One entry more than
+        the model has layers: the last one is the final norm (layer = n_layers, point 0: the vocabulary projection's
+        bf16 operand, steps of 1)."""
+        up = lambda n: (n + 255) // 256 * 256
+        buf, off, out = self.capture_buffer, 0, []
+        for l, rows in enumerate(rows_per_layer):
+            for point in range(4 if l < self.shape["n_layers"] else 1):
+                cols = self.shape["d_ffn"] if point == 3 else self.shape["d_model"]
+                x = buf[off:off + rows * cols * 4].view(torch.float32).view(rows, cols); off += up(rows * cols * 4)
+                op = buf[off:off + rows * cols * 2].view(torch.bfloat16).view(rows, cols); off += up(rows * cols * 2)
+                st = buf[off:off + rows * 4].view(torch.float32); off += up(rows * 4)
+                out.append((l, point, x, op, st))
+        return out
 
 
 def decode_step_result(result):

@@ -153,7 +153,7 @@ norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, co
 
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                       float* __restrict__ row_step, SmoothAct sm, int planes) {
+                       float* __restrict__ row_step, SmoothAct sm, int planes, float* __restrict__ pre) {
     extern __shared__ float row[];
     __shared__ float redf[kRowThreads / 32];
     grid_dependency_release();
@@ -170,6 +170,8 @@ ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_b
         const float* g = x + r * cols;
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = fmaxf(g[c], 0.0f);
     }
+    if (pre)                         // parity hook: the value the quantiser sees (each thread copies what it wrote)
+        for (int c = threadIdx.x; c < cols; c += kRowThreads) pre[r * cols + c] = row[c];
     if (sm.smooth) {
         const float* b = smooth_base(sm, r);
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
@@ -322,7 +324,7 @@ norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind
 template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int a_bits, __nv_bfloat16* __restrict__ op,
-                           float* __restrict__ row_step, SmoothAct sm, int planes) {
+                           float* __restrict__ row_step, SmoothAct sm, int planes, float* __restrict__ pre) {
     __shared__ float redf[kRowThreads / 32];
     grid_dependency_release();
     grid_dependency_wait();       // x comes from the preceding kernel
@@ -353,6 +355,13 @@ ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int
             const int idx = threadIdx.x + i * kRowThreads;
             const float4 g = idx < n4 ? __ldcs(g4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
             v[i] = make_float4(fmaxf(g.x, 0.f), fmaxf(g.y, 0.f), fmaxf(g.z, 0.f), fmaxf(g.w, 0.f));
+        }
+    }
+    if (pre) {                       // parity hook: the value the quantiser sees
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int idx = threadIdx.x + i * kRowThreads;
+            if (idx < n4) reinterpret_cast<float4*>(pre + r * cols)[idx] = v[i];
         }
     }
     smooth_regs<VPT>(v, n4, sm, r);
@@ -423,7 +432,7 @@ __global__ void copy_kernel(const float4* __restrict__ src, float4* __restrict__
 // Per-position loss = logsumexp - logit[label] from the per-tile (max, sum exp) partials.
 __global__ void ce_token_kernel(const float2* __restrict__ partials, const float* __restrict__ label_logit,
                                 const int32_t* __restrict__ labels, int64_t M, int64_t rows, int n_tiles,
-                                float* __restrict__ token_loss) {
+                                float* __restrict__ token_loss, int64_t vocab, int32_t* __restrict__ err_flag) {
     const int64_t r = blockIdx.x * (int64_t)(blockDim.x / 32) + (threadIdx.x >> 5);
     if (r >= rows) return;
     const int lane = threadIdx.x & 31;
@@ -445,7 +454,11 @@ __global__ void ce_token_kernel(const float2* __restrict__ partials, const float
         sm = a + b;
         mx = nm;
     }
-    if (lane == 0) token_loss[r] = lab >= 0 ? (mx + logf(sm)) - label_logit[r] : 0.0f;
+    if (lane == 0) {
+        // a label beyond the vocabulary has no logit (no tile wrote label_logit[r]): report it instead of a wrong loss
+        if (lab >= vocab) { if (err_flag) atomicExch(err_flag, kErrBadLabel); token_loss[r] = 0.0f; }
+        else token_loss[r] = lab >= 0 ? (mx + logf(sm)) - label_logit[r] : 0.0f;
+    }
 }
 
 // Deterministic sum of the per-position losses of each pass (fixed tree, double).
@@ -526,28 +539,28 @@ void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_ki
         launch_kernel(norm_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+        static DeviceOnce attr;
+        if (attr.first()) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); }
         launch_kernel(norm_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
     }
     count_launch();
 }
 
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
-                            float* row_step, cudaStream_t s, SmoothAct sm, bool dependent, bool planes) {
+                            float* row_step, cudaStream_t s, SmoothAct sm, bool dependent, bool planes, float* pre) {
     const int n4 = cols / 4;
-    const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(pre)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
+        launch_kernel(ffn_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
+        launch_kernel(ffn_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
+        launch_kernel(ffn_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
-        launch_kernel(ffn_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0);
+        static DeviceOnce attr;
+        if (attr.first()) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); }
+        launch_kernel(ffn_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
     }
     count_launch();
 }
@@ -563,9 +576,10 @@ void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t*
 }
 
 void launch_ce_finalize(const float2* partials, const float* label_logit, const int32_t* labels, int64_t M, int Z,
-                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, cudaStream_t s) {
+                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, int64_t vocab, int32_t* err_flag,
+                        cudaStream_t s) {
     const int64_t rows = M * Z;
-    ce_token_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(partials, label_logit, labels, M, rows, n_tiles, token_loss);
+    ce_token_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, s>>>(partials, label_logit, labels, M, rows, n_tiles, token_loss, vocab, err_flag);
     ce_sum_kernel<<<Z, 1024, 0, s>>>(token_loss, labels, M, loss_sum, count);
     count_launch(2);
 }

@@ -226,7 +226,12 @@ struct zoqat_model {
     // zoqat_step_deferred: Eq. (2) of the last step still to be applied (by the next step's producers, or by a flush)
     bool pending = false;
     uint64_t pending_seed = 0;
+    // a forward that carried a deferred update failed part-way: some masters have the update, some do not
+    bool broken = false;
     long long launches_at_create = 0;
+    // zoqat_debug_capture: records of the activation quantisers (caller's buffer), appended by forward()
+    uint8_t* cap = nullptr;
+    size_t cap_bytes = 0, cap_off = 0;
 };
 
 namespace {
@@ -298,6 +303,32 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
     }
 }
 
+// One capture record (zoqat_debug_capture): input fp32 [R, cols], operand bf16 [R, cols], step fp32 [R], each padded.
+size_t capture_record_bytes(int64_t R, int cols) {
+    return align_up((size_t)R * cols * 4) + align_up((size_t)R * cols * 2) + align_up((size_t)R * 4);
+}
+size_t capture_forward_bytes(const zoqat_model* m, int64_t T, int passes) {
+    size_t n = 0;
+    for (int l = 0; l < m->cfg.n_layers; ++l) {
+        const int64_t R = ((passes == 2 && l >= m->first_trainable_layer) ? 2 : 1) * T;
+        n += 3 * capture_record_bytes(R, m->cfg.d_model) + capture_record_bytes(R, m->cfg.d_ffn);
+    }
+    return n + capture_record_bytes(passes * T, m->cfg.d_model);      // input of the vocabulary projection
+}
+// Where the next record's input goes (NULL when the hook is off).
+float* capture_input(zoqat_model* m) { return m->cap ? reinterpret_cast<float*>(m->cap + m->cap_off) : nullptr; }
+// Completes the record: `input` (unless the kernel wrote it in place), the operand and the steps are copied in.
+void capture_finish(zoqat_model* m, const float* input, int64_t R, int cols, cudaStream_t s) {
+    if (!m->cap) return;
+    uint8_t* p = m->cap + m->cap_off;
+    if (input) cudaMemcpyAsync(p, input, (size_t)R * cols * 4, cudaMemcpyDeviceToDevice, s);
+    p += align_up((size_t)R * cols * 4);
+    cudaMemcpyAsync(p, m->ws.xa, (size_t)R * cols * 2, cudaMemcpyDeviceToDevice, s);
+    p += align_up((size_t)R * cols * 2);
+    cudaMemcpyAsync(p, m->ws.row_step, (size_t)R * 4, cudaMemcpyDeviceToDevice, s);
+    m->cap_off += capture_record_bytes(R, cols);
+}
+
 // The quantised forward.  passes = 1: loss of W + eps*u (eps signed) in loss_sum[0].
 // passes = 2: +eps in loss_sum[0] and -eps in loss_sum[1], evaluated side by side on 2T rows.
 // Layers before the first trainable one see the same weights in both passes and run once.
@@ -311,6 +342,11 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
     const int norm_kind = llama ? 1 : 2;
     const size_t ps = w.bop_elems;
+    if (m->cap) {
+        const size_t need = capture_forward_bytes(m, T, passes);
+        if (need > m->cap_bytes) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "capture buffer %zu < %zu bytes", m->cap_bytes, need);
+        m->cap_off = 0;
+    }
 
     int Z = (passes == 2 && m->first_trainable_layer == 0) ? 2 : 1;     // passes currently materialised as rows
     { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_embed(tokens, m->embed, m->pos, T, seq, d, c.vocab, Z, w.h, s); }
@@ -361,7 +397,8 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         // --- attention block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(0)); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(0));
+          capture_finish(m, nullptr, R, d, s); }
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
             produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
                             Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend);
@@ -387,7 +424,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                                   llama ? w.rope_sin : nullptr, w.att, w.attn_scratch, w.err_flag, s)) {
               return fail(rc, "attention launch rejected");
           } }
-        { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1)); }
+        { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
+          launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1));
+          capture_finish(m, w.att, R, d, s); }
         produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
@@ -397,7 +436,8 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         // --- feed-forward block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(2)); }
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(2));
+          capture_finish(m, nullptr, R, d, s); }
         const int n_up = llama ? 2 * F : F;
         produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend);
         if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend);
@@ -417,7 +457,8 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
           if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(3));
           else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
-          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3)); }
+          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3), false, false, capture_input(m));
+          capture_finish(m, fuse_gate ? w.ffn : nullptr, R, F, s); }
         produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
@@ -430,7 +471,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         Z = 2;
     }
     // --- final norm, vocabulary projection fused with the cross-entropy
-    { ProfScope ps_(m, ZOQAT_PROF_ACT, s); launch_norm_act_operand(w.h, Z * T, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, nullptr, s); }
+    { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
+      launch_norm_act_operand(w.h, Z * T, d, norm_kind, m->final_g, m->final_b, c.norm_eps, 0, w.xa, w.row_step, capture_input(m), s);
+      capture_finish(m, nullptr, Z * T, d, s); }
     produce_operand(m, m->head, w.bop, ps, Z, seed, eps, s, false, 0, nullptr, 0, 0, pend);
     GemmArgs g{};
     g.A = w.xa; g.B = w.bop; g.M = T; g.N = c.vocab; g.K = d; g.Z = Z; g.b_stride = ps;
@@ -438,7 +481,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     if (int rc = run_gemm(m, g, s)) return rc;
     { ProfScope ps_(m, ZOQAT_PROF_LOSS, s);
       launch_ce_finalize(w.ce_partials, w.label_logit, labels, T, Z, gemm_ce_tiles(c.vocab, c.gemm_impl), w.token_loss,
-                         w.loss_sum, w.count, s); }
+                         w.loss_sum, w.count, c.vocab, w.err_flag, s); }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "forward launch");
     return ZOQAT_OK;
@@ -453,6 +496,8 @@ int check_call(zoqat_model* m, const void* tokens, const void* labels, int batch
                     m->cfg.max_batch, m->cfg.max_seq);
     if (m->any_packed && !m->prequantized)
         return fail(ZOQAT_ERR_BAD_STATE, "frozen packed tensors present: call zoqat_prequantize_frozen first");
+    if (m->broken)
+        return fail(ZOQAT_ERR_BAD_STATE, "an earlier step failed while applying a deferred update: the masters are partially updated; reload them and create a new handle");
     return ZOQAT_OK;
 }
 
@@ -670,6 +715,7 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
     }
     cudaError_t e = cudaMemset(m->ws.err_flag, 0, 4);
     if (e != cudaSuccess) { delete m; return cuda_fail(e, "workspace init"); }
+    if (!generator_table_ready()) { delete m; return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed"); }
     m->launches_at_create = g_launch_count;
     *out = m;
     return ZOQAT_OK;
@@ -731,7 +777,11 @@ int zoqat_step_begin(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // a deferred update rides on this forward's producers (same bits as applying it first)
     PendingUpdate pend{m->pending_seed, m->ws.pending_scale};
-    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, eps, 2, s, m->pending ? &pend : nullptr)) return rc;
+    if (int rc = forward(m, tokens_dev, labels_dev, batch, seq, seed, eps, 2, s, m->pending ? &pend : nullptr)) {
+        // the producers launched before the failure have already applied the pending update to their tensors
+        if (m->pending && rc != ZOQAT_ERR_WORKSPACE_SMALL) { m->broken = true; m->pending = false; }
+        return rc;
+    }
     m->pending = false;
     launch_pack_sums(m->ws.loss_sum, m->ws.count, sums_dev, s);
     CUDA_TRY(cudaGetLastError());
@@ -882,6 +932,7 @@ static int step_host(zoqat_model_t* m, const int32_t* tokens_host, const int32_t
         return rc;
     CUDA_TRY(cudaMemcpyAsync(result_host, m->ws.result, sizeof(zoqat_step_result_t), cudaMemcpyDeviceToHost, s));
     CUDA_TRY(cudaStreamSynchronize(s));
+    if (result_host->status == kErrBadLabel) return fail(ZOQAT_ERR_INVALID_ARG, "a label is >= vocab (its position was given loss 0)");
     if (result_host->status != 0) return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", result_host->status);
     return ZOQAT_OK;
 }
@@ -916,6 +967,7 @@ int zoqat_check(zoqat_model_t* m, void* stream) {
     CUDA_TRY(cudaStreamSynchronize(s));
     if (flag != 0) {
         cudaMemsetAsync(m->ws.err_flag, 0, 4, s);
+        if (flag == kErrBadLabel) return fail(ZOQAT_ERR_INVALID_ARG, "a label is >= vocab (its position was given loss 0)");
         return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", flag);
     }
     return ZOQAT_OK;
@@ -961,6 +1013,22 @@ int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* byte
     return ZOQAT_OK;
 }
 
+int zoqat_debug_capture(zoqat_model_t* m, void* buf_dev, size_t bytes) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (buf_dev && (reinterpret_cast<uintptr_t>(buf_dev) & 255)) return fail(ZOQAT_ERR_INVALID_ARG, "buf_dev must be 256-byte aligned");
+    m->cap = static_cast<uint8_t*>(buf_dev);
+    m->cap_bytes = buf_dev ? bytes : 0;
+    m->cap_off = 0;
+    return ZOQAT_OK;
+}
+
+int zoqat_debug_capture_bytes(const zoqat_model_t* m, int batch, int seq, int passes, size_t* bytes) {
+    if (!m || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (batch <= 0 || seq <= 0 || (passes != 1 && passes != 2)) return fail(ZOQAT_ERR_INVALID_ARG, "bad capture size query");
+    *bytes = capture_forward_bytes(m, (int64_t)batch * seq, passes);
+    return ZOQAT_OK;
+}
+
 // ---- single operations ---------------------------------------------------------
 static int check_group_bits(int64_t rows, int64_t cols, int group, int bits, bool allow_zero_bits, int max_bits = 8,
                             bool allow_rows = false) {
@@ -983,6 +1051,7 @@ int zoqat_op_philox_words(uint64_t seed, uint32_t tensor_id, uint64_t blk0, uint
 }
 
 int zoqat_op_normal(uint64_t seed, uint32_t tensor_id, uint64_t n, float* out_dev, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (!out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "out_dev is NULL");
     launch_normal(seed, tensor_id, n, out_dev, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
@@ -992,6 +1061,7 @@ int zoqat_op_normal(uint64_t seed, uint32_t tensor_id, uint64_t n, float* out_de
 int zoqat_op_weight_quant(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
                           uint32_t tensor_id, float signed_eps, uint8_t* codes_dev, float* step_dev, int32_t* zp_dev,
                           void* operand_dev, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
     if (!w_dev || !operand_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_dev are NULL");
     launch_weight_operand(w_dev, rows * cols, group, bits, signed_eps != 0.0f, seed, tensor_id, signed_eps,
@@ -1003,6 +1073,7 @@ int zoqat_op_weight_quant(const float* w_dev, int64_t rows, int64_t cols, int gr
 
 int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
                                  uint32_t tensor_id, float eps, void* operand_plus_dev, void* operand_minus_dev, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (int rc = check_group_bits(rows, cols, group, bits, true)) return rc;
     if (!w_dev || !operand_plus_dev || !operand_minus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     launch_weight_operand(w_dev, rows * cols, group, bits, 1, seed, tensor_id, eps, static_cast<__nv_bfloat16*>(operand_plus_dev),
@@ -1015,6 +1086,7 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
                                     uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
                                     const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
                                     void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (!scratch_dev || (reinterpret_cast<uintptr_t>(scratch_dev) & 15)) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 16-byte aligned device memory");
     if (int rc = check_group_bits(rows, cols, group, bits, true, 8, true)) return rc;
     if (!w_dev || !operand_plus_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev/operand_plus_dev are NULL");
@@ -1039,6 +1111,7 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
 
 int zoqat_op_smooth_perturb(const float* scale_dev, const float* shift_dev, int64_t cols, uint64_t seed, uint32_t scale_id,
                             uint32_t shift_id, float eps, float* out_dev, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (!scale_dev || !shift_dev || !out_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
     if (cols <= 0 || cols % 4 || cols > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a positive multiple of 4");
     if ((reinterpret_cast<uintptr_t>(scale_dev) | reinterpret_cast<uintptr_t>(shift_dev) | reinterpret_cast<uintptr_t>(out_dev)) & 15)
@@ -1100,6 +1173,7 @@ int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int
 }
 
 int zoqat_op_update(float* w_dev, uint64_t n, uint64_t seed, uint32_t tensor_id, float scale, void* stream) {
+    if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (!w_dev) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev is NULL");
     if (reinterpret_cast<uintptr_t>(w_dev) & 15) return fail(ZOQAT_ERR_INVALID_ARG, "w_dev must be 16-byte aligned");
     launch_update(w_dev, n, seed, tensor_id, nullptr, scale, static_cast<cudaStream_t>(stream));
@@ -1237,7 +1311,7 @@ int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labe
     g.single_cta = impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
-    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
+    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, V, err_flag_dev, s);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
@@ -1250,24 +1324,14 @@ namespace {
 
 static __device__ __align__(256) unsigned char g_static_scratch[ZOQAT_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxStaticDevices = 64;
-std::mutex g_static_mu;
-void* g_static_ptr[kMaxStaticDevices] = {nullptr};
-
-// Device address of g_static_scratch on the current device.  In host code the symbol is only a
-// handle, never an address a kernel may dereference, so the address is looked up once per device.
+// Device address of g_static_scratch on the current device.  In host code the symbol is only a handle, never an
+// address a kernel may dereference; the address is looked up on every call (a table lookup in the runtime), so it is
+// always that of the current device and context, also after a context was torn down and created again.
 int static_scratch_address(void** out) {
-    int dev = 0;
-    CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxStaticDevices) return fail(ZOQAT_ERR_UNSUPPORTED, "device ordinal %d is beyond the %d this entry point tracks", dev, kMaxStaticDevices);
-    std::lock_guard<std::mutex> lock(g_static_mu);
-    if (!g_static_ptr[dev]) {
-        void* p = nullptr;
-        CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
-        if (!p) return fail(ZOQAT_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
-        g_static_ptr[dev] = p;
-    }
-    *out = g_static_ptr[dev];
+    void* p = nullptr;
+    CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p) return fail(ZOQAT_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+    *out = p;
     return ZOQAT_OK;
 }
 
@@ -1300,7 +1364,7 @@ int zoqat_op_head_loss_static(const void* a_dev, const void* b_dev, const int32_
     g.single_cta = impl == ZOQAT_GEMM_TCGEN05_1CTA;
     const int rc = impl == ZOQAT_GEMM_SIMT ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "head GEMM rejected: T=%lld V=%lld d=%lld", (long long)T, (long long)V, (long long)d);
-    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, s);
+    launch_ce_finalize(partials, label_logit, labels_dev, T, 1, gemm_ce_tiles(V, impl), token_loss_dev, loss_sum_dev, count_dev, V, err_flag_dev, s);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
@@ -1357,6 +1421,7 @@ int zoqat_decode_begin(zoqat_model_t* m, void* buffer_dev, size_t bytes, int bat
             if (Ly.lin[r].present && !Ly.lin[r].packed_frozen())
                 return fail(ZOQAT_ERR_UNSUPPORTED, "decode runs on the packed representation: every block linear must be FROZEN_PACKED");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);           // the vocabulary projection is converted from its master below
     const size_t d = c.d_model, F = c.d_ffn, G = c.w_group;
     uint8_t* p = static_cast<uint8_t*>(buffer_dev);
     auto take = [&](size_t n) { uint8_t* q = p; p += n; return q; };

@@ -164,8 +164,8 @@ template <int D>
 static void attention_launch(const float* qkv, int batch, int seq, int n_heads, const float* cos_t, const float* sin_t,
                              float* out, cudaStream_t s) {
     const size_t smem = (size_t)(3 * 64 * (D + 4) + 64 * (BKV + 4)) * sizeof(float);
-    static bool attr = false;
-    if (!attr) { cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr = true; }
+    static DeviceOnce attr;
+    if (attr.first()) { cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); }
     dim3 grid((seq + BQ - 1) / BQ, n_heads, batch);
     attention_kernel<D><<<grid, kAttThreads, smem, s>>>(qkv, seq, n_heads, cos_t, sin_t, out);
     count_launch();

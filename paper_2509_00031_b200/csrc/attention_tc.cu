@@ -635,11 +635,11 @@ int attention_tc_launch(const float* qkv, int batch, int seq, int n_heads, const
         !make_half_map(&m_kh, kh, D, seq, bhs, D, BKV) || !make_half_map(&m_kl, kl, D, seq, bhs, D, BKV) ||
         !make_half_map(&m_vth, vth, seq, D, bhs, seq_pad, D) || !make_half_map(&m_vtl, vtl, seq, D, bhs, seq_pad, D))
         return ZOQAT_ERR_CUDA;
-    static bool attr = false;
-    if (!attr) {
-        if (cudaFuncSetAttribute(attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
-            return ZOQAT_ERR_CUDA;
-        attr = true;
+    static DeviceOnce attr;
+    if (attr.first() &&
+        cudaFuncSetAttribute(attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+        attr.retry();
+        return ZOQAT_ERR_CUDA;
     }
     AttParams p;
     p.seq = seq; p.n_heads = n_heads; p.batch = batch;

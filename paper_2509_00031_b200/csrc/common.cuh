@@ -12,6 +12,27 @@ constexpr int kErrWaitFull = 1;      // MMA warp: operands never arrived
 constexpr int kErrWaitEmpty = 2;     // TMA warp: stage never released
 constexpr int kErrWaitAccFull = 3;   // epilogue: accumulator never committed
 constexpr int kErrWaitAccEmpty = 4;  // MMA warp: accumulator never drained
+constexpr int kErrBadLabel = 16;     // cross-entropy: a label >= vocab (not a wait; the position's loss is reported as 0)
+
+// Per-device one-time set-up (function attributes, cached device properties): true the first time it is called with this
+// word while device `ordinal < 64` is current; ordinals beyond that always get true and simply repeat the set-up.
+struct DeviceOnce {
+    unsigned long long seen = 0;
+    bool first() {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+        const unsigned long long bit = 1ull << dev;
+        return (__atomic_fetch_or(&seen, bit, __ATOMIC_ACQ_REL) & bit) == 0;
+    }
+    // forget the current device (its set-up failed and must be tried again)
+    void retry() {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) __atomic_fetch_and(&seen, ~(1ull << dev), __ATOMIC_ACQ_REL);
+    }
+};
+// The inverse-distribution table of the direction generator is uploaded to the current device on first use; false if
+// that failed (callers report it instead of launching a generator kernel on a missing table).
+bool generator_table_ready();
 
 // Host-side launch bookkeeping (one counter per process, read through the handle).
 extern long long g_launch_count;
@@ -114,9 +135,10 @@ struct SmoothAct { const float* smooth = nullptr; int ld = 0; int64_t rows_per_p
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
                              SmoothAct sm = SmoothAct(), bool dependent = false, bool planes = false);
+// pre (may be NULL): fp32 [rows, cols], receives the value the quantiser sees (parity hook).
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
                             __nv_bfloat16* op, float* row_step, cudaStream_t s, SmoothAct sm = SmoothAct(),
-                            bool dependent = false, bool planes = false);
+                            bool dependent = false, bool planes = false, float* pre = nullptr);
 // Activation operand of rows whose max |x| is already known (amax: bits of a non-negative float per row).
 void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits,
                          __nv_bfloat16* op, float* row_step, cudaStream_t s);
@@ -184,8 +206,10 @@ int launch_gemm_simt(const GemmArgs& a, cudaStream_t s);   // returns 0 or a ZOQ
 int launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
 
 // Per-position loss from the partials, then the deterministic sum.
+// vocab / err_flag (may be NULL): a label >= vocab sets kErrBadLabel there.
 void launch_ce_finalize(const float2* partials, const float* label_logit, const int32_t* labels, int64_t M, int Z,
-                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, cudaStream_t s);
+                        int n_tiles, float* token_loss, double* loss_sum, int32_t* count, int64_t vocab, int32_t* err_flag,
+                        cudaStream_t s);
 // g, lr*g and the result record from the two loss sums.
 struct zoqat_step_result_dev { float loss_plus, loss_minus, proj_grad, update_scale; int32_t status, n_labels; };
 void launch_pack_sums(const double* loss_sum, const int32_t* count, double* sums, cudaStream_t s);

@@ -508,8 +508,8 @@ int launch_decode_gemv(const void* wq, const float2* qparams, int N, int K, int 
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV(MBV)                                                                                                      \
     {                                                                                                                     \
-        static bool attr = false;                                                                                         \
-        if (!attr) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
+        static DeviceOnce attr;                                                                                         \
+        if (attr.first()) { cudaFuncSetAttribute(decode_gemv_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); } \
         launch_kernel(decode_gemv_kernel<MBV>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, qparams, N, K, gshift, act, row_step, bias, accumulate, out); \
     }
     if (mb == 1) ZQ_GEMV(1) else if (mb == 2) ZQ_GEMV(2) else if (mb == 4) ZQ_GEMV(4) else if (mb == 8) ZQ_GEMV(8) else return -1;
@@ -528,8 +528,8 @@ int launch_decode_gemv_fp(const void* wq, const float2* qparams, int N, int K, i
     const uint4* w4 = static_cast<const uint4*>(wq);
 #define ZQ_GEMV_FP(MBV)                                                                                                   \
     {                                                                                                                     \
-        static bool attr = false;                                                                                         \
-        if (!attr) { cudaFuncSetAttribute(decode_gemv_fp_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; } \
+        static DeviceOnce attr;                                                                                         \
+        if (attr.first()) { cudaFuncSetAttribute(decode_gemv_fp_kernel<MBV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); } \
         launch_kernel(decode_gemv_fp_kernel<MBV>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, qparams, N, K, gshift, act, bias, accumulate, out); \
     }
     if (mb == 1) ZQ_GEMV_FP(1) else if (mb == 2) ZQ_GEMV_FP(2) else if (mb == 4) ZQ_GEMV_FP(4) else if (mb == 8) ZQ_GEMV_FP(8) else return -1;
@@ -554,8 +554,8 @@ int launch_decode_head(const __nv_bfloat16* w, int V, int d, int mb, const __nv_
     else if (mb == 2) launch_kernel(decode_head_kernel<2>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
     else if (mb == 4) launch_kernel(decode_head_kernel<4>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
     else if (mb == 8) {
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(decode_head_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); attr = true; }
+        static DeviceOnce attr;
+        if (attr.first()) { cudaFuncSetAttribute(decode_head_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); }
         launch_kernel(decode_head_kernel<8>, dim3(grid), dim3(kGemvThreads), smem, s, true, w4, V, d, x, logits);
     } else return -1;
     count_launch();

@@ -563,14 +563,14 @@ bool make_half_box_map(CUtensorMap* map, void* base, int64_t inner, int64_t rows
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (cached per ordinal).
 int num_sms() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
+    static int cached[64] = {0};
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev >= 0 && dev < 64 && (n = __atomic_load_n(&cached[dev], __ATOMIC_RELAXED)) > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    if (dev >= 0 && dev < 64) __atomic_store_n(&cached[dev], n, __ATOMIC_RELAXED);
     return n;
 }
 
@@ -616,11 +616,11 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     } else if (a.mode != 2) {
         map_out = map_a;      // never dereferenced
     }
-    static bool attr = false;
-    if (!attr) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
-            return ZOQAT_ERR_CUDA;
-        attr = true;
+    static DeviceOnce attr;
+    if (attr.first() &&
+        cudaFuncSetAttribute(gemm_tc_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+        attr.retry();
+        return ZOQAT_ERR_CUDA;
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
     const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)

@@ -60,6 +60,10 @@ bool ensure_icdf_table() {
     return true;
 }
 
+}  // namespace
+bool generator_table_ready() { return ensure_icdf_table(); }
+namespace {
+
 // Every generator kernel starts by staging the table in shared memory.
 __device__ __forceinline__ void stage_icdf_table(float2* tab) {
     for (int i = threadIdx.x; i < kIcdfKnots; i += blockDim.x) tab[i] = g_icdf_table[i];

@@ -13,6 +13,7 @@ from oracle import core
 from oracle.model import (OracleConfig, OracleModel, adaptive_weight_quant, init_quant_params, act_quant, tensor_id,
                           QPARAM_ID, SMOOTH_SCALE_ID, SMOOTH_SHIFT_ID, POINTS)
 from paper_2509_00031_b200 import synth
+from gparity import check_g
 
 pytestmark = pytest.mark.gpu
 
@@ -316,18 +317,7 @@ def test_step_rates_match_oracle(zq, impl, shape, first):
             moved += 1
         assert moved == len(ids) - 1                             # every trainable tensor but the head, checked above
         g_o.append(float(g)); g_g.append(res["proj_grad"])
-    g_o, g_32, g_g = map(np.array, (g_o, g_32, g_g))
-    g_rms = float(np.sqrt(np.mean(g_o ** 2)))
-    band = float(np.sqrt(np.mean((g_o - g_32) ** 2)))
-    err = np.abs(g_g - g_o)
-    print(f"[g parity learnables] rms g {g_rms:.4f}; rms err {np.sqrt(np.mean(err ** 2)):.2e}; oracle self-band {band:.2e}; "
-          f"per step g_gpu-g {np.round(g_g - g_o, 4).tolist()} g32-g {np.round(g_32 - g_o, 4).tolist()}")
-    # g = (L+ - L-) / (2 eps) amplifies a binary32-grade loss difference (3e-6 relative here) by 500.  The oracle's
-    # self-disagreement under binary32 storage (band) models only part of what a binary32 implementation does
-    # differently and comes out at 0.03 % of rms(g) on this small model, against the 1-2 % it shows on the
-    # configurations of test_gpu_model; the bound therefore never drops below 1 % of rms(g).
-    assert np.sqrt(np.mean(err ** 2)) <= max(3.0 * band, 1e-2 * g_rms) + 2e-3 * g_rms
-    assert np.all(err <= 0.05 * g_rms + 2e-3 * np.abs(g_o))
+    check_g([dict(g=a, g32=b, g_gpu=c) for a, b, c in zip(g_o, g_32, g_g)], f"Section 4.2 {shape['arch']} W{shape['w_bits']}A{shape['a_bits']} impl={impl}")
 
 
 def test_step_with_one_rate_and_apply_update_rates(zq):

@@ -12,16 +12,21 @@ disagrees with ITSELF by 1-2 % of rms(g) when its stored activations are merely 
 to binary32 (OracleConfig.store_f32), so a 2e-3 relative bound on g cannot be met by any
 implementation that is not bit-identical to the oracle in every intermediate.  The test
 therefore (1) compares steps state-synced (GPU masters copied from the oracle before each
-step), (2) measures that self-disagreement ("band") on the same inputs, and (3) requires
-rms|g_gpu - g_oracle| <= 3 * rms(band) and every |g_gpu - g_oracle| <= 5 % of rms(g);
-it also reports how many steps meet 2e-3 * max(|g|, rms g).
+step), (2) measures that self-disagreement ("band") on the same inputs, and (3) applies the rule of
+gparity.check_g (rms error against the band, every error against 5 % of rms g); it also reports how many steps meet
+2e-3 * max(|g|, rms g).  Every assertion on g in the GPU tests is this one
+rule, over several seeds so that a band can be formed; the steps in which no quantised code differs
+from the oracle's are held to 2e-3 itself in test_gpu_forward_elementwise.py.
 """
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
 
 from oracle.model import OracleConfig, OracleModel
 from paper_2509_00031_b200 import synth
+from gparity import check_g
 
 pytestmark = pytest.mark.gpu
 
@@ -88,51 +93,57 @@ def sync_masters(model, oracle):
     model.params["lm_head"].copy_(torch.from_numpy(oracle.p["lm_head"]))
 
 
-def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr, **cfg_kw):
-    """n state-synced steps; returns per-step records and checks everything except g."""
+def default_step(zq, model, td, ld, seed, eps, lr):
+    return [zq.decode_step_result(model.zoqat_step(td, ld, seed, eps, lr))]
+
+
+def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr, step_fn=default_step, seed0=1000):
+    """n state-synced steps; returns per-step records and checks everything except g.  step_fn runs the GPU step and
+    returns the result records of the directions it evaluated (one for zoqat_step); direction i uses seed + i and
+    the factor lr / len(records)."""
     from oracle import core
     from oracle.model import tensor_id, LM_HEAD_ID
     recs = []
     n_lab = int((labels >= 0).sum())
+    td, ld = dev(tokens), dev(labels)
     for t in range(n_steps):
-        seed = 1000 + t
         sync_masters(model, oracle)
-        # the oracle's self-disagreement under binary32 storage of activations, same weights
-        o32 = OracleModel(oracle_cfg(shape, store_f32=True, **cfg_kw), oracle.p)
-        _, _, g32 = o32.projected_gradient(tokens, labels, seed, eps)
         w_before = {(l, n): oracle.p["layers"][l][n].copy() for l in range(shape["n_layers"]) for n in oracle.linear_names()}
-        res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), seed, eps, lr))
+        head_before = oracle.p["lm_head"].copy()
+        results = step_fn(zq, model, td, ld, seed0 + 8 * t, eps, lr)
         model.zoqat_check()
-        lp, lm, g = oracle.step(tokens, labels, seed, eps, lr)
-        assert res["status"] == 0 and res["n_labels"] == n_lab
-        assert abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
-        assert res["update_scale"] == float(np.float32(lr) * np.float32(res["proj_grad"]))
-        first = oracle.cfg.first_trainable_layer
+        q = len(results)
+        lr_q = np.float32(lr) if q == 1 else np.float32(np.float32(lr) / np.float32(q))
+        # the oracle's self-disagreement under binary32 storage of activations, same weights
+        o32 = OracleModel(dataclasses.replace(oracle.cfg, store_f32=True), oracle.p)
+        g32s = [o32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
+        want = oracle.step_multi(tokens, labels, seed0 + 8 * t, q, eps, lr) if q > 1 else [oracle.step(tokens, labels, seed0 + 8 * t, eps, lr)]
+        for i, (res, (lp, lm, g)) in enumerate(zip(results, want)):
+            assert res["status"] == 0 and res["n_labels"] == n_lab
+            assert abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
+            assert res["update_scale"] == float(lr_q * np.float32(res["proj_grad"]))
+            recs.append(dict(g=float(g), g32=float(g32s[i]), g_gpu=res["proj_grad"]))
         for (l, n), wb in w_before.items():
             got = model.params["layers"][l][n].cpu().numpy()
-            if l < first:
-                assert np.array_equal(got, wb)
+            if not oracle.is_trainable(l, n):
+                assert np.array_equal(got, wb), (l, n)
                 continue
             assert np.abs(got - oracle.p["layers"][l][n]).max() <= 1e-5, (l, n)
-            # Eq. (2) with the step's own factor is reproduced bit for bit
-            want = core.update_(wb.copy(), seed, tensor_id(l, oracle._ROLE[n]), np.float32(res["update_scale"]))
-            assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), (l, n)
-        recs.append(dict(g=float(g), g32=float(g32), g_gpu=res["proj_grad"]))
+            # Eq. (2) with the step's own factors is reproduced bit for bit
+            want_w = wb.copy()
+            for i, res in enumerate(results):
+                core.update_(want_w, seed0 + 8 * t + i, tensor_id(l, oracle._ROLE[n]), np.float32(res["update_scale"]))
+            assert np.array_equal(got.view(np.uint32), want_w.view(np.uint32)), (l, n)
+        got_h = model.params["lm_head"].cpu().numpy()
+        if oracle.cfg.head_trainable:
+            want_h = head_before.copy()
+            for i, res in enumerate(results):
+                core.update_(want_h, seed0 + 8 * t + i, LM_HEAD_ID, np.float32(res["update_scale"]))
+            assert np.array_equal(got_h.view(np.uint32), want_h.view(np.uint32))
+            assert np.abs(got_h - oracle.p["lm_head"]).max() <= 1e-5
+        else:
+            assert np.array_equal(got_h, head_before)
     return recs
-
-
-def check_g(recs, label):
-    g = np.array([r["g"] for r in recs]); g32 = np.array([r["g32"] for r in recs]); gg = np.array([r["g_gpu"] for r in recs])
-    g_rms = float(np.sqrt(np.mean(g * g)))
-    band_rms = float(np.sqrt(np.mean((g - g32) ** 2)))
-    err = np.abs(gg - g)
-    err_rms = float(np.sqrt(np.mean(err ** 2)))
-    within_target = int(np.sum(err <= 2e-3 * np.maximum(np.abs(g), g_rms)))
-    print(f"[g parity {label}] rms g {g_rms:.4f}; rms |g_gpu-g_oracle| {err_rms:.2e} ({err_rms / g_rms:.2%}); "
-          f"oracle self-band rms {band_rms:.2e}; steps within 2e-3: {within_target}/{len(recs)}")
-    assert err_rms <= 3.0 * band_rms + 2e-3 * g_rms, (err_rms, band_rms, g_rms)
-    assert np.all(err <= 0.05 * g_rms + 2e-3 * np.abs(g)), (err.max(), g_rms)
-    assert np.corrcoef(g, gg)[0, 1] > 0.995
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -141,7 +152,7 @@ def test_step_matches_oracle(zq, impl, shape, batch, seq):
     model, oracle = build_pair(zq, shape, batch, seq, impl)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=12)
     recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 8, 1e-3, 1e-6)
-    check_g(recs, f"{shape['arch']} impl={impl}")
+    check_g(recs, f"small {shape['arch']} W{shape['w_bits']}A{shape['a_bits']} impl={impl}")
     assert np.array_equal(model.params["embed"].cpu().numpy(), oracle.p["embed"])
 
 
@@ -221,9 +232,10 @@ def test_lightweight_variant(zq, impl):
     lp, lm, g = oracle.step(tokens, labels, 3, eps, lr)
     assert res == res2
     assert res["loss_plus"] == a
-    assert abs(res["loss_minus"] - lm) <= 1e-4 * abs(lm) and abs(res["proj_grad"] - g) <= 0.1 * max(abs(g), 1.0)
+    assert abs(res["loss_minus"] - lm) <= 1e-4 * abs(lm)
     assert torch.equal(frozen_before, plain.params["layers"][0]["wq"])
     assert np.abs(plain.params["layers"][2]["wq"].cpu().numpy() - oracle.p["layers"][2]["wq"]).max() <= 1e-5
+    check_g(run_synced_steps(zq, packed, oracle, shape, tokens, labels, 6, eps, lr), f"lightweight (packed prefix) impl={impl}")
     # nothing trainable: the loss ignores (seed, eps)
     none, _ = build_pair(zq, shape, batch, seq, impl, first_trainable_layer=3, head_trainable=False, packed=True)
     assert float(none.zoqat_forward_loss(td, ld, 1, 1e-3).item()) == float(none.zoqat_forward_loss(td, ld, 9, -1e-2).item())
@@ -254,11 +266,12 @@ def test_step_host_buffers(zq):
     model, oracle = build_pair(zq, shape, batch, seq, 0)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=15)
     th, lh = torch.from_numpy(tokens).pin_memory(), torch.from_numpy(labels).pin_memory()
-    res = model.zoqat_step_host(th, lh, 5, 1e-3, 1e-4)
-    lp, lm, g = oracle.step(tokens, labels, 5, 1e-3, 1e-4)
-    assert res.status == 0
-    assert abs(res.loss_plus - lp) <= 1e-3 * abs(lp) and abs(res.loss_minus - lm) <= 1e-3 * abs(lm)
-    assert abs(res.proj_grad - g) <= 0.1 * max(abs(g), 1.0)          # see the module docstring on g
+    def host_step(zq_, m, td, ld, seed, eps, lr):
+        r = m.zoqat_step_host(th, lh, seed, eps, lr)
+        return [dict(loss_plus=r.loss_plus, loss_minus=r.loss_minus, proj_grad=r.proj_grad, update_scale=r.update_scale,
+                     status=r.status, n_labels=r.n_labels)]
+
+    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 6, 1e-3, 1e-4, step_fn=host_step), "host buffers")
 
 
 # ---- the five workloads at their real layer dimensions ------------------------------------------------------------
@@ -281,7 +294,8 @@ WORKLOAD_CUTS = [
 def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packed):
     """Every workload with its real d_model / heads / d_ffn / vocabulary / quantiser, cut to one layer (two for the
     lightweight one: a frozen packed layer under a trainable one) and a short sequence so that the oracle finishes:
-    one full step against the oracle - both losses, the update of a block tensor and of the vocabulary projection."""
+    four state-synced steps against the oracle - both losses, every updated tensor bit for bit given the step's own
+    factor and within 1e-5 of the oracle's, g under the band rule."""
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq,
@@ -289,56 +303,55 @@ def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packe
     if packed:
         model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
-    eps, lr, seed = 1e-3, 1e-6, 1000
-    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), seed, eps, lr))
-    model.zoqat_check()
-    lp, lm, g = oracle.step(tokens, labels, seed, eps, lr)
-    assert res["status"] == 0
-    assert abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
-    print(f"[{shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} W{shape['w_bits']}A{shape['a_bits']}] "
-          f"L+ {res['loss_plus']:.6f} / {lp:.6f}  L- {res['loss_minus']:.6f} / {lm:.6f}  g {res['proj_grad']:.4f} / {g:.4f}")
-    last = shape["n_layers"] - 1
-    name = "w_down" if shape["arch"] == "llama" else "fc2"
-    # the update uses the step's own g: compare against the oracle's update with that factor (bit for bit), and
-    # against the oracle's own step within the weight tolerance scaled by the difference in g
-    from oracle import core
-    from oracle.model import tensor_id, LM_HEAD_ID
-    w0 = params["layers"][last][name]
-    want = core.update_(w0.copy(), seed, tensor_id(last, oracle._ROLE[name]), np.float32(res["update_scale"]))
-    assert np.array_equal(model.params["layers"][last][name].cpu().numpy().view(np.uint32), want.view(np.uint32))
-    want_h = core.update_(params["lm_head"].copy(), seed, LM_HEAD_ID, np.float32(res["update_scale"]))
-    assert np.array_equal(model.params["lm_head"].cpu().numpy().view(np.uint32), want_h.view(np.uint32))
-    assert np.abs(model.params["layers"][last][name].cpu().numpy() - oracle.p["layers"][last][name]).max() <= 1e-5
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 4, 1e-3, 1e-6)
+    check_g(recs, f"workload dims {shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} "
+                  f"W{shape['w_bits']}A{shape['a_bits']} g{shape['w_group']} T={batch * seq}")
     if first_trainable:
         assert np.array_equal(model.params["layers"][0]["wq"].cpu().numpy(), params["layers"][0]["wq"])
 
 
+def test_full_token_count_layer_step(zq):
+    """The bench workload's own token count through one layer and the vocabulary projection: LLaMA-7B dimensions,
+    W4A8 g128, batch 4 x seq 1024 - 16 row tiles and 8 attention query tiles per sequence in every GEMM, both passes
+    side by side on 8192 rows, the schedule the benchmark times.  Full zoqat_step against the oracle: both losses,
+    every updated tensor (bit for bit given the step's own factor, 1e-5 against the oracle's own step), g under the
+    band rule over three seeds, and the per-position losses of the last step's + pass element by element."""
+    shape = _cut("llama7b_w4a8", 1)
+    batch, seq = shape["batch"], shape["seq"]
+    params = synth.make_params(shape, seed=3, max_seq=seq)
+    oracle = OracleModel(oracle_cfg(shape), synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=1234)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3, 1e-3, 1e-6)
+    check_g(recs, "llama7b_w4a8, one layer, full 4 x 1024 tokens")
+    # per-position losses of both passes of one more (unsynced) step: rows [0, T) are the + pass, [T, 2T) the - pass
+    T = batch * seq
+    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), 77, 1e-3, 0.0))
+    tl_gpu = model.zoqat_debug_buffer(zq.BUF_TOKEN_LOSS)[:2 * T].cpu().numpy().astype(np.float64)
+    sync_masters(model, oracle)        # lr = 0 left the masters where the oracle's are; make it exact anyway
+    for z, sign in enumerate((1.0, -1.0)):
+        tl, valid = oracle.token_losses(tokens, labels, 77, sign * float(np.float32(1e-3)))
+        rel = np.abs(tl_gpu[z * T:(z + 1) * T] - tl)[valid] / tl[valid]
+        print(f"[full token count] pass {'+-'[z]}: per-position loss rel err max {rel.max():.2e} median {np.median(rel):.2e}")
+        assert rel.max() <= 1e-3
+    assert res["status"] == 0
+
+
 def test_step_multi_directions(zq):
-    """q = 3 directions per step: every g_i at the same weights, one fused update; against the oracle, and
-    q = 1 against zoqat_step bit for bit."""
-    from oracle import core
-    from oracle.model import tensor_id
+    """q = 3 directions per step: every g_i at the same weights, one fused update; against the oracle (losses, the
+    fused update bit for bit given the step's own factors, every g_i under the band rule), and q = 1 against
+    zoqat_step bit for bit."""
     shape, batch, seq = SMALL_LLAMA, 2, 96
     model, oracle = build_pair(zq, shape, batch, seq, 0)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=16)
     td, ld = dev(tokens), dev(labels)
     eps, lr, seed, q = 1e-3, 1e-4, 400, 3
-    w0 = oracle.p["layers"][1]["w_down"].copy()
-    res = model.zoqat_step_multi(td, ld, seed, q, eps, lr).cpu()
-    model.zoqat_check()
-    recs = [zq.decode_step_result(res[i]) for i in range(q)]
-    want = oracle.step_multi(tokens, labels, seed, q, eps, lr)
-    lr_q = np.float32(np.float32(lr) / np.float32(q))
-    upd = w0.copy()
-    for i, (r, (lp, lm, g)) in enumerate(zip(recs, want)):
-        assert r["status"] == 0
-        assert abs(r["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(r["loss_minus"] - lm) <= 1e-3 * abs(lm)
-        assert abs(r["proj_grad"] - g) <= 0.1 * max(abs(g), 1.0)          # see the module docstring on g
-        assert r["update_scale"] == float(lr_q * np.float32(r["proj_grad"]))
-        core.update_(upd, seed + i, tensor_id(1, oracle._ROLE["w_down"]), np.float32(r["update_scale"]))
-    got = model.params["layers"][1]["w_down"].cpu().numpy()
-    assert np.array_equal(got.view(np.uint32), upd.view(np.uint32))     # the fused update, given the step's own factors
-    assert np.abs(got - oracle.p["layers"][1]["w_down"]).max() <= 1e-5
+
+    def multi_step(zq_, m, td_, ld_, seed_, eps_, lr_):
+        res = m.zoqat_step_multi(td_, ld_, seed_, q, eps_, lr_).cpu()
+        return [zq_.decode_step_result(res[i]) for i in range(q)]
+
+    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 3, eps, lr, step_fn=multi_step, seed0=seed), "q = 3 directions")
     # q = 1 is zoqat_step
     a, _ = build_pair(zq, shape, batch, seq, 0)
     b, _ = build_pair(zq, shape, batch, seq, 0)
@@ -360,13 +373,8 @@ def test_query_value_only_selection(zq):
                           trainable_names=names, head_trainable=False)
     model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=17)
-    eps, lr, seed = 1e-3, 1e-4, 9
-    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), seed, eps, lr))
-    model.zoqat_check()
-    lp, lm, g = oracle.step(tokens, labels, seed, eps, lr)
-    assert res["status"] == 0
-    assert abs(res["loss_plus"] - lp) <= 1e-4 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-4 * abs(lm)
-    assert abs(res["proj_grad"] - g) <= 0.1 * max(abs(g), 1.0)
+    eps, lr = 1e-3, 1e-4
+    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 6, eps, lr, seed0=9), "query/value only")
     for l in range(2):
         for n in oracle.linear_names():
             got = model.params["layers"][l][n].cpu().numpy()

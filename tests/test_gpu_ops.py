@@ -134,7 +134,7 @@ def _check_codes(codes_gpu, step_gpu, x_gpu_f32, x_oracle_f64):
         inv = (np.float32(1.0) / s_or)[:, None]
         v = x_oracle_f64.astype(np.float32) * inv
         dist = np.abs(np.abs(v - np.floor(v)) - 0.5)
-        assert np.all(dist[diff] <= 1e-6 * np.maximum(1.0, np.abs(v[diff])) + 2e-5), "code differs away from a rounding boundary"
+        assert np.all(dist[diff] <= 1e-6 * np.maximum(1.0, np.abs(v[diff]))), "code differs away from a rounding boundary"
     return int(diff.sum())
 
 
@@ -150,7 +150,8 @@ def test_norm_act_operand(zq, kind, cols):
     normed = normed.cpu().numpy()
     assert np.allclose(normed, want, rtol=2e-6, atol=2e-6)
     excused = _check_codes(bf16_to_f32(op).astype(np.float64), step.cpu().numpy(), normed, want)
-    assert excused <= 3
+    print(f"[norm + quantiser kind {kind} cols {cols}] codes excused within 1e-6 of a boundary: {excused}/{rows * cols}")
+    assert excused <= max(3, int(2e-4 * rows * cols))
     # unquantised activations: operand = bf16(x), row step 1
     op16, step16, _ = zq.zoqat_op_norm_act_operand(dev(x), kind, dev(g), dev(b), 1e-5, 0, want_normed=False)
     assert np.array_equal(bf16_to_f32(op16), core.round_bf16(normed)) and np.all(step16.cpu().numpy() == 1.0)
@@ -181,7 +182,14 @@ def test_ffn_act_operand(zq, gated, cols):
     assert np.allclose(step.cpu().numpy(), np.abs(want).max(1) / 127, rtol=1e-6)
     q_or, s_or = act_quant(want)
     diff = codes != q_or
-    assert diff.mean() < 2e-4                      # only values that sit on a rounding boundary move
+    # only values that sit on a rounding boundary move: every differing code is one away and its pre-rounding value
+    # (oracle side) lies within 1e-6 relative of the half-integer between the two codes
+    inv = (np.float32(1.0) / s_or)[:, None]
+    v = want.astype(np.float32) * inv
+    dist = np.abs(v.astype(np.float64) - 0.5 * (codes + q_or))
+    print(f"[ffn non-linearity + quantiser gated {gated} cols {cols}] codes excused within 1e-6 of a boundary: {int(diff.sum())}/{codes.size}")
+    assert np.all(dist[diff] <= 1e-6 * np.maximum(1.0, np.abs(v[diff]))), float(dist[diff].max())
+    assert diff.mean() < 2e-4
     assert np.all(np.abs(codes - q_or) <= 1)
     deq = codes * step.cpu().numpy()[:, None]
     assert np.all(np.abs(deq - want) <= 0.5001 * s_or[:, None] + 1e-6)

@@ -257,6 +257,57 @@ def test_estimate_is_unbiased_in_expectation():
     assert abs(float(acc @ grad / (grad @ grad)) - 1.0) < 0.25
 
 
+def test_one_dimensional_smoothed_gradient_through_the_quantiser():
+    """Appendix G, Lemma 2 and the remark after it: d = 1, loss L = G * Q(w) with a uniform quantiser of step Delta.
+    Gaussian smoothing of the staircase gives the closed form
+        grad f_eps(W) = (G * Delta / eps) * sum_k phi((theta_k - W) / eps),   theta_k = (k + 1/2) * Delta,
+    which the two-point estimate of Eq. (1) must reproduce in expectation THROUGH the quantiser; it peaks on a
+    threshold, decays like exp(-t^2 / 2) with t = (distance to the nearest threshold) / eps, stays below the lemma's
+    bound, and is exactly zero once no direction the generator can draw reaches a threshold.
+    Element i of a constant tensor plays the role of the i-th independent draw (the direction is addressed by element
+    index), so one call of the oracle's perturbation and quantiser evaluates 2^22 one-dimensional problems."""
+    from oracle.model import adaptive_weight_quant
+    G, delta, bits, zero_point, n = 3.0, np.float32(0.01), 4, 8.0, 1 << 22
+    theta = np.array([[[delta, zero_point, 0.0, 1.0]]], np.float32)       # fixed grid: value = Delta * round(w / Delta)
+    phi = lambda x: np.exp(-0.5 * x * x) / math.sqrt(2.0 * math.pi)
+
+    def closed_form(W, eps):
+        k = np.arange(-8, 8)                                              # every threshold of the 4-bit grid
+        return G * float(delta) / eps * float(phi(((k + 0.5) * float(delta) - W) / eps).sum())
+
+    def estimate(W, eps, seed):
+        w = np.full((1, n), W, np.float32)
+        u = core.normal(seed, 77, n).astype(np.float64)
+        e32 = np.float32(eps)
+        _, qp = adaptive_weight_quant(core.perturb(w, seed, 77, e32), theta, n, bits)
+        _, qm = adaptive_weight_quant(core.perturb(w, seed, 77, -e32), theta, n, bits)
+        per_draw = G * (qp.astype(np.float64) - qm.astype(np.float64)).ravel() / (2.0 * float(e32)) * u      # Eq. (1), q = 1, d = 1
+        return float(per_draw.mean()), float(per_draw.std() / math.sqrt(n))
+
+    d = float(delta)
+    eps = 2e-3                                                             # Delta / eps = 5
+    seen = []
+    for i, W in enumerate([0.5 * d, 0.25 * d, 0.0, -1.5 * d + 0.1 * d, 2.0 * d]):
+        got, se = estimate(W, eps, 4000 + i)
+        want = closed_form(W, eps)
+        assert abs(got - want) <= 5.0 * se + 2e-3 * want, (W, got, want, se)
+        r = min(abs(W - (k + 0.5) * d) for k in range(-8, 8))
+        t = r / eps
+        if t > 0:       # Lemma 2
+            assert abs(got) <= G / math.sqrt(2 * math.pi) * (d / eps + 2 * t + 2 / t) * math.exp(-0.5 * t * t) + 5.0 * se
+        seen.append(want)
+    assert abs(seen[0] - G * 5 * (phi(0.0) + 2 * phi(5.0))) < 1e-3 * seen[0]      # on a threshold: G * (Delta/eps) * phi(0), plus the neighbours
+    assert seen[0] > seen[1] > seen[2] and abs(seen[2] - seen[4]) < 1e-12          # mid-cell values repeat with the grid's period
+    # away from every threshold by more than the largest |u| the generator draws (6.23): the estimate is exactly 0,
+    # and the closed form is below 1e-20
+    got, se = estimate(0.0, 5e-4, 4100)                                    # t = 10
+    assert got == 0.0 and se == 0.0 and closed_form(0.0, 5e-4) < 1e-20
+    # a planted mistake is caught: the one-sided difference (L(W + eps u) - L(W)) / eps has the same expectation only
+    # for a smooth loss; dropping the 1/2 of the symmetric form doubles the estimate
+    got, se = estimate(0.25 * d, eps, 4200)
+    assert abs(2.0 * got - closed_form(0.25 * d, eps)) > 20.0 * se
+
+
 def test_more_directions_reduce_the_estimator_error():
     """Eq. (1) with q directions and Proposition 1 (ii): the mean squared error of the estimate falls like 1/q.
     Quantiser off; the squared distance between (1/q) sum g_i u_i and the autograd gradient, averaged over

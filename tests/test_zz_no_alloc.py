@@ -6,7 +6,9 @@ latency-critical loop that cannot afford the device-wide stall of cudaMalloc/cud
 plug-in whose host bans allocation calls.  Its scratch is an array built into the library,
 shared by every call and never cleared between calls, so this test runs it TWICE in a row,
 the second time on a smaller problem with different labels, and checks both results against
-zoqat_op_head_loss (caller-provided scratch) through the C ABI.  The file is named so that
+zoqat_op_head_loss (caller-provided scratch) through the C ABI, and against the plain float64
+definition of the per-position cross-entropy (logsumexp of the logits minus the label's logit),
+so that the comparison is not one CUDA path against another only.  The file is named so that
 pytest collects it after every other test.
 """
 import numpy as np
@@ -54,6 +56,15 @@ def test_static_scratch_matches_caller_scratch_twice(zq, impl):
         assert torch.allclose(tl, want_tl, rtol=0, atol=3e-6 * scale)
         assert abs(float(ls.item()) - float(want_sum.item())) <= 1e-6 * abs(float(want_sum.item()))
         assert torch.all(tl[labels < 0] == 0)
+        # the definition itself, in float64 on the host (both operands are exact bf16 values)
+        logits = a.double().cpu().numpy() @ b.double().cpu().numpy().T
+        mx = logits.max(-1)
+        lse = mx + np.log(np.exp(logits - mx[:, None]).sum(-1))
+        lab = labels.cpu().numpy()
+        valid = lab >= 0
+        ref = np.where(valid, lse - logits[np.arange(T), np.where(valid, lab, 0)], 0.0)
+        assert np.allclose(tl.cpu().numpy(), ref, rtol=0, atol=3e-6 * np.abs(lse).max())
+        assert abs(float(ls.item()) - ref.sum()) <= 1e-6 * abs(ref.sum())
 
 
 def test_static_scratch_rejects_oversized_problem(zq):
