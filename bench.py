@@ -1,12 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the ZO-QAT step (two quantised forwards + seeded update) on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference] [--mode batch|directions]
 
 One step = one full pass of the hot path over one synthetic batch.  Default
 workload: LLaMA-7B shape, W4A8 (group-128 asymmetric weights, per-token int8
 activations), batch 4 x seq 1024.  Prints ONE JSON line (rank 0).
 --impl reference times the CPU oracle on a bounded sample of the same workload.
+
+--gpus N > 1: one process per GPU.  Under a launcher (torchrun: RANK / WORLD_SIZE / LOCAL_RANK set) this process is one
+rank; started plainly it launches the N ranks itself (torch.distributed.run on 127.0.0.1) and relays rank 0's line.
+--mode batch (default): replicas shard the mini-batch, one 24-byte all-reduce per step.  --mode directions: every
+replica evaluates its own direction on the same batch (Eq. (1) with q = N) and applies all N updates.
 """
 import argparse
 import json
@@ -176,7 +181,7 @@ def run_reference(args, w, rank, world):
 def run_ours(args, w, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_2509_00031_b200 import binding, synth
+    from paper_2509_00031_b200 import binding, replicas, synth
 
     torch.cuda.set_device(local_rank)
     if world > 1:
@@ -202,28 +207,28 @@ def run_ours(args, w, rank, world, local_rank):
                 if l < ftl or (names is not None and name not in names):
                     params["layers"][l][name] = None
         torch.cuda.empty_cache()
-    # weak scaling: each rank gets its own batch shard of the workload's size
-    tok_np, lab_np = synth.make_batch(w["batch"], w["seq"], w["vocab"], seed=1234 + rank)
+    # weak scaling: each rank gets its own batch shard of the workload's size (its own direction on the same batch in
+    # --mode directions)
+    tok_np, lab_np = synth.make_batch(w["batch"], w["seq"], w["vocab"], seed=1234 + (0 if args.mode == "directions" else rank))
     tokens, labels = torch.from_numpy(tok_np).cuda(), torch.from_numpy(lab_np).cuda()
     tok_host, lab_host = torch.from_numpy(tok_np).pin_memory(), torch.from_numpy(lab_np).pin_memory()
     result = torch.zeros(6, dtype=torch.float32, device="cuda")
     sums = torch.zeros(3, dtype=torch.float64, device="cuda")
 
     learned = bool(w.get("adaptive_quant") or w.get("smoothing"))
+    scales = torch.zeros(world, dtype=torch.float32, device="cuda")
 
     def step(t):
-        if world == 1 and learned:
+        if args.mode == "directions":                      # q = world directions per step, one per replica, same batch
+            replicas.direction_parallel_step(model, dist, rank, world, tokens, labels, 1000 + world * t, EPS, LR, sums, result, scales)
+        elif world == 1 and learned:
             model.zoqat_step_rates(tokens, labels, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
         elif world == 1:
             # Eq. (2) of step t rides on the operand producers of step t + 1; the last one is flushed inside the timed region
             model.zoqat_step_deferred(tokens, labels, 1000 + t, EPS, LR, result)
         else:                                              # data-parallel replicas: 24-byte all-reduce between the halves
-            model.zoqat_step_begin(tokens, labels, 1000 + t, EPS, sums)
-            dist.all_reduce(sums)
-            if learned:
-                model.zoqat_step_finish_rates(sums, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
-            else:
-                model.zoqat_step_finish_deferred(sums, 1000 + t, EPS, LR, result)
+            replicas.batch_sharded_step(model, dist, world, tokens, labels, 1000 + t, EPS, LR, sums, result,
+                                        (LR_QUANT, LR_SMOOTH) if learned else None)
 
     def barrier():
         if world > 1:
@@ -257,7 +262,7 @@ def run_ours(args, w, rank, world, local_rank):
     res = binding.decode_step_result(result)
     # ---- end-to-end: the host-buffer entry point, copies inside the timed region
     e2e_ms = None
-    if world == 1:
+    if world == 1 and args.mode == "batch":
         barrier()
         t0 = time.perf_counter()
         for t in range(args.steps):
@@ -289,6 +294,7 @@ def run_ours(args, w, rank, world, local_rank):
         data="synthetic", fwd_tokens_per_s=2 * nums["T"] * steps_per_s,
         config=dict(workload=args.workload, l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
                     gemm="simt" if args.simt else "tcgen05",
+                    mode="batch-sharded replicas" if args.mode == "batch" else "direction-parallel replicas (q = n_gpus, value counts two-point evaluations)",
                     **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab", "w_bits", "w_group",
                                          "a_bits", "batch", "seq")}),
         step_roofline=dict(bound="tensor" if t_flop >= t_hbm else "hbm", flops_per_step=nums["flops"],
@@ -304,6 +310,8 @@ def run_ours(args, w, rank, world, local_rank):
         gpu_launches=launches, clocks=clocks,
         last_step=dict(loss_plus=res["loss_plus"], loss_minus=res["loss_minus"], proj_grad=res["proj_grad"], status=res["status"]),
     )
+    if args.mode == "directions":
+        line["step_roofline"] = None          # the roofline model below is that of the one-direction step
     if e2e_ms is not None:
         line["e2e"] = dict(value=1e3 * args.steps / e2e_ms, unit=UNIT, h2d_bytes_per_step=2 * nums["T"] * 4, d2h_bytes_per_step=24)
     # release the device before the CPU baseline runs
@@ -317,6 +325,21 @@ def run_ours(args, w, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def launch_ranks(n, argv):
+    """Starts n local ranks of this script (one per GPU) under torch.distributed.run and relays their output; returns
+    the launcher's exit code.  NCCL's communicator summary is left on (NCCL_DEBUG=INFO unless the caller set it)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -327,12 +350,19 @@ def main():
     ap.add_argument("--simt", action="store_true", help="use the CUDA-core cross-check GEMM instead of tcgen05")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="time every kernel category, not only the GEMM launches (adds ~1 %% to the step)")
+    ap.add_argument("--mode", default="batch", choices=["batch", "directions"])
+    ap.add_argument("--rank-probe", action="store_true", help="print this process' rank / world size as JSON and exit before any device is touched")
     args = ap.parse_args()
-    from paper_2509_00031_b200 import synth
-    w = dict(synth.WORKLOADS[args.workload])
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1 and (args.impl == "ours" or args.rank_probe):
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.rank_probe:
+        print(json.dumps(dict(rank=rank, world=world, local_rank=local_rank, pid=os.getpid())), flush=True)
+        return
+    from paper_2509_00031_b200 import synth
+    w = dict(synth.WORKLOADS[args.workload])
     if args.impl == "reference":
         run_reference(args, w, rank, world)
         return

@@ -258,6 +258,21 @@ int zoqat_step_host_deferred(zoqat_model_t* m, const int32_t* tokens_host, const
 /* Eq. (2) alone: W <- W - scale * u(seed) on every TRAINABLE tensor (and on the Section 4.2 parameters);
  * the _rates form takes one factor per parameter class. */
 int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream);
+
+/* Eq. (2) for q = n_dirs directions with caller-supplied seeds and factors (Eq. (1) averages over q directions;
+ * Appendix G, Proposition 1 (ii): the estimator's error falls like 1/q): W <- W - sum_i scales[i] * u(seeds[i]),
+ * applied direction by direction (i = 0, 1, ...: one binary32 fma per element each) in ONE pass over every TRAINABLE
+ * tensor and over the Section 4.2 parameters, every class with the same factor.  It is the update half of
+ * zoqat_step_multi, for callers that evaluated the directions elsewhere - e.g. q replicas that each ran both passes
+ * of one direction on the same batch and exchanged (seed_i, fl((lr/q) g_i)): every replica then applies all q updates
+ * and the masters stay bit-identical.  seeds_host: host memory, read before the call returns; scales_dev: device
+ * memory, fp32 [n_dirs], read when the kernels run; 1 <= n_dirs <= 64.  A pending deferred update is applied first. */
+int zoqat_apply_update_multi(zoqat_model_t* m, const uint64_t* seeds_host, const float* scales_dev, int n_dirs, void* stream);
+
+/* Eq. (1) alone, from the sums zoqat_step_begin produced (all-reduced or not): fills the result record - L+, L-,
+ * g = (L+ - L-) / (2 eps), fl(lr * g) - and leaves every master untouched.  With zoqat_apply_update_multi it lets a
+ * caller separate the evaluation of a direction from the update (pass lr / q as lr for q directions). */
+int zoqat_step_result(zoqat_model_t* m, const double* sums_dev, float eps, float lr, zoqat_step_result_t* result_dev, void* stream);
 int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float scale_quant, float scale_smooth,
                              void* stream);
 

@@ -445,8 +445,12 @@ class OracleModel:
         """Eq. (1) with q = n_dirs directions u_1..u_q (seeds seed, seed+1, ...), all evaluated at the same W, then
         Eq. (2): W <- W - (lr/q) sum_i g_i u_i, applied direction by direction (one binary32 fma per element each).
         Returns the list of (L+, L-, g_i)."""
-        out = [self.projected_gradient(tokens, labels, seed + i, eps) for i in range(n_dirs)]
-        lr_q = F32(F32(lr) / F32(n_dirs))
-        for i, (_, _, g) in enumerate(out):
-            self.apply_update(seed + i, F32(lr_q * g))
+        return self.step_seeds(tokens, labels, [seed + i for i in range(n_dirs)], eps, lr)
+
+    def step_seeds(self, tokens, labels, seeds, eps, lr):
+        """step_multi with the directions named by an explicit list of seeds."""
+        out = [self.projected_gradient(tokens, labels, sd, eps) for sd in seeds]
+        lr_q = F32(F32(lr) / F32(len(seeds)))
+        for sd, (_, _, g) in zip(seeds, out):
+            self.apply_update(sd, F32(lr_q * g))
         return [(lp, lm, float(g)) for lp, lm, g in out]

@@ -28,7 +28,7 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
     "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_finish_deferred", "zoqat_flush_update", "zoqat_step_multi",
-    "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates",
+    "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates", "zoqat_apply_update_multi", "zoqat_step_result",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_debug_capture", "zoqat_debug_capture_bytes", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
@@ -104,6 +104,8 @@ def lib():
             "zoqat_step_begin": [vp, vp, vp, i32, i32, u64, f32, vp, vp],
             "zoqat_step_finish": [vp, vp, u64, f32, f32, vp, vp],
             "zoqat_apply_update": [vp, u64, f32, vp],
+            "zoqat_apply_update_multi": [vp, P(u64), vp, i32, vp],
+            "zoqat_step_result": [vp, vp, f32, f32, vp, vp],
             "zoqat_check": [vp, vp],
             "zoqat_launch_count": [vp, P(i64)],
             "zoqat_debug_buffer": [vp, i32, P(vp), P(sz)],
@@ -553,6 +555,18 @@ class ZoqatModel:
 
     def zoqat_apply_update(self, seed, scale):
         _check(lib().zoqat_apply_update(self.handle, seed, scale, _stream()))
+
+    def zoqat_apply_update_multi(self, seeds, scales):
+        """seeds: sequence of q integers (host); scales: float32 device tensor [q]."""
+        q = len(seeds)
+        arr = (ctypes.c_uint64 * q)(*[int(x) for x in seeds])
+        _check(lib().zoqat_apply_update_multi(self.handle, arr, _p(scales), q, _stream()))
+
+    def zoqat_step_result(self, sums, eps, lr, result=None):
+        """Eq. (1) from the sums of zoqat_step_begin; no update."""
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        _check(lib().zoqat_step_result(self.handle, _p(sums), eps, lr, _p(result), _stream()))
+        return result
 
     def zoqat_check(self):
         _check(lib().zoqat_check(self.handle, _stream()))

@@ -535,6 +535,33 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
         launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
 }
 
+// Eq. (2) for n_dirs directions in one pass over every trainable tensor (Section 4.2 parameters included): direction i
+// under seeds.s[i] with the factor scales[i * stride] (device memory), applied in the order i = 0, 1, ...
+void update_all_multi(zoqat_model* m, const SeedList& seeds, int n_dirs, const float* scales, int stride, cudaStream_t s) {
+    ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r) {
+            Linear& L = Ly.lin[r];
+            if (L.present && L.trainable()) {
+                launch_update_multi(L.w_mut, (uint64_t)(L.rows * L.cols), seeds, n_dirs, L.tid, scales, stride, s);
+                if (L.adaptive())
+                    launch_update_multi(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, seeds, n_dirs, L.tid_q(), scales, stride, s);
+            }
+        }
+    for (size_t l = 0; l < m->layers.size(); ++l) {
+        Layer& Ly = m->layers[l];
+        if (!Ly.smoothing) continue;
+        for (int pt = 0; pt < 4; ++pt) {
+            const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
+            const uint64_t n = pt == 3 ? (uint64_t)m->cfg.d_ffn : (uint64_t)m->cfg.d_model;
+            launch_update_multi(Ly.smooth_s[pt], n, seeds, n_dirs, 0x20000u + base, scales, stride, s);
+            launch_update_multi(Ly.smooth_d[pt], n, seeds, n_dirs, 0x30000u + base, scales, stride, s);
+        }
+    }
+    if (m->head.trainable())
+        launch_update_multi(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seeds, n_dirs, m->head.tid, scales, stride, s);
+}
+
 // Applies a deferred update now (every entry point that reads or changes the masters starts with this).
 void flush_pending(zoqat_model* m, cudaStream_t s) {
     if (!m->pending) return;
@@ -889,31 +916,9 @@ int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
         launch_finish_step(m->ws.sums, eps, lr_q, m->ws.err_flag, res + i, s);
     }
     // ... then Eq. (2) for all of them in one pass over each trainable tensor
-    {
-        ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
-        const int stride = (int)(sizeof(zoqat_step_result_dev) / sizeof(float));
-        for (auto& Ly : m->layers)
-            for (int r = 0; r < 7; ++r) {
-                Linear& L = Ly.lin[r];
-                if (L.present && L.trainable()) {
-                    launch_update_multi(L.w_mut, (uint64_t)(L.rows * L.cols), seed, n_dirs, L.tid, &res->update_scale, stride, s);
-                    if (L.adaptive())
-                        launch_update_multi(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, seed, n_dirs, L.tid_q(), &res->update_scale, stride, s);
-                }
-            }
-        for (size_t l = 0; l < m->layers.size(); ++l) {
-            Layer& Ly = m->layers[l];
-            if (!Ly.smoothing) continue;
-            for (int pt = 0; pt < 4; ++pt) {
-                const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
-                const uint64_t n = pt == 3 ? (uint64_t)m->cfg.d_ffn : (uint64_t)m->cfg.d_model;
-                launch_update_multi(Ly.smooth_s[pt], n, seed, n_dirs, 0x20000u + base, &res->update_scale, stride, s);
-                launch_update_multi(Ly.smooth_d[pt], n, seed, n_dirs, 0x30000u + base, &res->update_scale, stride, s);
-            }
-        }
-        if (m->head.trainable())
-            launch_update_multi(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, n_dirs, m->head.tid, &res->update_scale, stride, s);
-    }
+    SeedList seeds{};
+    for (int i = 0; i < n_dirs; ++i) seeds.s[i] = seed + (uint64_t)i;
+    update_all_multi(m, seeds, n_dirs, &res->update_scale, (int)(sizeof(zoqat_step_result_dev) / sizeof(float)), s);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
@@ -957,6 +962,28 @@ int zoqat_apply_update_rates(zoqat_model_t* m, uint64_t seed, float scale, float
 
 int zoqat_apply_update(zoqat_model_t* m, uint64_t seed, float scale, void* stream) {
     return zoqat_apply_update_rates(m, seed, scale, scale, scale, stream);
+}
+
+int zoqat_apply_update_multi(zoqat_model_t* m, const uint64_t* seeds_host, const float* scales_dev, int n_dirs, void* stream) {
+    if (!m || !seeds_host || !scales_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (n_dirs < 1 || n_dirs > kMaxDirections) return fail(ZOQAT_ERR_INVALID_ARG, "n_dirs %d (supported: 1..%d)", n_dirs, kMaxDirections);
+    if (m->broken) return fail(ZOQAT_ERR_BAD_STATE, "the masters are partially updated (an earlier step failed): create a new handle");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    flush_pending(m, s);
+    SeedList seeds{};
+    for (int i = 0; i < n_dirs; ++i) seeds.s[i] = seeds_host[i];
+    update_all_multi(m, seeds, n_dirs, scales_dev, 1, s);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_step_result(zoqat_model_t* m, const double* sums_dev, float eps, float lr, zoqat_step_result_t* result_dev, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (!sums_dev || !result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev/result_dev are NULL");
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, reinterpret_cast<zoqat_step_result_dev*>(result_dev), static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
 }
 
 int zoqat_check(zoqat_model_t* m, void* stream) {

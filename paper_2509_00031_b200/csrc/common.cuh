@@ -121,8 +121,10 @@ void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_
 // w <- w - scale*u; scale = *scale_ptr if scale_ptr != NULL else scale_val.
 void launch_update(float* w, uint64_t n, uint64_t seed, uint32_t tid, const float* scale_ptr, float scale_val, cudaStream_t s);
 
-// q directions at once: w <- fma(-scales[i*scale_stride], u(seed + i), w), i = 0..n_dirs-1 in order.
-void launch_update_multi(float* w, uint64_t n, uint64_t seed, int n_dirs, uint32_t tid, const float* scales,
+// q directions at once: w <- fma(-scales[i*scale_stride], u(seeds.s[i]), w), i = 0..n_dirs-1 in order.
+constexpr int kMaxDirections = 64;
+struct SeedList { uint64_t s[kMaxDirections]; };
+void launch_update_multi(float* w, uint64_t n, const SeedList& seeds, int n_dirs, uint32_t tid, const float* scales,
                          int scale_stride, cudaStream_t s);
 
 void launch_embed(const int32_t* tokens, const float* embed, const float* pos, int64_t T, int seq, int d,

@@ -21,6 +21,7 @@
 #include "../../include/zoqat.h"
 #include "tc_ptx.cuh"
 #include <cuda_fp16.h>
+#include <cstdlib>
 
 namespace zq {
 namespace {
@@ -67,6 +68,10 @@ struct TcParams {
     float* label_logit;
     int32_t* err_flag;
     int tiles_m, tiles_n;
+    // tile order inside a pass (tile_coords): group_n == 0: blocks of `group` row tiles, column tiles swept inside a
+    // block with the row tile fastest; group_n == 1: blocks of `group` column tiles, the column tile fastest
+    int group, group_n;
+    int hint_a, hint_b, hint_out;      // kL2* eviction priority of the A loads, the B loads and the result stores
     int tma_out;              // 1: mode-0 results leave through map_out (needs N % 4 == 0)
     uint32_t* row_amax;       // mode 3: [Z*M] running max |act| per row (bit pattern of a non-negative float)
     // mode 2: the q | k | v projection writes the attention operands
@@ -86,6 +91,20 @@ __device__ __forceinline__ void split_half(float x, __half& hi, __half& lo) {
 }
 __device__ __forceinline__ uint32_t pack_half2(__half a, __half b) {
     return (uint32_t)__half_as_ushort(a) | ((uint32_t)__half_as_ushort(b) << 16);
+}
+
+// Tile r of a pass -> (row tile, column tile).  The persistent CTAs take tiles r, r + units, ..., so the tiles in flight
+// at any time are consecutive r: a block of `group` tiles of one operand (kept in L2) times a sliding window of the other.
+__device__ __forceinline__ void tile_coords(const TcParams& p, int r, int& tm, int& tn) {
+    if (p.group_n == 0) {
+        const int per = p.group * p.tiles_n, g = r / per, rr = r - g * per, m0 = g * p.group;
+        const int gm = min(p.group, p.tiles_m - m0);
+        tm = m0 + rr % gm; tn = rr / gm;
+    } else {
+        const int per = p.group * p.tiles_m, g = r / per, rr = r - g * per, n0 = g * p.group;
+        const int gn = min(p.group, p.tiles_n - n0);
+        tn = n0 + rr % gn; tm = rr / gn;
+    }
 }
 
 template <int BN, int CG>
@@ -140,9 +159,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            const uint64_t pol_a = l2_policy(p.hint_a), pol_b = l2_policy(p.hint_b);
             for (int t = unit; t < total_tiles && ok; t += n_units) {
                 const int z = t / tiles_per_z, r = t % tiles_per_z;
-                const int tm = r % p.tiles_m, tn = r / p.tiles_m;     // m fastest: neighbours share B
+                int tm, tn;
+                tile_coords(p, r, tm, tn);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u)) { atomicExch(p.err_flag, kErrWaitEmpty); ok = false; break; }
                     const uint32_t a_dst = tiles + stage * Cfg::kStageBytes;
@@ -150,14 +171,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         // both CTAs' bytes are counted on the leader's barrier, which expects them all
                         if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::kStageBytes);
                         const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
-                        tma_load_3d_pair(a_dst, &map_a, lead_full, kb * BK, tm * TM + (int)rank * BM, z);
+                        tma_load_3d_pair_hint(a_dst, &map_a, lead_full, kb * BK, tm * TM + (int)rank * BM, z, pol_a);
                         // mode 3: the tile's first 128 columns are gate features, the last 128 the matching up features
                         const int b_row = p.mode == 3 ? (int)rank * (int)(p.N / 2) + tn * (BN / 2) : tn * BN + (int)rank * (BN / 2);
-                        tma_load_3d_pair(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, b_row, z);
+                        tma_load_3d_pair_hint(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, b_row, z, pol_b);
                     } else {
                         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
-                        tma_load_3d(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z);
-                        tma_load_3d(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z);
+                        tma_load_3d_hint(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z, pol_a);
+                        tma_load_3d_hint(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z, pol_b);
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -209,9 +230,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter+32)
         int acc = 0; uint32_t acc_phase = 0;
         int out_buf = 0;
+        const uint64_t pol_out = l2_policy(p.hint_out);
         for (int t = unit; t < total_tiles; t += n_units) {
             const int z = t / tiles_per_z, r = t % tiles_per_z;
-            const int tm = r % p.tiles_m, tn = r / p.tiles_m;
+            int tm, tn;
+            tile_coords(p, r, tm, tn);
             // the whole warp takes the same decision: the TMEM loads below are warp-collective
             if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc), acc_phase))) {
                 if (lane == 0) atomicExch(p.err_flag, kErrWaitAccFull);
@@ -382,7 +405,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_3d(&map_out, box, tn * (BN / 2) + c * 32, tm * TM + (int)rank * BM + quarter * 32, z);
+                        tma_store_3d_hint(&map_out, box, tn * (BN / 2) + c * 32, tm * TM + (int)rank * BM + quarter * 32, z, pol_out);
                         bulk_commit();
                     }
                     out_buf ^= 1;
@@ -429,8 +452,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) {
                         const int y0 = tm * TM + (int)rank * BM + quarter * 32;
-                        if (p.accumulate) tma_reduce_add_3d(&map_out, box, (int)n0, y0, z);
-                        else tma_store_3d(&map_out, box, (int)n0, y0, z);
+                        if (p.accumulate) tma_reduce_add_3d_hint(&map_out, box, (int)n0, y0, z, pol_out);
+                        else tma_store_3d_hint(&map_out, box, (int)n0, y0, z, pol_out);
                         bulk_commit();
                     }
                     out_buf ^= 1;
@@ -574,6 +597,47 @@ int num_sms() {
     return n;
 }
 
+// Tile order and L2 priorities of one launch.  A pass reads A (M x K) and B (N x K) once each at best; what is re-read
+// depends on which operand block stays in L2 while the other streams past it.  With blocks of g row tiles resident,
+// B is streamed once per block: bytes = A + B * ceil(tiles_m / g); with blocks of column tiles, the mirror image.
+// The cheaper of the two is taken, with the block sized to `resident` bytes of L2 (well below the 126 MB, which also
+// hold the stream in flight and the results), blocks evened out, the block's operand loaded evict_last and the rest
+// evict_first.
+struct TileOrder { int group, group_n, hint_a, hint_b, hint_out; };
+
+long env_long(const char* name, long dflt) {
+    const char* v = getenv(name);
+    return v ? atol(v) : dflt;
+}
+
+TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows) {
+    const double resident = (double)env_long("ZOQAT_GEMM_RESIDENT_MB", 48) * 1048576.0;
+    const long hints = env_long("ZOQAT_GEMM_HINTS", 3), force = env_long("ZOQAT_GEMM_ORDER", -1);
+    const double a_bytes = (double)M * K * 2, b_bytes = (double)N * K * 2;
+    auto even = [](int tiles, double strip, double cap) {
+        int g = (int)(cap / strip);
+        if (g < 1) g = 1;
+        if (g > tiles) g = tiles;
+        const int blocks = (tiles + g - 1) / g;
+        return (tiles + blocks - 1) / blocks;
+    };
+    const int gm = even(tiles_m, (double)tm_rows * K * 2, resident), gn = even(tiles_n, (double)tn_rows * K * 2, resident);
+    const double cost_m = a_bytes + b_bytes * ((tiles_m + gm - 1) / gm), cost_n = b_bytes + a_bytes * ((tiles_n + gn - 1) / gn);
+    TileOrder o;
+    const bool by_n = force < 0 ? cost_n < cost_m : force == 2;
+    o.group_n = by_n ? 1 : 0;
+    o.group = by_n ? gn : gm;
+    if (force == 0) { o.group_n = 0; o.group = tiles_m; }          // every row tile of a pass, column by column
+    const bool all_fit = a_bytes + b_bytes <= resident;
+    o.hint_a = o.hint_b = kL2Normal;
+    if ((hints & 1) && !all_fit) {
+        o.hint_a = o.group_n ? kL2EvictFirst : kL2EvictLast;
+        o.hint_b = o.group_n ? kL2EvictLast : kL2EvictFirst;
+    }
+    o.hint_out = (hints & 2) ? kL2EvictFirst : kL2Normal;
+    return o;
+}
+
 template <int BN, int CG>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
     using Cfg = TileCfg<BN, CG>;
@@ -621,6 +685,10 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
         cudaFuncSetAttribute(gemm_tc_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
         attr.retry();
         return ZOQAT_ERR_CUDA;
+    }
+    {
+        const TileOrder o = choose_order(a.M, a.N, a.K, p.tiles_m, p.tiles_n, BM * CG, BN);
+        p.group = o.group; p.group_n = o.group_n; p.hint_a = o.hint_a; p.hint_b = o.hint_b; p.hint_out = o.hint_out;
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
     const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)

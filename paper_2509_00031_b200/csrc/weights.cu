@@ -726,9 +726,9 @@ update_kernel(float* __restrict__ w, uint64_t n, const PhiloxKeys rk, uint32_t t
 }
 
 // Eq. (2) with q directions in one pass over the tensor: w <- fma(-c_i, u_i, w) for i = 0..q-1 in that order,
-// direction i under seed + i, c_i read from scales[i * scale_stride] (device memory).
+// direction i under seeds.s[i], c_i read from scales[i * scale_stride] (device memory).
 __global__ void __launch_bounds__(kThreads)
-update_multi_kernel(float* __restrict__ w, uint64_t n, uint64_t seed, int n_dirs, uint32_t tid,
+update_multi_kernel(float* __restrict__ w, uint64_t n, const SeedList seeds, int n_dirs, uint32_t tid,
                     const float* __restrict__ scales, int scale_stride) {
     __shared__ float2 tab[kIcdfKnots];
     stage_icdf_table(tab);
@@ -740,7 +740,7 @@ update_multi_kernel(float* __restrict__ w, uint64_t n, uint64_t seed, int n_dirs
         if (whole) { const float4 t = w4[b]; x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
         else for (int j = 0; j < 4; ++j) x[j] = 4 * b + j < n ? w[4 * b + j] : 0.0f;
         for (int i = 0; i < n_dirs; ++i) {
-            const uint64_t sd = seed + (uint64_t)i;
+            const uint64_t sd = seeds.s[i];
             const float c = -scales[(size_t)i * scale_stride];
             const float4 z = direction4(tab, (uint32_t)sd, (uint32_t)(sd >> 32), tid, b);
             x[0] = __fmaf_rn(c, z.x, x[0]); x[1] = __fmaf_rn(c, z.y, x[1]);
@@ -753,10 +753,10 @@ update_multi_kernel(float* __restrict__ w, uint64_t n, uint64_t seed, int n_dirs
 
 }  // namespace
 
-void launch_update_multi(float* w, uint64_t n, uint64_t seed, int n_dirs, uint32_t tid, const float* scales,
+void launch_update_multi(float* w, uint64_t n, const SeedList& seeds, int n_dirs, uint32_t tid, const float* scales,
                          int scale_stride, cudaStream_t s) {
-    if (n == 0 || n_dirs <= 0 || !ensure_icdf_table()) return;
-    update_multi_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(w, n, seed, n_dirs, tid, scales, scale_stride);
+    if (n == 0 || n_dirs <= 0 || n_dirs > kMaxDirections || !ensure_icdf_table()) return;
+    update_multi_kernel<<<stream_grid((int64_t)((n + 3) / 4), kThreads), kThreads, 0, s>>>(w, n, seeds, n_dirs, tid, scales, scale_stride);
     count_launch();
 }
 

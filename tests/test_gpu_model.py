@@ -361,6 +361,48 @@ def test_step_multi_directions(zq):
     assert torch.equal(a.params["layers"][0]["wq"], b.params["layers"][0]["wq"]) and torch.equal(a.params["lm_head"], b.params["lm_head"])
 
 
+def test_apply_update_multi_and_direction_parallel_step(zq):
+    """Eq. (2) for caller-supplied (seed_i, factor_i): one fused pass, bit for bit the oracle's direction-by-direction
+    update (arbitrary, non-consecutive seeds); zoqat_step_result leaves the masters alone; and the direction-parallel
+    call order on one replica (q = 1) is zoqat_step."""
+    from oracle import core
+    from oracle.model import tensor_id, LM_HEAD_ID
+    from paper_2509_00031_b200 import replicas
+    shape, batch, seq = SMALL_LLAMA, 2, 96
+    model, oracle = build_pair(zq, shape, batch, seq, 0)
+    seeds = [17, 2 ** 40 + 5, 3, 18]
+    scales = np.array([3e-4, -1e-4, 2.5e-5, 7e-4], np.float32)
+    model.zoqat_apply_update_multi(seeds, dev(scales))
+    model.zoqat_check()
+    for sd, c in zip(seeds, scales):
+        oracle.apply_update(sd, c)
+    for l in range(shape["n_layers"]):
+        for n in oracle.linear_names():
+            assert np.array_equal(model.params["layers"][l][n].cpu().numpy().view(np.uint32), oracle.p["layers"][l][n].view(np.uint32)), (l, n)
+    assert np.array_equal(model.params["lm_head"].cpu().numpy().view(np.uint32), oracle.p["lm_head"].view(np.uint32))
+    with pytest.raises(zq.ZoqatError):
+        model.zoqat_apply_update_multi(list(range(65)), dev(np.zeros(65, np.float32)))
+    # the two halves of a direction-parallel step on a single replica against zoqat_step
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=19)
+    td, ld = dev(tokens), dev(labels)
+    twin, _ = build_pair(zq, shape, batch, seq, 0)
+    sync_masters(twin, oracle)
+    before = model.params["layers"][1]["wq"].clone()
+    sums = torch.zeros(3, dtype=torch.float64, device="cuda")
+    model.zoqat_step_begin(td, ld, 900, 1e-3, sums)
+    rec = model.zoqat_step_result(sums, 1e-3, 1e-4)
+    assert torch.equal(before, model.params["layers"][1]["wq"])                     # Eq. (1) only
+    result, sc = torch.zeros(6, device="cuda"), torch.zeros(1, device="cuda")
+    replicas.direction_parallel_step(model, None, 0, 1, td, ld, 900, 1e-3, 1e-4, sums, result, sc)
+    want = twin.zoqat_step(td, ld, 900, 1e-3, 1e-4)
+    assert torch.equal(result.view(torch.int32), want.view(torch.int32)) and torch.equal(rec.view(torch.int32), want.view(torch.int32))
+    for l in range(shape["n_layers"]):
+        for n in oracle.linear_names():
+            assert torch.equal(model.params["layers"][l][n], twin.params["layers"][l][n]), (l, n)
+    assert torch.equal(model.params["lm_head"], twin.params["lm_head"])
+    model.zoqat_check()
+
+
 def test_query_value_only_selection(zq):
     """Section 4.3 as the paper runs it: only the query and value projections keep full-precision masters and are
     perturbed / updated; every other block linear is frozen and pre-quantised to packed codes."""
