@@ -119,6 +119,10 @@ class OracleConfig:
     store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
                                      # residual stream) to binary32, as an implementation that keeps activations in
                                      # fp32 does; used only to measure how far two correct implementations can differ
+    accum_f32: bool = False          # True (implies store_f32) also takes every sum - linear layers, norm statistics,
+                                     # attention scores and averages, log-sum-exp - in binary32 with the library's
+                                     # summation order, as a plain binary32 implementation does; used only to measure
+                                     # how far two correct implementations can differ
     operand_bf16: bool = True        # False (with w_bits = 0, a_bits = 0) gives the unquantised float64 model, used only to pin the forward
 
 
@@ -155,8 +159,9 @@ def apply_rope(x, cos, sin):
     return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
 
 
-def causal_attention(q, k, v, n_heads, cos=None, sin=None):
-    """softmax(q k^T / sqrt(d_head) + causal mask) v per head, float64.
+def causal_attention(q, k, v, n_heads, cos=None, sin=None, dtype=np.float64):
+    """softmax(q k^T / sqrt(d_head) + causal mask) v per head, float64 (dtype = float32 only for the
+    self-disagreement measurement of OracleConfig.accum_f32).
     q, k, v: [B, S, d_model]; cos/sin: rotary tables [S, d_head/2] or None."""
     B, S, d = q.shape
     dh = d // n_heads
@@ -164,12 +169,13 @@ def causal_attention(q, k, v, n_heads, cos=None, sin=None):
     if cos is not None:
         q = apply_rope(q, cos, sin)
         k = apply_rope(k, cos, sin)
-    sc = np.einsum("bshd,bthd->bhst", q, k) / np.sqrt(np.float64(dh))
+    q, k, v = q.astype(dtype), k.astype(dtype), v.astype(dtype)
+    sc = np.einsum("bshd,bthd->bhst", q, k) / np.sqrt(dtype(dh))
     sc = np.where(np.tril(np.ones((S, S), dtype=bool))[None, None], sc, -np.inf)
     sc = sc - sc.max(axis=-1, keepdims=True)
     pr = np.exp(sc)
     pr = pr / pr.sum(axis=-1, keepdims=True)
-    return np.einsum("bhst,bthd->bshd", pr, v).reshape(B, S, d)
+    return np.einsum("bhst,bthd->bshd", pr, v).reshape(B, S, d).astype(np.float64)
 
 
 class OracleModel:
@@ -319,10 +325,10 @@ class OracleModel:
             extra = self.perturbed_weight(l, name, seed, signed_eps).astype(np.float64) @ d_.astype(np.float64)
         if self.cfg.a_bits:
             a, s = act_quant(x, self.cfg.a_bits)
-            y = (a @ self.block_operand(l, name, seed, signed_eps).T) * s.astype(np.float64)[:, None]
+            y = self._matmul_t(a, self.block_operand(l, name, seed, signed_eps)) * s.astype(np.float64)[:, None]
         else:
             a = self._operand_round(x)
-            y = a @ self.block_operand(l, name, seed, signed_eps).T
+            y = self._matmul_t(a, self.block_operand(l, name, seed, signed_eps))
         if bias is not None:
             y = y + bias.astype(np.float64)[None, :]
         if extra is not None:
@@ -330,10 +336,18 @@ class OracleModel:
         return self._store(y)
 
     def _store(self, x):
-        return x.astype(F32).astype(np.float64) if self.cfg.store_f32 else x
+        return x.astype(F32).astype(np.float64) if (self.cfg.store_f32 or self.cfg.accum_f32) else x
+
+    def _matmul_t(self, a, b):
+        """a @ b.T in float64 (binary32 with the library's summation order under accum_f32)."""
+        if self.cfg.accum_f32:
+            return (a.astype(F32) @ b.astype(F32).T).astype(np.float64)
+        return a @ b.T
 
     def norm(self, h, g, b=None):
         cfg = self.cfg
+        if cfg.accum_f32:
+            h = h.astype(F32)
         if cfg.arch == "llama":
             ms = np.mean(h * h, axis=-1, keepdims=True)
             y = h / np.sqrt(ms + np.float64(F32(cfg.norm_eps))) * g.astype(np.float64)
@@ -353,6 +367,8 @@ class OracleModel:
         """tokens, labels int [B, S]; labels < 0 are ignored.  Returns the per-position
         cross-entropy (float64 [B*S], 0 where ignored) and the valid mask."""
         logits = self.logits(tokens, seed, signed_eps)
+        if self.cfg.accum_f32:
+            logits = logits.astype(F32)
         T = logits.shape[0]
         lab = labels.reshape(-1)
         valid = lab >= 0
@@ -386,7 +402,8 @@ class OracleModel:
             self._tap(f"l{l}.q", q); self._tap(f"l{l}.k", k); self._tap(f"l{l}.v", v)
             att = causal_attention(q.reshape(B, S, d), k.reshape(B, S, d), v.reshape(B, S, d), H,
                                    cos if cfg.arch == "llama" else None,
-                                   sin if cfg.arch == "llama" else None).reshape(T, d)
+                                   sin if cfg.arch == "llama" else None,
+                                   dtype=F32 if cfg.accum_f32 else np.float64).reshape(T, d)
             att = self._store(att)
             self._tap(f"l{l}.attn", att)
             h = self._store(h + self.lin(att, l, "wo", seed, signed_eps, P.get("bo")))
@@ -407,7 +424,7 @@ class OracleModel:
         x = self.norm(h, self.p["final_norm_g"], self.p.get("final_norm_b"))
         self._tap("final_norm", x)
         a = self._operand_round(x)
-        logits = a @ self.head_operand(seed, signed_eps).T
+        logits = self._matmul_t(a, self.head_operand(seed, signed_eps))
         self._tap("logits", logits)
         return logits
 

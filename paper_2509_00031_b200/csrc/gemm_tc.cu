@@ -600,9 +600,12 @@ int num_sms() {
 // Tile order and L2 priorities of one launch.  A pass reads A (M x K) and B (N x K) once each at best; what is re-read
 // depends on which operand block stays in L2 while the other streams past it.  With blocks of g row tiles resident,
 // B is streamed once per block: bytes = A + B * ceil(tiles_m / g); with blocks of column tiles, the mirror image.
-// The cheaper of the two is taken, with the block sized to `resident` bytes of L2 (well below the 126 MB, which also
-// hold the stream in flight and the results), blocks evened out, the block's operand loaded evict_last and the rest
-// evict_first.
+// The cheaper of the two is taken, with the block sized to `resident` bytes of L2 (measured: a 32 MB block survives
+// between waves, a 64 MB one does not), blocks evened out, the block's operand loaded evict_last and everything that
+// streams (the other operand, the results) evict_first.  When the block plus the window of the streamed operand that
+// one wave of CTAs walks does not fit either (long K: every strip is K * 512 bytes), nothing survives between waves
+// and evict_first would drop strips other CTAs of the wave still need: the wave is then made as square as possible
+// (fewest distinct strips per wave) and the operands keep the default priority.
 struct TileOrder { int group, group_n, hint_a, hint_b, hint_out; };
 
 long env_long(const char* name, long dflt) {
@@ -610,31 +613,41 @@ long env_long(const char* name, long dflt) {
     return v ? atol(v) : dflt;
 }
 
-TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows) {
+TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows, int units) {
     const double resident = (double)env_long("ZOQAT_GEMM_RESIDENT_MB", 48) * 1048576.0;
     const long hints = env_long("ZOQAT_GEMM_HINTS", 3), force = env_long("ZOQAT_GEMM_ORDER", -1);
     const double a_bytes = (double)M * K * 2, b_bytes = (double)N * K * 2;
-    auto even = [](int tiles, double strip, double cap) {
-        int g = (int)(cap / strip);
+    const double strip_a = (double)tm_rows * K * 2, strip_b = (double)tn_rows * K * 2;
+    auto even = [](int tiles, int g) {
         if (g < 1) g = 1;
         if (g > tiles) g = tiles;
         const int blocks = (tiles + g - 1) / g;
         return (tiles + blocks - 1) / blocks;
     };
-    const int gm = even(tiles_m, (double)tm_rows * K * 2, resident), gn = even(tiles_n, (double)tn_rows * K * 2, resident);
+    const int gm = even(tiles_m, (int)(resident / strip_a)), gn = even(tiles_n, (int)(resident / strip_b));
     const double cost_m = a_bytes + b_bytes * ((tiles_m + gm - 1) / gm), cost_n = b_bytes + a_bytes * ((tiles_n + gn - 1) / gn);
+    // block + the streamed operand's strips one wave touches
+    const double foot_m = gm * strip_a + ((double)units / gm + 1.0) * strip_b, foot_n = gn * strip_b + ((double)units / gn + 1.0) * strip_a;
     TileOrder o;
-    const bool by_n = force < 0 ? cost_n < cost_m : force == 2;
-    o.group_n = by_n ? 1 : 0;
-    o.group = by_n ? gn : gm;
-    if (force == 0) { o.group_n = 0; o.group = tiles_m; }          // every row tile of a pass, column by column
-    const bool all_fit = a_bytes + b_bytes <= resident;
     o.hint_a = o.hint_b = kL2Normal;
-    if ((hints & 1) && !all_fit) {
-        o.hint_a = o.group_n ? kL2EvictFirst : kL2EvictLast;
-        o.hint_b = o.group_n ? kL2EvictLast : kL2EvictFirst;
-    }
     o.hint_out = (hints & 2) ? kL2EvictFirst : kL2Normal;
+    if (force == 0) { o.group_n = 0; o.group = tiles_m; return o; }          // every row tile of a pass, column by column
+    const bool by_n = cost_n < cost_m;
+    const double foot = by_n ? foot_n : foot_m;
+    if (foot <= 1.5 * resident || force == 1) {
+        o.group_n = by_n ? 1 : 0;
+        o.group = by_n ? gn : gm;
+        if ((hints & 1) && a_bytes + b_bytes > resident) {
+            o.hint_a = by_n ? kL2EvictFirst : kL2EvictLast;
+            o.hint_b = by_n ? kL2EvictLast : kL2EvictFirst;
+        }
+        return o;
+    }
+    // square wave: g row tiles x units / g column tiles with g * strip_a ~ (units / g) * strip_b
+    int g = 1;
+    while ((double)(g + 1) * (g + 1) * strip_a <= (double)units * strip_b && g + 1 <= tiles_m) ++g;
+    o.group_n = 0;
+    o.group = even(tiles_m, g);
     return o;
 }
 
@@ -686,12 +699,12 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
         attr.retry();
         return ZOQAT_ERR_CUDA;
     }
+    const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)
     {
-        const TileOrder o = choose_order(a.M, a.N, a.K, p.tiles_m, p.tiles_n, BM * CG, BN);
+        const TileOrder o = choose_order(a.M, a.N, a.K, p.tiles_m, p.tiles_n, BM * CG, BN, units);
         p.group = o.group; p.group_n = o.group_n; p.hint_a = o.hint_a; p.hint_b = o.hint_b; p.hint_out = o.hint_out;
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
-    const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)
     const int grid = (int)(total < units ? total : units) * CG;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);

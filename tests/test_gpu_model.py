@@ -117,18 +117,27 @@ def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr,
         # the oracle's self-disagreement under binary32 storage of activations, same weights
         o32 = OracleModel(dataclasses.replace(oracle.cfg, store_f32=True), oracle.p)
         g32s = [o32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
+        oa32 = OracleModel(dataclasses.replace(oracle.cfg, accum_f32=True), oracle.p)
+        ga32s = [oa32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
         want = oracle.step_multi(tokens, labels, seed0 + 8 * t, q, eps, lr) if q > 1 else [oracle.step(tokens, labels, seed0 + 8 * t, eps, lr)]
         for i, (res, (lp, lm, g)) in enumerate(zip(results, want)):
             assert res["status"] == 0 and res["n_labels"] == n_lab
             assert abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
             assert res["update_scale"] == float(lr_q * np.float32(res["proj_grad"]))
-            recs.append(dict(g=float(g), g32=float(g32s[i]), g_gpu=res["proj_grad"]))
+            recs.append(dict(g=float(g), g32=float(g32s[i]), ga32=float(ga32s[i]), g_gpu=res["proj_grad"]))
+        # updated masters against the oracle's own step: 1e-5 absolute, or - where the two g are farther apart than that
+        # allows (see gparity) - their distance times the rate times the largest |u| the generator draws (6.23); the
+        # bit-for-bit check below, with the step's own factor, is the one that pins Eq. (2)
+        dg = sum(abs(res["proj_grad"] - g) for res, (_, _, g) in zip(results, want))
+        w_tol = max(1e-5, 6.3 * float(lr_q) * dg + 1e-7)
+        if w_tol > 1e-5:
+            print(f"[updated masters] step {t}: |g_gpu - g_oracle| = {dg:.3e} moves the masters by up to {w_tol:.2e} (rate {float(lr_q):.1e})")
         for (l, n), wb in w_before.items():
             got = model.params["layers"][l][n].cpu().numpy()
             if not oracle.is_trainable(l, n):
                 assert np.array_equal(got, wb), (l, n)
                 continue
-            assert np.abs(got - oracle.p["layers"][l][n]).max() <= 1e-5, (l, n)
+            assert np.abs(got - oracle.p["layers"][l][n]).max() <= w_tol, (l, n, w_tol)
             # Eq. (2) with the step's own factors is reproduced bit for bit
             want_w = wb.copy()
             for i, res in enumerate(results):
@@ -140,7 +149,7 @@ def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr,
             for i, res in enumerate(results):
                 core.update_(want_h, seed0 + 8 * t + i, LM_HEAD_ID, np.float32(res["update_scale"]))
             assert np.array_equal(got_h.view(np.uint32), want_h.view(np.uint32))
-            assert np.abs(got_h - oracle.p["lm_head"]).max() <= 1e-5
+            assert np.abs(got_h - oracle.p["lm_head"]).max() <= w_tol
         else:
             assert np.array_equal(got_h, head_before)
     return recs
