@@ -292,7 +292,8 @@ def run_ours(args, w, rank, world, local_rank):
         metric=METRIC, value=steps_per_s, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
         ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
         data="synthetic", fwd_tokens_per_s=2 * nums["T"] * steps_per_s,
-        config=dict(workload=args.workload, l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
+        config=dict(workload=args.workload + (f" cut to {w['n_layers']} layers" if args.layers > 0 else ""),
+                    l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
                     gemm="simt" if args.simt else "tcgen05",
                     mode="batch-sharded replicas" if args.mode == "batch" else "direction-parallel replicas (q = n_gpus, value counts two-point evaluations)",
                     **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab", "w_bits", "w_group",
@@ -305,7 +306,7 @@ def run_ours(args, w, rank, world, local_rank):
                       frac=(achieved_tf / peak_tf) if achieved_tf else None,
                       peak_source=peaks["source"] + " sustained bf16 (kernel timed inside a long step)",
                       launches_per_step=gemm_n / args.steps, avg_launch_ms=gemm_ms / max(gemm_n, 1),
-                      traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)),
+                      traffic=None if args.layers > 0 else NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload)),
         kernel_ms_per_step={k: v[0] / args.steps for k, v in prof.items() if v[1] > 0},
         gpu_launches=launches, clocks=clocks,
         last_step=dict(loss_plus=res["loss_plus"], loss_minus=res["loss_minus"], proj_grad=res["proj_grad"], status=res["status"]),
@@ -351,6 +352,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="time every kernel category, not only the GEMM launches (adds ~1 %% to the step)")
     ap.add_argument("--mode", default="batch", choices=["batch", "directions"])
+    ap.add_argument("--layers", type=int, default=0, help="cut the workload to its first N layers (small profiler captures; the line's config says so)")
     ap.add_argument("--rank-probe", action="store_true", help="print this process' rank / world size as JSON and exit before any device is touched")
     args = ap.parse_args()
     if "WORLD_SIZE" not in os.environ and args.gpus > 1 and (args.impl == "ours" or args.rank_probe):
@@ -363,6 +365,9 @@ def main():
         return
     from paper_2509_00031_b200 import synth
     w = dict(synth.WORKLOADS[args.workload])
+    if args.layers > 0:
+        w["n_layers"] = min(args.layers, w["n_layers"])
+        w["first_trainable_layer"] = min(w.get("first_trainable_layer", 0), w["n_layers"])
     if args.impl == "reference":
         run_reference(args, w, rank, world)
         return

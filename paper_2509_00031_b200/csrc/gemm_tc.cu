@@ -21,7 +21,6 @@
 #include "../../include/zoqat.h"
 #include "tc_ptx.cuh"
 #include <cuda_fp16.h>
-#include <cstdlib>
 
 namespace zq {
 namespace {
@@ -601,21 +600,15 @@ int num_sms() {
 // depends on which operand block stays in L2 while the other streams past it.  With blocks of g row tiles resident,
 // B is streamed once per block: bytes = A + B * ceil(tiles_m / g); with blocks of column tiles, the mirror image.
 // The cheaper of the two is taken, with the block sized to `resident` bytes of L2 (measured: a 32 MB block survives
-// between waves, a 64 MB one does not), blocks evened out, the block's operand loaded evict_last and everything that
+// between waves, 42 MB and 64 MB ones do not), blocks evened out, the block's operand loaded evict_last and everything that
 // streams (the other operand, the results) evict_first.  When the block plus the window of the streamed operand that
 // one wave of CTAs walks does not fit either (long K: every strip is K * 512 bytes), nothing survives between waves
 // and evict_first would drop strips other CTAs of the wave still need: the wave is then made as square as possible
 // (fewest distinct strips per wave) and the operands keep the default priority.
 struct TileOrder { int group, group_n, hint_a, hint_b, hint_out; };
 
-long env_long(const char* name, long dflt) {
-    const char* v = getenv(name);
-    return v ? atol(v) : dflt;
-}
-
 TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows, int units) {
-    const double resident = (double)env_long("ZOQAT_GEMM_RESIDENT_MB", 48) * 1048576.0;
-    const long hints = env_long("ZOQAT_GEMM_HINTS", 3), force = env_long("ZOQAT_GEMM_ORDER", -1);
+    const double resident = 36.0 * 1048576.0;
     const double a_bytes = (double)M * K * 2, b_bytes = (double)N * K * 2;
     const double strip_a = (double)tm_rows * K * 2, strip_b = (double)tn_rows * K * 2;
     auto even = [](int tiles, int g) {
@@ -630,14 +623,13 @@ TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n
     const double foot_m = gm * strip_a + ((double)units / gm + 1.0) * strip_b, foot_n = gn * strip_b + ((double)units / gn + 1.0) * strip_a;
     TileOrder o;
     o.hint_a = o.hint_b = kL2Normal;
-    o.hint_out = (hints & 2) ? kL2EvictFirst : kL2Normal;
-    if (force == 0) { o.group_n = 0; o.group = tiles_m; return o; }          // every row tile of a pass, column by column
+    o.hint_out = kL2EvictFirst;
     const bool by_n = cost_n < cost_m;
     const double foot = by_n ? foot_n : foot_m;
-    if (foot <= 1.5 * resident || force == 1) {
+    if (foot <= 2.0 * resident) {
         o.group_n = by_n ? 1 : 0;
         o.group = by_n ? gn : gm;
-        if ((hints & 1) && a_bytes + b_bytes > resident) {
+        if (a_bytes + b_bytes > resident) {
             o.hint_a = by_n ? kL2EvictFirst : kL2EvictLast;
             o.hint_b = by_n ? kL2EvictLast : kL2EvictFirst;
         }

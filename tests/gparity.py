@@ -35,7 +35,9 @@ def check_g(recs, label):
           f"rms |g_gpu-g_oracle(store_f32)| {err32_rms:.2e} "
           f"({err32_rms / g_rms:.2%}); steps within 2e-3: {within_target}/{len(recs)} "
           f"(the oracle against its own store_f32 run: {band_within}/{len(recs)})")
-    assert err_rms <= max(3.0 * band_rms, 1e-2 * g_rms) + 2e-3 * g_rms, (label, err_rms, band_rms, g_rms)
-    assert np.all(err <= 0.05 * g_rms + 2e-3 * np.abs(g)), (label, float(err.max()), g_rms)
+    rms_bound = max(3.0 * band_rms, 1e-2 * g_rms) + 2e-3 * g_rms
+    assert err_rms <= rms_bound, (label, err_rms, band_rms, g_rms)
+    # single steps: heavy-tailed, so three times the rms bound (at least 5 % of rms g)
+    assert np.all(err <= max(3.0 * rms_bound, 0.05 * g_rms) + 2e-3 * np.abs(g)), (label, float(err.max()), g_rms, band_rms)
     if len(recs) >= 8:
         assert np.corrcoef(g, gg)[0, 1] > 0.995, label
