@@ -324,10 +324,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 __syncwarp();
                                 if (lane == 0) {
                                     const int bh = bseq * p.n_heads + head0 + hh;
-                                    tma_store_3d(mh, stage, part * 32, pos0, bh);
-                                    tma_store_3d(ml, stage + 2048, part * 32, pos0, bh);
-                                    tma_store_3d(mh, stage + 4096, hd + part * 32, pos0, bh);
-                                    tma_store_3d(ml, stage + 6144, hd + part * 32, pos0, bh);
+                                    tma_store_3d_hint(mh, stage, part * 32, pos0, bh, pol_out);
+                                    tma_store_3d_hint(ml, stage + 2048, part * 32, pos0, bh, pol_out);
+                                    tma_store_3d_hint(mh, stage + 4096, hd + part * 32, pos0, bh, pol_out);
+                                    tma_store_3d_hint(ml, stage + 6144, hd + part * 32, pos0, bh, pol_out);
                                     bulk_commit();
                                 }
                             }
@@ -359,8 +359,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             if (lane == 0) {
                                 const int hh = (c * 32) / dh, d0 = (c * 32) % dh;
                                 const int bh = bseq * p.n_heads + head0 + hh;
-                                tma_store_3d(&att.vh, box, pos0, d0, bh);
-                                tma_store_3d(&att.vl, box + 2048, pos0, d0, bh);
+                                tma_store_3d_hint(&att.vh, box, pos0, d0, bh, pol_out);
+                                tma_store_3d_hint(&att.vl, box + 2048, pos0, d0, bh, pol_out);
                                 bulk_commit();
                             }
                         }

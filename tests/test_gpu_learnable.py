@@ -286,7 +286,7 @@ def test_step_rates_match_oracle(zq, impl, shape, first):
     model, oracle = build_pair(zq, shape, batch, seq, impl, True, True, first=first)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=13)
     keys = learnable_keys(oracle)
-    g_o, g_32, g_g = [], [], []
+    g_o, g_32, g_a32, g_g = [], [], [], []
     for t in range(10):
         seed = 2000 + t
         for l, k in keys:          # state sync: the GPU starts every compared step from the oracle's parameters
@@ -294,6 +294,8 @@ def test_step_rates_match_oracle(zq, impl, shape, first):
         model.params["lm_head"].copy_(torch.from_numpy(oracle.p["lm_head"]))
         o32 = OracleModel(oracle_cfg(shape, adaptive_quant=True, smoothing=True, first_trainable_layer=first, store_f32=True), oracle.p)
         g_32.append(float(o32.projected_gradient(tokens, labels, seed, eps)[2]))
+        oa32 = OracleModel(oracle_cfg(shape, adaptive_quant=True, smoothing=True, first_trainable_layer=first, accum_f32=True), oracle.p)
+        g_a32.append(float(oa32.projected_gradient(tokens, labels, seed, eps)[2]))
         before = {(l, k): oracle.p["layers"][l][k].copy() for l, k in keys}
         res = zq.decode_step_result(model.zoqat_step_rates(dev(tokens), dev(labels), seed, eps, lr, lrq, lrs))
         model.zoqat_check()
@@ -317,7 +319,7 @@ def test_step_rates_match_oracle(zq, impl, shape, first):
             moved += 1
         assert moved == len(ids) - 1                             # every trainable tensor but the head, checked above
         g_o.append(float(g)); g_g.append(res["proj_grad"])
-    check_g([dict(g=a, g32=b, g_gpu=c) for a, b, c in zip(g_o, g_32, g_g)], f"Section 4.2 {shape['arch']} W{shape['w_bits']}A{shape['a_bits']} impl={impl}")
+    check_g([dict(g=a, g32=b, ga32=d, g_gpu=c) for a, b, c, d in zip(g_o, g_32, g_g, g_a32)], f"Section 4.2 {shape['arch']} W{shape['w_bits']}A{shape['a_bits']} impl={impl}")
 
 
 def test_step_with_one_rate_and_apply_update_rates(zq):

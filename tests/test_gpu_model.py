@@ -97,10 +97,12 @@ def default_step(zq, model, td, ld, seed, eps, lr):
     return [zq.decode_step_result(model.zoqat_step(td, ld, seed, eps, lr))]
 
 
-def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr, step_fn=default_step, seed0=1000):
+def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr, step_fn=default_step, seed0=1000,
+                     store_band=True):
     """n state-synced steps; returns per-step records and checks everything except g.  step_fn runs the GPU step and
     returns the result records of the directions it evaluated (one for zoqat_step); direction i uses seed + i and
-    the factor lr / len(records)."""
+    the factor lr / len(records).  store_band = False skips the oracle's store_f32 run (the accum_f32 run, which
+    also stores in binary32, is always made): the large cases keep the suite's run time down that way."""
     from oracle import core
     from oracle.model import tensor_id, LM_HEAD_ID
     recs = []
@@ -115,10 +117,12 @@ def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr,
         q = len(results)
         lr_q = np.float32(lr) if q == 1 else np.float32(np.float32(lr) / np.float32(q))
         # the oracle's self-disagreement under binary32 storage of activations, same weights
-        o32 = OracleModel(dataclasses.replace(oracle.cfg, store_f32=True), oracle.p)
-        g32s = [o32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
         oa32 = OracleModel(dataclasses.replace(oracle.cfg, accum_f32=True), oracle.p)
         ga32s = [oa32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
+        g32s = ga32s
+        if store_band:
+            o32 = OracleModel(dataclasses.replace(oracle.cfg, store_f32=True), oracle.p)
+            g32s = [o32.projected_gradient(tokens, labels, seed0 + 8 * t + i, eps)[2] for i in range(q)]
         want = oracle.step_multi(tokens, labels, seed0 + 8 * t, q, eps, lr) if q > 1 else [oracle.step(tokens, labels, seed0 + 8 * t, eps, lr)]
         for i, (res, (lp, lm, g)) in enumerate(zip(results, want)):
             assert res["status"] == 0 and res["n_labels"] == n_lab
@@ -303,8 +307,8 @@ WORKLOAD_CUTS = [
 def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packed):
     """Every workload with its real d_model / heads / d_ffn / vocabulary / quantiser, cut to one layer (two for the
     lightweight one: a frozen packed layer under a trainable one) and a short sequence so that the oracle finishes:
-    four state-synced steps against the oracle - both losses, every updated tensor bit for bit given the step's own
-    factor and within 1e-5 of the oracle's, g under the band rule."""
+    three state-synced steps against the oracle - both losses, every updated tensor bit for bit given the step's own
+    factor, g under the band rule."""
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq,
@@ -312,7 +316,7 @@ def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packe
     if packed:
         model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 4, 1e-3, 1e-6)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3, 1e-3, 1e-6, store_band=False)
     check_g(recs, f"workload dims {shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} "
                   f"W{shape['w_bits']}A{shape['a_bits']} g{shape['w_group']} T={batch * seq}")
     if first_trainable:
@@ -324,14 +328,14 @@ def test_full_token_count_layer_step(zq):
     W4A8 g128, batch 4 x seq 1024 - 16 row tiles and 8 attention query tiles per sequence in every GEMM, both passes
     side by side on 8192 rows, the schedule the benchmark times.  Full zoqat_step against the oracle: both losses,
     every updated tensor (bit for bit given the step's own factor, 1e-5 against the oracle's own step), g under the
-    band rule over three seeds, and the per-position losses of both passes of one more step."""
+    band rule over two seeds, and the per-position losses of both passes of one more step."""
     shape = _cut("llama7b_w4a8", 1)
     batch, seq = shape["batch"], shape["seq"]
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=1234)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3, 1e-3, 1e-6)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 2, 1e-3, 1e-6, store_band=False)
     check_g(recs, "llama7b_w4a8, one layer, full 4 x 1024 tokens")
     # per-position losses of both passes of one more (unsynced) step: rows [0, T) are the + pass, [T, 2T) the - pass
     T = batch * seq
