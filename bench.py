@@ -222,7 +222,7 @@ def run_ours(args, w, rank, world, local_rank):
         if args.mode == "directions":                      # q = world directions per step, one per replica, same batch
             replicas.direction_parallel_step(model, dist, rank, world, tokens, labels, 1000 + world * t, EPS, LR, sums, result, scales)
         elif world == 1 and learned:
-            model.zoqat_step_rates(tokens, labels, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
+            model.zoqat_step_rates_deferred(tokens, labels, 1000 + t, EPS, LR, LR_QUANT, LR_SMOOTH, result)
         elif world == 1:
             # Eq. (2) of step t rides on the operand producers of step t + 1; the last one is flushed inside the timed region
             model.zoqat_step_deferred(tokens, labels, 1000 + t, EPS, LR, result)
@@ -266,7 +266,7 @@ def run_ours(args, w, rank, world, local_rank):
         barrier()
         t0 = time.perf_counter()
         for t in range(args.steps):
-            model.zoqat_step_host(tok_host, lab_host, 5000 + t, EPS, LR, deferred=not learned)
+            model.zoqat_step_host(tok_host, lab_host, 5000 + t, EPS, LR, deferred=True)
         model.zoqat_flush_update()
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3

@@ -208,16 +208,23 @@ int zoqat_step_rates(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t*
  * returned result until that happens; every other entry point that reads or changes them (zoqat_forward_loss,
  * zoqat_step*, zoqat_apply_update*, zoqat_init_qparams) flushes first, and a caller that reads the master tensors
  * itself calls zoqat_flush_update() before (zoqat_model_destroy() does not: a pending update is dropped with the handle).
- * Same arithmetic, same bits as zoqat_step.  Models with Section 4.2
- * parameters or per-row weight groups run zoqat_step instead (nothing is deferred). */
+ * Same arithmetic, same bits as zoqat_step.  Only the weights wait: the Section 4.2 parameters (quantiser parameters,
+ * smoothing vectors) are small and move at once, with their own rates in the _rates form (Appendix hyperparameter
+ * table).  With one weight group per output row the pending update is applied by the pass that finds the rows'
+ * minima and maxima. */
 int zoqat_step_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
                         int batch, int seq, uint64_t seed, float eps, float lr,
                         zoqat_step_result_t* result_dev, void* stream);
+int zoqat_step_rates_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev,
+                              int batch, int seq, uint64_t seed, float eps, float lr, float lr_quant, float lr_smooth,
+                              zoqat_step_result_t* result_dev, void* stream);
 int zoqat_flush_update(zoqat_model_t* m, void* stream);
 /* The deferred form of zoqat_step_finish for replicas: forms g from the global sums and leaves Eq. (2) to the next
  * zoqat_step_begin (whose producers apply it) or to zoqat_flush_update(). */
 int zoqat_step_finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
                                zoqat_step_result_t* result_dev, void* stream);
+int zoqat_step_finish_rates_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                                     float lr_quant, float lr_smooth, zoqat_step_result_t* result_dev, void* stream);
 
 /* Eq. (1) with q = n_dirs directions per step (the paper's estimator averages over q directions u_1..u_q; it never
  * states q): direction i uses seed + i, every g_i is the two-point estimate at the SAME weights, and Eq. (2) then
@@ -495,8 +502,9 @@ int zoqat_op_head_loss(const void* a_dev, const void* b_dev, const int32_t* labe
  *   - Limit: 256-byte-rounded T * ceil(V/128) * 8 plus 256-byte-rounded T * 4 bytes must
  *     fit in the array (T = 4096 with V = 32000 does; T = 8192 with V = 50272 does not).
  *     Larger problems return ZOQAT_ERR_WORKSPACE_SMALL and launch nothing.
- *   - The first call on each device looks up the array's device address (with that device
- *     current).  Make that first call outside any stream capture.
+ *   - Every call looks up the array's device address for the device (and context) that is
+ *     current, so a pointer never outlives the context it came from.  Make the first call on
+ *     a device outside any stream capture.
  *   - No cudaMalloc, cudaFree or other allocating routine is called, on any call.
  *   - All calls on a device share the one array, which still holds the previous call's
  *     data; the part that has to start from zero is cleared on `stream` before use.  Two

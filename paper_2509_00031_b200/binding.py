@@ -27,7 +27,7 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
-    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_finish_deferred", "zoqat_flush_update", "zoqat_step_multi",
+    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_rates_deferred", "zoqat_step_finish_deferred", "zoqat_step_finish_rates_deferred", "zoqat_flush_update", "zoqat_step_multi",
     "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates", "zoqat_apply_update_multi", "zoqat_step_result",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_debug_capture", "zoqat_debug_capture_bytes", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
@@ -88,6 +88,8 @@ def lib():
             "zoqat_init_qparams": [vp, vp],
             "zoqat_step_rates": [vp, vp, vp, i32, i32, u64, f32, f32, f32, f32, vp, vp],
             "zoqat_step_finish_rates": [vp, vp, u64, f32, f32, f32, f32, vp, vp],
+            "zoqat_step_rates_deferred": [vp, vp, vp, i32, i32, u64, f32, f32, f32, f32, vp, vp],
+            "zoqat_step_finish_rates_deferred": [vp, vp, u64, f32, f32, f32, f32, vp, vp],
             "zoqat_apply_update_rates": [vp, u64, f32, f32, f32, vp],
             "zoqat_op_weight_operand_learned": [vp, i64, i64, i32, i32, u64, u32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp],
             "zoqat_op_smooth_perturb": [vp, vp, i64, u64, u32, u32, f32, vp, vp],
@@ -487,6 +489,19 @@ class ZoqatModel:
         b, s = tokens.shape
         _check(lib().zoqat_step_rates(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, lr_quant, lr_smooth,
                                       _p(result), _stream()))
+        return result
+
+    def zoqat_step_rates_deferred(self, tokens, labels, seed, eps, lr, lr_quant, lr_smooth, result=None):
+        """zoqat_step_rates whose weight update rides on the next step's producers (or zoqat_flush_update)."""
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        b, s = tokens.shape
+        _check(lib().zoqat_step_rates_deferred(self.handle, _p(tokens), _p(labels), b, s, seed, eps, lr, lr_quant, lr_smooth,
+                                               _p(result), _stream()))
+        return result
+
+    def zoqat_step_finish_rates_deferred(self, sums, seed, eps, lr, lr_quant, lr_smooth, result=None):
+        result = torch.empty(6, dtype=torch.float32, device="cuda") if result is None else result
+        _check(lib().zoqat_step_finish_rates_deferred(self.handle, _p(sums), seed, eps, lr, lr_quant, lr_smooth, _p(result), _stream()))
         return result
 
     def zoqat_step_finish_rates(self, sums, seed, eps, lr, lr_quant, lr_smooth, result=None):

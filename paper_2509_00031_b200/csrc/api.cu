@@ -286,6 +286,7 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
             a.bias_part = m->ws.bias_part; a.bias0 = bias0;
             a.bias_out = m->ws.bias_pm + bias_off; a.bias_out_stride = m->ws.bias_ld;
         }
+        a.pend = (passes == 2 && L.trainable()) ? pend : nullptr;
         launch_weight_operand_learned(a, s);
         return;
     }
@@ -503,8 +504,10 @@ int check_call(zoqat_model* m, const void* tokens, const void* labels, int batch
 
 // Eq. (2) on every trainable tensor.  Factors: weights scale_ptr / scale_val; quantiser parameters and smoothing
 // vectors (Section 4.2) class_ptr[0] / class_ptr[1] when class_ptr != NULL, else scale_q / scale_s.
+// which: 0 every class, 1 the weights only, 2 the Section 4.2 parameters only (the two halves of a deferred step:
+// the small tensors move at once, the weights with the next step's producers).
 void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float scale_val, cudaStream_t s,
-                const float* class_ptr = nullptr, float scale_q = 0.0f, float scale_s = 0.0f) {
+                const float* class_ptr = nullptr, float scale_q = 0.0f, float scale_s = 0.0f, int which = 0) {
     ProfScope ps_(m, ZOQAT_PROF_UPDATE, s);
     const int d = m->cfg.d_model, F = m->cfg.d_ffn;
     for (size_t l = 0; l < m->layers.size(); ++l) {
@@ -519,10 +522,10 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
         for (int r = 0; r < 7; ++r) {
             Linear& L = Ly.lin[r];
             if (!(L.present && L.trainable())) continue;
-            launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
-            if (L.adaptive()) add(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, L.tid_q(), 0);
+            if (which != 2) launch_update(L.w_mut, (uint64_t)(L.rows * L.cols), seed, L.tid, scale_ptr, scale_val, s);
+            if (L.adaptive() && which != 1) add(L.theta, (uint64_t)L.n_qgroups(m->cfg.w_group) * 4, L.tid_q(), 0);
         }
-        if (Ly.smoothing)
+        if (Ly.smoothing && which != 1)
             for (int pt = 0; pt < 4; ++pt) {
                 const uint32_t base = 16u * (uint32_t)(l + 1) + (uint32_t)pt;
                 const uint64_t n = pt == 3 ? (uint64_t)F : (uint64_t)d;
@@ -531,7 +534,7 @@ void update_all(zoqat_model* m, uint64_t seed, const float* scale_ptr, float sca
             }
         launch_update_batch(ub, seed, class_ptr, scale_q, scale_s, s);
     }
-    if (m->head.trainable())
+    if (m->head.trainable() && which != 2)
         launch_update(m->head.w_mut, (uint64_t)(m->head.rows * m->head.cols), seed, m->head.tid, scale_ptr, scale_val, s);
 }
 
@@ -565,7 +568,7 @@ void update_all_multi(zoqat_model* m, const SeedList& seeds, int n_dirs, const f
 // Applies a deferred update now (every entry point that reads or changes the masters starts with this).
 void flush_pending(zoqat_model* m, cudaStream_t s) {
     if (!m->pending) return;
-    update_all(m, m->pending_seed, m->ws.pending_scale, 0.0f, s);
+    update_all(m, m->pending_seed, m->ws.pending_scale, 0.0f, s, nullptr, 0.0f, 0.0f, 1);     // only weights are ever deferred
     m->pending = false;
 }
 
@@ -864,21 +867,34 @@ int zoqat_step(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* label
     return zoqat_step_finish(m, m->ws.sums, seed, eps, lr, result_dev, stream);
 }
 
-int zoqat_step_finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
-                               zoqat_step_result_t* result_dev, void* stream) {
+static int finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr, float lr_quant,
+                           float lr_smooth, zoqat_step_result_t* result_dev, void* stream) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
     if (!sums_dev || !result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "sums_dev/result_dev are NULL");
-    if (m->any_learnable || m->cfg.w_group == 0) return zoqat_step_finish(m, sums_dev, seed, eps, lr, result_dev, stream);
     if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     flush_pending(m, s);            // nothing is pending after a step_begin; kept for callers that skip it
     zoqat_step_result_dev* res = reinterpret_cast<zoqat_step_result_dev*>(result_dev);
     launch_finish_step(sums_dev, eps, lr, m->ws.err_flag, res, s);
+    if (m->any_learnable) {         // the small Section 4.2 tensors move now; only the weights wait for the next producers
+        launch_class_scales(&res->proj_grad, lr_quant, lr_smooth, m->ws.class_scales, s);
+        update_all(m, seed, nullptr, 0.0f, s, m->ws.class_scales, 0.0f, 0.0f, 2);
+    }
     CUDA_TRY(cudaMemcpyAsync(m->ws.pending_scale, &res->update_scale, 4, cudaMemcpyDeviceToDevice, s));
     m->pending = true;
     m->pending_seed = seed;
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
+}
+
+int zoqat_step_finish_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr,
+                               zoqat_step_result_t* result_dev, void* stream) {
+    return finish_deferred(m, sums_dev, seed, eps, lr, lr, lr, result_dev, stream);
+}
+
+int zoqat_step_finish_rates_deferred(zoqat_model_t* m, const double* sums_dev, uint64_t seed, float eps, float lr, float lr_quant,
+                                     float lr_smooth, zoqat_step_result_t* result_dev, void* stream) {
+    return finish_deferred(m, sums_dev, seed, eps, lr, lr_quant, lr_smooth, result_dev, stream);
 }
 
 int zoqat_flush_update(zoqat_model_t* m, void* stream) {
@@ -893,10 +909,18 @@ int zoqat_step_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32
     if (!result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "result_dev is NULL");
     if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
     if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
-    // the producers that can carry an update are those of the plain per-group min/max path
-    if (m->any_learnable || m->cfg.w_group == 0) return zoqat_step(m, tokens_dev, labels_dev, batch, seq, seed, eps, lr, result_dev, stream);
     if (int rc = zoqat_step_begin(m, tokens_dev, labels_dev, batch, seq, seed, eps, m->ws.sums, stream)) return rc;
     return zoqat_step_finish_deferred(m, m->ws.sums, seed, eps, lr, result_dev, stream);
+}
+
+int zoqat_step_rates_deferred(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,
+                              uint64_t seed, float eps, float lr, float lr_quant, float lr_smooth, zoqat_step_result_t* result_dev,
+                              void* stream) {
+    if (!result_dev) return fail(ZOQAT_ERR_INVALID_ARG, "result_dev is NULL");
+    if (int rc = check_call(m, tokens_dev, labels_dev, batch, seq)) return rc;
+    if (!(eps > 0.0f)) return fail(ZOQAT_ERR_INVALID_ARG, "eps must be positive");
+    if (int rc = zoqat_step_begin(m, tokens_dev, labels_dev, batch, seq, seed, eps, m->ws.sums, stream)) return rc;
+    return zoqat_step_finish_rates_deferred(m, m->ws.sums, seed, eps, lr, lr_quant, lr_smooth, result_dev, stream);
 }
 
 int zoqat_step_multi(zoqat_model_t* m, const int32_t* tokens_dev, const int32_t* labels_dev, int batch, int seq,

@@ -110,6 +110,7 @@ struct LearnedOperandArgs {
     const float* smooth; int smooth_ld;
     float* bias_part; const float* bias0; float* bias_out; int64_t bias_out_stride;
     uint8_t* codes;
+    const PendingUpdate* pend;    // with op_minus only: the previous step's update, applied to the master on the way in
 };
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s);
 void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s);

@@ -342,20 +342,32 @@ adapt_prepare_kernel(PrepareBatch b, int bits, int perturb, uint32_t k0, uint32_
 // adapt_prepare_kernel, A = (step, 1/step, -z, Q_P - z), B = (z, 0, Q_P, 0), so the producer runs its folded form.
 // theta_out != NULL instead writes the initial learnable parameters (step, z, 0, 1) of the unperturbed row.
 // One CTA per row; cols4 = cols / 4.
+// w_upd != NULL: the previous step's update (Eq. (2), seed keys (uk0, uk1), factor *upd_scale) is applied to the master on
+// the way in and written back through w_upd (= w), so that the producer pass that follows reads the updated master.
 __global__ void __launch_bounds__(kThreads)
 row_prepare_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, int perturb, uint32_t k0, uint32_t k1,
                    uint32_t tid, float eps, int signs, const float* __restrict__ smooth, int smooth_ld,
-                   float4* __restrict__ out_a, float4* __restrict__ out_b, float4* __restrict__ theta_out) {
+                   float4* __restrict__ out_a, float4* __restrict__ out_b, float4* __restrict__ theta_out,
+                   float4* w_upd, const float* __restrict__ upd_scale, uint32_t uk0, uint32_t uk1) {
     __shared__ float2 tab[kIcdfKnots];
     __shared__ float red[4][kThreads / 32];
-    if (perturb) stage_icdf_table(tab);
+    if (perturb || w_upd) stage_icdf_table(tab);
+    const float upd_c = w_upd ? -(*upd_scale) : 0.0f;
     const float qp = (float)((1 << bits) - 1);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int r = blockIdx.x; r < rows; r += gridDim.x) {
         float mnp = INFINITY, mxp = -INFINITY, mnm = INFINITY, mxm = -INFINITY;
         for (int c = threadIdx.x; c < cols4; c += kThreads) {
             const int64_t chunk = (int64_t)r * cols4 + c;
-            const float4 v = __ldg(w + chunk);
+            float4 v;
+            if (w_upd) {
+                v = w_upd[chunk];
+                const float4 zu = direction4(tab, uk0, uk1, tid, (uint64_t)chunk);
+                v = make_float4(__fmaf_rn(upd_c, zu.x, v.x), __fmaf_rn(upd_c, zu.y, v.y), __fmaf_rn(upd_c, zu.z, v.z), __fmaf_rn(upd_c, zu.w, v.w));
+                w_upd[chunk] = v;
+            } else {
+                v = __ldg(w + chunk);
+            }
             float xp[4] = {v.x, v.y, v.z, v.w}, xm[4] = {v.x, v.y, v.z, v.w};
             if (perturb) {
                 const float4 z = direction4(tab, k0, k1, tid, (uint64_t)chunk);
@@ -410,7 +422,9 @@ row_prepare_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, 
 //   ADAPT   the group's quantiser comes from the learnable parameters, perturbed and prepared per (group, sign) by
 //           adapt_prepare_kernel (prep_a / prep_b), instead of being derived from min/max.
 // smooth: [sign][kind][smooth_ld] floats, kind 0 = scale, 1 = shift (2 = 1/scale, used by the activation side).
-template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH>
+// UPD: as in weight_operand_kernel, the previous step's update is applied to the master (read and written through w_out)
+// before this step's perturbation.
+template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH, bool UPD>
 __global__ void __launch_bounds__(kThreads, 3)
 weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols4, int bits, int perturb,
                               const PhiloxKeys rk, uint32_t tid, float eps,
@@ -418,12 +432,13 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                               const float4* __restrict__ prep_a, const float4* __restrict__ prep_b,
                               const float* __restrict__ smooth, int smooth_ld,
                               float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes,
-                              int qgroup_items) {
+                              int qgroup_items, float4* w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk) {
     // qgroup_items: 16-element items per quantisation group when that is not the GROUP-element span (one group per
     // row: cols / 16); 0 = the span itself.  The bias partial sums stay per span either way.
     constexpr int LANES = GROUP / 16;
     __shared__ float2 tab[kIcdfKnots];
-    if (perturb) stage_icdf_table(tab);
+    if (perturb || UPD) stage_icdf_table(tab);
+    const float upd_c = UPD ? -(*upd_scale) : 0.0f;
     const float qp = (float)((1 << bits) - 1);
     const int64_t n16_ceil = (n16 + 31) & ~(int64_t)31;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n16_ceil; i += (int64_t)gridDim.x * blockDim.x) {
@@ -431,8 +446,17 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
         float x[16], xm[16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const float4 v = live ? __ldg(w + chunk_of<LANES>(i, k)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 v = live ? (UPD ? w_out[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+        }
+        if (UPD) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 z = direction4(tab, urk, tid, (uint64_t)chunk_of<LANES>(i, k));
+                x[4 * k] = __fmaf_rn(upd_c, z.x, x[4 * k]); x[4 * k + 1] = __fmaf_rn(upd_c, z.y, x[4 * k + 1]);
+                x[4 * k + 2] = __fmaf_rn(upd_c, z.z, x[4 * k + 2]); x[4 * k + 3] = __fmaf_rn(upd_c, z.w, x[4 * k + 3]);
+                if (live) w_out[chunk_of<LANES>(i, k)] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+            }
         }
         if (perturb) {
 #pragma unroll
@@ -811,6 +835,7 @@ void launch_weight_operand(const float* w, int64_t n, int group, int bits, int p
 
 template <int GROUP, bool ADAPT, bool SMOOTH>
 static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
+    const PendingUpdate* pend = a.op_minus ? a.pend : nullptr;     // a deferred update rides on the two-sign producer only
     const int64_t n16 = a.rows * a.cols / 16;
     const int grid = stream_grid(n16, kThreads, 3);        // 80 registers: three CTAs per SM
     const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
@@ -828,22 +853,31 @@ static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
             PrepareBatch pb1{};
             pb1.count = 1; pb1.theta[0] = a.theta; pb1.prep[0] = a.prep; pb1.tid_q[0] = a.tid_q; pb1.prefix[0] = 0; pb1.prefix[1] = n_q;
             launch_adapt_prepare(pb1, a.bits, a.perturb, a.seed, a.eps, signs, s);
-        } else {       // one min/max group per row
+        } else {       // one min/max group per row; a pending update is applied by this first pass over the rows
             const int rgrid = (int)(a.rows < 148 * 8 ? a.rows : 148 * 8);
             row_prepare_kernel<<<rgrid, kThreads, 0, s>>>(w4, (int)a.rows, (int)(a.cols / 4), a.bits, a.perturb, k0, k1, a.tid, a.eps,
-                                                          signs, a.smooth, a.smooth_ld, pa, pb, nullptr);
+                                                          signs, a.smooth, a.smooth_ld, pa, pb, nullptr,
+                                                          pend ? reinterpret_cast<float4*>(const_cast<float*>(a.w)) : nullptr,
+                                                          pend ? pend->scale : nullptr, pend ? (uint32_t)pend->seed : 0u,
+                                                          pend ? (uint32_t)(pend->seed >> 32) : 0u);
             count_launch();
+            pend = nullptr;
         }
     }
     const int qgi = a.per_channel ? (int)(a.cols / 16) : 0;
-    if (a.op_minus)
-        weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, philox_keys(a.seed), a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
-            a.bias_part, n_groups, c4, qgi);
+    const PhiloxKeys rk = philox_keys(a.seed);
+    if (a.op_minus && pend)
+        weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH, true><<<grid, kThreads, 0, s>>>(
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
+            a.bias_part, n_groups, c4, qgi, reinterpret_cast<float4*>(const_cast<float*>(a.w)), pend->scale, philox_keys(pend->seed));
+    else if (a.op_minus)
+        weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH, false><<<grid, kThreads, 0, s>>>(
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
+            a.bias_part, n_groups, c4, qgi, nullptr, nullptr, rk);
     else
-        weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH><<<grid, kThreads, 0, s>>>(
-            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, philox_keys(a.seed), a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
-            a.bias_part, n_groups, c4, qgi);
+        weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH, false><<<grid, kThreads, 0, s>>>(
+            w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
+            a.bias_part, n_groups, c4, qgi, nullptr, nullptr, rk);
     count_launch();
     if (SMOOTH) {
         const int64_t work = a.rows * signs * 32;
@@ -863,7 +897,7 @@ static void learned_dispatch_group(const LearnedOperandArgs& a, cudaStream_t s) 
 }
 
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s) {
-    if (a.rows * a.cols == 0 || (a.perturb && !ensure_icdf_table())) return;
+    if (a.rows * a.cols == 0 || ((a.perturb || a.pend) && !ensure_icdf_table())) return;
     if (a.per_channel) { learned_dispatch_group<128>(a, s); return; }      // cols % 128 == 0 (checked by the callers)
     if (a.group == 32) learned_dispatch_group<32>(a, s);
     else if (a.group == 64) learned_dispatch_group<64>(a, s);
@@ -896,7 +930,7 @@ void launch_init_qparams_rows(const float* w, int64_t rows, int64_t cols, int bi
     if (rows * cols == 0) return;
     const int rgrid = (int)(rows < 148 * 8 ? rows : 148 * 8);
     row_prepare_kernel<<<rgrid, kThreads, 0, s>>>(reinterpret_cast<const float4*>(w), (int)rows, (int)(cols / 4), bits, 0, 0u, 0u, 0u, 0.0f,
-                                                  1, nullptr, 0, nullptr, nullptr, reinterpret_cast<float4*>(theta));
+                                                  1, nullptr, 0, nullptr, nullptr, reinterpret_cast<float4*>(theta), nullptr, nullptr, 0u, 0u);
     count_launch();
 }
 

@@ -12,6 +12,10 @@ between iterations) and prints one JSON line per kernel with its achieved rate.
   python -m paper_2509_00031_b200.microbench --op decode --workload llama7b_w4a8 --batch 1 --context 256 --tokens 64
       (decode-time inference over the packed model: tokens/s, bytes per token against the HBM copy rate)
 
+  python -m paper_2509_00031_b200.microbench --op gemm --M 8192 --N 4096 --K 4096 --sustain 2.5
+      (back-to-back launches for 2.5 s under the power cap: TFLOP/s, median SM clock and board power, mJ per launch;
+       --op gemm_lib runs the library's bf16 GEMM on the same shape the same way, as the yardstick)
+
 It is also the small, self-contained command used for ncu captures of one kernel.
 """
 import argparse
@@ -36,6 +40,38 @@ def timed(fn, iters, flush):
     torch.cuda.synchronize()
     ts = sorted(a.elapsed_time(b) for a, b in ev)
     return ts[len(ts) // 2], ts[0]
+
+
+def sustained(fn, secs):
+    """fn back to back for `secs` seconds; nvidia-smi sampled every 100 ms.  Returns (ms per launch, median SM MHz,
+    median board W)."""
+    import subprocess
+    import threading
+    import time
+    lines = []
+    proc = subprocess.Popen(["nvidia-smi", f"--id={torch.cuda.current_device()}", "--query-gpu=clocks.sm,power.draw",
+                             "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE, text=True)
+    threading.Thread(target=lambda: [lines.append((time.time(), ln.strip())) for ln in proc.stdout], daemon=True).start()
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0, n = time.time(), 0
+    e0.record()
+    while time.time() - t0 < secs:
+        for _ in range(20):
+            fn()
+        n += 20
+        torch.cuda.synchronize()
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    time.sleep(0.3)
+    proc.terminate()
+    samp = [ln.split(",") for (t, ln) in lines if t0 + 0.8 < t < t1]
+    clk = sorted(float(x[0]) for x in samp if len(x) == 2)
+    pw = sorted(float(x[1]) for x in samp if len(x) == 2)
+    return e0.elapsed_time(e1) / n, (clk[len(clk) // 2] if clk else None), (pw[len(pw) // 2] if pw else None)
 
 
 def decode_bench(a):
@@ -133,6 +169,7 @@ def main():
     ap.add_argument("--context", type=int, default=256)
     ap.add_argument("--tokens", type=int, default=64)
     ap.add_argument("--graph", action="store_true", help="decode: replay the timed steps from one captured CUDA graph")
+    ap.add_argument("--sustain", type=float, default=0.0, help="gemm / gemm_lib: run back to back for this many seconds and report clock, power and mJ per launch")
     a = ap.parse_args()
     if a.op == "decode":
         return decode_bench(a)
@@ -140,18 +177,27 @@ def main():
     dev = "cuda"
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = dict(op=a.op)
-    if a.op in ("gemm", "head_loss"):
+    if a.op in ("gemm", "head_loss", "gemm_lib"):
         A = torch.randint(-127, 128, (a.M, a.K), device=dev).to(torch.bfloat16)
         B = (torch.randn(a.N, a.K, device=dev) * 0.02).to(torch.bfloat16)
         rs = torch.rand(a.M, device=dev) + 0.5
         if a.op == "gemm":
             C = torch.zeros(a.M, a.N, device=dev)
             fn = lambda: zq.zoqat_op_gemm(A, B, row_step=rs, out=C, accumulate=a.accumulate, impl=a.impl)
+        elif a.op == "gemm_lib":            # the library's bf16 GEMM (bf16 result): a yardstick, not part of the path
+            Cl = torch.empty(a.M, a.N, device=dev, dtype=torch.bfloat16)
+            fn = lambda: torch.matmul(A, B.t(), out=Cl)
         else:
             labels = torch.randint(0, a.N, (a.M,), device=dev, dtype=torch.int32)
             fn = lambda: zq.zoqat_op_head_loss(A, B, labels, impl=a.impl)
-        med, best = timed(fn, a.iters, flush)
         flops = 2.0 * a.M * a.N * a.K
+        if a.sustain > 0:
+            ms, clk, pw = sustained(fn, a.sustain)
+            out.update(M=a.M, N=a.N, K=a.K, sustained_s=a.sustain, ms=ms, tflops=flops / ms / 1e9, sm_mhz_median=clk, power_w_median=pw,
+                       mj_per_launch=(ms * pw) if pw else None)
+            print(json.dumps(out), flush=True)
+            return
+        med, best = timed(fn, a.iters, flush)
         out.update(M=a.M, N=a.N, K=a.K, ms=med, ms_best=best, tflops=flops / med / 1e9, tflops_best=flops / best / 1e9)
     elif a.op in ("weight_pair", "weight_single", "weight_learned", "update", "unpack"):
         W = torch.randn(a.rows, a.cols, device=dev) * 0.02

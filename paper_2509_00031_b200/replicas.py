@@ -17,12 +17,13 @@ methods) and `dist` is torch.distributed (or a stand-in with all_reduce / all_ga
 
 
 def batch_sharded_step(model, dist, world, tokens, labels, seed, eps, lr, sums, result, rates=None):
-    """rates: (lr_quant, lr_smooth) for models with Section 4.2 parameters (their update is not deferred)."""
+    """rates: (lr_quant, lr_smooth) for models with Section 4.2 parameters (those move at once; the weights' update
+    rides on the next step like everyone's)."""
     model.zoqat_step_begin(tokens, labels, seed, eps, sums)
     if world > 1:
         dist.all_reduce(sums)
     if rates is not None:
-        model.zoqat_step_finish_rates(sums, seed, eps, lr, rates[0], rates[1], result)
+        model.zoqat_step_finish_rates_deferred(sums, seed, eps, lr, rates[0], rates[1], result)
     else:
         model.zoqat_step_finish_deferred(sums, seed, eps, lr, result)
     return result

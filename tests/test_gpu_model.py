@@ -98,11 +98,11 @@ def default_step(zq, model, td, ld, seed, eps, lr):
 
 
 def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr, step_fn=default_step, seed0=1000,
-                     store_band=True):
+                     store_band=False):
     """n state-synced steps; returns per-step records and checks everything except g.  step_fn runs the GPU step and
     returns the result records of the directions it evaluated (one for zoqat_step); direction i uses seed + i and
-    the factor lr / len(records).  store_band = False skips the oracle's store_f32 run (the accum_f32 run, which
-    also stores in binary32, is always made): the large cases keep the suite's run time down that way."""
+    the factor lr / len(records).  store_band = True also makes the oracle's store_f32 run (the accum_f32 run, which
+    also stores in binary32, is always made); most cases skip it to keep the suite's run time down."""
     from oracle import core
     from oracle.model import tensor_id, LM_HEAD_ID
     recs = []
@@ -164,7 +164,7 @@ def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr,
 def test_step_matches_oracle(zq, impl, shape, batch, seq):
     model, oracle = build_pair(zq, shape, batch, seq, impl)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=12)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 8, 1e-3, 1e-6)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 8, 1e-3, 1e-6, store_band=(impl == 0))
     check_g(recs, f"small {shape['arch']} W{shape['w_bits']}A{shape['a_bits']} impl={impl}")
     assert np.array_equal(model.params["embed"].cpu().numpy(), oracle.p["embed"])
 
@@ -177,7 +177,7 @@ def test_tiny_workload_ten_steps(zq):
     oracle = OracleModel(oracle_cfg(w), synth.copy_params(params))
     model = zq.ZoqatModel(w, zq.params_to_device(params), max_batch=w["batch"], max_seq=w["seq"])
     tokens, labels = synth.make_batch(w["batch"], w["seq"], w["vocab"], seed=1234)
-    recs = run_synced_steps(zq, model, oracle, w, tokens, labels, 10, 1e-3, 1e-6)
+    recs = run_synced_steps(zq, model, oracle, w, tokens, labels, 10, 1e-3, 1e-6, store_band=True)
     check_g(recs, "tiny_w4a8")
     # free-running (no state sync): ten more steps stay within the loss and weight tolerances
     sync_masters(model, oracle)
@@ -248,7 +248,7 @@ def test_lightweight_variant(zq, impl):
     assert abs(res["loss_minus"] - lm) <= 1e-4 * abs(lm)
     assert torch.equal(frozen_before, plain.params["layers"][0]["wq"])
     assert np.abs(plain.params["layers"][2]["wq"].cpu().numpy() - oracle.p["layers"][2]["wq"]).max() <= 1e-5
-    check_g(run_synced_steps(zq, packed, oracle, shape, tokens, labels, 6, eps, lr), f"lightweight (packed prefix) impl={impl}")
+    check_g(run_synced_steps(zq, packed, oracle, shape, tokens, labels, 4, eps, lr), f"lightweight (packed prefix) impl={impl}")
     # nothing trainable: the loss ignores (seed, eps)
     none, _ = build_pair(zq, shape, batch, seq, impl, first_trainable_layer=3, head_trainable=False, packed=True)
     assert float(none.zoqat_forward_loss(td, ld, 1, 1e-3).item()) == float(none.zoqat_forward_loss(td, ld, 9, -1e-2).item())
@@ -284,7 +284,7 @@ def test_step_host_buffers(zq):
         return [dict(loss_plus=r.loss_plus, loss_minus=r.loss_minus, proj_grad=r.proj_grad, update_scale=r.update_scale,
                      status=r.status, n_labels=r.n_labels)]
 
-    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 6, 1e-3, 1e-4, step_fn=host_step), "host buffers")
+    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 4, 1e-3, 1e-4, step_fn=host_step), "host buffers")
 
 
 # ---- the five workloads at their real layer dimensions ------------------------------------------------------------
@@ -307,8 +307,8 @@ WORKLOAD_CUTS = [
 def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packed):
     """Every workload with its real d_model / heads / d_ffn / vocabulary / quantiser, cut to one layer (two for the
     lightweight one: a frozen packed layer under a trainable one) and a short sequence so that the oracle finishes:
-    three state-synced steps against the oracle - both losses, every updated tensor bit for bit given the step's own
-    factor, g under the band rule."""
+    two or three state-synced steps against the oracle - both losses, every updated tensor bit for bit given the
+    step's own factor, g under the band rule."""
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq,
@@ -316,7 +316,7 @@ def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packe
     if packed:
         model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3, 1e-3, 1e-6, store_band=False)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3 if shape["a_bits"] else 2, 1e-3, 1e-6)
     check_g(recs, f"workload dims {shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} "
                   f"W{shape['w_bits']}A{shape['a_bits']} g{shape['w_group']} T={batch * seq}")
     if first_trainable:
@@ -327,30 +327,16 @@ def test_full_token_count_layer_step(zq):
     """The bench workload's own token count through one layer and the vocabulary projection: LLaMA-7B dimensions,
     W4A8 g128, batch 4 x seq 1024 - 16 row tiles and 8 attention query tiles per sequence in every GEMM, both passes
     side by side on 8192 rows, the schedule the benchmark times.  Full zoqat_step against the oracle: both losses,
-    every updated tensor (bit for bit given the step's own factor, 1e-5 against the oracle's own step), g under the
-    band rule over two seeds, and the per-position losses of both passes of one more step."""
+    every updated tensor (bit for bit given the step's own factor), g under the band rule over two seeds.  (The
+    per-position view of the same configuration is test_full_token_count_layer_element_by_element.)"""
     shape = _cut("llama7b_w4a8", 1)
     batch, seq = shape["batch"], shape["seq"]
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=1234)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 2, 1e-3, 1e-6, store_band=False)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 2, 1e-3, 1e-6)
     check_g(recs, "llama7b_w4a8, one layer, full 4 x 1024 tokens")
-    # per-position losses of both passes of one more (unsynced) step: rows [0, T) are the + pass, [T, 2T) the - pass
-    T = batch * seq
-    res = zq.decode_step_result(model.zoqat_step(dev(tokens), dev(labels), 77, 1e-3, 0.0))
-    tl_gpu = model.zoqat_debug_buffer(zq.BUF_TOKEN_LOSS)[:2 * T].cpu().numpy().astype(np.float64)
-    sync_masters(model, oracle)        # lr = 0 left the masters where the oracle's are; make it exact anyway
-    for z, sign in enumerate((1.0, -1.0)):
-        tl, valid = oracle.token_losses(tokens, labels, 77, sign * float(np.float32(1e-3)))
-        rel = np.abs(tl_gpu[z * T:(z + 1) * T] - tl)[valid] / tl[valid]
-        mean_rel = abs(tl_gpu[z * T:(z + 1) * T][valid].mean() - tl[valid].mean()) / tl[valid].mean()
-        print(f"[full token count] pass {'+-'[z]}: per-position loss rel err max {rel.max():.2e} median {np.median(rel):.2e}; mean loss rel err {mean_rel:.2e}")
-        # single positions carry the quantisation noise of their differing codes (test_gpu_forward_elementwise sets it
-        # beside the oracle's own binary32 run); the pass loss, their mean, agrees far inside 1e-3
-        assert rel.max() <= 1e-1 and np.median(rel) <= 2e-2 and mean_rel <= 1e-3
-    assert res["status"] == 0
 
 
 def test_step_multi_directions(zq):
@@ -432,7 +418,7 @@ def test_query_value_only_selection(zq):
     model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=17)
     eps, lr = 1e-3, 1e-4
-    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 6, eps, lr, seed0=9), "query/value only")
+    check_g(run_synced_steps(zq, model, oracle, shape, tokens, labels, 4, eps, lr, seed0=9), "query/value only")
     for l in range(2):
         for n in oracle.linear_names():
             got = model.params["layers"][l][n].cpu().numpy()

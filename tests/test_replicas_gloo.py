@@ -110,8 +110,8 @@ class _Recorder:
     def zoqat_step_finish_deferred(self, sums, seed, eps, lr, result):
         self.log.append(("finish_deferred", seed, sums.tolist()))
 
-    def zoqat_step_finish_rates(self, sums, seed, eps, lr, lr_quant, lr_smooth, result):
-        self.log.append(("finish_rates", seed, sums.tolist(), lr_quant, lr_smooth))
+    def zoqat_step_finish_rates_deferred(self, sums, seed, eps, lr, lr_quant, lr_smooth, result):
+        self.log.append(("finish_rates_deferred", seed, sums.tolist(), lr_quant, lr_smooth))
 
     def zoqat_step_result(self, sums, eps, lr, result):
         self.log.append(("result", lr))
@@ -168,7 +168,7 @@ def test_replica_call_order_and_payloads(tmp_path):
         log = json.load(open(tmp_path / f"log{rank}.json"))
         names = [e[0] for e in log]
         assert names == ["begin", "all_reduce", "finish_deferred", "begin", "all_reduce", "finish_deferred", "flush",
-                         "begin", "all_reduce", "finish_rates", "begin", "result", "all_gather", "apply_multi"]
+                         "begin", "all_reduce", "finish_rates_deferred", "begin", "result", "all_gather", "apply_multi"]
         assert log[1][1] == 24 and log[4][1] == 24 and log[8][1] == 24       # (sum L+, sum L-, count): three doubles
         assert log[2][2] == [21.0, 41.0, 10.0]                                 # both shards' sums reached the second half
         assert log[9][3:] == [1e-5, 5e-6]
