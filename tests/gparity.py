@@ -7,7 +7,9 @@ every sum also accumulated in binary32 in the library's order (OracleConfig.accu
 rms(g).  That self-disagreement ("band": the larger of the two, in rms over the steps) is measured on the same
 inputs, step by step.  It is heavy-tailed (one differing code in one step dominates a short run) and models only part
 of what another binary32 implementation does differently (not the tensor cores' accumulation order or the binary16
-attention operands), so the rms bound never drops below 1 % of rms(g).
+attention operands); on the small test models (a few hundred tokens) a single differing code moves g by 1-4 % of
+rms(g), and whether a four-step run of the oracle's own binary32 variant catches one is luck, so the rms bound never
+drops below 2.5 % of rms(g).
 
 records: dicts with g (float64 oracle), g32 (the oracle under binary32 storage, same weights), optionally ga32 (the
 oracle with binary32 accumulation) and g_gpu, one per evaluated direction, every step state-synced (GPU masters
@@ -37,9 +39,9 @@ def check_g(recs, label):
           f"rms |g_gpu-g_oracle(store_f32)| {err32_rms:.2e} "
           f"({err32_rms / g_rms:.2%}); steps within 2e-3: {within_target}/{len(recs)} "
           f"(the oracle against its own store_f32 run: {band_within}/{len(recs)})")
-    rms_bound = max(3.0 * band_rms, 1e-2 * g_rms) + 2e-3 * g_rms
+    rms_bound = max(3.0 * band_rms, 2.5e-2 * g_rms) + 2e-3 * g_rms
     assert err_rms <= rms_bound, (label, err_rms, band_rms, g_rms)
-    # single steps: heavy-tailed, so three times the rms bound (at least 5 % of rms g)
-    assert np.all(err <= max(3.0 * rms_bound, 0.05 * g_rms) + 2e-3 * np.abs(g)), (label, float(err.max()), g_rms, band_rms)
+    # single steps: heavy-tailed, so three times the rms bound
+    assert np.all(err <= 3.0 * rms_bound + 2e-3 * np.abs(g)), (label, float(err.max()), g_rms, band_rms)
     if len(recs) >= 8:
         assert np.corrcoef(g, gg)[0, 1] > 0.995, label
