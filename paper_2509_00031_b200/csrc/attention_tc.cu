@@ -14,12 +14,15 @@
 //   attn_prep_kernel   fp32 q|k|v -> rotary embedding, q * log2(e)/sqrt(d_head), hi/lo split;
 //                      q and k as [batch][head][seq][d_head], v transposed [batch][head][d_head][seq]
 //                      so that every tensor-core operand is K-major.
-//   attention_tc_kernel  persistent, one CTA per SM, 192 threads:
+//   attention_tc_kernel  persistent, one CTA per SM, 224 threads:
 //     warp 0     TMA producer: Q tile (128 queries) once per work item, then K / V^T tiles of 64 keys
 //                (hi and lo) into a two-stage ring.
-//     warp 1     MMA issuer: S_j = Q K_j^T (N = 64) into one of two TMEM score buffers - issued one
-//                tile ahead of the softmax - and O += P_j V_j (N = d_head), accumulated in TMEM over
-//                the whole work item.
+//     warp 1     MMA issuer of the scores: S_j = Q K_j^T (N = 64) into one of two TMEM score buffers,
+//                as far ahead of the softmax as the two buffers allow.
+//     warp 6     MMA issuer of the outputs: O += P_j V_j (N = d_head), accumulated in TMEM over the whole
+//                work item.  A thread of its own: the MMAs are small (32-48 cycles each), and one thread
+//                that also waits for every P tile cannot keep the score products of the next tiles flowing
+//                (measured: 304 -> 271 us per call at d_head 128, 304 -> 210 us at d_head 64).
 //     warps 2-5  softmax, one thread per query row (kRowThreads = 2 gives each row two threads that share the
 //                columns and exchange their maxima; it measured no faster): read S_j from TMEM, base-2 exponentials relative
 //                to a reference maximum, write P_j hi/lo to shared memory in the operand layout.  The
@@ -40,7 +43,8 @@ namespace {
 
 constexpr int BQ = 128, BKV = 64;
 constexpr int kRowThreads = 1;          // softmax threads per query row (each takes 1/kRowThreads of the columns)
-constexpr int kAttThreadsTC = 64 + 128 * kRowThreads;
+constexpr int kAttThreadsTC = 96 + 128 * kRowThreads;   // producer, two MMA issuers, softmax warps
+constexpr int kPvWarp = 2 + 4 * kRowThreads;            // the warp whose lane 0 issues the P V products
 constexpr float kRefSlack = 8.0f;      // the softmax reference may lag the row maximum by up to 2^8
 constexpr float kLoScale = 2048.0f, kLoInv = 1.0f / 2048.0f;
 constexpr int kErrAttnSmem = 16;       // dynamic shared memory window too small after alignment
@@ -318,8 +322,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc_s = idesc_f16(BKV), idesc_o = idesc_f16(D);
-            uint32_t kv_it = 0, t_it = 0, q_it = 0;
+            const uint32_t idesc_s = idesc_f16(BKV);
+            uint32_t kv_it = 0, q_it = 0;
             bool ok = true;
             // S of global tile g (stage / score buffer g & 1)
             auto issue_s = [&](uint32_t g) -> bool {
@@ -350,18 +354,31 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
                 umma_commit(k_empty(st));          // the K tile is free once these products have completed
                 return true;
             };
+            // the score products of every tile of every item, as far ahead as the two score buffers allow
             for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
                 const int n = n_kv_tiles(item_qt(it));
                 if (!mbar_wait(q_full, q_it & 1u)) { ok = false; break; }
-                if (!issue_s(kv_it)) { ok = false; break; }
-                if (n == 1) umma_commit(q_empty);
+                for (int j = 0; j < n; ++j) {
+                    if (!issue_s(kv_it + j)) { ok = false; break; }
+                }
+                if (!ok) break;
+                umma_commit(q_empty);                 // Q is free once the last S of the item has completed
+                kv_it += n;
+            }
+            if (!ok) atomicExch(p.err_flag, kErrAttnWait);
+        }
+    } else if (warp == kPvWarp) {
+        // ---------------- second MMA issuer: O += P_j V_j.  Its own thread, so that waiting for a P tile never holds
+        // back the score products of the tiles ahead (small MMAs: one issuing thread could not keep the pipe fed)
+        if (lane == 0) {
+            const uint32_t idesc_o = idesc_f16(D);
+            uint32_t kv_it = 0, t_it = 0, q_it = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < p.total_items && ok; it += gridDim.x, ++q_it) {
+                const int n = n_kv_tiles(item_qt(it));
                 // the O accumulators are free once the softmax warps have read out the previous item
                 if (!mbar_wait(o_empty, (q_it & 1u) ^ 1u)) { ok = false; break; }
                 for (int j = 0; j < n; ++j, ++t_it) {
-                    if (j + 1 < n) {
-                        if (!issue_s(kv_it + j + 1)) { ok = false; break; }
-                        if (j + 2 == n) umma_commit(q_empty);     // Q is free once the last S of the item has completed
-                    }
                     const int st = (kv_it + j) & 1u;
                     if (!mbar_wait(p_full, t_it & 1u) ||                         // P_j stored (and O rescaled if needed)
                         !mbar_wait(v_full(st), ((kv_it + j) >> 1) & 1u)) { ok = false; break; }
@@ -392,7 +409,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_qh, const __grid_con
             }
             if (!ok) atomicExch(p.err_flag, kErrAttnWait);
         }
-    } else {
+    } else if (warp >= 2 && warp < kPvWarp) {
         // ---------------- softmax / output warps: kRowThreads threads per query row, each on its share of the columns
         constexpr int CW = BKV / kRowThreads;               // score columns per thread
         constexpr int DW = D / kRowThreads;                 // output columns per thread
