@@ -30,9 +30,10 @@ UNIT = "steps/s"
 EPS, LR = 1e-3, 1e-6
 LR_QUANT, LR_SMOOTH = 1e-5, 5e-6      # rates of the Section 4.2 parameter classes (the paper's hyperparameter table)
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant (GEMM) kernel, averaged over the 129 GEMM
-# launches of one step, from the committed ncu capture (profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by
-# workload; absent for workloads that have not been captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 842.7e6}
+# launches of one step: captured with ncu on a two-layer cut of the workload and scaled by the layer count (the
+# per-layer launches repeat unchanged; profiles/zoqat_step_llama7b_w4a8_launch_list.md), keyed by workload; absent
+# for workloads that have not been captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"llama7b_w4a8": 779.7e6}
 
 
 def load_peaks():
