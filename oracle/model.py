@@ -116,6 +116,11 @@ class OracleConfig:
     integer_linear: bool = False     # deployment arithmetic of the frozen (packed) linears, used by the decode path: integer
                                      # dot products of activation codes and weight codes inside each group, the group step
                                      # and the token step applied outside (no bfloat16 rounding of the dequantised weight)
+    integer_gemm: bool = False       # the same integer arithmetic for EVERY quantised block linear, trainable ones included
+                                     # (perturbed weights, learnable quantiser, smoothing): with one weight group per output
+                                     # row and per-token activation codes the product of the two fake-quantised operands is
+                                     # exactly  s_t * Delta_n * sum_k a[t, k] * (c[n, k] - z_n), the plain definition of
+                                     # Q(x) Q(w)^T with no operand rounding at all
     store_f32: bool = False          # True rounds every stored activation (linear, attention and norm outputs, the
                                      # residual stream) to binary32, as an implementation that keeps activations in
                                      # fp32 does; used only to measure how far two correct implementations can differ
@@ -292,37 +297,71 @@ class OracleModel:
     def _operand_round(self, x):
         return core.round_bf16(x.astype(F32)).astype(np.float64) if self.cfg.operand_bf16 else x
 
-    def lin_integer(self, x, l, name, bias=None):
+    def block_codes(self, l, name, seed, signed_eps):
+        """Integer form of the fake-quantised weight of a block linear: (c - z) as float64 integers [out, in] and the
+        step Delta float32 [out, in / group], from the same quantiser (min/max or learnable, after perturbation and
+        smoothing) that block_operand() uses; the dequantised value is their product."""
+        cfg = self.cfg
+        w = self.perturbed_weight(l, name, seed, signed_eps)
+        if self.has_smoothing(l):
+            s_, _ = self.smoothing_params(l, name, seed, signed_eps)
+            w = (w * s_[None, :]).astype(F32)
+        g = self.group_of(w)
+        N, K = w.shape
+        if self.has_adaptive(l, name):
+            th = self.p["layers"][l]["theta_" + name]
+            if signed_eps != 0.0:
+                th = core.perturb(th, seed, tensor_id(l, self._ROLE[name]) + QPARAM_ID, signed_eps)
+            q, _ = adaptive_weight_quant(w, th, g, cfg.w_bits)
+            th = np.asarray(th, dtype=F32).reshape(N, K // g, 4)
+            delta = np.maximum(th[..., 0], F32(1e-8))
+            z = np.rint(th[..., 1]).astype(np.float64)
+        else:
+            q, delta, zp, _ = core.weight_quant(w, g, cfg.w_bits)
+            z = zp.astype(np.float64)
+        cz = q.astype(np.float64).reshape(N, K // g, g) - z[:, :, None]
+        return cz.reshape(N, K), delta
+
+    def lin_integer(self, x, l, name, seed=0, signed_eps=0.0, bias=None, extra=None):
         """The linear as an integer runtime evaluates it (Section 4.3 representation: stored codes, one step and zero
         point per group; per-token activation codes):
             y[t, n] = s_t * sum_g Delta[n, g] * ( sum_{k in g} a[t, k] * (c[n, k] - z[n, g]) )
-        with the inner sums exact integers."""
+        with the inner sums exact integers.  x is the input after smoothing, if any."""
         cfg = self.cfg
-        w = self.p["layers"][l][name]
-        g = self.group_of(w)
-        codes, delta, zp, _ = core.weight_quant(w, g, cfg.w_bits)
+        cz, delta = self.block_codes(l, name, seed, signed_eps)
         a, s = act_quant(x, cfg.a_bits)
         T, K = a.shape
-        N = w.shape[0]
-        cz = codes.reshape(N, K // g, g).astype(np.float64) - zp.astype(np.float64)[:, :, None]
-        inner = np.einsum("tgk,ngk->tng", a.reshape(T, K // g, g), cz)          # exact: integers far below 2^53
-        y = (inner * delta.astype(np.float64)[None, :, :]).sum(axis=-1) * s.astype(np.float64)[:, None]
+        N, G = delta.shape
+        g = K // G
+        inner = np.einsum("tgk,ngk->tng", a.reshape(T, G, g), cz.reshape(N, G, g))   # exact: integers far below 2^53
+        if cfg.accum_f32:       # binary32 outside the integer sums: convert, scale by the group step, by the token step
+            y = ((inner.astype(F32) * delta[None, :, :]).astype(F32).sum(axis=-1, dtype=F32) * s[:, None]).astype(F32).astype(np.float64)
+        else:
+            y = (inner * delta.astype(np.float64)[None, :, :]).sum(axis=-1) * s.astype(np.float64)[:, None]
         if bias is not None:
             y = y + bias.astype(np.float64)[None, :]
+        if extra is not None:
+            y = y + extra[None, :]
         return self._store(y)
+
+    def uses_integer(self, l, name):
+        cfg = self.cfg
+        if not (cfg.a_bits and cfg.w_bits):
+            return False
+        return cfg.integer_gemm or (cfg.integer_linear and not self.is_trainable(l, name))
 
     def lin(self, x, l, name, seed, signed_eps, bias=None):
         """x [T, in] float64 -> [T, out] float64 through the quantised linear.  With smoothing
         (Section 4.2): Y = Q_a((X - delta) / s) Q_w(s (.) W)^T + (B + delta W^T), the division taken in
         binary32 as a multiplication by 1/s rounded once, the shift term with the unquantised W."""
-        if self.cfg.integer_linear and self.cfg.a_bits and self.cfg.w_bits and not self.is_trainable(l, name):
-            return self.lin_integer(x, l, name, bias)
         extra = None
         if self.has_smoothing(l):
             s_, d_ = self.smoothing_params(l, name, seed, signed_eps)
             inv = (F32(1.0) / s_).astype(F32)
             x = (((x.astype(F32) - d_[None, :]).astype(F32)) * inv[None, :]).astype(F32).astype(np.float64)
             extra = self.perturbed_weight(l, name, seed, signed_eps).astype(np.float64) @ d_.astype(np.float64)
+        if self.uses_integer(l, name):
+            return self.lin_integer(x, l, name, seed, signed_eps, bias, extra)
         if self.cfg.a_bits:
             a, s = act_quant(x, self.cfg.a_bits)
             y = self._matmul_t(a, self.block_operand(l, name, seed, signed_eps)) * s.astype(np.float64)[:, None]

@@ -169,3 +169,61 @@ def test_estimate_sees_the_learnables():
     # zero perturbation: both passes coincide
     lp = m.loss(tokens, labels, 5, 0.0)
     assert lp == plain.loss(tokens, labels, 5, 0.0)
+
+
+# ---- integer form of the quantised linears (per-row weight groups, per-token activation codes) ----------------
+def test_integer_form_hand_cases():
+    """block_codes / lin_integer with the learnable quantiser, by hand: bits 2, Delta 0.5, z 2, levels [0, 3];
+    w / Delta = [-2, -0.5, 1, 4] rounds (ties to even) to [-2, -0, 1, 4], + z = [0, 2, 3, 6], clamped [0, 2, 3, 3],
+    minus z = [-2, 0, 1, 1]; with activation codes [127, -64, 32, 1] at step 1: -254 + 32 + 1 = -221, times Delta."""
+    cfg = OracleConfig(arch="llama", n_layers=1, d_model=4, n_heads=1, d_ffn=4, vocab=4, w_bits=2, w_group=0, a_bits=8,
+                       adaptive_quant=True, integer_gemm=True, head_trainable=False)
+    w = np.array([[-1.0, -0.25, 0.5, 2.0], [0.0, 1.5, 2.5, 3.0]], np.float32)
+    th = np.array([[[0.5, 2.0, 0.0, 1.0]], [[1.0, 0.0, 0.0, 1.0]]], np.float32)
+    m = OracleModel(cfg, {"layers": [{"wq": w, "theta_wq": th}]})
+    cz, delta = m.block_codes(0, "wq", 0, 0.0)
+    assert cz.tolist() == [[-2.0, 0.0, 1.0, 1.0], [0.0, 2.0, 2.0, 3.0]] and delta.tolist() == [[0.5], [1.0]]
+    x = np.array([[127.0, -64.0, 32.0, 1.0], [63.5, 0.0, 0.0, 0.0]])    # second token: step 0.5, codes [127, 0, 0, 0]
+    y = m.lin_integer(x, 0, "wq", bias=np.array([0.25, 0.0], np.float32))
+    assert y.tolist() == [[-110.5 + 0.25, -128.0 + 64.0 + 3.0], [0.5 * 0.5 * 127 * -2 + 0.25, 0.0]]
+
+
+@pytest.mark.parametrize("arch,adaptive,smoothing", [("llama", False, False), ("llama", True, True), ("opt", True, True)])
+def test_integer_form_is_the_product_of_the_two_fake_quantised_operands(arch, adaptive, smoothing):
+    """With one group per row, s_t * Delta_n * sum a (c - z) is Q(x) Q(w)^T itself.  The forward that multiplies the
+    dequantised binary32 operands in float64 (no bfloat16 rounding) differs only by the rounding of (c - z) * Delta to
+    binary32, 2^-24 relative per weight; the training forward (bfloat16 operands) by 2^-9."""
+    shape = dict(arch=arch, n_layers=2, d_model=32, n_heads=4, d_ffn=64, vocab=50)
+    p = synth.make_params(shape, seed=5, max_seq=16, jitter=True)
+    cfg = OracleConfig(w_bits=4, w_group=0, a_bits=8, adaptive_quant=adaptive, smoothing=smoothing, **shape)
+    m = OracleModel(cfg, p)
+    m.init_learnable()
+    if smoothing:
+        _randomise_smoothing(m, np.random.default_rng(8))
+    tokens, labels = synth.make_batch(2, 12, 50, seed=2)
+    out, loss = {}, {}
+    eps = float(np.float32(1e-3))
+    for key, kw in (("bf16", {}), ("f32", dict(operand_bf16=False)), ("int", dict(integer_gemm=True))):
+        for k, v in {"operand_bf16": True, "integer_gemm": False, **kw}.items():
+            setattr(m.cfg, k, v)
+        taps = {}
+        m.tap = lambda name, arr: taps.__setitem__(name, np.array(arr))
+        loss[key] = m.token_losses(tokens, labels, seed=9, signed_eps=eps)[0]
+        m.tap = None
+        out[key] = taps["l1.h_out"]        # the residual stream after the last block: every block linear is behind it
+    scale = np.abs(out["f32"]).max()
+    assert np.abs(out["int"] - out["f32"]).max() < 2e-6 * scale
+    d = np.abs(out["int"] - out["bf16"]).max()
+    assert 1e-5 * scale < d < 5e-2 * scale
+    # the two-point estimate goes through the same arithmetic
+    m.cfg.operand_bf16, m.cfg.integer_gemm = True, True
+    lp, lm, g = m.projected_gradient(tokens, labels, 9, 1e-3)
+    assert lp == pytest.approx(float(loss["int"].sum() / (labels >= 0).sum()), rel=1e-12)
+    assert g == pytest.approx((lp - lm) / (2 * eps), rel=1e-6)
+
+
+def test_integer_form_needs_quantised_inputs_and_weights():
+    shape = dict(arch="llama", n_layers=1, d_model=32, n_heads=4, d_ffn=64, vocab=50)
+    p = synth.make_params(shape, seed=5, max_seq=16, jitter=True)
+    m = OracleModel(OracleConfig(w_bits=4, w_group=0, a_bits=0, integer_gemm=True, **shape), p)
+    assert not m.uses_integer(0, "wq")
