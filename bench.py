@@ -139,7 +139,8 @@ def oracle_sample(w, budget_note=True):
     cores = os.cpu_count() or 1
     cfg = OracleConfig(arch=w["arch"], n_layers=1, d_model=w["d_model"], n_heads=w["n_heads"], d_ffn=w["d_ffn"],
                        vocab=w["vocab"], w_bits=w["w_bits"], w_group=w["w_group"], a_bits=w["a_bits"],
-                       adaptive_quant=bool(w.get("adaptive_quant")), smoothing=bool(w.get("smoothing")))
+                       adaptive_quant=bool(w.get("adaptive_quant")), smoothing=bool(w.get("smoothing")),
+                       integer_gemm=bool(w.get("integer_gemm")))
     params = synth.make_params(one, seed=0, max_seq=seq2)
     model = OracleModel(cfg, params)
     model.init_learnable()
@@ -197,7 +198,7 @@ def run_ours(args, w, rank, world, local_rank):
     any_packed = ftl > 0 or names is not None
     model = binding.ZoqatModel(w, params, max_batch=w["batch"], max_seq=w["seq"], first_trainable_layer=ftl,
                                packed_frozen=any_packed, trainable_names=names, head_trainable=w.get("head_trainable", True),
-                               gemm_impl=binding.GEMM_SIMT if args.simt else binding.GEMM_TCGEN05,
+                               gemm_impl=binding.GEMM_SIMT if args.simt else (binding.GEMM_TCGEN05_I8 if w.get("integer_gemm") else binding.GEMM_TCGEN05),
                                adaptive_quant=bool(w.get("adaptive_quant")), smoothing=bool(w.get("smoothing")))
     if w.get("adaptive_quant"):
         model.zoqat_init_qparams()
@@ -288,14 +289,22 @@ def run_ours(args, w, rank, world, local_rank):
     peak_tf = peaks["tf_sustained"]
     t_flop = nums["flops"] / (peaks["tf_burst"] * 1e12)
     t_hbm = nums["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    i8 = bool(w.get("integer_gemm")) and not args.simt
+    if i8:
+        # block linears on 8-bit integers: their peak is the measured bf16 peak x 2 (nominal int8 : bf16 ratio of the part);
+        # the vocabulary projection and the attention stay on the bf16 / fp16 peak
+        head_flops = 2 * nums["T"] * 2 * nums["head_params"]
+        t_flop_bf16 = t_flop
+        t_flop = ((nums["linear_flops"] - head_flops) / 2 + head_flops + nums["attn_flops"]) / (peaks["tf_burst"] * 1e12)
     roof_s = max(t_flop, t_hbm)
     line = dict(
         metric=METRIC, value=steps_per_s, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
-        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+        ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="s8 (block linears, s32 sums) + bf16 (vocabulary projection)" if i8 else "bf16",
         data="synthetic", fwd_tokens_per_s=2 * nums["T"] * steps_per_s,
         config=dict(workload=args.workload + (f" cut to {w['n_layers']} layers" if args.layers > 0 else ""),
                     l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
-                    gemm="simt" if args.simt else "tcgen05",
+                    gemm="simt" if args.simt else ("tcgen05 kind::i8 (block linears) + kind::f16" if i8 else "tcgen05"),
                     mode="batch-sharded replicas" if args.mode == "batch" else "direction-parallel replicas (q = n_gpus, value counts two-point evaluations)",
                     **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab", "w_bits", "w_group",
                                          "a_bits", "batch", "seq")}),
@@ -312,6 +321,12 @@ def run_ours(args, w, rank, world, local_rank):
         gpu_launches=launches, clocks=clocks,
         last_step=dict(loss_plus=res["loss_plus"], loss_minus=res["loss_minus"], proj_grad=res["proj_grad"], status=res["status"]),
     )
+    if i8:
+        line["step_roofline"]["peak_source"] = peaks["source"] + " (burst bf16 x 2 for the 8-bit block linears: nominal ratio; copy HBM)"
+        line["step_roofline"]["frac_of_bf16_roofline"] = max(t_flop_bf16, t_hbm) * 1e3 / ms_per_step
+        line["roofline"]["peak"] = 2 * peak_tf
+        line["roofline"]["frac"] = (achieved_tf / (2 * peak_tf)) if achieved_tf else None
+        line["roofline"]["peak_source"] = peaks["source"] + " sustained bf16 x 2 (nominal int8 : bf16 ratio); the launches include the bf16 vocabulary projection"
     if args.mode == "directions":
         line["step_roofline"] = None          # the roofline model below is that of the one-direction step
     if e2e_ms is not None:

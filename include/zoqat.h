@@ -105,6 +105,16 @@ extern "C" {
                                   pair of CTAs on two SMs with one cta_group::2 MMA                                  */
 #define ZOQAT_GEMM_SIMT    1   /* plain CUDA-core kernels, kept as an on-device cross-check                          */
 #define ZOQAT_GEMM_TCGEN05_1CTA 2 /* as 0, but every GEMM tile (128 rows) belongs to a single CTA                    */
+#define ZOQAT_GEMM_TCGEN05_I8  3  /* as 0, with every block linear evaluated on integers (appendix on quantisation
+                                     settings: one weight scale per output channel, one activation scale per token):
+                                       y[t, n] = s_t * (Delta_n * sum_k a[t, k] * (c[n, k] - z_n)) (+ bias),
+                                     the sum exact (tcgen05.mma kind::i8 on signed bytes, 32-bit accumulators), which
+                                     is Q(x) Q(w)^T of Section 2 with no rounding of the operands; ZOQAT_GEMM_TCGEN05
+                                     instead rounds the dequantised weight (c - z) * Delta to bf16.  Needs w_group = 0,
+                                     a_bits != 0, w_bits <= 7, every block linear QUANTIZED and none FROZEN_PACKED; the
+                                     vocabulary projection stays bf16.  A weight row whose c - z leaves [-128, 127]
+                                     (zero point far outside the code range) makes the step report status 32 and
+                                     zoqat_check() return ZOQAT_ERR_UNSUPPORTED; results of that call are not usable. */
 
 typedef struct zoqat_config {
     int32_t arch;          /* ZOQAT_ARCH_*                                                        */
@@ -323,7 +333,8 @@ int zoqat_debug_buffer(zoqat_model_t* m, int which, void** dev_ptr, size_t* byte
  * ffn_in, ffn_out) and in execution order, one record into `buf_dev`:
  *   input   fp32 [rows, cols]   the value the quantiser saw (after the norm / non-linearity, before the Section 4.2
  *                               shift and scale if the layer has them)
- *   operand bf16 [rows, cols]   what the quantiser wrote for the GEMM (integer codes, or bf16(x) when a_bits = 0)
+ *   operand bf16 [rows, cols]   what the quantiser wrote for the GEMM (integer codes, or bf16(x) when a_bits = 0); with
+ *                               ZOQAT_GEMM_TCGEN05_I8 the block records hold int8 [rows, cols] in the first half of the slot
  *   step    fp32 [rows]         the per-token step
  * each part padded to a multiple of 256 bytes; rows = passes * batch * seq as materialised at that layer (a frozen
  * prefix is evaluated once: rows = batch * seq there), cols = d_model (d_ffn at ffn_out).  One more record follows
@@ -447,6 +458,31 @@ int zoqat_op_gemm(const void* a_dev, const void* b_dev, int64_t M, int64_t N, in
 int zoqat_op_gemm_silu_gate(const void* a_dev, const void* b_dev, int64_t M, int64_t F, int64_t K,
                             const float* row_step_dev, float* act_dev, uint32_t* row_amax_dev,
                             int32_t* err_flag_dev, void* stream);
+
+/* The linear on 8-bit integers (ZOQAT_GEMM_TCGEN05_I8; Section 2 quantisers with one weight group per output row):
+ *   out[m, n] (+)= row_step[m] * (col_step[n] * sum_k A[m, k] * B[n, k]) (+ bias[n]),
+ * the sum an exact 32-bit integer, converted to fp32 once (round to nearest) before the two multiplications.
+ * a_dev int8 [M, K] (activation codes), b_dev int8 [N, K] (weight codes minus zero point), col_step_dev fp32 [N]
+ * (required), row_step_dev / bias_dev may be NULL; K % 16 == 0, N % 32 == 0, 16-byte aligned pointers.
+ * gated = 1: the SiLU-gated pair of zoqat_op_gemm_silu_gate (N = 2F, b_dev gate rows then up rows, out_dev fp32
+ * [M, F], row_amax_dev uint32 [M] required, no accumulation); gated = 0: out_dev fp32 [M, N]. */
+int zoqat_op_gemm_i8(const void* a_dev, const void* b_dev, int64_t M, int64_t N, int64_t K,
+                     const float* row_step_dev, const float* col_step_dev, const float* bias_dev, int accumulate,
+                     int gated, float* out_dev, uint32_t* row_amax_dev, int32_t* err_flag_dev, void* stream);
+
+/* zoqat_op_weight_operand_learned with one group per row, writing the operands of the integer GEMM: operand_plus_dev /
+ * operand_minus_dev int8 [rows, cols] = code minus zero point (16-byte aligned; the second may be NULL), col_step_dev
+ * fp32 [2][rows] (or [rows]) = the rows' steps per sign.  err_flag_dev (int32, zeroed by the caller) is set to 32 if a
+ * row's code minus zero point leaves [-128, 127].  bits 2..7; other arguments as there. */
+int zoqat_op_weight_operand_i8(const float* w_dev, int64_t rows, int64_t cols, int bits, uint64_t seed,
+                               uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
+                               const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
+                               void* operand_minus_dev, float* col_step_dev, int32_t* err_flag_dev, void* stream);
+
+/* zoqat_op_norm_act_operand writing the per-token codes as signed bytes: operand_dev int8 [rows, cols]; a_bits 4, 6, 8. */
+int zoqat_op_norm_act_operand_i8(const float* x_dev, int64_t rows, int64_t cols, int norm_kind,
+                                 const float* gain_dev, const float* bias_dev, float norm_eps, int a_bits,
+                                 void* operand_dev, float* row_step_dev, void* stream);
 
 /* Causal softmax attention of one layer (the architecture of the workloads; the paper's
  * forward pass of Section 4.1 runs the unmodified decoder between the quantised linears).

@@ -20,7 +20,7 @@ ARCH_LLAMA, ARCH_OPT = 0, 1
 ROLE_SMOOTH_SCALE, ROLE_SMOOTH_SHIFT = 22, 26      # + quantisation point 0..3 (Section 4.2)
 SMOOTH_POINTS = ("attn_in", "attn_out", "ffn_in", "ffn_out")
 TENSOR_TRAINABLE, TENSOR_QUANTIZED, TENSOR_FROZEN_PACKED, TENSOR_ADAPTIVE = 1, 2, 4, 8
-GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_1CTA = 0, 1, 2
+GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_1CTA, GEMM_TCGEN05_I8 = 0, 1, 2, 3
 BUF_RESIDUAL, BUF_QKV, BUF_ATTN, BUF_FFN, BUF_TOKEN_LOSS = range(5)
 PROF_GEMM, PROF_WEIGHT, PROF_ACT, PROF_ATTENTION, PROF_LOSS, PROF_UPDATE = range(6)
 PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "update"]
@@ -33,7 +33,7 @@ EXPORTS = [
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
     "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
-    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_qkv_attention", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
+    "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_gemm_i8", "zoqat_op_weight_operand_i8", "zoqat_op_norm_act_operand_i8", "zoqat_op_qkv_attention", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
     "zoqat_decode_bytes", "zoqat_decode_begin", "zoqat_decode_step", "zoqat_op_decode_gemv",
@@ -126,6 +126,9 @@ def lib():
             "zoqat_op_ffn_act_operand": [vp, i64, i64, i32, i32, vp, vp, vp],
             "zoqat_op_gemm": [vp, vp, i64, i64, i64, vp, vp, i32, i32, vp, i32, vp, vp],
             "zoqat_op_gemm_silu_gate": [vp, vp, i64, i64, i64, vp, vp, vp, vp, vp],
+            "zoqat_op_gemm_i8": [vp, vp, i64, i64, i64, vp, vp, vp, i32, i32, vp, vp, vp, vp],
+            "zoqat_op_weight_operand_i8": [vp, i64, i64, i32, u64, u32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "zoqat_op_norm_act_operand_i8": [vp, i64, i64, i32, vp, vp, f32, i32, vp, vp, vp],
             "zoqat_op_attention_scratch_bytes": [i32, i32, i32, i32, P(sz)],
             "zoqat_op_qkv_attention": [vp, vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp],
             "zoqat_op_attention": [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp, vp],
@@ -301,6 +304,42 @@ def zoqat_op_gemm_silu_gate(a, b_gate_up, row_step=None):
     return act, amax.view(torch.float32), err
 
 
+def zoqat_op_gemm_i8(a, b, col_step, row_step=None, bias=None, out=None, accumulate=False, gated=False):
+    """a int8 [M, K], b int8 [N, K] -> (out fp32 [M, N] or [M, N/2] when gated, row maxima or None, error word)."""
+    M, K = a.shape
+    N = b.shape[0]
+    if out is None:
+        out = torch.empty((M, N // 2 if gated else N), dtype=torch.float32, device=a.device)
+    amax = torch.empty(M, dtype=torch.int32, device=a.device) if gated else None
+    err = torch.zeros(1, dtype=torch.int32, device=a.device)
+    _check(lib().zoqat_op_gemm_i8(_p(a), _p(b), M, N, K, _p(row_step), _p(col_step), _p(bias), int(accumulate), int(gated),
+                                  _p(out), _p(amax), _p(err), _stream()))
+    return out, (amax.view(torch.float32) if gated else None), err
+
+
+def zoqat_op_weight_operand_i8(w, bits, seed, tensor_id, eps, theta=None, smooth=None, bias0=None, dual=True):
+    """-> (int8 operand of +eps, of -eps or None, steps [signs, rows], smoothed bias or None, error word)."""
+    rows, cols = w.shape
+    plus = torch.empty((rows, cols), dtype=torch.int8, device=w.device)
+    minus = torch.empty_like(plus) if dual else None
+    steps = torch.zeros((2 if dual else 1, rows), dtype=torch.float32, device=w.device)
+    scratch = torch.empty(18 * rows * (cols // 128), dtype=torch.float32, device=w.device)
+    bias = torch.empty((2 if dual else 1, rows), dtype=torch.float32, device=w.device) if smooth is not None else None
+    err = torch.zeros(1, dtype=torch.int32, device=w.device)
+    _check(lib().zoqat_op_weight_operand_i8(_p(w), rows, cols, bits, seed, tensor_id, eps, _p(theta), _p(smooth), _p(bias0),
+                                            _p(bias), _p(scratch), _p(plus), _p(minus), _p(steps), _p(err), _stream()))
+    return plus, minus, steps, bias, err
+
+
+def zoqat_op_norm_act_operand_i8(x, norm_kind, gain, bias, norm_eps, a_bits):
+    rows, cols = x.shape
+    operand = torch.empty((rows, cols), dtype=torch.int8, device=x.device)
+    row_step = torch.empty(rows, dtype=torch.float32, device=x.device)
+    _check(lib().zoqat_op_norm_act_operand_i8(_p(x), rows, cols, norm_kind, _p(gain), _p(bias), norm_eps, a_bits,
+                                              _p(operand), _p(row_step), _stream()))
+    return operand, row_step
+
+
 def zoqat_op_attention(qkv, batch, seq, n_heads, d_head, cos=None, sin=None, impl=GEMM_TCGEN05, scratch=None, err=None):
     out = torch.empty((batch * seq, n_heads * d_head), dtype=torch.float32, device=qkv.device)
     if impl == GEMM_TCGEN05:
@@ -402,6 +441,7 @@ class ZoqatModel:
                           d_model=shape["d_model"], n_heads=shape["n_heads"], d_ffn=shape["d_ffn"], vocab=shape["vocab"],
                           max_batch=max_batch, max_seq=max_seq, w_bits=shape["w_bits"], w_group=shape["w_group"],
                           a_bits=shape["a_bits"], gemm_impl=gemm_impl, norm_eps=norm_eps, rope_base=rope_base)
+        self.gemm_impl = gemm_impl
         nbytes = ctypes.c_size_t()
         _check(L.zoqat_query_workspace(ctypes.byref(self.cfg), ctypes.byref(nbytes)))
         self.workspace_bytes = nbytes.value
@@ -632,7 +672,11 @@ class ZoqatModel:
             for point in range(4 if l < self.shape["n_layers"] else 1):
                 cols = self.shape["d_ffn"] if point == 3 else self.shape["d_model"]
                 x = buf[off:off + rows * cols * 4].view(torch.float32).view(rows, cols); off += up(rows * cols * 4)
-                op = buf[off:off + rows * cols * 2].view(torch.bfloat16).view(rows, cols); off += up(rows * cols * 2)
+                if self.gemm_impl == GEMM_TCGEN05_I8 and l < self.shape["n_layers"]:     # signed bytes in the first half
+                    op = buf[off:off + rows * cols].view(torch.int8).view(rows, cols)
+                else:
+                    op = buf[off:off + rows * cols * 2].view(torch.bfloat16).view(rows, cols)
+                off += up(rows * cols * 2)
                 st = buf[off:off + rows * 4].view(torch.float32); off += up(rows * 4)
                 out.append((l, point, x, op, st))
         return out

@@ -72,6 +72,15 @@ __device__ __forceinline__ void store_code_planes(const CodePlanes& pl, int idx,
     }
 }
 
+// planes == 2: the codes as signed bytes in row-major order (the operand of the 8-bit integer GEMM), row r at byte r * cols.
+__device__ __forceinline__ __nv_bfloat16* operand_row(__nv_bfloat16* op, int64_t r, int cols, int planes) {
+    return planes == 2 ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(op) + r * cols) : op + r * cols;
+}
+__device__ __forceinline__ uint32_t s8x4(float a, float b, float c, float d) {
+    return ((uint32_t)__float2int_rn(a) & 0xFFu) | (((uint32_t)__float2int_rn(b) & 0xFFu) << 8) |
+           (((uint32_t)__float2int_rn(c) & 0xFFu) << 16) | ((uint32_t)__float2int_rn(d) << 24);
+}
+
 // Writes the operand row from the fp32 row held in shared memory.
 __device__ __forceinline__ void write_operand_row(const float* row, int cols, int a_bits, __nv_bfloat16* op_row,
                                                   float* row_step, float* redf, int planes = 0) {
@@ -83,6 +92,16 @@ __device__ __forceinline__ void write_operand_row(const float* row, int cols, in
         const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
+        if (planes == 2) {                     // cols % 4 == 0
+            uint32_t* o = reinterpret_cast<uint32_t*>(op_row);
+            for (int idx = threadIdx.x; idx < (cols >> 2); idx += kRowThreads) {
+                float q[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) q[j] = fminf(fmaxf(rintf(__fmul_rn(row[4 * idx + j], inv)), qmin), qmax);
+                o[idx] = s8x4(q[0], q[1], q[2], q[3]);
+            }
+            return;
+        }
         if (planes) {                          // cols % 32 == 0: every warp runs every round, loads and stores are guarded
             const CodePlanes pl = code_planes(op_row, cols);
             const int n4 = cols >> 2;
@@ -148,7 +167,7 @@ norm_act_operand_kernel(const float* __restrict__ x, int cols, int norm_kind, co
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
         __syncthreads();
     }
-    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf, planes);
+    write_operand_row(row, cols, a_bits, operand_row(op, r, cols, planes), row_step + r, redf, planes);
 }
 
 __global__ void __launch_bounds__(kRowThreads)
@@ -177,7 +196,7 @@ ffn_act_operand_kernel(const float* __restrict__ x, int cols, int gated, int a_b
         for (int c = threadIdx.x; c < cols; c += kRowThreads) row[c] = smooth1(row[c], b[sm.ld + c], b[2 * (size_t)sm.ld + c]);
     }
     __syncthreads();
-    write_operand_row(row, cols, a_bits, op + r * cols, row_step + r, redf, planes);
+    write_operand_row(row, cols, a_bits, operand_row(op, r, cols, planes), row_step + r, redf, planes);
 }
 
 // ---- register-resident variants (rows up to 12288 columns) ------------------------------------------------
@@ -202,6 +221,19 @@ __device__ __forceinline__ void write_operand_regs(const float4 (&v)[VPT], int n
         const float step = fmaxf(__fdiv_rn(amax, qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) *row_step = step;
+        if (planes == 2) {
+            uint32_t* o = reinterpret_cast<uint32_t*>(op_row);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int idx = threadIdx.x + i * kRowThreads;
+                if (idx < n4)
+                    o[idx] = s8x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), qmin), qmax));
+            }
+            return;
+        }
         if (planes) {
             const CodePlanes pl = code_planes(reinterpret_cast<__nv_bfloat16*>(op_row), 4 * n4);
 #pragma unroll
@@ -318,7 +350,7 @@ norm_act_operand_reg_kernel(const float* __restrict__ x, int cols, int norm_kind
         }
     }
     smooth_regs<VPT>(v, n4, sm, r);
-    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf, planes);
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(operand_row(op, r, cols, planes)), row_step + r, redf, planes);
 }
 
 template <int VPT>
@@ -365,18 +397,18 @@ ffn_act_operand_reg_kernel(const float* __restrict__ x, int cols, int gated, int
         }
     }
     smooth_regs<VPT>(v, n4, sm, r);
-    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(op + r * cols), row_step + r, redf, planes);
+    write_operand_regs<VPT>(v, n4, a_bits, reinterpret_cast<uint2*>(operand_row(op, r, cols, planes)), row_step + r, redf, planes);
 }
 
 // Activation operand of a row whose max |x| has already been collected (by the GEMM that produced x).
 template <int VPT>
 __global__ void __launch_bounds__(kRowThreads)
 rows_operand_reg_kernel(const float* __restrict__ x, int cols, const uint32_t* __restrict__ amax_bits, int a_bits,
-                        __nv_bfloat16* __restrict__ op, float* __restrict__ row_step) {
+                        __nv_bfloat16* __restrict__ op, float* __restrict__ row_step, int planes) {
     const int64_t r = blockIdx.x;
     const int n4 = cols >> 2;
     const float4* xr = reinterpret_cast<const float4*>(x + r * cols);
-    uint2* op_row = reinterpret_cast<uint2*>(op + r * cols);
+    uint2* op_row = reinterpret_cast<uint2*>(operand_row(op, r, cols, planes));
     float4 v[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
@@ -388,6 +420,19 @@ rows_operand_reg_kernel(const float* __restrict__ x, int cols, const uint32_t* _
         const float step = fmaxf(__fdiv_rn(__uint_as_float(amax_bits[r]), qmax), 1e-8f);
         const float inv = __fdiv_rn(1.0f, step);
         if (threadIdx.x == 0) row_step[r] = step;
+        if (planes == 2) {
+            uint32_t* o = reinterpret_cast<uint32_t*>(op_row);
+#pragma unroll
+            for (int i = 0; i < VPT; ++i) {
+                const int idx = threadIdx.x + i * kRowThreads;
+                if (idx < n4)
+                    o[idx] = s8x4(fminf(fmaxf(rintf(__fmul_rn(v[i].x, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].y, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].z, inv)), qmin), qmax),
+                                  fminf(fmaxf(rintf(__fmul_rn(v[i].w, inv)), qmin), qmax));
+            }
+            return;
+        }
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int idx = threadIdx.x + i * kRowThreads;
@@ -527,51 +572,51 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
-                             SmoothAct sm, bool dependent, bool planes) {
+                             SmoothAct sm, bool dependent, int planes) {
     const int n4 = cols / 4;
     const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gain) | reinterpret_cast<uintptr_t>(bias) |
                            reinterpret_cast<uintptr_t>(normed)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        launch_kernel(norm_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
+        launch_kernel(norm_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        launch_kernel(norm_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
+        launch_kernel(norm_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        launch_kernel(norm_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
+        launch_kernel(norm_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static DeviceOnce attr;
         if (attr.first()) { cudaFuncSetAttribute(norm_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); }
-        launch_kernel(norm_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes ? 1 : 0);
+        launch_kernel(norm_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, norm_kind, gain, bias, norm_eps, a_bits, op, row_step, normed, sm, planes);
     }
     count_launch();
 }
 
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits, __nv_bfloat16* op,
-                            float* row_step, cudaStream_t s, SmoothAct sm, bool dependent, bool planes, float* pre) {
+                            float* row_step, cudaStream_t s, SmoothAct sm, bool dependent, int planes, float* pre) {
     const int n4 = cols / 4;
     const bool aligned = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(pre)) & 15) == 0 && (reinterpret_cast<uintptr_t>(op) & 7) == 0;
     if (aligned && n4 <= 4 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
+        launch_kernel(ffn_act_operand_reg_kernel<4>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes, pre);
     } else if (aligned && n4 <= 8 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
+        launch_kernel(ffn_act_operand_reg_kernel<8>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes, pre);
     } else if (aligned && n4 <= 12 * kRowThreads) {
-        launch_kernel(ffn_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
+        launch_kernel(ffn_act_operand_reg_kernel<12>, dim3((unsigned)rows), dim3(kRowThreads), 0, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes, pre);
     } else {
         const size_t smem = (size_t)cols * sizeof(float);
         static DeviceOnce attr;
         if (attr.first()) { cudaFuncSetAttribute(ffn_act_operand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024); }
-        launch_kernel(ffn_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes ? 1 : 0, pre);
+        launch_kernel(ffn_act_operand_kernel, dim3((unsigned)rows), dim3(kRowThreads), smem, s, dependent, x, cols, gated, a_bits, op, row_step, sm, planes, pre);
     }
     count_launch();
 }
 
 void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits, __nv_bfloat16* op,
-                         float* row_step, cudaStream_t s) {
+                         float* row_step, cudaStream_t s, int planes) {
     const int n4 = cols / 4;       // callers guarantee cols % 4 == 0, cols <= 16384 and 16-byte aligned rows
-    if (n4 <= 4 * kRowThreads) rows_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
-    else if (n4 <= 8 * kRowThreads) rows_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
-    else if (n4 <= 12 * kRowThreads) rows_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
-    else rows_operand_reg_kernel<16><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step);
+    if (n4 <= 4 * kRowThreads) rows_operand_reg_kernel<4><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step, planes);
+    else if (n4 <= 8 * kRowThreads) rows_operand_reg_kernel<8><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step, planes);
+    else if (n4 <= 12 * kRowThreads) rows_operand_reg_kernel<12><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step, planes);
+    else rows_operand_reg_kernel<16><<<(unsigned)rows, kRowThreads, 0, s>>>(x, cols, amax, a_bits, op, row_step, planes);
     count_launch();
 }
 

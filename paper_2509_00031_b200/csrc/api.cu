@@ -86,6 +86,7 @@ struct Workspace {
     uint8_t* qprep;                     // prepared (perturbed) quantiser parameters of the current layer's linears
     size_t qprep_off[8];                // byte offset of each block linear's block inside qprep
     float* bias_pm;                     // smoothed bias per pass: [sign][bias_ld]
+    float* col_step;                    // 8-bit integer GEMM: step of every output column per pass: [sign][bias_ld]
     float* class_scales;                // {lr_quant * g, lr_smooth * g}
     float* pending_scale;               // factor lr * g of a deferred update
     int smooth_ld, bias_ld;
@@ -141,6 +142,7 @@ void layout_workspace(const zoqat_config_t& c, uint8_t* base, Workspace& w) {
     }
     w.bias_ld = (int)(3 * d > ffn_cols ? 3 * d : ffn_cols);
     w.bias_pm = (float*)take((size_t)2 * w.bias_ld * 4);
+    w.col_step = (float*)take((size_t)2 * w.bias_ld * 4);
     w.class_scales = (float*)take(2 * 4);
     w.pending_scale = (float*)take(4);
     w.total = off;
@@ -160,7 +162,11 @@ int validate_config(const zoqat_config_t* c) {
     if (c->w_group == 0 && (c->d_model % 128 || c->d_ffn % 128)) return fail(ZOQAT_ERR_UNSUPPORTED, "per-row weight groups need d_model and d_ffn to be multiples of 128");
     if (c->w_group != 0 && (c->d_model % c->w_group || c->d_ffn % c->w_group)) return fail(ZOQAT_ERR_INVALID_ARG, "w_group must divide d_model and d_ffn");
     if (c->a_bits != 0 && c->a_bits != 4 && c->a_bits != 6 && c->a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (supported: 0, 4, 6, 8)", c->a_bits);
-    if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT && c->gemm_impl != ZOQAT_GEMM_TCGEN05_1CTA) return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
+    if (c->gemm_impl != ZOQAT_GEMM_TCGEN05 && c->gemm_impl != ZOQAT_GEMM_SIMT && c->gemm_impl != ZOQAT_GEMM_TCGEN05_1CTA &&
+        c->gemm_impl != ZOQAT_GEMM_TCGEN05_I8)
+        return fail(ZOQAT_ERR_INVALID_ARG, "unknown gemm_impl %d", c->gemm_impl);
+    if (c->gemm_impl == ZOQAT_GEMM_TCGEN05_I8 && (c->w_group != 0 || c->a_bits == 0 || c->w_bits > 7))
+        return fail(ZOQAT_ERR_UNSUPPORTED, "the 8-bit integer GEMM needs one weight group per output row (w_group 0), quantised activations and w_bits <= 7");
     if ((int64_t)c->max_batch * c->max_seq > (1 << 24)) return fail(ZOQAT_ERR_UNSUPPORTED, "max_batch*max_seq too large");
     return ZOQAT_OK;
 }
@@ -254,6 +260,9 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
     ProfScope ps(m, ZOQAT_PROF_GEMM, s);
     g.err_flag = m->ws.err_flag;
     g.single_cta = m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_1CTA;
+    if (m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_I8 && g.mode != 1) {     // every block linear; the vocabulary projection stays bf16
+        g.int8 = 1; g.col_step = m->ws.col_step; g.col_stride = (size_t)m->ws.bias_ld;
+    }
     const int rc = (m->cfg.gemm_impl == ZOQAT_GEMM_SIMT) ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "GEMM launch rejected (M=%lld N=%lld K=%lld)", (long long)g.M, (long long)g.N, (long long)g.K);
     return ZOQAT_OK;
@@ -266,11 +275,19 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
 // NULL).  Adaptive tensors read the parameters forward() prepared for block linear `role`.
 void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t pass_stride, int passes,
                      uint64_t seed, float eps, cudaStream_t s, bool smoothing = false, size_t bias_off = 0,
-                     const float* bias0 = nullptr, int role = 0, int point = 0, const PendingUpdate* pend = nullptr) {
+                     const float* bias0 = nullptr, int role = 0, int point = 0, const PendingUpdate* pend = nullptr,
+                     bool i8 = false) {
     ProfScope ps(m, ZOQAT_PROF_WEIGHT, s);
     const int64_t n = L.rows * L.cols;
     const int bits = L.bits(m->cfg.w_bits);
     const bool per_channel = m->cfg.w_group == 0 && bits != 0;
+    if (i8) {
+        // signed bytes at the same element offsets: dst and the pass stride count bytes; the steps of this linear's
+        // output columns sit where its bias does (bias_off)
+        uint8_t* base = reinterpret_cast<uint8_t*>(m->ws.bop) + (dst - m->ws.bop);
+        dst = reinterpret_cast<__nv_bfloat16*>(base);
+        pass_stride /= 2;                             // added to a bf16 pointer below
+    }
     if (smoothing || per_channel || (L.adaptive() && bits != 0)) {
         LearnedOperandArgs a{};
         a.w = L.w; a.rows = L.rows; a.cols = L.cols; a.group = m->cfg.w_group ? m->cfg.w_group : 128; a.bits = bits;
@@ -287,6 +304,7 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
             a.bias_out = m->ws.bias_pm + bias_off; a.bias_out_stride = m->ws.bias_ld;
         }
         a.pend = (passes == 2 && L.trainable()) ? pend : nullptr;
+        if (i8) { a.i8 = 1; a.col_step = m->ws.col_step + bias_off; a.col_stride = m->ws.bias_ld; a.err_flag = m->ws.err_flag; }
         launch_weight_operand_learned(a, s);
         return;
     }
@@ -343,6 +361,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     const bool llama = c.arch == ZOQAT_ARCH_LLAMA;
     const int norm_kind = llama ? 1 : 2;
     const size_t ps = w.bop_elems;
+    const bool i8 = c.gemm_impl == ZOQAT_GEMM_TCGEN05_I8;      // block linears on signed bytes (pair kernel otherwise as 0)
+    const bool pair = c.gemm_impl == ZOQAT_GEMM_TCGEN05 || i8;
+    const int planes = i8 ? 2 : 0;
     if (m->cap) {
         const size_t need = capture_forward_bytes(m, T, passes);
         if (need > m->cap_bytes) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "capture buffer %zu < %zu bytes", m->cap_bytes, need);
@@ -398,11 +419,11 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         // --- attention block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(0));
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(0), false, planes);
           capture_finish(m, nullptr, R, d, s); }
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
             produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
-                            Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend);
+                            Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend, i8);
         GemmArgs g{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = llama ? nullptr : w.bias_qkv + (size_t)l * 3 * d;
@@ -410,7 +431,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         g.out = w.qkv; g.b_stride = ps;
         // on the pair kernel the epilogue of this GEMM writes the attention operands itself (rotary embedding, q
         // scaling, binary16 hi / lo split, v transposed): q | k | v never exist as fp32 and no preparation kernel runs
-        const bool fuse_qkv = c.gemm_impl == ZOQAT_GEMM_TCGEN05 && d % 256 == 0 && seq % 32 == 0;
+        const bool fuse_qkv = pair && d % 256 == 0 && seq % 32 == 0;
         if (fuse_qkv) {
             g.mode = 2; g.out = nullptr;
             g.att = attention_tc_operands(w.attn_scratch, Z * batch, seq, H, dh);
@@ -426,9 +447,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
               return fail(rc, "attention launch rejected");
           } }
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
-          launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1));
+          launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1), false, planes);
           capture_finish(m, w.att, R, d, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
@@ -437,18 +458,18 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         // --- feed-forward block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_FFN_NORM_G], Ly.vec[ZOQAT_ROLE_FFN_NORM_B],
-                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(2));
+                                  c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(2), false, planes);
           capture_finish(m, nullptr, R, d, s); }
         const int n_up = llama ? 2 * F : F;
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend);
-        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend, i8);
+        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         // SiLU-gated FFN on the pair kernel: the epilogue multiplies silu(gate) by up and collects the row maxima,
         // so the intermediate is half as wide and the quantiser that follows needs a single pass
-        const bool fuse_gate = llama && c.gemm_impl == ZOQAT_GEMM_TCGEN05 && F % 128 == 0 && F <= 16384;
+        const bool fuse_gate = llama && pair && F % 128 == 0 && F <= 16384;
         if (fuse_gate) {
             cudaMemsetAsync(w.row_amax, 0, (size_t)R * 4, s);
             g.mode = 3; g.row_amax = w.row_amax;
@@ -456,11 +477,11 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
-          if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(3));
-          else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s);
-          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3), false, false, capture_input(m));
+          if (fuse_gate && smo) launch_norm_act_operand(w.ffn, R, F, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(3), false, planes);
+          else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s, planes);
+          else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3), false, planes, capture_input(m));
           capture_finish(m, fuse_gate ? w.ffn : nullptr, R, F, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend);
+        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
@@ -719,6 +740,12 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
         }
         if (Ly.smoothing) m->any_learnable = true;
         for (int r = 0; r < 7; ++r) if (Ly.lin[r].adaptive()) m->any_learnable = true;
+        if (cfg->gemm_impl == ZOQAT_GEMM_TCGEN05_I8)
+            for (int r = 0; r < 7; ++r)
+                if (Ly.lin[r].present && (Ly.lin[r].bits(cfg->w_bits) == 0 || Ly.lin[r].packed_frozen())) {
+                    delete m;
+                    return fail(ZOQAT_ERR_UNSUPPORTED, "layer %d: the 8-bit integer GEMM needs every block linear QUANTIZED and not FROZEN_PACKED", l);
+                }
     }
     // one-time tables: rotary cos/sin (evaluated in double, stored fp32) and concatenated q|k|v biases
     if (llama) {
@@ -1019,6 +1046,7 @@ int zoqat_check(zoqat_model_t* m, void* stream) {
     if (flag != 0) {
         cudaMemsetAsync(m->ws.err_flag, 0, 4, s);
         if (flag == kErrBadLabel) return fail(ZOQAT_ERR_INVALID_ARG, "a label is >= vocab (its position was given loss 0)");
+        if (flag == kErrCodeRange) return fail(ZOQAT_ERR_UNSUPPORTED, "8-bit integer GEMM: a weight row's code minus zero point left [-128, 127]");
         return fail(ZOQAT_ERR_TIMEOUT, "device wait ran out (code %d)", flag);
     }
     return ZOQAT_OK;
@@ -1133,10 +1161,11 @@ int zoqat_op_weight_operand_pair(const float* w_dev, int64_t rows, int64_t cols,
     return ZOQAT_OK;
 }
 
-int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
-                                    uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
-                                    const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
-                                    void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
+static int op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
+                                     uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
+                                     const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
+                                     void* operand_minus_dev, uint8_t* codes_dev, void* stream, float* col_step_dev,
+                                     int32_t* err_flag_dev) {
     if (!generator_table_ready()) return fail(ZOQAT_ERR_CUDA, "upload of the direction generator's table failed");
     if (!scratch_dev || (reinterpret_cast<uintptr_t>(scratch_dev) & 15)) return fail(ZOQAT_ERR_INVALID_ARG, "scratch_dev must be 16-byte aligned device memory");
     if (int rc = check_group_bits(rows, cols, group, bits, true, 8, true)) return rc;
@@ -1155,9 +1184,30 @@ int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t co
     a.prep = scratch_dev;
     a.bias_part = scratch_dev + 16 * (rows * cols / a.group); a.bias0 = bias0_dev; a.bias_out = bias_dev; a.bias_out_stride = rows;
     a.codes = codes_dev;
+    if (col_step_dev) { a.i8 = 1; a.col_step = col_step_dev; a.col_stride = rows; a.err_flag = err_flag_dev; }
     launch_weight_operand_learned(a, static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
+}
+
+int zoqat_op_weight_operand_learned(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, uint64_t seed,
+                                    uint32_t tensor_id, float eps, const float* theta_dev, const float* smooth_dev,
+                                    const float* bias0_dev, float* bias_dev, float* scratch_dev, void* operand_plus_dev,
+                                    void* operand_minus_dev, uint8_t* codes_dev, void* stream) {
+    return op_weight_operand_learned(w_dev, rows, cols, group, bits, seed, tensor_id, eps, theta_dev, smooth_dev, bias0_dev, bias_dev,
+                                     scratch_dev, operand_plus_dev, operand_minus_dev, codes_dev, stream, nullptr, nullptr);
+}
+
+int zoqat_op_weight_operand_i8(const float* w_dev, int64_t rows, int64_t cols, int bits, uint64_t seed, uint32_t tensor_id,
+                               float eps, const float* theta_dev, const float* smooth_dev, const float* bias0_dev,
+                               float* bias_dev, float* scratch_dev, void* operand_plus_dev, void* operand_minus_dev,
+                               float* col_step_dev, int32_t* err_flag_dev, void* stream) {
+    if (!col_step_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "col_step_dev/err_flag_dev are NULL");
+    if (bits < 2 || bits > 7) return fail(ZOQAT_ERR_UNSUPPORTED, "bits %d (2..7: code minus zero point must fit a signed byte)", bits);
+    if ((reinterpret_cast<uintptr_t>(operand_plus_dev) | reinterpret_cast<uintptr_t>(operand_minus_dev)) & 15)
+        return fail(ZOQAT_ERR_INVALID_ARG, "operands must be 16-byte aligned");
+    return op_weight_operand_learned(w_dev, rows, cols, 0, bits, seed, tensor_id, eps, theta_dev, smooth_dev, bias0_dev, bias_dev,
+                                     scratch_dev, operand_plus_dev, operand_minus_dev, nullptr, stream, col_step_dev, err_flag_dev);
 }
 
 int zoqat_op_smooth_perturb(const float* scale_dev, const float* shift_dev, int64_t cols, uint64_t seed, uint32_t scale_id,
@@ -1245,6 +1295,20 @@ int zoqat_op_norm_act_operand(const float* x_dev, int64_t rows, int64_t cols, in
     return ZOQAT_OK;
 }
 
+int zoqat_op_norm_act_operand_i8(const float* x_dev, int64_t rows, int64_t cols, int norm_kind, const float* gain_dev,
+                                 const float* bias_dev, float norm_eps, int a_bits, void* operand_dev, float* row_step_dev,
+                                 void* stream) {
+    if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (rows <= 0 || cols <= 0 || cols % 4 || cols > 32768) return fail(ZOQAT_ERR_UNSUPPORTED, "cols must be a multiple of 4, at most 32768");
+    if (norm_kind < 0 || norm_kind > 2 || (norm_kind >= 1 && !gain_dev) || (norm_kind == 2 && !bias_dev)) return fail(ZOQAT_ERR_INVALID_ARG, "bad norm arguments");
+    if (a_bits != 4 && a_bits != 6 && a_bits != 8) return fail(ZOQAT_ERR_UNSUPPORTED, "a_bits %d (4, 6 or 8)", a_bits);
+    launch_norm_act_operand(x_dev, rows, (int)cols, norm_kind, gain_dev, bias_dev, norm_eps, a_bits,
+                            static_cast<__nv_bfloat16*>(operand_dev), row_step_dev, nullptr, static_cast<cudaStream_t>(stream),
+                            SmoothAct(), false, 2);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
 int zoqat_op_ffn_act_operand(const float* x_dev, int64_t rows, int64_t cols, int gated, int a_bits, void* operand_dev,
                              float* row_step_dev, void* stream) {
     if (!x_dev || !operand_dev || !row_step_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
@@ -1284,6 +1348,26 @@ int zoqat_op_gemm_silu_gate(const void* a_dev, const void* b_dev, int64_t M, int
     g.b_stride = (size_t)2 * F * K; g.mode = 3; g.row_amax = row_amax_dev;
     const int rc = launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "gated GEMM rejected: M=%lld F=%lld K=%lld (K %% 8 == 0, 16-byte aligned pointers)", (long long)M, (long long)F, (long long)K);
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
+int zoqat_op_gemm_i8(const void* a_dev, const void* b_dev, int64_t M, int64_t N, int64_t K, const float* row_step_dev,
+                     const float* col_step_dev, const float* bias_dev, int accumulate, int gated, float* out_dev,
+                     uint32_t* row_amax_dev, int32_t* err_flag_dev, void* stream) {
+    if (!a_dev || !b_dev || !out_dev || !col_step_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (M <= 0 || N <= 0 || K <= 0 || K % 16 || N % 32) return fail(ZOQAT_ERR_UNSUPPORTED, "needs K %% 16 == 0 and N %% 32 == 0");
+    if (gated && (N % 256 || !row_amax_dev || accumulate)) return fail(ZOQAT_ERR_UNSUPPORTED, "gated: N = 2 F with F %% 128 == 0, row_amax_dev given, no accumulation");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (gated) CUDA_TRY(cudaMemsetAsync(row_amax_dev, 0, (size_t)M * 4, s));
+    GemmArgs g{};
+    g.A = static_cast<const __nv_bfloat16*>(a_dev); g.B = static_cast<const __nv_bfloat16*>(b_dev);
+    g.M = M; g.N = N; g.K = K; g.Z = 1; g.row_step = row_step_dev; g.bias = bias_dev; g.accumulate = accumulate;
+    g.out = out_dev; g.err_flag = err_flag_dev; g.b_stride = (size_t)N * K;
+    g.int8 = 1; g.col_step = col_step_dev; g.col_stride = (size_t)N;
+    if (gated) { g.mode = 3; g.row_amax = row_amax_dev; }
+    const int rc = launch_gemm_tc(g, s);
+    if (rc != ZOQAT_OK) return fail(rc, "8-bit GEMM rejected: M=%lld N=%lld K=%lld (16-byte aligned pointers)", (long long)M, (long long)N, (long long)K);
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }

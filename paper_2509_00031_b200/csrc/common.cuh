@@ -12,6 +12,7 @@ constexpr int kErrWaitFull = 1;      // MMA warp: operands never arrived
 constexpr int kErrWaitEmpty = 2;     // TMA warp: stage never released
 constexpr int kErrWaitAccFull = 3;   // epilogue: accumulator never committed
 constexpr int kErrWaitAccEmpty = 4;  // MMA warp: accumulator never drained
+constexpr int kErrCodeRange = 32;    // 8-bit operands: a weight code minus its zero point does not fit a signed byte
 constexpr int kErrBadLabel = 16;     // cross-entropy: a label >= vocab (not a wait; the position's loss is reported as 0)
 
 // Per-device one-time set-up (function attributes, cached device properties): true the first time it is called with this
@@ -111,6 +112,9 @@ struct LearnedOperandArgs {
     float* bias_part; const float* bias0; float* bias_out; int64_t bias_out_stride;
     uint8_t* codes;
     const PendingUpdate* pend;    // with op_minus only: the previous step's update, applied to the master on the way in
+    // per_channel with bits != 0 only: the operands are signed bytes (code - zero point, rows of `cols` bytes at op_plus /
+    // op_minus) and the steps go to col_step[sign * col_stride + row]; err_flag receives kErrCodeRange if a row does not fit
+    int i8; float* col_step; int64_t col_stride; int32_t* err_flag;
 };
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s);
 void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* theta, cudaStream_t s);
@@ -133,18 +137,20 @@ void launch_embed(const int32_t* tokens, const float* embed, const float* pos, i
 // Smoothing of Section 4.2 on the activation side (smooth may be NULL): the quantiser sees (x - shift') * (1 / scale')
 // with the vectors of launch_smooth_perturb; rows [0, rows_per_pass) use sign 0, the rest sign 1.
 struct SmoothAct { const float* smooth = nullptr; int ld = 0; int64_t rows_per_pass = 0; };
-// planes = true (a_bits != 0, cols % 32 == 0): the operand row holds, instead of bf16 codes, the integer form the
+// planes = 1 (a_bits != 0, cols % 32 == 0): the operand row holds, instead of bf16 codes, the integer form the
 // decode-time matrix-vector kernels read (int8 codes of even columns, of odd columns, int32 sums of every 32 codes).
+// planes = 2 (a_bits != 0, cols % 4 == 0): the codes as signed bytes, row r at byte r * cols of op (the A operand of the
+// 8-bit integer GEMM).
 void launch_norm_act_operand(const float* x, int64_t rows, int cols, int norm_kind, const float* gain, const float* bias,
                              float norm_eps, int a_bits, __nv_bfloat16* op, float* row_step, float* normed, cudaStream_t s,
-                             SmoothAct sm = SmoothAct(), bool dependent = false, bool planes = false);
+                             SmoothAct sm = SmoothAct(), bool dependent = false, int planes = 0);
 // pre (may be NULL): fp32 [rows, cols], receives the value the quantiser sees (parity hook).
 void launch_ffn_act_operand(const float* x, int64_t rows, int cols, int gated, int a_bits,
                             __nv_bfloat16* op, float* row_step, cudaStream_t s, SmoothAct sm = SmoothAct(),
-                            bool dependent = false, bool planes = false, float* pre = nullptr);
+                            bool dependent = false, int planes = 0, float* pre = nullptr);
 // Activation operand of rows whose max |x| is already known (amax: bits of a non-negative float per row).
 void launch_rows_operand(const float* x, int64_t rows, int cols, const uint32_t* amax, int a_bits,
-                         __nv_bfloat16* op, float* row_step, cudaStream_t s);
+                         __nv_bfloat16* op, float* row_step, cudaStream_t s, int planes = 0);
 // fp32 CUDA-core attention (cross-check) and the tensor-core attention (needs scratch and an error word).
 void launch_attention(const float* qkv, int batch, int seq, int n_heads, int d_head,
                       const float* cos_t, const float* sin_t, float* out, cudaStream_t s);
@@ -179,7 +185,11 @@ void launch_decode_argmax(const float* logits, int batch, int V, int32_t* next, 
 struct GemmArgs {
     const __nv_bfloat16* A;   // [Z*M, K]
     const __nv_bfloat16* B;   // [Z][N, K], pass z starts at B + z*b_stride
-    size_t b_stride;          // elements between the B matrices of consecutive passes (multiple of 8)
+    size_t b_stride;          // elements between the B matrices of consecutive passes (multiple of 8; of 16 with int8)
+    int int8;                 // 1 (tcgen05 pair kernel only, modes 0 / 2 / 3): A and B hold signed 8-bit integers instead of
+                              // bf16 (K % 16 == 0, N % 32 == 0); the exact integer sums are scaled by col_step, then row_step
+    const float* col_step;    // int8: [Z][col_stride] step of every output column (16-byte aligned, col_stride % 4 == 0)
+    size_t col_stride;
     int64_t M, N, K;
     int Z;
     const float* row_step;    // [Z*M] or NULL

@@ -15,6 +15,11 @@
 // Two accumulators (2*BN of the 512 TMEM columns) let the epilogue of tile i
 // overlap the MMAs of tile i+1.
 //
+// I8 (pair kernel only): A and B hold signed 8-bit integers - activation codes and weight codes minus their zero
+// point, one weight step per output row - multiplied by tcgen05.mma kind::i8 into exact 32-bit sums (128 of them per
+// 128-byte swizzle row, so a stage covers twice the depth); the epilogue converts a sum once, multiplies by the step
+// of its output column (col_step) and then by the row step:  out = row_step * (col_step * sum a (c - z)) (+ bias).
+//
 // Every wait is bounded: a wait that runs out records a code in *err_flag and
 // the role leaves its loop; the CTA then drains, frees its TMEM and returns.
 #include "common.cuh"
@@ -26,8 +31,8 @@ namespace zq {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
-constexpr int UMMA_K = 16;
+constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row (128 int8)
+constexpr int UMMA_K = 16;             // 32 bytes of the row per MMA: 16 bf16 or 32 int8
 constexpr int kThreadsTC = 192;
 
 // CG = CTAs per tile: 1, or 2 (a cluster of two CTAs on an SM pair computes a 256 x BN tile with one
@@ -53,10 +58,35 @@ __device__ __forceinline__ uint32_t idesc_bf16() {
          | ((uint32_t)((BM * CG) >> 4) << 24); // M / 16
 }
 
+// Instruction descriptor, kind::i8: 32-bit integer accumulate, signed 8-bit A and B, both K-major.
+template <int BN, int CG>
+__device__ __forceinline__ uint32_t idesc_s8() {
+    return (2u << 4)                           // D format: s32
+         | (1u << 7)                           // A format: signed 8-bit
+         | (1u << 10)                          // B format: signed 8-bit
+         | ((uint32_t)(BN >> 3) << 17)         // N / 8
+         | ((uint32_t)((BM * CG) >> 4) << 24); // M / 16
+}
+
+// accumulator word -> fp32 value: the bits themselves (f16 kind) or col_step * (float)sum (i8 kind)
+template <bool I8>
+__device__ __forceinline__ float acc_value(uint32_t v, float cs) {
+    return I8 ? __fmul_rn(__int2float_rn((int)v), cs) : __uint_as_float(v);
+}
+
+// four consecutive column steps (16-byte aligned: column a multiple of 4), or ones when the kind has none
+template <bool I8>
+__device__ __forceinline__ float4 col_steps4(const float* csb, int64_t n) {
+    return I8 ? __ldg(reinterpret_cast<const float4*>(csb + n)) : make_float4(1.f, 1.f, 1.f, 1.f);
+}
+__device__ __forceinline__ float pick4(const float4& v, int i) { return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w)); }
+
 struct TcParams {
     int64_t M, N, K;
     int Z;
     const float* row_step;
+    const float* col_step;    // I8: [Z][col_stride] step of every output column
+    int64_t col_stride;
     const float* bias;
     int64_t bias_stride;      // elements between the bias vectors of consecutive passes (0: shared)
     int relu, accumulate;
@@ -106,7 +136,7 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int r, int& tm, i
     }
 }
 
-template <int BN, int CG>
+template <int BN, int CG, bool I8>
 __global__ void __launch_bounds__(kThreadsTC, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ AttMaps att, TcParams p) {
@@ -130,7 +160,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t* tmem_slot_ptr = reinterpret_cast<uint32_t*>(smem_raw + (tmem_slot - raw));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_kb = (int)((p.K + BK - 1) / BK);
+    constexpr int KB = I8 ? 2 * BK : BK;                         // elements per 128-byte row of a stage
+    const int num_kb = (int)((p.K + KB - 1) / KB);
     const int tiles_per_z = p.tiles_m * p.tiles_n;
     const int total_tiles = tiles_per_z * p.Z;
 
@@ -170,14 +201,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         // both CTAs' bytes are counted on the leader's barrier, which expects them all
                         if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * Cfg::kStageBytes);
                         const uint32_t lead_full = mapa_shared(full_bar(stage), 0);
-                        tma_load_3d_pair_hint(a_dst, &map_a, lead_full, kb * BK, tm * TM + (int)rank * BM, z, pol_a);
+                        tma_load_3d_pair_hint(a_dst, &map_a, lead_full, kb * KB, tm * TM + (int)rank * BM, z, pol_a);
                         // mode 3: the tile's first 128 columns are gate features, the last 128 the matching up features
                         const int b_row = p.mode == 3 ? (int)rank * (int)(p.N / 2) + tn * (BN / 2) : tn * BN + (int)rank * (BN / 2);
-                        tma_load_3d_pair_hint(a_dst + Cfg::kABytes, &map_b, lead_full, kb * BK, b_row, z, pol_b);
+                        tma_load_3d_pair_hint(a_dst + Cfg::kABytes, &map_b, lead_full, kb * KB, b_row, z, pol_b);
                     } else {
                         mbar_arrive_expect_tx(full_bar(stage), Cfg::kStageBytes);
-                        tma_load_3d_hint(a_dst, &map_a, full_bar(stage), kb * BK, tm * BM, z, pol_a);
-                        tma_load_3d_hint(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * BK, tn * BN, z, pol_b);
+                        tma_load_3d_hint(a_dst, &map_a, full_bar(stage), kb * KB, tm * BM, z, pol_a);
+                        tma_load_3d_hint(a_dst + Cfg::kABytes, &map_b, full_bar(stage), kb * KB, tn * BN, z, pol_b);
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -193,7 +224,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0 && rank == 0) {
-            const uint32_t idesc = idesc_bf16<BN, CG>();
+            const uint32_t idesc = I8 ? idesc_s8<BN, CG>() : idesc_bf16<BN, CG>();
             int stage = 0; uint32_t phase = 0;
             int acc = 0; uint32_t acc_phase = 0;
             bool ok = true;
@@ -209,8 +240,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint64_t b_desc = smem_desc_sw128(a_addr + Cfg::kABytes);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advance 16 elements = 32 bytes inside the swizzled row: +2 in the (addr/16) field
-                        if (CG == 2) umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                        // advance 32 bytes inside the swizzled row: +2 in the (addr/16) field
+                        if (I8) umma_s8_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                             (kb > 0 || k > 0) ? 1u : 0u);
+                        else if (CG == 2) umma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                                     (kb > 0 || k > 0) ? 1u : 0u);
                         else umma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                        (kb > 0 || k > 0) ? 1u : 0u);
@@ -249,7 +282,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             float ce_m = -INFINITY, ce_s = 0.0f;
             const int32_t lab = (p.mode == 1 && row_ok) ? p.labels[m] : -1;
             const float* bias = p.bias ? p.bias + (int64_t)z * p.bias_stride : nullptr;
-            (void)lab;
+            const float* csb = I8 ? p.col_step + (int64_t)z * p.col_stride : nullptr;      // column steps of this pass
+            (void)lab; (void)csb;
             if (p.mode == 2) {
                 // q | k | v projection: rotary embedding, q scaling, hi / lo split and the layouts of the attention kernel,
                 // written from here so that q | k | v never exist as fp32 in memory.  A warp's 32 rows are 32 consecutive
@@ -293,13 +327,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                                 for (int j = 0; j < 32; j += 8) {
                                     uint32_t w[4][4];       // [lo-half hi, lo-half lo, hi-half hi, hi-half lo][4 x half2]
+                                    const float4 ca0 = col_steps4<I8>(csb, n_lo + j), ca1 = col_steps4<I8>(csb, n_lo + j + 4);
+                                    const float4 cb0 = col_steps4<I8>(csb, n_lo + hd + j), cb1 = col_steps4<I8>(csb, n_lo + hd + j + 4);
 #pragma unroll
                                     for (int e = 0; e < 8; e += 2) {
                                         __half h[4][2];
 #pragma unroll
                                         for (int u = 0; u < 2; ++u) {
-                                            float a = rs * __uint_as_float(va[j + e + u]);
-                                            float b = rs * __uint_as_float(vb[j + e + u]);
+                                            float a = rs * acc_value<I8>(va[j + e + u], pick4(e < 4 ? ca0 : ca1, (e + u) & 3));
+                                            float b = rs * acc_value<I8>(vb[j + e + u], pick4(e < 4 ? cb0 : cb1, (e + u) & 3));
                                             if (bias) { a += bias[n_lo + j + e + u]; b += bias[n_lo + hd + j + e + u]; }
                                             float lo = a, hi = b;
                                             if (p.cos_t) {
@@ -343,9 +379,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             if (lane == 0) bulk_wait_read_1();
                             __syncwarp();
                             const int64_t n0 = n_base + c * 32;
+                            float4 c4 = make_float4(1.f, 1.f, 1.f, 1.f);
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                float x = rs * __uint_as_float(v[j]);
+                                if ((j & 3) == 0) c4 = col_steps4<I8>(csb, n0 + j);
+                                float x = rs * acc_value<I8>(v[j], pick4(c4, j & 3));
                                 if (bias) x += bias[n0 + j];
                                 __half h, l;
                                 split_half(x, h, l);
@@ -391,10 +429,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             bu = *reinterpret_cast<const float4*>(bias + p.N / 2 + f0 + j);
                         }
                         const float bgs[4] = {bg.x, bg.y, bg.z, bg.w}, bus[4] = {bu.x, bu.y, bu.z, bu.w};
+                        const float4 cg = col_steps4<I8>(csb, f0 + j), cu = col_steps4<I8>(csb, p.N / 2 + f0 + j);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float g = rs * __uint_as_float(vg[j + e]) + bgs[e];
-                            const float u = rs * __uint_as_float(vu[j + e]) + bus[e];
+                            const float g = rs * acc_value<I8>(vg[j + e], pick4(cg, e)) + bgs[e];
+                            const float u = rs * acc_value<I8>(vu[j + e], pick4(cu, e)) + bus[e];
                             a4[e] = __fdiv_rn(g, 1.0f + expf(-g)) * u;
                             amax = fmaxf(amax, fabsf(a4[e]));
                         }
@@ -430,8 +469,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         float4 x;
-                        x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
-                        x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
+                        const float4 c4 = col_steps4<I8>(csb, n0 + j);         // I8: N % 32 == 0, the chunk is whole
+                        x.x = rs * acc_value<I8>(v[j], c4.x);     x.y = rs * acc_value<I8>(v[j + 1], c4.y);
+                        x.z = rs * acc_value<I8>(v[j + 2], c4.z); x.w = rs * acc_value<I8>(v[j + 3], c4.w);
                         if (bias) {
                             if (full) {
                                 const float4 b = *reinterpret_cast<const float4*>(bias + n0 + j);
@@ -463,8 +503,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 x;
-                            x.x = rs * __uint_as_float(v[j]);     x.y = rs * __uint_as_float(v[j + 1]);
-                            x.z = rs * __uint_as_float(v[j + 2]); x.w = rs * __uint_as_float(v[j + 3]);
+                            const float4 c4 = col_steps4<I8>(csb, n0 + j);
+                            x.x = rs * acc_value<I8>(v[j], c4.x);     x.y = rs * acc_value<I8>(v[j + 1], c4.y);
+                            x.z = rs * acc_value<I8>(v[j + 2], c4.z); x.w = rs * acc_value<I8>(v[j + 3], c4.w);
                             if (bias) {
                                 const float4 b = *reinterpret_cast<const float4*>(bias + n0 + j);
                                 x.x += b.x; x.y += b.y; x.z += b.z; x.w += b.w;
@@ -479,7 +520,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else {
                         for (int j = 0; j < 32; ++j) {
                             if (n0 + j >= p.N) break;
-                            float x = rs * __uint_as_float(v[j]);
+                            float x = rs * acc_value<I8>(v[j], I8 ? __ldg(csb + n0 + j) : 1.0f);
                             if (bias) x += bias[n0 + j];
                             if (p.relu) x = fmaxf(x, 0.f);
                             if (p.accumulate) x += o[j];
@@ -491,7 +532,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     float x[32], cm = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        x[j] = (n0 + j < p.N) ? rs * __uint_as_float(v[j]) : -INFINITY;
+                        x[j] = (n0 + j < p.N) ? rs * acc_value<I8>(v[j], I8 ? __ldg(csb + n0 + j) : 1.0f) : -INFINITY;
                         cm = fmaxf(cm, x[j]);
                         if (n0 + j == lab) p.label_logit[row] = x[j];
                     }
@@ -545,16 +586,17 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 3-D map over a [Z][rows][K] bf16 array (K innermost), box = 64 x box_rows x 1, 128-byte swizzle,
+// 3-D map over a [Z][rows][K] bf16 (or 8-bit) array (K innermost), box = 128 bytes x box_rows x 1, 128-byte swizzle,
 // out-of-range elements read as zero.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int Z, size_t z_stride_elems, int box_rows) {
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int Z, size_t z_stride_elems, int box_rows, bool bytes8 = false) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const cuuint64_t esz = bytes8 ? 1 : 2;
     const cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)Z};
-    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)z_stride_elems * 2};
-    const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * esz, (cuuint64_t)z_stride_elems * esz};
+    const cuuint32_t box[3] = {(cuuint32_t)(bytes8 ? 2 * BK : BK), (cuuint32_t)box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+    return fn(map, bytes8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -607,10 +649,10 @@ int num_sms() {
 // (fewest distinct strips per wave) and the operands keep the default priority.
 struct TileOrder { int group, group_n, hint_a, hint_b, hint_out; };
 
-TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows, int units) {
+TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n, int tm_rows, int tn_rows, int units, int esz) {
     const double resident = 36.0 * 1048576.0;
-    const double a_bytes = (double)M * K * 2, b_bytes = (double)N * K * 2;
-    const double strip_a = (double)tm_rows * K * 2, strip_b = (double)tn_rows * K * 2;
+    const double a_bytes = (double)M * K * esz, b_bytes = (double)N * K * esz;
+    const double strip_a = (double)tm_rows * K * esz, strip_b = (double)tn_rows * K * esz;
     auto even = [](int tiles, int g) {
         if (g < 1) g = 1;
         if (g > tiles) g = tiles;
@@ -643,16 +685,17 @@ TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n
     return o;
 }
 
-template <int BN, int CG>
+template <int BN, int CG, bool I8 = false>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
     using Cfg = TileCfg<BN, CG>;
     alignas(64) CUtensorMap map_a, map_b, map_out;
     alignas(64) AttMaps att;
     const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
-    if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN / CG))
+    if (!make_map(&map_a, a.A, a.M, a.K, a.Z, (size_t)a.M * a.K, BM, I8) || !make_map(&map_b, a.B, a.N, a.K, a.Z, b_stride, BN / CG, I8))
         return ZOQAT_ERR_CUDA;
     TcParams p;
     p.M = a.M; p.N = a.N; p.K = a.K; p.Z = a.Z;
+    p.col_step = a.col_step; p.col_stride = (int64_t)a.col_stride;
     p.row_step = a.row_step; p.bias = a.bias; p.bias_stride = (int64_t)a.bias_stride; p.relu = a.relu; p.accumulate = a.accumulate;
     p.out = a.out; p.mode = a.mode; p.labels = a.labels; p.partials = a.partials; p.label_logit = a.label_logit;
     p.err_flag = a.err_flag;
@@ -687,13 +730,13 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     }
     static DeviceOnce attr;
     if (attr.first() &&
-        cudaFuncSetAttribute(gemm_tc_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
+        cudaFuncSetAttribute(gemm_tc_kernel<BN, CG, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess) {
         attr.retry();
         return ZOQAT_ERR_CUDA;
     }
     const int units = num_sms() / CG;                      // persistent CTAs (CG = 1) or CTA pairs (CG = 2)
     {
-        const TileOrder o = choose_order(a.M, a.N, a.K, p.tiles_m, p.tiles_n, BM * CG, BN, units);
+        const TileOrder o = choose_order(a.M, a.N, a.K, p.tiles_m, p.tiles_n, BM * CG, BN, units, I8 ? 1 : 2);
         p.group = o.group; p.group_n = o.group_n; p.hint_a = o.hint_a; p.hint_b = o.hint_b; p.hint_out = o.hint_out;
     }
     const int64_t total = (int64_t)p.tiles_m * p.tiles_n * a.Z;
@@ -708,7 +751,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, CG>, map_a, map_b, map_out, att, p) != cudaSuccess) return ZOQAT_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, CG, I8>, map_a, map_b, map_out, att, p) != cudaSuccess) return ZOQAT_ERR_CUDA;
     count_launch();
     return ZOQAT_OK;
 }
@@ -718,12 +761,20 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
 int launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
     if (a.M <= 0 || a.N <= 0 || a.K <= 0 || a.Z <= 0) return ZOQAT_ERR_INVALID_ARG;
     if (a.K % 8 != 0 || a.err_flag == nullptr || (a.Z > 1 && (a.b_stride % 8 != 0 || a.b_stride < (size_t)a.N * a.K))) return ZOQAT_ERR_INVALID_ARG;
+    if (a.int8) {
+        // signed 8-bit operands: pair kernel only, whole 32-column chunks, one step per output column
+        if (a.single_cta || a.mode == 1) return ZOQAT_ERR_UNSUPPORTED;
+        if (a.K % 16 != 0 || a.N % 32 != 0 || !a.col_step || a.col_stride % 4 != 0 || (a.Z > 1 && a.b_stride % 16 != 0) ||
+            (reinterpret_cast<uintptr_t>(a.col_step) & 15))
+            return ZOQAT_ERR_INVALID_ARG;
+    }
     if (a.bias_stride % 4 != 0) return ZOQAT_ERR_INVALID_ARG;      // the epilogue reads the bias with 16-byte loads
     if ((reinterpret_cast<uintptr_t>(a.A) | reinterpret_cast<uintptr_t>(a.B) | reinterpret_cast<uintptr_t>(a.out) |
          reinterpret_cast<uintptr_t>(a.bias)) & 15)
         return ZOQAT_ERR_INVALID_ARG;
     // the cross-entropy epilogue always uses 256-column tiles (gemm_ce_tiles)
     if ((a.mode == 3 || a.mode == 2) && a.single_cta) return ZOQAT_ERR_UNSUPPORTED;
+    if (a.int8) return launch_tc<256, 2, true>(a, s);
     if (a.mode != 0 || a.N > 128) return a.single_cta ? launch_tc<256, 1>(a, s) : launch_tc<256, 2>(a, s);
     return launch_tc<128, 1>(a, s);
 }

@@ -304,6 +304,24 @@ __device__ __forceinline__ void quantise16_folded(float (&x)[16], const float4& 
     for (int j = 0; j < 16; ++j) x[j] = __fmul_rn(fminf(fmaxf(rintf(__fmul_rn(x[j], a.y)), a.z), a.w), a.x);
 }
 
+// Integer form: the code minus its zero point, clamp(round(x * inv), lo - z, hi - z), left as it is (no step).
+__device__ __forceinline__ void quantise16_integer(float (&x)[16], const float4& a) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) x[j] = fminf(fmaxf(rintf(__fmul_rn(x[j], a.y)), a.z), a.w);
+}
+
+// Four integer-valued floats in [-128, 127] -> four signed bytes, first value in the low byte.
+__device__ __forceinline__ uint32_t pack_s8x4(float a, float b, float c, float d) {
+    return ((uint32_t)__float2int_rn(a) & 0xFFu) | (((uint32_t)__float2int_rn(b) & 0xFFu) << 8) |
+           (((uint32_t)__float2int_rn(c) & 0xFFu) << 16) | ((uint32_t)__float2int_rn(d) << 24);
+}
+
+template <int LANES>
+__device__ __forceinline__ void store_s8x16(uint32_t* dst, int64_t i, const float (&x)[16]) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) dst[chunk_of<LANES>(i, k)] = pack_s8x4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+}
+
 // Perturbs the quantiser parameters of every group once (one Philox block per group, tensor id tid_q) and derives
 // what the producer needs, per (group, sign): A = (step, 1/step, lo - z, hi - z), B = (z, lo, hi, 0), all after
 // rounding / limiting.  A.z is NaN when the folded form is not exact for the group (|z| >= 2^24 - 16).
@@ -424,7 +442,10 @@ row_prepare_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, 
 // smooth: [sign][kind][smooth_ld] floats, kind 0 = scale, 1 = shift (2 = 1/scale, used by the activation side).
 // UPD: as in weight_operand_kernel, the previous step's update is applied to the master (read and written through w_out)
 // before this step's perturbation.
-template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH, bool UPD>
+// I8 (one group per row, prepared parameters): the operands are the signed bytes code - z instead of bf16 values
+// (op_plus / op_minus then point at rows of cols bytes) and the row's step goes to col_step[sign * col_stride + row]; a
+// row whose code - z leaves [-128, 127] (or whose zero point is beyond exact integer arithmetic) sets kErrCodeRange.
+template <int GROUP, bool DUAL, bool ADAPT, bool SMOOTH, bool UPD, bool I8 = false>
 __global__ void __launch_bounds__(kThreads, 3)
 weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int cols4, int bits, int perturb,
                               const PhiloxKeys rk, uint32_t tid, float eps,
@@ -432,7 +453,8 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                               const float4* __restrict__ prep_a, const float4* __restrict__ prep_b,
                               const float* __restrict__ smooth, int smooth_ld,
                               float* __restrict__ bias_part, int64_t n_groups, uchar4* __restrict__ codes,
-                              int qgroup_items, float4* w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk) {
+                              int qgroup_items, float4* w_out, const float* __restrict__ upd_scale, const PhiloxKeys urk,
+                              float* __restrict__ col_step = nullptr, int64_t col_stride = 0, int32_t* err_flag = nullptr) {
     // qgroup_items: 16-element items per quantisation group when that is not the GROUP-element span (one group per
     // row: cols / 16); 0 = the span itself.  The bias partial sums stay per span either way.
     constexpr int LANES = GROUP / 16;
@@ -532,6 +554,16 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
                 const int64_t qg = qgroup_items ? (int64_t)((uint32_t)i / (uint32_t)qgroup_items) : i / LANES;
                 const int64_t slot = qg * SG + sg;
                 const float4 a = live ? __ldg(prep_a + slot) : make_float4(1.f, 1.f, 0.f, 0.f);
+                if (I8) {
+                    // the first item of a row records the row's step and checks that code - z fits a signed byte
+                    if (live && (uint32_t)i % (uint32_t)qgroup_items == 0) {
+                        col_step[(int64_t)sg * col_stride + qg] = a.x;
+                        if (!(a.z >= -128.0f && a.w <= 127.0f)) atomicExch(err_flag, kErrCodeRange);
+                    }
+                    quantise16_integer(v, a);
+                    if (live) store_s8x16<LANES>(reinterpret_cast<uint32_t*>(sg == 0 ? op_plus : op_minus), i, v);
+                    continue;
+                }
                 const bool literal = (a.z != a.z) || cdp != nullptr;
                 if (__any_sync(0xffffffffu, literal)) {       // zero point beyond exact integer arithmetic, or codes wanted
                     const float4 b = live ? __ldg(prep_b + slot) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -866,6 +898,31 @@ static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
     }
     const int qgi = a.per_channel ? (int)(a.cols / 16) : 0;
     const PhiloxKeys rk = philox_keys(a.seed);
+    if constexpr (GROUP == 128 && ADAPT) {
+        if (a.i8) {
+            float4* wm = reinterpret_cast<float4*>(const_cast<float*>(a.w));
+            if (a.op_minus && pend)
+                weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH, true, true><<<grid, kThreads, 0, s>>>(
+                    w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
+                    a.bias_part, n_groups, nullptr, qgi, wm, pend->scale, philox_keys(pend->seed), a.col_step, a.col_stride, a.err_flag);
+            else if (a.op_minus)
+                weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH, false, true><<<grid, kThreads, 0, s>>>(
+                    w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,
+                    a.bias_part, n_groups, nullptr, qgi, nullptr, nullptr, rk, a.col_step, a.col_stride, a.err_flag);
+            else
+                weight_operand_learned_kernel<GROUP, false, ADAPT, SMOOTH, false, true><<<grid, kThreads, 0, s>>>(
+                    w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, nullptr, pa, pb, a.smooth, a.smooth_ld,
+                    a.bias_part, n_groups, nullptr, qgi, nullptr, nullptr, rk, a.col_step, a.col_stride, a.err_flag);
+            count_launch();
+            if (SMOOTH) {
+                const int64_t work = a.rows * signs * 32;
+                bias_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, s>>>(a.bias_part, n_groups, (int)(a.cols / GROUP), (int)a.rows,
+                                                                                  signs, a.bias0, a.bias_out, a.bias_out_stride);
+                count_launch();
+            }
+            return;
+        }
+    }
     if (a.op_minus && pend)
         weight_operand_learned_kernel<GROUP, true, ADAPT, SMOOTH, true><<<grid, kThreads, 0, s>>>(
             w4, n16, (int)(a.cols / 4), a.bits, a.perturb, rk, a.tid, a.eps, p, m, pa, pb, a.smooth, a.smooth_ld,

@@ -14,7 +14,8 @@ between iterations) and prints one JSON line per kernel with its achieved rate.
 
   python -m paper_2509_00031_b200.microbench --op gemm --M 8192 --N 4096 --K 4096 --sustain 2.5
       (back-to-back launches for 2.5 s under the power cap: TFLOP/s, median SM clock and board power, mJ per launch;
-       --op gemm_lib runs the library's bf16 GEMM on the same shape the same way, as the yardstick)
+       --op gemm_lib runs the library's bf16 GEMM on the same shape the same way, as the yardstick;
+       --op gemm_i8 the 8-bit integer GEMM of the per-channel workloads, --op gemm_i8_lib the library's int8 GEMM)
 
 It is also the small, self-contained command used for ncu captures of one kernel.
 """
@@ -177,11 +178,21 @@ def main():
     dev = "cuda"
     flush = None if a.no_flush else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = dict(op=a.op)
-    if a.op in ("gemm", "head_loss", "gemm_lib"):
+    if a.op in ("gemm", "head_loss", "gemm_lib", "gemm_i8", "gemm_i8_lib"):
         A = torch.randint(-127, 128, (a.M, a.K), device=dev).to(torch.bfloat16)
         B = (torch.randn(a.N, a.K, device=dev) * 0.02).to(torch.bfloat16)
         rs = torch.rand(a.M, device=dev) + 0.5
-        if a.op == "gemm":
+        if a.op in ("gemm_i8", "gemm_i8_lib"):      # signed-byte operands: our kind::i8 kernel, or the library's int8 GEMM as a yardstick
+            A8 = torch.randint(-127, 128, (a.M, a.K), device=dev, dtype=torch.int8)
+            B8 = torch.randint(-15, 16, (a.N, a.K), device=dev, dtype=torch.int8)
+            cs = torch.rand(a.N, device=dev) * 1e-3 + 1e-3
+            if a.op == "gemm_i8":
+                C = torch.zeros(a.M, a.N, device=dev)
+                fn = lambda: zq.zoqat_op_gemm_i8(A8, B8, cs, row_step=rs, out=C, accumulate=a.accumulate)
+            else:
+                Bt = B8.t()
+                fn = lambda: torch._int_mm(A8, Bt)
+        elif a.op == "gemm":
             C = torch.zeros(a.M, a.N, device=dev)
             fn = lambda: zq.zoqat_op_gemm(A, B, row_step=rs, out=C, accumulate=a.accumulate, impl=a.impl)
         elif a.op == "gemm_lib":            # the library's bf16 GEMM (bf16 result): a yardstick, not part of the path

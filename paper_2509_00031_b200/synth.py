@@ -40,6 +40,14 @@ WORKLOADS = {
                                     adaptive_quant=True, smoothing=True),
     "llama7b_w6a6_perchannel": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
                                     w_bits=6, w_group=0, a_bits=6, batch=4, seq=1024, bf16_init=True),
+    # the same settings with the block linears evaluated on integers (exact sums of 8-bit codes, steps applied outside)
+    "llama7b_w4a4_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                         w_bits=4, w_group=0, a_bits=4, batch=4, seq=1024, bf16_init=True,
+                                         adaptive_quant=True, smoothing=True, integer_gemm=True),
+    "llama7b_w6a6_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                         w_bits=6, w_group=0, a_bits=6, batch=4, seq=1024, bf16_init=True, integer_gemm=True),
+    "llama7b_w4a8_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                         w_bits=4, w_group=0, a_bits=8, batch=4, seq=1024, bf16_init=True, integer_gemm=True),
 }
 
 
