@@ -33,18 +33,21 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row (128 int8)
 constexpr int UMMA_K = 16;             // 32 bytes of the row per MMA: 16 bf16 or 32 int8
-constexpr int kThreadsTC = 192;
+constexpr int kThreadsTC = 192;        // four epilogue warps
+constexpr int kThreadsTC8 = 320;       // eight epilogue warps (8-bit kind: half the MMA time per tile, the same epilogue work)
 
 // CG = CTAs per tile: 1, or 2 (a cluster of two CTAs on an SM pair computes a 256 x BN tile with one
 // cta_group::2 MMA; each CTA stages its 128 rows of A and its half of the B rows, so a stage is a third smaller).
-template <int BN, int CG> struct TileCfg {
-    static constexpr int kStages = (BN == 256 && CG == 1) ? 4 : 6;
+// EW = epilogue warps: 4 (one per 32-lane quarter of the accumulator), or 8 (two per quarter, each taking every other
+// 32-column chunk; their staging boxes cost one stage of the ring).
+template <int BN, int CG, int EW = 4> struct TileCfg {
+    static constexpr int kStages = (BN == 256 && CG == 1) ? 4 : (EW == 8 ? 5 : 6);
     static constexpr int kABytes = BM * BK * 2;
     static constexpr int kBBytes = (BN / CG) * BK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     // output staging for the TMA stores of the epilogue: two 32x32 fp32 boxes per epilogue warp
     static constexpr int kOutBoxBytes = 32 * 32 * 4;
-    static constexpr int kOutStageBytes = 4 * 2 * kOutBoxBytes;
+    static constexpr int kOutStageBytes = EW * 2 * kOutBoxBytes;
     static constexpr int kSmemBytes = kStages * kStageBytes + kOutStageBytes + 1024 /*align slack*/ + 256 /*barriers*/;
 };
 
@@ -137,10 +140,12 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int r, int& tm, i
 }
 
 template <int BN, int CG, bool I8>
-__global__ void __launch_bounds__(kThreadsTC, 1)
+__global__ void __launch_bounds__(I8 ? kThreadsTC8 : kThreadsTC, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ AttMaps att, TcParams p) {
-    using Cfg = TileCfg<BN, CG>;
+    constexpr int EW = I8 ? 8 : 4;
+    constexpr int EH = EW / 4;                                   // epilogue warps per quarter: chunk stride
+    using Cfg = TileCfg<BN, CG, EW>;
     constexpr int S = Cfg::kStages;
     constexpr int TM = BM * CG;                                  // rows of a tile
     const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;     // CTA 0 of a pair leads: it issues the MMAs
@@ -167,7 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4 * CG); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), EW * CG); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b);
@@ -260,6 +265,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ---------------- epilogue (warps 2..5) ----------------
         const int quarter = warp & 3;                        // TMEM lanes [32*quarter, 32*quarter+32)
+        const int ew = warp - 2;                             // epilogue warp 0 .. EW-1: staging boxes 2*ew, 2*ew + 1
+        const int eh = ew >> 2;                              // which of the quarter's EH warps: chunks eh, eh + EH, ...
         int acc = 0; uint32_t acc_phase = 0;
         int out_buf = 0;
         const uint64_t pol_out = l2_policy(p.hint_out);
@@ -295,7 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int dh = p.d_head, hd = dh >> 1;
                     const int sel = (int)((int64_t)tn * BN / p.d_model);           // 0 q, 1 k, 2 v
                     const int head0 = (int)(((int64_t)tn * BN - (int64_t)sel * p.d_model) / dh);
-                    const uint32_t stage = out_stage + (uint32_t)(quarter * 2 * Cfg::kOutBoxBytes);     // 8 KB of this warp
+                    const uint32_t stage = out_stage + (uint32_t)(ew * 2 * Cfg::kOutBoxBytes);     // 8 KB of this warp
                     if (sel < 2) {
                         const CUtensorMap* mh = sel == 0 ? &att.qh : &att.kh;
                         const CUtensorMap* ml = sel == 0 ? &att.ql : &att.kl;
@@ -315,7 +322,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 }
                             }
 #pragma unroll 1
-                            for (int hh = 0; hh < BN / dh; ++hh) {
+                            for (int hh = eh; hh < BN / dh; hh += EH) {
                                 uint32_t va[32], vb[32];
                                 __syncwarp();
                                 tmem_ld32(t_addr + (uint32_t)(hh * dh + part * 32), va);
@@ -370,12 +377,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     } else {
 #pragma unroll 1
-                        for (int c = 0; c < BN / 32; ++c) {
+                        for (int c = eh; c < BN / 32; c += EH) {
                             uint32_t v[32];
                             __syncwarp();
                             tmem_ld32(t_addr + (uint32_t)(c * 32), v);
                             tmem_ld_wait();
-                            const uint32_t box = stage + (uint32_t)((c & 1) * 4096);    // hi box, lo box 2 KB further
+                            const uint32_t box = stage + (uint32_t)(((c / EH) & 1) * 4096);    // hi box, lo box 2 KB further
                             if (lane == 0) bulk_wait_read_1();
                             __syncwarp();
                             const int64_t n0 = n_base + c * 32;
@@ -410,13 +417,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // collected for the activation quantiser that follows.
                 float amax = 0.0f;
 #pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
+                for (int c = eh; c < BN / 64; c += EH) {
                     uint32_t vg[32], vu[32];
                     __syncwarp();
                     tmem_ld32(t_addr + (uint32_t)(c * 32), vg);
                     tmem_ld32(t_addr + (uint32_t)(BN / 2 + c * 32), vu);
                     tmem_ld_wait();
-                    const uint32_t box = out_stage + (uint32_t)((quarter * 2 + out_buf) * Cfg::kOutBoxBytes);
+                    const uint32_t box = out_stage + (uint32_t)((ew * 2 + out_buf) * Cfg::kOutBoxBytes);
                     if (lane == 0) bulk_wait_read_1();
                     __syncwarp();
                     const int64_t f0 = (int64_t)tn * (BN / 2) + c * 32;     // feature of column 0 of this chunk
@@ -451,7 +458,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (row_ok) atomicMax(p.row_amax + row, __float_as_uint(amax));
             }
 #pragma unroll 1
-            for (int c = 0; c < ((p.mode == 3 || p.mode == 2) ? 0 : BN / 32); ++c) {
+            for (int c = eh; c < ((p.mode == 3 || p.mode == 2) ? 0 : BN / 32); c += EH) {
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)(c * 32), v);
@@ -462,7 +469,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     // Stage the warp's 32x32 box in shared memory (128-byte rows, 16-byte chunks XOR-swizzled by
                     // row so that the writes spread over all banks) and hand it to the TMA unit, which writes
                     // whole rows (or adds them into the residual stream) and clips the box at the matrix edge.
-                    const uint32_t box = out_stage + (uint32_t)((quarter * 2 + out_buf) * Cfg::kOutBoxBytes);
+                    const uint32_t box = out_stage + (uint32_t)((ew * 2 + out_buf) * Cfg::kOutBoxBytes);
                     if (lane == 0) bulk_wait_read_1();          // the box written two chunks ago has been read
                     __syncwarp();
                     const bool full = n0 + 32 <= p.N;
@@ -544,7 +551,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     ce_m = nm;
                 }
             }
-            if (p.mode == 1 && row_ok) p.partials[row * p.tiles_n + tn] = make_float2(ce_m, ce_s);
+            // (the cross-entropy partials are per row and tile: four epilogue warps only - the 8-bit kind never runs mode 1)
+            if (p.mode == 1 && row_ok && EW == 4) p.partials[row * p.tiles_n + tn] = make_float2(ce_m, ce_s);
             // accumulator drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
@@ -687,7 +695,7 @@ TileOrder choose_order(int64_t M, int64_t N, int64_t K, int tiles_m, int tiles_n
 
 template <int BN, int CG, bool I8 = false>
 int launch_tc(const GemmArgs& a, cudaStream_t s) {
-    using Cfg = TileCfg<BN, CG>;
+    using Cfg = TileCfg<BN, CG, I8 ? 8 : 4>;
     alignas(64) CUtensorMap map_a, map_b, map_out;
     alignas(64) AttMaps att;
     const size_t b_stride = a.Z > 1 ? a.b_stride : (size_t)a.N * a.K;
@@ -743,7 +751,7 @@ int launch_tc(const GemmArgs& a, cudaStream_t s) {
     const int grid = (int)(total < units ? total : units) * CG;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(kThreadsTC, 1, 1);
+    cfg.blockDim = dim3(I8 ? kThreadsTC8 : kThreadsTC, 1, 1);
     cfg.dynamicSmemBytes = Cfg::kSmemBytes;
     cfg.stream = s;
     cudaLaunchAttribute at[1];
