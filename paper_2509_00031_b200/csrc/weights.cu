@@ -586,6 +586,100 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
     }
 }
 
+// One quantisation group per output row, min/max quantiser, both signs, in ONE pass over the row: a CTA owns a row,
+// every thread up to NI items of 16 elements.  The +eps values stay in registers and the -eps values in shared memory
+// while the row's four extrema are reduced over the CTA; then both operands are quantised with the folded form of
+// row_prepare_kernel + weight_operand_learned_kernel (the same operations on the same numbers, so the same bits) and
+// written.  The direction is evaluated once (the two-pass form evaluates it in both passes).
+// UPD / I8 as in weight_operand_learned_kernel.  Dynamic shared memory: NI * 16 * kThreads floats.
+template <int NI, bool UPD, bool I8>
+__global__ void __launch_bounds__(kThreads, NI == 1 ? 4 : (NI == 2 ? 3 : 2))
+weight_operand_row_kernel(const float4* __restrict__ w, int rows, int items_per_row, int bits, const PhiloxKeys rk, uint32_t tid,
+                          float eps, void* __restrict__ op_plus, void* __restrict__ op_minus, float4* w_out,
+                          const float* __restrict__ upd_scale, const PhiloxKeys urk, float* __restrict__ col_step,
+                          int64_t col_stride, int32_t* err_flag) {
+    constexpr int LANES = 8;                       // chunk interleave of 128-element spans, as in the other producers
+    extern __shared__ float xm_s[];                // [NI][16][kThreads]
+    __shared__ float2 tab[kIcdfKnots];
+    __shared__ float red[2][4][kThreads / 32];
+    stage_icdf_table(tab);
+    const float upd_c = UPD ? -(*upd_scale) : 0.0f;
+    const float qp = (float)((1 << bits) - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int par = 0;
+    for (int r = blockIdx.x; r < rows; r += gridDim.x, par ^= 1) {
+        float x[NI][16];
+        float mnp = INFINITY, mxp = -INFINITY, mnm = INFINITY, mxm = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < NI; ++j) {
+            const int li = threadIdx.x + j * kThreads;
+            if (li >= items_per_row) continue;
+            const int64_t i = (int64_t)r * items_per_row + li;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int64_t chunk = chunk_of<LANES>(i, k);
+                float4 v = UPD ? w_out[chunk] : __ldg(w + chunk);
+                if (UPD) {
+                    const float4 zu = direction4(tab, urk, tid, (uint64_t)chunk);
+                    v = make_float4(__fmaf_rn(upd_c, zu.x, v.x), __fmaf_rn(upd_c, zu.y, v.y), __fmaf_rn(upd_c, zu.z, v.z), __fmaf_rn(upd_c, zu.w, v.w));
+                    w_out[chunk] = v;
+                }
+                const float4 z = direction4(tab, rk, tid, (uint64_t)chunk);
+                const float vv[4] = {v.x, v.y, v.z, v.w}, zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float a = __fmaf_rn(eps, zz[e], vv[e]), b = __fmaf_rn(-eps, zz[e], vv[e]);
+                    x[j][4 * k + e] = a;
+                    xm_s[(j * 16 + 4 * k + e) * kThreads + threadIdx.x] = b;
+                    mnp = fminf(mnp, a); mxp = fmaxf(mxp, a);
+                    mnm = fminf(mnm, b); mxm = fmaxf(mxm, b);
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mnp = fminf(mnp, __shfl_xor_sync(0xffffffffu, mnp, o)); mxp = fmaxf(mxp, __shfl_xor_sync(0xffffffffu, mxp, o));
+            mnm = fminf(mnm, __shfl_xor_sync(0xffffffffu, mnm, o)); mxm = fmaxf(mxm, __shfl_xor_sync(0xffffffffu, mxm, o));
+        }
+        if (lane == 0) { red[par][0][warp] = mnp; red[par][1][warp] = mxp; red[par][2][warp] = mnm; red[par][3][warp] = mxm; }
+        __syncthreads();        // red[par] is next written two rows on, after the barrier of the row in between
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) {
+            mnp = fminf(mnp, red[par][0][i]); mxp = fmaxf(mxp, red[par][1][i]);
+            mnm = fminf(mnm, red[par][2][i]); mxm = fmaxf(mxm, red[par][3][i]);
+        }
+        const GroupQ gp = group_params(mnp, mxp, qp), gm = group_params(mnm, mxm, qp);
+        const float zp_ = __fadd_rn(gp.zp, 0.0f), zm_ = __fadd_rn(gm.zp, 0.0f);        // -0 -> +0
+        const float4 ap = make_float4(gp.step, gp.inv, -zp_, __fadd_rn(qp, -zp_));
+        const float4 am = make_float4(gm.step, gm.inv, -zm_, __fadd_rn(qp, -zm_));
+        if (I8 && threadIdx.x == 0) {
+            col_step[r] = ap.x;
+            col_step[col_stride + r] = am.x;
+            if (!(ap.z >= -128.0f && ap.w <= 127.0f && am.z >= -128.0f && am.w <= 127.0f)) atomicExch(err_flag, kErrCodeRange);
+        }
+#pragma unroll
+        for (int j = 0; j < NI; ++j) {
+            const int li = threadIdx.x + j * kThreads;
+            if (li >= items_per_row) continue;
+            const int64_t i = (int64_t)r * items_per_row + li;
+            float y[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) y[e] = xm_s[(j * 16 + e) * kThreads + threadIdx.x];
+            if (I8) {
+                quantise16_integer(x[j], ap);
+                quantise16_integer(y, am);
+                store_s8x16<LANES>(reinterpret_cast<uint32_t*>(op_plus), i, x[j]);
+                store_s8x16<LANES>(reinterpret_cast<uint32_t*>(op_minus), i, y);
+            } else {
+                quantise16_folded(x[j], ap);
+                quantise16_folded(y, am);
+                store_bf16x16<LANES>(reinterpret_cast<uint2*>(op_plus), i, x[j]);
+                store_bf16x16<LANES>(reinterpret_cast<uint2*>(op_minus), i, y);
+            }
+        }
+    }
+}
+
 // out[sign][row] = bias0[row] + sum over the row's groups of bias_part[sign][row * gpr + g]; one warp per (sign, row),
 // lane-strided partial sums in double and a fixed shuffle tree, so the result does not depend on timing.
 __global__ void bias_reduce_kernel(const float* __restrict__ part, int64_t n_groups, int gpr, int rows, int signs,
@@ -953,8 +1047,43 @@ static void learned_dispatch_group(const LearnedOperandArgs& a, cudaStream_t s) 
     else learned_dispatch<GROUP, false, true>(a, s);
 }
 
+template <int NI, bool UPD, bool I8>
+static void row_launch(const LearnedOperandArgs& a, cudaStream_t s) {
+    const PendingUpdate* pend = UPD ? a.pend : nullptr;
+    // static + dynamic shared memory exceed the default limit from NI = 2 on: every instantiation opts in
+    const size_t smem = (size_t)NI * 16 * kThreads * sizeof(float);
+    static DeviceOnce attr;
+    if (attr.first() && cudaFuncSetAttribute(weight_operand_row_kernel<NI, UPD, I8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem) != cudaSuccess)
+        attr.retry();
+    const int per_sm = NI == 1 ? 4 : (NI == 2 ? 3 : 2);
+    const int64_t cap = (int64_t)148 * per_sm;
+    const int grid = (int)(a.rows < cap ? a.rows : cap);
+    const PhiloxKeys rk = philox_keys(a.seed), urk = pend ? philox_keys(pend->seed) : rk;
+    weight_operand_row_kernel<NI, UPD, I8><<<grid, kThreads, smem, s>>>(
+        reinterpret_cast<const float4*>(a.w), (int)a.rows, (int)(a.cols / 16), a.bits, rk, a.tid, a.eps, a.op_plus, a.op_minus,
+        pend ? reinterpret_cast<float4*>(const_cast<float*>(a.w)) : nullptr, pend ? pend->scale : nullptr, urk, a.col_step,
+        a.col_stride, a.err_flag);
+    count_launch();
+}
+
+template <int NI>
+static void row_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
+    if (a.i8) { if (a.pend) row_launch<NI, true, true>(a, s); else row_launch<NI, false, true>(a, s); }
+    else { if (a.pend) row_launch<NI, true, false>(a, s); else row_launch<NI, false, false>(a, s); }
+}
+
 void launch_weight_operand_learned(const LearnedOperandArgs& a, cudaStream_t s) {
     if (a.rows * a.cols == 0 || ((a.perturb || a.pend) && !ensure_icdf_table())) return;
+    // plain min/max rows, both signs, perturbed: one pass per row with a single evaluation of the direction
+    if (a.per_channel && a.bits != 0 && !a.theta && !a.smooth && a.op_minus && a.perturb && !a.codes && a.cols <= 16 * kThreads * 4) {
+        const int64_t items = a.cols / 16;
+        if (items <= kThreads) row_dispatch<1>(a, s);
+        else if (items <= 2 * kThreads) row_dispatch<2>(a, s);
+        else if (items <= 3 * kThreads) row_dispatch<3>(a, s);
+        else row_dispatch<4>(a, s);
+        return;
+    }
     if (a.per_channel) { learned_dispatch_group<128>(a, s); return; }      // cols % 128 == 0 (checked by the callers)
     if (a.group == 32) learned_dispatch_group<32>(a, s);
     else if (a.group == 64) learned_dispatch_group<64>(a, s);

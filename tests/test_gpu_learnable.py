@@ -196,6 +196,26 @@ def test_per_row_groups_match_oracle(zq, bits, adaptive, smoothing):
             assert np.array_equal(codes.cpu().numpy(), np.asarray(q).astype(np.uint8))
 
 
+@pytest.mark.parametrize("cols", [640, 4224, 11008, 12416], ids=["one_item", "two_items", "three_items", "four_items"])
+@pytest.mark.parametrize("bits", [4, 6])
+def test_per_row_one_pass_producer_matches_oracle(zq, cols, bits):
+    """Plain min/max rows with both signs take the one-pass producer (a CTA per row, the direction evaluated once):
+    bf16 operands and the signed-byte operands with their row steps, bit for bit."""
+    rng = np.random.default_rng(cols + bits)
+    rows = 45
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    w[3] *= 4.0
+    seed, tid, eps = 123, 20, np.float32(1e-3)
+    plus, minus, _, _ = zq.zoqat_op_weight_operand_learned(dev(w), 0, bits, seed, tid, float(eps))
+    p8, m8, steps, _, err = zq.zoqat_op_weight_operand_i8(dev(w), bits, seed, tid, float(eps))
+    assert int(err.item()) == 0
+    for sg, (e, op, o8) in enumerate(((eps, plus, p8), (-eps, minus, m8))):
+        q, delta, zp, deq = core.weight_quant(core.perturb(w, seed, tid, e), cols, bits)
+        assert np.array_equal(bf16_to_f32(op), core.round_bf16(deq)), sg
+        assert np.array_equal(o8.cpu().numpy().astype(np.int64), q.astype(np.int64) - zp.astype(np.int64)), sg
+        assert np.array_equal(steps[sg].cpu().numpy().view(np.uint32), delta.reshape(rows).view(np.uint32)), sg
+
+
 # ---- the model ---------------------------------------------------------------------------------------------------
 SMALL_LLAMA = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=600, w_bits=4, w_group=64, a_bits=8)
 SMALL_LLAMA_UNFUSED = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=320, vocab=600, w_bits=4, w_group=64, a_bits=8)
