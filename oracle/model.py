@@ -333,7 +333,8 @@ class OracleModel:
         T, K = a.shape
         N, G = delta.shape
         g = K // G
-        inner = np.einsum("tgk,ngk->tng", a.reshape(T, G, g), cz.reshape(N, G, g))   # exact: integers far below 2^53
+        # inner[t, n, group] = sum over the group's columns of a * (c - z): exact, integers far below 2^53
+        inner = np.stack([a[:, j * g:(j + 1) * g] @ cz[:, j * g:(j + 1) * g].T for j in range(G)], axis=-1)
         if cfg.accum_f32:       # binary32 outside the integer sums: convert, scale by the group step, by the token step
             y = ((inner.astype(F32) * delta[None, :, :]).astype(F32).sum(axis=-1, dtype=F32) * s[:, None]).astype(F32).astype(np.float64)
         else:

@@ -64,7 +64,8 @@ def quantise_like_oracle(x, a_bits):
     return core.round_bf16(x32).astype(np.float64), np.ones(x32.shape[0], np.float32), None
 
 
-def compare_forward(zq, model, oracle, shape, tokens, labels, seed, eps, label, max_diff_frac=None, self_check=False):
+def compare_forward(zq, model, oracle, shape, tokens, labels, seed, eps, label, max_diff_frac=None, self_check=False,
+                    noise_bound=1e-1):
     """One forward on both sides; returns (stats dict, GPU token losses float64, oracle token losses, valid).
     self_check: also run the oracle with binary32 accumulation (OracleConfig.accum_f32) and count ITS codes that
     differ from the float64 run's - what another correct binary32 implementation does on the same inputs."""
@@ -83,8 +84,8 @@ def compare_forward(zq, model, oracle, shape, tokens, labels, seed, eps, label, 
     # tokens whose history is free of differing codes: position s of a sequence sees positions <= s of earlier quantisers
     dirty = np.zeros((B, S), dtype=bool)
     # one differing code moves its token's later values by about a quantisation step over sqrt(fan-in), relative to the
-    # row's largest value; products of two such values (the gated FFN) by a few times that
-    noise_bound = 1e-1
+    # row's largest value; products of two such values (the gated FFN) by a few times that (noise_bound: 1e-1 unless the
+    # caller knows better - one 6-bit code is 1/31 of its row's largest value)
     # differing codes multiply from one quantiser to the next (each re-draws its token's rounding noise): a few per
     # mille of all int8 codes after two layers, a few per cent of all bf16 roundings (256 times finer steps)
     if max_diff_frac is None:

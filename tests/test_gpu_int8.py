@@ -256,6 +256,25 @@ def test_forward_element_by_element(zq, shape, batch, seq):
                         max_diff_frac=0.1)
 
 
+def test_workload_dimensions_element_by_element(zq):
+    """The W6A6 per-channel workload's own dimensions (rows of 4096 and 11008 weights, 32 heads, the fused epilogues),
+    one layer, 128 tokens: every quantisation point, the residual stream and the per-position loss against the oracle.
+    Norm gains are jittered: with gains of exactly 1 the first quantiser sees bf16-valued embedding rows divided by
+    their largest element, which puts about two values per token exactly on a rounding boundary of the 6-bit grid, and
+    then almost no token is free of a differing code (the benchmark's inputs keep gains of 1; this test wants tokens it
+    can compare to binary32 accuracy)."""
+    shape = dict(synth.WORKLOADS["llama7b_w6a6_perchannel_int8"], n_layers=1)
+    batch, seq = 1, 128
+    params = synth.make_params(shape, seed=3, max_seq=seq, jitter=True)
+    oracle = OracleModel(oracle_cfg(shape, integer_gemm=True), synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq, gemm_impl=zq.GEMM_TCGEN05_I8)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
+    # 6-bit activation codes: one differing code is 1/31 of its row's largest value; behind a token with a differing
+    # code the next quantiser re-draws a third of its codes, so such tokens agree only to the quantisation noise itself
+    compare_forward(zq, model, oracle, shape, tokens, labels, 1000, 1e-3, "integer GEMM, 7B dimensions, W6A6 per-channel", max_diff_frac=0.3,
+                    noise_bound=3e-1)
+
+
 def test_integer_gemm_needs_per_row_groups(zq):
     shape = dict(I8_LLAMA, w_group=128)
     params = synth.make_params(shape, seed=3, max_seq=32, jitter=True)

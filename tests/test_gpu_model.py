@@ -300,6 +300,8 @@ WORKLOAD_CUTS = [
     pytest.param(_cut("llama7b_w2", 1), 1, 128, 0, False, id="llama7b_w2"),
     pytest.param(_cut("llama7b_w3", 1), 1, 128, 0, False, id="llama7b_w3"),
     pytest.param(_cut("llama13b_light", 2), 1, 96, 1, True, id="llama13b_light"),
+    # one weight group per output row on the 8-bit integer GEMM (rows of 4096 and 11008 weights through the one-pass producer)
+    pytest.param(_cut("llama7b_w4a8_perchannel_int8", 1), 1, 128, 0, False, id="llama7b_w4a8_perchannel_int8"),
 ]
 
 
@@ -310,13 +312,16 @@ def test_workload_layer_dimensions(zq, shape, batch, seq, first_trainable, packe
     two or three state-synced steps against the oracle - both losses, every updated tensor bit for bit given the
     step's own factor, g under the band rule."""
     params = synth.make_params(shape, seed=3, max_seq=seq)
-    oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable), synth.copy_params(params))
+    i8 = bool(shape.get("integer_gemm"))
+    oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first_trainable, integer_gemm=i8), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq,
-                          first_trainable_layer=first_trainable, packed_frozen=packed)
+                          first_trainable_layer=first_trainable, packed_frozen=packed,
+                          gemm_impl=zq.GEMM_TCGEN05_I8 if i8 else zq.GEMM_TCGEN05)
     if packed:
         model.zoqat_prequantize_frozen()
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=21)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 3 if shape["a_bits"] else 2, 1e-3, 1e-6)
+    n_steps = 2 if (first_trainable or i8 or not shape["a_bits"]) else 3         # (the two-layer cut is the slowest: two steps)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, 1e-3, 1e-6)
     check_g(recs, f"workload dims {shape['arch']} d={shape['d_model']} F={shape['d_ffn']} V={shape['vocab']} "
                   f"W{shape['w_bits']}A{shape['a_bits']} g{shape['w_group']} T={batch * seq}")
     if first_trainable:
@@ -327,15 +332,16 @@ def test_full_token_count_layer_step(zq):
     """The bench workload's own token count through one layer and the vocabulary projection: LLaMA-7B dimensions,
     W4A8 g128, batch 4 x seq 1024 - 16 row tiles and 8 attention query tiles per sequence in every GEMM, both passes
     side by side on 8192 rows, the schedule the benchmark times.  Full zoqat_step against the oracle: both losses,
-    every updated tensor (bit for bit given the step's own factor), g under the band rule over two seeds.  (The
-    per-position view of the same configuration is test_full_token_count_layer_element_by_element.)"""
+    every updated tensor (bit for bit given the step's own factor), g under the band rule.  One step: the oracle needs
+    about half a minute per evaluation at this size.  (The per-position view of the same configuration is
+    test_full_token_count_layer_element_by_element.)"""
     shape = _cut("llama7b_w4a8", 1)
     batch, seq = shape["batch"], shape["seq"]
     params = synth.make_params(shape, seed=3, max_seq=seq)
     oracle = OracleModel(oracle_cfg(shape), synth.copy_params(params))
     model = zq.ZoqatModel(shape, zq.params_to_device(params), max_batch=batch, max_seq=seq)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=1234)
-    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 2, 1e-3, 1e-6)
+    recs = run_synced_steps(zq, model, oracle, shape, tokens, labels, 1, 1e-3, 1e-6)
     check_g(recs, "llama7b_w4a8, one layer, full 4 x 1024 tokens")
 
 
