@@ -196,6 +196,38 @@ def test_per_row_groups_match_oracle(zq, bits, adaptive, smoothing):
             assert np.array_equal(codes.cpu().numpy(), np.asarray(q).astype(np.uint8))
 
 
+@pytest.mark.parametrize("cols,rows,group", [(4096, 304, 128), (11008, 120, 128), (4096, 304, 0), (5120, 250, 64)],
+                         ids=["d4096_g128", "f11008_g128", "d4096_per_row", "d5120_g64"])
+def test_learned_producer_on_wide_tensors(zq, cols, rows, group):
+    """The Section 4.2 producer on rows as wide as the workloads' (4096, 5120, 11008 columns: every thread wraps around
+    the smoothing vectors several times): operands of both signs, the shift term of the bias and, with one group per
+    row, the signed-byte operands."""
+    bits = 4
+    rng = np.random.default_rng(cols + rows)
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    seed, tid, eps = 777, 52, np.float32(1e-3)
+    g = group or cols
+    theta = random_theta(w, g, bits, rng)
+    s = rng.uniform(0.5, 2.0, cols).astype(np.float32)
+    d = (0.3 * rng.standard_normal(cols)).astype(np.float32)
+    smooth = zq.zoqat_op_smooth_perturb(dev(s), dev(d), seed, 0x20021, 0x30021, float(eps))
+    plus, minus, bias, _ = zq.zoqat_op_weight_operand_learned(dev(w), group, bits, seed, tid, float(eps), theta=dev(theta), smooth=smooth)
+    ops8 = zq.zoqat_op_weight_operand_i8(dev(w), bits, seed, tid, float(eps), theta=dev(theta), smooth=smooth) if group == 0 else None
+    for sg, (e, op) in enumerate(((eps, plus), (-eps, minus))):
+        wp = core.perturb(w, seed, tid, e)
+        x = (wp * core.perturb(s, seed, 0x20021, e)[None, :]).astype(np.float32)
+        want_bias = wp.astype(np.float64) @ core.perturb(d, seed, 0x30021, e).astype(np.float64)
+        assert np.allclose(bias[sg].cpu().numpy(), want_bias, rtol=0, atol=2e-6 * np.abs(want_bias).max() + 1e-7)
+        thp = core.perturb(theta, seed, tid + QPARAM_ID, e)
+        q, deq = adaptive_weight_quant(x, thp, g, bits)
+        assert np.array_equal(bf16_to_f32(op), core.round_bf16(deq)), sg
+        if ops8 is not None:
+            z = np.rint(thp[..., 1]).reshape(rows, 1)
+            assert int(ops8[4].item()) == 0
+            assert np.array_equal(ops8[sg].cpu().numpy().astype(np.int64), np.asarray(q).astype(np.int64) - z.astype(np.int64)), sg
+            assert torch.equal(ops8[3][sg], bias[sg])
+
+
 @pytest.mark.parametrize("cols", [640, 4224, 11008, 12416], ids=["one_item", "two_items", "three_items", "four_items"])
 @pytest.mark.parametrize("bits", [4, 6])
 def test_per_row_one_pass_producer_matches_oracle(zq, cols, bits):
