@@ -77,8 +77,11 @@ __device__ __forceinline__ __nv_bfloat16* operand_row(__nv_bfloat16* op, int64_t
     return planes == 2 ? reinterpret_cast<__nv_bfloat16*>(reinterpret_cast<uint8_t*>(op) + r * cols) : op + r * cols;
 }
 __device__ __forceinline__ uint32_t s8x4(float a, float b, float c, float d) {
-    return ((uint32_t)__float2int_rn(a) & 0xFFu) | (((uint32_t)__float2int_rn(b) & 0xFFu) << 8) |
-           (((uint32_t)__float2int_rn(c) & 0xFFu) << 16) | ((uint32_t)__float2int_rn(d) << 24);
+    // adding 1.5 * 2^23 leaves the integer (two's complement) in the low mantissa bits: the low byte is the signed byte
+    constexpr float kMagic = 12582912.0f;
+    const uint32_t ua = __float_as_uint(__fadd_rn(a, kMagic)), ub = __float_as_uint(__fadd_rn(b, kMagic));
+    const uint32_t uc = __float_as_uint(__fadd_rn(c, kMagic)), ud = __float_as_uint(__fadd_rn(d, kMagic));
+    return __byte_perm(__byte_perm(ua, ub, 0x0040), __byte_perm(uc, ud, 0x0040), 0x5410);
 }
 
 // Writes the operand row from the fp32 row held in shared memory.

@@ -312,8 +312,11 @@ __device__ __forceinline__ void quantise16_integer(float (&x)[16], const float4&
 
 // Four integer-valued floats in [-128, 127] -> four signed bytes, first value in the low byte.
 __device__ __forceinline__ uint32_t pack_s8x4(float a, float b, float c, float d) {
-    return ((uint32_t)__float2int_rn(a) & 0xFFu) | (((uint32_t)__float2int_rn(b) & 0xFFu) << 8) |
-           (((uint32_t)__float2int_rn(c) & 0xFFu) << 16) | ((uint32_t)__float2int_rn(d) << 24);
+    // adding 1.5 * 2^23 leaves the integer (two's complement) in the low mantissa bits: the low byte is the signed byte
+    constexpr float kMagic = 12582912.0f;
+    const uint32_t ua = __float_as_uint(__fadd_rn(a, kMagic)), ub = __float_as_uint(__fadd_rn(b, kMagic));
+    const uint32_t uc = __float_as_uint(__fadd_rn(c, kMagic)), ud = __float_as_uint(__fadd_rn(d, kMagic));
+    return __byte_perm(__byte_perm(ua, ub, 0x0040), __byte_perm(uc, ud, 0x0040), 0x5410);
 }
 
 template <int LANES>

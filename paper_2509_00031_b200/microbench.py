@@ -210,7 +210,7 @@ def main():
             return
         med, best = timed(fn, a.iters, flush)
         out.update(M=a.M, N=a.N, K=a.K, ms=med, ms_best=best, tflops=flops / med / 1e9, tflops_best=flops / best / 1e9)
-    elif a.op in ("weight_pair", "weight_single", "weight_learned", "update", "unpack"):
+    elif a.op in ("weight_pair", "weight_single", "weight_learned", "weight_row", "weight_row_i8", "update", "unpack"):
         W = torch.randn(a.rows, a.cols, device=dev) * 0.02
         n = a.rows * a.cols
         if a.op == "weight_learned":
@@ -218,6 +218,12 @@ def main():
             smooth = zq.zoqat_op_smooth_perturb(torch.ones(a.cols, device=dev), torch.zeros(a.cols, device=dev), 1000, 0x20010, 0x30010, 1e-3)
             fn = lambda: zq.zoqat_op_weight_operand_learned(W, a.group, a.bits, 1000, 16, 1e-3, theta=theta, smooth=smooth)
             nbytes = n * (4 + 2 + 2 + 16 / a.group)
+        elif a.op == "weight_row":           # one min/max group per row, both signs, bf16 operands (one-pass row producer)
+            fn = lambda: zq.zoqat_op_weight_operand_learned(W, 0, a.bits, 1000, 16, 1e-3)
+            nbytes = n * (4 + 2 + 2)
+        elif a.op == "weight_row_i8":        # the same with signed-byte operands and the row steps
+            fn = lambda: zq.zoqat_op_weight_operand_i8(W, a.bits, 1000, 16, 1e-3)
+            nbytes = n * (4 + 1 + 1)
         elif a.op == "weight_pair":
             fn = lambda: zq.zoqat_op_weight_operand_pair(W, a.group, a.bits, 1000, 16, 1e-3)
             nbytes = n * (4 + 2 + 2)
