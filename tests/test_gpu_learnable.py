@@ -331,8 +331,9 @@ def test_initial_learnables_leave_the_model_unchanged(zq, shape):
     assert np.array_equal(th, init_quant_params(params["layers"][1]["wq"], shape["w_group"], shape["w_bits"]))
 
 
-@pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("shape,first", [(SMALL_LLAMA, 0), (SMALL_OPT, 1), (PER_ROW_W6A6, 0)], ids=["llama", "opt_last_layer", "per_row_w6a6"])
+# (the CUDA-core cross-check GEMM runs one of the three shapes: every case costs five oracle steps)
+@pytest.mark.parametrize("impl,shape,first", [(0, SMALL_LLAMA, 0), (1, SMALL_LLAMA, 0), (0, SMALL_OPT, 1), (0, PER_ROW_W6A6, 0)],
+                         ids=["llama-tcgen05", "llama-simt", "opt_last_layer-tcgen05", "per_row_w6a6-tcgen05"])
 def test_step_rates_match_oracle(zq, impl, shape, first):
     batch, seq, eps, lr, lrq, lrs = 2, 80, 1e-3, 1e-4, 3e-5, 5e-4
     model, oracle = build_pair(zq, shape, batch, seq, impl, True, True, first=first)

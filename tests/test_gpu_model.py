@@ -159,8 +159,9 @@ def run_synced_steps(zq, model, oracle, shape, tokens, labels, n_steps, eps, lr,
     return recs
 
 
-@pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("shape,batch,seq", [(SMALL_LLAMA, 2, 96), (SMALL_OPT, 3, 50)], ids=["llama_w4a8", "opt_w4"])
+# (the CUDA-core cross-check GEMM runs one of the two shapes: every case costs eight oracle steps and their band runs)
+@pytest.mark.parametrize("impl,shape,batch,seq", [(0, SMALL_LLAMA, 2, 96), (1, SMALL_LLAMA, 2, 96), (0, SMALL_OPT, 3, 50)],
+                         ids=["llama_w4a8-tcgen05", "llama_w4a8-simt", "opt_w4-tcgen05"])
 def test_step_matches_oracle(zq, impl, shape, batch, seq):
     model, oracle = build_pair(zq, shape, batch, seq, impl)
     tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=12)
