@@ -216,6 +216,28 @@ def test_step_rates_match_oracle(zq, shape):
     check_g(recs, f"integer GEMM {shape['arch']} W{shape['w_bits']}A{shape['a_bits']}")
 
 
+def test_frozen_first_layer_and_step_multi(zq):
+    """A frozen (unperturbed, never updated) first layer under a trainable one: its linears run once on T rows with
+    byte operands of the unperturbed weights; then q = 2 directions in one step.  Against the oracle's integer form."""
+    shape, batch, seq = I8_LLAMA, 2, 96
+    model, oracle = build_pair(zq, shape, batch, seq, zq.GEMM_TCGEN05_I8, False, False, first=1, integer_gemm=True)
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=29)
+    frozen = {k: oracle.p["layers"][0][k].copy() for k in oracle.linear_names()}
+    for seed, eps in [(3, 0.0), (3, 1e-3)]:
+        got = float(model.zoqat_forward_loss(dev(tokens), dev(labels), seed, eps).item())
+        want = oracle.loss(tokens, labels, seed, float(F32(eps)))
+        assert abs(got - want) <= 1e-4 * abs(want), (seed, eps, got, want)
+    res = model.zoqat_step_multi(dev(tokens), dev(labels), 50, 2, 1e-3, 1e-4).cpu()
+    model.zoqat_check()
+    want = oracle.step_multi(tokens, labels, 50, 2, 1e-3, 1e-4)
+    for i, (lp, lm, g) in enumerate(want):
+        r = zq.decode_step_result(res[i])
+        assert r["status"] == 0 and abs(r["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(r["loss_minus"] - lm) <= 1e-3 * abs(lm)
+    for k, wb in frozen.items():
+        assert np.array_equal(model.params["layers"][0][k].cpu().numpy(), wb), k
+    assert not np.array_equal(model.params["layers"][1]["wq"].cpu().numpy(), frozen["wq"])
+
+
 @pytest.mark.parametrize("shape,learned", [(I8_LLAMA, True), (I8_LLAMA_W6A6, False)], ids=["llama_learned", "llama_w6a6_minmax"])
 def test_deferred_update_gives_the_same_bits(zq, shape, learned):
     """The weights' update riding on the next step's producers (on the row min/max pass without learnable parameters):
