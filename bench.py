@@ -204,6 +204,8 @@ def run_ours(args, w, rank, world, local_rank):
         model.zoqat_init_qparams()
     if any_packed:
         model.zoqat_prequantize_frozen()
+        if w.get("integer_gemm") and not args.simt:
+            model.zoqat_expand_frozen()                    # frozen tensors as byte operands, once: no per-step work on them
         for l in range(w["n_layers"]):                     # the fp32 copies of packed tensors are no longer needed
             for name in synth.linear_shapes(w):
                 if l < ftl or (names is not None and name not in names):

@@ -111,8 +111,9 @@ extern "C" {
                                      the sum exact (tcgen05.mma kind::i8 on signed bytes, 32-bit accumulators), which
                                      is Q(x) Q(w)^T of Section 2 with no rounding of the operands; ZOQAT_GEMM_TCGEN05
                                      instead rounds the dequantised weight (c - z) * Delta to bf16.  Needs w_group = 0,
-                                     a_bits != 0, w_bits <= 7, every block linear QUANTIZED and none FROZEN_PACKED; the
-                                     vocabulary projection stays bf16.  A weight row whose c - z leaves [-128, 127]
+                                     a_bits != 0, w_bits <= 7, every block linear QUANTIZED or FROZEN_PACKED (packed
+                                     tensors expand straight into byte operands: no per-step work on their weights
+                                     beyond that); the vocabulary projection stays bf16.  A weight row whose c - z leaves [-128, 127]
                                      (zero point far outside the code range) makes the step report status 32 and
                                      zoqat_check() return ZOQAT_ERR_UNSUPPORTED; results of that call are not usable. */
 
@@ -127,8 +128,8 @@ typedef struct zoqat_config {
     int32_t max_seq;       /* ... and sequence length a call will pass                            */
     int32_t w_bits;        /* 2..8 (FROZEN_PACKED tensors: 2, 3 or 4)                             */
     int32_t w_group;       /* 32, 64 or 128 (divides d_model and d_ffn), or 0 = one group per output
-                              row ("per-channel" weights; d_model, d_ffn multiples of 128; not for
-                              FROZEN_PACKED tensors)                                              */
+                              row ("per-channel" weights; d_model, d_ffn multiples of 128; FROZEN_PACKED
+                              tensors then carry one (step, zero point) per row; not in decode)   */
     int32_t a_bits;        /* 4, 6 or 8 = per-token symmetric N-bit codes on block-linear inputs, 0 = none */
     int32_t gemm_impl;     /* ZOQAT_GEMM_*                                                        */
     float   norm_eps;
@@ -182,6 +183,17 @@ int zoqat_model_destroy(zoqat_model_t* m);
  * values into `packed` / `qparams`.  Idempotent.  Must run before the first
  * forward when such tensors exist. */
 int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream);
+
+/* ZOQAT_GEMM_TCGEN05_I8 only, optional, after zoqat_prequantize_frozen: expands every FROZEN_PACKED tensor once into the
+ * integer GEMM's operand (signed bytes code - zero point, and the rows' steps) inside `buffer_dev` (caller-owned, 256-byte
+ * aligned, zoqat_expand_frozen_bytes() bytes: one byte per block-linear weight plus four per output row; in use until the
+ * handle is destroyed or the call is repeated; buffer_dev = NULL returns to expanding on every step).  Afterwards a linear
+ * layer whose tensors are all frozen reads them in place, both passes as one product, and a frozen tensor that shares a
+ * GEMM with trainable ones (a frozen key projection next to trainable query / value projections) is copied instead of
+ * decoded: Section 4.3's frozen tensors then cost no arithmetic per step.  Results are bit-identical either way.  A row
+ * that does not fit a signed byte is reported through zoqat_check() (status 32). */
+int zoqat_expand_frozen_bytes(const zoqat_model_t* m, size_t* bytes);
+int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* stream);
 
 /* Section 4.2: writes the initial quantiser parameters of every ADAPTIVE tensor - step and zero point of the
  * default min/max scheme on the current (unperturbed) weights, alpha = 0, beta = 1 - at which the adaptive
@@ -415,9 +427,15 @@ int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int gr
                           void* stream);
 
 /* Packing of Section 4.3: quantise W (unperturbed) into packed codes + qparams,
- * and expansion of a packed tensor into the bf16 operand. */
+ * and expansion of a packed tensor into the bf16 operand.  group = 0: one group per row
+ * (cols % 128 == 0; qparams_dev then holds rows (step, zero point) pairs, zoqat_packed_bytes
+ * gives the sizes); zoqat_op_unpack_operand_i8 (group 0 only) expands into the integer GEMM's
+ * operand instead: operand_dev int8 [rows, cols] = code - zero point, col_step_dev fp32 [rows]
+ * the rows' steps, err_flag_dev (int32, zeroed by the caller) set to 32 if a row does not fit. */
 int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int group, int bits,
                          void* packed_dev, void* qparams_dev, void* stream);
+int zoqat_op_unpack_operand_i8(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols,
+                               int bits, void* operand_dev, float* col_step_dev, int32_t* err_flag_dev, void* stream);
 int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols,
                             int group, int bits, void* operand_dev, void* stream);
 

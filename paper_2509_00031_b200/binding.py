@@ -27,12 +27,12 @@ PROF_NAMES = ["gemm", "weight_operand", "act_operand", "attention", "loss", "upd
 
 EXPORTS = [
     "zoqat_query_workspace", "zoqat_packed_bytes", "zoqat_model_create", "zoqat_model_destroy",
-    "zoqat_prequantize_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_rates_deferred", "zoqat_step_finish_deferred", "zoqat_step_finish_rates_deferred", "zoqat_flush_update", "zoqat_step_multi",
+    "zoqat_prequantize_frozen", "zoqat_expand_frozen_bytes", "zoqat_expand_frozen", "zoqat_init_qparams", "zoqat_forward_loss", "zoqat_step", "zoqat_step_rates", "zoqat_step_deferred", "zoqat_step_rates_deferred", "zoqat_step_finish_deferred", "zoqat_step_finish_rates_deferred", "zoqat_flush_update", "zoqat_step_multi",
     "zoqat_step_begin", "zoqat_step_finish", "zoqat_step_finish_rates", "zoqat_step_host", "zoqat_step_host_deferred", "zoqat_apply_update", "zoqat_apply_update_rates", "zoqat_apply_update_multi", "zoqat_step_result",
     "zoqat_check", "zoqat_launch_count", "zoqat_profile_enable", "zoqat_profile_read", "zoqat_debug_buffer", "zoqat_debug_capture", "zoqat_debug_capture_bytes", "zoqat_status_string", "zoqat_last_error",
     "zoqat_op_philox_words", "zoqat_op_normal", "zoqat_op_weight_quant", "zoqat_op_weight_operand_pair",
     "zoqat_op_weight_operand_learned", "zoqat_op_smooth_perturb", "zoqat_op_smooth_act_operand", "zoqat_op_init_qparams",
-    "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_update", "zoqat_op_norm_act_operand",
+    "zoqat_op_pack_frozen", "zoqat_op_unpack_operand", "zoqat_op_unpack_operand_i8", "zoqat_op_update", "zoqat_op_norm_act_operand",
     "zoqat_op_ffn_act_operand", "zoqat_op_gemm", "zoqat_op_gemm_silu_gate", "zoqat_op_gemm_i8", "zoqat_op_weight_operand_i8", "zoqat_op_norm_act_operand_i8", "zoqat_op_qkv_attention", "zoqat_op_attention_scratch_bytes", "zoqat_op_attention",
     "zoqat_op_head_loss_scratch_bytes",
     "zoqat_op_head_loss", "zoqat_op_head_loss_static",
@@ -85,6 +85,8 @@ def lib():
             "zoqat_model_create": [P(Config), P(TensorDesc), i32, vp, sz, P(vp)],
             "zoqat_model_destroy": [vp],
             "zoqat_prequantize_frozen": [vp, vp],
+            "zoqat_expand_frozen_bytes": [vp, P(sz)],
+            "zoqat_expand_frozen": [vp, vp, sz, vp],
             "zoqat_init_qparams": [vp, vp],
             "zoqat_step_rates": [vp, vp, vp, i32, i32, u64, f32, f32, f32, f32, vp, vp],
             "zoqat_step_finish_rates": [vp, vp, u64, f32, f32, f32, f32, vp, vp],
@@ -121,6 +123,7 @@ def lib():
             "zoqat_op_weight_operand_pair": [vp, i64, i64, i32, i32, u64, u32, f32, vp, vp, vp],
             "zoqat_op_pack_frozen": [vp, i64, i64, i32, i32, vp, vp, vp],
             "zoqat_op_unpack_operand": [vp, vp, i64, i64, i32, i32, vp, vp],
+            "zoqat_op_unpack_operand_i8": [vp, vp, i64, i64, i32, vp, vp, vp, vp],
             "zoqat_op_update": [vp, u64, u64, u32, f32, vp],
             "zoqat_op_norm_act_operand": [vp, i64, i64, i32, vp, vp, f32, i32, vp, vp, vp, vp],
             "zoqat_op_ffn_act_operand": [vp, i64, i64, i32, i32, vp, vp, vp],
@@ -257,6 +260,15 @@ def zoqat_op_unpack_operand(packed, qparams, rows, cols, group, bits):
     operand = torch.empty((rows, cols), dtype=torch.bfloat16, device=packed.device)
     _check(lib().zoqat_op_unpack_operand(_p(packed), _p(qparams), rows, cols, group, bits, _p(operand), _stream()))
     return operand
+
+
+def zoqat_op_unpack_operand_i8(packed, qparams, rows, cols, bits):
+    """Per-row packed tensor -> (int8 operand code - zero point, row steps, error word)."""
+    operand = torch.empty((rows, cols), dtype=torch.int8, device=packed.device)
+    steps = torch.empty(rows, dtype=torch.float32, device=packed.device)
+    err = torch.zeros(1, dtype=torch.int32, device=packed.device)
+    _check(lib().zoqat_op_unpack_operand_i8(_p(packed), _p(qparams), rows, cols, bits, _p(operand), _p(steps), _p(err), _stream()))
+    return operand, steps, err
 
 
 def zoqat_op_update(w, seed, tensor_id, scale):
@@ -502,6 +514,17 @@ class ZoqatModel:
 
     def zoqat_prequantize_frozen(self):
         _check(lib().zoqat_prequantize_frozen(self.handle, _stream()))
+
+    def zoqat_expand_frozen(self, on=True):
+        """Expands the packed tensors once into byte operands (buffer kept alive by this object); on=False undoes it."""
+        if not on:
+            _check(lib().zoqat_expand_frozen(self.handle, None, 0, _stream()))
+            self.expand_buffer = None
+            return
+        nb = ctypes.c_size_t()
+        _check(lib().zoqat_expand_frozen_bytes(self.handle, ctypes.byref(nb)))
+        self.expand_buffer = torch.empty(nb.value, dtype=torch.uint8, device="cuda")
+        _check(lib().zoqat_expand_frozen(self.handle, _p(self.expand_buffer), nb.value, _stream()))
 
     def zoqat_decode_begin(self, batch, max_len):
         """Allocates the decode buffer (kept alive by this object) and converts the packed model for decoding."""

@@ -52,6 +52,9 @@ struct Linear {
     const uint32_t* packed = nullptr;
     const float2* qparams = nullptr;
     float* theta = nullptr;             // Section 4.2: learnable (step, zero point, alpha, beta) per group
+    // zoqat_expand_frozen (8-bit integer GEMM): the packed tensor as signed bytes code - zero point, and its rows' steps
+    const uint8_t* expanded = nullptr;
+    const float* expanded_step = nullptr;
     bool present = false;
     bool adaptive() const { return theta != nullptr; }
     uint32_t tid_q() const { return tid + 0x10000u; }
@@ -261,7 +264,8 @@ int run_gemm(zoqat_model* m, GemmArgs& g, cudaStream_t s) {
     g.err_flag = m->ws.err_flag;
     g.single_cta = m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_1CTA;
     if (m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_I8 && g.mode != 1) {     // every block linear; the vocabulary projection stays bf16
-        g.int8 = 1; g.col_step = m->ws.col_step; g.col_stride = (size_t)m->ws.bias_ld;
+        g.int8 = 1;
+        if (!g.col_step) { g.col_step = m->ws.col_step; g.col_stride = (size_t)m->ws.bias_ld; }
     }
     const int rc = (m->cfg.gemm_impl == ZOQAT_GEMM_SIMT) ? launch_gemm_simt(g, s) : launch_gemm_tc(g, s);
     if (rc != ZOQAT_OK) return fail(rc, "GEMM launch rejected (M=%lld N=%lld K=%lld)", (long long)g.M, (long long)g.N, (long long)g.K);
@@ -287,6 +291,22 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
         uint8_t* base = reinterpret_cast<uint8_t*>(m->ws.bop) + (dst - m->ws.bop);
         dst = reinterpret_cast<__nv_bfloat16*>(base);
         pass_stride /= 2;                             // added to a bf16 pointer below
+    }
+    if (L.packed_frozen() && i8 && L.expanded) {
+        // expanded once (zoqat_expand_frozen): bytes and steps are copied next to the operands of the trainable tensors
+        // that share this GEMM (a GEMM whose tensors are all expanded reads them in place and never gets here)
+        for (int pz = 0; pz < passes; ++pz) {
+            cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dst) + (size_t)pz * 2 * pass_stride, L.expanded, (size_t)n, cudaMemcpyDeviceToDevice, s);
+            cudaMemcpyAsync(m->ws.col_step + bias_off + (size_t)pz * m->ws.bias_ld, L.expanded_step, (size_t)L.rows * 4, cudaMemcpyDeviceToDevice, s);
+        }
+        return;
+    }
+    if (L.packed_frozen() && m->cfg.w_group == 0) {
+        // one group per row: bf16 operand, or the signed bytes and the rows' steps; the second pass sees the same tensor
+        launch_unpack_rows(L.packed, L.qparams, L.rows, L.cols, m->cfg.w_bits, dst, i8, m->ws.col_step + bias_off, m->ws.bias_ld,
+                           passes, m->ws.err_flag, s);
+        if (passes == 2) cudaMemcpyAsync(dst + pass_stride, dst, (size_t)n * (i8 ? 1 : 2), cudaMemcpyDeviceToDevice, s);
+        return;
     }
     if (smoothing || per_channel || (L.adaptive() && bits != 0)) {
         LearnedOperandArgs a{};
@@ -364,6 +384,19 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     const bool i8 = c.gemm_impl == ZOQAT_GEMM_TCGEN05_I8;      // block linears on signed bytes (pair kernel otherwise as 0)
     const bool pair = c.gemm_impl == ZOQAT_GEMM_TCGEN05 || i8;
     const int planes = i8 ? 2 : 0;
+    // A GEMM whose tensors were all expanded by zoqat_expand_frozen reads them in place: they are the same in both passes,
+    // so the passes run as one product over all materialised rows.
+    auto all_expanded = [&](const Layer& Ly_, int r0, int r1) {
+        if (!i8) return false;
+        for (int r = r0; r <= r1; ++r)
+            if (Ly_.lin[r].present && !(Ly_.lin[r].packed_frozen() && Ly_.lin[r].expanded)) return false;
+        return true;
+    };
+    auto use_expanded = [&](GemmArgs& g_, const Linear& first, int Z_) {
+        g_.B = reinterpret_cast<const __nv_bfloat16*>(first.expanded);
+        g_.col_step = first.expanded_step; g_.col_stride = (size_t)g_.N;
+        g_.M = (int64_t)Z_ * g_.M; g_.Z = 1; g_.b_stride = (size_t)g_.N * g_.K; g_.bias_stride = 0;
+    };
     if (m->cap) {
         const size_t need = capture_forward_bytes(m, T, passes);
         if (need > m->cap_bytes) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "capture buffer %zu < %zu bytes", m->cap_bytes, need);
@@ -421,7 +454,8 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           launch_norm_act_operand(w.h, R, d, norm_kind, Ly.vec[ZOQAT_ROLE_ATTN_NORM_G], Ly.vec[ZOQAT_ROLE_ATTN_NORM_B],
                                   c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(0), false, planes);
           capture_finish(m, nullptr, R, d, s); }
-        for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV; ++r)
+        const bool qkv_exp = all_expanded(Ly, ZOQAT_ROLE_WQ, ZOQAT_ROLE_WV);
+        for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV && !qkv_exp; ++r)
             produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
                             Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend, i8);
         GemmArgs g{};
@@ -438,6 +472,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             g.seq = seq; g.n_heads = H; g.d_head = dh;
             g.cos_t = llama ? w.rope_cos : nullptr; g.sin_t = llama ? w.rope_sin : nullptr;
         }
+        if (qkv_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_WQ], Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s);
           if (c.gemm_impl == ZOQAT_GEMM_SIMT) {
@@ -449,11 +484,13 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1), false, planes);
           capture_finish(m, w.att, R, d, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend, i8);
+        const bool o_exp = all_expanded(Ly, ZOQAT_ROLE_WO, ZOQAT_ROLE_WO);
+        if (!o_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
+        if (o_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_WO], Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         // --- feed-forward block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
@@ -461,8 +498,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                   c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(2), false, planes);
           capture_finish(m, nullptr, R, d, s); }
         const int n_up = llama ? 2 * F : F;
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend, i8);
-        if (llama) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend, i8);
+        const bool up_exp = all_expanded(Ly, ZOQAT_ROLE_W_GATE, ZOQAT_ROLE_W_UP);
+        if (!up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend, i8);
+        if (llama && !up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
@@ -474,6 +512,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             cudaMemsetAsync(w.row_amax, 0, (size_t)R * 4, s);
             g.mode = 3; g.row_amax = w.row_amax;
         }
+        if (up_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_W_GATE], Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
@@ -481,11 +520,13 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           else if (fuse_gate) launch_rows_operand(w.ffn, R, F, w.row_amax, c.a_bits, w.xa, w.row_step, s, planes);
           else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3), false, planes, capture_input(m));
           capture_finish(m, fuse_gate ? w.ffn : nullptr, R, F, s); }
-        produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend, i8);
+        const bool down_exp = all_expanded(Ly, ZOQAT_ROLE_W_DOWN, ZOQAT_ROLE_W_DOWN);
+        if (!down_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
+        if (down_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_W_DOWN], Z);
         if (int rc = run_gemm(m, g, s)) return rc;
     }
     if (passes == 2 && Z == 1) {
@@ -623,11 +664,11 @@ int zoqat_query_workspace(const zoqat_config_t* cfg, size_t* bytes) {
 }
 
 int zoqat_packed_bytes(int64_t rows, int64_t cols, int bits, int group, size_t* code_bytes, size_t* qparam_bytes) {
-    if (rows <= 0 || cols <= 0 || (bits != 2 && bits != 3 && bits != 4) || (group != 32 && group != 64 && group != 128))
+    if (rows <= 0 || cols <= 0 || (bits != 2 && bits != 3 && bits != 4) || (group != 0 && group != 32 && group != 64 && group != 128))
         return fail(ZOQAT_ERR_INVALID_ARG, "bad packed-size query");
-    if (cols % group || (rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128 and cols of the group");
+    if (cols % (group ? group : 128) || (rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128 and cols of the group (of 128 with one group per row)");
     if (code_bytes) *code_bytes = (size_t)(rows * cols / 128) * 16 * bits;
-    if (qparam_bytes) *qparam_bytes = (size_t)(rows * cols / group) * 8;
+    if (qparam_bytes) *qparam_bytes = (size_t)(group ? rows * cols / group : rows) * 8;
     return ZOQAT_OK;
 }
 
@@ -680,7 +721,7 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
                 if (is_packed) {
                     if (!t.packed || !t.qparams) { delete m; return fail(ZOQAT_ERR_INVALID_ARG, "tensor %d: packed/qparams are NULL", i); }
                     if ((L.rows * L.cols) % 128) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need rows*cols %% 128 == 0", i); }
-                    if (cfg->w_bits > 4 || cfg->w_group == 0) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need w_bits <= 4 and a column group of 32, 64 or 128", i); }
+                    if (cfg->w_bits > 4) { delete m; return fail(ZOQAT_ERR_UNSUPPORTED, "tensor %d: packed tensors need w_bits <= 4", i); }
                     L.packed = static_cast<const uint32_t*>(t.packed);
                     L.qparams = static_cast<const float2*>(t.qparams);
                     m->any_packed = true;
@@ -742,9 +783,9 @@ int zoqat_model_create(const zoqat_config_t* cfg, const zoqat_tensor_desc_t* ten
         for (int r = 0; r < 7; ++r) if (Ly.lin[r].adaptive()) m->any_learnable = true;
         if (cfg->gemm_impl == ZOQAT_GEMM_TCGEN05_I8)
             for (int r = 0; r < 7; ++r)
-                if (Ly.lin[r].present && (Ly.lin[r].bits(cfg->w_bits) == 0 || Ly.lin[r].packed_frozen())) {
+                if (Ly.lin[r].present && Ly.lin[r].bits(cfg->w_bits) == 0) {
                     delete m;
-                    return fail(ZOQAT_ERR_UNSUPPORTED, "layer %d: the 8-bit integer GEMM needs every block linear QUANTIZED and not FROZEN_PACKED", l);
+                    return fail(ZOQAT_ERR_UNSUPPORTED, "layer %d: the 8-bit integer GEMM needs every block linear QUANTIZED or FROZEN_PACKED", l);
                 }
     }
     // one-time tables: rotary cos/sin (evaluated in double, stored fp32) and concatenated q|k|v biases
@@ -791,11 +832,57 @@ int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream) {
             Linear& L = Ly.lin[r];
             if (!L.present || !L.packed_frozen()) continue;
             if (!L.w) return fail(ZOQAT_ERR_BAD_STATE, "frozen tensor has no fp32 source to quantise");
-            launch_pack_frozen(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, const_cast<uint32_t*>(L.packed),
-                               const_cast<float2*>(L.qparams), s);
+            if (m->cfg.w_group == 0)
+                launch_pack_frozen_rows(L.w, L.rows, L.cols, m->cfg.w_bits, const_cast<uint32_t*>(L.packed), const_cast<float2*>(L.qparams), s);
+            else
+                launch_pack_frozen(L.w, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, const_cast<uint32_t*>(L.packed),
+                                   const_cast<float2*>(L.qparams), s);
         }
     CUDA_TRY(cudaGetLastError());
     m->prequantized = true;
+    return ZOQAT_OK;
+}
+
+int zoqat_expand_frozen_bytes(const zoqat_model_t* m, size_t* bytes) {
+    if (!m || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    size_t n = 0;
+    for (const auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r)
+            if (Ly.lin[r].present) n += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols) + (size_t)Ly.lin[r].rows * 4;
+    *bytes = align_up(n);
+    return ZOQAT_OK;
+}
+
+int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* stream) {
+    if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
+    if (m->cfg.gemm_impl != ZOQAT_GEMM_TCGEN05_I8) return fail(ZOQAT_ERR_UNSUPPORTED, "byte operands belong to ZOQAT_GEMM_TCGEN05_I8");
+    if (m->any_packed && !m->prequantized) return fail(ZOQAT_ERR_BAD_STATE, "call zoqat_prequantize_frozen first");
+    size_t need = 0;
+    zoqat_expand_frozen_bytes(m, &need);
+    if (!buffer_dev) {                       // back to expanding on every step
+        for (auto& Ly : m->layers) for (int r = 0; r < 7; ++r) { Ly.lin[r].expanded = nullptr; Ly.lin[r].expanded_step = nullptr; }
+        return ZOQAT_OK;
+    }
+    if (bytes < need) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "expansion buffer %zu < %zu bytes", bytes, need);
+    if (reinterpret_cast<uintptr_t>(buffer_dev) & 255) return fail(ZOQAT_ERR_INVALID_ARG, "buffer_dev must be 256-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // all byte operands first (the tensors of one GEMM back to back: q | k | v, o, gate | up, down), then all steps in the same order
+    size_t total_bytes = 0;
+    for (const auto& Ly : m->layers) for (int r = 0; r < 7; ++r) if (Ly.lin[r].present) total_bytes += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols);
+    uint8_t* pb = static_cast<uint8_t*>(buffer_dev);
+    float* pstep = reinterpret_cast<float*>(pb + total_bytes);      // total_bytes is a multiple of 4096
+    for (auto& Ly : m->layers)
+        for (int r = 0; r < 7; ++r) {
+            Linear& L = Ly.lin[r];
+            if (!L.present) continue;
+            if (L.packed_frozen()) {
+                launch_unpack_rows(L.packed, L.qparams, L.rows, L.cols, m->cfg.w_bits, pb, true, pstep, 0, 1, m->ws.err_flag, s);
+                L.expanded = pb; L.expanded_step = pstep;
+            }
+            pb += (size_t)(L.rows * L.cols);
+            pstep += L.rows;
+        }
+    CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
 
@@ -1253,20 +1340,42 @@ int zoqat_op_init_qparams(const float* w_dev, int64_t rows, int64_t cols, int gr
 
 int zoqat_op_pack_frozen(const float* w_dev, int64_t rows, int64_t cols, int group, int bits, void* packed_dev,
                          void* qparams_dev, void* stream) {
-    if (int rc = check_group_bits(rows, cols, group, bits, false, 4)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 4, true)) return rc;
     if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
     if (!w_dev || !packed_dev || !qparams_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (group == 0) {
+        launch_pack_frozen_rows(w_dev, rows, cols, bits, static_cast<uint32_t*>(packed_dev), static_cast<float2*>(qparams_dev),
+                                static_cast<cudaStream_t>(stream));
+        CUDA_TRY(cudaGetLastError());
+        return ZOQAT_OK;
+    }
     launch_pack_frozen(w_dev, rows * cols, group, bits, static_cast<uint32_t*>(packed_dev), static_cast<float2*>(qparams_dev),
                        static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
 }
 
+int zoqat_op_unpack_operand_i8(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int bits,
+                               void* operand_dev, float* col_step_dev, int32_t* err_flag_dev, void* stream) {
+    if (int rc = check_group_bits(rows, cols, 0, bits, false, 4, true)) return rc;
+    if (!packed_dev || !qparams_dev || !operand_dev || !col_step_dev || !err_flag_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    launch_unpack_rows(static_cast<const uint32_t*>(packed_dev), static_cast<const float2*>(qparams_dev), rows, cols, bits, operand_dev,
+                       true, col_step_dev, rows, 1, err_flag_dev, static_cast<cudaStream_t>(stream));
+    CUDA_TRY(cudaGetLastError());
+    return ZOQAT_OK;
+}
+
 int zoqat_op_unpack_operand(const void* packed_dev, const void* qparams_dev, int64_t rows, int64_t cols, int group,
                             int bits, void* operand_dev, void* stream) {
-    if (int rc = check_group_bits(rows, cols, group, bits, false, 4)) return rc;
+    if (int rc = check_group_bits(rows, cols, group, bits, false, 4, true)) return rc;
     if ((rows * cols) % 128) return fail(ZOQAT_ERR_UNSUPPORTED, "rows*cols must be a multiple of 128");
     if (!packed_dev || !qparams_dev || !operand_dev) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    if (group == 0) {
+        launch_unpack_rows(static_cast<const uint32_t*>(packed_dev), static_cast<const float2*>(qparams_dev), rows, cols, bits, operand_dev,
+                           false, nullptr, 0, 0, nullptr, static_cast<cudaStream_t>(stream));
+        CUDA_TRY(cudaGetLastError());
+        return ZOQAT_OK;
+    }
     launch_unpack_operand(static_cast<const uint32_t*>(packed_dev), static_cast<const float2*>(qparams_dev), rows * cols,
                           group, bits, static_cast<__nv_bfloat16*>(operand_dev), static_cast<cudaStream_t>(stream));
     CUDA_TRY(cudaGetLastError());

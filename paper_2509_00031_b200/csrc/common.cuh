@@ -121,6 +121,11 @@ void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* 
 void launch_init_qparams_rows(const float* w, int64_t rows, int64_t cols, int bits, float* theta, cudaStream_t s);   // one group per row
 void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s);
 void launch_pack_frozen(const float* w, int64_t n, int group, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);
+// One group per output row (cols % 128 == 0): qparams holds one (step, zero point) per row.  Unpacking gives the bf16
+// operand, or (i8) the signed bytes code - zero point with the rows' steps in col_step[sign * col_stride + row].
+void launch_pack_frozen_rows(const float* w, int64_t rows, int64_t cols, int bits, uint32_t* packed, float2* qparams, cudaStream_t s);
+void launch_unpack_rows(const uint32_t* packed, const float2* qparams, int64_t rows, int64_t cols, int bits, void* op, bool i8,
+                        float* col_step, int64_t col_stride, int signs, int32_t* err_flag, cudaStream_t s);
 void launch_unpack_operand(const uint32_t* packed, const float2* qparams, int64_t n, int group, int bits,
                            __nv_bfloat16* op, cudaStream_t s);
 // w <- w - scale*u; scale = *scale_ptr if scale_ptr != NULL else scale_val.

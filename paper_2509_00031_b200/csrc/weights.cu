@@ -839,6 +839,99 @@ unpack_operand_kernel(const uint32_t* __restrict__ packed, const float2* __restr
     }
 }
 
+// ---- packed frozen tensors with one quantisation group per output row --------------------------------------------
+// (step, zero point) of every row by the min/max scheme of Section 2: one CTA per row.
+__global__ void __launch_bounds__(kThreads)
+row_qparams_kernel(const float4* __restrict__ w, int rows, int cols4, int bits, float2* __restrict__ qparams) {
+    __shared__ float red[2][kThreads / 32];
+    const float qp = (float)((1 << bits) - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        float mn = INFINITY, mx = -INFINITY;
+        for (int c = threadIdx.x; c < cols4; c += kThreads) {
+            const float4 v = __ldg(w + (int64_t)r * cols4 + c);
+            mn = fminf(mn, fminf(fminf(v.x, v.y), fminf(v.z, v.w)));
+            mx = fmaxf(mx, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        __syncthreads();
+        if (lane == 0) { red[0][warp] = mn; red[1][warp] = mx; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int i = 1; i < kThreads / 32; ++i) { mn = fminf(mn, red[0][i]); mx = fmaxf(mx, red[1][i]); }
+            const GroupQ g = group_params(mn, mx, qp);
+            qparams[r] = make_float2(g.step, g.zp);
+        }
+    }
+}
+
+// pack_frozen_kernel with the rows' (step, zero point) given (row_qparams_kernel): same bit-plane layout.
+__global__ void __launch_bounds__(kThreads)
+pack_frozen_rows_kernel(const float4* __restrict__ w, int64_t n4, int cols4, int bits, uint32_t* __restrict__ packed,
+                        const float2* __restrict__ qparams) {
+    const float qp = (float)((1 << bits) - 1);
+    const int lane = threadIdx.x & 31;
+    const int64_t n4_ceil = (n4 + 31) & ~(int64_t)31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4_ceil; i += (int64_t)gridDim.x * blockDim.x) {
+        const bool live = i < n4;
+        const float4 x = live ? __ldg(w + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float2 q = live ? __ldg(qparams + i / cols4) : make_float2(1.f, 0.f);
+        GroupQ g;
+        g.step = q.x; g.inv = __fdiv_rn(1.0f, q.x); g.zp = q.y;
+        const uint32_t c[4] = {(uint32_t)quant_code(x.x, g, qp), (uint32_t)quant_code(x.y, g, qp),
+                               (uint32_t)quant_code(x.z, g, qp), (uint32_t)quant_code(x.w, g, qp)};
+        const int64_t chunk = i >> 5;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            for (int b = 0; b < bits; ++b) {
+                const uint32_t word = __ballot_sync(0xffffffffu, (c[j] >> b) & 1u);
+                if (lane == j * bits + b) packed[chunk * (4 * bits) + lane] = word;
+            }
+    }
+}
+
+// Packed codes of per-row groups -> the matmul operand: bf16 (c - z) * step, or (I8) the signed bytes c - z with the rows'
+// steps to col_step[sign * col_stride + row] for `signs` passes (the frozen tensor is the same in both); a row whose
+// c - z leaves [-128, 127] sets kErrCodeRange.
+template <int BITS, bool I8>
+__global__ void __launch_bounds__(kThreads)
+unpack_rows_kernel(const uint32_t* __restrict__ packed, const float2* __restrict__ qparams, int64_t n4, int cols4,
+                   void* __restrict__ op, float* __restrict__ col_step, int64_t col_stride, int signs, int32_t* err_flag) {
+    const int lane = threadIdx.x & 31;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint4* run = reinterpret_cast<const uint4*>(packed + (i >> 5) * (4 * BITS));
+        uint32_t wd[4 * BITS];
+#pragma unroll
+        for (int q = 0; q < BITS; ++q) {
+            const uint4 t = __ldg(run + q);
+            wd[4 * q] = t.x; wd[4 * q + 1] = t.y; wd[4 * q + 2] = t.z; wd[4 * q + 3] = t.w;
+        }
+        const int64_t row = i / cols4;
+        const float2 qpv = __ldg(qparams + row);
+        float v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t c = 0;
+#pragma unroll
+            for (int b = 0; b < BITS; ++b) c |= ((wd[j * BITS + b] >> lane) & 1u) << b;
+            v[j] = __fadd_rn((float)c, -qpv.y);
+        }
+        if (I8) {
+            reinterpret_cast<uint32_t*>(op)[i] = pack_s8x4(v[0], v[1], v[2], v[3]);
+            if (i - row * cols4 == 0) {
+                for (int sg = 0; sg < signs; ++sg) col_step[(int64_t)sg * col_stride + row] = qpv.x;
+                if (!(-qpv.y >= -128.0f && (float)((1 << BITS) - 1) - qpv.y <= 127.0f)) atomicExch(err_flag, kErrCodeRange);
+            }
+        } else {
+            reinterpret_cast<uint2*>(op)[i] = pack_bf16x4(__fmul_rn(v[0], qpv.x), __fmul_rn(v[1], qpv.x), __fmul_rn(v[2], qpv.x), __fmul_rn(v[3], qpv.x));
+        }
+    }
+}
+
 // Eq. (2): w <- w - scale*u, one fused multiply-add per element.
 __global__ void __launch_bounds__(kThreads)
 update_kernel(float* __restrict__ w, uint64_t n, const PhiloxKeys rk, uint32_t tid,
@@ -1137,6 +1230,34 @@ void launch_init_qparams(const float* w, int64_t n, int group, int bits, float* 
 
 void launch_class_scales(const float* proj_grad, float lr_quant, float lr_smooth, float* out, cudaStream_t s) {
     class_scales_kernel<<<1, 1, 0, s>>>(proj_grad, lr_quant, lr_smooth, out);
+    count_launch();
+}
+
+void launch_pack_frozen_rows(const float* w, int64_t rows, int64_t cols, int bits, uint32_t* packed, float2* qparams, cudaStream_t s) {
+    if (rows * cols == 0) return;
+    const float4* w4 = reinterpret_cast<const float4*>(w);
+    const int rgrid = (int)(rows < 148 * 8 ? rows : 148 * 8);
+    row_qparams_kernel<<<rgrid, kThreads, 0, s>>>(w4, (int)rows, (int)(cols / 4), bits, qparams);
+    const int64_t n4 = rows * cols / 4;
+    pack_frozen_rows_kernel<<<stream_grid(n4, kThreads), kThreads, 0, s>>>(w4, n4, (int)(cols / 4), bits, packed, qparams);
+    count_launch(2);
+}
+
+void launch_unpack_rows(const uint32_t* packed, const float2* qparams, int64_t rows, int64_t cols, int bits, void* op, bool i8,
+                        float* col_step, int64_t col_stride, int signs, int32_t* err_flag, cudaStream_t s) {
+    if (rows * cols == 0) return;
+    const int64_t n4 = rows * cols / 4;
+    const int grid = stream_grid(n4, kThreads);
+    const int c4 = (int)(cols / 4);
+    if (i8) {
+        if (bits == 2) unpack_rows_kernel<2, true><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, col_step, col_stride, signs, err_flag);
+        else if (bits == 3) unpack_rows_kernel<3, true><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, col_step, col_stride, signs, err_flag);
+        else unpack_rows_kernel<4, true><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, col_step, col_stride, signs, err_flag);
+    } else {
+        if (bits == 2) unpack_rows_kernel<2, false><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, nullptr, 0, 0, nullptr);
+        else if (bits == 3) unpack_rows_kernel<3, false><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, nullptr, 0, 0, nullptr);
+        else unpack_rows_kernel<4, false><<<grid, kThreads, 0, s>>>(packed, qparams, n4, c4, op, nullptr, 0, 0, nullptr);
+    }
     count_launch();
 }
 

@@ -46,6 +46,11 @@ WORKLOADS = {
                                          adaptive_quant=True, smoothing=True, integer_gemm=True),
     "llama7b_w6a6_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
                                          w_bits=6, w_group=0, a_bits=6, batch=4, seq=1024, bf16_init=True, integer_gemm=True),
+    # Section 4.3 as the paper runs it, in its weight-activation setting, on the integer GEMM: query and value projections
+    # trainable, everything else packed (expanded straight into byte operands: no per-step work on the frozen weights)
+    "llama7b_qv_light_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
+                                             w_bits=4, w_group=0, a_bits=8, batch=4, seq=1024, bf16_init=True,
+                                             trainable_names=("wq", "wv"), head_trainable=False, integer_gemm=True),
     "llama7b_w4a8_perchannel_int8": dict(arch="llama", n_layers=32, d_model=4096, n_heads=32, d_ffn=11008, vocab=32000,
                                          w_bits=4, w_group=0, a_bits=8, batch=4, seq=1024, bf16_init=True, integer_gemm=True),
 }

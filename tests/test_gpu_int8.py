@@ -165,6 +165,33 @@ def test_act_operand_i8_is_the_bf16_operand_as_bytes(zq, kind, cols, a_bits):
         assert np.array_equal(op8.cpu().numpy().astype(np.float64), q) and np.array_equal(st8.cpu().numpy(), st)
 
 
+@pytest.mark.parametrize("bits,rows,cols", [(4, 96, 512), (2, 37, 4096), (3, 130, 1408), (4, 64, 11008)])
+def test_pack_unpack_frozen_per_row(zq, bits, rows, cols):
+    """Section 4.3 packing with one group per output row: the rows' (step, zero point), the bit planes (decoded here to
+    the oracle's codes), the bf16 operand and the signed-byte operand with the rows' steps."""
+    rng = np.random.default_rng(bits + cols)
+    w = (rng.standard_normal((rows, cols)) * 0.02).astype(F32)
+    w[5] *= 3.0
+    packed, qparams = zq.zoqat_op_pack_frozen(dev(w), 0, bits)
+    assert packed.numel() == rows * cols * bits // 8 and qparams.numel() == 2 * rows
+    o_codes, o_step, o_zp, o_deq = core.weight_quant(w, cols, bits)
+    qp = qparams.cpu().numpy().reshape(-1, 2)
+    assert np.array_equal(qp[:, 0].view(np.uint32), o_step.ravel().view(np.uint32)) and np.array_equal(qp[:, 1], o_zp.ravel().astype(F32))
+    words = packed.cpu().numpy().view(np.uint32).reshape(-1, 4, bits)
+    lanes = np.arange(32, dtype=np.uint32)
+    dec = np.zeros((words.shape[0], 32, 4), np.uint8)
+    for j in range(4):
+        for b in range(bits):
+            dec[:, :, j] |= (((words[:, j, b][:, None] >> lanes[None, :]) & 1) << b).astype(np.uint8)
+    assert np.array_equal(dec.reshape(rows, cols), o_codes)
+    op = zq.zoqat_op_unpack_operand(packed, qparams, rows, cols, 0, bits)
+    assert np.array_equal(op.float().cpu().numpy(), core.round_bf16(o_deq))
+    op8, steps, err = zq.zoqat_op_unpack_operand_i8(packed, qparams, rows, cols, bits)
+    assert int(err.item()) == 0
+    assert np.array_equal(op8.cpu().numpy().astype(np.int64), o_codes.astype(np.int64) - o_zp.astype(np.int64))
+    assert np.array_equal(steps.cpu().numpy().view(np.uint32), o_step.ravel().view(np.uint32))
+
+
 # ---- the model ---------------------------------------------------------------------------------------------------
 I8_LLAMA = dict(arch="llama", n_layers=2, d_model=256, n_heads=2, d_ffn=384, vocab=500, w_bits=4, w_group=0, a_bits=8)
 I8_LLAMA_W6A6 = dict(arch="llama", n_layers=2, d_model=128, n_heads=2, d_ffn=384, vocab=500, w_bits=6, w_group=0, a_bits=6)
@@ -236,6 +263,78 @@ def test_frozen_first_layer_and_step_multi(zq):
     for k, wb in frozen.items():
         assert np.array_equal(model.params["layers"][0][k].cpu().numpy(), wb), k
     assert not np.array_equal(model.params["layers"][1]["wq"].cpu().numpy(), frozen["wq"])
+
+
+@pytest.mark.parametrize("impl_i8", [True, False], ids=["integer", "bf16"])
+@pytest.mark.parametrize("names", [None, ("wq", "wv")], ids=["packed_first_layer", "query_value_only"])
+def test_lightweight_variant_per_row(zq, impl_i8, names):
+    """Section 4.3 with one weight group per output row: frozen tensors packed (expanded into byte operands on the integer
+    GEMM, into bf16 operands otherwise), either the whole first layer or everything but the query and value projections."""
+    import dataclasses
+    shape, batch, seq = I8_LLAMA, 2, 96
+    first = 1 if names is None else 0
+    params = synth.make_params(shape, seed=3, max_seq=seq, jitter=True)
+    oracle = OracleModel(oracle_cfg(shape, first_trainable_layer=first, trainable_names=names, head_trainable=names is None,
+                                    integer_gemm=impl_i8), synth.copy_params(params))
+    model = zq.ZoqatModel(shape, zq.params_to_device(synth.copy_params(params)), max_batch=batch, max_seq=seq,
+                          gemm_impl=zq.GEMM_TCGEN05_I8 if impl_i8 else zq.GEMM_TCGEN05, first_trainable_layer=first,
+                          packed_frozen=True, trainable_names=names, head_trainable=names is None)
+    model.zoqat_prequantize_frozen()
+    tokens, labels = synth.make_batch(batch, seq, shape["vocab"], seed=31)
+    for seed, eps in [(3, 0.0), (3, 1e-3)]:
+        got = float(model.zoqat_forward_loss(dev(tokens), dev(labels), seed, eps).item())
+        model.zoqat_check()
+        want = oracle.loss(tokens, labels, seed, float(F32(eps)))
+        assert abs(got - want) <= 1e-4 * abs(want), (seed, eps, got, want)
+    recs = []
+    for t in range(3):
+        seed = 900 + t
+        for l in range(shape["n_layers"]):
+            for k in oracle.linear_names():
+                if oracle.is_trainable(l, k):
+                    model.params["layers"][l][k].copy_(torch.from_numpy(oracle.p["layers"][l][k]))
+        model.params["lm_head"].copy_(torch.from_numpy(oracle.p["lm_head"]))
+        oa32 = OracleModel(dataclasses.replace(oracle.cfg, accum_f32=True), oracle.p)
+        ga32 = float(oa32.projected_gradient(tokens, labels, seed, 1e-3)[2])
+        before = oracle.p["layers"][1]["wq"].copy()
+        res = zq.decode_step_result(model.zoqat_step_deferred(dev(tokens), dev(labels), seed, 1e-3, 1e-4))
+        model.zoqat_flush_update()
+        model.zoqat_check()
+        lp, lm, g = oracle.step(tokens, labels, seed, 1e-3, 1e-4)
+        assert res["status"] == 0 and abs(res["loss_plus"] - lp) <= 1e-3 * abs(lp) and abs(res["loss_minus"] - lm) <= 1e-3 * abs(lm)
+        want_w = core.update_(before.reshape(-1), seed, 16 * 2 + 0, F32(res["update_scale"])).reshape(before.shape)
+        assert np.array_equal(model.params["layers"][1]["wq"].cpu().numpy().view(np.uint32), want_w.view(np.uint32))
+        recs.append(dict(g=float(g), g32=ga32, ga32=ga32, g_gpu=res["proj_grad"]))
+    check_g(recs, f"per-row lightweight {'integer' if impl_i8 else 'bf16'} {names}")
+    if impl_i8:
+        # the packed tensors expanded once: linears that are all frozen read them in place (both passes as one product),
+        # a frozen key projection is copied next to the trainable query / value operands - the same bits either way
+        t, l = dev(tokens), dev(labels)
+        trainable = [(li, k) for li in range(shape["n_layers"]) for k in oracle.linear_names() if oracle.is_trainable(li, k)]
+        snap = {key: model.params["layers"][key[0]][key[1]].clone() for key in trainable}
+        snap_head = model.params["lm_head"].clone()
+        a = model.zoqat_forward_loss(t, l, 77, 1e-3).clone()
+        ra = model.zoqat_step(t, l, 78, 1e-3, 1e-4).clone()
+        wa = model.params["layers"][1]["wq"].clone()
+        for key in trainable:
+            model.params["layers"][key[0]][key[1]].copy_(snap[key])
+        model.params["lm_head"].copy_(snap_head)
+        model.zoqat_expand_frozen()
+        b = model.zoqat_forward_loss(t, l, 77, 1e-3).clone()
+        rb = model.zoqat_step(t, l, 78, 1e-3, 1e-4).clone()
+        model.zoqat_check()
+        assert torch.equal(a, b) and torch.equal(ra.view(torch.int32), rb.view(torch.int32))
+        assert torch.equal(wa, model.params["layers"][1]["wq"])
+        launches_before = model.zoqat_launch_count()
+        model.zoqat_forward_loss(t, l, 77, 1e-3)
+        with_cache = model.zoqat_launch_count() - launches_before
+        model.zoqat_expand_frozen(False)
+        launches_before = model.zoqat_launch_count()
+        model.zoqat_forward_loss(t, l, 77, 1e-3)
+        assert model.zoqat_launch_count() - launches_before > with_cache          # the per-step expansions are back
+    # frozen tensors never move
+    frozen_name = "wk" if names else "wq"
+    assert np.array_equal(model.params["layers"][0][frozen_name].cpu().numpy(), params["layers"][0][frozen_name])
 
 
 @pytest.mark.parametrize("shape,learned", [(I8_LLAMA, True), (I8_LLAMA_W6A6, False)], ids=["llama_learned", "llama_w6a6_minmax"])
