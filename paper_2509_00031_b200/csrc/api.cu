@@ -397,6 +397,16 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
         g_.col_step = first.expanded_step; g_.col_stride = (size_t)g_.N;
         g_.M = (int64_t)Z_ * g_.M; g_.Z = 1; g_.b_stride = (size_t)g_.N * g_.K; g_.bias_stride = 0;
     };
+    // The same for packed tensors that are decoded on every step (any GEMM kind): one operand, one product over all rows,
+    // instead of a copy of the operand for the second pass.
+    auto all_frozen = [&](const Layer& Ly_, int r0, int r1) {
+        for (int r = r0; r <= r1; ++r)
+            if (Ly_.lin[r].present && !Ly_.lin[r].packed_frozen()) return false;
+        return true;
+    };
+    auto one_product = [&](GemmArgs& g_, int Z_) {
+        g_.M = (int64_t)Z_ * g_.M; g_.Z = 1; g_.b_stride = (size_t)g_.N * g_.K; g_.bias_stride = 0;
+    };
     if (m->cap) {
         const size_t need = capture_forward_bytes(m, T, passes);
         if (need > m->cap_bytes) return fail(ZOQAT_ERR_WORKSPACE_SMALL, "capture buffer %zu < %zu bytes", m->cap_bytes, need);
@@ -455,8 +465,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
                                   c.norm_eps, c.a_bits, w.xa, w.row_step, capture_input(m), s, smooth_at(0), false, planes);
           capture_finish(m, nullptr, R, d, s); }
         const bool qkv_exp = all_expanded(Ly, ZOQAT_ROLE_WQ, ZOQAT_ROLE_WV);
+        const bool qkv_one = !qkv_exp && all_frozen(Ly, ZOQAT_ROLE_WQ, ZOQAT_ROLE_WV);
         for (int r = ZOQAT_ROLE_WQ; r <= ZOQAT_ROLE_WV && !qkv_exp; ++r)
-            produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, Z, seed, eps, s, smo, (size_t)r * d,
+            produce_operand(m, Ly.lin[r], w.bop + (size_t)r * d * d, ps, qkv_one ? 1 : Z, seed, eps, s, smo, (size_t)r * d,
                             Ly.vec[ZOQAT_ROLE_BQ + r], r, 0, pend, i8);
         GemmArgs g{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = 3 * d; g.K = d; g.Z = Z;
@@ -473,6 +484,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             g.cos_t = llama ? w.rope_cos : nullptr; g.sin_t = llama ? w.rope_sin : nullptr;
         }
         if (qkv_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_WQ], Z);
+        else if (qkv_one) one_product(g, Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ATTENTION, s);
           if (c.gemm_impl == ZOQAT_GEMM_SIMT) {
@@ -485,12 +497,14 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           launch_norm_act_operand(w.att, R, d, 0, nullptr, nullptr, 0.f, c.a_bits, w.xa, w.row_step, nullptr, s, smooth_at(1), false, planes);
           capture_finish(m, w.att, R, d, s); }
         const bool o_exp = all_expanded(Ly, ZOQAT_ROLE_WO, ZOQAT_ROLE_WO);
-        if (!o_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend, i8);
+        const bool o_one = !o_exp && all_frozen(Ly, ZOQAT_ROLE_WO, ZOQAT_ROLE_WO);
+        if (!o_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_WO], w.bop, ps, o_one ? 1 : Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_BO], ZOQAT_ROLE_WO, 1, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_BO]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         if (o_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_WO], Z);
+        else if (o_one) one_product(g, Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         // --- feed-forward block
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
@@ -499,8 +513,9 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           capture_finish(m, nullptr, R, d, s); }
         const int n_up = llama ? 2 * F : F;
         const bool up_exp = all_expanded(Ly, ZOQAT_ROLE_W_GATE, ZOQAT_ROLE_W_UP);
-        if (!up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend, i8);
-        if (llama && !up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend, i8);
+        const bool up_one = !up_exp && all_frozen(Ly, ZOQAT_ROLE_W_GATE, ZOQAT_ROLE_W_UP);
+        if (!up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_GATE], w.bop, ps, up_one ? 1 : Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC1], ZOQAT_ROLE_W_GATE, 2, pend, i8);
+        if (llama && !up_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_UP], w.bop + (size_t)F * d, ps, up_one ? 1 : Z, seed, eps, s, smo, (size_t)F, nullptr, ZOQAT_ROLE_W_UP, 2, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = n_up; g.K = d; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC1]; g.out = w.ffn; g.b_stride = ps;
@@ -513,6 +528,7 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
             g.mode = 3; g.row_amax = w.row_amax;
         }
         if (up_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_W_GATE], Z);
+        else if (up_one) one_product(g, Z);
         if (int rc = run_gemm(m, g, s)) return rc;
         { ProfScope ps_(m, ZOQAT_PROF_ACT, s);
           // with smoothing the row maxima of the gated epilogue are not those of the shifted and scaled values
@@ -521,12 +537,14 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
           else launch_ffn_act_operand(w.ffn, R, F, llama ? 1 : 0, c.a_bits, w.xa, w.row_step, s, smooth_at(3), false, planes, capture_input(m));
           capture_finish(m, fuse_gate ? w.ffn : nullptr, R, F, s); }
         const bool down_exp = all_expanded(Ly, ZOQAT_ROLE_W_DOWN, ZOQAT_ROLE_W_DOWN);
-        if (!down_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend, i8);
+        const bool down_one = !down_exp && all_frozen(Ly, ZOQAT_ROLE_W_DOWN, ZOQAT_ROLE_W_DOWN);
+        if (!down_exp) produce_operand(m, Ly.lin[ZOQAT_ROLE_W_DOWN], w.bop, ps, down_one ? 1 : Z, seed, eps, s, smo, 0, Ly.vec[ZOQAT_ROLE_B_FC2], ZOQAT_ROLE_W_DOWN, 3, pend, i8);
         g = GemmArgs{};
         g.A = w.xa; g.B = w.bop; g.M = T; g.N = d; g.K = F; g.Z = Z;
         g.row_step = w.row_step; g.bias = Ly.vec[ZOQAT_ROLE_B_FC2]; g.accumulate = 1; g.out = w.h; g.b_stride = ps;
         if (smo) { g.bias = w.bias_pm; g.bias_stride = (size_t)w.bias_ld; }
         if (down_exp) use_expanded(g, Ly.lin[ZOQAT_ROLE_W_DOWN], Z);
+        else if (down_one) one_product(g, Z);
         if (int rc = run_gemm(m, g, s)) return rc;
     }
     if (passes == 2 && Z == 1) {
