@@ -204,8 +204,8 @@ def run_ours(args, w, rank, world, local_rank):
         model.zoqat_init_qparams()
     if any_packed:
         model.zoqat_prequantize_frozen()
-        if w.get("integer_gemm") and not args.simt:
-            model.zoqat_expand_frozen()                    # frozen tensors as byte operands, once: no per-step work on them
+        if not args.packed_only:
+            model.zoqat_expand_frozen()                    # frozen tensors as GEMM operands, once: no per-step work on them
         for l in range(w["n_layers"]):                     # the fp32 copies of packed tensors are no longer needed
             for name in synth.linear_shapes(w):
                 if l < ftl or (names is not None and name not in names):
@@ -307,6 +307,7 @@ def run_ours(args, w, rank, world, local_rank):
         config=dict(workload=args.workload + (f" cut to {w['n_layers']} layers" if args.layers > 0 else ""),
                     l2="inputs larger than L2 (fp32 masters stream from HBM every step)",
                     gemm="simt" if args.simt else ("tcgen05 kind::i8 (block linears) + kind::f16" if i8 else "tcgen05"),
+                    frozen=("none" if not any_packed else ("packed, decoded every step" if args.packed_only else "packed, expanded once into GEMM operands")),
                     mode="batch-sharded replicas" if args.mode == "batch" else "direction-parallel replicas (q = n_gpus, value counts two-point evaluations)",
                     **{k: w[k] for k in ("arch", "n_layers", "d_model", "n_heads", "d_ffn", "vocab", "w_bits", "w_group",
                                          "a_bits", "batch", "seq")}),
@@ -366,6 +367,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b_w4a8")
+    ap.add_argument("--packed-only", action="store_true", help="lightweight workloads: decode the packed frozen tensors on every step instead of expanding them once (saves their 1-2 bytes per weight of device memory)")
     ap.add_argument("--simt", action="store_true", help="use the CUDA-core cross-check GEMM instead of tcgen05")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="time every kernel category, not only the GEMM launches (adds ~1 %% to the step)")

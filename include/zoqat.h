@@ -184,14 +184,15 @@ int zoqat_model_destroy(zoqat_model_t* m);
  * forward when such tensors exist. */
 int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream);
 
-/* ZOQAT_GEMM_TCGEN05_I8 only, optional, after zoqat_prequantize_frozen: expands every FROZEN_PACKED tensor once into the
- * integer GEMM's operand (signed bytes code - zero point, and the rows' steps) inside `buffer_dev` (caller-owned, 256-byte
- * aligned, zoqat_expand_frozen_bytes() bytes: one byte per block-linear weight plus four per output row; in use until the
- * handle is destroyed or the call is repeated; buffer_dev = NULL returns to expanding on every step).  Afterwards a linear
- * layer whose tensors are all frozen reads them in place, both passes as one product, and a frozen tensor that shares a
- * GEMM with trainable ones (a frozen key projection next to trainable query / value projections) is copied instead of
- * decoded: Section 4.3's frozen tensors then cost no arithmetic per step.  Results are bit-identical either way.  A row
- * that does not fit a signed byte is reported through zoqat_check() (status 32). */
+/* Optional, after zoqat_prequantize_frozen: expands every FROZEN_PACKED tensor once into the operand the GEMM reads - the
+ * bf16 values (code - zero point) * step, or with ZOQAT_GEMM_TCGEN05_I8 the signed bytes code - zero point and the rows'
+ * steps - inside `buffer_dev` (caller-owned, 256-byte aligned, zoqat_expand_frozen_bytes() bytes: two bytes per block-linear
+ * weight, or one plus four per output row; in use until the handle is destroyed or the call is repeated; buffer_dev = NULL
+ * returns to decoding the packed codes on every step).  Afterwards a linear layer whose tensors are all frozen reads them in
+ * place, both passes as one product, and a frozen tensor that shares a GEMM with trainable ones (a frozen key projection
+ * next to trainable query / value projections) is copied instead of decoded: Section 4.3's frozen tensors then cost no
+ * arithmetic per step, at the price of the memory the packed form saves.  Results are bit-identical either way.  With byte
+ * operands a row that does not fit a signed byte is reported through zoqat_check() (status 32). */
 int zoqat_expand_frozen_bytes(const zoqat_model_t* m, size_t* bytes);
 int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* stream);
 

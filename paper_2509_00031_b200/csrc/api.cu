@@ -52,7 +52,8 @@ struct Linear {
     const uint32_t* packed = nullptr;
     const float2* qparams = nullptr;
     float* theta = nullptr;             // Section 4.2: learnable (step, zero point, alpha, beta) per group
-    // zoqat_expand_frozen (8-bit integer GEMM): the packed tensor as signed bytes code - zero point, and its rows' steps
+    // zoqat_expand_frozen: the packed tensor as the GEMM reads it - the bf16 operand, or (8-bit integer GEMM) the signed
+    // bytes code - zero point and the rows' steps
     const uint8_t* expanded = nullptr;
     const float* expanded_step = nullptr;
     bool present = false;
@@ -292,12 +293,13 @@ void produce_operand(zoqat_model* m, const Linear& L, __nv_bfloat16* dst, size_t
         dst = reinterpret_cast<__nv_bfloat16*>(base);
         pass_stride /= 2;                             // added to a bf16 pointer below
     }
-    if (L.packed_frozen() && i8 && L.expanded) {
-        // expanded once (zoqat_expand_frozen): bytes and steps are copied next to the operands of the trainable tensors
-        // that share this GEMM (a GEMM whose tensors are all expanded reads them in place and never gets here)
+    if (L.packed_frozen() && L.expanded) {
+        // expanded once (zoqat_expand_frozen): the operand (and, for byte operands, the steps) is copied next to the operands
+        // of the trainable tensors that share this GEMM (a GEMM whose tensors are all expanded reads them in place and
+        // never gets here)
         for (int pz = 0; pz < passes; ++pz) {
-            cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dst) + (size_t)pz * 2 * pass_stride, L.expanded, (size_t)n, cudaMemcpyDeviceToDevice, s);
-            cudaMemcpyAsync(m->ws.col_step + bias_off + (size_t)pz * m->ws.bias_ld, L.expanded_step, (size_t)L.rows * 4, cudaMemcpyDeviceToDevice, s);
+            cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dst) + (size_t)pz * 2 * pass_stride, L.expanded, (size_t)n * (i8 ? 1 : 2), cudaMemcpyDeviceToDevice, s);
+            if (i8) cudaMemcpyAsync(m->ws.col_step + bias_off + (size_t)pz * m->ws.bias_ld, L.expanded_step, (size_t)L.rows * 4, cudaMemcpyDeviceToDevice, s);
         }
         return;
     }
@@ -387,14 +389,13 @@ int forward(zoqat_model* m, const int32_t* tokens, const int32_t* labels, int ba
     // A GEMM whose tensors were all expanded by zoqat_expand_frozen reads them in place: they are the same in both passes,
     // so the passes run as one product over all materialised rows.
     auto all_expanded = [&](const Layer& Ly_, int r0, int r1) {
-        if (!i8) return false;
         for (int r = r0; r <= r1; ++r)
             if (Ly_.lin[r].present && !(Ly_.lin[r].packed_frozen() && Ly_.lin[r].expanded)) return false;
         return true;
     };
     auto use_expanded = [&](GemmArgs& g_, const Linear& first, int Z_) {
         g_.B = reinterpret_cast<const __nv_bfloat16*>(first.expanded);
-        g_.col_step = first.expanded_step; g_.col_stride = (size_t)g_.N;
+        if (i8) { g_.col_step = first.expanded_step; g_.col_stride = (size_t)g_.N; }
         g_.M = (int64_t)Z_ * g_.M; g_.Z = 1; g_.b_stride = (size_t)g_.N * g_.K; g_.bias_stride = 0;
     };
     // The same for packed tensors that are decoded on every step (any GEMM kind): one operand, one product over all rows,
@@ -863,17 +864,19 @@ int zoqat_prequantize_frozen(zoqat_model_t* m, void* stream) {
 
 int zoqat_expand_frozen_bytes(const zoqat_model_t* m, size_t* bytes) {
     if (!m || !bytes) return fail(ZOQAT_ERR_INVALID_ARG, "NULL argument");
+    const bool i8 = m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_I8;
     size_t n = 0;
     for (const auto& Ly : m->layers)
         for (int r = 0; r < 7; ++r)
-            if (Ly.lin[r].present) n += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols) + (size_t)Ly.lin[r].rows * 4;
+            if (Ly.lin[r].present) n += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols) * (i8 ? 1 : 2) + (i8 ? (size_t)Ly.lin[r].rows * 4 : 0);
     *bytes = align_up(n);
     return ZOQAT_OK;
 }
 
 int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* stream) {
     if (!m) return fail(ZOQAT_ERR_INVALID_ARG, "model is NULL");
-    if (m->cfg.gemm_impl != ZOQAT_GEMM_TCGEN05_I8) return fail(ZOQAT_ERR_UNSUPPORTED, "byte operands belong to ZOQAT_GEMM_TCGEN05_I8");
+    const bool i8 = m->cfg.gemm_impl == ZOQAT_GEMM_TCGEN05_I8;
+    const size_t esz = i8 ? 1 : 2;
     if (m->any_packed && !m->prequantized) return fail(ZOQAT_ERR_BAD_STATE, "call zoqat_prequantize_frozen first");
     size_t need = 0;
     zoqat_expand_frozen_bytes(m, &need);
@@ -886,7 +889,7 @@ int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // all byte operands first (the tensors of one GEMM back to back: q | k | v, o, gate | up, down), then all steps in the same order
     size_t total_bytes = 0;
-    for (const auto& Ly : m->layers) for (int r = 0; r < 7; ++r) if (Ly.lin[r].present) total_bytes += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols);
+    for (const auto& Ly : m->layers) for (int r = 0; r < 7; ++r) if (Ly.lin[r].present) total_bytes += (size_t)(Ly.lin[r].rows * Ly.lin[r].cols) * esz;
     uint8_t* pb = static_cast<uint8_t*>(buffer_dev);
     float* pstep = reinterpret_cast<float*>(pb + total_bytes);      // total_bytes is a multiple of 4096
     for (auto& Ly : m->layers)
@@ -894,11 +897,14 @@ int zoqat_expand_frozen(zoqat_model_t* m, void* buffer_dev, size_t bytes, void* 
             Linear& L = Ly.lin[r];
             if (!L.present) continue;
             if (L.packed_frozen()) {
-                launch_unpack_rows(L.packed, L.qparams, L.rows, L.cols, m->cfg.w_bits, pb, true, pstep, 0, 1, m->ws.err_flag, s);
-                L.expanded = pb; L.expanded_step = pstep;
+                if (m->cfg.w_group == 0)
+                    launch_unpack_rows(L.packed, L.qparams, L.rows, L.cols, m->cfg.w_bits, pb, i8, pstep, 0, 1, m->ws.err_flag, s);
+                else
+                    launch_unpack_operand(L.packed, L.qparams, L.rows * L.cols, m->cfg.w_group, m->cfg.w_bits, reinterpret_cast<__nv_bfloat16*>(pb), s);
+                L.expanded = pb; L.expanded_step = i8 ? pstep : nullptr;
             }
-            pb += (size_t)(L.rows * L.cols);
-            pstep += L.rows;
+            pb += (size_t)(L.rows * L.cols) * esz;
+            if (i8) pstep += L.rows;
         }
     CUDA_TRY(cudaGetLastError());
     return ZOQAT_OK;
