@@ -82,3 +82,28 @@ def test_null_handles_and_new_config_values_are_rejected_on_the_host(zq):
     assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.OK
     cfg.w_bits = 1
     assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.ERR_UNSUPPORTED
+
+
+def test_integer_gemm_configuration_and_per_row_packing_are_validated_on_the_host(zq):
+    L = zq.lib()
+    n = ctypes.c_size_t()
+    cfg = zq.Config(arch=zq.ARCH_LLAMA, n_layers=1, d_model=256, n_heads=4, d_ffn=512, vocab=64, max_batch=1,
+                    max_seq=32, w_bits=4, w_group=0, a_bits=8, gemm_impl=zq.GEMM_TCGEN05_I8, norm_eps=1e-5, rope_base=10000.0)
+    assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.OK
+    # the integer GEMM needs one weight group per row, quantised activations and code - zero point inside a signed byte
+    for field, bad in (("w_group", 128), ("a_bits", 0), ("w_bits", 8)):
+        c2 = zq.Config.from_buffer_copy(cfg)
+        setattr(c2, field, bad)
+        assert L.zoqat_query_workspace(ctypes.byref(c2), ctypes.byref(n)) == zq.ERR_UNSUPPORTED, field
+    cfg.gemm_impl = 4
+    assert L.zoqat_query_workspace(ctypes.byref(cfg), ctypes.byref(n)) == zq.ERR_INVALID_ARG
+    # packed sizes with one group per row: one (step, zero point) pair per row
+    assert zq.zoqat_packed_bytes(4096, 11008, 4, 0) == (4096 * 11008 // 2, 4096 * 8)
+    with pytest.raises(zq.ZoqatError):
+        zq.zoqat_packed_bytes(64, 192, 4, 0)        # cols not a multiple of 128
+    # handles and buffers are checked before anything is launched
+    assert L.zoqat_expand_frozen(None, None, 0, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_expand_frozen_bytes(None, ctypes.byref(n)) == zq.ERR_INVALID_ARG
+    assert L.zoqat_op_gemm_i8(None, None, 128, 32, 16, None, None, None, 0, 0, None, None, None, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_op_weight_operand_i8(None, 8, 128, 4, 0, 0, 0.0, None, None, None, None, None, None, None, None, None, None) == zq.ERR_INVALID_ARG
+    assert L.zoqat_op_unpack_operand_i8(None, None, 8, 128, 4, None, None, None, None) == zq.ERR_INVALID_ARG
