@@ -214,6 +214,23 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
             const float4 v = live ? (UPD ? w_out[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
         }
+        if (UPD && perturb) {
+            // both directions of a chunk side by side: two independent Philox chains per chunk for the scheduler to interleave
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 zu = direction4(tab, urk, tid, (uint64_t)chunk_of<LANES>(i, k));
+                const float4 z = direction4(tab, rk, tid, (uint64_t)chunk_of<LANES>(i, k));
+                x[4 * k] = __fmaf_rn(upd_c, zu.x, x[4 * k]); x[4 * k + 1] = __fmaf_rn(upd_c, zu.y, x[4 * k + 1]);
+                x[4 * k + 2] = __fmaf_rn(upd_c, zu.z, x[4 * k + 2]); x[4 * k + 3] = __fmaf_rn(upd_c, zu.w, x[4 * k + 3]);
+                if (live) w_out[chunk_of<LANES>(i, k)] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+                const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (DUAL) xm[4 * k + j] = __fmaf_rn(-eps, zz[j], x[4 * k + j]);
+                    x[4 * k + j] = __fmaf_rn(eps, zz[j], x[4 * k + j]);
+                }
+            }
+        } else {
         if (UPD) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -237,6 +254,7 @@ weight_operand_kernel(const float4* __restrict__ w, int64_t n16, int bits, int p
         } else if (DUAL) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) xm[j] = x[j];
+        }
         }
         if (bits == 0) {
             if (live) {
@@ -474,6 +492,23 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
             const float4 v = live ? (UPD ? w_out[chunk_of<LANES>(i, k)] : __ldg(w + chunk_of<LANES>(i, k))) : make_float4(0.f, 0.f, 0.f, 0.f);
             x[4 * k] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
         }
+        if (UPD && perturb) {
+            // both directions of a chunk side by side: two independent Philox chains per chunk for the scheduler to interleave
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float4 zu = direction4(tab, urk, tid, (uint64_t)chunk_of<LANES>(i, k));
+                const float4 z = direction4(tab, rk, tid, (uint64_t)chunk_of<LANES>(i, k));
+                x[4 * k] = __fmaf_rn(upd_c, zu.x, x[4 * k]); x[4 * k + 1] = __fmaf_rn(upd_c, zu.y, x[4 * k + 1]);
+                x[4 * k + 2] = __fmaf_rn(upd_c, zu.z, x[4 * k + 2]); x[4 * k + 3] = __fmaf_rn(upd_c, zu.w, x[4 * k + 3]);
+                if (live) w_out[chunk_of<LANES>(i, k)] = make_float4(x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+                const float zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (DUAL) xm[4 * k + j] = __fmaf_rn(-eps, zz[j], x[4 * k + j]);
+                    x[4 * k + j] = __fmaf_rn(eps, zz[j], x[4 * k + j]);
+                }
+            }
+        } else {
         if (UPD) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -497,6 +532,7 @@ weight_operand_learned_kernel(const float4* __restrict__ w, int64_t n16, int col
         } else if (DUAL) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) xm[j] = x[j];
+        }
         }
         if (SMOOTH) {
             // column (in 16-byte chunks) of chunk 0; the following chunks are LANES further, wrapping at the row end
