@@ -1095,7 +1095,7 @@ template <int GROUP, bool ADAPT, bool SMOOTH>
 static void learned_dispatch(const LearnedOperandArgs& a, cudaStream_t s) {
     const PendingUpdate* pend = a.op_minus ? a.pend : nullptr;     // a deferred update rides on the two-sign producer only
     const int64_t n16 = a.rows * a.cols / 16;
-    const int grid = stream_grid(n16, kThreads, 3);        // 80 registers: three CTAs per SM
+    const int grid = stream_grid(n16, kThreads, 8);        // more CTAs than are resident (three per SM): the tail balances itself
     const uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
     const float4* w4 = reinterpret_cast<const float4*>(a.w);
     uint2* p = reinterpret_cast<uint2*>(a.op_plus);
@@ -1189,7 +1189,7 @@ static void row_launch(const LearnedOperandArgs& a, cudaStream_t s) {
                                              (int)smem) != cudaSuccess)
         attr.retry();
     const int per_sm = NI == 1 ? 4 : (NI == 2 ? 3 : 2);
-    const int64_t cap = (int64_t)148 * per_sm;
+    const int64_t cap = (int64_t)148 * per_sm * 3;         // about three waves: the tail balances itself
     const int grid = (int)(a.rows < cap ? a.rows : cap);
     const PhiloxKeys rk = philox_keys(a.seed), urk = pend ? philox_keys(pend->seed) : rk;
     weight_operand_row_kernel<NI, UPD, I8><<<grid, kThreads, smem, s>>>(
